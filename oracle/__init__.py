@@ -1,0 +1,195 @@
+"""ctypes front end of the CPU oracle (``sdgp_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's
+CPU-baseline leg import this; the GPU library never does, and nothing here
+touches the GPU library. Arrays are numpy; bf16 tensors are ``uint16`` bit
+patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sdgp_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+RANDOM, MAGNITUDE, RESCALED = 0, 1, 2
+
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".%d.tmp" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+             "-fno-fast-math", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build())
+            i64, u64, i32, vp, dbl = (ctypes.c_int64, ctypes.c_uint64, ctypes.c_int, ctypes.c_void_p,
+                                      ctypes.c_double)
+            lib.oracle_prune.argtypes = [vp, i64, i64, i32, i32, i32, u64, vp, vp, vp, vp]
+            lib.oracle_prune.restype = i32
+            lib.oracle_expand.argtypes = [vp, vp, i64, i64, vp]
+            lib.oracle_expand.restype = i32
+            lib.oracle_dgrad_linear.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64]
+            lib.oracle_dgrad_linear.restype = i32
+            lib.oracle_dgrad_conv2d.argtypes = [vp, vp, vp] + [i32] * 9 + [vp, i64]
+            lib.oracle_dgrad_conv2d.restype = i32
+            lib.oracle_conv2d_forward_f64.argtypes = [vp, vp, vp] + [i32] * 9
+            lib.oracle_conv2d_forward_f64.restype = i32
+            lib.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+            lib.oracle_philox4x32_10.restype = None
+            lib.oracle_random_key16.argtypes = [u64, u64]
+            lib.oracle_random_key16.restype = ctypes.c_uint16
+            lib.oracle_f32_to_bf16.argtypes = [ctypes.c_float]
+            lib.oracle_f32_to_bf16.restype = ctypes.c_uint16
+            lib.oracle_bf16_to_f64.argtypes = [ctypes.c_uint16]
+            lib.oracle_bf16_to_f64.restype = dbl
+            lib.oracle_runtime_reduction.argtypes = [dbl, i32, i32]
+            lib.oracle_runtime_reduction.restype = dbl
+            _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _u16(a, shape=None):
+    a = np.ascontiguousarray(a)
+    if a.dtype != np.uint16:
+        raise TypeError("bf16 tensors are passed as uint16 bit patterns")
+    return a if shape is None else a.reshape(shape)
+
+
+def compressible(n: int, m: int) -> bool:
+    return n <= 2 and m % 4 == 0
+
+
+def prune(dO, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask")):
+    """Algorithm 1 with the Section 3.2 pruning function ``scheme`` on a
+    ``[rows, K]`` uint16 array. Returns a dict with the requested outputs."""
+    dO = _u16(dO)
+    rows, K = dO.shape
+    out = {}
+    if "dense" in want:
+        out["dense"] = np.empty((rows, K), np.uint16)
+    if "values" in want:
+        out["values"] = np.empty((rows, K // 2), np.uint16)
+    if "meta" in want:
+        out["meta"] = np.empty((rows, K // 16), np.uint16)
+    if "mask" in want:
+        out["mask"] = np.empty((rows, K // 32), np.uint32)
+    rc = _load().oracle_prune(_ptr(dO), rows, K, n, m, scheme, seed, _ptr(out.get("dense")),
+                              _ptr(out.get("values")), _ptr(out.get("meta")), _ptr(out.get("mask")))
+    if rc != 0:
+        raise ValueError("oracle_prune rejected its arguments (rc=%d)" % rc)
+    return out
+
+
+def expand(values, meta):
+    values, meta = _u16(values), _u16(meta)
+    rows, K = values.shape[0], values.shape[1] * 2
+    dense = np.empty((rows, K), np.uint16)
+    rc = _load().oracle_expand(_ptr(values), _ptr(meta), rows, K, _ptr(dense))
+    if rc != 0:
+        raise ValueError("oracle_expand rejected its arguments")
+    return dense
+
+
+def dgrad_linear(dOp, W, row_index=None):
+    """dD = dOp @ W in fp64 from bf16 bit patterns; ``row_index`` evaluates a subset of rows."""
+    dOp, W = _u16(dOp), _u16(W)
+    rows, K = dOp.shape
+    K2, N = W.shape
+    if K != K2:
+        raise ValueError("shape mismatch")
+    idx = None if row_index is None else np.ascontiguousarray(row_index, dtype=np.int64)
+    count = rows if idx is None else idx.shape[0]
+    dD = np.empty((count, N), np.float64)
+    rc = _load().oracle_dgrad_linear(_ptr(dOp), _ptr(W), _ptr(dD), rows, K, N, _ptr(idx), count)
+    if rc != 0:
+        raise ValueError("oracle_dgrad_linear rejected its arguments")
+    return dD
+
+
+def dgrad_conv2d(dOp, W, H, Wd, stride=1, pad=0, pixel_index=None):
+    """dD (NHWC, fp64) from dOp NHWC ``[B,P,Q,Cout]`` and W ``[Cout,R,S,Cin]`` (uint16)."""
+    dOp, W = _u16(dOp), _u16(W)
+    B, P, Q, Cout = dOp.shape
+    Cout2, R, S, Cin = W.shape
+    if Cout != Cout2 or P != (H + 2 * pad - R) // stride + 1 or Q != (Wd + 2 * pad - S) // stride + 1:
+        raise ValueError("shape mismatch")
+    idx = None if pixel_index is None else np.ascontiguousarray(pixel_index, dtype=np.int64)
+    count = B * H * Wd if idx is None else idx.shape[0]
+    dD = np.empty((count, Cin), np.float64)
+    rc = _load().oracle_dgrad_conv2d(_ptr(dOp), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S, stride,
+                                     pad, _ptr(idx), count)
+    if rc != 0:
+        raise ValueError("oracle_dgrad_conv2d rejected its arguments")
+    return dD.reshape(B, H, Wd, Cin) if idx is None else dD
+
+
+def conv2d_forward_f64(D, W, stride=1, pad=0):
+    D = np.ascontiguousarray(D, dtype=np.float64)
+    W = _u16(W)
+    B, H, Wd, Cin = D.shape
+    Cout, R, S, _ = W.shape
+    P = (H + 2 * pad - R) // stride + 1
+    Q = (Wd + 2 * pad - S) // stride + 1
+    O = np.empty((B, P, Q, Cout), np.float64)
+    rc = _load().oracle_conv2d_forward_f64(_ptr(D), _ptr(W), _ptr(O), B, H, Wd, Cin, Cout, R, S,
+                                           stride, pad)
+    if rc != 0:
+        raise ValueError("oracle_conv2d_forward_f64 rejected its arguments")
+    return O
+
+
+def philox4x32_10(ctr, key):
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    o = np.empty(4, np.uint32)
+    _load().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(o))
+    return o
+
+
+def random_key16(seed, e):
+    return int(_load().oracle_random_key16(seed, e))
+
+
+def f32_to_bf16(x):
+    return int(_load().oracle_f32_to_bf16(float(x)))
+
+
+def bf16_to_f64(bits):
+    return float(_load().oracle_bf16_to_f64(int(bits)))
+
+
+def bf16_array_to_f64(a):
+    """Vectorised bf16 bits -> float64 (pure bit widening)."""
+    a = _u16(a)
+    return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def runtime_reduction(share, n, m):
+    """Section 4.3 closed form: share * (1 - n/m)."""
+    return float(_load().oracle_runtime_reduction(share, n, m))
+
+
+def omp_threads() -> int:
+    return int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))

@@ -1,0 +1,362 @@
+/*
+ * CPU oracle for Structured Data Gradient Pruning (SDGP).
+ *
+ * TEST INFRASTRUCTURE ONLY. This file is the slow, plain, obviously-correct
+ * statement of what the GPU library computes. It shares no code, header,
+ * table or helper with the CUDA path and is never called from it; only the
+ * tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * What follows the paper directly:
+ *   - Algorithm 1 (group loop over the last, stride-1 dimension, zero-initialised
+ *     copy, pruning function P applied to each m-element group);
+ *   - Section 3.2 pruning functions (random / magnitude / rescaled magnitude) and
+ *     the worked example there (rank by magnitude, prune the smallest m-n,
+ *     restore survivors to their original positions);
+ *   - Section 2.1 / Fig. 2-3 data-gradient contraction (the reduction runs over the
+ *     output-channel dimension, which is the pruned one).
+ *
+ * Readings taken where the paper is silent (each is listed in the design notes):
+ *   - ties between equal magnitudes go to the lower index;
+ *   - magnitude order is the order of the bf16 bit pattern with the sign cleared;
+ *   - the L1 rescale is per group, in fp32, with a fixed balanced summation tree;
+ *   - "random" ranks elements by 16-bit keys drawn from Philox4x32-10
+ *     (Salmon et al., SC'11) at a counter fixed by the element's linear index;
+ *   - pruned positions hold +0.0.
+ *
+ * Parity status: prune (magnitude, rescaled), compressed format, dgrad linear and
+ * dgrad conv are pinned by tests/ (paper's worked example, brute force,
+ * invariants, library fp64 matmul / transposed convolution). The Philox round
+ * function is pinned against an independent open-source engine at test time;
+ * agreement with the authors' published known-answer vectors: parity unpinned.
+ *
+ * Storage: bf16 tensors travel as uint16_t bit patterns, row-major.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_ARG 1
+
+enum { ORACLE_RANDOM = 0, ORACLE_MAGNITUDE = 1, ORACLE_RESCALED = 2 };
+#define ORACLE_MAX_M 32 /* Section 3.1: the implementation supports groups up to m = 32 */
+
+/* ------------------------------------------------------------------ bf16 */
+
+static float bf16_to_f32(uint16_t h) {
+  uint32_t u = (uint32_t)h << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return f;
+}
+
+double oracle_bf16_to_f64(uint16_t h) { return (double)bf16_to_f32(h); }
+
+/* fp32 -> bf16, round to nearest, ties to even; NaN stays NaN (quiet bit set). */
+uint16_t oracle_f32_to_bf16(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x0040u);
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7FFFu + lsb;
+  return (uint16_t)(u >> 16);
+}
+
+/* ---------------------------------------------------------------- Philox */
+
+/* Philox4x32-10, Salmon et al. SC'11: ten rounds of two 32x32->64 multiplies
+ * with a Weyl-sequence key schedule. */
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+  const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    if (round > 0) {
+      k0 += W0;
+      k1 += W1;
+    }
+    uint64_t p0 = (uint64_t)M0 * c0;
+    uint64_t p1 = (uint64_t)M1 * c2;
+    uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+    uint32_t n0 = hi1 ^ c1 ^ k0;
+    uint32_t n1 = lo1;
+    uint32_t n2 = hi0 ^ c3 ^ k1;
+    uint32_t n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* 16-bit random key of the element with linear index e = row*K + k.
+ * One Philox block serves 8 consecutive elements: block number e>>3 is the
+ * counter, the seed is the key, and element e takes half-word (e & 7) of the
+ * 128-bit output (little-endian half-words of words 0..3). */
+uint16_t oracle_random_key16(uint64_t seed, uint64_t e) {
+  uint64_t q = e >> 3;
+  uint32_t ctr[4] = {(uint32_t)q, (uint32_t)(q >> 32), 0u, 0u};
+  uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t o[4];
+  oracle_philox4x32_10(ctr, key, o);
+  uint32_t w = o[(e >> 1) & 3];
+  return (uint16_t)((e & 1) ? (w >> 16) : (w & 0xFFFFu));
+}
+
+/* ----------------------------------------------------------------- prune */
+
+/* Balanced-tree fp32 sum: level l adds aligned neighbours of width 2^l, the
+ * input padded with +0.0f up to the next power of two. */
+static float tree_sum_f32(const float* a, int m) {
+  float buf[ORACLE_MAX_M];
+  int p = 1;
+  while (p < m) p <<= 1;
+  for (int j = 0; j < p; ++j) buf[j] = (j < m) ? a[j] : 0.0f;
+  for (int width = p; width > 1; width >>= 1)
+    for (int j = 0; j < width / 2; ++j) {
+      volatile float s = buf[2 * j] + buf[2 * j + 1]; /* one rounding per add */
+      buf[j] = s;
+    }
+  return buf[0];
+}
+
+/* P(group, n): Section 3.2. Fills keep[j] in {0,1} and out[j] (bf16 bits).
+ * e0 is the linear index of the group's first element (random scheme only). */
+static void prune_group(const uint16_t* x, int n, int m, int scheme, uint64_t seed, uint64_t e0,
+                        uint8_t* keep, uint16_t* out) {
+  /* Rank: an index permutation ordered best-first, by a stable insertion sort
+   * so that equal keys stay in index order (the lower index wins a tie). */
+  int order[ORACLE_MAX_M];
+  uint32_t rank_key[ORACLE_MAX_M];
+  for (int j = 0; j < m; ++j) {
+    order[j] = j;
+    if (scheme == ORACLE_RANDOM)
+      rank_key[j] = oracle_random_key16(seed, e0 + (uint64_t)j); /* smaller key ranks first */
+    else
+      rank_key[j] = (uint32_t)(x[j] & 0x7FFFu); /* |x| as an integer; larger ranks first */
+  }
+  for (int i = 1; i < m; ++i) {
+    int idx = order[i];
+    int pos = i;
+    while (pos > 0) {
+      int prev = order[pos - 1];
+      int prev_is_worse = (scheme == ORACLE_RANDOM) ? (rank_key[prev] > rank_key[idx])
+                                                    : (rank_key[prev] < rank_key[idx]);
+      if (!prev_is_worse) break;
+      order[pos] = prev;
+      --pos;
+    }
+    order[pos] = idx;
+  }
+  /* Keep the first n of the ranking; restore them to their original positions. */
+  for (int j = 0; j < m; ++j) {
+    keep[j] = 0;
+    out[j] = 0x0000u; /* zeros_like: pruned slots are +0.0 */
+  }
+  for (int i = 0; i < n; ++i) {
+    keep[order[i]] = 1;
+    out[order[i]] = x[order[i]];
+  }
+  if (scheme == ORACLE_RESCALED) {
+    /* Rescale the survivors so that the group's L1 norm is preserved. */
+    float mag_all[ORACLE_MAX_M], mag_kept[ORACLE_MAX_M];
+    for (int j = 0; j < m; ++j) {
+      float a = fabsf(bf16_to_f32(x[j]));
+      mag_all[j] = a;
+      mag_kept[j] = keep[j] ? a : 0.0f;
+    }
+    float T = tree_sum_f32(mag_all, m);
+    float S = tree_sum_f32(mag_kept, m);
+    volatile float scale = (S == 0.0f) ? 1.0f : T / S;
+    for (int j = 0; j < m; ++j)
+      if (keep[j]) {
+        volatile float y = bf16_to_f32(x[j]) * scale;
+        out[j] = oracle_f32_to_bf16(y);
+      }
+  }
+}
+
+static int compressible(int n, int m) { return n <= 2 && (m % 4) == 0; }
+
+/* Algorithm 1 over a [rows, K] tensor, groups of m along K.
+ * Outputs (each may be NULL):
+ *   dense  [rows, K]     bf16  pruned copy
+ *   values [rows, K/2]   bf16  two slots per aligned 4-chunk, ascending position
+ *   meta   [rows, K/16]  u16   one nibble per 4-chunk: pos0 | pos1 << 2
+ *   mask   [rows, K/32]  u32   bit k%32 of word k/32 set iff element k is kept
+ * values/meta need every 4-chunk to hold at most two survivors (n <= 2, m % 4 == 0)
+ * and K % 16 == 0; mask needs K % 32 == 0. */
+int oracle_prune(const uint16_t* dO, int64_t rows, int64_t K, int n, int m, int scheme,
+                 uint64_t seed, uint16_t* dense, uint16_t* values, uint16_t* meta, uint32_t* mask) {
+  if (!dO || rows < 0 || K < 0 || m < 1 || m > ORACLE_MAX_M || n < 1 || n > m) return ORACLE_ERR_ARG;
+  if (K % m != 0) return ORACLE_ERR_ARG;
+  if (scheme < 0 || scheme > 2) return ORACLE_ERR_ARG;
+  if ((values || meta) && (!compressible(n, m) || K % 16 != 0)) return ORACLE_ERR_ARG;
+  if (mask && K % 32 != 0) return ORACLE_ERR_ARG;
+  if (mask) memset(mask, 0, (size_t)(rows * (K / 32)) * sizeof(uint32_t));
+  if (meta) memset(meta, 0, (size_t)(rows * (K / 16)) * sizeof(uint16_t));
+
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r) {
+    uint16_t* row_out = (uint16_t*)malloc((size_t)(K > 0 ? K : 1) * sizeof(uint16_t));
+    uint8_t* row_keep = (uint8_t*)malloc((size_t)(K > 0 ? K : 1));
+    for (int64_t g = 0; g < K / m; ++g) {
+      uint64_t e0 = (uint64_t)r * (uint64_t)K + (uint64_t)(g * m);
+      prune_group(dO + r * K + g * m, n, m, scheme, seed, e0, row_keep + g * m, row_out + g * m);
+    }
+    if (dense) memcpy(dense + r * K, row_out, (size_t)K * sizeof(uint16_t));
+    if (mask)
+      for (int64_t k = 0; k < K; ++k)
+        if (row_keep[k]) mask[r * (K / 32) + k / 32] |= (1u << (k % 32));
+    if (values || meta)
+      for (int64_t c = 0; c < K / 4; ++c) {
+        /* survivor positions of this 4-chunk, padded with the lowest free
+         * positions up to two, then sorted ascending */
+        int pos[2], cnt = 0;
+        uint8_t taken[4] = {0, 0, 0, 0};
+        for (int j = 0; j < 4; ++j)
+          if (row_keep[4 * c + j]) {
+            if (cnt < 2) pos[cnt] = j;
+            ++cnt;
+            taken[j] = 1;
+          }
+        for (int j = 0; j < 4 && cnt < 2; ++j)
+          if (!taken[j]) {
+            pos[cnt++] = j;
+            taken[j] = 1;
+          }
+        if (pos[0] > pos[1]) {
+          int t = pos[0];
+          pos[0] = pos[1];
+          pos[1] = t;
+        }
+        if (values) {
+          values[r * (K / 2) + 2 * c + 0] = row_keep[4 * c + pos[0]] ? row_out[4 * c + pos[0]] : 0;
+          values[r * (K / 2) + 2 * c + 1] = row_keep[4 * c + pos[1]] ? row_out[4 * c + pos[1]] : 0;
+        }
+        if (meta) {
+          uint16_t nib = (uint16_t)(pos[0] | (pos[1] << 2));
+          meta[r * (K / 16) + c / 4] |= (uint16_t)(nib << (4 * (c % 4)));
+        }
+      }
+    free(row_out);
+    free(row_keep);
+  }
+  return ORACLE_OK;
+}
+
+/* Inverse of the compressed format: rebuild the dense [rows, K] tensor. */
+int oracle_expand(const uint16_t* values, const uint16_t* meta, int64_t rows, int64_t K,
+                  uint16_t* dense) {
+  if (!values || !meta || !dense || K % 16 != 0) return ORACLE_ERR_ARG;
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t c = 0; c < K / 4; ++c) {
+      uint16_t word = meta[r * (K / 16) + c / 4];
+      int nib = (word >> (4 * (c % 4))) & 0xF;
+      int p0 = nib & 3, p1 = (nib >> 2) & 3;
+      for (int j = 0; j < 4; ++j) dense[r * K + 4 * c + j] = 0;
+      dense[r * K + 4 * c + p0] = values[r * (K / 2) + 2 * c + 0];
+      dense[r * K + 4 * c + p1] = values[r * (K / 2) + 2 * c + 1];
+    }
+  return ORACLE_OK;
+}
+
+/* ----------------------------------------------------------------- dgrad */
+
+/* Fully connected data gradient (Fig. 2): dD[r, c] = sum_k dOp[r, k] * W[k, c],
+ * dOp [rows, K], W [K, N] (output channels x input channels), fp64 accumulation
+ * in ascending k. Rows may be a subset: row_index (nullable) lists which rows
+ * of dOp to evaluate; dD then has n_rows rows in that order. */
+int oracle_dgrad_linear(const uint16_t* dOp, const uint16_t* W, double* dD, int64_t rows, int64_t K,
+                        int64_t N, const int64_t* row_index, int64_t n_rows) {
+  if (!dOp || !W || !dD || rows < 0 || K < 0 || N < 0) return ORACLE_ERR_ARG;
+  int64_t count = row_index ? n_rows : rows;
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < count; ++i) {
+    int64_t r = row_index ? row_index[i] : i;
+    for (int64_t c = 0; c < N; ++c) {
+      double acc = 0.0;
+      for (int64_t k = 0; k < K; ++k)
+        acc += oracle_bf16_to_f64(dOp[r * K + k]) * oracle_bf16_to_f64(W[k * N + c]);
+      dD[i * N + c] = acc;
+    }
+  }
+  return ORACLE_OK;
+}
+
+/* Convolution data gradient (Fig. 3). Forward layer: cross-correlation
+ *   O[b,p,q,co] = sum_{r,s,ci} D[b, p*stride - pad + r, q*stride - pad + s, ci] * W[co,r,s,ci]
+ * so the gradient w.r.t. the input is
+ *   dD[b,h,w,ci] = sum over (r,s,co) and the (p,q) with p*stride - pad + r == h,
+ *                  q*stride - pad + s == w of dOp[b,p,q,co] * W[co,r,s,ci].
+ * dOp NHWC [B,P,Q,Cout], W [Cout,R,S,Cin], dD NHWC [B,H,Wd,Cin] in fp64.
+ * pixel_index (nullable) lists flattened (b*H + h)*Wd + w positions to evaluate. */
+int oracle_dgrad_conv2d(const uint16_t* dOp, const uint16_t* W, double* dD, int B, int H, int Wd,
+                        int Cin, int Cout, int R, int S, int stride, int pad,
+                        const int64_t* pixel_index, int64_t n_pixels) {
+  if (!dOp || !W || !dD || stride < 1 || pad < 0 || R < 1 || S < 1) return ORACLE_ERR_ARG;
+  int P = (H + 2 * pad - R) / stride + 1;
+  int Q = (Wd + 2 * pad - S) / stride + 1;
+  if (P < 1 || Q < 1) return ORACLE_ERR_ARG;
+  int64_t count = pixel_index ? n_pixels : (int64_t)B * H * Wd;
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < count; ++i) {
+    int64_t pix = pixel_index ? pixel_index[i] : i;
+    int w = (int)(pix % Wd);
+    int h = (int)((pix / Wd) % H);
+    int b = (int)(pix / ((int64_t)Wd * H));
+    for (int ci = 0; ci < Cin; ++ci) {
+      double acc = 0.0;
+      for (int r = 0; r < R; ++r) {
+        int hp = h + pad - r;
+        if (hp < 0 || hp % stride != 0) continue;
+        int p = hp / stride;
+        if (p >= P) continue;
+        for (int s = 0; s < S; ++s) {
+          int wq = w + pad - s;
+          if (wq < 0 || wq % stride != 0) continue;
+          int q = wq / stride;
+          if (q >= Q) continue;
+          const uint16_t* g = dOp + (((int64_t)b * P + p) * Q + q) * Cout;
+          for (int co = 0; co < Cout; ++co)
+            acc += oracle_bf16_to_f64(g[co]) *
+                   oracle_bf16_to_f64(W[(((int64_t)co * R + r) * S + s) * Cin + ci]);
+        }
+      }
+      dD[i * Cin + ci] = acc;
+    }
+  }
+  return ORACLE_OK;
+}
+
+/* Direct forward convolution in fp64 on fp64 inputs; used only by the adjoint
+ * identity test <conv(D), G> == <D, dgrad(G)>. */
+int oracle_conv2d_forward_f64(const double* D, const uint16_t* W, double* O, int B, int H, int Wd,
+                              int Cin, int Cout, int R, int S, int stride, int pad) {
+  int P = (H + 2 * pad - R) / stride + 1;
+  int Q = (Wd + 2 * pad - S) / stride + 1;
+  if (P < 1 || Q < 1) return ORACLE_ERR_ARG;
+  for (int b = 0; b < B; ++b)
+    for (int p = 0; p < P; ++p)
+      for (int q = 0; q < Q; ++q)
+        for (int co = 0; co < Cout; ++co) {
+          double acc = 0.0;
+          for (int r = 0; r < R; ++r)
+            for (int s = 0; s < S; ++s) {
+              int h = p * stride - pad + r, w = q * stride - pad + s;
+              if (h < 0 || h >= H || w < 0 || w >= Wd) continue;
+              for (int ci = 0; ci < Cin; ++ci)
+                acc += D[(((int64_t)b * H + h) * Wd + w) * Cin + ci] *
+                       oracle_bf16_to_f64(W[(((int64_t)co * R + r) * S + s) * Cin + ci]);
+            }
+          O[(((int64_t)b * P + p) * Q + q) * Cout + co] = acc;
+        }
+  return ORACLE_OK;
+}
+
+/* Section 4.3 estimator: removing a fraction (1 - n/m) of a pass that takes
+ * share f of the runtime reduces the total by f * (1 - n/m). */
+double oracle_runtime_reduction(double share, int n, int m) {
+  return share * (1.0 - (double)n / (double)m);
+}

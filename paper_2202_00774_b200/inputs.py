@@ -1,0 +1,144 @@
+"""Seeded synthetic inputs for SDGP tests and benchmarks.
+
+This module only draws random tensors and describes workload shapes; it holds
+none of the pruning or contraction arithmetic. Everything is numpy on the
+host; bf16 tensors are returned as ``uint16`` bit patterns (row-major) so the
+same bits can be handed to any consumer.
+
+Workloads (synthetic stand-ins for the gradients and weights of the paper's
+CIFAR-10 / ImageNet training runs, Section 4):
+  * ``fc_small``       one fully connected layer, dO [256, 512], W [512, 256]
+  * ``resnet9``        3x3 stride-1 pad-1 convolution layers of a 9-layer ResNet at batch 512
+  * ``resnet50``       1x1 / 3x3 bottleneck convolutions of ResNet-50 at batch 256
+  * ``gemm_large``     dO [16384, 4096], W [4096, 4096]
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List
+
+import numpy as np
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 to bf16 (nearest, ties to even) and return the bit patterns."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    u = u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))
+    return (u >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def _rng(seed: int, stream: int) -> np.random.Generator:
+    return np.random.Generator(np.random.PCG64([int(seed), int(stream)]))
+
+
+def normal_bf16(shape, std: float, seed: int, stream: int = 0) -> np.ndarray:
+    """N(0, std^2) rounded to bf16."""
+    g = _rng(seed, stream)
+    return f32_to_bf16_bits(g.standard_normal(shape, dtype=np.float32) * np.float32(std))
+
+
+def relu_masked_laplace_bf16(shape, seed: int, stream: int = 0, zero_fraction: float = 0.5) -> np.ndarray:
+    """Laplace(0, 1) values with a Bernoulli(zero_fraction) share forced to exact +0.0,
+    as a gradient that has passed back through a ReLU would look (Section 3.3 reports a
+    large share of exact zeros in real data gradients)."""
+    g = _rng(seed, stream)
+    n = int(np.prod(shape))
+    out = np.empty(n, np.uint16)
+    step = 1 << 24
+    for lo in range(0, n, step):
+        hi = min(n, lo + step)
+        v = g.laplace(0.0, 1.0, hi - lo).astype(np.float32)
+        v[g.random(hi - lo, dtype=np.float32) < zero_fraction] = 0.0
+        out[lo:hi] = f32_to_bf16_bits(v)
+    return out.reshape(shape)
+
+
+def adversarial_groups_bf16(rows: int, K: int, seed: int) -> np.ndarray:
+    """Rows full of ranking edge cases: ties, signed zeros, infinities, NaNs, denormals."""
+    g = _rng(seed, 99)
+    pool = np.array([0x0000, 0x8000, 0x3F80, 0xBF80, 0x3F80, 0x4000, 0xC000, 0x7F80, 0xFF80,
+                     0x7FC0, 0xFFC1, 0x0001, 0x8001, 0x007F, 0x7F7F, 0xFF7F, 0x3F81, 0xBF81],
+                    dtype=np.uint16)
+    return pool[g.integers(0, pool.size, size=(rows, K))]
+
+
+# ------------------------------------------------------------------ shapes
+
+
+@dataclass(frozen=True)
+class ConvLayer:
+    name: str
+    B: int
+    H: int      # input (dD) height
+    W: int      # input (dD) width
+    Cin: int
+    Cout: int
+    R: int
+    S: int
+    stride: int
+    pad: int
+
+    @property
+    def P(self) -> int:
+        return (self.H + 2 * self.pad - self.R) // self.stride + 1
+
+    @property
+    def Q(self) -> int:
+        return (self.W + 2 * self.pad - self.S) // self.stride + 1
+
+    @property
+    def dense_macs(self) -> int:
+        """True multiply-accumulates of the dense data-gradient contraction."""
+        return self.B * self.P * self.Q * self.Cout * self.R * self.S * self.Cin
+
+    def dO_shape(self):
+        return (self.B, self.P, self.Q, self.Cout)
+
+    def W_shape(self):
+        return (self.Cout, self.R, self.S, self.Cin)
+
+    def dD_shape(self):
+        return (self.B, self.H, self.W, self.Cin)
+
+
+def resnet9_layers(batch: int = 512) -> List[ConvLayer]:
+    """3x3, stride 1, pad 1 layers (Cin -> Cout @ HxW) of the CIFAR-sized 9-layer ResNet."""
+    spec = [(64, 128, 32), (128, 128, 16), (128, 128, 16), (128, 256, 16), (256, 512, 8),
+            (512, 512, 4), (512, 512, 4)]
+    return [ConvLayer("r9_%d_%dto%d_at%d" % (i, ci, co, hw), batch, hw, hw, ci, co, 3, 3, 1, 1)
+            for i, (ci, co, hw) in enumerate(spec)]
+
+
+def resnet50_stride1_layers(batch: int = 256) -> List[ConvLayer]:
+    """Distinct stride-1 1x1 / 3x3 bottleneck convolutions of ResNet-50 (stages 1-4)."""
+    out = []
+    for stage, (hw, mid) in enumerate([(56, 64), (28, 128), (14, 256), (7, 512)], start=1):
+        wide = 4 * mid
+        out.append(ConvLayer("r50_s%d_1x1_%dto%d" % (stage, wide, mid), batch, hw, hw, wide, mid, 1, 1, 1, 0))
+        out.append(ConvLayer("r50_s%d_3x3_%dto%d" % (stage, mid, mid), batch, hw, hw, mid, mid, 3, 3, 1, 1))
+        out.append(ConvLayer("r50_s%d_1x1_%dto%d" % (stage, mid, wide), batch, hw, hw, mid, wide, 1, 1, 1, 0))
+    out.insert(0, ConvLayer("r50_s1_1x1_64to64", batch, 56, 56, 64, 64, 1, 1, 1, 0))
+    return out
+
+
+def conv_layer_tensors(layer: ConvLayer, seed: int):
+    """(dO, W) for one layer: dO = ReLU-masked Laplace, W = He-normal N(0, 2/(R*S*Cin))."""
+    dO = relu_masked_laplace_bf16(layer.dO_shape(), seed, stream=1)
+    W = normal_bf16(layer.W_shape(), float(np.sqrt(2.0 / (layer.R * layer.S * layer.Cin))), seed, stream=2)
+    return dO, W
+
+
+def fc_tensors(rows: int, K: int, N: int, seed: int):
+    """(dO, W) for a fully connected layer: dO ~ N(0,1), W ~ N(0, 1/K)."""
+    dO = normal_bf16((rows, K), 1.0, seed, stream=1)
+    W = normal_bf16((K, N), float(1.0 / np.sqrt(K)), seed, stream=2)
+    return dO, W
+
+
+FC_SMALL = dict(rows=256, K=512, N=256, seed=0)
+GEMM_LARGE = dict(rows=16384, K=4096, N=4096, seed=0)
+NM_SWEEP = [(1, 4), (2, 4), (2, 8), (2, 16)]
