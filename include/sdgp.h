@@ -1,0 +1,134 @@
+/*
+ * sdgp.h - C ABI of the Structured Data Gradient Pruning (SDGP) GPU library.
+ *
+ * During back-propagation SDGP prunes the output data gradient dL/dO of a layer to an N:M
+ * pattern along the output-channel dimension (keep n of every m consecutive elements) and
+ * then computes the input data gradient dL/dD = prune(dL/dO) . W from the pruned tensor
+ * (Algorithm 1; Section 2.1, Fig. 2 and Fig. 3; Section 3.2 for the pruning functions).
+ *
+ * Conventions common to every entry point
+ *   - All tensor pointers are DEVICE pointers (global memory of the current CUDA device),
+ *     caller-owned, 16-byte aligned, contiguous, row-major; bf16 unless stated.
+ *   - Inputs are never written (dL/dO is still needed for the weight gradient, Section 3.1).
+ *     Outputs are fully overwritten.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream). Work is enqueued
+ *     asynchronously; the call returns before it finishes.
+ *   - The library allocates no device memory; scratch is the caller's `workspace`.
+ *   - Argument errors are found on the host and returned BEFORE anything is launched.
+ *     Nothing aborts, throws or traps. A kernel whose internal wait runs out raises a flag
+ *     that sdgp_last_device_error() reports.
+ *   - n == m is legal and prunes nothing (the dense data gradient).
+ *
+ * Pruning functions P (Section 3.2), applied to each group of m consecutive elements:
+ *   SDGP_RANDOM              keep the n elements with the smallest 16-bit random keys. Keys come
+ *                            from Philox4x32-10 (Salmon et al., SC'11): key = seed, counter =
+ *                            (e >> 3) with e the element's linear index row*K + k, element e taking
+ *                            little-endian half-word (e & 7) of the 128-bit output. Equal keys:
+ *                            lower index wins.
+ *   SDGP_MAGNITUDE           keep the n largest magnitudes (order of the bf16 bit pattern with the
+ *                            sign cleared); equal magnitudes: lower index wins; survivors keep
+ *                            their exact bits.
+ *   SDGP_RESCALED_MAGNITUDE  same survivors, each multiplied by sum|group| / sum|survivors| so the
+ *                            group's L1 norm is preserved: fp32 magnitudes, balanced pairwise
+ *                            summation in index order, IEEE division, fp32 multiply, round to
+ *                            nearest-even bf16; a zero denominator gives scale 1; a NaN result is
+ *                            stored as 0x7FC0.
+ *   Pruned positions hold +0.0.
+ *
+ * Compressed form (for patterns with n <= 2 and m % 4 == 0, where every aligned 4-element chunk
+ * holds at most two survivors - the form a 2:4 sparse tensor core consumes):
+ *   values [rows, K/2]  two slots per 4-chunk: the chunk's survivor positions, padded with the
+ *                       lowest unused positions up to two and sorted ascending (p0 < p1); slot i
+ *                       holds the pruned tensor's value at p_i (a pad slot therefore holds +0.0).
+ *   meta   [rows, K/16] uint16; chunk c of a row sits in bits [4*(c%4), 4*(c%4)+3] of word c/4 and
+ *                       is p0 | p1 << 2.
+ */
+#ifndef SDGP_H_
+#define SDGP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SDGP_OK = 0,
+  SDGP_ERR_INVALID_ARG = 1, /* null pointer, negative size, n/m out of range, K % m != 0, ... */
+  SDGP_ERR_UNSUPPORTED = 2, /* legal request this build has no kernel for */
+  SDGP_ERR_ALIGNMENT = 3,   /* pointer not 16-byte aligned / extent not a multiple the layout needs */
+  SDGP_ERR_WORKSPACE = 4,   /* workspace missing or smaller than sdgp_workspace_size_*() */
+  SDGP_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, tensor-map encode, ...) */
+  SDGP_ERR_TIMEOUT = 6      /* a bounded wait inside a kernel ran out (see sdgp_last_device_error) */
+} sdgp_status;
+
+typedef enum { SDGP_RANDOM = 0, SDGP_MAGNITUDE = 1, SDGP_RESCALED_MAGNITUDE = 2 } sdgp_scheme;
+
+/* `flags` of the dgrad entry points. */
+enum {
+  SDGP_FLAG_TWO_PASS = 0, /* prune kernel writes compressed dL/dO into the workspace, sparse GEMM reads it */
+  SDGP_FLAG_FUSED = 1,    /* pruning happens inside the GEMM's producer; no compressed tensor in global memory */
+  SDGP_FLAG_DENSE = 2     /* no pruning: dense tensor-core data gradient of dL/dO itself (n, m, scheme ignored) */
+};
+
+/* Algorithm 1 with pruning function `scheme` on dO viewed as [rows, K], groups of m along K.
+ * Requirements: 1 <= n <= m <= 32, m in {4, 8, 16, 32}, K % m == 0, K % 16 == 0 (K % 32 == 0 when
+ * `mask` is requested). Any of the four outputs may be NULL; values/meta additionally need
+ * n <= 2 (else SDGP_ERR_UNSUPPORTED).
+ *   dOp_dense [rows, K]    bf16  pruned copy (the tensor the paper's implementation produces)
+ *   values    [rows, K/2]  bf16  compressed survivors      (see file header)
+ *   meta      [rows, K/16] u16   survivor positions        (see file header)
+ *   mask      [rows, K/32] u32   bit k%32 of word k/32 set iff element k is kept
+ * rows == 0 or K == 0 is a no-op returning SDGP_OK. */
+sdgp_status sdgp_prune(const void* dO, int64_t rows, int64_t K, int n, int m, sdgp_scheme scheme,
+                       uint64_t seed, void* dOp_dense, void* values, void* meta, void* mask,
+                       void* stream);
+
+/* Fully connected data gradient (Section 2.1, Fig. 2): dD[r, c] = sum_k prune(dO)[r, k] * W[k, c].
+ *   dO [rows, K] bf16, W [K, N] bf16 (output channels x input channels), dD [rows, N] bf16,
+ *   fp32 accumulation, round-to-nearest-even bf16 result.
+ * Requirements: K % 64 == 0, N % 64 == 0 (any rows >= 0); pruned modes need n <= 2, m in {4,8,16,32}
+ * dividing K. Workspace: sdgp_workspace_size_linear() bytes, 256-byte aligned. */
+sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,
+                              int64_t N, int n, int m, sdgp_scheme scheme, uint64_t seed,
+                              void* workspace, size_t workspace_bytes, uint32_t flags, void* stream);
+
+/* Convolution data gradient (Section 3.1, Fig. 3), NHWC, for the forward cross-correlation
+ *   O[b,p,q,co] = sum_{r,s,ci} D[b, p*stride - pad + r, q*stride - pad + s, ci] * W[co,r,s,ci]:
+ *   dD[b,h,w,ci] = sum over r, s, co and the (p, q) with p*stride - pad + r == h and
+ *                  q*stride - pad + s == w of prune(dO)[b,p,q,co] * W[co,r,s,ci].
+ *   dO [B,P,Q,Cout] with P = (H + 2*pad - R)/stride + 1, Q likewise; W [Cout,R,S,Cin];
+ *   dD [B,H,Wd,Cin]. Groups of m run along Cout at a fixed (b,p,q).
+ * Requirements: stride == 1 (other strides: SDGP_ERR_UNSUPPORTED), Cout % 64 == 0, Cin % 64 == 0,
+ * pad <= R-1 and pad <= S-1. Workspace: sdgp_workspace_size_conv2d() bytes. */
+sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, int H, int Wd, int Cin,
+                              int Cout, int R, int S, int stride, int pad, int n, int m,
+                              sdgp_scheme scheme, uint64_t seed, void* workspace,
+                              size_t workspace_bytes, uint32_t flags, void* stream);
+
+/* The contraction alone, from an already compressed dL/dO (output of sdgp_prune):
+ * values [rows, K/2] bf16 and meta [rows, K/16] u16 in place of dO. No workspace. */
+sdgp_status sdgp_spmm_linear(const void* values, const void* meta, const void* W, void* dD,
+                             int64_t rows, int64_t K, int64_t N, void* stream);
+sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W, void* dD, int B,
+                             int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
+                             void* stream);
+
+/* Bytes of workspace the matching dgrad call needs for these shapes and flags (0 for
+ * SDGP_FLAG_DENSE and SDGP_FLAG_FUSED). */
+size_t sdgp_workspace_size_linear(int64_t rows, int64_t K, int64_t N, uint32_t flags);
+size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R, int S, int stride,
+                                  int pad, uint32_t flags);
+
+/* Reads and clears the device-side error word of the current device (synchronises the device).
+ * SDGP_OK, or SDGP_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last call. */
+sdgp_status sdgp_last_device_error(void);
+
+/* Static, NUL-terminated description of a status code. */
+const char* sdgp_status_string(sdgp_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDGP_H_ */

@@ -53,11 +53,14 @@ static float bf16_to_f32(uint16_t h) {
 
 double oracle_bf16_to_f64(uint16_t h) { return (double)bf16_to_f32(h); }
 
-/* fp32 -> bf16, round to nearest, ties to even; NaN stays NaN (quiet bit set). */
+/* fp32 -> bf16, round to nearest, ties to even. A NaN result is stored as the one
+ * canonical quiet NaN 0x7FC0: which payload an fp32 multiply by NaN returns differs
+ * between processors, so the stored pattern is fixed here (a reading; the paper does
+ * not discuss non-finite gradients). */
 uint16_t oracle_f32_to_bf16(float f) {
   uint32_t u;
   memcpy(&u, &f, 4);
-  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x0040u);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)0x7FC0u;
   uint32_t lsb = (u >> 16) & 1u;
   u += 0x7FFFu + lsb;
   return (uint16_t)(u >> 16);
