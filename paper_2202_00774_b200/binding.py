@@ -1,0 +1,149 @@
+"""Python binding of the SDGP C ABI (``include/sdgp.h``): argument marshalling only.
+
+Tensors are torch CUDA tensors (device memory and streams come from torch); every
+computation happens inside ``libsdgp.so``. There is no fallback: a missing library or a
+non-OK status raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+RANDOM, MAGNITUDE, RESCALED_MAGNITUDE = 0, 1, 2
+FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE = 0, 1, 2
+
+EXPORTS = ["sdgp_prune", "sdgp_dgrad_linear", "sdgp_dgrad_conv2d", "sdgp_spmm_linear", "sdgp_spmm_conv2d",
+           "sdgp_workspace_size_linear", "sdgp_workspace_size_conv2d", "sdgp_last_device_error",
+           "sdgp_status_string"]
+
+_lib = None
+
+
+class SdgpError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__("%s failed: %s (status %d)" % (what, status_string(status), status))
+        self.status = status
+
+
+def lib() -> ctypes.CDLL:
+    """Loads (building first if the sources are newer) the C-ABI library."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if _build.needs_build():
+            path = _build.build()
+        if not os.path.exists(path):
+            raise RuntimeError("libsdgp.so is missing; run paper_2202_00774_b200/build.py")
+        L = ctypes.CDLL(path)
+        i64, u64, i32, u32, vp, sz = (ctypes.c_int64, ctypes.c_uint64, ctypes.c_int, ctypes.c_uint32,
+                                      ctypes.c_void_p, ctypes.c_size_t)
+        L.sdgp_prune.argtypes = [vp, i64, i64, i32, i32, i32, u64, vp, vp, vp, vp, vp]
+        L.sdgp_prune.restype = i32
+        L.sdgp_dgrad_linear.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, u64, vp, sz, u32, vp]
+        L.sdgp_dgrad_linear.restype = i32
+        L.sdgp_dgrad_conv2d.argtypes = [vp, vp, vp] + [i32] * 9 + [i32, i32, i32, u64, vp, sz, u32, vp]
+        L.sdgp_dgrad_conv2d.restype = i32
+        L.sdgp_spmm_linear.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
+        L.sdgp_spmm_linear.restype = i32
+        L.sdgp_spmm_conv2d.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
+        L.sdgp_spmm_conv2d.restype = i32
+        L.sdgp_workspace_size_linear.argtypes = [i64, i64, i64, u32]
+        L.sdgp_workspace_size_linear.restype = sz
+        L.sdgp_workspace_size_conv2d.argtypes = [i32] * 9 + [u32]
+        L.sdgp_workspace_size_conv2d.restype = sz
+        L.sdgp_last_device_error.argtypes = []
+        L.sdgp_last_device_error.restype = i32
+        L.sdgp_status_string.argtypes = [i32]
+        L.sdgp_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().sdgp_status_string(int(status)).decode()
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise SdgpError(status, what)
+
+
+def _dev(t, name):
+    if t is not None and (not t.is_cuda or not t.is_contiguous()):
+        raise ValueError("%s must be a contiguous CUDA tensor" % name)
+
+
+def sdgp_prune(dO, n, m, scheme, seed=0, dense=None, values=None, meta=None, mask=None):
+    """``sdgp_prune`` of sdgp.h. ``dO`` is a 2-byte-element tensor whose last dimension is K;
+    outputs are caller-allocated tensors (or None)."""
+    for t, name in ((dO, "dO"), (dense, "dense"), (values, "values"), (meta, "meta"), (mask, "mask")):
+        _dev(t, name)
+    K = dO.shape[-1] if dO.dim() else 0
+    rows = dO.numel() // K if K else 0
+    _check(lib().sdgp_prune(_ptr(dO), rows, K, n, m, scheme, seed, _ptr(dense), _ptr(values), _ptr(meta),
+                            _ptr(mask), _stream()), "sdgp_prune")
+
+
+def sdgp_workspace_size_linear(rows, K, N, flags=FLAG_TWO_PASS) -> int:
+    return int(lib().sdgp_workspace_size_linear(rows, K, N, flags))
+
+
+def sdgp_workspace_size_conv2d(B, H, Wd, Cin, Cout, R, S, stride, pad, flags=FLAG_TWO_PASS) -> int:
+    return int(lib().sdgp_workspace_size_conv2d(B, H, Wd, Cin, Cout, R, S, stride, pad, flags))
+
+
+def sdgp_dgrad_linear(dO, W, dD, n, m, scheme, seed=0, workspace=None, flags=FLAG_TWO_PASS):
+    """``sdgp_dgrad_linear``: dO [rows,K], W [K,N], dD [rows,N] (bf16 or 2-byte views)."""
+    for t, name in ((dO, "dO"), (W, "W"), (dD, "dD"), (workspace, "workspace")):
+        _dev(t, name)
+    rows, K = dO.shape
+    N = W.shape[1]
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().sdgp_dgrad_linear(_ptr(dO), _ptr(W), _ptr(dD), rows, K, N, n, m, scheme, seed,
+                                   _ptr(workspace), ws_bytes, flags, _stream()), "sdgp_dgrad_linear")
+
+
+def sdgp_dgrad_conv2d(dO, W, dD, stride, pad, n, m, scheme, seed=0, workspace=None, flags=FLAG_TWO_PASS):
+    """``sdgp_dgrad_conv2d``: dO NHWC [B,P,Q,Cout], W [Cout,R,S,Cin], dD NHWC [B,H,Wd,Cin]."""
+    for t, name in ((dO, "dO"), (W, "W"), (dD, "dD"), (workspace, "workspace")):
+        _dev(t, name)
+    B, H, Wd, Cin = dD.shape
+    Cout, R, S, _ = W.shape
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().sdgp_dgrad_conv2d(_ptr(dO), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S, stride, pad, n, m,
+                                   scheme, seed, _ptr(workspace), ws_bytes, flags, _stream()),
+           "sdgp_dgrad_conv2d")
+
+
+def sdgp_spmm_linear(values, meta, W, dD):
+    for t, name in ((values, "values"), (meta, "meta"), (W, "W"), (dD, "dD")):
+        _dev(t, name)
+    rows, N = dD.shape
+    K = W.shape[0]
+    _check(lib().sdgp_spmm_linear(_ptr(values), _ptr(meta), _ptr(W), _ptr(dD), rows, K, N, _stream()),
+           "sdgp_spmm_linear")
+
+
+def sdgp_spmm_conv2d(values, meta, W, dD, stride, pad):
+    for t, name in ((values, "values"), (meta, "meta"), (W, "W"), (dD, "dD")):
+        _dev(t, name)
+    B, H, Wd, Cin = dD.shape
+    Cout, R, S, _ = W.shape
+    _check(lib().sdgp_spmm_conv2d(_ptr(values), _ptr(meta), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S,
+                                  stride, pad, _stream()), "sdgp_spmm_conv2d")
+
+
+def sdgp_last_device_error() -> int:
+    return int(lib().sdgp_last_device_error())

@@ -1,0 +1,147 @@
+// extern "C" entry points: argument validation, workspace carving, dispatch.
+#include "sdgp_internal.cuh"
+
+namespace {
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+sdgp_status check_prune_args(int64_t rows, int64_t K, int n, int m, int scheme) {
+  if (rows < 0 || K < 0) return SDGP_ERR_INVALID_ARG;
+  if (scheme < 0 || scheme > 2) return SDGP_ERR_INVALID_ARG;
+  if (m < 1 || m > 32 || n < 1 || n > m) return SDGP_ERR_INVALID_ARG;
+  if (m != 4 && m != 8 && m != 16 && m != 32) return SDGP_ERR_UNSUPPORTED;
+  if (K % m != 0) return SDGP_ERR_INVALID_ARG;
+  return SDGP_OK;
+}
+
+struct Carve {
+  void* values;
+  void* meta;
+  size_t bytes;
+};
+
+Carve carve_compressed(void* workspace, int64_t elements) {
+  Carve c;
+  const size_t values_bytes = round_up((size_t)elements, 256);      // elements/2 bf16
+  const size_t meta_bytes = round_up((size_t)elements / 8, 256);    // elements/16 uint16
+  c.values = workspace;
+  c.meta = workspace ? (void*)((uint8_t*)workspace + values_bytes) : nullptr;
+  c.bytes = values_bytes + meta_bytes;
+  return c;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sdgp_status_string(sdgp_status status) {
+  switch (status) {
+    case SDGP_OK: return "ok";
+    case SDGP_ERR_INVALID_ARG: return "invalid argument";
+    case SDGP_ERR_UNSUPPORTED: return "unsupported configuration";
+    case SDGP_ERR_ALIGNMENT: return "misaligned pointer or extent";
+    case SDGP_ERR_WORKSPACE: return "workspace missing or too small";
+    case SDGP_ERR_CUDA: return "CUDA call failed";
+    case SDGP_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+  }
+  return "unknown status";
+}
+
+sdgp_status sdgp_prune(const void* dO, int64_t rows, int64_t K, int n, int m, sdgp_scheme scheme,
+                       uint64_t seed, void* dOp_dense, void* values, void* meta, void* mask,
+                       void* stream) {
+  sdgp_status st = check_prune_args(rows, K, n, m, (int)scheme);
+  if (st != SDGP_OK) return st;
+  if (rows == 0 || K == 0) return SDGP_OK;
+  if (!dO) return SDGP_ERR_INVALID_ARG;
+  if ((values || meta) && n > 2) return SDGP_ERR_UNSUPPORTED;
+  if (K % 16 != 0 || (mask && K % 32 != 0)) return SDGP_ERR_ALIGNMENT;
+  if (!aligned16(dO) || !aligned16(dOp_dense) || !aligned16(values) || !aligned16(meta) || !aligned16(mask))
+    return SDGP_ERR_ALIGNMENT;
+  cudaError_t e = sdgp::launch_prune(dO, rows, K, n, m, (int)scheme, seed, dOp_dense, values, meta, mask,
+                                     (cudaStream_t)stream);
+  return e == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
+}
+
+size_t sdgp_workspace_size_linear(int64_t rows, int64_t K, int64_t N, uint32_t flags) {
+  (void)N;
+  if (flags != SDGP_FLAG_TWO_PASS || rows <= 0 || K <= 0) return 0;
+  return carve_compressed(nullptr, rows * K).bytes;
+}
+
+size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R, int S, int stride,
+                                  int pad, uint32_t flags) {
+  (void)Cin;
+  if (flags != SDGP_FLAG_TWO_PASS || stride < 1) return 0;
+  const int64_t P = (H + 2 * pad - R) / stride + 1, Q = (Wd + 2 * pad - S) / stride + 1;
+  if (B <= 0 || P <= 0 || Q <= 0 || Cout <= 0) return 0;
+  return carve_compressed(nullptr, (int64_t)B * P * Q * Cout).bytes;
+}
+
+sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W, void* dD, int B,
+                             int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
+                             void* stream) {
+  if (B < 0 || H < 0 || Wd < 0 || Cin < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0)
+    return SDGP_ERR_INVALID_ARG;
+  if (stride != 1) return SDGP_ERR_UNSUPPORTED;
+  if (pad > R - 1 || pad > S - 1) return SDGP_ERR_UNSUPPORTED;
+  if ((int64_t)B * H * Wd == 0) return SDGP_OK;
+  if (!values || !meta || !W || !dD) return SDGP_ERR_INVALID_ARG;
+  if (!aligned16(values) || !aligned16(meta) || !aligned16(W) || !aligned16(dD)) return SDGP_ERR_ALIGNMENT;
+  return sdgp::launch_dgrad(true, values, meta, W, dD, B, H, Wd, Cin, Cout, R, S, pad, (cudaStream_t)stream);
+}
+
+sdgp_status sdgp_spmm_linear(const void* values, const void* meta, const void* W, void* dD,
+                             int64_t rows, int64_t K, int64_t N, void* stream) {
+  if (rows < 0 || K < 1 || N < 1) return SDGP_ERR_INVALID_ARG;
+  if (rows > 0x7FFFFFFF || K > 0x7FFFFFFF || N > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
+  return sdgp_spmm_conv2d(values, meta, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 1, 0, stream);
+}
+
+sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, int H, int Wd, int Cin,
+                              int Cout, int R, int S, int stride, int pad, int n, int m,
+                              sdgp_scheme scheme, uint64_t seed, void* workspace,
+                              size_t workspace_bytes, uint32_t flags, void* stream) {
+  if (B < 0 || H < 0 || Wd < 0 || Cin < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0)
+    return SDGP_ERR_INVALID_ARG;
+  if (flags > SDGP_FLAG_DENSE) return SDGP_ERR_INVALID_ARG;
+  if (stride != 1) return SDGP_ERR_UNSUPPORTED;
+  if (pad > R - 1 || pad > S - 1) return SDGP_ERR_UNSUPPORTED;
+  if (flags != SDGP_FLAG_DENSE) {
+    sdgp_status st = check_prune_args(0, Cout, n, m, (int)scheme);
+    if (st != SDGP_OK) return st;
+    if (n > 2 && n != m) return SDGP_ERR_UNSUPPORTED;
+  }
+  if ((int64_t)B * H * Wd == 0) return SDGP_OK;
+  const int64_t P = H + 2 * pad - R + 1, Q = Wd + 2 * pad - S + 1;
+  if (P < 1 || Q < 1) return SDGP_ERR_INVALID_ARG;
+  if (!dO || !W || !dD) return SDGP_ERR_INVALID_ARG;
+  if (!aligned16(dO) || !aligned16(W) || !aligned16(dD)) return SDGP_ERR_ALIGNMENT;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (flags == SDGP_FLAG_DENSE || n == m)
+    return sdgp::launch_dgrad(false, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, pad, s);
+  if (flags == SDGP_FLAG_FUSED) return SDGP_ERR_UNSUPPORTED;
+  if (Cin % 64 != 0 || Cout % 128 != 0) return SDGP_ERR_UNSUPPORTED;
+  const Carve c = carve_compressed(workspace, (int64_t)B * P * Q * Cout);
+  if (!workspace || workspace_bytes < c.bytes) return SDGP_ERR_WORKSPACE;
+  if (((uintptr_t)workspace & 255u) != 0) return SDGP_ERR_ALIGNMENT;
+  cudaError_t e = sdgp::launch_prune(dO, (int64_t)B * P * Q, Cout, n, m, (int)scheme, seed, nullptr, c.values,
+                                     c.meta, nullptr, s);
+  if (e != cudaSuccess) return SDGP_ERR_CUDA;
+  return sdgp::launch_dgrad(true, c.values, c.meta, W, dD, B, H, Wd, Cin, Cout, R, S, pad, s);
+}
+
+sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,
+                              int64_t N, int n, int m, sdgp_scheme scheme, uint64_t seed,
+                              void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
+  if (rows < 0 || K < 1 || N < 1) return SDGP_ERR_INVALID_ARG;
+  if (rows > 0x7FFFFFFF || K > 0x7FFFFFFF || N > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
+  return sdgp_dgrad_conv2d(dO, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 1, 0, n, m, scheme, seed,
+                           workspace, workspace_bytes, flags, stream);
+}
+
+sdgp_status sdgp_last_device_error(void) { return sdgp::read_device_error(); }
+
+}  // extern "C"

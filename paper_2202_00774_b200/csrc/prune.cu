@@ -1,0 +1,220 @@
+// N:M pruning of the output data gradient (Algorithm 1, Section 3.2), sm_100a.
+//
+// One thread owns one aligned run of 8 bf16 elements (a single 128-bit load). Groups of
+// m = 4 (two per thread) and m = 8 (one per thread) are ranked inside the thread; groups of
+// 16 and 32 span 2 and 4 neighbouring lanes, which trade their keys with warp shuffles.
+// The kernel is a pure stream: 2 B read per element, 1 B of compressed values, 1/8 B of
+// position metadata (+ 1/8 B mask, + 2 B dense copy when asked for), every output indexed by
+// the same 8-element vector number so all stores coalesce.
+#include "sdgp_internal.cuh"
+
+namespace sdgp {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kVecPerThread = 4;
+
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds, Weyl key schedule.
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+// fp32 -> bf16 bits, round to nearest even; any NaN becomes 0x7FC0.
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
+  uint32_t u = __float_as_uint(f);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FC0u;
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return u >> 16;
+}
+
+// Survivor positions of a 4-chunk from its 4-bit keep mask: pad with the lowest unused
+// positions up to two, ascending; entry = p0 | p1 << 2 (16 nibbles packed in 64 bits).
+__device__ __forceinline__ uint32_t chunk_nibble(uint32_t keep4) {
+  return (uint32_t)(0x444E4DCC49884444ull >> (4 * keep4)) & 0xFu;
+}
+
+// M: group size; LANES = lanes that share a group (1, 2 or 4).
+template <int M, int SCHEME>
+__global__ void __launch_bounds__(kThreads)
+prune_kernel(const uint4* __restrict__ dO, int64_t nvec, int n, uint32_t seed_lo, uint32_t seed_hi,
+             uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
+             uint8_t* __restrict__ mask) {
+  constexpr int LANES = (M <= 8) ? 1 : M / 8;
+  constexpr int SUB = (M == 4) ? 4 : 8;  // elements of this thread that share a group
+  const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
+
+  uint4 in[kVecPerThread];
+#pragma unroll
+  for (int it = 0; it < kVecPerThread; ++it) {
+    const int64_t v = base + (int64_t)it * kThreads;
+    in[it] = (v < nvec) ? __ldg(dO + v) : make_uint4(0, 0, 0, 0);
+  }
+
+#pragma unroll
+  for (int it = 0; it < kVecPerThread; ++it) {
+    const int64_t v = base + (int64_t)it * kThreads;
+    const uint32_t w[4] = {in[it].x, in[it].y, in[it].z, in[it].w};
+    uint32_t x[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = (i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu);
+
+    // ---- ranking key: larger composite = better; unique inside a group ----
+    uint32_t key16[8];
+    if (SCHEME == SDGP_RANDOM) {
+      const uint4 o = philox4x32_10((uint32_t)v, (uint32_t)((uint64_t)v >> 32), 0u, 0u, seed_lo, seed_hi);
+      const uint32_t r[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t r16 = (i & 1) ? (r[i >> 1] >> 16) : (r[i >> 1] & 0xFFFFu);
+        key16[i] = 0xFFFFu - r16;  // smallest random key ranks first
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) key16[i] = x[i] & 0x7FFFu;  // |x| as an integer
+    }
+    const int lane_in_group = (LANES == 1) ? 0 : (threadIdx.x & (LANES - 1));
+    uint32_t c[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int j = (M == 4) ? (i & 3) : (lane_in_group * 8 + i);  // position inside the group
+      c[i] = (key16[i] << 5) | (uint32_t)(31 - j);                 // ties: lower position wins
+    }
+
+    // ---- keep <=> fewer than n elements of the group rank above ----
+    int above[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int cnt = 0;
+#pragma unroll
+      for (int o = 0; o < 8; ++o)
+        if (o != i && (o / SUB) == (i / SUB)) cnt += (c[o] > c[i]) ? 1 : 0;
+      above[i] = cnt;
+    }
+    if (LANES > 1) {
+#pragma unroll
+      for (int d = 1; d < LANES; ++d) {
+#pragma unroll
+        for (int o = 0; o < 8; ++o) {
+          const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, c[o], d);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) above[i] += (other > c[i]) ? 1 : 0;
+        }
+      }
+    }
+    uint32_t keep8 = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) keep8 |= (above[i] < n ? 1u : 0u) << i;
+
+    // ---- survivor values ----
+    uint32_t y[8];
+    if (SCHEME == SDGP_RESCALED_MAGNITUDE) {
+      float a[8], t[8], s[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        a[i] = __uint_as_float((x[i] & 0x7FFFu) << 16);
+        t[i] = a[i];
+        s[i] = ((keep8 >> i) & 1u) ? a[i] : 0.0f;
+      }
+      // balanced pairwise sums in index order; every add rounds once
+#pragma unroll
+      for (int width = 8; width > (8 / SUB); width >>= 1) {
+#pragma unroll
+        for (int i = 0; i < width / 2; ++i) {
+          t[i] = __fadd_rn(t[2 * i], t[2 * i + 1]);
+          s[i] = __fadd_rn(s[2 * i], s[2 * i + 1]);
+        }
+      }
+      // M == 4: t[0], t[1] are the two groups' sums; otherwise t[0] is this lane's partial
+      if (LANES > 1) {
+#pragma unroll
+        for (int d = 1; d < LANES; d <<= 1) {
+          t[0] = __fadd_rn(t[0], __shfl_xor_sync(0xFFFFFFFFu, t[0], d));
+          s[0] = __fadd_rn(s[0], __shfl_xor_sync(0xFFFFFFFFu, s[0], d));
+        }
+      }
+      float scale[2];
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        const int src = (M == 4) ? g : 0;
+        scale[g] = (s[src] == 0.0f) ? 1.0f : __fdiv_rn(t[src], s[src]);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float xf = __uint_as_float(x[i] << 16);
+        y[i] = ((keep8 >> i) & 1u) ? f32_to_bf16_bits(__fmul_rn(xf, scale[i >> 2])) : 0u;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) y[i] = ((keep8 >> i) & 1u) ? x[i] : 0u;
+    }
+
+    if (v >= nvec) continue;
+
+    // ---- emit ----
+    if (dense) dense[v] = make_uint4(y[0] | (y[1] << 16), y[2] | (y[3] << 16), y[4] | (y[5] << 16), y[6] | (y[7] << 16));
+    if (mask) mask[v] = (uint8_t)keep8;
+    if (values || meta) {
+      uint32_t slots[4];
+      uint32_t nib2 = 0;
+#pragma unroll
+      for (int ch = 0; ch < 2; ++ch) {
+        const uint32_t nib = chunk_nibble((keep8 >> (4 * ch)) & 0xFu);
+        const uint64_t quad = (uint64_t)(y[4 * ch] | (y[4 * ch + 1] << 16)) |
+                              ((uint64_t)(y[4 * ch + 2] | (y[4 * ch + 3] << 16)) << 32);
+        slots[2 * ch] = (uint32_t)(quad >> (16 * (nib & 3u))) & 0xFFFFu;
+        slots[2 * ch + 1] = (uint32_t)(quad >> (16 * (nib >> 2))) & 0xFFFFu;
+        nib2 |= nib << (4 * ch);
+      }
+      if (values) values[v] = make_uint2(slots[0] | (slots[1] << 16), slots[2] | (slots[3] << 16));
+      if (meta) meta[v] = (uint8_t)nib2;
+    }
+  }
+}
+
+template <int M>
+cudaError_t launch_m(int scheme, const void* dO, int64_t nvec, int n, uint64_t seed, void* dense,
+                     void* values, void* meta, void* mask, cudaStream_t stream) {
+  const int64_t per_block = (int64_t)kThreads * kVecPerThread;
+  const int64_t blocks = (nvec + per_block - 1) / per_block;
+  if (blocks == 0) return cudaSuccess;
+  if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
+  const dim3 grid((unsigned)blocks), block(kThreads);
+  const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
+#define SDGP_LAUNCH(S)                                                                              \
+  prune_kernel<M, S><<<grid, block, 0, stream>>>((const uint4*)dO, nvec, n, lo, hi, (uint4*)dense, \
+                                                 (uint2*)values, (uint8_t*)meta, (uint8_t*)mask)
+  switch (scheme) {
+    case SDGP_RANDOM: SDGP_LAUNCH(SDGP_RANDOM); break;
+    case SDGP_MAGNITUDE: SDGP_LAUNCH(SDGP_MAGNITUDE); break;
+    default: SDGP_LAUNCH(SDGP_RESCALED_MAGNITUDE); break;
+  }
+#undef SDGP_LAUNCH
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, int scheme,
+                         uint64_t seed, void* dense, void* values, void* meta, void* mask,
+                         cudaStream_t stream) {
+  const int64_t nvec = rows * (K / 8);
+  switch (m) {
+    case 4: return launch_m<4>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
+    case 8: return launch_m<8>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
+    case 16: return launch_m<16>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
+    case 32: return launch_m<32>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace sdgp

@@ -1,0 +1,78 @@
+"""Host-only checks of the C-ABI library: it loads without a GPU, exports every symbol the
+header declares, and rejects bad arguments before any launch."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2202_00774_b200 import binding
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "sdgp.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sdgp_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert "sdgp_prune" in names and "sdgp_dgrad_linear" in names and "sdgp_dgrad_conv2d" in names
+    for name in names:
+        assert hasattr(lib, name), name
+
+
+def test_binding_lists_the_same_symbols():
+    from paper_2202_00774_b200 import binding
+    assert sorted(binding.EXPORTS) == declared_symbols()
+
+
+def test_status_strings(lib):
+    seen = {lib.sdgp_status_string(i).decode() for i in range(7)}
+    assert len(seen) == 7 and "ok" in seen
+    assert lib.sdgp_status_string(99).decode() == "unknown status"
+
+
+FAKE = ctypes.c_void_p(0x1000)  # aligned, never dereferenced: every call below fails validation first
+
+
+def test_prune_rejects_bad_arguments_before_launch(lib):
+    P = lib.sdgp_prune
+    assert P(FAKE, 4, 64, 2, 4, 1, 0, None, None, None, None, None) in (0, 5)  # valid args: OK, or CUDA error with no GPU
+    assert P(FAKE, 4, 64, 0, 4, 1, 0, FAKE, None, None, None, None) == 1   # n < 1
+    assert P(FAKE, 4, 64, 5, 4, 1, 0, FAKE, None, None, None, None) == 1   # n > m
+    assert P(FAKE, 4, 64, 2, 64, 1, 0, FAKE, None, None, None, None) == 1  # m > 32
+    assert P(FAKE, 4, 64, 2, 6, 1, 0, FAKE, None, None, None, None) == 2   # m not a supported group size
+    assert P(FAKE, 4, 72, 2, 16, 1, 0, FAKE, None, None, None, None) == 1  # K % m != 0
+    assert P(FAKE, 4, 64, 2, 4, 7, 0, FAKE, None, None, None, None) == 1   # unknown scheme
+    assert P(FAKE, -1, 64, 2, 4, 1, 0, FAKE, None, None, None, None) == 1
+    assert P(None, 4, 64, 2, 4, 1, 0, FAKE, None, None, None, None) == 1   # null input
+    assert P(FAKE, 4, 64, 4, 8, 1, 0, None, FAKE, FAKE, None, None) == 2   # 4:8 has no compressed form
+    assert P(FAKE, 4, 40, 2, 4, 1, 0, FAKE, None, None, None, None) == 3   # K % 16 != 0
+    assert P(FAKE, 4, 48, 2, 4, 1, 0, None, None, None, FAKE, None) == 3   # mask needs K % 32 == 0
+    assert P(ctypes.c_void_p(0x1008), 4, 64, 2, 4, 1, 0, FAKE, None, None, None, None) == 3
+    assert P(None, 0, 64, 2, 4, 1, 0, None, None, None, None, None) == 0   # empty tensor: no-op
+
+
+def test_dgrad_rejects_bad_arguments_before_launch(lib):
+    L, C = lib.sdgp_dgrad_linear, lib.sdgp_dgrad_conv2d
+    ws = ctypes.c_void_p(0x10000)
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 2, 4, 1, 0, None, 0, 0, None) == 4        # no workspace
+    need = lib.sdgp_workspace_size_linear(128, 256, 128, 0)
+    assert need == 128 * 256 + 128 * 256 // 8
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 2, 4, 1, 0, ws, need - 1, 0, None) == 4   # short workspace
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 3, 4, 1, 0, ws, need, 0, None) == 2       # 3:4 not 2:4-compatible
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 2, 4, 1, 0, ws, need, 9, None) == 1       # unknown flags
+    assert L(FAKE, FAKE, FAKE, 128, 250, 128, 2, 4, 1, 0, ws, need, 0, None) == 1       # K % m != 0
+    assert L(None, FAKE, FAKE, 128, 256, 128, 2, 4, 1, 0, ws, need, 0, None) == 1
+    assert L(FAKE, FAKE, FAKE, 0, 256, 128, 2, 4, 1, 0, None, 0, 0, None) == 0          # rows == 0: no-op
+    assert C(FAKE, FAKE, FAKE, 2, 8, 8, 64, 128, 3, 3, 2, 1, 2, 4, 1, 0, ws, 1 << 30, 0, None) == 2  # stride 2
+    assert C(FAKE, FAKE, FAKE, 2, 8, 8, 64, 128, 3, 3, 1, 1, 2, 4, 1, 0, None, 0, 0, None) == 4
+    assert lib.sdgp_workspace_size_conv2d(2, 8, 8, 64, 128, 3, 3, 1, 1, 0) == 2 * 8 * 8 * 128 * 9 // 8
+    assert lib.sdgp_workspace_size_conv2d(2, 8, 8, 64, 128, 3, 3, 1, 1, 2) == 0

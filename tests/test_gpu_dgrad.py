@@ -1,0 +1,137 @@
+"""GPU data-gradient kernels vs the fp64 CPU oracle, through the C ABI.
+
+Tolerance: relative Frobenius error <= 5e-3 against the fp64 result computed from the same
+pruned bf16 inputs (fp32 accumulation plus one bf16 rounding per output sits near 2e-3)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2202_00774_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = 5e-3
+
+
+def dev16(a):
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
+
+
+def to_f64(t):
+    return inputs.bf16_bits_to_f32(t.cpu().numpy().view(np.uint16)).astype(np.float64)
+
+
+def rel_fro(got, ref):
+    return np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+
+
+def check_no_device_error():
+    import paper_2202_00774_b200 as sdgp
+    assert sdgp.sdgp_last_device_error() == 0
+
+
+# ------------------------------------------------------------------- linear
+
+
+@pytest.mark.parametrize("rows,K,N", [(256, 512, 256), (300, 256, 128), (77, 128, 64), (1000, 384, 192), (128, 64, 64)])
+def test_dense_linear(rows, K, N):
+    import paper_2202_00774_b200 as sdgp
+    dO, W = inputs.fc_tensors(rows, K, N, seed=rows)
+    dD = torch.full((rows, N), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, 4, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
+    check_no_device_error()
+    assert rel_fro(to_f64(dD), oracle.dgrad_linear(dO, W)) <= TOL
+
+
+@pytest.mark.parametrize("rows,K,N", [(256, 512, 256), (300, 256, 128), (77, 128, 64), (1000, 384, 192)])
+def test_spmm_linear_from_oracle_compressed(rows, K, N):
+    """The contraction alone: feed the oracle's compressed tensors to the sparse kernel."""
+    import paper_2202_00774_b200 as sdgp
+    dO, W = inputs.fc_tensors(rows, K, N, seed=rows + 1)
+    ref = oracle.prune(dO, 2, 4, oracle.MAGNITUDE, want=("dense", "values", "meta"))
+    dD = torch.full((rows, N), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_spmm_linear(dev16(ref["values"]), dev16(ref["meta"]), dev16(W), dD)
+    check_no_device_error()
+    assert rel_fro(to_f64(dD), oracle.dgrad_linear(ref["dense"], W)) <= TOL
+
+
+@pytest.mark.parametrize("scheme", [oracle.RANDOM, oracle.MAGNITUDE, oracle.RESCALED])
+@pytest.mark.parametrize("n,m", [(2, 4), (1, 4), (2, 8), (2, 16), (2, 32), (4, 4)])
+def test_pruned_linear_two_pass(n, m, scheme):
+    import paper_2202_00774_b200 as sdgp
+    rows, K, N = 333, 512, 128
+    dO, W = inputs.fc_tensors(rows, K, N, seed=n + m)
+    ws = torch.empty(sdgp.sdgp_workspace_size_linear(rows, K, N), dtype=torch.uint8, device="cuda")
+    dD = torch.full((rows, N), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, n, m, scheme, seed=42, workspace=ws)
+    check_no_device_error()
+    pruned = oracle.prune(dO, n, m, scheme, 42, want=("dense",))["dense"]
+    assert rel_fro(to_f64(dD), oracle.dgrad_linear(pruned, W)) <= TOL
+
+
+def test_fc_small_config_full():
+    """The single-FC workload: dO [256,512], W [512,256], 2:4 magnitude, seed 0."""
+    import paper_2202_00774_b200 as sdgp
+    c = inputs.FC_SMALL
+    dO, W = inputs.fc_tensors(c["rows"], c["K"], c["N"], c["seed"])
+    ws = torch.empty(sdgp.sdgp_workspace_size_linear(c["rows"], c["K"], c["N"]), dtype=torch.uint8, device="cuda")
+    dD = torch.empty((c["rows"], c["N"]), dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, 2, 4, sdgp.MAGNITUDE, workspace=ws)
+    check_no_device_error()
+    pruned = oracle.prune(dO, 2, 4, oracle.MAGNITUDE, want=("dense",))["dense"]
+    assert rel_fro(to_f64(dD), oracle.dgrad_linear(pruned, W)) <= TOL
+
+
+# --------------------------------------------------------------------- conv
+
+
+CONV_CASES = [
+    # B, H, W, Cin, Cout, R, S, pad
+    (3, 8, 8, 64, 128, 3, 3, 1),
+    (2, 16, 16, 128, 128, 3, 3, 1),
+    (5, 4, 4, 64, 256, 3, 3, 1),      # several images per tile, ragged batch
+    (1, 32, 32, 64, 128, 3, 3, 1),
+    (2, 14, 14, 64, 128, 1, 1, 0),    # 1x1, image width not a power of two
+    (3, 7, 7, 128, 128, 3, 3, 1),
+    (1, 10, 12, 64, 128, 3, 3, 0),    # no padding: output grid smaller than input grid
+    (1, 9, 9, 64, 128, 5, 5, 2),
+]
+
+
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_dense_conv(case):
+    import paper_2202_00774_b200 as sdgp
+    B, H, Wd, Cin, Cout, R, S, pad = case
+    layer = inputs.ConvLayer("t", B, H, Wd, Cin, Cout, R, S, 1, pad)
+    dO, W = inputs.conv_layer_tensors(layer, seed=H)
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, pad, 4, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
+    check_no_device_error()
+    assert rel_fro(to_f64(dD), oracle.dgrad_conv2d(dO, W, H, Wd, 1, pad)) <= TOL
+
+
+@pytest.mark.parametrize("scheme", [oracle.RANDOM, oracle.MAGNITUDE, oracle.RESCALED])
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_pruned_conv_two_pass(case, scheme):
+    import paper_2202_00774_b200 as sdgp
+    B, H, Wd, Cin, Cout, R, S, pad = case
+    layer = inputs.ConvLayer("t", B, H, Wd, Cin, Cout, R, S, 1, pad)
+    dO, W = inputs.conv_layer_tensors(layer, seed=H + 1)
+    ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(B, H, Wd, Cin, Cout, R, S, 1, pad), dtype=torch.uint8,
+                     device="cuda")
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, pad, 2, 4, scheme, seed=7, workspace=ws)
+    check_no_device_error()
+    pruned = oracle.prune(dO.reshape(-1, Cout), 2, 4, scheme, 7, want=("dense",))["dense"].reshape(dO.shape)
+    assert rel_fro(to_f64(dD), oracle.dgrad_conv2d(pruned, W, H, Wd, 1, pad)) <= TOL
+
+
+def test_unsupported_requests_raise():
+    import paper_2202_00774_b200 as sdgp
+    dO = torch.zeros((2, 4, 4, 128), dtype=torch.int16, device="cuda")
+    W = torch.zeros((128, 3, 3, 64), dtype=torch.int16, device="cuda")
+    dD = torch.zeros((2, 8, 8, 64), dtype=torch.int16, device="cuda")
+    with pytest.raises(sdgp.SdgpError) as e:
+        sdgp.sdgp_dgrad_conv2d(dO, W, dD, 2, 1, 2, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
+    assert e.value.status == 2
