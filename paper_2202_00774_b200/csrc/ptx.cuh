@@ -58,8 +58,9 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after ~2 s of wall time, records `code` in *error_word and
-// returns false; the caller carries on so that the kernel always terminates.
+// Bounded wait: gives up after ~2 s of wall time (or as soon as another wait has given up),
+// records `code` in *error_word and returns false; the caller carries on, so the kernel
+// always terminates.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* error_word,
                                           unsigned int code) {
   if (mbar_test(bar, parity)) return true;
@@ -68,6 +69,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsign
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_test(bar, parity)) return true;
+    // once any wait of any CTA has given up, no other wait lingers
+    if (*(volatile unsigned int*)error_word != 0u) return false;
     if (globaltimer_ns() - t0 > 2000000000ull) {
       atomicCAS(error_word, 0u, code);
       return false;
