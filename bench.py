@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the SDGP hot path: N:M pruning of dL/dO followed by the sparse tensor-core
+data gradient, on synthetic tensors shaped like a network's convolution layers.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet9|gemm_large|fc_small]
+                  [--scheme magnitude|rescaled|random] [--nm 2:4] [--impl ours|reference]
+
+One step = every layer of the workload once: prune kernel + sparse dgrad kernel per layer
+(the whole step replayed as one CUDA graph). Prints ONE JSON line.
+
+  value      dense-equivalent TFLOP/s of the data gradient (2*M*N*K of the implicit GEMM,
+             M = output pixels, N = Cin, K = R*S*Cout), prune time included, inputs resident.
+  e2e        same metric with the step's dL/dO copied from pinned host memory and dL/dD copied
+             back inside the timed region.
+  roofline   the dominant kernel (sparse dgrad) against twice the measured dense bf16 peak.
+  cpu_baseline  the CPU oracle on a bounded sample of the same workload.
+
+With --impl reference the CPU oracle is the timed arm (there is no other implementation of
+the paper's method to run); with more than one rank every rank runs an independent replica of
+the workload (the path shards by batch with nothing to exchange).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2202_00774_b200 import inputs  # noqa: E402
+
+SCHEMES = {"random": 0, "magnitude": 1, "rescaled": 2}
+METRIC = "dgrad_dense_equiv_tflops"
+UNIT = "TFLOP/s"
+
+
+def workload_layers(name):
+    if name == "resnet9":
+        return inputs.resnet9_layers(512)
+    if name == "gemm_large":
+        c = inputs.GEMM_LARGE
+        return [inputs.ConvLayer("gemm_16384x4096x4096", 1, 1, c["rows"], c["N"], c["K"], 1, 1, 1, 0)]
+    if name == "fc_small":
+        c = inputs.FC_SMALL
+        return [inputs.ConvLayer("fc_256x512x256", 1, 1, c["rows"], c["N"], c["K"], 1, 1, 1, 0)]
+    raise SystemExit("unknown workload " + name)
+
+
+def layer_flops(l):
+    return 2.0 * l.B * l.H * l.W * l.Cin * l.R * l.S * l.Cout
+
+
+def layer_inputs(l, workload, seed):
+    if workload == "resnet9":
+        return inputs.conv_layer_tensors(l, seed)
+    dO, W = inputs.fc_tensors(l.W, l.Cout, l.Cin, seed)
+    return dO.reshape(l.dO_shape()), W.reshape(l.W_shape())
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------- CPU oracle arm
+
+
+class OracleArm:
+    """The CPU oracle on a bounded sample: per layer, prune `p` rows of dL/dO and evaluate the
+    fp64 data gradient at `p` output pixels (the pruned neighbourhood is prepared once, outside
+    the timed region). p is scaled so that a step lasts about `seconds`."""
+
+    def __init__(self, layers, workload, n, m, scheme):
+        import oracle
+        oracle.build()
+        self.oracle = oracle
+        self.n, self.m, self.scheme = n, m, scheme
+        self.layers = [inputs.ConvLayer(l.name, min(l.B, 4), l.H, min(l.W, 2048) if l.B == 1 and l.H == 1 else l.W,
+                                        l.Cin, l.Cout, l.R, l.S, l.stride, l.pad) for l in layers]
+        self.tensors = [layer_inputs(l, workload, 0) for l in self.layers]
+        self.pruned = [oracle.prune(dO.reshape(-1, l.Cout), n, m, scheme, 0, want=("dense",))["dense"].reshape(dO.shape)
+                       for l, (dO, _) in zip(self.layers, self.tensors)]
+        self.cores = oracle.omp_threads()
+
+    def step(self, pixels):
+        flops = 0.0
+        for l, (dO, W), pruned in zip(self.layers, self.tensors, self.pruned):
+            p = int(max(1, min(pixels, l.B * l.H * l.W, l.B * l.P * l.Q)))
+            self.oracle.prune(dO.reshape(-1, l.Cout)[:p], self.n, self.m, self.scheme, 0, want=("dense",))
+            self.oracle.dgrad_conv2d(pruned, W, l.H, l.W, l.stride, l.pad, pixel_index=np.arange(p, dtype=np.int64))
+            flops += 2.0 * p * l.Cin * l.R * l.S * l.Cout
+        return flops
+
+    def pixels_for(self, seconds):
+        probe = 8
+        t0 = time.perf_counter()
+        self.step(probe)
+        dt = max(time.perf_counter() - t0, 1e-6)
+        return int(max(1, probe * seconds / dt))
+
+
+def cpu_baseline(layers, workload, n, m, scheme, target_s=15.0):
+    arm = OracleArm(layers, workload, n, m, scheme)
+    pixels = arm.pixels_for(target_s)
+    t0 = time.perf_counter()
+    flops = arm.step(pixels)
+    dt = time.perf_counter() - t0
+    return dict(value=flops / dt / 1e12, unit=UNIT, cores=arm.cores, kind="oracle",
+                sample="up to %d rows pruned + %d output pixels of fp64 dgrad per layer, %.1f s" % (pixels, pixels, dt))
+
+
+def run_reference(args, layers):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n, m = [int(v) for v in args.nm.split(":")]
+    arm = OracleArm(layers, args.workload, n, m, SCHEMES[args.scheme])
+    budget = min(20.0, 150.0 / max(1, args.steps + args.warmup))  # whole run stays within a few minutes
+    pixels = arm.pixels_for(budget)
+    for _ in range(args.warmup):
+        arm.step(pixels)
+    t0 = time.perf_counter()
+    flops = 0.0
+    for _ in range(args.steps):
+        flops += arm.step(pixels)
+    dt = time.perf_counter() - t0
+    value = flops / dt / 1e12
+    sample = "each step: up to %d rows pruned + %d output pixels of fp64 dgrad per layer" % (pixels, pixels)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "nm": args.nm, "scheme": args.scheme, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": arm.cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# -------------------------------------------------------------------- GPU arm
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(device_index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(smax)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+def run_ours(args, layers):
+    import torch
+    import paper_2202_00774_b200 as sdgp
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    n, m = [int(v) for v in args.nm.split(":")]
+    scheme = SCHEMES[args.scheme]
+    pk = peaks()
+
+    def dev16(a):
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
+
+    host_tensors = [layer_inputs(l, args.workload, seed=rank) for l in layers]
+    dO = [dev16(t[0]) for t in host_tensors]
+    Wt = [dev16(t[1]) for t in host_tensors]
+    dD = [torch.empty(l.dD_shape(), dtype=torch.int16, device="cuda") for l in layers]
+    ws = [torch.empty(max(16, sdgp.sdgp_workspace_size_conv2d(l.B, l.H, l.W, l.Cin, l.Cout, l.R, l.S, l.stride, l.pad)),
+                      dtype=torch.uint8, device="cuda") for l in layers]
+    total_flops = sum(layer_flops(l) for l in layers)
+    order = list(range(len(layers)))[::-1]  # backward pass: last layer first
+
+    def sparse_step():
+        for i in order:
+            l = layers[i]
+            sdgp.sdgp_dgrad_conv2d(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, seed=1234, workspace=ws[i],
+                                   flags=sdgp.FLAG_TWO_PASS)
+
+    def dense_step():
+        for i in order:
+            l = layers[i]
+            sdgp.sdgp_dgrad_conv2d(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, flags=sdgp.FLAG_DENSE)
+
+    def capture(fn):
+        stream = torch.cuda.Stream()
+        stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(stream):
+            fn()  # warm-up outside capture: first calls configure kernel attributes
+        torch.cuda.current_stream().wait_stream(stream)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g
+
+    def timed(replay, steps, warmup):
+        for _ in range(warmup):
+            replay()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dist.barrier()
+            ms = float(t.item())
+        torch.cuda.synchronize()
+        return ms
+
+    g_sparse = capture(sparse_step)
+    g_dense = capture(dense_step)
+
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    ms_sparse = timed(g_sparse.replay, args.steps, args.warmup)
+    clocks = sampler.stop() if sampler else None
+    dense_steps = max(3, args.steps // 4)
+    ms_dense = timed(g_dense.replay, dense_steps, max(3, args.warmup // 2))
+
+    ms_per_step = ms_sparse / args.steps
+    value = world * total_flops / (ms_per_step * 1e-3) / 1e12
+    dense_value = world * total_flops / (ms_dense / dense_steps * 1e-3) / 1e12
+
+    # ---- per-kernel timing (eager launches with events around each kernel) ----
+    per_steps = min(args.steps, 20)
+    prune_ms = [0.0] * len(layers)
+    dgrad_ms = [0.0] * len(layers)
+    vals = [torch.empty(l.B * l.P * l.Q * l.Cout // 2, dtype=torch.int16, device="cuda") for l in layers]
+    metas = [torch.empty(l.B * l.P * l.Q * l.Cout // 16, dtype=torch.int16, device="cuda") for l in layers]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in layers]
+    for it in range(per_steps + 3):
+        for i in order:
+            l = layers[i]
+            evs[i][0].record()
+            sdgp.sdgp_prune(dO[i].view(-1, l.Cout), n, m, scheme, 1234, values=vals[i], meta=metas[i])
+            evs[i][1].record()
+            sdgp.sdgp_spmm_conv2d(vals[i].view(l.B, l.P, l.Q, l.Cout // 2), metas[i].view(l.B, l.P, l.Q, l.Cout // 16),
+                                  Wt[i], dD[i], l.stride, l.pad)
+            evs[i][2].record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            for i in order:
+                prune_ms[i] += evs[i][0].elapsed_time(evs[i][1])
+                dgrad_ms[i] += evs[i][1].elapsed_time(evs[i][2])
+    status = sdgp.sdgp_last_device_error()
+    if status != 0:
+        raise SystemExit("device error: " + sdgp.status_string(status))
+    prune_bytes = sum(l.B * l.P * l.Q * l.Cout * 3.125 for l in layers)
+    prune_gbs = prune_bytes * per_steps / (sum(prune_ms) * 1e-3) / 1e9
+    dgrad_tflops = total_flops * per_steps / (sum(dgrad_ms) * 1e-3) / 1e12
+    sparse_peak = 2.0 * pk["bf16_sustained"]
+    per_layer = [{"layer": l.name, "prune_us": 1e3 * prune_ms[i] / per_steps, "dgrad_us": 1e3 * dgrad_ms[i] / per_steps,
+                  "dgrad_dense_equiv_tflops": layer_flops(l) / (dgrad_ms[i] / per_steps * 1e-3) / 1e12,
+                  "prune_gbs": l.B * l.P * l.Q * l.Cout * 3.125 / (prune_ms[i] / per_steps * 1e-3) / 1e9}
+                 for i, l in enumerate(layers)]
+
+    # ---- end to end: dL/dO from pinned host memory, dL/dD back to the host, every step ----
+    h_in = [torch.from_numpy(np.ascontiguousarray(t[0]).view(np.int16)).pin_memory() for t in host_tensors]
+    h_out = [torch.empty(l.dD_shape(), dtype=torch.int16).pin_memory() for l in layers]
+    h2d = sum(t.numel() * 2 for t in h_in)
+    d2h = sum(t.numel() * 2 for t in h_out)
+
+    def e2e_step():
+        for i in order:
+            dO[i].copy_(h_in[i], non_blocking=True)
+        sparse_step()
+        for i in order:
+            h_out[i].copy_(dD[i], non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    ms_e2e = timed(e2e_step, e2e_steps, 3)
+    e2e_value = world * total_flops / (ms_e2e / e2e_steps * 1e-3) / 1e12
+
+    if rank == 0:
+        base = cpu_baseline(layers, args.workload, n, m, scheme) if world == 1 and not args.no_cpu_baseline else None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "layers": len(layers), "nm": args.nm, "scheme": args.scheme,
+                       "mode": "two_pass", "flops": "2*M*N*K of the implicit GEMM per layer",
+                       "l2": "inputs larger than L2 (step touches %.0f MB)" % ((prune_bytes + d2h) / 1e6),
+                       "launch": "one CUDA graph per step", "replicas": world},
+            "speedup_vs_dense": value / dense_value, "dense_tflops": dense_value,
+            "prune_gbs": prune_gbs, "prune_frac_of_hbm": prune_gbs / pk["hbm"],
+            "roofline": {"bound": "tensor", "kernel": "dgrad_kernel<sparse>", "achieved": dgrad_tflops,
+                         "peak": sparse_peak, "unit": "TFLOP/s", "frac": dgrad_tflops / sparse_peak,
+                         "traffic": None,
+                         "note": "dense-equivalent FLOPs of all sparse dgrad launches / their summed event time; "
+                                 "peak = 2 x %s sustained dense bf16" % pk["source"]},
+            "per_layer": per_layer,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": 2 * len(layers) * args.steps,
+            "clocks": clocks,
+        }
+        if base is not None:
+            line["cpu_baseline"] = base
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet9", choices=["resnet9", "gemm_large", "fc_small"])
+    ap.add_argument("--scheme", default="magnitude", choices=sorted(SCHEMES))
+    ap.add_argument("--nm", default="2:4")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    layers = workload_layers(args.workload)
+    if args.impl == "reference":
+        run_reference(args, layers)
+    else:
+        run_ours(args, layers)
+
+
+if __name__ == "__main__":
+    main()
