@@ -60,7 +60,8 @@ typedef enum {
   SDGP_ERR_ALIGNMENT = 3,   /* pointer not 16-byte aligned / extent not a multiple the layout needs */
   SDGP_ERR_WORKSPACE = 4,   /* workspace missing or smaller than sdgp_workspace_size_*() */
   SDGP_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, tensor-map encode, ...) */
-  SDGP_ERR_TIMEOUT = 6      /* a bounded wait inside a kernel ran out (see sdgp_last_device_error) */
+  SDGP_ERR_TIMEOUT = 6,     /* a bounded wait inside a kernel ran out (see sdgp_last_device_error) */
+  SDGP_ERR_TOO_LARGE = 7    /* problem exceeds the fixed scratch of sdgp_dgrad_linear_static */
 } sdgp_status;
 
 typedef enum { SDGP_RANDOM = 0, SDGP_MAGNITUDE = 1, SDGP_RESCALED_MAGNITUDE = 2 } sdgp_scheme;
@@ -114,6 +115,23 @@ sdgp_status sdgp_spmm_linear(const void* values, const void* meta, const void* W
 sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W, void* dD, int B,
                              int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
                              void* stream);
+
+/* No counterpart in the paper: a convenience variant of sdgp_dgrad_linear (two-pass mode) that
+ * takes no workspace and allocates nothing - for callers that cannot call cudaMalloc where
+ * the gradient is computed (inside another runtime's no-allocation region, in a plugin whose
+ * host owns all device memory, in a latency-critical loop). The compressed dL/dO goes into a
+ * 9 MiB array that is part of the library image in device memory, so every GPU that loads the
+ * library holds those 9 MiB until the process exits.
+ *   Limit: rows * K <= 8,388,608 elements (e.g. 4096 x 2048); larger -> SDGP_ERR_TOO_LARGE.
+ *   Same requirements as sdgp_dgrad_linear otherwise (K % 128 == 0, N % 64 == 0, n <= 2, ...).
+ *   The first call on each device looks up the array's device address (one host-side runtime
+ *   query, no allocation); make that first call outside any stream capture.
+ *   All calls on a device share the one array: two calls whose kernels may overlap on the GPU
+ *   (different streams, no dependency) race on it and give wrong results - serialise them.
+ *   Nothing in the array has to be cleared between calls: each call rewrites what it reads. */
+sdgp_status sdgp_dgrad_linear_static(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,
+                                     int64_t N, int n, int m, sdgp_scheme scheme, uint64_t seed,
+                                     void* stream);
 
 /* Bytes of workspace the matching dgrad call needs for these shapes and flags (0 for
  * SDGP_FLAG_DENSE and SDGP_FLAG_FUSED). */

@@ -17,6 +17,7 @@ RANDOM, MAGNITUDE, RESCALED_MAGNITUDE = 0, 1, 2
 FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE = 0, 1, 2
 
 EXPORTS = ["sdgp_prune", "sdgp_dgrad_linear", "sdgp_dgrad_conv2d", "sdgp_spmm_linear", "sdgp_spmm_conv2d",
+           "sdgp_dgrad_linear_static",
            "sdgp_workspace_size_linear", "sdgp_workspace_size_conv2d", "sdgp_last_device_error",
            "sdgp_status_string"]
 
@@ -47,6 +48,8 @@ def lib() -> ctypes.CDLL:
         L.sdgp_dgrad_linear.restype = i32
         L.sdgp_dgrad_conv2d.argtypes = [vp, vp, vp] + [i32] * 9 + [i32, i32, i32, u64, vp, sz, u32, vp]
         L.sdgp_dgrad_conv2d.restype = i32
+        L.sdgp_dgrad_linear_static.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, u64, vp]
+        L.sdgp_dgrad_linear_static.restype = i32
         L.sdgp_spmm_linear.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
         L.sdgp_spmm_linear.restype = i32
         L.sdgp_spmm_conv2d.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
@@ -113,6 +116,18 @@ def sdgp_dgrad_linear(dO, W, dD, n, m, scheme, seed=0, workspace=None, flags=FLA
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().sdgp_dgrad_linear(_ptr(dO), _ptr(W), _ptr(dD), rows, K, N, n, m, scheme, seed,
                                    _ptr(workspace), ws_bytes, flags, _stream()), "sdgp_dgrad_linear")
+
+
+def sdgp_dgrad_linear_static(dO, W, dD, n, m, scheme, seed=0):
+    """``sdgp_dgrad_linear_static``: like :func:`sdgp_dgrad_linear` in two-pass mode, but the
+    scratch is the library's own fixed device array - for callers that cannot allocate a
+    workspace. rows*K is limited to 8Mi elements; calls must not overlap on the GPU."""
+    for t, name in ((dO, "dO"), (W, "W"), (dD, "dD")):
+        _dev(t, name)
+    rows, K = dO.shape
+    N = W.shape[1]
+    _check(lib().sdgp_dgrad_linear_static(_ptr(dO), _ptr(W), _ptr(dD), rows, K, N, n, m, scheme, seed,
+                                          _stream()), "sdgp_dgrad_linear_static")
 
 
 def sdgp_dgrad_conv2d(dO, W, dD, stride, pad, n, m, scheme, seed=0, workspace=None, flags=FLAG_TWO_PASS):

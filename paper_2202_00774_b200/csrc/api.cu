@@ -45,6 +45,7 @@ const char* sdgp_status_string(sdgp_status status) {
     case SDGP_ERR_WORKSPACE: return "workspace missing or too small";
     case SDGP_ERR_CUDA: return "CUDA call failed";
     case SDGP_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case SDGP_ERR_TOO_LARGE: return "problem exceeds the library's fixed scratch capacity";
   }
   return "unknown status";
 }
