@@ -43,6 +43,8 @@ struct DgradParams {
   int tiles_w, tiles_h, tiles_b, tiles_n;
   int total_tiles;
   int k_blocks_per_tap; // ceil(Cout / channels per stage)
+  int m_tiles;          // tiles_w * tiles_h * tiles_b
+  int pair_tiles;       // CTA-pair kernel: ceil(m_tiles / 2) * tiles_n
   uint16_t* dD;
 };
 
@@ -64,6 +66,53 @@ struct Cfg {
 __host__ __device__ constexpr uint32_t make_idesc(int n, bool sparse) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
          ((uint32_t)(kBM >> 4) << 24) | (sparse ? (1u << 2) : 0u);
+}
+
+
+// One row of a stage's metadata: from the row-major order TMA delivers (8 uint16 per pixel,
+// one per 16 channels) to the order tcgen05.cp moves into TMEM. For the MMA covering channels
+// [32*k2, 32*k2+32) of the stage the tensor core reads one 32-bit TMEM column: lane
+// (row%8) + 8*half + 16*(row/16) holds in its low 16 bits the four position nibbles of channels
+// 32*k2 + 16*half + [0,16) of the row with bit 3 clear and in its high 16 bits those of row + 8.
+__device__ __forceinline__ void rearrange_metadata(const uint8_t* raw_stage, uint8_t* hw_stage, int row,
+                                                   int rows_used) {
+  const uint4 raw = *(const uint4*)(raw_stage + row * 16);
+  const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
+  uint16_t* hw = (uint16_t*)hw_stage;
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    uint32_t v = (u & 1) ? (w4[u >> 1] >> 16) : (w4[u >> 1] & 0xFFFFu);
+    // rows outside the patch or outside the image carry no data: give them the well-formed
+    // position pair (0,1) in every chunk
+    if (row >= rows_used || v == 0u) v = 0x4444u;
+    const int tl = (row & 7) + 8 * (u & 1) + 16 * (row >> 4);
+    hw[tl * 8 + 2 * (u >> 1) + ((row >> 3) & 1)] = (uint16_t)v;
+  }
+}
+
+// This warp's 32 accumulator rows x BN columns: TMEM -> registers -> bf16 -> global.
+template <int BN>
+__device__ __forceinline__ void store_accumulator(uint32_t taddr, uint16_t* out, bool valid) {
+#pragma unroll 1
+  for (int c0 = 0; c0 < BN; c0 += 32) {
+    uint32_t v[32];
+    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
+    ptx::tmem_ld_wait();
+    if (valid) {
+      uint4* dst = (uint4*)(out + c0);
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        uint32_t w2[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * g + 2 * e]),
+                                                          __uint_as_float(v[8 * g + 2 * e + 1]));
+          w2[e] = *(const uint32_t*)&h2;
+        }
+        dst[g] = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+      }
+    }
+  }
 }
 
 template <bool SPARSE, int BN>
@@ -205,22 +254,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           const int st = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           ptx::mbar_wait(&full[st], ph, err, 0x500u + st);
-          const uint4 raw = *(const uint4*)(sEraw + st * kEBytes + row * 16);
-          const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
-          uint16_t* hw = (uint16_t*)(sEhw + st * kEBytes);
-          // The tensor core reads, for the MMA covering channels [32*k2, 32*k2+32) of the stage,
-          // one 32-bit TMEM column: lane (row%8) + 8*half + 16*(row/16) holds in its low 16 bits
-          // the four position nibbles of channels 32*k2 + 16*half + [0,16) of row (row with bit 3
-          // clear) and in its high 16 bits those of row + 8.
-#pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            uint32_t v = (u & 1) ? (w4[u >> 1] >> 16) : (w4[u >> 1] & 0xFFFFu);
-            // rows outside the patch or outside the image carry no data: give them the
-            // well-formed position pair (0,1) in every chunk
-            if (row >= rows_used || v == 0u) v = 0x4444u;
-            const int tl = (row & 7) + 8 * (u & 1) + 16 * (row >> 4);
-            hw[tl * 8 + 2 * (u >> 1) + ((row >> 3) & 1)] = (uint16_t)v;
-          }
+          rearrange_metadata(sEraw + st * kEBytes, sEhw + st * kEBytes, row, rows_used);
           ptx::fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&meta_ready[st]);
@@ -248,26 +282,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       ptx::mbar_wait(&acc_full[acc], aph, err, 0x600u + acc);
       ptx::tc_fence_after_sync();
       uint16_t* out = p.dD + (((int64_t)b * p.H + h) * p.W + w) * (int64_t)p.Cin + (int64_t)nt * BN;
-#pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
-        ptx::tmem_ld_wait();
-        if (valid) {
-          uint4* dst = (uint4*)(out + c0);
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint32_t w2[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * g + 2 * e]),
-                                                              __uint_as_float(v[8 * g + 2 * e + 1]));
-              w2[e] = *(const uint32_t*)&h2;
-            }
-            dst[g] = make_uint4(w2[0], w2[1], w2[2], w2[3]);
-          }
-        }
-      }
+      store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), out, valid);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
@@ -278,6 +293,227 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   __syncthreads();
   ptx::tc_fence_after_sync();
   if (warp == 1) ptx::tmem_dealloc(tmem_base, kTmemCols);
+}
+
+
+// ------------------------------------------------------------------------------------------
+// CTA-pair variant (cta_group::2). Two CTAs of a cluster own two neighbouring 128-pixel
+// patches and one BN-wide column block: each stages its own A patch (+ metadata) and HALF of
+// the W columns, and a single thread of the pair's first CTA issues 256-row MMAs that read
+// both halves. Per CTA this halves the W bytes and TMA requests per FLOP and the shared-memory
+// reads of B, and leaves room in TMEM for BN = 256.
+//
+// Barriers: full / meta_ready / acc_empty are waited on by the first CTA only and collect
+// arrivals from both; empty / acc_full exist in both CTAs and are signalled together by a
+// multicast tcgen05.commit; meta_full is local (each CTA's own metadata box).
+
+template <bool SPARSE, int BN>
+struct PairCfg {
+  static constexpr int kKB = SPARSE ? 128 : 64;
+  static constexpr int kBCols = BN / 2;                    // W columns staged by one CTA
+  static constexpr int kBBytes = kKB * kBCols * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes + (SPARSE ? 2 * kEBytes : 0);
+  static constexpr int kSmemBudget = 232448 - 2048;
+  static constexpr int kStagesFit = kSmemBudget / kStageBytes;
+  static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
+  static constexpr int kAcc = (2 * BN + (SPARSE ? 4 * kStages : 0) <= (int)kTmemCols) ? 2 : 1;
+  static constexpr int kMetaCol = kAcc * BN;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 2048;
+  static_assert(kBCols % 64 == 0, "each CTA stages whole 64-column swizzle blocks of W");
+  static_assert(kStages >= 2, "pipeline needs at least two stages");
+};
+
+__host__ __device__ constexpr uint32_t make_idesc_pair(int n, bool sparse) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(256 >> 4) << 24) | (sparse ? (1u << 2) : 0u);
+}
+
+template <bool SPARSE, int BN>
+__global__ void __launch_bounds__(kThreadsGemm, 1)
+dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmE,
+                  const __grid_constant__ CUtensorMap tmB, const DgradParams p) {
+  using C = PairCfg<SPARSE, BN>;
+  constexpr int STAGES = C::kStages;
+  constexpr int NACC = C::kAcc;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sA = smem;
+  uint8_t* sB = sA + STAGES * kABytes;
+  uint8_t* sEraw = sB + STAGES * C::kBBytes;
+  uint8_t* sEhw = sEraw + (SPARSE ? STAGES * kEBytes : 0);
+  uint64_t* bars = (uint64_t*)(sEhw + (SPARSE ? STAGES * kEBytes : 0));
+  uint64_t* full = bars;
+  uint64_t* empty = full + STAGES;
+  uint64_t* meta_full = empty + STAGES;
+  uint64_t* meta_ready = meta_full + STAGES;
+  uint64_t* acc_full = meta_ready + STAGES;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();  // 0: issues the MMAs
+  unsigned int* err = &g_device_error;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+      ptx::mbar_init(&meta_full[s], 1);
+      ptx::mbar_init(&meta_ready[s], 8);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&acc_full[a], 1);
+      ptx::mbar_init(&acc_empty[a], 8);
+    }
+    ptx::fence_mbar_init();
+  }
+  if (warp == 0 && lane == 0) {
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+    if (SPARSE) ptx::prefetch_tensormap(&tmE);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before_sync();
+  ptx::cluster_sync();  // barrier inits and TMEM of both CTAs are ready before any cross-CTA signal
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int rows_used = p.TW * p.TH * p.TB;
+  const int taps = p.R * p.S;
+  const int k_iters = taps * p.k_blocks_per_tap;
+  const int pair_stride = gridDim.x >> 1;
+  const int first_pair = blockIdx.x >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer
+    if (ptx::elect_one()) {
+      const uint32_t pair_tx = 2u * (uint32_t)(rows_used * 128 + C::kBBytes);
+      uint32_t it = 0;
+      for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride) {
+        const int nt = pt % p.tiles_n;
+        int t = 2 * (pt / p.tiles_n) + (int)rank;  // this CTA's patch; may lie past the last one
+        const int wt = t % p.tiles_w; t /= p.tiles_w;
+        const int ht = t % p.tiles_h; t /= p.tiles_h;
+        const int bt = t;
+        const int n0 = nt * BN + (int)rank * C::kBCols;
+        const int w0 = wt * p.TW, h0 = ht * p.TH, b0 = bt * p.TB;
+        for (int tap = 0; tap < taps; ++tap) {
+          const int r = tap / p.S, s = tap - r * p.S;
+          const int q0 = w0 + p.pad - s, p0 = h0 + p.pad - r;
+          for (int cb = 0; cb < p.k_blocks_per_tap; ++cb, ++it) {
+            const int st = it % STAGES;
+            const uint32_t ph = (it / STAGES) & 1u;
+            ptx::mbar_wait(&empty[st], ph ^ 1u, err, 0x1100u + st);
+            if (rank == 0) ptx::mbar_arrive_expect_tx(&full[st], pair_tx);
+            if (SPARSE) {
+              ptx::mbar_arrive_expect_tx(&meta_full[st], (uint32_t)(rows_used * 16));
+              ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &meta_full[st], cb * 8, q0, p0, b0);
+            }
+            ptx::tma_load_4d_pair(sA + st * kABytes, &tmA, &full[st], cb * 64, q0, p0, b0);
+#pragma unroll
+            for (int j = 0; j < C::kBCols / 64; ++j)
+              ptx::tma_load_2d_pair(sB + st * C::kBBytes + j * (C::kKB * 128), &tmB, &full[st],
+                                    tap * p.Cin + n0 + 64 * j, cb * C::kKB);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------- MMA issuer (first CTA only)
+    if (rank == 0 && ptx::elect_one()) {
+      constexpr uint32_t idesc = make_idesc_pair(BN, SPARSE);
+      uint32_t it = 0, lt = 0;
+      for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride, ++lt) {
+        const int acc = lt % NACC;
+        const uint32_t aph = (lt / NACC) & 1u;
+        ptx::mbar_wait(&acc_empty[acc], aph ^ 1u, err, 0x1200u + acc);
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < k_iters; ++kb, ++it) {
+          const int st = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          ptx::mbar_wait(&full[st], ph, err, 0x1300u + st);
+          if (SPARSE) ptx::mbar_wait(&meta_ready[st], ph, err, 0x1400u + st);
+          ptx::tc_fence_after_sync();
+          const uint64_t adesc = ptx::make_smem_desc(ptx::smem_u32(sA + st * kABytes), 16, 1024, 2);
+          const uint64_t bdesc =
+              ptx::make_smem_desc(ptx::smem_u32(sB + st * C::kBBytes), C::kKB * 128, 1024, 2);
+          if (SPARSE) {
+            const uint64_t edesc = ptx::make_smem_desc(ptx::smem_u32(sEhw + st * kEBytes), 128, 128, 0);
+            ptx::tc_cp_128x128b_pair(tmem_base + (uint32_t)(C::kMetaCol + 4 * st), edesc);
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t accumulate = (kb > 0 || j > 0) ? 1u : 0u;
+            const uint64_t a_j = adesc + (uint64_t)(j * 2);
+            const uint64_t b_j = bdesc + (uint64_t)(j * (C::kKB / 4) * 128 / 16);
+            if (SPARSE) {
+              const uint32_t col = (uint32_t)(C::kMetaCol + 4 * st + j);
+              ptx::mma_sp_f16_ss_pair(d_tmem, a_j, b_j, tmem_base + (col & ~1u), idesc | (col & 1u), accumulate);
+            } else {
+              ptx::mma_f16_ss_pair(d_tmem, a_j, b_j, idesc, accumulate);
+            }
+          }
+          ptx::tc_commit_pair(&empty[st], 3);
+        }
+        ptx::tc_commit_pair(&acc_full[acc], 3);
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------- metadata rearranger
+    if (SPARSE) {
+      const int row = threadIdx.x - 64;
+      uint32_t it = 0;
+      for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride) {
+        for (int kb = 0; kb < k_iters; ++kb, ++it) {
+          const int st = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          ptx::mbar_wait(&meta_full[st], ph, err, 0x1500u + st);
+          rearrange_metadata(sEraw + st * kEBytes, sEhw + st * kEBytes, row, rows_used);
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(&meta_ready[st], 0);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const int tw = row % p.TW;
+    const int th = (row / p.TW) % p.TH;
+    const int tb = row / (p.TW * p.TH);
+    uint32_t lt = 0;
+    for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride, ++lt) {
+      const int nt = pt % p.tiles_n;
+      int t = 2 * (pt / p.tiles_n) + (int)rank;
+      const int wt = t % p.tiles_w; t /= p.tiles_w;
+      const int ht = t % p.tiles_h; t /= p.tiles_h;
+      const int bt = t;
+      const int w = wt * p.TW + tw, h = ht * p.TH + th, b = bt * p.TB + tb;
+      const bool valid = row < rows_used && w < p.W && h < p.H && b < p.B;
+      const int acc = lt % NACC;
+      const uint32_t aph = (lt / NACC) & 1u;
+      ptx::mbar_wait(&acc_full[acc], aph, err, 0x1600u + acc);
+      ptx::tc_fence_after_sync();
+      uint16_t* out = p.dD + (((int64_t)b * p.H + h) * p.W + w) * (int64_t)p.Cin + (int64_t)nt * BN;
+      store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), out, valid);
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
+    }
+  }
+
+  ptx::tc_fence_before_sync();
+  __syncwarp();
+  ptx::cluster_sync();  // neither CTA leaves (or frees TMEM) while the other may still touch it
+  ptx::tc_fence_after_sync();
+  if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
 }
 
 // ------------------------------------------------------------------- host
@@ -363,6 +599,34 @@ sdgp_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmE, const CUt
   return cudaGetLastError() == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
+template <bool SPARSE, int BN>
+sdgp_status launch_pair_cfg(const CUtensorMap& tmA, const CUtensorMap& tmE, const CUtensorMap& tmB,
+                            const DgradParams& p, cudaStream_t stream) {
+  using C = PairCfg<SPARSE, BN>;
+  static bool configured = false;
+  auto kernel = dgrad_pair_kernel<SPARSE, BN>;
+  if (!configured) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
+      return SDGP_ERR_CUDA;
+    configured = true;
+  }
+  const int max_pairs = sm_count() / 2;
+  const int pairs = p.pair_tiles < max_pairs ? p.pair_tiles : max_pairs;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3(kThreadsGemm);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, tmA, tmE, tmB, p) == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
+}
+
 }  // namespace
 
 // A: dense dL/dO [B,P,Q,Cout] (sparse == false) or compressed values [B,P,Q,Cout/2] with
@@ -375,18 +639,25 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
   if (Cin % 64 != 0 || Cout % (sparse ? 128 : 64) != 0) return SDGP_ERR_UNSUPPORTED;
   if ((int64_t)R * S * Cin > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
 
+  // CTA pairs whenever the column count allows whole 64-column halves; the single-CTA kernel
+  // serves Cin = 64 (mod 128).
+  const bool pair = (Cin % 128 == 0);
+  const int BN = pair ? ((Cin % 256 == 0) ? 256 : 128) : 64;
+  const int kb_channels = sparse ? 128 : 64;
+
   DgradParams p;
   p.B = B; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout; p.R = R; p.S = S; p.pad = pad;
   choose_patch(B, H, W, &p.TW, &p.TH, &p.TB);
-  const int BN = (Cin % 128 == 0) ? 128 : 64;
   p.tiles_w = (W + p.TW - 1) / p.TW;
   p.tiles_h = (H + p.TH - 1) / p.TH;
   p.tiles_b = (B + p.TB - 1) / p.TB;
   p.tiles_n = Cin / BN;
-  const int64_t total = (int64_t)p.tiles_w * p.tiles_h * p.tiles_b * p.tiles_n;
-  if (total > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
+  const int64_t m_tiles = (int64_t)p.tiles_w * p.tiles_h * p.tiles_b;
+  const int64_t total = m_tiles * p.tiles_n;
+  if (total > 0x3FFFFFFF) return SDGP_ERR_UNSUPPORTED;
+  p.m_tiles = (int)m_tiles;
   p.total_tiles = (int)total;
-  const int kb_channels = sparse ? 128 : 64;
+  p.pair_tiles = (int)((m_tiles + 1) / 2) * p.tiles_n;
   p.k_blocks_per_tap = (Cout + kb_channels - 1) / kb_channels;
   p.dD = (uint16_t*)dD;
 
@@ -417,12 +688,14 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
       return SDGP_ERR_CUDA;
   }
 
-  if (sparse) {
-    return BN == 128 ? launch_cfg<true, 128>(tmA, tmE, tmB, p, stream)
-                     : launch_cfg<true, 64>(tmA, tmE, tmB, p, stream);
+  if (pair) {
+    if (sparse)
+      return BN == 256 ? launch_pair_cfg<true, 256>(tmA, tmE, tmB, p, stream)
+                       : launch_pair_cfg<true, 128>(tmA, tmE, tmB, p, stream);
+    return BN == 256 ? launch_pair_cfg<false, 256>(tmA, tmE, tmB, p, stream)
+                     : launch_pair_cfg<false, 128>(tmA, tmE, tmB, p, stream);
   }
-  return BN == 128 ? launch_cfg<false, 128>(tmA, tmE, tmB, p, stream)
-                   : launch_cfg<false, 64>(tmA, tmE, tmB, p, stream);
+  return sparse ? launch_cfg<true, 64>(tmA, tmE, tmB, p, stream) : launch_cfg<false, 64>(tmA, tmE, tmB, p, stream);
 }
 
 sdgp_status read_device_error() {
