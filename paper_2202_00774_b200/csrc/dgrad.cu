@@ -10,10 +10,10 @@
 //               box of metadata, and BN/64 boxes of W.
 //   warp 1      MMA issuer: copies the stage's metadata into TMEM (tcgen05.cp), issues four
 //               MMAs per stage into a TMEM accumulator, commits to the stage's "empty" barrier.
-//   warps 2-5   (sparse only) rearrange the stage's row-major metadata into the lane/column
-//               order the tensor core reads from TMEM.
-//   warps 6-9   epilogue: TMEM -> registers -> bf16 -> global, overlapped with the next tile's
-//               main loop through a second accumulator.
+//   warps 2-5   (sparse only) rearrange the stages' row-major metadata into the lane/column
+//               order the tensor core reads from TMEM, one warp per stage, four stages at once.
+//   warps 6-9   epilogue: TMEM -> registers -> bf16 -> swizzled staging tile -> TMA store,
+//               overlapped with the next tile's main loop through a second accumulator.
 //
 // Every mbarrier wait is bounded; a wait that runs out records a code in g_device_error and
 // the kernel still runs to completion and frees its TMEM.
@@ -34,6 +34,7 @@ constexpr int kThreadsGemm = 320;  // 10 warps
 constexpr int kABytes = kBM * 128; // one A stage: 128 rows x 128 B (64 bf16, dense or compressed)
 constexpr int kEBytes = kBM * 16;  // one metadata stage: 128 rows x 8 uint16
 constexpr uint32_t kTmemCols = 512;
+constexpr int kOutBytes = kBM * 128;  // epilogue staging: 128 rows x 64 bf16 columns
 
 struct DgradParams {
   int B, H, W;          // dD pixel grid (fully connected: B = H = 1, W = rows)
@@ -54,11 +55,12 @@ struct Cfg {
   static constexpr int kBBytes = kKB * BN * 2;
   static constexpr int kStageBytes = kABytes + kBBytes + (SPARSE ? 2 * kEBytes : 0);
   static constexpr int kSmemBudget = 232448 - 2048;       // max dynamic smem minus barriers/alignment slack
-  static constexpr int kStagesFit = kSmemBudget / kStageBytes;
+  static constexpr int kOutBufs = ((kSmemBudget - 2 * kOutBytes) / kStageBytes >= 4) ? 2 : 1;
+  static constexpr int kStagesFit = (kSmemBudget - kOutBufs * kOutBytes) / kStageBytes;
   static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
   static constexpr int kAcc = (2 * BN + (SPARSE ? 4 * kStages : 0) <= (int)kTmemCols) ? 2 : 1;
   static constexpr int kMetaCol = kAcc * BN;              // first TMEM column of the metadata slots
-  static constexpr int kSmemBytes = kStages * kStageBytes + 2048;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kOutBufs * kOutBytes + 2048;
   static_assert(kStages >= 2, "pipeline needs at least two stages");
 };
 
@@ -74,8 +76,8 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool sparse) {
 // [32*k2, 32*k2+32) of the stage the tensor core reads one 32-bit TMEM column: lane
 // (row%8) + 8*half + 16*(row/16) holds in its low 16 bits the four position nibbles of channels
 // 32*k2 + 16*half + [0,16) of the row with bit 3 clear and in its high 16 bits those of row + 8.
-__device__ __forceinline__ void rearrange_metadata(const uint8_t* raw_stage, uint8_t* hw_stage, int row,
-                                                   int rows_used) {
+__device__ __forceinline__ void rearrange_metadata_row(const uint8_t* raw_stage, uint8_t* hw_stage, int row,
+                                                       int rows_used) {
   const uint4 raw = *(const uint4*)(raw_stage + row * 16);
   const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
   uint16_t* hw = (uint16_t*)hw_stage;
@@ -90,27 +92,50 @@ __device__ __forceinline__ void rearrange_metadata(const uint8_t* raw_stage, uin
   }
 }
 
-// This warp's 32 accumulator rows x BN columns: TMEM -> registers -> bf16 -> global.
-template <int BN>
-__device__ __forceinline__ void store_accumulator(uint32_t taddr, uint16_t* out, bool valid) {
+// One warp rearranges a whole stage (lane l takes rows l, l+32, l+64, l+96); the four
+// rearranger warps work on four different stages at once, so the per-stage latency of
+// wait -> shuffle -> proxy fence -> arrive is overlapped four ways.
+__device__ __forceinline__ void rearrange_metadata_stage(const uint8_t* raw_stage, uint8_t* hw_stage, int lane,
+                                                         int rows_used) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) rearrange_metadata_row(raw_stage, hw_stage, lane + 32 * i, rows_used);
+}
+
+// The four epilogue warps move one 128-row x BN accumulator to global memory in 64-column
+// slabs: TMEM -> registers -> bf16 -> a 128-byte-swizzled staging tile in shared memory -> one
+// TMA store of the whole pixel patch (full-line writes; rows and pixels outside the tensor are
+// clipped by the TMA unit). With NBUF = 2 the store of one slab overlaps the packing of the next.
+// `chunk` counts slabs over the kernel's lifetime and picks the staging buffer.
+template <int BN, int NBUF>
+__device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* staging, const CUtensorMap* tmD,
+                                                  int n0, int w0, int h0, int b0, bool tile_in_range, int row,
+                                                  bool issuer, uint32_t& chunk) {
 #pragma unroll 1
-  for (int c0 = 0; c0 < BN; c0 += 32) {
-    uint32_t v[32];
-    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
-    ptx::tmem_ld_wait();
-    if (valid) {
-      uint4* dst = (uint4*)(out + c0);
+  for (int c0 = 0; c0 < BN; c0 += 64, ++chunk) {
+    uint32_t packed[32];
 #pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        uint32_t w2[4];
+    for (int half = 0; half < 2; ++half) {
+      uint32_t v[32];
+      ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32 * half), v);
+      ptx::tmem_ld_wait();
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * g + 2 * e]),
-                                                          __uint_as_float(v[8 * g + 2 * e + 1]));
-          w2[e] = *(const uint32_t*)&h2;
-        }
-        dst[g] = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+      for (int e = 0; e < 16; ++e) {
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+        packed[16 * half + e] = *(const uint32_t*)&h2;
       }
+    }
+    uint8_t* buf = staging + (chunk % NBUF) * kOutBytes;
+    if (issuer) ptx::bulk_wait_group_read<NBUF - 1>();  // the store that last used this buffer has read it
+    ptx::named_bar_sync(1, 128);
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+      *(uint4*)(buf + row * 128 + ((c ^ (row & 7)) << 4)) =
+          make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+    ptx::fence_proxy_async_smem();
+    ptx::named_bar_sync(1, 128);
+    if (issuer && tile_in_range) {
+      ptx::tma_store_4d(tmD, buf, n0 + c0, w0, h0, b0);
+      ptx::bulk_commit_group();
     }
   }
 }
@@ -118,7 +143,8 @@ __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint16_t* out,
 template <bool SPARSE, int BN>
 __global__ void __launch_bounds__(kThreadsGemm, 1)
 dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmE,
-             const __grid_constant__ CUtensorMap tmB, const DgradParams p) {
+             const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
+             const DgradParams p) {
   using C = Cfg<SPARSE, BN>;
   constexpr int STAGES = C::kStages;
   constexpr int NACC = C::kAcc;
@@ -130,7 +156,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   uint8_t* sB = sA + STAGES * kABytes;
   uint8_t* sEraw = sB + STAGES * C::kBBytes;
   uint8_t* sEhw = sEraw + (SPARSE ? STAGES * kEBytes : 0);
-  uint64_t* bars = (uint64_t*)(sEhw + (SPARSE ? STAGES * kEBytes : 0));
+  uint8_t* sOut = sEhw + (SPARSE ? STAGES * kEBytes : 0);
+  uint64_t* bars = (uint64_t*)(sOut + C::kOutBufs * kOutBytes);
   uint64_t* full = bars;
   uint64_t* empty = full + STAGES;
   uint64_t* meta_ready = empty + STAGES;
@@ -146,7 +173,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     for (int s = 0; s < STAGES; ++s) {
       ptx::mbar_init(&full[s], 1);
       ptx::mbar_init(&empty[s], 1);
-      ptx::mbar_init(&meta_ready[s], 4);
+      ptx::mbar_init(&meta_ready[s], 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&acc_full[a], 1);
@@ -157,6 +184,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   if (warp == 0 && lane == 0) {
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
+    ptx::prefetch_tensormap(&tmD);
     if (SPARSE) ptx::prefetch_tensormap(&tmE);
   }
   if (warp == 1) {
@@ -247,14 +275,14 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   } else if (warp < 6) {
     // ------------------------------------------------- metadata rearranger
     if (SPARSE) {
-      const int row = threadIdx.x - 64;  // 0..127: A-tile row = TMEM lane of the accumulator
       uint32_t it = 0;
       for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
         for (int kb = 0; kb < k_iters; ++kb, ++it) {
+          if ((int)(it & 3u) != warp - 2) continue;  // this warp's turn: every fourth stage use
           const int st = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           ptx::mbar_wait(&full[st], ph, err, 0x500u + st);
-          rearrange_metadata(sEraw + st * kEBytes, sEhw + st * kEBytes, row, rows_used);
+          rearrange_metadata_stage(sEraw + st * kEBytes, sEhw + st * kEBytes, lane, rows_used);
           ptx::fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&meta_ready[st]);
@@ -265,28 +293,25 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     // ------------------------------------------------------------ epilogue
     const int q = warp & 3;  // a warp may only touch TMEM lanes [32*(warp%4), +32)
     const int row = q * 32 + lane;
-    const int tw = row % p.TW;
-    const int th = (row / p.TW) % p.TH;
-    const int tb = row / (p.TW * p.TH);
-    uint32_t lt = 0;
+    const bool issuer = (threadIdx.x == 192);
+    uint32_t lt = 0, chunk = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++lt) {
       int t = tile;
       const int nt = t % p.tiles_n; t /= p.tiles_n;
       const int wt = t % p.tiles_w; t /= p.tiles_w;
       const int ht = t % p.tiles_h; t /= p.tiles_h;
       const int bt = t;
-      const int w = wt * p.TW + tw, h = ht * p.TH + th, b = bt * p.TB + tb;
-      const bool valid = row < rows_used && w < p.W && h < p.H && b < p.B;
       const int acc = lt % NACC;
       const uint32_t aph = (lt / NACC) & 1u;
       ptx::mbar_wait(&acc_full[acc], aph, err, 0x600u + acc);
       ptx::tc_fence_after_sync();
-      uint16_t* out = p.dD + (((int64_t)b * p.H + h) * p.W + w) * (int64_t)p.Cin + (int64_t)nt * BN;
-      store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), out, valid);
+      store_accumulator<BN, C::kOutBufs>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), sOut, &tmD,
+                                         nt * BN, wt * p.TW, ht * p.TH, bt * p.TB, true, row, issuer, chunk);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
     }
+    if (issuer) ptx::bulk_wait_group_all();  // dD is written before the CTA leaves
   }
 
   ptx::tc_fence_before_sync();
@@ -314,11 +339,12 @@ struct PairCfg {
   static constexpr int kBBytes = kKB * kBCols * 2;
   static constexpr int kStageBytes = kABytes + kBBytes + (SPARSE ? 2 * kEBytes : 0);
   static constexpr int kSmemBudget = 232448 - 2048;
-  static constexpr int kStagesFit = kSmemBudget / kStageBytes;
+  static constexpr int kOutBufs = ((kSmemBudget - 2 * kOutBytes) / kStageBytes >= 4) ? 2 : 1;
+  static constexpr int kStagesFit = (kSmemBudget - kOutBufs * kOutBytes) / kStageBytes;
   static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
   static constexpr int kAcc = (2 * BN + (SPARSE ? 4 * kStages : 0) <= (int)kTmemCols) ? 2 : 1;
   static constexpr int kMetaCol = kAcc * BN;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 2048;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kOutBufs * kOutBytes + 2048;
   static_assert(kBCols % 64 == 0, "each CTA stages whole 64-column swizzle blocks of W");
   static_assert(kStages >= 2, "pipeline needs at least two stages");
 };
@@ -331,7 +357,8 @@ __host__ __device__ constexpr uint32_t make_idesc_pair(int n, bool sparse) {
 template <bool SPARSE, int BN>
 __global__ void __launch_bounds__(kThreadsGemm, 1)
 dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmE,
-                  const __grid_constant__ CUtensorMap tmB, const DgradParams p) {
+                  const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
+                  const DgradParams p) {
   using C = PairCfg<SPARSE, BN>;
   constexpr int STAGES = C::kStages;
   constexpr int NACC = C::kAcc;
@@ -342,7 +369,8 @@ dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   uint8_t* sB = sA + STAGES * kABytes;
   uint8_t* sEraw = sB + STAGES * C::kBBytes;
   uint8_t* sEhw = sEraw + (SPARSE ? STAGES * kEBytes : 0);
-  uint64_t* bars = (uint64_t*)(sEhw + (SPARSE ? STAGES * kEBytes : 0));
+  uint8_t* sOut = sEhw + (SPARSE ? STAGES * kEBytes : 0);
+  uint64_t* bars = (uint64_t*)(sOut + C::kOutBufs * kOutBytes);
   uint64_t* full = bars;
   uint64_t* empty = full + STAGES;
   uint64_t* meta_full = empty + STAGES;
@@ -361,7 +389,7 @@ dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ptx::mbar_init(&full[s], 1);
       ptx::mbar_init(&empty[s], 1);
       ptx::mbar_init(&meta_full[s], 1);
-      ptx::mbar_init(&meta_ready[s], 8);
+      ptx::mbar_init(&meta_ready[s], 2);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&acc_full[a], 1);
@@ -372,6 +400,7 @@ dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   if (warp == 0 && lane == 0) {
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
+    ptx::prefetch_tensormap(&tmD);
     if (SPARSE) ptx::prefetch_tensormap(&tmE);
   }
   if (warp == 1) {
@@ -467,14 +496,14 @@ dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   } else if (warp < 6) {
     // ------------------------------------------------- metadata rearranger
     if (SPARSE) {
-      const int row = threadIdx.x - 64;
       uint32_t it = 0;
       for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride) {
         for (int kb = 0; kb < k_iters; ++kb, ++it) {
+          if ((int)(it & 3u) != warp - 2) continue;
           const int st = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           ptx::mbar_wait(&meta_full[st], ph, err, 0x1500u + st);
-          rearrange_metadata(sEraw + st * kEBytes, sEhw + st * kEBytes, row, rows_used);
+          rearrange_metadata_stage(sEraw + st * kEBytes, sEhw + st * kEBytes, lane, rows_used);
           ptx::fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive_cluster(&meta_ready[st], 0);
@@ -485,28 +514,27 @@ dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // ------------------------------------------------------------ epilogue
     const int q = warp & 3;
     const int row = q * 32 + lane;
-    const int tw = row % p.TW;
-    const int th = (row / p.TW) % p.TH;
-    const int tb = row / (p.TW * p.TH);
-    uint32_t lt = 0;
+    const bool issuer = (threadIdx.x == 192);
+    uint32_t lt = 0, chunk = 0;
     for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride, ++lt) {
       const int nt = pt % p.tiles_n;
-      int t = 2 * (pt / p.tiles_n) + (int)rank;
+      const int mt = 2 * (pt / p.tiles_n) + (int)rank;
+      int t = mt;
       const int wt = t % p.tiles_w; t /= p.tiles_w;
       const int ht = t % p.tiles_h; t /= p.tiles_h;
       const int bt = t;
-      const int w = wt * p.TW + tw, h = ht * p.TH + th, b = bt * p.TB + tb;
-      const bool valid = row < rows_used && w < p.W && h < p.H && b < p.B;
       const int acc = lt % NACC;
       const uint32_t aph = (lt / NACC) & 1u;
       ptx::mbar_wait(&acc_full[acc], aph, err, 0x1600u + acc);
       ptx::tc_fence_after_sync();
-      uint16_t* out = p.dD + (((int64_t)b * p.H + h) * p.W + w) * (int64_t)p.Cin + (int64_t)nt * BN;
-      store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), out, valid);
+      store_accumulator<BN, C::kOutBufs>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), sOut, &tmD,
+                                         nt * BN, wt * p.TW, ht * p.TH, bt * p.TB, mt < p.m_tiles, row, issuer,
+                                         chunk);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
     }
+    if (issuer) ptx::bulk_wait_group_all();
   }
 
   ptx::tc_fence_before_sync();
@@ -585,7 +613,7 @@ int sm_count() {
 
 template <bool SPARSE, int BN>
 sdgp_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmE, const CUtensorMap& tmB,
-                       const DgradParams& p, cudaStream_t stream) {
+                       const CUtensorMap& tmD, const DgradParams& p, cudaStream_t stream) {
   using C = Cfg<SPARSE, BN>;
   static bool configured = false;
   auto kernel = dgrad_kernel<SPARSE, BN>;
@@ -595,13 +623,13 @@ sdgp_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmE, const CUt
     configured = true;
   }
   const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
-  kernel<<<grid, kThreadsGemm, C::kSmemBytes, stream>>>(tmA, tmE, tmB, p);
+  kernel<<<grid, kThreadsGemm, C::kSmemBytes, stream>>>(tmA, tmE, tmB, tmD, p);
   return cudaGetLastError() == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
 template <bool SPARSE, int BN>
 sdgp_status launch_pair_cfg(const CUtensorMap& tmA, const CUtensorMap& tmE, const CUtensorMap& tmB,
-                            const DgradParams& p, cudaStream_t stream) {
+                            const CUtensorMap& tmD, const DgradParams& p, cudaStream_t stream) {
   using C = PairCfg<SPARSE, BN>;
   static bool configured = false;
   auto kernel = dgrad_pair_kernel<SPARSE, BN>;
@@ -624,7 +652,7 @@ sdgp_status launch_pair_cfg(const CUtensorMap& tmA, const CUtensorMap& tmE, cons
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, tmA, tmE, tmB, p) == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
+  return cudaLaunchKernelEx(&cfg, kernel, tmA, tmE, tmB, tmD, p) == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
 }  // namespace
@@ -688,14 +716,24 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
       return SDGP_ERR_CUDA;
   }
 
+  CUtensorMap tmD;
+  {
+    const uint64_t dims[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)B};
+    const uint64_t strides[3] = {(uint64_t)Cin * 2, (uint64_t)Cin * 2 * W, (uint64_t)Cin * 2 * W * H};
+    const uint32_t box[4] = {64, (uint32_t)p.TW, (uint32_t)p.TH, (uint32_t)p.TB};
+    if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, dD, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+      return SDGP_ERR_CUDA;
+  }
+
   if (pair) {
     if (sparse)
-      return BN == 256 ? launch_pair_cfg<true, 256>(tmA, tmE, tmB, p, stream)
-                       : launch_pair_cfg<true, 128>(tmA, tmE, tmB, p, stream);
-    return BN == 256 ? launch_pair_cfg<false, 256>(tmA, tmE, tmB, p, stream)
-                     : launch_pair_cfg<false, 128>(tmA, tmE, tmB, p, stream);
+      return BN == 256 ? launch_pair_cfg<true, 256>(tmA, tmE, tmB, tmD, p, stream)
+                       : launch_pair_cfg<true, 128>(tmA, tmE, tmB, tmD, p, stream);
+    return BN == 256 ? launch_pair_cfg<false, 256>(tmA, tmE, tmB, tmD, p, stream)
+                     : launch_pair_cfg<false, 128>(tmA, tmE, tmB, tmD, p, stream);
   }
-  return sparse ? launch_cfg<true, 64>(tmA, tmE, tmB, p, stream) : launch_cfg<false, 64>(tmA, tmE, tmB, p, stream);
+  return sparse ? launch_cfg<true, 64>(tmA, tmE, tmB, tmD, p, stream)
+                : launch_cfg<false, 64>(tmA, tmE, tmB, tmD, p, stream);
 }
 
 sdgp_status read_device_error() {
