@@ -46,6 +46,7 @@ struct DgradParams {
   int k_blocks_per_tap; // ceil(Cout / channels per stage)
   int m_tiles;          // tiles_w * tiles_h * tiles_b
   int pair_tiles;       // CTA-pair kernel: ceil(m_tiles / 2) * tiles_n
+  int meta_merged;      // metadata box spans whole pixel rows (8*TW uint16 per TMA request)
   uint16_t* dD;
 };
 
@@ -221,7 +222,10 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             ptx::mbar_wait(&empty[st], ph ^ 1u, err, 0x100u + st);
             ptx::mbar_arrive_expect_tx(&full[st], tx_bytes);
             ptx::tma_load_4d(sA + st * kABytes, &tmA, &full[st], cb * 64, q0, p0, b0);
-            if (SPARSE) ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &full[st], cb * 8, q0, p0, b0);
+            if (SPARSE) {
+              if (p.meta_merged) ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &full[st], 8 * q0, p0, b0, 0);
+              else ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &full[st], cb * 8, q0, p0, b0);
+            }
 #pragma unroll
             for (int j = 0; j < BN / 64; ++j)
               ptx::tma_load_2d(sB + st * C::kBBytes + j * (C::kKB * 128), &tmB, &full[st],
@@ -441,7 +445,8 @@ dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (rank == 0) ptx::mbar_arrive_expect_tx(&full[st], pair_tx);
             if (SPARSE) {
               ptx::mbar_arrive_expect_tx(&meta_full[st], (uint32_t)(rows_used * 16));
-              ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &meta_full[st], cb * 8, q0, p0, b0);
+              if (p.meta_merged) ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &meta_full[st], 8 * q0, p0, b0, 0);
+              else ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &meta_full[st], cb * 8, q0, p0, b0);
             }
             ptx::tma_load_4d_pair(sA + st * kABytes, &tmA, &full[st], cb * 64, q0, p0, b0);
 #pragma unroll
@@ -698,7 +703,17 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
     if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
   }
-  if (sparse) {
+  p.meta_merged = 0;
+  if (sparse && Cout == 128 && p.TW <= 32) {
+    // One pixel's metadata is a single 16-byte run and pixels of an image row are contiguous:
+    // fetch whole rows of the patch per TMA request instead of one request per pixel.
+    p.meta_merged = 1;
+    const uint64_t dims[4] = {8ull * Q, (uint64_t)P, (uint64_t)B, 1};
+    const uint64_t strides[3] = {16ull * Q, 16ull * Q * P, 16ull * Q * P * B};
+    const uint32_t box[4] = {8u * (uint32_t)p.TW, (uint32_t)p.TH, (uint32_t)p.TB, 1};
+    if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
+      return SDGP_ERR_CUDA;
+  } else if (sparse) {
     const uint64_t CE = (uint64_t)Cout / 16;
     const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)P, (uint64_t)B};
     const uint64_t strides[3] = {CE * 2, CE * 2 * Q, CE * 2 * Q * P};
