@@ -1,22 +1,38 @@
 // Data-gradient contraction dD = dOp . W on the sm_100a tensor cores (Section 2.1, Fig. 2/3).
 //
 // One persistent, warp-specialised kernel serves the fully connected layer and the stride-1
-// convolution (an implicit GEMM whose K axis runs tap-major, output-channel-minor, so a
-// 4-element pruning chunk never straddles two filter taps), with A either dense dL/dO
-// (tcgen05.mma) or 2:4-compressed dL/dO plus position metadata (tcgen05.mma.sp):
+// convolution (an implicit GEMM whose K axis covers filter taps x output channels; a 4-element
+// pruning chunk never straddles two taps), with A either dense dL/dO (tcgen05.mma) or
+// 2:4-compressed dL/dO plus position metadata (tcgen05.mma.sp).
 //
-//   warp 0      TMA producer: per K-block one 4-D box of A (a TW x TH x TB patch of pixels,
-//               shifted by the filter tap; out-of-image pixels arrive as zeros), the matching
-//               box of metadata, and BN/64 boxes of W.
-//   warp 1      MMA issuer: copies the stage's metadata into TMEM (tcgen05.cp), issues four
-//               MMAs per stage into a TMEM accumulator, commits to the stage's "empty" barrier.
-//   warps 2-5   (sparse only) rearrange the stages' row-major metadata into the lane/column
-//               order the tensor core reads from TMEM, one warp per stage, four stages at once.
+// CTA pairs (cta_group::2): the two CTAs of a cluster own two neighbouring 128-pixel patches
+// and one BN-wide block of input channels. Each CTA stages its own A patch (+ metadata) and
+// HALF of the W columns; one thread of the pair's first CTA issues 256-row MMAs that read
+// both halves. What limits this kernel is the bytes an SM can pull in from L2 (about 64 B per
+// clock), so everything is arranged to reuse what is already in shared memory:
+//   * W column halves: half the W bytes per CTA and half the shared-memory reads of B;
+//   * filter-row reuse: for an R x S filter one A "image" of TH + R - 1 pixel rows serves all R
+//     vertical taps - a tap is just a row offset (a multiple of 8 rows, i.e. of the 1024-byte
+//     swizzle period) in the A descriptor - so A is fetched S times instead of R*S times;
+//   * resident W: when the layer's whole W slice fits next to two A stages it is loaded once
+//     per CTA and never streamed again.
+//
+// Warp roles
+//   warp 0      TMA producer (both CTAs): per stage one 4-D box of A (pixels outside the image
+//               arrive as zeros), the matching box of metadata, and the W boxes of its half.
+//   warp 1      MMA issuer (first CTA only): tcgen05.cp of the stage's metadata into TMEM,
+//               four MMAs per (tap, channel block), tcgen05.commit to the stage's "empty" barrier.
+//   warps 2-5   (sparse only) rearrange metadata from the row-major order TMA delivers into
+//               the lane/column order the tensor core reads from TMEM (one thread per A-tile row).
 //   warps 6-9   epilogue: TMEM -> registers -> bf16 -> swizzled staging tile -> TMA store,
 //               overlapped with the next tile's main loop through a second accumulator.
 //
-// Every mbarrier wait is bounded; a wait that runs out records a code in g_device_error and
-// the kernel still runs to completion and frees its TMEM.
+// Barriers: full / meta_ready / acc_empty / w_full are waited on by the first CTA only and
+// collect arrivals from both; empty / acc_full exist in both CTAs and are signalled together
+// by a multicast tcgen05.commit; meta_full is local (each CTA's own metadata box).
+// Every wait is bounded: a wait that runs out records a code in g_device_error, the role
+// stops issuing work, every other wait then gives up at once, and the kernel frees its TMEM
+// and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -29,59 +45,67 @@ __device__ unsigned int g_device_error = 0;
 
 namespace {
 
-constexpr int kBM = 128;           // output pixels (rows) per tile = TMEM lanes
-constexpr int kThreadsGemm = 320;  // 10 warps
-constexpr int kABytes = kBM * 128; // one A stage: 128 rows x 128 B (64 bf16, dense or compressed)
-constexpr int kEBytes = kBM * 16;  // one metadata stage: 128 rows x 8 uint16
+constexpr int kBM = 128;             // output pixels (rows) per CTA tile = TMEM lanes
+constexpr int kThreadsGemm = 320;    // 10 warps
+constexpr int kEHwBytes = kBM * 16;  // rearranged metadata of one (tap, channel block): 128 lanes x 16 B
+constexpr int kOutBytes = kBM * 128; // epilogue staging slab: 128 rows x 64 bf16 columns
 constexpr uint32_t kTmemCols = 512;
-constexpr int kOutBytes = kBM * 128;  // epilogue staging: 128 rows x 64 bf16 columns
+constexpr int kMaxImgRows = 192;     // pixel rows of one A stage (filter-row reuse: TW * (TH + R - 1))
+constexpr int kSmemLimit = 232448;   // opt-in dynamic shared memory per CTA
+constexpr int kSmemSlack = 1536;     // 1024-byte alignment of the carve + barrier block
+constexpr int kMaxStages = 8;
 
 struct DgradParams {
-  int B, H, W;          // dD pixel grid (fully connected: B = H = 1, W = rows)
+  int B, H, W;            // dD pixel grid (fully connected: B = H = 1, W = rows)
   int Cin, Cout;
   int R, S, pad;
-  int TW, TH, TB;       // pixel patch of one tile, TW * TH * TB <= 128
+  int TW, TH, TB;         // pixel patch of one CTA tile, TW * TH * TB <= 128
   int tiles_w, tiles_h, tiles_b, tiles_n;
-  int total_tiles;
-  int k_blocks_per_tap; // ceil(Cout / channels per stage)
-  int m_tiles;          // tiles_w * tiles_h * tiles_b
-  int pair_tiles;       // CTA-pair kernel: ceil(m_tiles / 2) * tiles_n
-  int meta_merged;      // metadata box spans whole pixel rows (8*TW uint16 per TMA request)
-  uint16_t* dD;
+  int m_tiles;            // tiles_w * tiles_h * tiles_b
+  int pair_tiles;         // ceil(m_tiles / 2) * tiles_n
+  int k_blocks;           // channel blocks per tap: ceil(Cout / channels per stage)
+  int rr;                 // vertical taps served by one A stage: 1, or R (filter-row reuse)
+  int img_rows;           // pixel rows of one A stage: TW * (TH + rr - 1) * TB
+  int stages;             // shared-memory pipeline depth
+  int nacc;               // TMEM accumulators (2 = epilogue overlaps the next tile)
+  int meta_col;           // first TMEM column of the metadata slots
+  int w_resident;         // whole W half-slice kept in shared memory
+  int out_bufs;           // epilogue staging slabs (1 or 2)
+  // shared-memory carve (byte offsets from the 1024-aligned base) and per-stage sizes
+  int a_bytes, b_bytes, eraw_bytes, ehw_bytes;
+  int off_b, off_eraw, off_ehw, off_w, off_out, off_bar;
+  int smem_bytes;
 };
 
 template <bool SPARSE, int BN>
 struct Cfg {
-  static constexpr int kKB = SPARSE ? 128 : 64;           // W rows (output channels) per stage
-  static constexpr int kBBytes = kKB * BN * 2;
-  static constexpr int kStageBytes = kABytes + kBBytes + (SPARSE ? 2 * kEBytes : 0);
-  static constexpr int kSmemBudget = 232448 - 2048;       // max dynamic smem minus barriers/alignment slack
-  static constexpr int kOutBufs = ((kSmemBudget - 2 * kOutBytes) / kStageBytes >= 4) ? 2 : 1;
-  static constexpr int kStagesFit = (kSmemBudget - kOutBufs * kOutBytes) / kStageBytes;
-  static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
-  static constexpr int kAcc = (2 * BN + (SPARSE ? 4 * kStages : 0) <= (int)kTmemCols) ? 2 : 1;
-  static constexpr int kMetaCol = kAcc * BN;              // first TMEM column of the metadata slots
-  static constexpr int kSmemBytes = kStages * kStageBytes + kOutBufs * kOutBytes + 2048;
-  static_assert(kStages >= 2, "pipeline needs at least two stages");
+  static constexpr int kKB = SPARSE ? 128 : 64;               // W rows (output channels) per MMA group
+  static constexpr int kBCols = BN / 2;                       // W columns staged by one CTA
+  static constexpr int kBoxCols = kBCols < 64 ? kBCols : 64;  // columns of one W box
+  static constexpr int kBoxes = kBCols / kBoxCols;
+  static constexpr int kRowB = kBoxCols * 2;                  // bytes of one W row in shared memory
+  static constexpr uint32_t kBSwizzle = (kRowB == 128) ? 2u : 4u;  // descriptor code: 128-/64-byte swizzle
+  static constexpr int kBoxBytes = kKB * kRowB;
+  static constexpr int kTapBBytes = kBoxBytes * kBoxes;       // one CTA's W bytes of one (tap, channel block)
+  static_assert(kBCols == 32 || kBCols % 64 == 0, "W half must be 32 columns or whole 64-column blocks");
 };
 
-// Instruction descriptor: fp32 accumulate, bf16 A and B, A K-major, B MN-major, M = 128.
+// Instruction descriptor: fp32 accumulate, bf16 A and B, A K-major, B MN-major, M = 256 (pair).
 __host__ __device__ constexpr uint32_t make_idesc(int n, bool sparse) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
-         ((uint32_t)(kBM >> 4) << 24) | (sparse ? (1u << 2) : 0u);
+         ((uint32_t)(256 >> 4) << 24) | (sparse ? (1u << 2) : 0u);
 }
 
-
-// One row of a stage's metadata: from the row-major order TMA delivers (8 uint16 per pixel,
-// one per 16 channels) to the order tcgen05.cp moves into TMEM. For the MMA covering channels
-// [32*k2, 32*k2+32) of the stage the tensor core reads one 32-bit TMEM column: lane
+// One row of metadata: from the row-major order TMA delivers (8 uint16 per pixel, one per 16
+// channels) to the order tcgen05.cp moves into TMEM. For the MMA covering channels
+// [32*k2, 32*k2+32) of the block the tensor core reads one 32-bit TMEM column: lane
 // (row%8) + 8*half + 16*(row/16) holds in its low 16 bits the four position nibbles of channels
 // 32*k2 + 16*half + [0,16) of the row with bit 3 clear and in its high 16 bits those of row + 8.
-__device__ __forceinline__ void rearrange_metadata_row(const uint8_t* raw_stage, uint8_t* hw_stage, int row,
+__device__ __forceinline__ void rearrange_metadata_row(const uint8_t* raw_rows, uint8_t* hw_tile, int row,
                                                        int rows_used) {
-  const uint4 raw = *(const uint4*)(raw_stage + row * 16);
+  const uint4 raw = *(const uint4*)(raw_rows + row * 16);
   const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
-  uint16_t* hw = (uint16_t*)hw_stage;
+  uint16_t* hw = (uint16_t*)hw_tile;
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
     uint32_t v = (u & 1) ? (w4[u >> 1] >> 16) : (w4[u >> 1] & 0xFFFFu);
@@ -93,40 +117,34 @@ __device__ __forceinline__ void rearrange_metadata_row(const uint8_t* raw_stage,
   }
 }
 
-// One warp rearranges a whole stage (lane l takes rows l, l+32, l+64, l+96); the four
-// rearranger warps work on four different stages at once, so the per-stage latency of
-// wait -> shuffle -> proxy fence -> arrive is overlapped four ways.
-__device__ __forceinline__ void rearrange_metadata_stage(const uint8_t* raw_stage, uint8_t* hw_stage, int lane,
-                                                         int rows_used) {
-#pragma unroll
-  for (int i = 0; i < 4; ++i) rearrange_metadata_row(raw_stage, hw_stage, lane + 32 * i, rows_used);
-}
-
 // The four epilogue warps move one 128-row x BN accumulator to global memory in 64-column
-// slabs: TMEM -> registers -> bf16 -> a 128-byte-swizzled staging tile in shared memory -> one
-// TMA store of the whole pixel patch (full-line writes; rows and pixels outside the tensor are
-// clipped by the TMA unit). With NBUF = 2 the store of one slab overlaps the packing of the next.
-// `chunk` counts slabs over the kernel's lifetime and picks the staging buffer.
-template <int BN, int NBUF>
-__device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* staging, const CUtensorMap* tmD,
-                                                  int n0, int w0, int h0, int b0, bool tile_in_range, int row,
-                                                  bool issuer, uint32_t& chunk) {
+// slabs: TMEM -> registers -> bf16 -> a 128-byte-swizzled staging tile -> one TMA store of the
+// whole pixel patch (full-line writes; pixels outside the tensor are clipped by the TMA unit).
+// With two staging slabs the store of one overlaps the packing of the next. `chunk` counts
+// slabs over the kernel's lifetime and picks the slab.
+template <int BN>
+__device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* staging, int out_bufs,
+                                                  const CUtensorMap* tmD, int n0, int w0, int h0, int b0,
+                                                  bool tile_in_range, int row, bool issuer, uint32_t& chunk) {
 #pragma unroll 1
   for (int c0 = 0; c0 < BN; c0 += 64, ++chunk) {
     uint32_t packed[32];
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
+    for (int part = 0; part < 2; ++part) {
       uint32_t v[32];
-      ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32 * half), v);
+      ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32 * part), v);
       ptx::tmem_ld_wait();
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
         const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
-        packed[16 * half + e] = *(const uint32_t*)&h2;
+        packed[16 * part + e] = *(const uint32_t*)&h2;
       }
     }
-    uint8_t* buf = staging + (chunk % NBUF) * kOutBytes;
-    if (issuer) ptx::bulk_wait_group_read<NBUF - 1>();  // the store that last used this buffer has read it
+    uint8_t* buf = staging + (out_bufs == 2 ? (chunk & 1u) : 0u) * kOutBytes;
+    if (issuer) {  // the store that last used this slab has finished reading it
+      if (out_bufs == 2) ptx::bulk_wait_group_read<1>();
+      else ptx::bulk_wait_group_read<0>();
+    }
     ptx::named_bar_sync(1, 128);
 #pragma unroll
     for (int c = 0; c < 8; ++c)
@@ -147,258 +165,44 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
              const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
              const DgradParams p) {
   using C = Cfg<SPARSE, BN>;
-  constexpr int STAGES = C::kStages;
-  constexpr int NACC = C::kAcc;
 
   extern __shared__ uint8_t smem_raw[];
-  // 1024-byte alignment: required by the 128-byte swizzle of the A and B stages
+  // 1024-byte alignment: required by the 128-byte swizzle of the A, B and staging tiles
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;
-  uint8_t* sB = sA + STAGES * kABytes;
-  uint8_t* sEraw = sB + STAGES * C::kBBytes;
-  uint8_t* sEhw = sEraw + (SPARSE ? STAGES * kEBytes : 0);
-  uint8_t* sOut = sEhw + (SPARSE ? STAGES * kEBytes : 0);
-  uint64_t* bars = (uint64_t*)(sOut + C::kOutBufs * kOutBytes);
-  uint64_t* full = bars;
-  uint64_t* empty = full + STAGES;
-  uint64_t* meta_ready = empty + STAGES;
-  uint64_t* acc_full = meta_ready + STAGES;
+  uint8_t* sB = smem + p.off_b;
+  uint8_t* sEraw = smem + p.off_eraw;
+  uint8_t* sEhw = smem + p.off_ehw;
+  uint8_t* sW = smem + p.off_w;
+  uint8_t* sOut = smem + p.off_out;
+  uint64_t* full = (uint64_t*)(smem + p.off_bar);
+  uint64_t* empty = full + kMaxStages;
+  uint64_t* meta_full = empty + kMaxStages;
+  uint64_t* meta_ready = meta_full + kMaxStages;
+  uint64_t* acc_full = meta_ready + kMaxStages;
   uint64_t* acc_empty = acc_full + 2;
-  uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
-
-  const int warp = threadIdx.x >> 5;
-  const int lane = threadIdx.x & 31;
-  unsigned int* err = &g_device_error;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      ptx::mbar_init(&full[s], 1);
-      ptx::mbar_init(&empty[s], 1);
-      ptx::mbar_init(&meta_ready[s], 1);
-    }
-    for (int a = 0; a < 2; ++a) {
-      ptx::mbar_init(&acc_full[a], 1);
-      ptx::mbar_init(&acc_empty[a], 4);
-    }
-    ptx::fence_mbar_init();
-  }
-  if (warp == 0 && lane == 0) {
-    ptx::prefetch_tensormap(&tmA);
-    ptx::prefetch_tensormap(&tmB);
-    ptx::prefetch_tensormap(&tmD);
-    if (SPARSE) ptx::prefetch_tensormap(&tmE);
-  }
-  if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, kTmemCols);
-    ptx::tmem_relinquish();
-  }
-  ptx::tc_fence_before_sync();
-  __syncthreads();
-  ptx::tc_fence_after_sync();
-  const uint32_t tmem_base = *tmem_slot;
-
-  const int rows_used = p.TW * p.TH * p.TB;
-  const int taps = p.R * p.S;
-  const int k_iters = taps * p.k_blocks_per_tap;
-  const uint32_t tx_bytes = (uint32_t)(rows_used * 128 + C::kBBytes + (SPARSE ? rows_used * 16 : 0));
-
-  if (warp == 0) {
-    // ------------------------------------------------------------ producer
-    if (ptx::elect_one()) {
-      uint32_t it = 0;
-      for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
-        int t = tile;
-        const int nt = t % p.tiles_n; t /= p.tiles_n;
-        const int wt = t % p.tiles_w; t /= p.tiles_w;
-        const int ht = t % p.tiles_h; t /= p.tiles_h;
-        const int bt = t;
-        const int n0 = nt * BN, w0 = wt * p.TW, h0 = ht * p.TH, b0 = bt * p.TB;
-        for (int tap = 0; tap < taps; ++tap) {
-          const int r = tap / p.S, s = tap - r * p.S;
-          const int q0 = w0 + p.pad - s, p0 = h0 + p.pad - r;  // dO pixel of the patch's corner
-          for (int cb = 0; cb < p.k_blocks_per_tap; ++cb, ++it) {
-            const int st = it % STAGES;
-            const uint32_t ph = (it / STAGES) & 1u;
-            ptx::mbar_wait(&empty[st], ph ^ 1u, err, 0x100u + st);
-            ptx::mbar_arrive_expect_tx(&full[st], tx_bytes);
-            ptx::tma_load_4d(sA + st * kABytes, &tmA, &full[st], cb * 64, q0, p0, b0);
-            if (SPARSE) {
-              if (p.meta_merged) ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &full[st], 8 * q0, p0, b0, 0);
-              else ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &full[st], cb * 8, q0, p0, b0);
-            }
-#pragma unroll
-            for (int j = 0; j < BN / 64; ++j)
-              ptx::tma_load_2d(sB + st * C::kBBytes + j * (C::kKB * 128), &tmB, &full[st],
-                               tap * p.Cin + n0 + 64 * j, cb * C::kKB);
-          }
-        }
-      }
-    }
-  } else if (warp == 1) {
-    // ---------------------------------------------------------- MMA issuer
-    if (ptx::elect_one()) {
-      constexpr uint32_t idesc = make_idesc(BN, SPARSE);
-      uint32_t it = 0, lt = 0;
-      for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++lt) {
-        const int acc = lt % NACC;
-        const uint32_t aph = (lt / NACC) & 1u;
-        ptx::mbar_wait(&acc_empty[acc], aph ^ 1u, err, 0x200u + acc);
-        ptx::tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < k_iters; ++kb, ++it) {
-          const int st = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          ptx::mbar_wait(&full[st], ph, err, 0x300u + st);
-          if (SPARSE) ptx::mbar_wait(&meta_ready[st], ph, err, 0x400u + st);
-          ptx::tc_fence_after_sync();
-          const uint64_t adesc = ptx::make_smem_desc(ptx::smem_u32(sA + st * kABytes), 16, 1024, 2);
-          const uint64_t bdesc =
-              ptx::make_smem_desc(ptx::smem_u32(sB + st * C::kBBytes), C::kKB * 128, 1024, 2);
-          if (SPARSE) {
-            const uint64_t edesc = ptx::make_smem_desc(ptx::smem_u32(sEhw + st * kEBytes), 128, 128, 0);
-            ptx::tc_cp_128x128b(tmem_base + (uint32_t)(C::kMetaCol + 4 * st), edesc);
-          }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t accumulate = (kb > 0 || j > 0) ? 1u : 0u;
-            // A: 32 bytes of a 128-byte swizzled row per MMA; B: 16 (dense) or 32 (sparse) rows of 128 B
-            const uint64_t a_j = adesc + (uint64_t)(j * 2);
-            const uint64_t b_j = bdesc + (uint64_t)(j * (C::kKB / 4) * 128 / 16);
-            if (SPARSE) {
-              const uint32_t col = (uint32_t)(C::kMetaCol + 4 * st + j);
-              ptx::mma_sp_f16_ss(d_tmem, a_j, b_j, tmem_base + (col & ~1u), idesc | (col & 1u), accumulate);
-            } else {
-              ptx::mma_f16_ss(d_tmem, a_j, b_j, idesc, accumulate);
-            }
-          }
-          ptx::tc_commit(&empty[st]);
-        }
-        ptx::tc_commit(&acc_full[acc]);
-      }
-    }
-  } else if (warp < 6) {
-    // ------------------------------------------------- metadata rearranger
-    if (SPARSE) {
-      uint32_t it = 0;
-      for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
-        for (int kb = 0; kb < k_iters; ++kb, ++it) {
-          if ((int)(it & 3u) != warp - 2) continue;  // this warp's turn: every fourth stage use
-          const int st = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          ptx::mbar_wait(&full[st], ph, err, 0x500u + st);
-          rearrange_metadata_stage(sEraw + st * kEBytes, sEhw + st * kEBytes, lane, rows_used);
-          ptx::fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&meta_ready[st]);
-        }
-      }
-    }
-  } else {
-    // ------------------------------------------------------------ epilogue
-    const int q = warp & 3;  // a warp may only touch TMEM lanes [32*(warp%4), +32)
-    const int row = q * 32 + lane;
-    const bool issuer = (threadIdx.x == 192);
-    uint32_t lt = 0, chunk = 0;
-    for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++lt) {
-      int t = tile;
-      const int nt = t % p.tiles_n; t /= p.tiles_n;
-      const int wt = t % p.tiles_w; t /= p.tiles_w;
-      const int ht = t % p.tiles_h; t /= p.tiles_h;
-      const int bt = t;
-      const int acc = lt % NACC;
-      const uint32_t aph = (lt / NACC) & 1u;
-      ptx::mbar_wait(&acc_full[acc], aph, err, 0x600u + acc);
-      ptx::tc_fence_after_sync();
-      store_accumulator<BN, C::kOutBufs>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), sOut, &tmD,
-                                         nt * BN, wt * p.TW, ht * p.TH, bt * p.TB, true, row, issuer, chunk);
-      ptx::tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
-    }
-    if (issuer) ptx::bulk_wait_group_all();  // dD is written before the CTA leaves
-  }
-
-  ptx::tc_fence_before_sync();
-  __syncthreads();
-  ptx::tc_fence_after_sync();
-  if (warp == 1) ptx::tmem_dealloc(tmem_base, kTmemCols);
-}
-
-
-// ------------------------------------------------------------------------------------------
-// CTA-pair variant (cta_group::2). Two CTAs of a cluster own two neighbouring 128-pixel
-// patches and one BN-wide column block: each stages its own A patch (+ metadata) and HALF of
-// the W columns, and a single thread of the pair's first CTA issues 256-row MMAs that read
-// both halves. Per CTA this halves the W bytes and TMA requests per FLOP and the shared-memory
-// reads of B, and leaves room in TMEM for BN = 256.
-//
-// Barriers: full / meta_ready / acc_empty are waited on by the first CTA only and collect
-// arrivals from both; empty / acc_full exist in both CTAs and are signalled together by a
-// multicast tcgen05.commit; meta_full is local (each CTA's own metadata box).
-
-template <bool SPARSE, int BN>
-struct PairCfg {
-  static constexpr int kKB = SPARSE ? 128 : 64;
-  static constexpr int kBCols = BN / 2;                    // W columns staged by one CTA
-  static constexpr int kBBytes = kKB * kBCols * 2;
-  static constexpr int kStageBytes = kABytes + kBBytes + (SPARSE ? 2 * kEBytes : 0);
-  static constexpr int kSmemBudget = 232448 - 2048;
-  static constexpr int kOutBufs = ((kSmemBudget - 2 * kOutBytes) / kStageBytes >= 4) ? 2 : 1;
-  static constexpr int kStagesFit = (kSmemBudget - kOutBufs * kOutBytes) / kStageBytes;
-  static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
-  static constexpr int kAcc = (2 * BN + (SPARSE ? 4 * kStages : 0) <= (int)kTmemCols) ? 2 : 1;
-  static constexpr int kMetaCol = kAcc * BN;
-  static constexpr int kSmemBytes = kStages * kStageBytes + kOutBufs * kOutBytes + 2048;
-  static_assert(kBCols % 64 == 0, "each CTA stages whole 64-column swizzle blocks of W");
-  static_assert(kStages >= 2, "pipeline needs at least two stages");
-};
-
-__host__ __device__ constexpr uint32_t make_idesc_pair(int n, bool sparse) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
-         ((uint32_t)(256 >> 4) << 24) | (sparse ? (1u << 2) : 0u);
-}
-
-template <bool SPARSE, int BN>
-__global__ void __launch_bounds__(kThreadsGemm, 1)
-dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmE,
-                  const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
-                  const DgradParams p) {
-  using C = PairCfg<SPARSE, BN>;
-  constexpr int STAGES = C::kStages;
-  constexpr int NACC = C::kAcc;
-
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* sA = smem;
-  uint8_t* sB = sA + STAGES * kABytes;
-  uint8_t* sEraw = sB + STAGES * C::kBBytes;
-  uint8_t* sEhw = sEraw + (SPARSE ? STAGES * kEBytes : 0);
-  uint8_t* sOut = sEhw + (SPARSE ? STAGES * kEBytes : 0);
-  uint64_t* bars = (uint64_t*)(sOut + C::kOutBufs * kOutBytes);
-  uint64_t* full = bars;
-  uint64_t* empty = full + STAGES;
-  uint64_t* meta_full = empty + STAGES;
-  uint64_t* meta_ready = meta_full + STAGES;
-  uint64_t* acc_full = meta_ready + STAGES;
-  uint64_t* acc_empty = acc_full + 2;
-  uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+  uint64_t* w_full = acc_empty + 2;
+  uint32_t* tmem_slot = (uint32_t*)(w_full + 1);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t rank = ptx::cluster_ctarank();  // 0: issues the MMAs
   unsigned int* err = &g_device_error;
+  const int STAGES = p.stages;
+  const int NACC = p.nacc;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
+    for (int s = 0; s < kMaxStages; ++s) {
       ptx::mbar_init(&full[s], 1);
       ptx::mbar_init(&empty[s], 1);
       ptx::mbar_init(&meta_full[s], 1);
-      ptx::mbar_init(&meta_ready[s], 2);
+      ptx::mbar_init(&meta_ready[s], 8);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&acc_full[a], 1);
       ptx::mbar_init(&acc_empty[a], 8);
     }
+    ptx::mbar_init(w_full, 1);
     ptx::fence_mbar_init();
   }
   if (warp == 0 && lane == 0) {
@@ -418,130 +222,186 @@ dgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
   const int rows_used = p.TW * p.TH * p.TB;
   const int taps = p.R * p.S;
-  const int k_iters = taps * p.k_blocks_per_tap;
+  const bool reuse = (p.rr == p.R) && p.R > 1;
+  const int groups = reuse ? p.S : taps;  // stage uses per channel block and tile
+  const int uses_per_tile = groups * p.k_blocks;
   const int pair_stride = gridDim.x >> 1;
   const int first_pair = blockIdx.x >> 1;
+  const int n_half = (int)rank * C::kBCols;  // this CTA's column offset inside the BN block
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer
     if (ptx::elect_one()) {
-      const uint32_t pair_tx = 2u * (uint32_t)(rows_used * 128 + C::kBBytes);
-      uint32_t it = 0;
-      for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride) {
+      bool alive = true;
+      if (p.w_resident) {
+        // the layer's whole W half-slice, once: [tap][channel block][box] tiles of kKB rows
+        if (rank == 0) ptx::mbar_arrive_expect_tx(w_full, 2u * (uint32_t)(taps * p.k_blocks * C::kTapBBytes));
+        for (int t = 0; t < taps; ++t)
+          for (int cb = 0; cb < p.k_blocks; ++cb)
+#pragma unroll
+            for (int j = 0; j < C::kBoxes; ++j)
+              ptx::tma_load_2d_pair(sW + ((t * p.k_blocks + cb) * C::kBoxes + j) * C::kBoxBytes, &tmB, w_full,
+                                    t * p.Cin + n_half + C::kBoxCols * j, cb * C::kKB);
+      }
+      const uint32_t pair_tx = 2u * (uint32_t)(p.img_rows * 128 + (p.w_resident ? 0 : p.rr * C::kTapBBytes));
+      const uint32_t meta_tx = (uint32_t)(p.img_rows * 16);
+      int st = 0;
+      uint32_t ph = 0;
+      for (int pt = first_pair; alive && pt < p.pair_tiles; pt += pair_stride) {
         const int nt = pt % p.tiles_n;
         int t = 2 * (pt / p.tiles_n) + (int)rank;  // this CTA's patch; may lie past the last one
         const int wt = t % p.tiles_w; t /= p.tiles_w;
         const int ht = t % p.tiles_h; t /= p.tiles_h;
         const int bt = t;
-        const int n0 = nt * BN + (int)rank * C::kBCols;
+        const int n0 = nt * BN + n_half;
         const int w0 = wt * p.TW, h0 = ht * p.TH, b0 = bt * p.TB;
-        for (int tap = 0; tap < taps; ++tap) {
-          const int r = tap / p.S, s = tap - r * p.S;
+        // reuse: a group is the horizontal tap s and the image starts R-1 rows above the row
+        // the last vertical tap needs; otherwise a group is the single tap (r, s).
+        int r = reuse ? (p.R - 1) : 0, s = 0;
+        for (int g = 0; alive && g < groups; ++g) {
           const int q0 = w0 + p.pad - s, p0 = h0 + p.pad - r;
-          for (int cb = 0; cb < p.k_blocks_per_tap; ++cb, ++it) {
-            const int st = it % STAGES;
-            const uint32_t ph = (it / STAGES) & 1u;
-            ptx::mbar_wait(&empty[st], ph ^ 1u, err, 0x1100u + st);
+          for (int cb = 0; cb < p.k_blocks; ++cb) {
+            if (!ptx::mbar_wait(&empty[st], ph ^ 1u, err, 0x100u + st)) { alive = false; break; }
             if (rank == 0) ptx::mbar_arrive_expect_tx(&full[st], pair_tx);
             if (SPARSE) {
-              ptx::mbar_arrive_expect_tx(&meta_full[st], (uint32_t)(rows_used * 16));
-              if (p.meta_merged) ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &meta_full[st], 8 * q0, p0, b0, 0);
-              else ptx::tma_load_4d(sEraw + st * kEBytes, &tmE, &meta_full[st], cb * 8, q0, p0, b0);
+              ptx::mbar_arrive_expect_tx(&meta_full[st], meta_tx);
+              ptx::tma_load_4d(sEraw + st * p.eraw_bytes, &tmE, &meta_full[st], cb * 8, q0, p0, b0);
             }
-            ptx::tma_load_4d_pair(sA + st * kABytes, &tmA, &full[st], cb * 64, q0, p0, b0);
+            ptx::tma_load_4d_pair(sA + st * p.a_bytes, &tmA, &full[st], cb * 64, q0, p0, b0);
+            if (!p.w_resident) {
+              for (int u = 0; u < p.rr; ++u) {
+                const int tap = (reuse ? u : r) * p.S + s;
 #pragma unroll
-            for (int j = 0; j < C::kBCols / 64; ++j)
-              ptx::tma_load_2d_pair(sB + st * C::kBBytes + j * (C::kKB * 128), &tmB, &full[st],
-                                    tap * p.Cin + n0 + 64 * j, cb * C::kKB);
+                for (int j = 0; j < C::kBoxes; ++j)
+                  ptx::tma_load_2d_pair(sB + st * p.b_bytes + (u * C::kBoxes + j) * C::kBoxBytes, &tmB, &full[st],
+                                        tap * p.Cin + n0 + C::kBoxCols * j, cb * C::kKB);
+              }
+            }
+            if (++st == STAGES) { st = 0; ph ^= 1u; }
           }
+          if (++s == p.S) { s = 0; if (!reuse) ++r; }
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------- MMA issuer (first CTA only)
     if (rank == 0 && ptx::elect_one()) {
-      constexpr uint32_t idesc = make_idesc_pair(BN, SPARSE);
-      uint32_t it = 0, lt = 0;
-      for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride, ++lt) {
-        const int acc = lt % NACC;
-        const uint32_t aph = (lt / NACC) & 1u;
-        ptx::mbar_wait(&acc_empty[acc], aph ^ 1u, err, 0x1200u + acc);
+      constexpr uint32_t idesc = make_idesc(BN, SPARSE);
+      bool alive = true;
+      if (p.w_resident) alive = ptx::mbar_wait(w_full, 0u, err, 0x700u);
+      // descriptor constants; the 14-bit address field is added per use (all addresses < 256 KiB)
+      const uint64_t adesc0 = ptx::make_smem_desc(0, 16, 1024, 2);
+      const uint64_t bdesc0 = ptx::make_smem_desc(0, C::kBoxBytes, 8 * C::kRowB, C::kBSwizzle);
+      const uint64_t edesc0 = ptx::make_smem_desc(0, 128, 128, 0);
+      const uint32_t sA_u = ptx::smem_u32(sA), sB_u = ptx::smem_u32(sB), sW_u = ptx::smem_u32(sW),
+                     sE_u = ptx::smem_u32(sEhw);
+      int st = 0, acc = 0;
+      uint32_t ph = 0, aph = 0;
+      for (int pt = first_pair; alive && pt < p.pair_tiles; pt += pair_stride) {
+        if (!ptx::mbar_wait(&acc_empty[acc], aph ^ 1u, err, 0x200u + acc)) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < k_iters; ++kb, ++it) {
-          const int st = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          ptx::mbar_wait(&full[st], ph, err, 0x1300u + st);
-          if (SPARSE) ptx::mbar_wait(&meta_ready[st], ph, err, 0x1400u + st);
-          ptx::tc_fence_after_sync();
-          const uint64_t adesc = ptx::make_smem_desc(ptx::smem_u32(sA + st * kABytes), 16, 1024, 2);
-          const uint64_t bdesc =
-              ptx::make_smem_desc(ptx::smem_u32(sB + st * C::kBBytes), C::kKB * 128, 1024, 2);
-          if (SPARSE) {
-            const uint64_t edesc = ptx::make_smem_desc(ptx::smem_u32(sEhw + st * kEBytes), 128, 128, 0);
-            ptx::tc_cp_128x128b_pair(tmem_base + (uint32_t)(C::kMetaCol + 4 * st), edesc);
-          }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t accumulate = (kb > 0 || j > 0) ? 1u : 0u;
-            const uint64_t a_j = adesc + (uint64_t)(j * 2);
-            const uint64_t b_j = bdesc + (uint64_t)(j * (C::kKB / 4) * 128 / 16);
+        uint32_t accumulate = 0u;
+        int r_single = 0, s = 0;
+        for (int g = 0; alive && g < groups; ++g) {
+          for (int cb = 0; cb < p.k_blocks; ++cb) {
+            if (!ptx::mbar_wait(&full[st], ph, err, 0x300u + st)) { alive = false; break; }
+            if (SPARSE && !ptx::mbar_wait(&meta_ready[st], ph, err, 0x400u + st)) { alive = false; break; }
+            ptx::tc_fence_after_sync();
+            const uint32_t meta_slot = (uint32_t)(p.meta_col + st * p.rr * 4);
             if (SPARSE) {
-              const uint32_t col = (uint32_t)(C::kMetaCol + 4 * st + j);
-              ptx::mma_sp_f16_ss_pair(d_tmem, a_j, b_j, tmem_base + (col & ~1u), idesc | (col & 1u), accumulate);
-            } else {
-              ptx::mma_f16_ss_pair(d_tmem, a_j, b_j, idesc, accumulate);
+              for (int u = 0; u < p.rr; ++u)
+                ptx::tc_cp_128x128b_pair(tmem_base + meta_slot + 4u * u,
+                                         edesc0 + ((sE_u + st * p.ehw_bytes + u * kEHwBytes) >> 4));
             }
+            for (int u = 0; u < p.rr; ++u) {
+              // vertical tap r: the tile's rows start (R-1-r) image rows into the stage
+              const int r = reuse ? u : r_single;
+              const int row_off = reuse ? (p.R - 1 - r) * p.TW : 0;
+              const uint32_t b_addr = p.w_resident ? sW_u + ((r * p.S + s) * p.k_blocks + cb) * C::kTapBBytes
+                                                   : sB_u + st * p.b_bytes + u * C::kTapBBytes;
+              const uint64_t adesc = adesc0 + ((sA_u + st * p.a_bytes + row_off * 128) >> 4);
+              const uint64_t bdesc = bdesc0 + (b_addr >> 4);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                // A: 32 bytes of a 128-byte swizzled row per MMA; B: 16 (dense) or 32 (sparse) rows
+                const uint64_t a_j = adesc + (uint64_t)(j * 2);
+                const uint64_t b_j = bdesc + (uint64_t)(j * (C::kKB / 4) * C::kRowB / 16);
+                if (SPARSE) {
+                  const uint32_t col = meta_slot + 4u * u + j;
+                  ptx::mma_sp_f16_ss_pair(d_tmem, a_j, b_j, tmem_base + (col & ~1u), idesc | (col & 1u), accumulate);
+                } else {
+                  ptx::mma_f16_ss_pair(d_tmem, a_j, b_j, idesc, accumulate);
+                }
+                accumulate = 1u;
+              }
+            }
+            ptx::tc_commit_pair(&empty[st], 3);
+            if (++st == STAGES) { st = 0; ph ^= 1u; }
           }
-          ptx::tc_commit_pair(&empty[st], 3);
+          if (++s == p.S) { s = 0; ++r_single; }
         }
-        ptx::tc_commit_pair(&acc_full[acc], 3);
+        if (alive) ptx::tc_commit_pair(&acc_full[acc], 3);
+        if (++acc == NACC) { acc = 0; aph ^= 1u; }
       }
     }
   } else if (warp < 6) {
     // ------------------------------------------------- metadata rearranger
     if (SPARSE) {
-      uint32_t it = 0;
-      for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride) {
-        for (int kb = 0; kb < k_iters; ++kb, ++it) {
-          if ((int)(it & 3u) != warp - 2) continue;
-          const int st = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          ptx::mbar_wait(&meta_full[st], ph, err, 0x1500u + st);
-          rearrange_metadata_stage(sEraw + st * kEBytes, sEhw + st * kEBytes, lane, rows_used);
+      // thread = A-tile row; the four warps handle every stage use together, in order
+      const int row = threadIdx.x - 64;
+      bool alive = true;
+      int st = 0;
+      uint32_t ph = 0;
+      for (int pt = first_pair; alive && pt < p.pair_tiles; pt += pair_stride) {
+        for (int k = 0; k < uses_per_tile; ++k) {
+          if (!ptx::mbar_wait(&meta_full[st], ph, err, 0x500u + st)) { alive = false; break; }
+          for (int u = 0; u < p.rr; ++u) {
+            const int row_off = reuse ? (p.R - 1 - u) * p.TW : 0;
+            rearrange_metadata_row(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + u * kEHwBytes,
+                                   row, rows_used);
+          }
           ptx::fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive_cluster(&meta_ready[st], 0);
+          if (++st == STAGES) { st = 0; ph ^= 1u; }
         }
       }
     }
   } else {
     // ------------------------------------------------------------ epilogue
-    const int q = warp & 3;
+    const int q = warp & 3;  // a warp may only touch TMEM lanes [32*(warp%4), +32)
     const int row = q * 32 + lane;
     const bool issuer = (threadIdx.x == 192);
-    uint32_t lt = 0, chunk = 0;
-    for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride, ++lt) {
+    uint32_t chunk = 0, aph = 0;
+    int acc = 0;
+    for (int pt = first_pair; pt < p.pair_tiles; pt += pair_stride) {
       const int nt = pt % p.tiles_n;
       const int mt = 2 * (pt / p.tiles_n) + (int)rank;
       int t = mt;
       const int wt = t % p.tiles_w; t /= p.tiles_w;
       const int ht = t % p.tiles_h; t /= p.tiles_h;
       const int bt = t;
-      const int acc = lt % NACC;
-      const uint32_t aph = (lt / NACC) & 1u;
-      ptx::mbar_wait(&acc_full[acc], aph, err, 0x1600u + acc);
+      if (!ptx::mbar_wait(&acc_full[acc], aph, err, 0x600u + acc)) break;
       ptx::tc_fence_after_sync();
-      store_accumulator<BN, C::kOutBufs>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), sOut, &tmD,
-                                         nt * BN, wt * p.TW, ht * p.TH, bt * p.TB, mt < p.m_tiles, row, issuer,
-                                         chunk);
+      store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), sOut, p.out_bufs, &tmD,
+                            nt * BN, wt * p.TW, ht * p.TH, bt * p.TB, mt < p.m_tiles, row, issuer, chunk);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
+      if (++acc == NACC) { acc = 0; aph ^= 1u; }
     }
-    if (issuer) ptx::bulk_wait_group_all();
+    if (issuer) ptx::bulk_wait_group_all();  // dD is written before the CTA leaves
   }
 
+  __syncwarp();
+  if (*(volatile unsigned int*)err != 0u) {
+    // A wait gave up somewhere: loads may still be in flight towards this CTA's shared
+    // memory. Give them a bounded while to land before the CTA goes away.
+    const uint64_t t0 = ptx::globaltimer_ns();
+    while (ptx::globaltimer_ns() - t0 < 200000ull) {
+    }
+  }
   ptx::tc_fence_before_sync();
   __syncwarp();
   ptx::cluster_sync();  // neither CTA leaves (or frees TMEM) while the other may still touch it
@@ -616,30 +476,111 @@ int sm_count() {
   return n;
 }
 
+int round_up(int x, int a) { return (x + a - 1) / a * a; }
+
+// Shared-memory plan for one launch: decides filter-row reuse, resident W, pipeline depth,
+// accumulator count and the carve. Returns false if no variant fits.
 template <bool SPARSE, int BN>
-sdgp_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmE, const CUtensorMap& tmB,
-                       const CUtensorMap& tmD, const DgradParams& p, cudaStream_t stream) {
+bool plan(DgradParams* p) {
   using C = Cfg<SPARSE, BN>;
-  static bool configured = false;
-  auto kernel = dgrad_kernel<SPARSE, BN>;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-      return SDGP_ERR_CUDA;
-    configured = true;
+  const int taps = p->R * p->S;
+  const int budget = kSmemLimit - kSmemSlack;
+  // Filter-row reuse needs a single-image patch whose rows are whole groups of 8 pixels, so
+  // that every vertical tap is an offset of whole 1024-byte swizzle periods.
+  const bool can_reuse = p->R > 1 && p->TB == 1 && p->TW % 8 == 0 && p->TW * (p->TH + p->R - 1) <= kMaxImgRows;
+  const bool can_reside = p->tiles_n == 1 && p->pair_tiles > sm_count() / 2;  // pays only if tiles repeat
+  for (int attempt = 0; attempt < 4; ++attempt) {
+    // attempt 0: reuse + resident W, 1: reuse, 2: resident W, 3: neither
+    const bool reuse = attempt < 2;
+    const bool resident = (attempt == 0 || attempt == 2);
+    if ((reuse && !can_reuse) || (resident && !can_reside)) continue;
+    p->rr = reuse ? p->R : 1;
+    p->img_rows = p->TW * (p->TH + p->rr - 1) * p->TB;
+    p->w_resident = resident ? 1 : 0;
+    p->a_bytes = round_up(p->img_rows * 128, 1024);
+    p->b_bytes = resident ? 0 : p->rr * C::kTapBBytes;
+    p->eraw_bytes = SPARSE ? round_up(p->img_rows * 16, 128) : 0;
+    p->ehw_bytes = SPARSE ? p->rr * kEHwBytes : 0;
+    const int w_bytes = resident ? taps * p->k_blocks * C::kTapBBytes : 0;
+    const int stage_bytes = p->a_bytes + p->b_bytes + p->eraw_bytes + p->ehw_bytes;
+    int out_bufs = 2;
+    int stages = (budget - w_bytes - out_bufs * kOutBytes) / stage_bytes;
+    if (stages < 4) {
+      out_bufs = 1;
+      stages = (budget - w_bytes - out_bufs * kOutBytes) / stage_bytes;
+    }
+    if (stages > kMaxStages) stages = kMaxStages;
+    // TMEM: accumulators first, metadata slots (4 columns per tap and stage) behind them
+    const int meta_cols_per_stage = SPARSE ? 4 * p->rr : 0;
+    int nacc = (2 * BN + 2 * meta_cols_per_stage <= (int)kTmemCols) ? 2 : 1;
+    if (meta_cols_per_stage > 0) {
+      const int max_meta_stages = ((int)kTmemCols - nacc * BN) / meta_cols_per_stage;
+      if (stages > max_meta_stages) stages = max_meta_stages;
+    }
+    if (stages < ((resident || reuse) ? 2 : 3)) continue;  // a reuse stage is R taps long
+    p->stages = stages;
+    p->nacc = nacc;
+    p->meta_col = nacc * BN;
+    p->out_bufs = out_bufs;
+    p->off_b = stages * p->a_bytes;
+    p->off_eraw = p->off_b + stages * p->b_bytes;
+    p->off_ehw = round_up(p->off_eraw + stages * p->eraw_bytes, 1024);
+    p->off_w = round_up(p->off_ehw + stages * p->ehw_bytes, 1024);
+    p->off_out = round_up(p->off_w + w_bytes, 1024);
+    p->off_bar = p->off_out + out_bufs * kOutBytes;
+    p->smem_bytes = p->off_bar + 512 + 1024;
+    if (p->smem_bytes > kSmemLimit) continue;
+    return true;
   }
-  const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
-  kernel<<<grid, kThreadsGemm, C::kSmemBytes, stream>>>(tmA, tmE, tmB, tmD, p);
-  return cudaGetLastError() == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
+  return false;
 }
 
 template <bool SPARSE, int BN>
-sdgp_status launch_pair_cfg(const CUtensorMap& tmA, const CUtensorMap& tmE, const CUtensorMap& tmB,
-                            const CUtensorMap& tmD, const DgradParams& p, cudaStream_t stream) {
-  using C = PairCfg<SPARSE, BN>;
+sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, void* dD, DgradParams p, int P, int Q,
+                       cudaStream_t stream) {
+  using C = Cfg<SPARSE, BN>;
+  if (!plan<SPARSE, BN>(&p)) return SDGP_ERR_UNSUPPORTED;
+
+  CUtensorMap tmA, tmE, tmB, tmD;
+  const uint32_t img_h = (uint32_t)(p.TH + p.rr - 1);
+  const uint64_t CA = SPARSE ? (uint64_t)p.Cout / 2 : (uint64_t)p.Cout;  // stored elements per pixel
+  {
+    const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)P, (uint64_t)p.B};
+    const uint64_t strides[3] = {CA * 2, CA * 2 * Q, CA * 2 * Q * P};
+    const uint32_t box[4] = {64, (uint32_t)p.TW, img_h, (uint32_t)p.TB};
+    if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+      return SDGP_ERR_CUDA;
+  }
+  if (SPARSE) {
+    const uint64_t CE = (uint64_t)p.Cout / 16;
+    const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)P, (uint64_t)p.B};
+    const uint64_t strides[3] = {CE * 2, CE * 2 * Q, CE * 2 * Q * P};
+    const uint32_t box[4] = {8, (uint32_t)p.TW, img_h, (uint32_t)p.TB};
+    if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
+      return SDGP_ERR_CUDA;
+  } else {
+    tmE = tmA;
+  }
+  {
+    const uint64_t dims[2] = {(uint64_t)p.R * p.S * p.Cin, (uint64_t)p.Cout};
+    const uint64_t strides[1] = {(uint64_t)p.R * p.S * p.Cin * 2};
+    const uint32_t box[2] = {(uint32_t)C::kBoxCols, (uint32_t)C::kKB};
+    if (!encode(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Wt, dims, strides, box,
+                C::kRowB == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
+      return SDGP_ERR_CUDA;
+  }
+  {
+    const uint64_t dims[4] = {(uint64_t)p.Cin, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.B};
+    const uint64_t strides[3] = {(uint64_t)p.Cin * 2, (uint64_t)p.Cin * 2 * p.W, (uint64_t)p.Cin * 2 * p.W * p.H};
+    const uint32_t box[4] = {64, (uint32_t)p.TW, (uint32_t)p.TH, (uint32_t)p.TB};
+    if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, dD, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+      return SDGP_ERR_CUDA;
+  }
+
   static bool configured = false;
-  auto kernel = dgrad_pair_kernel<SPARSE, BN>;
+  auto kernel = dgrad_kernel<SPARSE, BN>;
   if (!configured) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
       return SDGP_ERR_CUDA;
     configured = true;
   }
@@ -648,7 +589,7 @@ sdgp_status launch_pair_cfg(const CUtensorMap& tmA, const CUtensorMap& tmE, cons
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs));
   cfg.blockDim = dim3(kThreadsGemm);
-  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -672,13 +613,10 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
   if (Cin % 64 != 0 || Cout % (sparse ? 128 : 64) != 0) return SDGP_ERR_UNSUPPORTED;
   if ((int64_t)R * S * Cin > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
 
-  // CTA pairs whenever the column count allows whole 64-column halves; the single-CTA kernel
-  // serves Cin = 64 (mod 128).
-  const bool pair = (Cin % 128 == 0);
-  const int BN = pair ? ((Cin % 256 == 0) ? 256 : 128) : 64;
+  const int BN = (Cin % 256 == 0) ? 256 : (Cin % 128 == 0) ? 128 : 64;
   const int kb_channels = sparse ? 128 : 64;
 
-  DgradParams p;
+  DgradParams p = {};
   p.B = B; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout; p.R = R; p.S = S; p.pad = pad;
   choose_patch(B, H, W, &p.TW, &p.TH, &p.TB);
   p.tiles_w = (W + p.TW - 1) / p.TW;
@@ -686,69 +624,19 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
   p.tiles_b = (B + p.TB - 1) / p.TB;
   p.tiles_n = Cin / BN;
   const int64_t m_tiles = (int64_t)p.tiles_w * p.tiles_h * p.tiles_b;
-  const int64_t total = m_tiles * p.tiles_n;
-  if (total > 0x3FFFFFFF) return SDGP_ERR_UNSUPPORTED;
+  if (m_tiles * p.tiles_n > 0x3FFFFFFF) return SDGP_ERR_UNSUPPORTED;
   p.m_tiles = (int)m_tiles;
-  p.total_tiles = (int)total;
   p.pair_tiles = (int)((m_tiles + 1) / 2) * p.tiles_n;
-  p.k_blocks_per_tap = (Cout + kb_channels - 1) / kb_channels;
-  p.dD = (uint16_t*)dD;
+  p.k_blocks = (Cout + kb_channels - 1) / kb_channels;
 
-  CUtensorMap tmA, tmE, tmB;
-  const uint64_t CA = sparse ? (uint64_t)Cout / 2 : (uint64_t)Cout;  // stored elements per pixel
-  {
-    const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)P, (uint64_t)B};
-    const uint64_t strides[3] = {CA * 2, CA * 2 * Q, CA * 2 * Q * P};
-    const uint32_t box[4] = {64, (uint32_t)p.TW, (uint32_t)p.TH, (uint32_t)p.TB};
-    if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
-      return SDGP_ERR_CUDA;
+  if (sparse) {
+    if (BN == 256) return launch_cfg<true, 256>(A, meta, Wt, dD, p, P, Q, stream);
+    if (BN == 128) return launch_cfg<true, 128>(A, meta, Wt, dD, p, P, Q, stream);
+    return launch_cfg<true, 64>(A, meta, Wt, dD, p, P, Q, stream);
   }
-  p.meta_merged = 0;
-  if (sparse && Cout == 128 && p.TW <= 32) {
-    // One pixel's metadata is a single 16-byte run and pixels of an image row are contiguous:
-    // fetch whole rows of the patch per TMA request instead of one request per pixel.
-    p.meta_merged = 1;
-    const uint64_t dims[4] = {8ull * Q, (uint64_t)P, (uint64_t)B, 1};
-    const uint64_t strides[3] = {16ull * Q, 16ull * Q * P, 16ull * Q * P * B};
-    const uint32_t box[4] = {8u * (uint32_t)p.TW, (uint32_t)p.TH, (uint32_t)p.TB, 1};
-    if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
-      return SDGP_ERR_CUDA;
-  } else if (sparse) {
-    const uint64_t CE = (uint64_t)Cout / 16;
-    const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)P, (uint64_t)B};
-    const uint64_t strides[3] = {CE * 2, CE * 2 * Q, CE * 2 * Q * P};
-    const uint32_t box[4] = {8, (uint32_t)p.TW, (uint32_t)p.TH, (uint32_t)p.TB};
-    if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
-      return SDGP_ERR_CUDA;
-  } else {
-    tmE = tmA;
-  }
-  {
-    const uint64_t dims[2] = {(uint64_t)R * S * Cin, (uint64_t)Cout};
-    const uint64_t strides[1] = {(uint64_t)R * S * Cin * 2};
-    const uint32_t box[2] = {64, (uint32_t)kb_channels};
-    if (!encode(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Wt, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
-      return SDGP_ERR_CUDA;
-  }
-
-  CUtensorMap tmD;
-  {
-    const uint64_t dims[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)B};
-    const uint64_t strides[3] = {(uint64_t)Cin * 2, (uint64_t)Cin * 2 * W, (uint64_t)Cin * 2 * W * H};
-    const uint32_t box[4] = {64, (uint32_t)p.TW, (uint32_t)p.TH, (uint32_t)p.TB};
-    if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, dD, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
-      return SDGP_ERR_CUDA;
-  }
-
-  if (pair) {
-    if (sparse)
-      return BN == 256 ? launch_pair_cfg<true, 256>(tmA, tmE, tmB, tmD, p, stream)
-                       : launch_pair_cfg<true, 128>(tmA, tmE, tmB, tmD, p, stream);
-    return BN == 256 ? launch_pair_cfg<false, 256>(tmA, tmE, tmB, tmD, p, stream)
-                     : launch_pair_cfg<false, 128>(tmA, tmE, tmB, tmD, p, stream);
-  }
-  return sparse ? launch_cfg<true, 64>(tmA, tmE, tmB, tmD, p, stream)
-                : launch_cfg<false, 64>(tmA, tmE, tmB, tmD, p, stream);
+  if (BN == 256) return launch_cfg<false, 256>(A, meta, Wt, dD, p, P, Q, stream);
+  if (BN == 128) return launch_cfg<false, 128>(A, meta, Wt, dD, p, P, Q, stream);
+  return launch_cfg<false, 64>(A, meta, Wt, dD, p, P, Q, stream);
 }
 
 sdgp_status read_device_error() {

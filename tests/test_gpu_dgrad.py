@@ -127,6 +127,48 @@ def test_pruned_conv_two_pass(case, scheme):
     assert rel_fro(to_f64(dD), oracle.dgrad_conv2d(pruned, W, H, Wd, 1, pad)) <= TOL
 
 
+# Shapes that switch on the kernel's shared-memory reuse modes: enough tiles that every CTA
+# pair gets several (resident W), 3x3 filters on 16- and 32-wide images (one A image serves the
+# three vertical taps), 64 input channels (32-column W halves), two channel blocks (streamed W).
+REUSE_CASES = [
+    (40, 16, 16, 128, 128, 3, 3, 1),
+    (20, 32, 32, 64, 128, 3, 3, 1),
+    (40, 16, 16, 128, 256, 3, 3, 1),
+    (3, 32, 32, 192, 128, 3, 3, 1),
+    (80, 8, 8, 64, 128, 3, 3, 1),
+    (24, 16, 16, 64, 64, 3, 3, 1),
+]
+
+
+@pytest.mark.parametrize("mode", ["dense", "sparse"])
+@pytest.mark.parametrize("case", REUSE_CASES)
+def test_conv_reuse_modes_sampled(case, mode):
+    import paper_2202_00774_b200 as sdgp
+    B, H, Wd, Cin, Cout, R, S, pad = case
+    if mode == "sparse" and Cout % 128:
+        pytest.skip("compressed path needs Cout % 128 == 0")
+    layer = inputs.ConvLayer("t", B, H, Wd, Cin, Cout, R, S, 1, pad)
+    dO, W = inputs.conv_layer_tensors(layer, seed=B + Cin)
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    if mode == "dense":
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, pad, 4, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
+        src = dO
+    else:
+        ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(B, H, Wd, Cin, Cout, R, S, 1, pad), dtype=torch.uint8,
+                         device="cuda")
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, pad, 2, 4, sdgp.MAGNITUDE, seed=3, workspace=ws)
+        src = oracle.prune(dO.reshape(-1, Cout), 2, 4, oracle.MAGNITUDE, 3, want=("dense",))["dense"].reshape(dO.shape)
+    check_no_device_error()
+    rng = np.random.default_rng(1)
+    npix = B * H * Wd
+    idx = np.unique(np.concatenate([rng.integers(0, npix, 1500), np.arange(0, 300), np.arange(npix - 300, npix)]))
+    want = oracle.dgrad_conv2d(src, W, H, Wd, 1, pad, pixel_index=idx)
+    got = to_f64(dD).reshape(npix, Cin)[idx]
+    assert rel_fro(got, want) <= TOL
+    # nothing outside the sample is left unwritten (the buffer was pre-filled with 0xFFFF = NaN)
+    assert not np.isnan(to_f64(dD)).any()
+
+
 def test_unsupported_requests_raise():
     import paper_2202_00774_b200 as sdgp
     dO = torch.zeros((2, 4, 4, 128), dtype=torch.int16, device="cuda")
