@@ -104,10 +104,15 @@ class OracleArm:
         return flops
 
     def pixels_for(self, seconds):
-        probe = 8
-        t0 = time.perf_counter()
-        self.step(probe)
-        dt = max(time.perf_counter() - t0, 1e-6)
+        # grow the probe until it is long enough to be dominated by the arithmetic, then scale
+        probe, dt = 8, 0.0
+        while True:
+            t0 = time.perf_counter()
+            self.step(probe)
+            dt = max(time.perf_counter() - t0, 1e-6)
+            if dt >= min(0.5, seconds / 4) or probe >= (1 << 20):
+                break
+            probe *= 4
         return int(max(1, probe * seconds / dt))
 
 
@@ -286,27 +291,51 @@ def run_ours(args, layers):
     value = world * total_flops / (ms_per_step * 1e-3) / 1e12
     dense_value = world * total_flops / (ms_dense / dense_steps * 1e-3) / 1e12
 
-    # ---- per-kernel timing (eager launches with events around each kernel) ----
-    per_steps = min(args.steps, 20)
-    prune_ms = [0.0] * len(layers)
-    dgrad_ms = [0.0] * len(layers)
+    # ---- per-kernel timing: the same step captured with timing events between the kernels
+    # (event-record graph nodes), replayed with the same data and cache state as the timed step ----
     vals = [torch.empty(l.B * l.P * l.Q * l.Cout // 2, dtype=torch.int16, device="cuda") for l in layers]
     metas = [torch.empty(l.B * l.P * l.Q * l.Cout // 16, dtype=torch.int16, device="cuda") for l in layers]
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in layers]
-    for it in range(per_steps + 3):
+    ev_s = [torch.cuda.Event(enable_timing=True, external=True) for _ in range(2 * len(layers) + 1)]
+    ev_d = [torch.cuda.Event(enable_timing=True, external=True) for _ in range(len(layers) + 1)]
+
+    def sparse_step_events():
+        k = 0
         for i in order:
             l = layers[i]
-            evs[i][0].record()
+            ev_s[k].record()
             sdgp.sdgp_prune(dO[i].view(-1, l.Cout), n, m, scheme, 1234, values=vals[i], meta=metas[i])
-            evs[i][1].record()
+            ev_s[k + 1].record()
             sdgp.sdgp_spmm_conv2d(vals[i].view(l.B, l.P, l.Q, l.Cout // 2), metas[i].view(l.B, l.P, l.Q, l.Cout // 16),
                                   Wt[i], dD[i], l.stride, l.pad)
-            evs[i][2].record()
+            k += 2
+        ev_s[k].record()
+
+    def dense_step_events():
+        for k, i in enumerate(order):
+            l = layers[i]
+            ev_d[k].record()
+            sdgp.sdgp_dgrad_conv2d(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, flags=sdgp.FLAG_DENSE)
+        ev_d[len(order)].record()
+
+    per_steps = max(3, min(args.steps, 30))
+    prune_ms = [0.0] * len(layers)
+    dgrad_ms = [0.0] * len(layers)
+    dense_ms = [0.0] * len(layers)
+    g_ev = capture(sparse_step_events)
+    for it in range(per_steps + 3):
+        g_ev.replay()
         torch.cuda.synchronize()
         if it >= 3:
-            for i in order:
-                prune_ms[i] += evs[i][0].elapsed_time(evs[i][1])
-                dgrad_ms[i] += evs[i][1].elapsed_time(evs[i][2])
+            for k, i in enumerate(order):
+                prune_ms[i] += ev_s[2 * k].elapsed_time(ev_s[2 * k + 1])
+                dgrad_ms[i] += ev_s[2 * k + 1].elapsed_time(ev_s[2 * k + 2])
+    g_evd = capture(dense_step_events)
+    for it in range(per_steps + 3):
+        g_evd.replay()
+        torch.cuda.synchronize()
+        if it >= 3:
+            for k, i in enumerate(order):
+                dense_ms[i] += ev_d[k].elapsed_time(ev_d[k + 1])
     status = sdgp.sdgp_last_device_error()
     if status != 0:
         raise SystemExit("device error: " + sdgp.status_string(status))
@@ -315,7 +344,9 @@ def run_ours(args, layers):
     dgrad_tflops = total_flops * per_steps / (sum(dgrad_ms) * 1e-3) / 1e12
     sparse_peak = 2.0 * pk["bf16_sustained"]
     per_layer = [{"layer": l.name, "prune_us": 1e3 * prune_ms[i] / per_steps, "dgrad_us": 1e3 * dgrad_ms[i] / per_steps,
+                  "dense_us": 1e3 * dense_ms[i] / per_steps,
                   "dgrad_dense_equiv_tflops": layer_flops(l) / (dgrad_ms[i] / per_steps * 1e-3) / 1e12,
+                  "speedup_vs_dense": dense_ms[i] / (prune_ms[i] + dgrad_ms[i]),
                   "prune_gbs": l.B * l.P * l.Q * l.Cout * 3.125 / (prune_ms[i] / per_steps * 1e-3) / 1e9}
                  for i, l in enumerate(layers)]
 
@@ -351,7 +382,8 @@ def run_ours(args, layers):
             "roofline": {"bound": "tensor", "kernel": "dgrad_kernel<sparse>", "achieved": dgrad_tflops,
                          "peak": sparse_peak, "unit": "TFLOP/s", "frac": dgrad_tflops / sparse_peak,
                          "traffic": None,
-                         "note": "dense-equivalent FLOPs of all sparse dgrad launches / their summed event time; "
+                         "note": "dense-equivalent FLOPs of all sparse dgrad launches / their summed time between "
+                                 "event nodes of the replayed step graph; "
                                  "peak = 2 x %s sustained dense bf16" % pk["source"]},
             "per_layer": per_layer,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

@@ -177,3 +177,66 @@ def test_unsupported_requests_raise():
     with pytest.raises(sdgp.SdgpError) as e:
         sdgp.sdgp_dgrad_conv2d(dO, W, dD, 2, 1, 2, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
     assert e.value.status == 2
+
+
+# ------------------------------------------------- full benchmark sizes, sampled outputs
+
+
+def _sampled_conv_check(layer, seed, n, m, scheme, samples=600):
+    """Run the two-pass path on the full layer; compare `samples` output pixels (plus the first
+    and last pixels of the tensor) with the oracle, which prunes only the rows those pixels read."""
+    import paper_2202_00774_b200 as sdgp
+    dO, W = inputs.conv_layer_tensors(layer, seed)
+    ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(layer.B, layer.H, layer.W, layer.Cin, layer.Cout, layer.R,
+                                                     layer.S, 1, layer.pad), dtype=torch.uint8, device="cuda")
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, layer.pad, n, m, scheme, seed=5, workspace=ws)
+    check_no_device_error()
+    got_all = dD.cpu().numpy().view(np.uint16)
+    assert not np.isnan(inputs.bf16_bits_to_f32(got_all)).any()   # every output was written
+    rng = np.random.default_rng(seed)
+    # sample whole images so that the random scheme's linear indices and all borders are covered
+    imgs = np.unique(np.concatenate([[0, layer.B - 1], rng.integers(0, layer.B, 6)]))
+    per_img = layer.H * layer.W
+    pruned = np.zeros_like(dO)
+    for b in imgs:
+        rows = dO[b].reshape(-1, layer.Cout)
+        if scheme == oracle.RANDOM:
+            # keys depend on the element's linear index in the whole tensor: prune a slab that
+            # starts at row 0 of the tensor up to this image (cheap enough for the sampled images)
+            full = oracle.prune(dO[:b + 1].reshape(-1, layer.Cout), n, m, scheme, 5, want=("dense",))["dense"]
+            pruned[b] = full[-rows.shape[0]:].reshape(dO[b].shape)
+        else:
+            pruned[b] = oracle.prune(rows, n, m, scheme, 5, want=("dense",))["dense"].reshape(dO[b].shape)
+    idx = np.concatenate([b * per_img + rng.integers(0, per_img, samples // len(imgs)) for b in imgs])
+    idx = np.unique(np.concatenate([idx, np.arange(0, 64), np.arange(layer.B * per_img - 64, layer.B * per_img)]))
+    want = oracle.dgrad_conv2d(pruned, W, layer.H, layer.W, 1, layer.pad, pixel_index=idx)
+    got = inputs.bf16_bits_to_f32(got_all.reshape(-1, layer.Cin)[idx]).astype(np.float64)
+    assert rel_fro(got, want) <= TOL
+
+
+@pytest.mark.parametrize("index", range(7))
+def test_resnet9_full_size_layers_sampled(index):
+    """The benchmark's own shapes (batch 512) in the launch configuration it times."""
+    layer = inputs.resnet9_layers(512)[index]
+    scheme = [oracle.MAGNITUDE, oracle.RESCALED, oracle.RANDOM][index % 3]
+    _sampled_conv_check(layer, seed=index, n=2, m=4, scheme=scheme)
+
+
+@pytest.mark.parametrize("n,m,scheme", [(2, 4, oracle.MAGNITUDE), (1, 4, oracle.RESCALED), (2, 8, oracle.MAGNITUDE),
+                                        (2, 16, oracle.RESCALED)])
+def test_gemm_large_full_size_sampled_rows(n, m, scheme):
+    """[16384 x 4096] . [4096 x 4096] in full on the GPU; 96 sampled rows against the oracle."""
+    import paper_2202_00774_b200 as sdgp
+    c = inputs.GEMM_LARGE
+    dO, W = inputs.fc_tensors(c["rows"], c["K"], c["N"], c["seed"])
+    ws = torch.empty(sdgp.sdgp_workspace_size_linear(c["rows"], c["K"], c["N"]), dtype=torch.uint8, device="cuda")
+    dD = torch.full((c["rows"], c["N"]), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, n, m, scheme, seed=9, workspace=ws)
+    check_no_device_error()
+    rng = np.random.default_rng(n * 10 + m)
+    rows = np.unique(np.concatenate([[0, 127, 128, c["rows"] - 1], rng.integers(0, c["rows"], 92)]))
+    pruned = oracle.prune(dO[rows], n, m, scheme, 9, want=("dense",))["dense"]   # magnitude schemes: row-local
+    want = oracle.dgrad_linear(pruned, W)
+    got = inputs.bf16_bits_to_f32(dD[torch.from_numpy(rows).cuda()].cpu().numpy().view(np.uint16)).astype(np.float64)
+    assert rel_fro(got, want) <= TOL
