@@ -69,6 +69,7 @@ struct DgradParams {
   int stages;             // shared-memory pipeline depth
   int nacc;               // TMEM accumulators (2 = epilogue overlaps the next tile)
   int meta_col;           // first TMEM column of the metadata slots
+  int meta_shared;        // metadata slots live in the first columns of the accumulator NOT being written
   int w_resident;         // whole W half-slice kept in shared memory
   int out_bufs;           // epilogue staging slabs (1 or 2)
   // shared-memory carve (byte offsets from the 1024-aligned base) and per-stage sizes
@@ -125,7 +126,8 @@ __device__ __forceinline__ void rearrange_metadata_row(const uint8_t* raw_rows, 
 template <int BN>
 __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* staging, int out_bufs,
                                                   const CUtensorMap* tmD, int n0, int w0, int h0, int b0,
-                                                  bool tile_in_range, int row, bool issuer, uint32_t& chunk) {
+                                                  bool tile_in_range, int row, bool issuer, uint32_t& chunk,
+                                                  uint64_t* first_slab_read) {
 #pragma unroll 1
   for (int c0 = 0; c0 < BN; c0 += 64, ++chunk) {
     uint32_t packed[32];
@@ -139,6 +141,13 @@ __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* stagi
         const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
         packed[16 * part + e] = *(const uint32_t*)&h2;
       }
+    }
+    if (c0 == 0 && first_slab_read != nullptr) {
+      // the accumulator's first 64 columns are in registers: they may now hold the next
+      // tile's metadata
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if ((threadIdx.x & 31) == 0) ptx::mbar_arrive_cluster(first_slab_read, 0);
     }
     uint8_t* buf = staging + (out_bufs == 2 ? (chunk & 1u) : 0u) * kOutBytes;
     if (issuer) {  // the store that last used this slab has finished reading it
@@ -182,7 +191,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   uint64_t* acc_full = meta_ready + kMaxStages;
   uint64_t* acc_empty = acc_full + 2;
   uint64_t* w_full = acc_empty + 2;
-  uint32_t* tmem_slot = (uint32_t*)(w_full + 1);
+  uint64_t* meta_free = w_full + 1;
+  uint32_t* tmem_slot = (uint32_t*)(meta_free + 2);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -201,6 +211,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&acc_full[a], 1);
       ptx::mbar_init(&acc_empty[a], 8);
+      ptx::mbar_init(&meta_free[a], 8);
     }
     ptx::mbar_init(w_full, 1);
     ptx::fence_mbar_init();
@@ -296,9 +307,15 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const uint32_t sA_u = ptx::smem_u32(sA), sB_u = ptx::smem_u32(sB), sW_u = ptx::smem_u32(sW),
                      sE_u = ptx::smem_u32(sEhw);
       int st = 0, acc = 0;
-      uint32_t ph = 0, aph = 0;
-      for (int pt = first_pair; alive && pt < p.pair_tiles; pt += pair_stride) {
+      uint32_t ph = 0, aph = 0, lt = 0;
+      for (int pt = first_pair; alive && pt < p.pair_tiles; pt += pair_stride, ++lt) {
         if (!ptx::mbar_wait(&acc_empty[acc], aph ^ 1u, err, 0x200u + acc)) break;
+        // Shared metadata region: this tile's slots are the first columns of the other
+        // accumulator, which the epilogue of the previous tile must have read out first.
+        if (p.meta_shared && lt > 0 &&
+            !ptx::mbar_wait(&meta_free[acc ^ 1], ((lt - 1u) >> 1) & 1u, err, 0x800u + acc))
+          break;
+        const int meta_base = p.meta_shared ? (acc ^ 1) * BN : p.meta_col;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         uint32_t accumulate = 0u;
@@ -308,7 +325,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             if (!ptx::mbar_wait(&full[st], ph, err, 0x300u + st)) { alive = false; break; }
             if (SPARSE && !ptx::mbar_wait(&meta_ready[st], ph, err, 0x400u + st)) { alive = false; break; }
             ptx::tc_fence_after_sync();
-            const uint32_t meta_slot = (uint32_t)(p.meta_col + st * p.rr * 4);
+            const uint32_t meta_slot = (uint32_t)(meta_base + st * p.rr * 4);
             if (SPARSE) {
               for (int u = 0; u < p.rr; ++u)
                 ptx::tc_cp_128x128b_pair(tmem_base + meta_slot + 4u * u,
@@ -385,7 +402,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       if (!ptx::mbar_wait(&acc_full[acc], aph, err, 0x600u + acc)) break;
       ptx::tc_fence_after_sync();
       store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), sOut, p.out_bufs, &tmD,
-                            nt * BN, wt * p.TW, ht * p.TH, bt * p.TB, mt < p.m_tiles, row, issuer, chunk);
+                            nt * BN, wt * p.TW, ht * p.TH, bt * p.TB, mt < p.m_tiles, row, issuer, chunk,
+                            p.meta_shared ? &meta_free[acc] : nullptr);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
@@ -512,15 +530,23 @@ bool plan(DgradParams* p) {
     if (stages > kMaxStages) stages = kMaxStages;
     // TMEM: accumulators first, metadata slots (4 columns per tap and stage) behind them
     const int meta_cols_per_stage = SPARSE ? 4 * p->rr : 0;
+    const int meta_div = SPARSE ? meta_cols_per_stage : 1;  // divisor that is never zero
     int nacc = (2 * BN + 2 * meta_cols_per_stage <= (int)kTmemCols) ? 2 : 1;
-    if (meta_cols_per_stage > 0) {
-      const int max_meta_stages = ((int)kTmemCols - nacc * BN) / meta_cols_per_stage;
+    p->meta_shared = 0;
+    if (meta_cols_per_stage > 0 && nacc == 1 && 2 * BN <= (int)kTmemCols) {
+      // Two accumulators fill TMEM: the metadata slots share the first 64 columns of whichever
+      // accumulator is being read out, released early by the epilogue.
+      nacc = 2;
+      p->meta_shared = 1;
+      if (stages > 64 / meta_div) stages = 64 / meta_div;
+    } else if (meta_cols_per_stage > 0) {
+      const int max_meta_stages = ((int)kTmemCols - nacc * BN) / meta_div;
       if (stages > max_meta_stages) stages = max_meta_stages;
     }
     if (stages < ((resident || reuse) ? 2 : 3)) continue;  // a reuse stage is R taps long
     p->stages = stages;
     p->nacc = nacc;
-    p->meta_col = nacc * BN;
+    p->meta_col = p->meta_shared ? 0 : nacc * BN;
     p->out_bufs = out_bufs;
     p->off_b = stages * p->a_bytes;
     p->off_eraw = p->off_b + stages * p->b_bytes;

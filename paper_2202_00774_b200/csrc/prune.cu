@@ -6,6 +6,8 @@
 // The kernel is a pure stream: 2 B read per element, 1 B of compressed values, 1/8 B of
 // position metadata (+ 1/8 B mask, + 2 B dense copy when asked for), every output indexed by
 // the same 8-element vector number so all stores coalesce.
+#include <cuda_bf16.h>
+
 #include "sdgp_internal.cuh"
 
 namespace sdgp {
@@ -214,6 +216,64 @@ __host__ __device__ constexpr int threshold_lut(bool na, bool nb, bool nc) {
   return lut;
 }
 
+
+// Survivors of both lanes times their group's scale, rounded to bf16 (nearest even). When both
+// group sums are finite every product is finite and the hardware's packed conversion applies;
+// otherwise (Inf or NaN in the group) each value goes through the explicit rounding, which
+// stores any NaN as 0x7FC0.
+__device__ __forceinline__ void rescale_packed(uint32_t& y0, uint32_t& y1, uint32_t& y2, uint32_t& y3, uint32_t km0,
+                                               uint32_t km1, uint32_t km2, uint32_t km3, float scA, float scB,
+                                               float tA, float tB) {
+  const bool finite = (__float_as_uint(tA) & 0x7F800000u) != 0x7F800000u &&
+                      (__float_as_uint(tB) & 0x7F800000u) != 0x7F800000u;
+  if (finite) {
+#define SDGP_RESCALE_FAST(y, km)                                                                    \
+  {                                                                                                 \
+    const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(__uint_as_float(y << 16), scA),        \
+                                                   __fmul_rn(__uint_as_float(y & 0xFFFF0000u), scB)); \
+    y = (*(const uint32_t*)&h) & km;                                                                \
+  }
+    SDGP_RESCALE_FAST(y0, km0) SDGP_RESCALE_FAST(y1, km1) SDGP_RESCALE_FAST(y2, km2) SDGP_RESCALE_FAST(y3, km3)
+#undef SDGP_RESCALE_FAST
+  } else {
+#define SDGP_RESCALE_SLOW(y, km)                                                                    \
+  y = (f32_to_bf16_bits(__fmul_rn(__uint_as_float(y << 16), scA)) |                                 \
+       (f32_to_bf16_bits(__fmul_rn(__uint_as_float(y & 0xFFFF0000u), scB)) << 16)) & km;
+    SDGP_RESCALE_SLOW(y0, km0) SDGP_RESCALE_SLOW(y1, km1) SDGP_RESCALE_SLOW(y2, km2) SDGP_RESCALE_SLOW(y3, km3)
+#undef SDGP_RESCALE_SLOW
+  }
+}
+
+// Writes one vector's outputs from the lane-paired form: y_i = (element i, element i + 4) after
+// pruning, km_i = 0xFFFF in the lanes of kept elements. COMPRESS: every 4-chunk holds at most two
+// survivors, so values / meta can be produced.
+template <bool COMPRESS>
+__device__ __forceinline__ void emit_packed(int64_t v, uint32_t y0, uint32_t y1, uint32_t y2, uint32_t y3,
+                                            uint32_t km0, uint32_t km1, uint32_t km2, uint32_t km3,
+                                            uint4* __restrict__ dense, uint2* __restrict__ values,
+                                            uint8_t* __restrict__ meta, uint8_t* __restrict__ mask) {
+  if (dense)
+    dense[v] = make_uint4(prmt(y0, y1, 0x5410), prmt(y2, y3, 0x5410), prmt(y0, y1, 0x7632), prmt(y2, y3, 0x7632));
+  if (mask) {
+    const uint32_t t = (km0 & 0x00010001u) | (km1 & 0x00020002u) | (km2 & 0x00040004u) | (km3 & 0x00080008u);
+    mask[v] = (uint8_t)((t & 0xFu) | (t >> 12));
+  }
+  if (COMPRESS && (values || meta)) {
+    // At most two survivors per chunk. Positions: p1 = last survivor, but at least 1;
+    // p0 = first survivor if there are two, else 0 (the pad takes the lowest free position).
+    const uint32_t k23 = km2 | km3;
+    const uint32_t slot0 = y0 | (y1 & k23) | (y2 & km3);
+    const uint32_t slot1 = y3 | (~km3 & (y2 | (~km2 & y1)));
+    if (values) values[v] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
+    if (meta) {
+      const uint32_t pos0 = (km1 & k23 & 0x00010001u) | (km2 & km3 & 0x00020002u);
+      const uint32_t pos1 = 0x00010001u + (k23 & 0x00010001u) + (km3 & 0x00010001u);
+      const uint32_t nib = pos0 + 4u * pos1;
+      meta[v] = (uint8_t)((nib & 0xFu) | (nib >> 12));
+    }
+  }
+}
+
 template <int N, int SCHEME>
 __global__ void __launch_bounds__(kThreads)
 prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
@@ -289,34 +349,10 @@ prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, ui
                                  __fadd_rn(__uint_as_float(y2 & 0x7FFF0000u), __uint_as_float(y3 & 0x7FFF0000u)));
       const float scA = (sA == 0.0f) ? 1.0f : __fdiv_rn(tA, sA);
       const float scB = (sB == 0.0f) ? 1.0f : __fdiv_rn(tB, sB);
-#define SDGP_RESCALE(y, km)                                                                        \
-  y = (f32_to_bf16_bits(__fmul_rn(__uint_as_float(y << 16), scA)) |                                \
-       (f32_to_bf16_bits(__fmul_rn(__uint_as_float(y & 0xFFFF0000u), scB)) << 16)) & km;
-      SDGP_RESCALE(y0, km0) SDGP_RESCALE(y1, km1) SDGP_RESCALE(y2, km2) SDGP_RESCALE(y3, km3)
-#undef SDGP_RESCALE
+      rescale_packed(y0, y1, y2, y3, km0, km1, km2, km3, scA, scB, tA, tB);
     }
 
-    if (dense)
-      dense[v] = make_uint4(prmt(y0, y1, 0x5410), prmt(y2, y3, 0x5410),
-                            prmt(y0, y1, 0x7632), prmt(y2, y3, 0x7632));
-    if (mask) {
-      const uint32_t t = (km0 & 0x00010001u) | (km1 & 0x00020002u) | (km2 & 0x00040004u) | (km3 & 0x00080008u);
-      mask[v] = (uint8_t)((t & 0xFu) | (t >> 12));
-    }
-    if (N <= 2 && (values || meta)) {
-      // At most two survivors per chunk. Positions: p1 = last survivor, but at least 1;
-      // p0 = first survivor if there are two, else 0 (the pad takes the lowest free position).
-      const uint32_t k23 = km2 | km3;
-      const uint32_t slot0 = y0 | (y1 & k23) | (y2 & km3);
-      const uint32_t slot1 = y3 | (~km3 & (y2 | (~km2 & y1)));
-      if (values) values[v] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
-      if (meta) {
-        const uint32_t pos0 = (km1 & k23 & 0x00010001u) | (km2 & km3 & 0x00020002u);
-        const uint32_t pos1 = 0x00010001u + (k23 & 0x00010001u) + (km3 & 0x00010001u);
-        const uint32_t nib = pos0 + 4u * pos1;
-        meta[v] = (uint8_t)((nib & 0xFu) | (nib >> 12));
-      }
-    }
+    emit_packed<(N <= 2)>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask);
   }
 }
 
@@ -338,6 +374,119 @@ cudaError_t launch_m4_n(int scheme, const void* dO, int64_t nvec, uint64_t seed,
     default: SDGP_LAUNCH4(SDGP_RESCALED_MAGNITUDE); break;
   }
 #undef SDGP_LAUNCH4
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Groups of 8, 16 or 32 with n <= 2: the survivors are the elements whose composite key
+// (rank key << 5 | 31 - position, unique inside a group) reaches the group's n-th largest key.
+// Each thread finds the two largest keys of its 8 elements with a max/min network, groups that
+// span 2 or 4 lanes merge their pairs through xor-shuffles, and the outputs are written from the
+// same lane-paired form as the m = 4 path.
+
+__device__ __forceinline__ void merge_top2(uint32_t& hi, uint32_t& lo, uint32_t hi2, uint32_t lo2) {
+  const uint32_t h = max(hi, hi2);
+  lo = max(min(hi, hi2), max(lo, lo2));
+  hi = h;
+}
+
+template <int M, int N, int SCHEME>
+__global__ void __launch_bounds__(kThreads)
+prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
+                  uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
+                  uint8_t* __restrict__ mask) {
+  constexpr int LANES = M / 8;
+  static_assert(N == 1 || N == 2, "threshold selection keeps one or two elements");
+  const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
+  const uint32_t pos0 = 31u - 8u * (uint32_t)(threadIdx.x & (LANES - 1));  // tie-break bits of element 0
+  uint4 in[kVecPerThread];
+#pragma unroll
+  for (int it = 0; it < kVecPerThread; ++it) {
+    const int64_t v = base + (int64_t)it * kThreads;
+    in[it] = (v < nvec) ? __ldg(dO + v) : make_uint4(0, 0, 0, 0);
+  }
+#pragma unroll
+  for (int it = 0; it < kVecPerThread; ++it) {
+    const int64_t v = base + (int64_t)it * kThreads;
+    const uint4 w = in[it];
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+    uint32_t c[8];
+    if (SCHEME == SDGP_RANDOM) {
+      const uint4 o = philox4x32_10((uint32_t)v, (uint32_t)((uint64_t)v >> 32), 0u, 0u, seed_lo, seed_hi);
+      const uint32_t r[4] = {~o.x, ~o.y, ~o.z, ~o.w};  // smallest random key ranks first
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        c[i] = (((i & 1) ? (r[i >> 1] >> 11) : (r[i >> 1] << 5)) & 0x1FFFE0u) | (pos0 - i);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        c[i] = (((i & 1) ? (ww[i >> 1] >> 11) : (ww[i >> 1] << 5)) & 0xFFFE0u) | (pos0 - i);  // |x| << 5 | tie-break
+    }
+    uint32_t hi, lo = 0;
+    if (N == 1) {
+      hi = max(max(max(c[0], c[1]), max(c[2], c[3])), max(max(c[4], c[5]), max(c[6], c[7])));
+#pragma unroll
+      for (int d = 1; d < LANES; d <<= 1) hi = max(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, d));
+    } else {
+      uint32_t h1 = max(c[2], c[3]), l1 = min(c[2], c[3]), h2 = max(c[4], c[5]), l2 = min(c[4], c[5]),
+               h3 = max(c[6], c[7]), l3 = min(c[6], c[7]);
+      hi = max(c[0], c[1]);
+      lo = min(c[0], c[1]);
+      merge_top2(hi, lo, h1, l1);
+      merge_top2(h2, l2, h3, l3);
+      merge_top2(hi, lo, h2, l2);
+#pragma unroll
+      for (int d = 1; d < LANES; d <<= 1) {
+        const uint32_t oh = __shfl_xor_sync(0xFFFFFFFFu, hi, d), ol = __shfl_xor_sync(0xFFFFFFFFu, lo, d);
+        merge_top2(hi, lo, oh, ol);
+      }
+    }
+    const uint32_t t1 = ((N == 1) ? hi : lo) - 1u;  // keep <=> key > t1; (t1 - key) is then negative
+    const uint32_t p0 = prmt(w.x, w.z, 0x5410), p1 = prmt(w.x, w.z, 0x7632);
+    const uint32_t p2 = prmt(w.y, w.w, 0x5410), p3 = prmt(w.y, w.w, 0x7632);
+    const uint32_t km0 = prmt(t1 - c[0], t1 - c[4], 0xFFBB), km1 = prmt(t1 - c[1], t1 - c[5], 0xFFBB);
+    const uint32_t km2 = prmt(t1 - c[2], t1 - c[6], 0xFFBB), km3 = prmt(t1 - c[3], t1 - c[7], 0xFFBB);
+    uint32_t y0 = p0 & km0, y1 = p1 & km1, y2 = p2 & km2, y3 = p3 & km3;
+    if (SCHEME == SDGP_RESCALED_MAGNITUDE) {
+      // balanced pairwise sums in index order: elements 0..3 are the low lanes, 4..7 the high lanes
+#define SDGP_SUM8(q0, q1, q2, q3)                                                                                 \
+  __fadd_rn(__fadd_rn(__fadd_rn(__uint_as_float((q0 << 16) & 0x7FFF0000u), __uint_as_float((q1 << 16) & 0x7FFF0000u)), \
+                      __fadd_rn(__uint_as_float((q2 << 16) & 0x7FFF0000u), __uint_as_float((q3 << 16) & 0x7FFF0000u))), \
+            __fadd_rn(__fadd_rn(__uint_as_float(q0 & 0x7FFF0000u), __uint_as_float(q1 & 0x7FFF0000u)),             \
+                      __fadd_rn(__uint_as_float(q2 & 0x7FFF0000u), __uint_as_float(q3 & 0x7FFF0000u))))
+      float tsum = SDGP_SUM8(p0, p1, p2, p3);
+      float ssum = SDGP_SUM8(y0, y1, y2, y3);
+#undef SDGP_SUM8
+#pragma unroll
+      for (int d = 1; d < LANES; d <<= 1) {
+        tsum = __fadd_rn(tsum, __shfl_xor_sync(0xFFFFFFFFu, tsum, d));
+        ssum = __fadd_rn(ssum, __shfl_xor_sync(0xFFFFFFFFu, ssum, d));
+      }
+      const float sc = (ssum == 0.0f) ? 1.0f : __fdiv_rn(tsum, ssum);
+      rescale_packed(y0, y1, y2, y3, km0, km1, km2, km3, sc, sc, tsum, tsum);
+    }
+    if (v < nvec) emit_packed<true>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask);
+  }
+}
+
+template <int M, int N>
+cudaError_t launch_top2(int scheme, const void* dO, int64_t nvec, uint64_t seed, void* dense, void* values,
+                        void* meta, void* mask, cudaStream_t stream) {
+  const int64_t per_block = (int64_t)kThreads * kVecPerThread;
+  const int64_t blocks = (nvec + per_block - 1) / per_block;
+  if (blocks == 0) return cudaSuccess;
+  if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
+  const dim3 grid((unsigned)blocks), block(kThreads);
+  const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
+#define SDGP_LAUNCH_T2(S)                                                                            \
+  prune_top2_kernel<M, N, S><<<grid, block, 0, stream>>>((const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
+                                                         (uint2*)values, (uint8_t*)meta, (uint8_t*)mask)
+  switch (scheme) {
+    case SDGP_RANDOM: SDGP_LAUNCH_T2(SDGP_RANDOM); break;
+    case SDGP_MAGNITUDE: SDGP_LAUNCH_T2(SDGP_MAGNITUDE); break;
+    default: SDGP_LAUNCH_T2(SDGP_RESCALED_MAGNITUDE); break;
+  }
+#undef SDGP_LAUNCH_T2
   return cudaGetLastError();
 }
 
@@ -376,9 +525,15 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
         case 3: return launch_m4_n<3>(scheme, dO, nvec, seed, dense, values, meta, mask, stream);
         default: return launch_m4_n<4>(scheme, dO, nvec, seed, dense, values, meta, mask, stream);
       }
-    case 8: return launch_m<8>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
-    case 16: return launch_m<16>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
-    case 32: return launch_m<32>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
+#define SDGP_M_CASE(M)                                                                              \
+  case M:                                                                                           \
+    if (n == 1) return launch_top2<M, 1>(scheme, dO, nvec, seed, dense, values, meta, mask, stream); \
+    if (n == 2) return launch_top2<M, 2>(scheme, dO, nvec, seed, dense, values, meta, mask, stream); \
+    return launch_m<M>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
+    SDGP_M_CASE(8)
+    SDGP_M_CASE(16)
+    SDGP_M_CASE(32)
+#undef SDGP_M_CASE
     default: return cudaErrorInvalidValue;
   }
 }
