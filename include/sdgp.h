@@ -90,7 +90,8 @@ sdgp_status sdgp_prune(const void* dO, int64_t rows, int64_t K, int n, int m, sd
  *   dO [rows, K] bf16, W [K, N] bf16 (output channels x input channels), dD [rows, N] bf16,
  *   fp32 accumulation, round-to-nearest-even bf16 result.
  * Requirements: K % 64 == 0, N % 64 == 0 (any rows >= 0); pruned modes need n <= 2, m in {4,8,16,32}
- * dividing K. Workspace: sdgp_workspace_size_linear() bytes, 256-byte aligned. */
+ * dividing K (or n == m, which prunes nothing). Workspace: sdgp_workspace_size_linear() bytes,
+ * 256-byte aligned (the compressed rows are padded to whole blocks of 128 channels). */
 sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,
                               int64_t N, int n, int m, sdgp_scheme scheme, uint64_t seed,
                               void* workspace, size_t workspace_bytes, uint32_t flags, void* stream);
@@ -101,15 +102,16 @@ sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t r
  *                  q*stride - pad + s == w of prune(dO)[b,p,q,co] * W[co,r,s,ci].
  *   dO [B,P,Q,Cout] with P = (H + 2*pad - R)/stride + 1, Q likewise; W [Cout,R,S,Cin];
  *   dD [B,H,Wd,Cin]. Groups of m run along Cout at a fixed (b,p,q).
- * Requirements: stride == 1 (other strides: SDGP_ERR_UNSUPPORTED), Cout % 64 == 0, Cin % 64 == 0,
- * pad <= R-1 and pad <= S-1. Workspace: sdgp_workspace_size_conv2d() bytes. */
+ * Requirements: stride 1 or 2 (other strides: SDGP_ERR_UNSUPPORTED), Cout % 64 == 0, Cin % 64 == 0,
+ * pad <= R-1 and pad <= S-1. Workspace: sdgp_workspace_size_conv2d() bytes, 256-byte aligned. */
 sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, int H, int Wd, int Cin,
                               int Cout, int R, int S, int stride, int pad, int n, int m,
                               sdgp_scheme scheme, uint64_t seed, void* workspace,
                               size_t workspace_bytes, uint32_t flags, void* stream);
 
 /* The contraction alone, from an already compressed dL/dO (output of sdgp_prune):
- * values [rows, K/2] bf16 and meta [rows, K/16] u16 in place of dO. No workspace. */
+ * values [rows, K/2] bf16 and meta [rows, K/16] u16 in place of dO. No workspace. Needs
+ * K % 128 == 0 (Cout % 128 == 0 for the convolution), N % 64 == 0, stride 1 or 2. */
 sdgp_status sdgp_spmm_linear(const void* values, const void* meta, const void* W, void* dD,
                              int64_t rows, int64_t K, int64_t N, void* stream);
 sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W, void* dD, int B,

@@ -7,6 +7,10 @@ bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// The sparse contraction works on whole blocks of 128 channels; the compressed workspace rows are
+// padded up to that.
+int64_t pad128(int64_t k) { return (k + 127) / 128 * 128; }
+
 sdgp_status check_prune_args(int64_t rows, int64_t K, int n, int m, int scheme) {
   if (rows < 0 || K < 0) return SDGP_ERR_INVALID_ARG;
   if (scheme < 0 || scheme > 2) return SDGP_ERR_INVALID_ARG;
@@ -69,7 +73,7 @@ sdgp_status sdgp_prune(const void* dO, int64_t rows, int64_t K, int n, int m, sd
 size_t sdgp_workspace_size_linear(int64_t rows, int64_t K, int64_t N, uint32_t flags) {
   (void)N;
   if (flags != SDGP_FLAG_TWO_PASS || rows <= 0 || K <= 0) return 0;
-  return carve_compressed(nullptr, rows * K).bytes;
+  return carve_compressed(nullptr, rows * pad128(K)).bytes;
 }
 
 size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R, int S, int stride,
@@ -78,7 +82,7 @@ size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R
   if (flags != SDGP_FLAG_TWO_PASS || stride < 1) return 0;
   const int64_t P = (H + 2 * pad - R) / stride + 1, Q = (Wd + 2 * pad - S) / stride + 1;
   if (B <= 0 || P <= 0 || Q <= 0 || Cout <= 0) return 0;
-  return carve_compressed(nullptr, (int64_t)B * P * Q * Cout).bytes;
+  return carve_compressed(nullptr, (int64_t)B * P * Q * pad128(Cout)).bytes;
 }
 
 sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W, void* dD, int B,
@@ -86,12 +90,13 @@ sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W
                              void* stream) {
   if (B < 0 || H < 0 || Wd < 0 || Cin < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0)
     return SDGP_ERR_INVALID_ARG;
-  if (stride != 1) return SDGP_ERR_UNSUPPORTED;
+  if (stride > 2) return SDGP_ERR_UNSUPPORTED;
   if (pad > R - 1 || pad > S - 1) return SDGP_ERR_UNSUPPORTED;
+  if (Cout % 128 != 0) return SDGP_ERR_UNSUPPORTED;  // caller-supplied compressed rows are not padded
   if ((int64_t)B * H * Wd == 0) return SDGP_OK;
   if (!values || !meta || !W || !dD) return SDGP_ERR_INVALID_ARG;
   if (!aligned16(values) || !aligned16(meta) || !aligned16(W) || !aligned16(dD)) return SDGP_ERR_ALIGNMENT;
-  return sdgp::launch_dgrad(true, values, meta, W, dD, B, H, Wd, Cin, Cout, R, S, pad, (cudaStream_t)stream);
+  return sdgp::launch_dgrad(true, values, meta, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, (cudaStream_t)stream);
 }
 
 sdgp_status sdgp_spmm_linear(const void* values, const void* meta, const void* W, void* dD,
@@ -108,7 +113,7 @@ sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, in
   if (B < 0 || H < 0 || Wd < 0 || Cin < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0)
     return SDGP_ERR_INVALID_ARG;
   if (flags > SDGP_FLAG_DENSE) return SDGP_ERR_INVALID_ARG;
-  if (stride != 1) return SDGP_ERR_UNSUPPORTED;
+  if (stride > 2) return SDGP_ERR_UNSUPPORTED;
   if (pad > R - 1 || pad > S - 1) return SDGP_ERR_UNSUPPORTED;
   if (flags != SDGP_FLAG_DENSE) {
     sdgp_status st = check_prune_args(0, Cout, n, m, (int)scheme);
@@ -116,22 +121,23 @@ sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, in
     if (n > 2 && n != m) return SDGP_ERR_UNSUPPORTED;
   }
   if ((int64_t)B * H * Wd == 0) return SDGP_OK;
-  const int64_t P = H + 2 * pad - R + 1, Q = Wd + 2 * pad - S + 1;
+  const int64_t P = (H + 2 * pad - R) / stride + 1, Q = (Wd + 2 * pad - S) / stride + 1;
   if (P < 1 || Q < 1) return SDGP_ERR_INVALID_ARG;
   if (!dO || !W || !dD) return SDGP_ERR_INVALID_ARG;
   if (!aligned16(dO) || !aligned16(W) || !aligned16(dD)) return SDGP_ERR_ALIGNMENT;
   cudaStream_t s = (cudaStream_t)stream;
   if (flags == SDGP_FLAG_DENSE || n == m)
-    return sdgp::launch_dgrad(false, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, pad, s);
+    return sdgp::launch_dgrad(false, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s);
   if (flags == SDGP_FLAG_FUSED) return SDGP_ERR_UNSUPPORTED;
-  if (Cin % 64 != 0 || Cout % 128 != 0) return SDGP_ERR_UNSUPPORTED;
-  const Carve c = carve_compressed(workspace, (int64_t)B * P * Q * Cout);
+  if (Cin % 64 != 0 || Cout % 64 != 0) return SDGP_ERR_UNSUPPORTED;
+  const int64_t Cpad = pad128(Cout);
+  const Carve c = carve_compressed(workspace, (int64_t)B * P * Q * Cpad);
   if (!workspace || workspace_bytes < c.bytes) return SDGP_ERR_WORKSPACE;
   if (((uintptr_t)workspace & 255u) != 0) return SDGP_ERR_ALIGNMENT;
   cudaError_t e = sdgp::launch_prune(dO, (int64_t)B * P * Q, Cout, n, m, (int)scheme, seed, nullptr, c.values,
-                                     c.meta, nullptr, s);
+                                     c.meta, nullptr, s, Cpad);
   if (e != cudaSuccess) return SDGP_ERR_CUDA;
-  return sdgp::launch_dgrad(true, c.values, c.meta, W, dD, B, H, Wd, Cin, Cout, R, S, pad, s);
+  return sdgp::launch_dgrad(true, c.values, c.meta, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s);
 }
 
 sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,

@@ -58,7 +58,9 @@ constexpr int kMaxStages = 8;
 struct DgradParams {
   int B, H, W;            // dD pixel grid (fully connected: B = H = 1, W = rows)
   int Cin, Cout;
-  int R, S, pad;
+  int R, S;               // filter taps of this launch (stride 2: the taps of one output-parity class)
+  int pad_h, pad_w;       // dO pixel of output pixel (h,w) under tap (r,s): (h + pad_h - r, w + pad_w - s)
+  int r_first, r_step, s_first, s_step, S_full;  // tap (r,s) of the launch is filter tap (r_first + r_step*r, s_first + s_step*s)
   int TW, TH, TB;         // pixel patch of one CTA tile, TW * TH * TB <= 128
   int tiles_w, tiles_h, tiles_b, tiles_n;
   int m_tiles;            // tiles_w * tiles_h * tiles_b
@@ -234,6 +236,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   const int rows_used = p.TW * p.TH * p.TB;
   const int taps = p.R * p.S;
   const bool reuse = (p.rr == p.R) && p.R > 1;
+  auto filter_tap = [&p](int r, int s) { return (p.r_first + p.r_step * r) * p.S_full + p.s_first + p.s_step * s; };
   const int groups = reuse ? p.S : taps;  // stage uses per channel block and tile
   const int uses_per_tile = groups * p.k_blocks;
   const int pair_stride = gridDim.x >> 1;
@@ -247,12 +250,14 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       if (p.w_resident) {
         // the layer's whole W half-slice, once: [tap][channel block][box] tiles of kKB rows
         if (rank == 0) ptx::mbar_arrive_expect_tx(w_full, 2u * (uint32_t)(taps * p.k_blocks * C::kTapBBytes));
-        for (int t = 0; t < taps; ++t)
+        for (int t = 0; t < taps; ++t) {
+          const int ft = filter_tap(t / p.S, t % p.S);
           for (int cb = 0; cb < p.k_blocks; ++cb)
 #pragma unroll
             for (int j = 0; j < C::kBoxes; ++j)
               ptx::tma_load_2d_pair(sW + ((t * p.k_blocks + cb) * C::kBoxes + j) * C::kBoxBytes, &tmB, w_full,
-                                    t * p.Cin + n_half + C::kBoxCols * j, cb * C::kKB);
+                                    ft * p.Cin + n_half + C::kBoxCols * j, cb * C::kKB);
+        }
       }
       const uint32_t pair_tx = 2u * (uint32_t)(p.img_rows * 128 + (p.w_resident ? 0 : p.rr * C::kTapBBytes));
       const uint32_t meta_tx = (uint32_t)(p.img_rows * 16);
@@ -270,7 +275,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // the last vertical tap needs; otherwise a group is the single tap (r, s).
         int r = reuse ? (p.R - 1) : 0, s = 0;
         for (int g = 0; alive && g < groups; ++g) {
-          const int q0 = w0 + p.pad - s, p0 = h0 + p.pad - r;
+          const int q0 = w0 + p.pad_w - s, p0 = h0 + p.pad_h - r;
           for (int cb = 0; cb < p.k_blocks; ++cb) {
             if (!ptx::mbar_wait(&empty[st], ph ^ 1u, err, 0x100u + st)) { alive = false; break; }
             if (rank == 0) ptx::mbar_arrive_expect_tx(&full[st], pair_tx);
@@ -281,7 +286,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             ptx::tma_load_4d_pair(sA + st * p.a_bytes, &tmA, &full[st], cb * 64, q0, p0, b0);
             if (!p.w_resident) {
               for (int u = 0; u < p.rr; ++u) {
-                const int tap = (reuse ? u : r) * p.S + s;
+                const int tap = filter_tap(reuse ? u : r, s);
 #pragma unroll
                 for (int j = 0; j < C::kBoxes; ++j)
                   ptx::tma_load_2d_pair(sB + st * p.b_bytes + (u * C::kBoxes + j) * C::kBoxBytes, &tmB, &full[st],
@@ -561,25 +566,37 @@ bool plan(DgradParams* p) {
   return false;
 }
 
+// Where one launch reads and writes: dO as stored (P x Q pixels of `a_channels` channels per image,
+// a multiple of the channel block; W holds only the first `Cout` of them), the full filter
+// width in W columns, and the (possibly strided) view of dD the launch fills.
+struct DgradView {
+  int P, Q, batch;
+  int a_channels;
+  int64_t w_cols;                 // R_full * S_full * Cin
+  void* d_base;
+  uint64_t d_stride_w, d_stride_h, d_stride_b;  // bytes
+};
+
 template <bool SPARSE, int BN>
-sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, void* dD, DgradParams p, int P, int Q,
+sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const DgradView& view, DgradParams p,
                        cudaStream_t stream) {
+  const int P = view.P, Q = view.Q;
   using C = Cfg<SPARSE, BN>;
   if (!plan<SPARSE, BN>(&p)) return SDGP_ERR_UNSUPPORTED;
 
   CUtensorMap tmA, tmE, tmB, tmD;
   const uint32_t img_h = (uint32_t)(p.TH + p.rr - 1);
-  const uint64_t CA = SPARSE ? (uint64_t)p.Cout / 2 : (uint64_t)p.Cout;  // stored elements per pixel
+  const uint64_t CA = SPARSE ? (uint64_t)view.a_channels / 2 : (uint64_t)view.a_channels;  // stored elements per pixel
   {
-    const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)P, (uint64_t)p.B};
+    const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
     const uint64_t strides[3] = {CA * 2, CA * 2 * Q, CA * 2 * Q * P};
     const uint32_t box[4] = {64, (uint32_t)p.TW, img_h, (uint32_t)p.TB};
     if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
   }
   if (SPARSE) {
-    const uint64_t CE = (uint64_t)p.Cout / 16;
-    const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)P, (uint64_t)p.B};
+    const uint64_t CE = (uint64_t)view.a_channels / 16;
+    const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
     const uint64_t strides[3] = {CE * 2, CE * 2 * Q, CE * 2 * Q * P};
     const uint32_t box[4] = {8, (uint32_t)p.TW, img_h, (uint32_t)p.TB};
     if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
@@ -588,8 +605,8 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, void* dD
     tmE = tmA;
   }
   {
-    const uint64_t dims[2] = {(uint64_t)p.R * p.S * p.Cin, (uint64_t)p.Cout};
-    const uint64_t strides[1] = {(uint64_t)p.R * p.S * p.Cin * 2};
+    const uint64_t dims[2] = {(uint64_t)view.w_cols, (uint64_t)p.Cout};
+    const uint64_t strides[1] = {(uint64_t)view.w_cols * 2};
     const uint32_t box[2] = {(uint32_t)C::kBoxCols, (uint32_t)C::kKB};
     if (!encode(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Wt, dims, strides, box,
                 C::kRowB == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
@@ -597,9 +614,9 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, void* dD
   }
   {
     const uint64_t dims[4] = {(uint64_t)p.Cin, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.B};
-    const uint64_t strides[3] = {(uint64_t)p.Cin * 2, (uint64_t)p.Cin * 2 * p.W, (uint64_t)p.Cin * 2 * p.W * p.H};
+    const uint64_t strides[3] = {view.d_stride_w, view.d_stride_h, view.d_stride_b};
     const uint32_t box[4] = {64, (uint32_t)p.TW, (uint32_t)p.TH, (uint32_t)p.TB};
-    if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, dD, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+    if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, view.d_base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
   }
 
@@ -629,40 +646,77 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, void* dD
 
 }  // namespace
 
-// A: dense dL/dO [B,P,Q,Cout] (sparse == false) or compressed values [B,P,Q,Cout/2] with
-// meta [B,P,Q,Cout/16]; Wt: [Cout, R, S, Cin]; dD: [B,H,W,Cin]. Stride 1.
+// A: dense dL/dO [B,P,Q,Cout] (sparse == false) or compressed values [B,P,Q,a_channels/2] with
+// meta [B,P,Q,a_channels/16], a_channels = Cout rounded up to 128 (pad channels hold zero values
+// and the position pair (0,1)); Wt: [Cout, R, S, Cin]; dD: [B,H,W,Cin].
+// Stride 2 is split by the parity of the output pixel: pixel (2h'+ph, 2w'+pw) only meets the taps
+// r = ph + pad (mod 2), s = pw + pad (mod 2), and on those it is a stride-1 problem from dO to
+// the strided view dD[:, ph::2, pw::2, :].
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
-                         int H, int W, int Cin, int Cout, int R, int S, int pad, cudaStream_t stream) {
-  const int P = H + 2 * pad - R + 1, Q = W + 2 * pad - S + 1;
+                         int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream) {
+  if (stride != 1 && stride != 2) return SDGP_ERR_UNSUPPORTED;
+  const int P = (H + 2 * pad - R) / stride + 1, Q = (W + 2 * pad - S) / stride + 1;
   if (P < 1 || Q < 1) return SDGP_ERR_INVALID_ARG;
   if ((int64_t)B * H * W == 0) return SDGP_OK;
-  if (Cin % 64 != 0 || Cout % (sparse ? 128 : 64) != 0) return SDGP_ERR_UNSUPPORTED;
+  if (Cin % 64 != 0 || Cout % 64 != 0) return SDGP_ERR_UNSUPPORTED;
   if ((int64_t)R * S * Cin > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
 
   const int BN = (Cin % 256 == 0) ? 256 : (Cin % 128 == 0) ? 128 : 64;
   const int kb_channels = sparse ? 128 : 64;
 
-  DgradParams p = {};
-  p.B = B; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout; p.R = R; p.S = S; p.pad = pad;
-  choose_patch(B, H, W, &p.TW, &p.TH, &p.TB);
-  p.tiles_w = (W + p.TW - 1) / p.TW;
-  p.tiles_h = (H + p.TH - 1) / p.TH;
-  p.tiles_b = (B + p.TB - 1) / p.TB;
-  p.tiles_n = Cin / BN;
-  const int64_t m_tiles = (int64_t)p.tiles_w * p.tiles_h * p.tiles_b;
-  if (m_tiles * p.tiles_n > 0x3FFFFFFF) return SDGP_ERR_UNSUPPORTED;
-  p.m_tiles = (int)m_tiles;
-  p.pair_tiles = (int)((m_tiles + 1) / 2) * p.tiles_n;
-  p.k_blocks = (Cout + kb_channels - 1) / kb_channels;
+  DgradView view;
+  view.P = P; view.Q = Q; view.batch = B;
+  view.a_channels = sparse ? (Cout + 127) / 128 * 128 : Cout;
+  view.w_cols = (int64_t)R * S * Cin;
 
-  if (sparse) {
-    if (BN == 256) return launch_cfg<true, 256>(A, meta, Wt, dD, p, P, Q, stream);
-    if (BN == 128) return launch_cfg<true, 128>(A, meta, Wt, dD, p, P, Q, stream);
-    return launch_cfg<true, 64>(A, meta, Wt, dD, p, P, Q, stream);
+  // Output parities that no tap reaches are zero: clear dD first if there is any such class.
+  bool any_empty = false;
+  for (int ph = 0; ph < stride; ++ph)
+    for (int pw = 0; pw < stride; ++pw)
+      if ((ph + pad) % stride >= R || (pw + pad) % stride >= S) any_empty = true;
+  if (any_empty && cudaMemsetAsync(dD, 0, (size_t)B * H * W * Cin * 2, stream) != cudaSuccess) return SDGP_ERR_CUDA;
+  for (int ph = 0; ph < stride; ++ph) {
+    for (int pw = 0; pw < stride; ++pw) {
+      const int Hs = (H - ph + stride - 1) / stride, Ws = (W - pw + stride - 1) / stride;  // pixels of this class
+      if (Hs <= 0 || Ws <= 0) continue;
+      DgradParams p = {};
+      p.r_first = (ph + pad) % stride; p.r_step = stride;
+      p.s_first = (pw + pad) % stride; p.s_step = stride;
+      p.S_full = S;
+      p.R = p.r_first < R ? (R - p.r_first + stride - 1) / stride : 0;
+      p.S = p.s_first < S ? (S - p.s_first + stride - 1) / stride : 0;
+      if (p.R == 0 || p.S == 0) continue;  // cleared above
+      p.pad_h = (ph + pad - p.r_first) / stride;
+      p.pad_w = (pw + pad - p.s_first) / stride;
+      p.B = B; p.H = Hs; p.W = Ws; p.Cin = Cin; p.Cout = Cout;
+      choose_patch(B, Hs, Ws, &p.TW, &p.TH, &p.TB);
+      p.tiles_w = (Ws + p.TW - 1) / p.TW;
+      p.tiles_h = (Hs + p.TH - 1) / p.TH;
+      p.tiles_b = (B + p.TB - 1) / p.TB;
+      p.tiles_n = Cin / BN;
+      const int64_t m_tiles = (int64_t)p.tiles_w * p.tiles_h * p.tiles_b;
+      if (m_tiles * p.tiles_n > 0x3FFFFFFF) return SDGP_ERR_UNSUPPORTED;
+      p.m_tiles = (int)m_tiles;
+      p.pair_tiles = (int)((m_tiles + 1) / 2) * p.tiles_n;
+      p.k_blocks = (Cout + kb_channels - 1) / kb_channels;
+      view.d_base = (uint8_t*)dD + ((size_t)ph * W + pw) * Cin * 2;
+      view.d_stride_w = (uint64_t)stride * Cin * 2;
+      view.d_stride_h = (uint64_t)stride * W * Cin * 2;
+      view.d_stride_b = (uint64_t)H * W * Cin * 2;
+      sdgp_status st;
+      if (sparse) {
+        st = BN == 256 ? launch_cfg<true, 256>(A, meta, Wt, view, p, stream)
+           : BN == 128 ? launch_cfg<true, 128>(A, meta, Wt, view, p, stream)
+                       : launch_cfg<true, 64>(A, meta, Wt, view, p, stream);
+      } else {
+        st = BN == 256 ? launch_cfg<false, 256>(A, meta, Wt, view, p, stream)
+           : BN == 128 ? launch_cfg<false, 128>(A, meta, Wt, view, p, stream)
+                       : launch_cfg<false, 64>(A, meta, Wt, view, p, stream);
+      }
+      if (st != SDGP_OK) return st;
+    }
   }
-  if (BN == 256) return launch_cfg<false, 256>(A, meta, Wt, dD, p, P, Q, stream);
-  if (BN == 128) return launch_cfg<false, 128>(A, meta, Wt, dD, p, P, Q, stream);
-  return launch_cfg<false, 64>(A, meta, Wt, dD, p, P, Q, stream);
+  return SDGP_OK;
 }
 
 sdgp_status read_device_error() {

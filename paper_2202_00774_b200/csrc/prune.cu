@@ -247,11 +247,31 @@ __device__ __forceinline__ void rescale_packed(uint32_t& y0, uint32_t& y1, uint3
 // Writes one vector's outputs from the lane-paired form: y_i = (element i, element i + 4) after
 // pruning, km_i = 0xFFFF in the lanes of kept elements. COMPRESS: every 4-chunk holds at most two
 // survivors, so values / meta can be produced.
+// Row pitch of the compressed outputs, in 8-element vectors: k8 per input row, kpad8 per output
+// row (kpad8 == 0: same as the input). The extra vectors of a padded row are written as zero
+// values with the position pair (0,1), by the thread that owns the row's last real vector.
+struct OutPitch {
+  int k8, kpad8;
+};
+
 template <bool COMPRESS>
 __device__ __forceinline__ void emit_packed(int64_t v, uint32_t y0, uint32_t y1, uint32_t y2, uint32_t y3,
                                             uint32_t km0, uint32_t km1, uint32_t km2, uint32_t km3,
                                             uint4* __restrict__ dense, uint2* __restrict__ values,
-                                            uint8_t* __restrict__ meta, uint8_t* __restrict__ mask) {
+                                            uint8_t* __restrict__ meta, uint8_t* __restrict__ mask,
+                                            OutPitch pitch) {
+  int64_t vo = v;
+  if (pitch.kpad8 != 0) {
+    const int64_t row = v / pitch.k8;
+    const int kv = (int)(v - row * pitch.k8);
+    vo = row * pitch.kpad8 + kv;
+    if (COMPRESS && kv == pitch.k8 - 1) {
+      for (int t = 1; t <= pitch.kpad8 - pitch.k8; ++t) {
+        if (values) values[vo + t] = make_uint2(0u, 0u);
+        if (meta) meta[vo + t] = (uint8_t)0x44;
+      }
+    }
+  }
   if (dense)
     dense[v] = make_uint4(prmt(y0, y1, 0x5410), prmt(y2, y3, 0x5410), prmt(y0, y1, 0x7632), prmt(y2, y3, 0x7632));
   if (mask) {
@@ -264,12 +284,12 @@ __device__ __forceinline__ void emit_packed(int64_t v, uint32_t y0, uint32_t y1,
     const uint32_t k23 = km2 | km3;
     const uint32_t slot0 = y0 | (y1 & k23) | (y2 & km3);
     const uint32_t slot1 = y3 | (~km3 & (y2 | (~km2 & y1)));
-    if (values) values[v] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
+    if (values) values[vo] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
     if (meta) {
       const uint32_t pos0 = (km1 & k23 & 0x00010001u) | (km2 & km3 & 0x00020002u);
       const uint32_t pos1 = 0x00010001u + (k23 & 0x00010001u) + (km3 & 0x00010001u);
       const uint32_t nib = pos0 + 4u * pos1;
-      meta[v] = (uint8_t)((nib & 0xFu) | (nib >> 12));
+      meta[vo] = (uint8_t)((nib & 0xFu) | (nib >> 12));
     }
   }
 }
@@ -278,7 +298,7 @@ template <int N, int SCHEME>
 __global__ void __launch_bounds__(kThreads)
 prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                 uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
-                uint8_t* __restrict__ mask) {
+                uint8_t* __restrict__ mask, OutPitch pitch) {
   constexpr int NEED = 4 - N;  // an element is kept iff it beats at least 4 - n of the other three
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
   uint4 in[kVecPerThread];
@@ -352,13 +372,13 @@ prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, ui
       rescale_packed(y0, y1, y2, y3, km0, km1, km2, km3, scA, scB, tA, tB);
     }
 
-    emit_packed<(N <= 2)>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask);
+    emit_packed<(N <= 2)>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask, pitch);
   }
 }
 
 template <int N>
 cudaError_t launch_m4_n(int scheme, const void* dO, int64_t nvec, uint64_t seed, void* dense, void* values,
-                        void* meta, void* mask, cudaStream_t stream) {
+                        void* meta, void* mask, OutPitch pitch, cudaStream_t stream) {
   const int64_t per_block = (int64_t)kThreads * kVecPerThread;
   const int64_t blocks = (nvec + per_block - 1) / per_block;
   if (blocks == 0) return cudaSuccess;
@@ -367,7 +387,7 @@ cudaError_t launch_m4_n(int scheme, const void* dO, int64_t nvec, uint64_t seed,
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
 #define SDGP_LAUNCH4(S)                                                                         \
   prune_m4_kernel<N, S><<<grid, block, 0, stream>>>((const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
-                                                    (uint2*)values, (uint8_t*)meta, (uint8_t*)mask)
+                                                    (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch)
   switch (scheme) {
     case SDGP_RANDOM: SDGP_LAUNCH4(SDGP_RANDOM); break;
     case SDGP_MAGNITUDE: SDGP_LAUNCH4(SDGP_MAGNITUDE); break;
@@ -394,7 +414,7 @@ template <int M, int N, int SCHEME>
 __global__ void __launch_bounds__(kThreads)
 prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                   uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
-                  uint8_t* __restrict__ mask) {
+                  uint8_t* __restrict__ mask, OutPitch pitch) {
   constexpr int LANES = M / 8;
   static_assert(N == 1 || N == 2, "threshold selection keeps one or two elements");
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
@@ -465,13 +485,13 @@ prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, 
       const float sc = (ssum == 0.0f) ? 1.0f : __fdiv_rn(tsum, ssum);
       rescale_packed(y0, y1, y2, y3, km0, km1, km2, km3, sc, sc, tsum, tsum);
     }
-    if (v < nvec) emit_packed<true>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask);
+    if (v < nvec) emit_packed<true>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask, pitch);
   }
 }
 
 template <int M, int N>
 cudaError_t launch_top2(int scheme, const void* dO, int64_t nvec, uint64_t seed, void* dense, void* values,
-                        void* meta, void* mask, cudaStream_t stream) {
+                        void* meta, void* mask, OutPitch pitch, cudaStream_t stream) {
   const int64_t per_block = (int64_t)kThreads * kVecPerThread;
   const int64_t blocks = (nvec + per_block - 1) / per_block;
   if (blocks == 0) return cudaSuccess;
@@ -480,7 +500,7 @@ cudaError_t launch_top2(int scheme, const void* dO, int64_t nvec, uint64_t seed,
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
 #define SDGP_LAUNCH_T2(S)                                                                            \
   prune_top2_kernel<M, N, S><<<grid, block, 0, stream>>>((const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
-                                                         (uint2*)values, (uint8_t*)meta, (uint8_t*)mask)
+                                                         (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch)
   switch (scheme) {
     case SDGP_RANDOM: SDGP_LAUNCH_T2(SDGP_RANDOM); break;
     case SDGP_MAGNITUDE: SDGP_LAUNCH_T2(SDGP_MAGNITUDE); break;
@@ -515,20 +535,25 @@ cudaError_t launch_m(int scheme, const void* dO, int64_t nvec, int n, uint64_t s
 
 cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, int scheme,
                          uint64_t seed, void* dense, void* values, void* meta, void* mask,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, int64_t k_pad) {
   const int64_t nvec = rows * (K / 8);
+  OutPitch pitch = {(int)(K / 8), 0};
+  if (k_pad != 0 && k_pad != K) {
+    if (k_pad < K || k_pad % 8 != 0 || n > 2) return cudaErrorInvalidValue;  // padded rows exist only for compressed outputs
+    pitch.kpad8 = (int)(k_pad / 8);
+  }
   switch (m) {
     case 4:
       switch (n) {
-        case 1: return launch_m4_n<1>(scheme, dO, nvec, seed, dense, values, meta, mask, stream);
-        case 2: return launch_m4_n<2>(scheme, dO, nvec, seed, dense, values, meta, mask, stream);
-        case 3: return launch_m4_n<3>(scheme, dO, nvec, seed, dense, values, meta, mask, stream);
-        default: return launch_m4_n<4>(scheme, dO, nvec, seed, dense, values, meta, mask, stream);
+        case 1: return launch_m4_n<1>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
+        case 2: return launch_m4_n<2>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
+        case 3: return launch_m4_n<3>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
+        default: return launch_m4_n<4>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
       }
-#define SDGP_M_CASE(M)                                                                              \
-  case M:                                                                                           \
-    if (n == 1) return launch_top2<M, 1>(scheme, dO, nvec, seed, dense, values, meta, mask, stream); \
-    if (n == 2) return launch_top2<M, 2>(scheme, dO, nvec, seed, dense, values, meta, mask, stream); \
+#define SDGP_M_CASE(M)                                                                                     \
+  case M:                                                                                                  \
+    if (n == 1) return launch_top2<M, 1>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream); \
+    if (n == 2) return launch_top2<M, 2>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream); \
     return launch_m<M>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
     SDGP_M_CASE(8)
     SDGP_M_CASE(16)

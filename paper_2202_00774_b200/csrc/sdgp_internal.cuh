@@ -7,15 +7,19 @@
 
 namespace sdgp {
 
+// k_pad (0 = none): row pitch, in elements, of the compressed outputs. When k_pad > K the extra
+// chunks of every row are written as zero values with the position pair (0,1), so a consumer can
+// treat the row as k_pad channels (used to bring a channel count up to a whole 128-channel block).
 cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, int scheme,
                          uint64_t seed, void* dense, void* values, void* meta, void* mask,
-                         cudaStream_t stream);
+                         cudaStream_t stream, int64_t k_pad = 0);
 
-// Stride-1 data gradient on the tensor cores. sparse == false: A is dense dL/dO [B,P,Q,Cout];
-// sparse == true: A is the compressed values [B,P,Q,Cout/2] and meta [B,P,Q,Cout/16].
+// Data gradient on the tensor cores (stride 1 or 2). sparse == false: A is dense dL/dO
+// [B,P,Q,Cout]; sparse == true: A is the compressed values [B,P,Q,Cp/2] and meta [B,P,Q,Cp/16]
+// with Cp = Cout rounded up to a multiple of 128 (see launch_prune's k_pad).
 // Wt [Cout,R,S,Cin], dD [B,H,W,Cin]. A fully connected layer is B = H = 1, W = rows, R = S = 1.
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
-                         int H, int W, int Cin, int Cout, int R, int S, int pad, cudaStream_t stream);
+                         int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream);
 
 // Synchronises the device, then reads and clears the kernels' error word.
 sdgp_status read_device_error();

@@ -61,5 +61,5 @@ extern "C" sdgp_status sdgp_dgrad_linear_static(const void* dO, const void* W, v
   // first, so what an earlier call left in the array never shows.
   if (sdgp::launch_prune(dO, rows, K, n, m, (int)scheme, seed, nullptr, values, meta, nullptr, s) != cudaSuccess)
     return SDGP_ERR_CUDA;
-  return sdgp::launch_dgrad(true, values, meta, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 0, s);
+  return sdgp::launch_dgrad(true, values, meta, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 1, 0, s);
 }

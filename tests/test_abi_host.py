@@ -72,7 +72,7 @@ def test_dgrad_rejects_bad_arguments_before_launch(lib):
     assert L(FAKE, FAKE, FAKE, 128, 250, 128, 2, 4, 1, 0, ws, need, 0, None) == 1       # K % m != 0
     assert L(None, FAKE, FAKE, 128, 256, 128, 2, 4, 1, 0, ws, need, 0, None) == 1
     assert L(FAKE, FAKE, FAKE, 0, 256, 128, 2, 4, 1, 0, None, 0, 0, None) == 0          # rows == 0: no-op
-    assert C(FAKE, FAKE, FAKE, 2, 8, 8, 64, 128, 3, 3, 2, 1, 2, 4, 1, 0, ws, 1 << 30, 0, None) == 2  # stride 2
+    assert C(FAKE, FAKE, FAKE, 2, 8, 8, 64, 128, 3, 3, 3, 1, 2, 4, 1, 0, ws, 1 << 30, 0, None) == 2  # stride 3
     assert C(FAKE, FAKE, FAKE, 2, 8, 8, 64, 128, 3, 3, 1, 1, 2, 4, 1, 0, None, 0, 0, None) == 4
     assert lib.sdgp_workspace_size_conv2d(2, 8, 8, 64, 128, 3, 3, 1, 1, 0) == 2 * 8 * 8 * 128 * 9 // 8
     assert lib.sdgp_workspace_size_conv2d(2, 8, 8, 64, 128, 3, 3, 1, 1, 2) == 0

@@ -169,13 +169,88 @@ def test_conv_reuse_modes_sampled(case, mode):
     assert not np.isnan(to_f64(dD)).any()
 
 
+STRIDE2_CASES = [
+    # B, H, W, Cin, Cout, R, S, pad      (stride 2)
+    (3, 16, 16, 64, 128, 3, 3, 1),
+    (2, 28, 28, 128, 128, 3, 3, 1),     # bottleneck 3x3 / 2
+    (2, 14, 14, 64, 128, 1, 1, 0),      # 1x1 / 2 projection: three of four output parities are zero
+    (2, 15, 13, 64, 128, 3, 3, 1),      # odd sizes: parity classes of different extent
+    (1, 12, 12, 64, 128, 5, 5, 2),
+]
+
+
+@pytest.mark.parametrize("mode", ["dense", "sparse"])
+@pytest.mark.parametrize("case", STRIDE2_CASES)
+def test_conv_stride2(case, mode):
+    import paper_2202_00774_b200 as sdgp
+    B, H, Wd, Cin, Cout, R, S, pad = case
+    layer = inputs.ConvLayer("t", B, H, Wd, Cin, Cout, R, S, 2, pad)
+    dO, W = inputs.conv_layer_tensors(layer, seed=H + Cin)
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    if mode == "dense":
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 2, pad, 4, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
+        src = dO
+    else:
+        ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(B, H, Wd, Cin, Cout, R, S, 2, pad), dtype=torch.uint8,
+                         device="cuda")
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 2, pad, 2, 4, sdgp.RESCALED_MAGNITUDE, seed=3, workspace=ws)
+        src = oracle.prune(dO.reshape(-1, Cout), 2, 4, oracle.RESCALED, 3, want=("dense",))["dense"].reshape(dO.shape)
+    check_no_device_error()
+    got = to_f64(dD)
+    assert not np.isnan(got).any()
+    assert rel_fro(got, oracle.dgrad_conv2d(src, W, H, Wd, 2, pad)) <= TOL
+
+
+# Output-channel counts that are not whole 128-channel blocks: the compressed rows are padded.
+PADDED_CASES = [
+    (2, 14, 14, 64, 64, 3, 3, 1, 1),     # B, H, W, Cin, Cout, R, S, stride, pad
+    (2, 14, 14, 256, 64, 1, 1, 1, 0),
+    (2, 8, 8, 64, 192, 3, 3, 1, 1),
+    (2, 16, 16, 64, 64, 3, 3, 2, 1),
+]
+
+
+@pytest.mark.parametrize("scheme", [oracle.MAGNITUDE, oracle.RANDOM])
+@pytest.mark.parametrize("case", PADDED_CASES)
+def test_pruned_conv_partial_channel_block(case, scheme):
+    import paper_2202_00774_b200 as sdgp
+    B, H, Wd, Cin, Cout, R, S, stride, pad = case
+    layer = inputs.ConvLayer("t", B, H, Wd, Cin, Cout, R, S, stride, pad)
+    dO, W = inputs.conv_layer_tensors(layer, seed=Cout)
+    ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(B, H, Wd, Cin, Cout, R, S, stride, pad), dtype=torch.uint8,
+                     device="cuda")
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, stride, pad, 2, 4, scheme, seed=11, workspace=ws)
+    check_no_device_error()
+    pruned = oracle.prune(dO.reshape(-1, Cout), 2, 4, scheme, 11, want=("dense",))["dense"].reshape(dO.shape)
+    assert rel_fro(to_f64(dD), oracle.dgrad_conv2d(pruned, W, H, Wd, stride, pad)) <= TOL
+
+
+def test_resnet50_bottleneck_shapes_small_batch():
+    """Every distinct stride-1 bottleneck convolution of ResNet-50 (batch 2), 2:4 magnitude."""
+    import paper_2202_00774_b200 as sdgp
+    for layer in inputs.resnet50_stride1_layers(batch=2):
+        dO, W = inputs.conv_layer_tensors(layer, seed=layer.Cin + layer.Cout)
+        ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(layer.B, layer.H, layer.W, layer.Cin, layer.Cout, layer.R,
+                                                         layer.S, 1, layer.pad), dtype=torch.uint8, device="cuda")
+        dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, layer.pad, 2, 4, sdgp.MAGNITUDE, workspace=ws)
+        check_no_device_error()
+        pruned = oracle.prune(dO.reshape(-1, layer.Cout), 2, 4, oracle.MAGNITUDE, 0, want=("dense",))["dense"]
+        rng = np.random.default_rng(layer.Cin)
+        idx = np.unique(rng.integers(0, layer.B * layer.H * layer.W, 400))
+        want = oracle.dgrad_conv2d(pruned.reshape(dO.shape), W, layer.H, layer.W, 1, layer.pad, pixel_index=idx)
+        got = to_f64(dD).reshape(-1, layer.Cin)[idx]
+        assert rel_fro(got, want) <= TOL, layer.name
+
+
 def test_unsupported_requests_raise():
     import paper_2202_00774_b200 as sdgp
     dO = torch.zeros((2, 4, 4, 128), dtype=torch.int16, device="cuda")
     W = torch.zeros((128, 3, 3, 64), dtype=torch.int16, device="cuda")
     dD = torch.zeros((2, 8, 8, 64), dtype=torch.int16, device="cuda")
     with pytest.raises(sdgp.SdgpError) as e:
-        sdgp.sdgp_dgrad_conv2d(dO, W, dD, 2, 1, 2, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
+        sdgp.sdgp_dgrad_conv2d(dO, W, dD, 3, 1, 2, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)   # stride 3
     assert e.value.status == 2
 
 
