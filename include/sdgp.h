@@ -69,7 +69,8 @@ typedef enum { SDGP_RANDOM = 0, SDGP_MAGNITUDE = 1, SDGP_RESCALED_MAGNITUDE = 2 
 /* `flags` of the dgrad entry points. */
 enum {
   SDGP_FLAG_TWO_PASS = 0, /* prune kernel writes compressed dL/dO into the workspace, sparse GEMM reads it */
-  SDGP_FLAG_FUSED = 1,    /* pruning happens inside the GEMM's producer; no compressed tensor in global memory */
+  SDGP_FLAG_FUSED = 1,    /* pruning happens inside the dgrad kernel (needs m == 4, n <= 2); no workspace, no
+                             compressed tensor in global memory */
   SDGP_FLAG_DENSE = 2     /* no pruning: dense tensor-core data gradient of dL/dO itself (n, m, scheme ignored) */
 };
 

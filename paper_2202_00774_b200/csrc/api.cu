@@ -128,8 +128,12 @@ sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, in
   cudaStream_t s = (cudaStream_t)stream;
   if (flags == SDGP_FLAG_DENSE || n == m)
     return sdgp::launch_dgrad(false, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s);
-  if (flags == SDGP_FLAG_FUSED) return SDGP_ERR_UNSUPPORTED;
   if (Cin % 64 != 0 || Cout % 64 != 0) return SDGP_ERR_UNSUPPORTED;
+  if (flags == SDGP_FLAG_FUSED) {
+    if (m != 4) return SDGP_ERR_UNSUPPORTED;  // the in-kernel prune handles groups of four
+    const sdgp::FusedPrune fp = {n, (int)scheme, seed};
+    return sdgp::launch_dgrad(true, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, &fp);
+  }
   const int64_t Cpad = pad128(Cout);
   const Carve c = carve_compressed(workspace, (int64_t)B * P * Q * Cpad);
   if (!workspace || workspace_bytes < c.bytes) return SDGP_ERR_WORKSPACE;

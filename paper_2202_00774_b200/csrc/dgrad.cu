@@ -36,6 +36,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include "prune_core.cuh"
 #include "ptx.cuh"
 #include "sdgp_internal.cuh"
 
@@ -74,6 +75,11 @@ struct DgradParams {
   int meta_shared;        // metadata slots live in the first columns of the accumulator NOT being written
   int w_resident;         // whole W half-slice kept in shared memory
   int out_bufs;           // epilogue staging slabs (1 or 2)
+  // fused pruning (the kernel reads dense dL/dO and prunes it while staging A)
+  int fused_n, fused_scheme;
+  uint32_t seed_lo, seed_hi;
+  int P, Q;               // dO pixel grid (for the linear element index of the random scheme)
+  int off_raw;            // dense dL/dO stages: 2 * a_bytes each (two boxes of 64 channels)
   // shared-memory carve (byte offsets from the 1024-aligned base) and per-stage sizes
   int a_bytes, b_bytes, eraw_bytes, ehw_bytes;
   int off_b, off_eraw, off_ehw, off_w, off_out, off_bar;
@@ -118,6 +124,28 @@ __device__ __forceinline__ void rearrange_metadata_row(const uint8_t* raw_rows, 
     const int tl = (row & 7) + 8 * (u & 1) + 16 * (row >> 4);
     hw[tl * 8 + 2 * (u >> 1) + ((row >> 3) & 1)] = (uint16_t)v;
   }
+}
+
+// Fused pruning of one pixel row of a stage: 128 dense channels (two 128-byte-swizzled boxes of
+// 64) -> 64 compressed values written straight into the A tile's swizzled row, plus the row's 16
+// bytes of position metadata in the row-major form the rearrangement step expects.
+// vbase = number of the row's first 8-element vector in the whole dL/dO tensor (random keys).
+template <int N, int SCHEME>
+__device__ __forceinline__ void fused_prune_row(const uint8_t* raw, int a_bytes, uint8_t* a_tile, uint8_t* meta_rows,
+                                                int i, int64_t vbase, uint32_t seed_lo, uint32_t seed_hi) {
+  uint32_t metaw[4] = {0u, 0u, 0u, 0u};
+  const int sw = i & 7;
+#pragma unroll 4
+  for (int j = 0; j < 16; ++j) {
+    const uint4 w = *(const uint4*)(raw + (j >> 3) * a_bytes + i * 128 + (((j & 7) ^ sw) << 4));
+    uint32_t y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2;
+    m4_prune_vector<N, SCHEME>(w, vbase + j, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
+    compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
+    *(uint2*)(a_tile + i * 128 + (((j >> 1) ^ sw) << 4) + (j & 1) * 8) =
+        make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
+    metaw[j >> 2] |= nib2 << (8 * (j & 3));
+  }
+  *(uint4*)(meta_rows + i * 16) = make_uint4(metaw[0], metaw[1], metaw[2], metaw[3]);
 }
 
 // The four epilogue warps move one 128-row x BN accumulator to global memory in 64-column
@@ -170,7 +198,7 @@ __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* stagi
   }
 }
 
-template <bool SPARSE, int BN>
+template <bool SPARSE, int BN, bool FUSED>
 __global__ void __launch_bounds__(kThreadsGemm, 1)
 dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmE,
              const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
@@ -186,6 +214,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   uint8_t* sEhw = smem + p.off_ehw;
   uint8_t* sW = smem + p.off_w;
   uint8_t* sOut = smem + p.off_out;
+  uint8_t* sRaw = smem + p.off_raw;
   uint64_t* full = (uint64_t*)(smem + p.off_bar);
   uint64_t* empty = full + kMaxStages;
   uint64_t* meta_full = empty + kMaxStages;
@@ -194,7 +223,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   uint64_t* acc_empty = acc_full + 2;
   uint64_t* w_full = acc_empty + 2;
   uint64_t* meta_free = w_full + 1;
-  uint32_t* tmem_slot = (uint32_t*)(meta_free + 2);
+  uint64_t* raw_full = meta_free + 2;
+  uint32_t* tmem_slot = (uint32_t*)(raw_full + kMaxStages);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -208,6 +238,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       ptx::mbar_init(&full[s], 1);
       ptx::mbar_init(&empty[s], 1);
       ptx::mbar_init(&meta_full[s], 1);
+      ptx::mbar_init(&raw_full[s], 1);
       ptx::mbar_init(&meta_ready[s], 8);
     }
     for (int a = 0; a < 2; ++a) {
@@ -259,7 +290,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                                     ft * p.Cin + n_half + C::kBoxCols * j, cb * C::kKB);
         }
       }
-      const uint32_t pair_tx = 2u * (uint32_t)(p.img_rows * 128 + (p.w_resident ? 0 : p.rr * C::kTapBBytes));
+      const uint32_t pair_tx =
+          2u * (uint32_t)((FUSED ? 0 : p.img_rows * 128) + (p.w_resident ? 0 : p.rr * C::kTapBBytes));
       const uint32_t meta_tx = (uint32_t)(p.img_rows * 16);
       int st = 0;
       uint32_t ph = 0;
@@ -279,11 +311,18 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           for (int cb = 0; cb < p.k_blocks; ++cb) {
             if (!ptx::mbar_wait(&empty[st], ph ^ 1u, err, 0x100u + st)) { alive = false; break; }
             if (rank == 0) ptx::mbar_arrive_expect_tx(&full[st], pair_tx);
-            if (SPARSE) {
-              ptx::mbar_arrive_expect_tx(&meta_full[st], meta_tx);
-              ptx::tma_load_4d(sEraw + st * p.eraw_bytes, &tmE, &meta_full[st], cb * 8, q0, p0, b0);
+            if (FUSED) {
+              // dense dL/dO of this CTA's patch: 128 channels as two boxes of 64
+              ptx::mbar_arrive_expect_tx(&raw_full[st], 2u * (uint32_t)(p.img_rows * 128));
+              ptx::tma_load_4d(sRaw + st * 2 * p.a_bytes, &tmA, &raw_full[st], cb * 128, q0, p0, b0);
+              ptx::tma_load_4d(sRaw + st * 2 * p.a_bytes + p.a_bytes, &tmA, &raw_full[st], cb * 128 + 64, q0, p0, b0);
+            } else {
+              if (SPARSE) {
+                ptx::mbar_arrive_expect_tx(&meta_full[st], meta_tx);
+                ptx::tma_load_4d(sEraw + st * p.eraw_bytes, &tmE, &meta_full[st], cb * 8, q0, p0, b0);
+              }
+              ptx::tma_load_4d_pair(sA + st * p.a_bytes, &tmA, &full[st], cb * 64, q0, p0, b0);
             }
-            ptx::tma_load_4d_pair(sA + st * p.a_bytes, &tmA, &full[st], cb * 64, q0, p0, b0);
             if (!p.w_resident) {
               for (int u = 0; u < p.rr; ++u) {
                 const int tap = filter_tap(reuse ? u : r, s);
@@ -375,9 +414,34 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       bool alive = true;
       int st = 0;
       uint32_t ph = 0;
+      const int img_h = p.TH + p.rr - 1;
       for (int pt = first_pair; alive && pt < p.pair_tiles; pt += pair_stride) {
+        int t = 2 * (pt / p.tiles_n) + (int)rank;
+        const int wt = t % p.tiles_w; t /= p.tiles_w;
+        const int ht = t % p.tiles_h; t /= p.tiles_h;
+        const int w0 = wt * p.TW, h0 = ht * p.TH, b0 = t * p.TB;
+        int r = reuse ? (p.R - 1) : 0, s = 0, cb = 0;
         for (int k = 0; k < uses_per_tile; ++k) {
-          if (!ptx::mbar_wait(&meta_full[st], ph, err, 0x500u + st)) { alive = false; break; }
+          if (FUSED) {
+            if (!ptx::mbar_wait(&raw_full[st], ph, err, 0x900u + st)) { alive = false; break; }
+            const int q0 = w0 + p.pad_w - s, p0 = h0 + p.pad_h - r;
+            for (int i = row; i < p.img_rows; i += 128) {
+              const int iw = i % p.TW, ih = (i / p.TW) % img_h, ib = i / (p.TW * img_h);
+              const int64_t pixel = ((int64_t)(b0 + ib) * p.P + (p0 + ih)) * p.Q + (q0 + iw);  // any value when outside
+              const int64_t vbase = pixel * (p.Cout >> 3) + cb * 16;
+              const uint8_t* raw = sRaw + st * 2 * p.a_bytes;
+              uint8_t* a_tile = sA + st * p.a_bytes;
+              uint8_t* meta_rows = sEraw + st * p.eraw_bytes;
+#define SDGP_FUSED_ROW(NN, SS) fused_prune_row<NN, SS>(raw, p.a_bytes, a_tile, meta_rows, i, vbase, p.seed_lo, p.seed_hi)
+              if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_MAGNITUDE); else SDGP_FUSED_ROW(2, SDGP_MAGNITUDE); }
+              else if (p.fused_scheme == SDGP_RANDOM) { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_RANDOM); else SDGP_FUSED_ROW(2, SDGP_RANDOM); }
+              else { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_RESCALED_MAGNITUDE); else SDGP_FUSED_ROW(2, SDGP_RESCALED_MAGNITUDE); }
+#undef SDGP_FUSED_ROW
+            }
+            ptx::named_bar_sync(2, 128);  // every row's metadata is in place before it is rearranged
+          } else {
+            if (!ptx::mbar_wait(&meta_full[st], ph, err, 0x500u + st)) { alive = false; break; }
+          }
           for (int u = 0; u < p.rr; ++u) {
             const int row_off = reuse ? (p.R - 1 - u) * p.TW : 0;
             rearrange_metadata_row(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + u * kEHwBytes,
@@ -387,6 +451,10 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive_cluster(&meta_ready[st], 0);
           if (++st == STAGES) { st = 0; ph ^= 1u; }
+          if (++cb == p.k_blocks) {
+            cb = 0;
+            if (++s == p.S) { s = 0; if (!reuse) ++r; }
+          }
         }
       }
     }
@@ -503,7 +571,7 @@ int round_up(int x, int a) { return (x + a - 1) / a * a; }
 
 // Shared-memory plan for one launch: decides filter-row reuse, resident W, pipeline depth,
 // accumulator count and the carve. Returns false if no variant fits.
-template <bool SPARSE, int BN>
+template <bool SPARSE, int BN, bool FUSED>
 bool plan(DgradParams* p) {
   using C = Cfg<SPARSE, BN>;
   const int taps = p->R * p->S;
@@ -525,7 +593,8 @@ bool plan(DgradParams* p) {
     p->eraw_bytes = SPARSE ? round_up(p->img_rows * 16, 128) : 0;
     p->ehw_bytes = SPARSE ? p->rr * kEHwBytes : 0;
     const int w_bytes = resident ? taps * p->k_blocks * C::kTapBBytes : 0;
-    const int stage_bytes = p->a_bytes + p->b_bytes + p->eraw_bytes + p->ehw_bytes;
+    const int raw_bytes = FUSED ? 2 * p->a_bytes : 0;
+    const int stage_bytes = p->a_bytes + p->b_bytes + p->eraw_bytes + p->ehw_bytes + raw_bytes;
     int out_bufs = 2;
     int stages = (budget - w_bytes - out_bufs * kOutBytes) / stage_bytes;
     if (stages < 4) {
@@ -548,7 +617,7 @@ bool plan(DgradParams* p) {
       const int max_meta_stages = ((int)kTmemCols - nacc * BN) / meta_div;
       if (stages > max_meta_stages) stages = max_meta_stages;
     }
-    if (stages < ((resident || reuse) ? 2 : 3)) continue;  // a reuse stage is R taps long
+    if (stages < ((resident || reuse || FUSED) ? 2 : 3)) continue;  // a reuse stage is R taps long
     p->stages = stages;
     p->nacc = nacc;
     p->meta_col = p->meta_shared ? 0 : nacc * BN;
@@ -558,7 +627,8 @@ bool plan(DgradParams* p) {
     p->off_ehw = round_up(p->off_eraw + stages * p->eraw_bytes, 1024);
     p->off_w = round_up(p->off_ehw + stages * p->ehw_bytes, 1024);
     p->off_out = round_up(p->off_w + w_bytes, 1024);
-    p->off_bar = p->off_out + out_bufs * kOutBytes;
+    p->off_raw = p->off_out + out_bufs * kOutBytes;
+    p->off_bar = p->off_raw + stages * raw_bytes;
     p->smem_bytes = p->off_bar + 512 + 1024;
     if (p->smem_bytes > kSmemLimit) continue;
     return true;
@@ -577,16 +647,16 @@ struct DgradView {
   uint64_t d_stride_w, d_stride_h, d_stride_b;  // bytes
 };
 
-template <bool SPARSE, int BN>
+template <bool SPARSE, int BN, bool FUSED = false>
 sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const DgradView& view, DgradParams p,
                        cudaStream_t stream) {
   const int P = view.P, Q = view.Q;
   using C = Cfg<SPARSE, BN>;
-  if (!plan<SPARSE, BN>(&p)) return SDGP_ERR_UNSUPPORTED;
+  if (!plan<SPARSE, BN, FUSED>(&p)) return SDGP_ERR_UNSUPPORTED;
 
   CUtensorMap tmA, tmE, tmB, tmD;
   const uint32_t img_h = (uint32_t)(p.TH + p.rr - 1);
-  const uint64_t CA = SPARSE ? (uint64_t)view.a_channels / 2 : (uint64_t)view.a_channels;  // stored elements per pixel
+  const uint64_t CA = (SPARSE && !FUSED) ? (uint64_t)view.a_channels / 2 : (uint64_t)view.a_channels;  // stored elements per pixel
   {
     const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
     const uint64_t strides[3] = {CA * 2, CA * 2 * Q, CA * 2 * Q * P};
@@ -594,7 +664,7 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const Dg
     if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
   }
-  if (SPARSE) {
+  if (SPARSE && !FUSED) {
     const uint64_t CE = (uint64_t)view.a_channels / 16;
     const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
     const uint64_t strides[3] = {CE * 2, CE * 2 * Q, CE * 2 * Q * P};
@@ -621,7 +691,7 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const Dg
   }
 
   static bool configured = false;
-  auto kernel = dgrad_kernel<SPARSE, BN>;
+  auto kernel = dgrad_kernel<SPARSE, BN, FUSED>;
   if (!configured) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
       return SDGP_ERR_CUDA;
@@ -652,8 +722,12 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const Dg
 // Stride 2 is split by the parity of the output pixel: pixel (2h'+ph, 2w'+pw) only meets the taps
 // r = ph + pad (mod 2), s = pw + pad (mod 2), and on those it is a stride-1 problem from dO to
 // the strided view dD[:, ph::2, pw::2, :].
+// fused != nullptr (with sparse == true): A is the DENSE dL/dO and the kernel prunes it itself
+// (m = 4, n = fused->n in {1, 2}); no compressed tensor exists in global memory.
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
-                         int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream) {
+                         int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
+                         const FusedPrune* fused) {
+  if (fused && (!sparse || fused->n < 1 || fused->n > 2)) return SDGP_ERR_UNSUPPORTED;
   if (stride != 1 && stride != 2) return SDGP_ERR_UNSUPPORTED;
   const int P = (H + 2 * pad - R) / stride + 1, Q = (W + 2 * pad - S) / stride + 1;
   if (P < 1 || Q < 1) return SDGP_ERR_INVALID_ARG;
@@ -666,7 +740,7 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
 
   DgradView view;
   view.P = P; view.Q = Q; view.batch = B;
-  view.a_channels = sparse ? (Cout + 127) / 128 * 128 : Cout;
+  view.a_channels = (sparse && !fused) ? (Cout + 127) / 128 * 128 : Cout;
   view.w_cols = (int64_t)R * S * Cin;
 
   // Output parities that no tap reaches are zero: clear dD first if there is any such class.
@@ -699,12 +773,21 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
       p.m_tiles = (int)m_tiles;
       p.pair_tiles = (int)((m_tiles + 1) / 2) * p.tiles_n;
       p.k_blocks = (Cout + kb_channels - 1) / kb_channels;
+      p.P = P; p.Q = Q;
+      if (fused) {
+        p.fused_n = fused->n; p.fused_scheme = fused->scheme;
+        p.seed_lo = (uint32_t)fused->seed; p.seed_hi = (uint32_t)(fused->seed >> 32);
+      }
       view.d_base = (uint8_t*)dD + ((size_t)ph * W + pw) * Cin * 2;
       view.d_stride_w = (uint64_t)stride * Cin * 2;
       view.d_stride_h = (uint64_t)stride * W * Cin * 2;
       view.d_stride_b = (uint64_t)H * W * Cin * 2;
       sdgp_status st;
-      if (sparse) {
+      if (fused) {
+        st = BN == 256 ? launch_cfg<true, 256, true>(A, meta, Wt, view, p, stream)
+           : BN == 128 ? launch_cfg<true, 128, true>(A, meta, Wt, view, p, stream)
+                       : launch_cfg<true, 64, true>(A, meta, Wt, view, p, stream);
+      } else if (sparse) {
         st = BN == 256 ? launch_cfg<true, 256>(A, meta, Wt, view, p, stream)
            : BN == 128 ? launch_cfg<true, 128>(A, meta, Wt, view, p, stream)
                        : launch_cfg<true, 64>(A, meta, Wt, view, p, stream);

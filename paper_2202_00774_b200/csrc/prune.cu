@@ -8,6 +8,7 @@
 // the same 8-element vector number so all stores coalesce.
 #include <cuda_bf16.h>
 
+#include "prune_core.cuh"
 #include "sdgp_internal.cuh"
 
 namespace sdgp {
@@ -15,29 +16,6 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kVecPerThread = 4;
-
-// Philox4x32-10 (Salmon et al., SC'11): ten rounds, Weyl key schedule.
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                               uint32_t k0, uint32_t k1) {
-#pragma unroll
-  for (int round = 0; round < 10; ++round) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
-    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
-  }
-  return make_uint4(c0, c1, c2, c3);
-}
-
-// fp32 -> bf16 bits, round to nearest even; any NaN becomes 0x7FC0.
-__device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
-  uint32_t u = __float_as_uint(f);
-  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FC0u;
-  u += 0x7FFFu + ((u >> 16) & 1u);
-  return u >> 16;
-}
 
 // Survivor positions of a 4-chunk from its 4-bit keep mask: pad with the lowest unused
 // positions up to two, ascending; entry = p0 | p1 << 2 (16 nibbles packed in 64 bits).
@@ -190,63 +168,6 @@ prune_kernel(const uint4* __restrict__ dO, int64_t nvec, int n, uint32_t seed_lo
 // element (a threshold on the number of wins), and the compressed slots / position nibbles
 // are computed on both lanes at once. About a quarter of the instructions of the generic path.
 
-template <int LUT>
-__device__ __forceinline__ uint32_t lop3(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("lop3.b32 %0, %1, %2, %3, %4;" : "=r"(d) : "r"(a), "r"(b), "r"(c), "n"(LUT));
-  return d;
-}
-
-// prmt.b32, default mode: result byte n = byte (sel nibble n & 7) of {b,a}; a nibble with its
-// top bit set replicates that byte's sign bit over the whole result byte instead.
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-  uint32_t d;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-  return d;
-}
-
-// Truth-table byte of "at least NEED of the three inputs are true", with optional input negation.
-template <int NEED>
-__host__ __device__ constexpr int threshold_lut(bool na, bool nb, bool nc) {
-  int lut = 0;
-  for (int idx = 0; idx < 8; ++idx) {
-    const int a = ((idx >> 2) & 1) ^ (na ? 1 : 0), b = ((idx >> 1) & 1) ^ (nb ? 1 : 0), c = (idx & 1) ^ (nc ? 1 : 0);
-    if (a + b + c >= NEED) lut |= 1 << idx;
-  }
-  return lut;
-}
-
-
-// Survivors of both lanes times their group's scale, rounded to bf16 (nearest even). When both
-// group sums are finite every product is finite and the hardware's packed conversion applies;
-// otherwise (Inf or NaN in the group) each value goes through the explicit rounding, which
-// stores any NaN as 0x7FC0.
-__device__ __forceinline__ void rescale_packed(uint32_t& y0, uint32_t& y1, uint32_t& y2, uint32_t& y3, uint32_t km0,
-                                               uint32_t km1, uint32_t km2, uint32_t km3, float scA, float scB,
-                                               float tA, float tB) {
-  const bool finite = (__float_as_uint(tA) & 0x7F800000u) != 0x7F800000u &&
-                      (__float_as_uint(tB) & 0x7F800000u) != 0x7F800000u;
-  if (finite) {
-#define SDGP_RESCALE_FAST(y, km)                                                                    \
-  {                                                                                                 \
-    const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(__uint_as_float(y << 16), scA),        \
-                                                   __fmul_rn(__uint_as_float(y & 0xFFFF0000u), scB)); \
-    y = (*(const uint32_t*)&h) & km;                                                                \
-  }
-    SDGP_RESCALE_FAST(y0, km0) SDGP_RESCALE_FAST(y1, km1) SDGP_RESCALE_FAST(y2, km2) SDGP_RESCALE_FAST(y3, km3)
-#undef SDGP_RESCALE_FAST
-  } else {
-#define SDGP_RESCALE_SLOW(y, km)                                                                    \
-  y = (f32_to_bf16_bits(__fmul_rn(__uint_as_float(y << 16), scA)) |                                 \
-       (f32_to_bf16_bits(__fmul_rn(__uint_as_float(y & 0xFFFF0000u), scB)) << 16)) & km;
-    SDGP_RESCALE_SLOW(y0, km0) SDGP_RESCALE_SLOW(y1, km1) SDGP_RESCALE_SLOW(y2, km2) SDGP_RESCALE_SLOW(y3, km3)
-#undef SDGP_RESCALE_SLOW
-  }
-}
-
-// Writes one vector's outputs from the lane-paired form: y_i = (element i, element i + 4) after
-// pruning, km_i = 0xFFFF in the lanes of kept elements. COMPRESS: every 4-chunk holds at most two
-// survivors, so values / meta can be produced.
 // Row pitch of the compressed outputs, in 8-element vectors: k8 per input row, kpad8 per output
 // row (kpad8 == 0: same as the input). The extra vectors of a padded row are written as zero
 // values with the position pair (0,1), by the thread that owns the row's last real vector.
@@ -254,6 +175,8 @@ struct OutPitch {
   int k8, kpad8;
 };
 
+// Writes one vector's outputs from the lane-paired form (see m4_prune_vector). COMPRESS: every
+// 4-chunk holds at most two survivors, so values / meta can be produced.
 template <bool COMPRESS>
 __device__ __forceinline__ void emit_packed(int64_t v, uint32_t y0, uint32_t y1, uint32_t y2, uint32_t y3,
                                             uint32_t km0, uint32_t km1, uint32_t km2, uint32_t km3,
@@ -279,18 +202,10 @@ __device__ __forceinline__ void emit_packed(int64_t v, uint32_t y0, uint32_t y1,
     mask[v] = (uint8_t)((t & 0xFu) | (t >> 12));
   }
   if (COMPRESS && (values || meta)) {
-    // At most two survivors per chunk. Positions: p1 = last survivor, but at least 1;
-    // p0 = first survivor if there are two, else 0 (the pad takes the lowest free position).
-    const uint32_t k23 = km2 | km3;
-    const uint32_t slot0 = y0 | (y1 & k23) | (y2 & km3);
-    const uint32_t slot1 = y3 | (~km3 & (y2 | (~km2 & y1)));
+    uint32_t slot0, slot1, nib2;
+    compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
     if (values) values[vo] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
-    if (meta) {
-      const uint32_t pos0 = (km1 & k23 & 0x00010001u) | (km2 & km3 & 0x00020002u);
-      const uint32_t pos1 = 0x00010001u + (k23 & 0x00010001u) + (km3 & 0x00010001u);
-      const uint32_t nib = pos0 + 4u * pos1;
-      meta[vo] = (uint8_t)((nib & 0xFu) | (nib >> 12));
-    }
+    if (meta) meta[vo] = (uint8_t)nib2;
   }
 }
 
@@ -299,7 +214,6 @@ __global__ void __launch_bounds__(kThreads)
 prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                 uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
                 uint8_t* __restrict__ mask, OutPitch pitch) {
-  constexpr int NEED = 4 - N;  // an element is kept iff it beats at least 4 - n of the other three
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
   uint4 in[kVecPerThread];
 #pragma unroll
@@ -312,66 +226,8 @@ prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, ui
     const int64_t v = base + (int64_t)it * kThreads;
     if (v >= nvec) continue;
     const uint4 w = in[it];
-    // lanes: low half = group A (elements 0..3), high half = group B (elements 4..7)
-    const uint32_t p0 = prmt(w.x, w.z, 0x5410), p1 = prmt(w.x, w.z, 0x7632);
-    const uint32_t p2 = prmt(w.y, w.w, 0x5410), p3 = prmt(w.y, w.w, 0x7632);
-
-    uint32_t km0, km1, km2, km3;  // 0xFFFF in a lane whose element is kept
-    if (N == 4) {
-      km0 = km1 = km2 = km3 = 0xFFFFFFFFu;
-    } else if (SCHEME == SDGP_RANDOM) {
-      const uint4 o = philox4x32_10((uint32_t)v, (uint32_t)((uint64_t)v >> 32), 0u, 0u, seed_lo, seed_hi);
-      // 16-bit keys; smaller ranks first, equal keys: lower index. e(i,j) = r_j - r_i has its
-      // sign bit set iff j ranks before i (j < i in key), i.e. iff i loses against j (for i < j).
-      const uint32_t rA0 = o.x & 0xFFFFu, rA1 = o.x >> 16, rA2 = o.y & 0xFFFFu, rA3 = o.y >> 16;
-      const uint32_t rB0 = o.z & 0xFFFFu, rB1 = o.z >> 16, rB2 = o.w & 0xFFFFu, rB3 = o.w >> 16;
-#define SDGP_KEEP4(r0, r1, r2, r3, k0, k1, k2, k3)                                                \
-  {                                                                                                \
-    const uint32_t e01 = r1 - r0, e02 = r2 - r0, e03 = r3 - r0, e12 = r2 - r1, e13 = r3 - r1,      \
-                   e23 = r3 - r2;                                                                  \
-    k0 = lop3<threshold_lut<NEED>(true, true, true)>(e01, e02, e03);                               \
-    k1 = lop3<threshold_lut<NEED>(false, true, true)>(e01, e12, e13);                              \
-    k2 = lop3<threshold_lut<NEED>(false, false, true)>(e02, e12, e23);                             \
-    k3 = lop3<threshold_lut<NEED>(false, false, false)>(e03, e13, e23);                            \
-  }
-      uint32_t a0, a1, a2, a3, b0, b1, b2, b3;  // keep flags in bit 31
-      SDGP_KEEP4(rA0, rA1, rA2, rA3, a0, a1, a2, a3)
-      SDGP_KEEP4(rB0, rB1, rB2, rB3, b0, b1, b2, b3)
-#undef SDGP_KEEP4
-      // replicate the two sign bits over their 16-bit lanes
-      km0 = prmt(a0, b0, 0xFFBB); km1 = prmt(a1, b1, 0xFFBB);
-      km2 = prmt(a2, b2, 0xFFBB); km3 = prmt(a3, b3, 0xFFBB);
-    } else {
-      // |x| as 15-bit integers. d(i,j) = (a_i | 0x8000) - a_j per lane never borrows across lanes
-      // and has bit 15 of the lane set iff a_i >= a_j, i.e. iff i beats j (i < j: ties to i).
-      constexpr uint32_t H = 0x80008000u;
-      const uint32_t h0 = p0 | H, h1 = p1 | H, h2 = p2 | H;
-      const uint32_t l1 = p1 & ~H, l2 = p2 & ~H, l3 = p3 & ~H;
-      const uint32_t d01 = h0 - l1, d02 = h0 - l2, d03 = h0 - l3, d12 = h1 - l2, d13 = h1 - l3, d23 = h2 - l3;
-      const uint32_t k0 = lop3<threshold_lut<NEED>(false, false, false)>(d01, d02, d03);
-      const uint32_t k1 = lop3<threshold_lut<NEED>(true, false, false)>(d01, d12, d13);
-      const uint32_t k2 = lop3<threshold_lut<NEED>(true, true, false)>(d02, d12, d23);
-      const uint32_t k3 = lop3<threshold_lut<NEED>(true, true, true)>(d03, d13, d23);
-      km0 = prmt(k0, 0, 0xBB99); km1 = prmt(k1, 0, 0xBB99);
-      km2 = prmt(k2, 0, 0xBB99); km3 = prmt(k3, 0, 0xBB99);
-    }
-
-    uint32_t y0 = p0 & km0, y1 = p1 & km1, y2 = p2 & km2, y3 = p3 & km3;  // pruned lanes are +0.0
-    if (SCHEME == SDGP_RESCALED_MAGNITUDE && N != 4) {
-      // per group: scale = sum|x| / sum|kept x|, balanced pairwise sums in index order
-      const float tA = __fadd_rn(__fadd_rn(__uint_as_float((p0 << 16) & 0x7FFF0000u), __uint_as_float((p1 << 16) & 0x7FFF0000u)),
-                                 __fadd_rn(__uint_as_float((p2 << 16) & 0x7FFF0000u), __uint_as_float((p3 << 16) & 0x7FFF0000u)));
-      const float tB = __fadd_rn(__fadd_rn(__uint_as_float(p0 & 0x7FFF0000u), __uint_as_float(p1 & 0x7FFF0000u)),
-                                 __fadd_rn(__uint_as_float(p2 & 0x7FFF0000u), __uint_as_float(p3 & 0x7FFF0000u)));
-      const float sA = __fadd_rn(__fadd_rn(__uint_as_float((y0 << 16) & 0x7FFF0000u), __uint_as_float((y1 << 16) & 0x7FFF0000u)),
-                                 __fadd_rn(__uint_as_float((y2 << 16) & 0x7FFF0000u), __uint_as_float((y3 << 16) & 0x7FFF0000u)));
-      const float sB = __fadd_rn(__fadd_rn(__uint_as_float(y0 & 0x7FFF0000u), __uint_as_float(y1 & 0x7FFF0000u)),
-                                 __fadd_rn(__uint_as_float(y2 & 0x7FFF0000u), __uint_as_float(y3 & 0x7FFF0000u)));
-      const float scA = (sA == 0.0f) ? 1.0f : __fdiv_rn(tA, sA);
-      const float scB = (sB == 0.0f) ? 1.0f : __fdiv_rn(tB, sB);
-      rescale_packed(y0, y1, y2, y3, km0, km1, km2, km3, scA, scB, tA, tB);
-    }
-
+    uint32_t y0, y1, y2, y3, km0, km1, km2, km3;
+    m4_prune_vector<N, SCHEME>(w, v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
     emit_packed<(N <= 2)>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask, pitch);
   }
 }

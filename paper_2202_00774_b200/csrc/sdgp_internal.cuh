@@ -18,8 +18,15 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
 // [B,P,Q,Cout]; sparse == true: A is the compressed values [B,P,Q,Cp/2] and meta [B,P,Q,Cp/16]
 // with Cp = Cout rounded up to a multiple of 128 (see launch_prune's k_pad).
 // Wt [Cout,R,S,Cin], dD [B,H,W,Cin]. A fully connected layer is B = H = 1, W = rows, R = S = 1.
+// fused != nullptr: A is the dense dL/dO and the kernel prunes it on the fly (groups of 4).
+struct FusedPrune {
+  int n;
+  int scheme;
+  uint64_t seed;
+};
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
-                         int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream);
+                         int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
+                         const FusedPrune* fused = nullptr);
 
 // Synchronises the device, then reads and clears the kernels' error word.
 sdgp_status read_device_error();

@@ -244,6 +244,50 @@ def test_resnet50_bottleneck_shapes_small_batch():
         assert rel_fro(got, want) <= TOL, layer.name
 
 
+# ------------------------------------------------------------------- fused
+
+
+FUSED_CASES = [
+    # B, H, W, Cin, Cout, R, S, stride, pad
+    (1, 1, 333, 128, 512, 1, 1, 1, 0),      # fully connected
+    (1, 1, 1000, 256, 256, 1, 1, 1, 0),
+    (3, 8, 8, 64, 128, 3, 3, 1, 1),
+    (40, 16, 16, 128, 128, 3, 3, 1, 1),     # filter-row reuse + resident W
+    (6, 32, 32, 64, 128, 3, 3, 1, 1),
+    (2, 14, 14, 64, 64, 3, 3, 1, 1),        # half a channel block
+    (2, 16, 16, 64, 128, 3, 3, 2, 1),       # stride 2
+    (2, 16, 16, 128, 256, 3, 3, 1, 1),      # two channel blocks
+]
+
+
+@pytest.mark.parametrize("scheme,n", [(oracle.MAGNITUDE, 2), (oracle.RESCALED, 2), (oracle.RANDOM, 2), (oracle.MAGNITUDE, 1),
+                                      (oracle.RANDOM, 1)])
+@pytest.mark.parametrize("case", FUSED_CASES)
+def test_fused_prune_and_dgrad(case, scheme, n):
+    """SDGP_FLAG_FUSED: no workspace; the kernel prunes dense dL/dO itself (groups of 4)."""
+    import paper_2202_00774_b200 as sdgp
+    B, H, Wd, Cin, Cout, R, S, stride, pad = case
+    layer = inputs.ConvLayer("t", B, H, Wd, Cin, Cout, R, S, stride, pad)
+    dO, W = inputs.conv_layer_tensors(layer, seed=B + Cout)
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, stride, pad, n, 4, scheme, seed=21, flags=sdgp.FLAG_FUSED)
+    check_no_device_error()
+    pruned = oracle.prune(dO.reshape(-1, Cout), n, 4, scheme, 21, want=("dense",))["dense"].reshape(dO.shape)
+    got = to_f64(dD)
+    assert not np.isnan(got).any()
+    assert rel_fro(got, oracle.dgrad_conv2d(pruned, W, H, Wd, stride, pad)) <= TOL
+
+
+def test_fused_needs_groups_of_four():
+    import paper_2202_00774_b200 as sdgp
+    dO = torch.zeros((2, 8, 8, 128), dtype=torch.int16, device="cuda")
+    W = torch.zeros((128, 3, 3, 64), dtype=torch.int16, device="cuda")
+    dD = torch.zeros((2, 8, 8, 64), dtype=torch.int16, device="cuda")
+    with pytest.raises(sdgp.SdgpError) as e:
+        sdgp.sdgp_dgrad_conv2d(dO, W, dD, 1, 1, 2, 8, sdgp.MAGNITUDE, flags=sdgp.FLAG_FUSED)
+    assert e.value.status == 2
+
+
 def test_unsupported_requests_raise():
     import paper_2202_00774_b200 as sdgp
     dO = torch.zeros((2, 4, 4, 128), dtype=torch.int16, device="cuda")
