@@ -237,7 +237,7 @@ def run_ours(args, layers):
         for i in order:
             l = layers[i]
             sdgp.sdgp_dgrad_conv2d(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, seed=1234, workspace=ws[i],
-                                   flags=sdgp.FLAG_TWO_PASS)
+                                   flags=sdgp.FLAG_FUSED if args.mode == "fused" else sdgp.FLAG_TWO_PASS)
 
     def dense_step():
         for i in order:
@@ -374,7 +374,7 @@ def run_ours(args, layers):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "layers": len(layers), "nm": args.nm, "scheme": args.scheme,
-                       "mode": "two_pass", "flops": "2*M*N*K of the implicit GEMM per layer",
+                       "mode": args.mode, "flops": "2*M*N*K of the implicit GEMM per layer",
                        "l2": "inputs larger than L2 (step touches %.0f MB)" % ((prune_bytes + d2h) / 1e6),
                        "launch": "one CUDA graph per step", "replicas": world},
             "speedup_vs_dense": value / dense_value, "dense_tflops": dense_value,
@@ -387,7 +387,7 @@ def run_ours(args, layers):
                                  "peak = 2 x %s sustained dense bf16" % pk["source"]},
             "per_layer": per_layer,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": 2 * len(layers) * args.steps,
+            "gpu_launches": (1 if args.mode == "fused" else 2) * len(layers) * args.steps,
             "clocks": clocks,
         }
         if base is not None:
@@ -406,6 +406,8 @@ def main():
     ap.add_argument("--workload", default="resnet9", choices=["resnet9", "gemm_large", "fc_small"])
     ap.add_argument("--scheme", default="magnitude", choices=sorted(SCHEMES))
     ap.add_argument("--nm", default="2:4")
+    ap.add_argument("--mode", default="two_pass", choices=["two_pass", "fused"],
+                    help="two_pass: prune kernel + sparse dgrad kernel per layer; fused: one kernel prunes and contracts")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     layers = workload_layers(args.workload)

@@ -581,9 +581,10 @@ bool plan(DgradParams* p) {
   const bool can_reuse = p->R > 1 && p->TB == 1 && p->TW % 8 == 0 && p->TW * (p->TH + p->R - 1) <= kMaxImgRows;
   const bool can_reside = p->tiles_n == 1 && p->pair_tiles > sm_count() / 2;  // pays only if tiles repeat
   for (int attempt = 0; attempt < 4; ++attempt) {
-    // attempt 0: reuse + resident W, 1: reuse, 2: resident W, 3: neither
+    // attempt 0: reuse with streamed W (measured best where it fits: more stages in flight),
+    // 1: reuse + resident W, 2: resident W, 3: neither
     const bool reuse = attempt < 2;
-    const bool resident = (attempt == 0 || attempt == 2);
+    const bool resident = (attempt == 1 || attempt == 2);
     if ((reuse && !can_reuse) || (resident && !can_reside)) continue;
     p->rr = reuse ? p->R : 1;
     p->img_rows = p->TW * (p->TH + p->rr - 1) * p->TB;
