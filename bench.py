@@ -204,6 +204,16 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(value, dist, device):
+    """Largest `value` over all ranks (every rank gets it); identity without a process group."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def run_ours(args, layers):
     import torch
     import paper_2202_00774_b200 as sdgp
@@ -271,10 +281,8 @@ def run_ours(args, layers):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1)
         if dist is not None:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = max_over_ranks(ms, dist, "cuda")
             dist.barrier()
-            ms = float(t.item())
         torch.cuda.synchronize()
         return ms
 
