@@ -65,6 +65,24 @@ def layer_inputs(l, workload, seed):
     return dO.reshape(l.dO_shape()), W.reshape(l.W_shape())
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the seven sparse dgrad launches of one
+# resnet9 two-pass step, from the ncu capture summarised in profiles/traffic_dgrad_sparse_resnet9.md,
+# and the hash of the kernel sources it was taken with (the figure is dropped once they change).
+NCU_TRAFFIC = {"workload": "resnet9", "mode": "two_pass", "bytes_per_step": 218.0e6, "sources_sha": "72e338b461f61d15"}
+KERNEL_SOURCES = ["dgrad.cu", "ptx.cuh", "prune_core.cuh"]
+
+
+def measured_traffic(workload, mode):
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2202_00774_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    if workload != NCU_TRAFFIC["workload"] or mode != NCU_TRAFFIC["mode"]:
+        return None
+    return NCU_TRAFFIC["bytes_per_step"] if h.hexdigest()[:16] == NCU_TRAFFIC["sources_sha"] else None
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -389,7 +407,8 @@ def run_ours(args, layers):
             "prune_gbs": prune_gbs, "prune_frac_of_hbm": prune_gbs / pk["hbm"],
             "roofline": {"bound": "tensor", "kernel": "dgrad_kernel<sparse>", "achieved": dgrad_tflops,
                          "peak": sparse_peak, "unit": "TFLOP/s", "frac": dgrad_tflops / sparse_peak,
-                         "traffic": None,
+                         "traffic": measured_traffic(args.workload, args.mode),
+                         "traffic_unit": "DRAM bytes of the sparse dgrad launches of one step (ncu)",
                          "note": "dense-equivalent FLOPs of all sparse dgrad launches / their summed time between "
                                  "event nodes of the replayed step graph; "
                                  "peak = 2 x %s sustained dense bf16" % pk["source"]},
