@@ -146,6 +146,11 @@ size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R
  * SDGP_OK, or SDGP_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last call. */
 sdgp_status sdgp_last_device_error(void);
 
+/* Self-test of the failure path (no counterpart in the paper): enqueues a one-CTA kernel that waits,
+ * with a 50 ms limit, on a barrier nothing signals. The kernel must end by itself and leave
+ * SDGP_ERR_TIMEOUT for the next sdgp_last_device_error() call; the context stays usable. */
+sdgp_status sdgp_selftest_bounded_wait(void* stream);
+
 /* Static, NUL-terminated description of a status code. */
 const char* sdgp_status_string(sdgp_status status);
 

@@ -17,7 +17,7 @@ RANDOM, MAGNITUDE, RESCALED_MAGNITUDE = 0, 1, 2
 FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE = 0, 1, 2
 
 EXPORTS = ["sdgp_prune", "sdgp_dgrad_linear", "sdgp_dgrad_conv2d", "sdgp_spmm_linear", "sdgp_spmm_conv2d",
-           "sdgp_dgrad_linear_static",
+           "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
            "sdgp_workspace_size_linear", "sdgp_workspace_size_conv2d", "sdgp_last_device_error",
            "sdgp_status_string"]
 
@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.sdgp_workspace_size_conv2d.restype = sz
         L.sdgp_last_device_error.argtypes = []
         L.sdgp_last_device_error.restype = i32
+        L.sdgp_selftest_bounded_wait.argtypes = [vp]
+        L.sdgp_selftest_bounded_wait.restype = i32
         L.sdgp_status_string.argtypes = [i32]
         L.sdgp_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -158,6 +160,11 @@ def sdgp_spmm_conv2d(values, meta, W, dD, stride, pad):
     Cout, R, S, _ = W.shape
     _check(lib().sdgp_spmm_conv2d(_ptr(values), _ptr(meta), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S,
                                   stride, pad, _stream()), "sdgp_spmm_conv2d")
+
+
+def sdgp_selftest_bounded_wait():
+    """Enqueues the kernel whose wait must run out (see sdgp.h); check with sdgp_last_device_error()."""
+    _check(lib().sdgp_selftest_bounded_wait(_stream()), "sdgp_selftest_bounded_wait")
 
 
 def sdgp_last_device_error() -> int:

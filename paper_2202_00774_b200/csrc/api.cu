@@ -155,4 +155,6 @@ sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t r
 
 sdgp_status sdgp_last_device_error(void) { return sdgp::read_device_error(); }
 
+sdgp_status sdgp_selftest_bounded_wait(void* stream) { return sdgp::launch_bounded_wait_selftest((cudaStream_t)stream); }
+
 }  // extern "C"

@@ -803,6 +803,24 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
   return SDGP_OK;
 }
 
+// One CTA waits, with a 50 ms limit, on a barrier that nothing ever signals: the wait must give
+// up, record its code and let the kernel end normally.
+__global__ void bounded_wait_selftest_kernel() {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) ptx::mbar_wait(&bar, 0u, &g_device_error, 0xE00u, 50000000ull);
+  __syncthreads();
+}
+
+sdgp_status launch_bounded_wait_selftest(cudaStream_t stream) {
+  bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>();
+  return cudaGetLastError() == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
+}
+
 sdgp_status read_device_error() {
   unsigned int word = 0;
   if (cudaDeviceSynchronize() != cudaSuccess) return SDGP_ERR_CUDA;

@@ -62,7 +62,7 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 // records `code` in *error_word and returns false; the caller carries on, so the kernel
 // always terminates.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* error_word,
-                                          unsigned int code) {
+                                          unsigned int code, uint64_t limit_ns = 2000000000ull) {
   if (mbar_test(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   for (;;) {
@@ -71,7 +71,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsign
       if (mbar_test(bar, parity)) return true;
     // once any wait of any CTA has given up, no other wait lingers
     if (*(volatile unsigned int*)error_word != 0u) return false;
-    if (globaltimer_ns() - t0 > 2000000000ull) {
+    if (globaltimer_ns() - t0 > limit_ns) {
       atomicCAS(error_word, 0u, code);
       return false;
     }

@@ -28,6 +28,9 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
                          int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
                          const FusedPrune* fused = nullptr);
 
+// Launches a one-CTA kernel whose only wait can never be satisfied (50 ms limit).
+sdgp_status launch_bounded_wait_selftest(cudaStream_t stream);
+
 // Synchronises the device, then reads and clears the kernels' error word.
 sdgp_status read_device_error();
 

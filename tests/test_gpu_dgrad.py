@@ -360,3 +360,18 @@ def test_gemm_large_full_size_sampled_rows(n, m, scheme):
     want = oracle.dgrad_linear(pruned, W)
     got = inputs.bf16_bits_to_f32(dD[torch.from_numpy(rows).cuda()].cpu().numpy().view(np.uint16)).astype(np.float64)
     assert rel_fro(got, want) <= TOL
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A wait that nothing satisfies gives up after its limit; the host sees SDGP_ERR_TIMEOUT once,
+    and the next kernels run normally."""
+    import paper_2202_00774_b200 as sdgp
+    assert sdgp.sdgp_last_device_error() == 0
+    sdgp.sdgp_selftest_bounded_wait()
+    assert sdgp.sdgp_last_device_error() == 6
+    assert sdgp.sdgp_last_device_error() == 0
+    dO, W = inputs.fc_tensors(128, 128, 64, seed=1)
+    dD = torch.empty((128, 64), dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, 4, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
+    check_no_device_error()
+    assert rel_fro(to_f64(dD), oracle.dgrad_linear(dO, W)) <= TOL
