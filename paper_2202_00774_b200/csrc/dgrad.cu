@@ -500,6 +500,340 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
 }
 
+// ---------------------------------------------------------------- whole-filter reuse
+//
+// Convolutions with more than one filter tap on images at least a strip (8 x 16 pixels) large.
+// The shared-memory matrix descriptor swizzles by absolute address bits, so an A operand may
+// start at ANY 128-byte row of a swizzled tile and its 8-row groups may lie any number of rows
+// apart. A tile is therefore an 8-pixel-wide, 16-pixel-tall strip of one image, and one TMA box
+// holding the strip plus its (R-1, S-1) halo serves EVERY filter tap: tap (r, s) is the row
+// offset (R-1-r) * pitch + (S-1-s) in the A descriptor, group stride = pitch rows. dL/dO is
+// read from L2 once per strip (plus halo) instead of once per horizontal tap, and with two
+// neighbouring strips per CTA (two accumulators) each W stage feeds twice the MMAs.
+//
+// Rings: A images (2 stages; one stage = one tile set and one block of output channels),
+// W taps (w_stages; one stage = the W rows of one tap and channel block, plus, for sparse A, the
+// rearranged metadata tiles of that tap). Roles as in dgrad_kernel; the metadata warps build one
+// 2 KB TMEM image per (tap, strip) from the raw metadata box of the A stage.
+
+constexpr int kHaloTH = 16;  // pixel rows of a strip: 8 x 16 pixels = the 128 rows of an accumulator
+constexpr int kHaloAStages = 2;
+
+struct HaloParams {
+  int B, H, W, Cin, Cout;
+  int R, S, pad_h, pad_w;
+  int r_first, r_step, s_first, s_step, S_full;  // as in DgradParams
+  int nt;                  // strips per CTA tile set (1 or 2), side by side, sharing every W stage
+  int sets_w, tiles_h, tiles_n;
+  int m_sets;              // sets_w * tiles_h * B
+  int pair_tiles;          // ceil(m_sets / 2) * tiles_n
+  int k_blocks;
+  int pitch;               // pixel columns of the A box: 8 * nt + S - 1
+  int img_h;               // pixel rows of the A box: kHaloTH + R - 1
+  int img_rows;            // pitch * img_h
+  int w_stages;
+  int meta_col, meta_shared, out_bufs;
+  int a_bytes, eraw_bytes, w_bytes, ehw_bytes;  // per stage
+  int off_eraw, off_w, off_ehw, off_out, off_bar;
+  int smem_bytes;
+};
+
+template <bool SPARSE, int BN, int NT>
+__global__ void __launch_bounds__(kThreadsGemm, 1)
+dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmE,
+                  const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
+                  const HaloParams p) {
+  using C = Cfg<SPARSE, BN>;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sA = smem;
+  uint8_t* sEraw = smem + p.off_eraw;
+  uint8_t* sW = smem + p.off_w;
+  uint8_t* sEhw = smem + p.off_ehw;
+  uint8_t* sOut = smem + p.off_out;
+  uint64_t* a_full = (uint64_t*)(smem + p.off_bar);
+  uint64_t* a_empty = a_full + kHaloAStages;
+  uint64_t* meta_full = a_empty + kHaloAStages;
+  uint64_t* w_ready = meta_full + kHaloAStages;  // W bytes landed AND (sparse) metadata tiles built
+  uint64_t* w_empty = w_ready + kMaxStages;
+  uint64_t* acc_full = w_empty + kMaxStages;
+  uint64_t* acc_empty = acc_full + 2;
+  uint64_t* meta_free = acc_empty + 2;
+  uint32_t* tmem_slot = (uint32_t*)(meta_free + 2);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();
+  unsigned int* err = &g_device_error;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kHaloAStages; ++s) {
+      ptx::mbar_init(&a_full[s], 1);
+      ptx::mbar_init(&a_empty[s], 1);
+      ptx::mbar_init(&meta_full[s], 1);
+    }
+    for (int s = 0; s < kMaxStages; ++s) {
+      // one arrival from the producer (with the byte count) plus, for sparse A, one from each
+      // metadata warp of both CTAs: the MMA thread waits once per tap
+      ptx::mbar_init(&w_ready[s], SPARSE ? 9 : 1);
+      ptx::mbar_init(&w_empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&acc_full[a], 1);
+      ptx::mbar_init(&acc_empty[a], 8);
+      ptx::mbar_init(&meta_free[a], 8);
+    }
+    ptx::fence_mbar_init();
+  }
+  if (warp == 0 && lane == 0) {
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+    ptx::prefetch_tensormap(&tmD);
+    if (SPARSE) ptx::prefetch_tensormap(&tmE);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before_sync();
+  ptx::cluster_sync();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int taps = p.R * p.S;
+  const int pair_stride = gridDim.x >> 1;
+  const int first_pair = blockIdx.x >> 1;
+  const int my_tiles = first_pair < p.pair_tiles ? (p.pair_tiles - first_pair + pair_stride - 1) / pair_stride : 0;
+  const int n_half = (int)rank * C::kBCols;
+  constexpr int set_cols = NT * BN;  // TMEM columns of one tile set's accumulators
+  const int WS = p.w_stages;
+  // tile set `pt` of this CTA: first input channel, first pixel column / row, image
+  auto locate = [&p, rank](int pt, int& n0, int& w0, int& h0, int& b0) -> bool {
+    n0 = (pt % p.tiles_n) * BN;
+    int t = 2 * (pt / p.tiles_n) + (int)rank;
+    const bool in_range = t < p.m_sets;  // a set past the last one loads zeros and stores nothing
+    w0 = (t % p.sets_w) * 8 * NT; t /= p.sets_w;
+    h0 = (t % p.tiles_h) * kHaloTH;
+    b0 = t / p.tiles_h;
+    return in_range;
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer
+    if (ptx::elect_one()) {
+      const uint32_t a_tx = 2u * (uint32_t)(p.img_rows * 128);
+      const uint32_t meta_tx = (uint32_t)(p.img_rows * 16);
+      const uint32_t w_tx = 2u * (uint32_t)C::kTapBBytes;
+      const int a_uses = my_tiles * p.k_blocks;
+      int ia = 0, ast = 0;
+      uint32_t aph = 0;
+      // Loads the A box (and raw metadata) of stage use `ia`. blocking == false: only if the
+      // stage is free right now. Returns 1 issued, 0 not free, -1 wait gave up.
+      auto issue_a = [&](bool blocking) -> int {
+        if (blocking) {
+          if (!ptx::mbar_wait(&a_empty[ast], aph ^ 1u, err, 0x100u + ast)) return -1;
+        } else if (!ptx::mbar_test(&a_empty[ast], aph ^ 1u)) {
+          return 0;
+        }
+        const int lt = ia / p.k_blocks, kb = ia - lt * p.k_blocks;
+        int n0, w0, h0, b0;
+        locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
+        const int q0 = w0 + p.pad_w - (p.S - 1), p0 = h0 + p.pad_h - (p.R - 1);
+        if (rank == 0) ptx::mbar_arrive_expect_tx(&a_full[ast], a_tx);
+        if (SPARSE) {
+          ptx::mbar_arrive_expect_tx(&meta_full[ast], meta_tx);
+          ptx::tma_load_4d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, p0, b0);
+        }
+        ptx::tma_load_4d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, p0, b0);
+        ++ia;
+        if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
+        return 1;
+      };
+      bool alive = true;
+      int wst = 0, use = 0;
+      uint32_t wph = 0;
+      for (int lt = 0; alive && lt < my_tiles; ++lt) {
+        const int pt = first_pair + lt * pair_stride;
+        const int n0 = (pt % p.tiles_n) * BN + n_half;
+        for (int kb = 0; alive && kb < p.k_blocks; ++kb, ++use) {
+          while (alive && ia <= use)
+            if (issue_a(true) < 0) alive = false;
+          for (int t = 0; alive && t < taps; ++t) {
+            // the next A box goes out as soon as its stage is released, between W taps
+            if (ia < a_uses && ia < use + kHaloAStages && issue_a(false) < 0) { alive = false; break; }
+            if (!ptx::mbar_wait(&w_empty[wst], wph ^ 1u, err, 0x180u + wst)) { alive = false; break; }
+            if (rank == 0) ptx::mbar_arrive_expect_tx(&w_ready[wst], w_tx);
+            const int r = t / p.S, s = t - r * p.S;
+            const int ft = (p.r_first + p.r_step * r) * p.S_full + p.s_first + p.s_step * s;
+#pragma unroll
+            for (int j = 0; j < C::kBoxes; ++j)
+              ptx::tma_load_2d_pair(sW + wst * p.w_bytes + j * C::kBoxBytes, &tmB, &w_ready[wst],
+                                    ft * p.Cin + n0 + C::kBoxCols * j, kb * C::kKB);
+            if (++wst == WS) { wst = 0; wph ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------- MMA issuer (first CTA only)
+    // One thread executes a few dependent instructions per ~10 clocks, so its path per tap is
+    // kept short: one barrier wait, running descriptor words updated by additions, compile-time
+    // offsets for the strips and the four MMAs of a channel block.
+    if (rank == 0 && ptx::elect_one()) {
+      constexpr uint32_t idesc = make_idesc(BN, SPARSE);
+      // descriptors as two 32-bit halves: the start address only ever changes the low word
+      const uint64_t adesc0 = ptx::make_smem_desc(0, 16, (uint32_t)p.pitch * 128u, 2);
+      const uint64_t bdesc0 = ptx::make_smem_desc(0, C::kBoxBytes, 8 * C::kRowB, C::kBSwizzle);
+      const uint64_t edesc0 = ptx::make_smem_desc(0, 128, 128, 0);
+      const uint32_t a_hi = (uint32_t)(adesc0 >> 32), b_hi = (uint32_t)(bdesc0 >> 32), e_hi = (uint32_t)(edesc0 >> 32);
+      const uint32_t a_lo0 = (uint32_t)adesc0 + (ptx::smem_u32(sA) >> 4);
+      const uint32_t b_lo0 = (uint32_t)bdesc0 + (ptx::smem_u32(sW) >> 4);
+      const uint32_t e_lo0 = (uint32_t)edesc0 + (ptx::smem_u32(sEhw) >> 4);
+      const uint32_t a_stage16 = (uint32_t)p.a_bytes >> 4, w_stage16 = (uint32_t)p.w_bytes >> 4,
+                     e_stage16 = (uint32_t)p.ehw_bytes >> 4;
+      const uint32_t a_first16 = (uint32_t)(((p.R - 1) * p.pitch + (p.S - 1)) * 8);  // tap (0,0), in 16-byte units
+      const uint32_t a_rowstep16 = (uint32_t)((p.pitch - (p.S - 1)) * 8);            // last tap of a filter row -> first of the next
+      constexpr uint32_t kBStep = (uint32_t)((C::kKB / 4) * C::kRowB / 16);  // W rows of one MMA
+      constexpr uint32_t kSlotCols = 4u * NT;                                // metadata columns of one W stage
+      bool alive = true;
+      int ast = 0, acc = 0, wst = 0;
+      uint32_t aph = 0, wph = 0, cph = 0;
+      // running words of the W ring: W descriptor, metadata descriptor, metadata column (relative)
+      uint32_t b_lo = b_lo0, e_lo = e_lo0, mcol = 0;
+      for (int lt = 0; alive && lt < my_tiles; ++lt) {
+        if (!ptx::mbar_wait(&acc_empty[acc], cph ^ 1u, err, 0x200u + acc)) break;
+        // shared metadata region: the first columns of the other tile set's accumulators,
+        // which the epilogue of the previous tile set reads out first
+        if (p.meta_shared && lt > 0 &&
+            !ptx::mbar_wait(&meta_free[acc ^ 1], (((uint32_t)lt - 1u) >> 1) & 1u, err, 0x800u + acc))
+          break;
+        const uint32_t meta_base = tmem_base + (uint32_t)(p.meta_shared ? (acc ^ 1) * set_cols : p.meta_col);
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * set_cols);
+        uint32_t accumulate = 0u;
+        for (int kb = 0; alive && kb < p.k_blocks; ++kb) {
+          if (!ptx::mbar_wait(&a_full[ast], aph, err, 0x300u + ast)) { alive = false; break; }
+          uint32_t a_lo = a_lo0 + (uint32_t)ast * a_stage16 + a_first16;
+          int s = p.S;
+          for (int t = 0; t < taps; ++t) {
+            if (!ptx::mbar_wait(&w_ready[wst], wph, err, 0x380u + wst)) { alive = false; break; }
+            ptx::tc_fence_after_sync();
+            const uint32_t e_col = meta_base + mcol;  // even: slots are 4 columns apart
+            if (SPARSE) {
+#pragma unroll
+              for (int j = 0; j < NT; ++j)
+                ptx::tc_cp_128x128b_pair(e_col + 4u * j, ((uint64_t)e_hi << 32) | (e_lo + (uint32_t)(j * (kEHwBytes / 16))));
+            }
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                // strip j: 8 pixels = 1024 bytes to the right; MMA q: 32 bytes along the row
+                const uint64_t a_q = ((uint64_t)a_hi << 32) | (a_lo + (uint32_t)(j * 64 + q * 2));
+                const uint64_t b_q = ((uint64_t)b_hi << 32) | (b_lo + (uint32_t)q * kBStep);
+                if (SPARSE)
+                  ptx::mma_sp_f16_ss_pair(d_tmem + (uint32_t)(j * BN), a_q, b_q, e_col + (uint32_t)(4 * j + (q & 2)),
+                                          idesc | (uint32_t)(q & 1), q == 0 ? accumulate : 1u);
+                else
+                  ptx::mma_f16_ss_pair(d_tmem + (uint32_t)(j * BN), a_q, b_q, idesc, q == 0 ? accumulate : 1u);
+              }
+            }
+            ptx::tc_commit_pair(&w_empty[wst], 3);
+            accumulate = 1u;
+            // next tap: one pixel to the left, or the end of the filter row above
+            if (--s == 0) { s = p.S; a_lo -= a_rowstep16; } else { a_lo -= 8u; }
+            if (++wst == WS) { wst = 0; wph ^= 1u; b_lo = b_lo0; e_lo = e_lo0; mcol = 0; }
+            else { b_lo += w_stage16; e_lo += e_stage16; mcol += kSlotCols; }
+          }
+          if (alive) ptx::tc_commit_pair(&a_empty[ast], 3);
+          if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
+        }
+        if (alive) ptx::tc_commit_pair(&acc_full[acc], 3);
+        if (++acc == 2) { acc = 0; cph ^= 1u; }
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------- metadata rearranger
+    if (SPARSE) {
+      // thread = TMEM lane: pixel column w of strip rows 2*h2 and 2*h2+1, channel half `half`
+      const int tl = threadIdx.x - 64;
+      const int w = tl & 7, h2 = tl >> 4;
+      const uint32_t sel = (tl & 8) ? 0x7632u : 0x5410u;
+      bool alive = true;
+      int ast = 0, wst = 0;
+      uint32_t aph = 0, wph = 0;
+      for (int lt = 0; alive && lt < my_tiles; ++lt) {
+        for (int kb = 0; alive && kb < p.k_blocks; ++kb) {
+          if (!ptx::mbar_wait(&meta_full[ast], aph, err, 0x500u + ast)) { alive = false; break; }
+          const uint8_t* raw = sEraw + ast * p.eraw_bytes;
+          int r = 0, s = 0;
+          for (int t = 0; t < taps; ++t) {
+            // the stage's previous tiles have been copied to TMEM and used
+            if (!ptx::mbar_wait(&w_empty[wst], wph ^ 1u, err, 0x580u + wst)) { alive = false; break; }
+            const int px = (2 * h2 + (p.R - 1 - r)) * p.pitch + w + (p.S - 1 - s);
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+              const uint4 lo = *(const uint4*)(raw + (px + 8 * j) * 16);
+              const uint4 hi = *(const uint4*)(raw + (px + 8 * j + p.pitch) * 16);
+              uint32_t x[4] = {prmt(lo.x, hi.x, sel), prmt(lo.y, hi.y, sel), prmt(lo.z, hi.z, sel),
+                               prmt(lo.w, hi.w, sel)};
+#pragma unroll
+              for (int k2 = 0; k2 < 4; ++k2) {
+                // pixels outside the image carry no metadata: give them the well-formed pair (0,1)
+                if ((x[k2] & 0xFFFFu) == 0u) x[k2] |= 0x4444u;
+                if ((x[k2] >> 16) == 0u) x[k2] |= 0x44440000u;
+              }
+              *(uint4*)(sEhw + wst * p.ehw_bytes + j * kEHwBytes + tl * 16) = make_uint4(x[0], x[1], x[2], x[3]);
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(&w_ready[wst], 0);
+            if (++wst == WS) { wst = 0; wph ^= 1u; }
+            if (++s == p.S) { s = 0; ++r; }
+          }
+          if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const bool issuer = (threadIdx.x == 192);
+    uint32_t chunk = 0, cph = 0;
+    int acc = 0;
+    for (int lt = 0; lt < my_tiles; ++lt) {
+      int n0, w0, h0, b0;
+      const bool in_range = locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
+      if (!ptx::mbar_wait(&acc_full[acc], cph, err, 0x600u + acc)) break;
+      ptx::tc_fence_after_sync();
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+        store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * set_cols + j * BN), sOut,
+                              p.out_bufs, &tmD, n0, w0 + 8 * j, h0, b0, in_range && (w0 + 8 * j < p.W), row, issuer,
+                              chunk, (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr);
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
+      if (++acc == 2) { acc = 0; cph ^= 1u; }
+    }
+    if (issuer) ptx::bulk_wait_group_all();
+  }
+
+  __syncwarp();
+  if (*(volatile unsigned int*)err != 0u) {
+    const uint64_t t0 = ptx::globaltimer_ns();
+    while (ptx::globaltimer_ns() - t0 < 200000ull) {
+    }
+  }
+  ptx::tc_fence_before_sync();
+  __syncwarp();
+  ptx::cluster_sync();
+  ptx::tc_fence_after_sync();
+  if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+}
+
 // ------------------------------------------------------------------- host
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -715,6 +1049,150 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const Dg
   return cudaLaunchKernelEx(&cfg, kernel, tmA, tmE, tmB, tmD, p) == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
+// Shared-memory and TMEM plan of the whole-filter-reuse kernel. Returns false if it does not fit.
+template <bool SPARSE, int BN>
+bool plan_halo(HaloParams* p, int nt) {
+  using C = Cfg<SPARSE, BN>;
+  const int budget = kSmemLimit - kSmemSlack;
+  {
+    if (nt * BN > 256) return false;         // two tile sets of accumulators must fit the 512 TMEM columns
+    if (nt == 2 && p->W <= 8) return false;  // a second strip would be empty
+    p->nt = nt;
+    p->pitch = 8 * nt + p->S - 1;
+    p->img_h = kHaloTH + p->R - 1;
+    p->img_rows = p->pitch * p->img_h;
+    if (p->pitch > 256 || p->img_h > 256) return false;
+    p->a_bytes = round_up(p->img_rows * 128, 1024);
+    p->eraw_bytes = SPARSE ? round_up(p->img_rows * 16, 128) : 0;
+    p->w_bytes = C::kTapBBytes;
+    p->ehw_bytes = SPARSE ? nt * kEHwBytes : 0;
+    const int fixed = kHaloAStages * (p->a_bytes + p->eraw_bytes) + 1024;
+    int out_bufs = 2;
+    int w_stages = (budget - fixed - out_bufs * kOutBytes) / (p->w_bytes + p->ehw_bytes);
+    if (w_stages < 4) {
+      out_bufs = 1;
+      w_stages = (budget - fixed - out_bufs * kOutBytes) / (p->w_bytes + p->ehw_bytes);
+    }
+    if (w_stages > kMaxStages) w_stages = kMaxStages;
+    p->meta_shared = 0;
+    p->meta_col = 2 * nt * BN;
+    if (SPARSE) {
+      const int slot_cols = 4 * nt;  // TMEM columns of one W stage's metadata
+      const int free_cols = (int)kTmemCols - 2 * nt * BN;
+      if (free_cols >= 3 * slot_cols) {
+        if (w_stages > free_cols / slot_cols) w_stages = free_cols / slot_cols;
+      } else {
+        p->meta_shared = 1;  // slots live in the first 64 columns of the tile set being read out
+        p->meta_col = 0;
+        if (w_stages > 64 / slot_cols) w_stages = 64 / slot_cols;
+      }
+    }
+    if (w_stages < 3) return false;
+    p->w_stages = w_stages;
+    p->out_bufs = out_bufs;
+    p->off_eraw = kHaloAStages * p->a_bytes;
+    p->off_w = round_up(p->off_eraw + kHaloAStages * p->eraw_bytes, 1024);
+    p->off_ehw = p->off_w + w_stages * p->w_bytes;
+    p->off_out = round_up(p->off_ehw + w_stages * p->ehw_bytes, 1024);
+    p->off_bar = p->off_out + out_bufs * kOutBytes;
+    p->smem_bytes = p->off_bar + 512 + 1024;
+    if (p->smem_bytes > kSmemLimit) return false;
+    p->sets_w = (p->W + 8 * nt - 1) / (8 * nt);
+    p->tiles_h = (p->H + kHaloTH - 1) / kHaloTH;
+    const int64_t m_sets = (int64_t)p->sets_w * p->tiles_h * p->B;
+    if (m_sets * p->tiles_n > 0x3FFFFFFF) return false;
+    p->m_sets = (int)m_sets;
+    p->pair_tiles = (int)((m_sets + 1) / 2) * p->tiles_n;
+    return true;
+  }
+  return false;
+}
+
+// Whole-filter reuse pays when there is more than one tap and strips of 8 x 16 pixels cover the
+// image without much padding.
+bool halo_applies(int H, int W, int taps) {
+  if (taps < 2 || W < 8 || H < 12) return false;
+  const int64_t covered = (int64_t)((W + 7) / 8 * 8) * ((H + kHaloTH - 1) / kHaloTH * kHaloTH);
+  return covered * 100 <= (int64_t)H * W * 135;
+}
+
+template <bool SPARSE, int BN, int NT>
+sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, const DgradView& view, HaloParams p,
+                           cudaStream_t stream) {
+  using C = Cfg<SPARSE, BN>;
+  if (!plan_halo<SPARSE, BN>(&p, NT)) return SDGP_ERR_UNSUPPORTED;
+
+  CUtensorMap tmA, tmE, tmB, tmD;
+  const int P = view.P, Q = view.Q;
+  const uint64_t CA = SPARSE ? (uint64_t)view.a_channels / 2 : (uint64_t)view.a_channels;
+  {
+    const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
+    const uint64_t strides[3] = {CA * 2, CA * 2 * Q, CA * 2 * Q * P};
+    const uint32_t box[4] = {64, (uint32_t)p.pitch, (uint32_t)p.img_h, 1};
+    if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+      return SDGP_ERR_CUDA;
+  }
+  if (SPARSE) {
+    const uint64_t CE = (uint64_t)view.a_channels / 16;
+    const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
+    const uint64_t strides[3] = {CE * 2, CE * 2 * Q, CE * 2 * Q * P};
+    const uint32_t box[4] = {8, (uint32_t)p.pitch, (uint32_t)p.img_h, 1};
+    if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
+      return SDGP_ERR_CUDA;
+  } else {
+    tmE = tmA;
+  }
+  {
+    const uint64_t dims[2] = {(uint64_t)view.w_cols, (uint64_t)p.Cout};
+    const uint64_t strides[1] = {(uint64_t)view.w_cols * 2};
+    const uint32_t box[2] = {(uint32_t)C::kBoxCols, (uint32_t)C::kKB};
+    if (!encode(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Wt, dims, strides, box,
+                C::kRowB == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
+      return SDGP_ERR_CUDA;
+  }
+  {
+    const uint64_t dims[4] = {(uint64_t)p.Cin, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.B};
+    const uint64_t strides[3] = {view.d_stride_w, view.d_stride_h, view.d_stride_b};
+    const uint32_t box[4] = {64, 8, (uint32_t)kHaloTH, 1};
+    if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, view.d_base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+      return SDGP_ERR_CUDA;
+  }
+
+  static bool configured = false;
+  auto kernel = dgrad_halo_kernel<SPARSE, BN, NT>;
+  if (!configured) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
+      return SDGP_ERR_CUDA;
+    configured = true;
+  }
+  const int max_pairs = sm_count() / 2;
+  const int pairs = p.pair_tiles < max_pairs ? p.pair_tiles : max_pairs;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3(kThreadsGemm);
+  cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, tmA, tmE, tmB, tmD, p) == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
+}
+
+// Two strips per CTA where the accumulators of two tile sets fit TMEM, else one.
+template <bool SPARSE, int BN>
+sdgp_status launch_halo(const void* A, const void* meta, const void* Wt, const DgradView& view, const HaloParams& p,
+                        cudaStream_t stream) {
+  if (BN <= 128) {
+    const sdgp_status st = launch_halo_nt<SPARSE, (BN <= 128 ? BN : 64), 2>(A, meta, Wt, view, p, stream);
+    if (st != SDGP_ERR_UNSUPPORTED) return st;
+  }
+  return launch_halo_nt<SPARSE, BN, 1>(A, meta, Wt, view, p, stream);
+}
+
 }  // namespace
 
 // A: dense dL/dO [B,P,Q,Cout] (sparse == false) or compressed values [B,P,Q,a_channels/2] with
@@ -783,7 +1261,26 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
       view.d_stride_w = (uint64_t)stride * Cin * 2;
       view.d_stride_h = (uint64_t)stride * W * Cin * 2;
       view.d_stride_b = (uint64_t)H * W * Cin * 2;
-      sdgp_status st;
+      sdgp_status st = SDGP_ERR_UNSUPPORTED;
+      if (!fused && halo_applies(Hs, Ws, p.R * p.S)) {
+        HaloParams hp = {};
+        hp.B = B; hp.H = Hs; hp.W = Ws; hp.Cin = Cin; hp.Cout = Cout;
+        hp.R = p.R; hp.S = p.S; hp.pad_h = p.pad_h; hp.pad_w = p.pad_w;
+        hp.r_first = p.r_first; hp.r_step = p.r_step; hp.s_first = p.s_first; hp.s_step = p.s_step;
+        hp.S_full = S;
+        hp.tiles_n = p.tiles_n; hp.k_blocks = p.k_blocks;
+        if (sparse) {
+          st = BN == 256 ? launch_halo<true, 256>(A, meta, Wt, view, hp, stream)
+             : BN == 128 ? launch_halo<true, 128>(A, meta, Wt, view, hp, stream)
+                         : launch_halo<true, 64>(A, meta, Wt, view, hp, stream);
+        } else {
+          st = BN == 256 ? launch_halo<false, 256>(A, meta, Wt, view, hp, stream)
+             : BN == 128 ? launch_halo<false, 128>(A, meta, Wt, view, hp, stream)
+                         : launch_halo<false, 64>(A, meta, Wt, view, hp, stream);
+        }
+        if (st == SDGP_OK) continue;
+        if (st != SDGP_ERR_UNSUPPORTED) return st;  // otherwise: does not fit, use the general kernel
+      }
       if (fused) {
         st = BN == 256 ? launch_cfg<true, 256, true>(A, meta, Wt, view, p, stream)
            : BN == 128 ? launch_cfg<true, 128, true>(A, meta, Wt, view, p, stream)
