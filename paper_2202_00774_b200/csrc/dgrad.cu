@@ -574,9 +574,9 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ptx::mbar_init(&meta_full[s], 1);
     }
     for (int s = 0; s < kMaxStages; ++s) {
-      // one arrival from the producer (with the byte count) plus, for sparse A, one from each
-      // metadata warp of both CTAs: the MMA thread waits once per tap
-      ptx::mbar_init(&w_ready[s], SPARSE ? 9 : 1);
+      // one arrival from the producer (with the byte count) plus, for sparse A, one from the
+      // metadata warp of each CTA that built the tap: the MMA thread waits once per tap
+      ptx::mbar_init(&w_ready[s], SPARSE ? 3 : 1);
       ptx::mbar_init(&w_empty[s], 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -756,44 +756,51 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   } else if (warp < 6) {
     // ------------------------------------------------- metadata rearranger
     if (SPARSE) {
-      // thread = TMEM lane: pixel column w of strip rows 2*h2 and 2*h2+1, channel half `half`
-      const int tl = threadIdx.x - 64;
-      const int w = tl & 7, h2 = tl >> 4;
-      const uint32_t sel = (tl & 8) ? 0x7632u : 0x5410u;
-      bool alive = true;
-      int ast = 0, wst = 0;
-      uint32_t aph = 0, wph = 0;
-      for (int lt = 0; alive && lt < my_tiles; ++lt) {
-        for (int kb = 0; alive && kb < p.k_blocks; ++kb) {
-          if (!ptx::mbar_wait(&meta_full[ast], aph, err, 0x500u + ast)) { alive = false; break; }
-          const uint8_t* raw = sEraw + ast * p.eraw_bytes;
-          int r = 0, s = 0;
-          for (int t = 0; t < taps; ++t) {
-            // the stage's previous tiles have been copied to TMEM and used
-            if (!ptx::mbar_wait(&w_empty[wst], wph ^ 1u, err, 0x580u + wst)) { alive = false; break; }
-            const int px = (2 * h2 + (p.R - 1 - r)) * p.pitch + w + (p.S - 1 - s);
+      // A lone warp runs a dependent instruction chain slowly, so the four warps do not share
+      // one tap: warp k builds the metadata of W-ring uses k, k+4, k+8, ... (a whole TMEM image
+      // per strip: four passes of 32 lanes), four taps in flight.
+      // lane = pixel column w, channel half, and odd/even pair of strip rows within a pass
+      const int w = lane & 7, hsub = lane >> 4;
+      const uint32_t sel = (lane & 8) ? 0x7632u : 0x5410u;
+      const int total_uses = my_tiles * p.k_blocks * taps;
+      int t = warp - 2;  // tap within the channel block
+      int ause = 0;      // A stage use = (tile set, channel block)
+      while (t >= taps) { t -= taps; ++ause; }
+      int wst = warp - 2;
+      uint32_t wph = 0;
+      while (wst >= WS) { wst -= WS; wph ^= 1u; }
+      for (int u = warp - 2; u < total_uses; u += 4) {
+        const int ast = ause & 1;  // kHaloAStages == 2
+        if (!ptx::mbar_wait(&meta_full[ast], (uint32_t)(ause >> 1) & 1u, err, 0x500u + ast)) break;
+        // the stage's previous tiles have been copied to TMEM and used
+        if (!ptx::mbar_wait(&w_empty[wst], wph ^ 1u, err, 0x580u + wst)) break;
+        const int r = t / p.S, s = t - r * p.S;
+        const uint8_t* raw = sEraw + ast * p.eraw_bytes;
+        uint8_t* dst = sEhw + wst * p.ehw_bytes + lane * 16;
+        // TMEM lane 32*i + lane holds strip rows 2*h2 and 2*h2 + 1 with h2 = 2*i + hsub
+        const int px0 = (2 * hsub + (p.R - 1 - r)) * p.pitch + w + (p.S - 1 - s);
 #pragma unroll
-            for (int j = 0; j < NT; ++j) {
-              const uint4 lo = *(const uint4*)(raw + (px + 8 * j) * 16);
-              const uint4 hi = *(const uint4*)(raw + (px + 8 * j + p.pitch) * 16);
-              uint32_t x[4] = {prmt(lo.x, hi.x, sel), prmt(lo.y, hi.y, sel), prmt(lo.z, hi.z, sel),
-                               prmt(lo.w, hi.w, sel)};
+        for (int i = 0; i < 4; ++i) {
 #pragma unroll
-              for (int k2 = 0; k2 < 4; ++k2) {
-                // pixels outside the image carry no metadata: give them the well-formed pair (0,1)
-                if ((x[k2] & 0xFFFFu) == 0u) x[k2] |= 0x4444u;
-                if ((x[k2] >> 16) == 0u) x[k2] |= 0x44440000u;
-              }
-              *(uint4*)(sEhw + wst * p.ehw_bytes + j * kEHwBytes + tl * 16) = make_uint4(x[0], x[1], x[2], x[3]);
-            }
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(&w_ready[wst], 0);
-            if (++wst == WS) { wst = 0; wph ^= 1u; }
-            if (++s == p.S) { s = 0; ++r; }
+          for (int j = 0; j < NT; ++j) {
+            const int px = px0 + 4 * i * p.pitch + 8 * j;
+            uint4 lo = *(const uint4*)(raw + px * 16);
+            uint4 hi = *(const uint4*)(raw + (px + p.pitch) * 16);
+            // pixels outside the image carry no metadata (TMA fills zeros; real metadata is never
+            // zero): give them the well-formed position pair (0,1) in every chunk
+            if (lo.x == 0u) lo = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+            if (hi.x == 0u) hi = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+            *(uint4*)(dst + j * kEHwBytes + i * 512) =
+                make_uint4(prmt(lo.x, hi.x, sel), prmt(lo.y, hi.y, sel), prmt(lo.z, hi.z, sel), prmt(lo.w, hi.w, sel));
           }
-          if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
         }
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive_cluster(&w_ready[wst], 0);
+        t += 4;
+        while (t >= taps) { t -= taps; ++ause; }
+        wst += 4;
+        while (wst >= WS) { wst -= WS; wph ^= 1u; }
       }
     }
   } else {
