@@ -22,13 +22,16 @@
 //               arrive as zeros), the matching box of metadata, and the W boxes of its half.
 //   warp 1      MMA issuer (first CTA only): tcgen05.cp of the stage's metadata into TMEM,
 //               four MMAs per (tap, channel block), tcgen05.commit to the stage's "empty" barrier.
-//   warps 2-5   (sparse only) rearrange metadata from the row-major order TMA delivers into
-//               the lane/column order the tensor core reads from TMEM (one thread per A-tile row).
+//   warps 2-5   (sparse only) build the stage's metadata images: from the row-major order TMA
+//               delivers to the lane/column order the tensor core reads from TMEM. Each warp
+//               takes every fourth stage use (four stages in flight); with fused pruning the
+//               four warps first prune the stage's pixel rows together.
 //   warps 6-9   epilogue: TMEM -> registers -> bf16 -> swizzled staging tile -> TMA store,
 //               overlapped with the next tile's main loop through a second accumulator.
 //
-// Barriers: full / meta_ready / acc_empty / w_full are waited on by the first CTA only and
-// collect arrivals from both; empty / acc_full exist in both CTAs and are signalled together
+// Barriers: full / acc_empty / w_full are waited on by the first CTA only and collect arrivals
+// from both (full: the producer's byte count plus the metadata warps' arrivals, so the MMA
+// thread waits once per stage); empty / acc_full exist in both CTAs and are signalled together
 // by a multicast tcgen05.commit; meta_full is local (each CTA's own metadata box).
 // Every wait is bounded: a wait that runs out records a code in g_device_error, the role
 // stops issuing work, every other wait then gives up at once, and the kernel frees its TMEM
@@ -105,25 +108,25 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool sparse) {
          ((uint32_t)(256 >> 4) << 24) | (sparse ? (1u << 2) : 0u);
 }
 
-// One row of metadata: from the row-major order TMA delivers (8 uint16 per pixel, one per 16
-// channels) to the order tcgen05.cp moves into TMEM. For the MMA covering channels
-// [32*k2, 32*k2+32) of the block the tensor core reads one 32-bit TMEM column: lane
-// (row%8) + 8*half + 16*(row/16) holds in its low 16 bits the four position nibbles of channels
-// 32*k2 + 16*half + [0,16) of the row with bit 3 clear and in its high 16 bits those of row + 8.
-__device__ __forceinline__ void rearrange_metadata_row(const uint8_t* raw_rows, uint8_t* hw_tile, int row,
-                                                       int rows_used) {
-  const uint4 raw = *(const uint4*)(raw_rows + row * 16);
-  const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
-  uint16_t* hw = (uint16_t*)hw_tile;
-#pragma unroll
-  for (int u = 0; u < 8; ++u) {
-    uint32_t v = (u & 1) ? (w4[u >> 1] >> 16) : (w4[u >> 1] & 0xFFFFu);
-    // rows outside the patch or outside the image carry no data: give them the well-formed
-    // position pair (0,1) in every chunk
-    if (row >= rows_used || v == 0u) v = 0x4444u;
-    const int tl = (row & 7) + 8 * (u & 1) + 16 * (row >> 4);
-    hw[tl * 8 + 2 * (u >> 1) + ((row >> 3) & 1)] = (uint16_t)v;
-  }
+// Metadata of an A tile: from the row-major order TMA delivers (16 bytes per pixel row: one uint16
+// per 16 channels of a 128-channel block) to the order tcgen05.cp moves into TMEM. For the MMA
+// covering channels [32*k2, 32*k2+32) of the block the tensor core reads one 32-bit TMEM column:
+// lane (row%8) + 8*half + 16*(row/16) holds in its low 16 bits the four position nibbles of
+// channels 32*k2 + 16*half + [0,16) of the row with bit 3 clear, in its high 16 bits those of
+// row + 8. One call builds the 16 bytes of TMEM lane `tl` from its two rows. Rows that carry no
+// data (past the patch, or outside the image where TMA filled zeros - real metadata is never
+// zero) get the well-formed position pair (0,1) in every chunk.
+__device__ __forceinline__ void build_metadata_lane(const uint8_t* raw_rows, uint8_t* hw_tile, int tl, int rows_used) {
+  const int row_a = ((tl >> 4) << 4) + (tl & 7), row_b = row_a + 8;
+  const uint32_t sel = (tl & 8) ? 0x7632u : 0x5410u;
+  const uint4 k01 = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+  uint4 lo = k01, hi = k01;
+  if (row_a < rows_used) lo = *(const uint4*)(raw_rows + row_a * 16);
+  if (row_b < rows_used) hi = *(const uint4*)(raw_rows + row_b * 16);
+  if (lo.x == 0u) lo = k01;
+  if (hi.x == 0u) hi = k01;
+  *(uint4*)(hw_tile + tl * 16) =
+      make_uint4(prmt(lo.x, hi.x, sel), prmt(lo.y, hi.y, sel), prmt(lo.z, hi.z, sel), prmt(lo.w, hi.w, sel));
 }
 
 // Fused pruning of one pixel row of a stage: 128 dense channels (two 128-byte-swizzled boxes of
@@ -161,23 +164,23 @@ __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* stagi
 #pragma unroll 1
   for (int c0 = 0; c0 < BN; c0 += 64, ++chunk) {
     uint32_t packed[32];
-#pragma unroll
-    for (int part = 0; part < 2; ++part) {
-      uint32_t v[32];
-      ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32 * part), v);
-      ptx::tmem_ld_wait();
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
-        packed[16 * part + e] = *(const uint32_t*)&h2;
-      }
-    }
+    uint32_t v0[32], v1[32];
+    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v0);
+    ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32), v1);
+    ptx::tmem_ld_wait();
     if (c0 == 0 && first_slab_read != nullptr) {
       // the accumulator's first 64 columns are in registers: they may now hold the next
-      // tile's metadata
+      // tile's metadata (signalled before the conversion work, the MMA thread is waiting)
       ptx::tc_fence_before_sync();
       __syncwarp();
       if ((threadIdx.x & 31) == 0) ptx::mbar_arrive_cluster(first_slab_read, 0);
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const __nv_bfloat162 a2 = __floats2bfloat162_rn(__uint_as_float(v0[2 * e]), __uint_as_float(v0[2 * e + 1]));
+      const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v1[2 * e]), __uint_as_float(v1[2 * e + 1]));
+      packed[e] = *(const uint32_t*)&a2;
+      packed[16 + e] = *(const uint32_t*)&b2;
     }
     uint8_t* buf = staging + (out_bufs == 2 ? (chunk & 1u) : 0u) * kOutBytes;
     if (issuer) {  // the store that last used this slab has finished reading it
@@ -218,8 +221,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   uint64_t* full = (uint64_t*)(smem + p.off_bar);
   uint64_t* empty = full + kMaxStages;
   uint64_t* meta_full = empty + kMaxStages;
-  uint64_t* meta_ready = meta_full + kMaxStages;
-  uint64_t* acc_full = meta_ready + kMaxStages;
+  uint64_t* acc_full = meta_full + kMaxStages;
   uint64_t* acc_empty = acc_full + 2;
   uint64_t* w_full = acc_empty + 2;
   uint64_t* meta_free = w_full + 1;
@@ -235,11 +237,13 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
-      ptx::mbar_init(&full[s], 1);
+      // full: the producer's arrival (with the stage's byte count) plus, for sparse A, the
+      // arrivals of the warps that built the stage's metadata images in both CTAs (one warp per
+      // CTA; all four when they also prune) - the MMA thread waits once per stage
+      ptx::mbar_init(&full[s], SPARSE ? (FUSED ? 9 : 3) : 1);
       ptx::mbar_init(&empty[s], 1);
       ptx::mbar_init(&meta_full[s], 1);
       ptx::mbar_init(&raw_full[s], 1);
-      ptx::mbar_init(&meta_ready[s], 8);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&acc_full[a], 1);
@@ -272,6 +276,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   const int uses_per_tile = groups * p.k_blocks;
   const int pair_stride = gridDim.x >> 1;
   const int first_pair = blockIdx.x >> 1;
+  const int my_tiles = first_pair < p.pair_tiles ? (p.pair_tiles - first_pair + pair_stride - 1) / pair_stride : 0;
   const int n_half = (int)rank * C::kBCols;  // this CTA's column offset inside the BN block
 
   if (warp == 0) {
@@ -340,26 +345,37 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     }
   } else if (warp == 1) {
     // ------------------------------------------- MMA issuer (first CTA only)
+    // A single thread executes roughly one dependent instruction per ten clocks, so its path
+    // per stage is short: one barrier wait, descriptor words kept as running sums.
     if (rank == 0 && ptx::elect_one()) {
       constexpr uint32_t idesc = make_idesc(BN, SPARSE);
       bool alive = true;
       if (p.w_resident) alive = ptx::mbar_wait(w_full, 0u, err, 0x700u);
-      // descriptor constants; the 14-bit address field is added per use (all addresses < 256 KiB)
+      // descriptors as two 32-bit halves: the start address only ever changes the low word
       const uint64_t adesc0 = ptx::make_smem_desc(0, 16, 1024, 2);
       const uint64_t bdesc0 = ptx::make_smem_desc(0, C::kBoxBytes, 8 * C::kRowB, C::kBSwizzle);
       const uint64_t edesc0 = ptx::make_smem_desc(0, 128, 128, 0);
-      const uint32_t sA_u = ptx::smem_u32(sA), sB_u = ptx::smem_u32(sB), sW_u = ptx::smem_u32(sW),
-                     sE_u = ptx::smem_u32(sEhw);
+      const uint32_t a_hi = (uint32_t)(adesc0 >> 32), b_hi = (uint32_t)(bdesc0 >> 32), e_hi = (uint32_t)(edesc0 >> 32);
+      const uint32_t a_lo0 = (uint32_t)adesc0 + (ptx::smem_u32(sA) >> 4);
+      const uint32_t b_lo0 = (uint32_t)bdesc0 + (ptx::smem_u32(sB) >> 4);
+      const uint32_t w_lo0 = (uint32_t)bdesc0 + (ptx::smem_u32(sW) >> 4);
+      const uint32_t e_lo0 = (uint32_t)edesc0 + (ptx::smem_u32(sEhw) >> 4);
+      const uint32_t a_stage16 = (uint32_t)p.a_bytes >> 4, b_stage16 = (uint32_t)p.b_bytes >> 4,
+                     e_stage16 = (uint32_t)p.ehw_bytes >> 4;
+      constexpr uint32_t kTapB16 = (uint32_t)C::kTapBBytes >> 4;
+      constexpr uint32_t kBStep = (uint32_t)((C::kKB / 4) * C::kRowB / 16);  // W rows of one MMA
+      const uint32_t slot_cols = 4u * (uint32_t)p.rr;                         // metadata columns of one stage
       int st = 0, acc = 0;
-      uint32_t ph = 0, aph = 0, lt = 0;
-      for (int pt = first_pair; alive && pt < p.pair_tiles; pt += pair_stride, ++lt) {
+      uint32_t ph = 0, aph = 0;
+      uint32_t a_lo = a_lo0, b_lo = b_lo0, e_lo = e_lo0, mcol = 0;  // running words of the stage ring
+      for (int lt = 0; alive && lt < my_tiles; ++lt) {
         if (!ptx::mbar_wait(&acc_empty[acc], aph ^ 1u, err, 0x200u + acc)) break;
         // Shared metadata region: this tile's slots are the first columns of the other
         // accumulator, which the epilogue of the previous tile must have read out first.
         if (p.meta_shared && lt > 0 &&
-            !ptx::mbar_wait(&meta_free[acc ^ 1], ((lt - 1u) >> 1) & 1u, err, 0x800u + acc))
+            !ptx::mbar_wait(&meta_free[acc ^ 1], (((uint32_t)lt - 1u) >> 1) & 1u, err, 0x800u + acc))
           break;
-        const int meta_base = p.meta_shared ? (acc ^ 1) * BN : p.meta_col;
+        const uint32_t meta_base = tmem_base + (uint32_t)(p.meta_shared ? (acc ^ 1) * BN : p.meta_col);
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         uint32_t accumulate = 0u;
@@ -367,38 +383,34 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         for (int g = 0; alive && g < groups; ++g) {
           for (int cb = 0; cb < p.k_blocks; ++cb) {
             if (!ptx::mbar_wait(&full[st], ph, err, 0x300u + st)) { alive = false; break; }
-            if (SPARSE && !ptx::mbar_wait(&meta_ready[st], ph, err, 0x400u + st)) { alive = false; break; }
             ptx::tc_fence_after_sync();
-            const uint32_t meta_slot = (uint32_t)(meta_base + st * p.rr * 4);
+            const uint32_t e_col = meta_base + mcol;  // even: slots are multiples of 4 columns apart
             if (SPARSE) {
               for (int u = 0; u < p.rr; ++u)
-                ptx::tc_cp_128x128b_pair(tmem_base + meta_slot + 4u * u,
-                                         edesc0 + ((sE_u + st * p.ehw_bytes + u * kEHwBytes) >> 4));
+                ptx::tc_cp_128x128b_pair(e_col + 4u * u, ((uint64_t)e_hi << 32) | (e_lo + (uint32_t)(u * (kEHwBytes / 16))));
             }
             for (int u = 0; u < p.rr; ++u) {
               // vertical tap r: the tile's rows start (R-1-r) image rows into the stage
               const int r = reuse ? u : r_single;
-              const int row_off = reuse ? (p.R - 1 - r) * p.TW : 0;
-              const uint32_t b_addr = p.w_resident ? sW_u + ((r * p.S + s) * p.k_blocks + cb) * C::kTapBBytes
-                                                   : sB_u + st * p.b_bytes + u * C::kTapBBytes;
-              const uint64_t adesc = adesc0 + ((sA_u + st * p.a_bytes + row_off * 128) >> 4);
-              const uint64_t bdesc = bdesc0 + (b_addr >> 4);
+              const uint32_t a_u = a_lo + (reuse ? (uint32_t)((p.R - 1 - r) * p.TW * 8) : 0u);
+              const uint32_t b_u = p.w_resident ? w_lo0 + (uint32_t)((r * p.S + s) * p.k_blocks + cb) * kTapB16
+                                                : b_lo + (uint32_t)u * kTapB16;
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
+              for (int q = 0; q < 4; ++q) {
                 // A: 32 bytes of a 128-byte swizzled row per MMA; B: 16 (dense) or 32 (sparse) rows
-                const uint64_t a_j = adesc + (uint64_t)(j * 2);
-                const uint64_t b_j = bdesc + (uint64_t)(j * (C::kKB / 4) * C::kRowB / 16);
-                if (SPARSE) {
-                  const uint32_t col = meta_slot + 4u * u + j;
-                  ptx::mma_sp_f16_ss_pair(d_tmem, a_j, b_j, tmem_base + (col & ~1u), idesc | (col & 1u), accumulate);
-                } else {
-                  ptx::mma_f16_ss_pair(d_tmem, a_j, b_j, idesc, accumulate);
-                }
-                accumulate = 1u;
+                const uint64_t a_q = ((uint64_t)a_hi << 32) | (a_u + (uint32_t)(q * 2));
+                const uint64_t b_q = ((uint64_t)b_hi << 32) | (b_u + (uint32_t)q * kBStep);
+                if (SPARSE)
+                  ptx::mma_sp_f16_ss_pair(d_tmem, a_q, b_q, e_col + 4u * u + (uint32_t)(q & 2), idesc | (uint32_t)(q & 1),
+                                          q == 0 ? accumulate : 1u);
+                else
+                  ptx::mma_f16_ss_pair(d_tmem, a_q, b_q, idesc, q == 0 ? accumulate : 1u);
               }
+              accumulate = 1u;
             }
             ptx::tc_commit_pair(&empty[st], 3);
-            if (++st == STAGES) { st = 0; ph ^= 1u; }
+            if (++st == STAGES) { st = 0; ph ^= 1u; a_lo = a_lo0; b_lo = b_lo0; e_lo = e_lo0; mcol = 0; }
+            else { a_lo += a_stage16; b_lo += b_stage16; e_lo += e_stage16; mcol += slot_cols; }
           }
           if (++s == p.S) { s = 0; ++r_single; }
         }
@@ -408,8 +420,33 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     }
   } else if (warp < 6) {
     // ------------------------------------------------- metadata rearranger
-    if (SPARSE) {
-      // thread = A-tile row; the four warps handle every stage use together, in order
+    if (SPARSE && !FUSED) {
+      // A lone warp runs a dependent chain slowly, so the four warps do not share a stage:
+      // warp k builds the TMEM metadata images of stage uses k, k+4, k+8, ... (four passes of
+      // 32 lanes per image), four stages in flight.
+      const int total_uses = my_tiles * uses_per_tile;
+      int st = warp - 2;
+      uint32_t ph = 0;
+      while (st >= STAGES) { st -= STAGES; ph ^= 1u; }
+      for (int u = warp - 2; u < total_uses; u += 4) {
+        // the metadata box was requested after the stage's previous use had been consumed
+        if (!ptx::mbar_wait(&meta_full[st], ph, err, 0x500u + st)) break;
+        for (int v = 0; v < p.rr; ++v) {
+          const int row_off = reuse ? (p.R - 1 - v) * p.TW : 0;
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            build_metadata_lane(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + v * kEHwBytes,
+                                32 * i + lane, rows_used);
+        }
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive_cluster(&full[st], 0);
+        st += 4;
+        while (st >= STAGES) { st -= STAGES; ph ^= 1u; }
+      }
+    } else if (SPARSE) {
+      // Fused pruning: the four warps prune the stage's pixel rows together (thread = row),
+      // then each thread builds one TMEM lane of every metadata image.
       const int row = threadIdx.x - 64;
       bool alive = true;
       int st = 0;
@@ -422,34 +459,30 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int w0 = wt * p.TW, h0 = ht * p.TH, b0 = t * p.TB;
         int r = reuse ? (p.R - 1) : 0, s = 0, cb = 0;
         for (int k = 0; k < uses_per_tile; ++k) {
-          if (FUSED) {
-            if (!ptx::mbar_wait(&raw_full[st], ph, err, 0x900u + st)) { alive = false; break; }
-            const int q0 = w0 + p.pad_w - s, p0 = h0 + p.pad_h - r;
-            for (int i = row; i < p.img_rows; i += 128) {
-              const int iw = i % p.TW, ih = (i / p.TW) % img_h, ib = i / (p.TW * img_h);
-              const int64_t pixel = ((int64_t)(b0 + ib) * p.P + (p0 + ih)) * p.Q + (q0 + iw);  // any value when outside
-              const int64_t vbase = pixel * (p.Cout >> 3) + cb * 16;
-              const uint8_t* raw = sRaw + st * 2 * p.a_bytes;
-              uint8_t* a_tile = sA + st * p.a_bytes;
-              uint8_t* meta_rows = sEraw + st * p.eraw_bytes;
+          if (!ptx::mbar_wait(&raw_full[st], ph, err, 0x900u + st)) { alive = false; break; }
+          const int q0 = w0 + p.pad_w - s, p0 = h0 + p.pad_h - r;
+          for (int i = row; i < p.img_rows; i += 128) {
+            const int iw = i % p.TW, ih = (i / p.TW) % img_h, ib = i / (p.TW * img_h);
+            const int64_t pixel = ((int64_t)(b0 + ib) * p.P + (p0 + ih)) * p.Q + (q0 + iw);  // any value when outside
+            const int64_t vbase = pixel * (p.Cout >> 3) + cb * 16;
+            const uint8_t* raw = sRaw + st * 2 * p.a_bytes;
+            uint8_t* a_tile = sA + st * p.a_bytes;
+            uint8_t* meta_rows = sEraw + st * p.eraw_bytes;
 #define SDGP_FUSED_ROW(NN, SS) fused_prune_row<NN, SS>(raw, p.a_bytes, a_tile, meta_rows, i, vbase, p.seed_lo, p.seed_hi)
-              if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_MAGNITUDE); else SDGP_FUSED_ROW(2, SDGP_MAGNITUDE); }
-              else if (p.fused_scheme == SDGP_RANDOM) { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_RANDOM); else SDGP_FUSED_ROW(2, SDGP_RANDOM); }
-              else { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_RESCALED_MAGNITUDE); else SDGP_FUSED_ROW(2, SDGP_RESCALED_MAGNITUDE); }
+            if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_MAGNITUDE); else SDGP_FUSED_ROW(2, SDGP_MAGNITUDE); }
+            else if (p.fused_scheme == SDGP_RANDOM) { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_RANDOM); else SDGP_FUSED_ROW(2, SDGP_RANDOM); }
+            else { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_RESCALED_MAGNITUDE); else SDGP_FUSED_ROW(2, SDGP_RESCALED_MAGNITUDE); }
 #undef SDGP_FUSED_ROW
-            }
-            ptx::named_bar_sync(2, 128);  // every row's metadata is in place before it is rearranged
-          } else {
-            if (!ptx::mbar_wait(&meta_full[st], ph, err, 0x500u + st)) { alive = false; break; }
           }
+          ptx::named_bar_sync(2, 128);  // every row's metadata is in place before it is rearranged
           for (int u = 0; u < p.rr; ++u) {
             const int row_off = reuse ? (p.R - 1 - u) * p.TW : 0;
-            rearrange_metadata_row(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + u * kEHwBytes,
-                                   row, rows_used);
+            build_metadata_lane(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + u * kEHwBytes, row,
+                                rows_used);
           }
           ptx::fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive_cluster(&meta_ready[st], 0);
+          if (lane == 0) ptx::mbar_arrive_cluster(&full[st], 0);
           if (++st == STAGES) { st = 0; ph ^= 1u; }
           if (++cb == p.k_blocks) {
             cb = 0;
