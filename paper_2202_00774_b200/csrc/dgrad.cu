@@ -424,11 +424,13 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       // A lone warp runs a dependent chain slowly, so the four warps do not share a stage:
       // warp k builds the TMEM metadata images of stage uses k, k+4, k+8, ... (four passes of
       // 32 lanes per image), four stages in flight.
-      const int total_uses = my_tiles * uses_per_tile;
+      // No more warps than stages take part: a warp's previous use then needed the use two ring
+      // passes back to be complete, so a parity wait can never be satisfied by a stale phase.
+      const int G = STAGES < 4 ? STAGES : 4;
+      const int total_uses = (warp - 2 < G) ? my_tiles * uses_per_tile : 0;
       int st = warp - 2;
       uint32_t ph = 0;
-      while (st >= STAGES) { st -= STAGES; ph ^= 1u; }
-      for (int u = warp - 2; u < total_uses; u += 4) {
+      for (int u = warp - 2; u < total_uses; u += G) {
         // the metadata box was requested after the stage's previous use had been consumed
         if (!ptx::mbar_wait(&meta_full[st], ph, err, 0x500u + st)) break;
         for (int v = 0; v < p.rr; ++v) {
@@ -441,7 +443,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive_cluster(&full[st], 0);
-        st += 4;
+        st += G;
         while (st >= STAGES) { st -= STAGES; ph ^= 1u; }
       }
     } else if (SPARSE) {
@@ -459,7 +461,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int w0 = wt * p.TW, h0 = ht * p.TH, b0 = t * p.TB;
         int r = reuse ? (p.R - 1) : 0, s = 0, cb = 0;
         for (int k = 0; k < uses_per_tile; ++k) {
-          if (!ptx::mbar_wait(&raw_full[st], ph, err, 0x900u + st)) { alive = false; break; }
+          // the four warps stay or leave together: they meet at a named barrier below
+          if (!ptx::named_bar_all(2, 128, ptx::mbar_wait(&raw_full[st], ph, err, 0x900u + st))) { alive = false; break; }
           const int q0 = w0 + p.pad_w - s, p0 = h0 + p.pad_h - r;
           for (int i = row; i < p.img_rows; i += 128) {
             const int iw = i % p.TW, ih = (i / p.TW) % img_h, ib = i / (p.TW * img_h);
@@ -551,6 +554,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
 constexpr int kHaloTH = 16;  // pixel rows of a strip: 8 x 16 pixels = the 128 rows of an accumulator
 constexpr int kHaloAStages = 2;
+constexpr int kPruneWarps = 8;  // fused pruning: warps 10..17 prune the dense A box in shared memory
+constexpr int kThreadsHaloFused = kThreadsGemm + 32 * kPruneWarps;
 
 struct HaloParams {
   int B, H, W, Cin, Cout;
@@ -567,12 +572,37 @@ struct HaloParams {
   int w_stages;
   int meta_col, meta_shared, out_bufs;
   int a_bytes, eraw_bytes, w_bytes, ehw_bytes;  // per stage
-  int off_eraw, off_w, off_ehw, off_out, off_bar;
+  int off_eraw, off_half1, off_w, off_ehw, off_out, off_bar;
   int smem_bytes;
+  // fused pruning (A is the dense dL/dO; m = 4)
+  int fused_n, fused_scheme;
+  uint32_t seed_lo, seed_hi;
+  int P, Q;                // dO pixel grid (linear element index of the random scheme)
 };
 
-template <bool SPARSE, int BN, int NT>
-__global__ void __launch_bounds__(kThreadsGemm, 1)
+// Fused pruning of one quarter (32 channels = 4 vectors) of one pixel row of a dense A box that
+// lies in shared memory as two 128-byte-swizzled halves of 64 channels: `half` points at the half
+// holding the quarter, c = quarter number (0..3). The results stay in registers (out, metaw)
+// until every thread of the round has read its input, because the compressed row overwrites the
+// first half in place.
+template <int N, int SCHEME>
+__device__ __forceinline__ void fused_prune_quarter(const uint8_t* half, int i, int c, int64_t vbase, uint32_t seed_lo,
+                                                    uint32_t seed_hi, uint2 (&out)[4], uint32_t& metaw) {
+  const int sw = i & 7;
+  metaw = 0u;
+#pragma unroll
+  for (int v = 0; v < 4; ++v) {
+    const uint4 w = *(const uint4*)(half + i * 128 + (((4 * (c & 1) + v) ^ sw) << 4));
+    uint32_t y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2;
+    m4_prune_vector<N, SCHEME>(w, vbase + 4 * c + v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
+    compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
+    out[v] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
+    metaw |= nib2 << (8 * v);
+  }
+}
+
+template <bool SPARSE, int BN, int NT, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? kThreadsHaloFused : kThreadsGemm, 1)
 dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmE,
                   const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
                   const HaloParams p) {
@@ -582,13 +612,15 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;
   uint8_t* sEraw = smem + p.off_eraw;
+  uint8_t* sHalf1 = smem + p.off_half1;  // fused: channels 64..127 of the dense box being pruned
   uint8_t* sW = smem + p.off_w;
   uint8_t* sEhw = smem + p.off_ehw;
   uint8_t* sOut = smem + p.off_out;
   uint64_t* a_full = (uint64_t*)(smem + p.off_bar);
   uint64_t* a_empty = a_full + kHaloAStages;
   uint64_t* meta_full = a_empty + kHaloAStages;
-  uint64_t* w_ready = meta_full + kHaloAStages;  // W bytes landed AND (sparse) metadata tiles built
+  uint64_t* raw_full = meta_full + kHaloAStages;  // fused: the dense box has landed
+  uint64_t* w_ready = raw_full + kHaloAStages;    // W bytes landed AND (sparse) metadata tiles built
   uint64_t* w_empty = w_ready + kMaxStages;
   uint64_t* acc_full = w_empty + kMaxStages;
   uint64_t* acc_empty = acc_full + 2;
@@ -602,9 +634,12 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kHaloAStages; ++s) {
-      ptx::mbar_init(&a_full[s], 1);
+      // fused: A and its metadata rows are complete when every pruning warp has arrived
+      // (a_full: the warps of both CTAs; meta_full: this CTA's)
+      ptx::mbar_init(&a_full[s], FUSED ? 2 * kPruneWarps : 1);
       ptx::mbar_init(&a_empty[s], 1);
-      ptx::mbar_init(&meta_full[s], 1);
+      ptx::mbar_init(&meta_full[s], FUSED ? kPruneWarps : 1);
+      ptx::mbar_init(&raw_full[s], 1);
     }
     for (int s = 0; s < kMaxStages; ++s) {
       // one arrival from the producer (with the byte count) plus, for sparse A, one from the
@@ -664,21 +699,34 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // Loads the A box (and raw metadata) of stage use `ia`. blocking == false: only if the
       // stage is free right now. Returns 1 issued, 0 not free, -1 wait gave up.
       auto issue_a = [&](bool blocking) -> int {
+        // fused: the box before this one must have been pruned, its second half lies in the
+        // single scratch buffer this load overwrites
+        uint64_t* pruned = &meta_full[ast ^ 1];
+        const uint32_t pruned_ph = ((uint32_t)(ia - 1) >> 1) & 1u;
         if (blocking) {
           if (!ptx::mbar_wait(&a_empty[ast], aph ^ 1u, err, 0x100u + ast)) return -1;
-        } else if (!ptx::mbar_test(&a_empty[ast], aph ^ 1u)) {
+          if (FUSED && ia > 0 && !ptx::mbar_wait(pruned, pruned_ph, err, 0x140u + ast)) return -1;
+        } else if (!ptx::mbar_test(&a_empty[ast], aph ^ 1u) || (FUSED && ia > 0 && !ptx::mbar_test(pruned, pruned_ph))) {
           return 0;
         }
         const int lt = ia / p.k_blocks, kb = ia - lt * p.k_blocks;
         int n0, w0, h0, b0;
         locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
         const int q0 = w0 + p.pad_w - (p.S - 1), p0 = h0 + p.pad_h - (p.R - 1);
-        if (rank == 0) ptx::mbar_arrive_expect_tx(&a_full[ast], a_tx);
-        if (SPARSE) {
-          ptx::mbar_arrive_expect_tx(&meta_full[ast], meta_tx);
-          ptx::tma_load_4d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, p0, b0);
+        if (FUSED) {
+          // dense dL/dO of this CTA's box: 128 channels as two halves of 64; the first half lands
+          // in the A stage itself and is compressed in place
+          ptx::mbar_arrive_expect_tx(&raw_full[ast], 2u * (uint32_t)(p.img_rows * 128));
+          ptx::tma_load_4d(sA + ast * p.a_bytes, &tmA, &raw_full[ast], kb * 128, q0, p0, b0);
+          ptx::tma_load_4d(sHalf1, &tmA, &raw_full[ast], kb * 128 + 64, q0, p0, b0);
+        } else {
+          if (rank == 0) ptx::mbar_arrive_expect_tx(&a_full[ast], a_tx);
+          if (SPARSE) {
+            ptx::mbar_arrive_expect_tx(&meta_full[ast], meta_tx);
+            ptx::tma_load_4d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, p0, b0);
+          }
+          ptx::tma_load_4d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, p0, b0);
         }
-        ptx::tma_load_4d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, p0, b0);
         ++ia;
         if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
         return 1;
@@ -795,14 +843,16 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // lane = pixel column w, channel half, and odd/even pair of strip rows within a pass
       const int w = lane & 7, hsub = lane >> 4;
       const uint32_t sel = (lane & 8) ? 0x7632u : 0x5410u;
-      const int total_uses = my_tiles * p.k_blocks * taps;
+      // No more warps than W stages take part: a warp's previous use then needed the use two
+      // ring passes back to be consumed, so a parity wait can never be satisfied by a stale phase.
+      const int G = WS < 4 ? WS : 4;
+      const int total_uses = (warp - 2 < G) ? my_tiles * p.k_blocks * taps : 0;
       int t = warp - 2;  // tap within the channel block
       int ause = 0;      // A stage use = (tile set, channel block)
       while (t >= taps) { t -= taps; ++ause; }
       int wst = warp - 2;
       uint32_t wph = 0;
-      while (wst >= WS) { wst -= WS; wph ^= 1u; }
-      for (int u = warp - 2; u < total_uses; u += 4) {
+      for (int u = warp - 2; u < total_uses; u += G) {
         const int ast = ause & 1;  // kHaloAStages == 2
         if (!ptx::mbar_wait(&meta_full[ast], (uint32_t)(ause >> 1) & 1u, err, 0x500u + ast)) break;
         // the stage's previous tiles have been copied to TMEM and used
@@ -830,11 +880,67 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive_cluster(&w_ready[wst], 0);
-        t += 4;
+        t += G;
         while (t >= taps) { t -= taps; ++ause; }
-        wst += 4;
+        wst += G;
         while (wst >= WS) { wst -= WS; wph ^= 1u; }
       }
+    }
+  } else if (FUSED && warp >= 10) {
+    // ------------------------------------------------------------ pruner
+    // The dense box is pruned quarter row by quarter row (32 channels per item, items dealt to
+    // the 256 threads round-robin: a round covers 64 whole pixel rows). Within a round every
+    // thread reads its input, all wait, then every thread writes: the compressed row replaces
+    // the first dense half in place.
+    const int tid = threadIdx.x - kThreadsGemm;  // 0 .. 32 * kPruneWarps - 1
+    constexpr int kPruners = 32 * kPruneWarps;
+    const int items = p.img_rows * 4;
+    const int rounds = (items + kPruners - 1) / kPruners;
+    const int a_uses = my_tiles * p.k_blocks;
+    int lt = 0, kb = 0;
+    for (int ia = 0; ia < a_uses; ++ia) {
+      const int ast = ia & 1;  // kHaloAStages == 2
+      // all pruning threads stay or leave together: they meet at named barriers below
+      if (!ptx::named_bar_all(3, kPruners, ptx::mbar_wait(&raw_full[ast], ((uint32_t)ia >> 1) & 1u, err, 0x900u + ast)))
+        break;
+      int n0, w0, h0, b0;
+      locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
+      const int q0 = w0 + p.pad_w - (p.S - 1), p0 = h0 + p.pad_h - (p.R - 1);
+      uint8_t* a_tile = sA + ast * p.a_bytes;
+      uint8_t* meta_rows = sEraw + ast * p.eraw_bytes;
+      for (int rd = 0; rd < rounds; ++rd) {
+        const int item = rd * kPruners + tid;
+        const int i = item >> 2, c = item & 3;  // pixel row of the box, quarter
+        const bool active = item < items;
+        uint2 out[4];
+        uint32_t metaw = 0u;
+        if (active) {
+          const int ih = i / p.pitch, iw = i - ih * p.pitch;
+          const int64_t pixel = ((int64_t)b0 * p.P + (p0 + ih)) * p.Q + (q0 + iw);  // any value when outside the image
+          const int64_t vbase = pixel * (p.Cout >> 3) + kb * 16;
+          const uint8_t* half = (c < 2) ? a_tile : sHalf1;
+#define SDGP_FUSED_Q(NN, SS) fused_prune_quarter<NN, SS>(half, i, c, vbase, p.seed_lo, p.seed_hi, out, metaw)
+          if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_Q(1, SDGP_MAGNITUDE); else SDGP_FUSED_Q(2, SDGP_MAGNITUDE); }
+          else if (p.fused_scheme == SDGP_RANDOM) { if (p.fused_n == 1) SDGP_FUSED_Q(1, SDGP_RANDOM); else SDGP_FUSED_Q(2, SDGP_RANDOM); }
+          else { if (p.fused_n == 1) SDGP_FUSED_Q(1, SDGP_RESCALED_MAGNITUDE); else SDGP_FUSED_Q(2, SDGP_RESCALED_MAGNITUDE); }
+#undef SDGP_FUSED_Q
+        }
+        ptx::named_bar_sync(3, kPruners);  // the round's inputs are in registers
+        if (active) {
+          const int sw = i & 7;
+          // vectors 4c .. 4c+3 of the row -> 8 bytes each at chunk (j >> 1), half (j & 1)
+          *(uint4*)(a_tile + i * 128 + (((2 * c) ^ sw) << 4)) = make_uint4(out[0].x, out[0].y, out[1].x, out[1].y);
+          *(uint4*)(a_tile + i * 128 + (((2 * c + 1) ^ sw) << 4)) = make_uint4(out[2].x, out[2].y, out[3].x, out[3].y);
+          *(uint32_t*)(meta_rows + i * 16 + 4 * c) = metaw;
+        }
+      }
+      ptx::fence_proxy_async_smem();  // the tensor core reads A through the async proxy
+      __syncwarp();
+      if (lane == 0) {
+        ptx::mbar_arrive(&meta_full[ast]);
+        ptx::mbar_arrive_cluster(&a_full[ast], 0);
+      }
+      if (++kb == p.k_blocks) { kb = 0; ++lt; }
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -1090,7 +1196,7 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const Dg
 }
 
 // Shared-memory and TMEM plan of the whole-filter-reuse kernel. Returns false if it does not fit.
-template <bool SPARSE, int BN>
+template <bool SPARSE, int BN, bool FUSED>
 bool plan_halo(HaloParams* p, int nt) {
   using C = Cfg<SPARSE, BN>;
   const int budget = kSmemLimit - kSmemSlack;
@@ -1106,7 +1212,8 @@ bool plan_halo(HaloParams* p, int nt) {
     p->eraw_bytes = SPARSE ? round_up(p->img_rows * 16, 128) : 0;
     p->w_bytes = C::kTapBBytes;
     p->ehw_bytes = SPARSE ? nt * kEHwBytes : 0;
-    const int fixed = kHaloAStages * (p->a_bytes + p->eraw_bytes) + 1024;
+    const int half1_bytes = FUSED ? p->a_bytes : 0;  // scratch for the second dense half
+    const int fixed = kHaloAStages * (p->a_bytes + p->eraw_bytes) + half1_bytes + 1024;
     int out_bufs = 2;
     int w_stages = (budget - fixed - out_bufs * kOutBytes) / (p->w_bytes + p->ehw_bytes);
     if (w_stages < 4) {
@@ -1131,7 +1238,8 @@ bool plan_halo(HaloParams* p, int nt) {
     p->w_stages = w_stages;
     p->out_bufs = out_bufs;
     p->off_eraw = kHaloAStages * p->a_bytes;
-    p->off_w = round_up(p->off_eraw + kHaloAStages * p->eraw_bytes, 1024);
+    p->off_half1 = round_up(p->off_eraw + kHaloAStages * p->eraw_bytes, 1024);
+    p->off_w = p->off_half1 + half1_bytes;
     p->off_ehw = p->off_w + w_stages * p->w_bytes;
     p->off_out = round_up(p->off_ehw + w_stages * p->ehw_bytes, 1024);
     p->off_bar = p->off_out + out_bufs * kOutBytes;
@@ -1156,15 +1264,15 @@ bool halo_applies(int H, int W, int taps) {
   return covered * 100 <= (int64_t)H * W * 135;
 }
 
-template <bool SPARSE, int BN, int NT>
+template <bool SPARSE, int BN, int NT, bool FUSED>
 sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, const DgradView& view, HaloParams p,
                            cudaStream_t stream) {
   using C = Cfg<SPARSE, BN>;
-  if (!plan_halo<SPARSE, BN>(&p, NT)) return SDGP_ERR_UNSUPPORTED;
+  if (!plan_halo<SPARSE, BN, FUSED>(&p, NT)) return SDGP_ERR_UNSUPPORTED;
 
   CUtensorMap tmA, tmE, tmB, tmD;
   const int P = view.P, Q = view.Q;
-  const uint64_t CA = SPARSE ? (uint64_t)view.a_channels / 2 : (uint64_t)view.a_channels;
+  const uint64_t CA = (SPARSE && !FUSED) ? (uint64_t)view.a_channels / 2 : (uint64_t)view.a_channels;
   {
     const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
     const uint64_t strides[3] = {CA * 2, CA * 2 * Q, CA * 2 * Q * P};
@@ -1172,7 +1280,7 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
     if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
   }
-  if (SPARSE) {
+  if (SPARSE && !FUSED) {
     const uint64_t CE = (uint64_t)view.a_channels / 16;
     const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
     const uint64_t strides[3] = {CE * 2, CE * 2 * Q, CE * 2 * Q * P};
@@ -1199,7 +1307,7 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
   }
 
   static bool configured = false;
-  auto kernel = dgrad_halo_kernel<SPARSE, BN, NT>;
+  auto kernel = dgrad_halo_kernel<SPARSE, BN, NT, FUSED>;
   if (!configured) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
       return SDGP_ERR_CUDA;
@@ -1209,7 +1317,7 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
   const int pairs = p.pair_tiles < max_pairs ? p.pair_tiles : max_pairs;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3(kThreadsGemm);
+  cfg.blockDim = dim3(FUSED ? kThreadsHaloFused : kThreadsGemm);
   cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -1223,14 +1331,14 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
 }
 
 // Two strips per CTA where the accumulators of two tile sets fit TMEM, else one.
-template <bool SPARSE, int BN>
+template <bool SPARSE, int BN, bool FUSED = false>
 sdgp_status launch_halo(const void* A, const void* meta, const void* Wt, const DgradView& view, const HaloParams& p,
                         cudaStream_t stream) {
   if (BN <= 128) {
-    const sdgp_status st = launch_halo_nt<SPARSE, (BN <= 128 ? BN : 64), 2>(A, meta, Wt, view, p, stream);
+    const sdgp_status st = launch_halo_nt<SPARSE, (BN <= 128 ? BN : 64), 2, FUSED>(A, meta, Wt, view, p, stream);
     if (st != SDGP_ERR_UNSUPPORTED) return st;
   }
-  return launch_halo_nt<SPARSE, BN, 1>(A, meta, Wt, view, p, stream);
+  return launch_halo_nt<SPARSE, BN, 1, FUSED>(A, meta, Wt, view, p, stream);
 }
 
 }  // namespace
@@ -1302,14 +1410,20 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
       view.d_stride_h = (uint64_t)stride * W * Cin * 2;
       view.d_stride_b = (uint64_t)H * W * Cin * 2;
       sdgp_status st = SDGP_ERR_UNSUPPORTED;
-      if (!fused && halo_applies(Hs, Ws, p.R * p.S)) {
+      if (halo_applies(Hs, Ws, p.R * p.S)) {
         HaloParams hp = {};
         hp.B = B; hp.H = Hs; hp.W = Ws; hp.Cin = Cin; hp.Cout = Cout;
         hp.R = p.R; hp.S = p.S; hp.pad_h = p.pad_h; hp.pad_w = p.pad_w;
         hp.r_first = p.r_first; hp.r_step = p.r_step; hp.s_first = p.s_first; hp.s_step = p.s_step;
         hp.S_full = S;
         hp.tiles_n = p.tiles_n; hp.k_blocks = p.k_blocks;
-        if (sparse) {
+        hp.P = P; hp.Q = Q;
+        if (fused) {
+          hp.fused_n = p.fused_n; hp.fused_scheme = p.fused_scheme; hp.seed_lo = p.seed_lo; hp.seed_hi = p.seed_hi;
+          st = BN == 256 ? launch_halo<true, 256, true>(A, meta, Wt, view, hp, stream)
+             : BN == 128 ? launch_halo<true, 128, true>(A, meta, Wt, view, hp, stream)
+                         : launch_halo<true, 64, true>(A, meta, Wt, view, hp, stream);
+        } else if (sparse) {
           st = BN == 256 ? launch_halo<true, 256>(A, meta, Wt, view, hp, stream)
              : BN == 128 ? launch_halo<true, 128>(A, meta, Wt, view, hp, stream)
                          : launch_halo<true, 64>(A, meta, Wt, view, hp, stream);

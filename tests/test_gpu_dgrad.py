@@ -278,6 +278,57 @@ def test_fused_prune_and_dgrad(case, scheme, n):
     assert rel_fro(got, oracle.dgrad_conv2d(pruned, W, H, Wd, stride, pad)) <= TOL
 
 
+# Shapes for the whole-filter-reuse kernel (more than one tap, images at least one 8 x 16 strip
+# large): ragged strips in both directions, one and two strips per tile set, odd strip counts,
+# wide filters, non-square filters, missing padding, two channel blocks, a half-empty last channel
+# block, 64 / 128 / 256 input channels, stride 2 (parity classes with 1 x 2, 2 x 1 and 2 x 2 taps).
+HALO_CASES = [
+    # B, H, W, Cin, Cout, R, S, stride, pad
+    (3, 20, 24, 64, 128, 3, 3, 1, 1),
+    (2, 16, 8, 128, 128, 3, 3, 1, 1),       # a single strip per image
+    (5, 12, 40, 64, 64, 3, 3, 1, 1),        # five strips: the last tile set has one
+    (2, 17, 17, 128, 256, 3, 3, 1, 1),
+    (1, 24, 24, 64, 128, 5, 5, 1, 2),
+    (2, 16, 16, 64, 128, 1, 3, 1, 0),       # one filter row, no padding
+    (2, 16, 16, 64, 128, 3, 1, 1, 0),       # one filter column, no padding
+    (3, 16, 16, 256, 128, 3, 3, 1, 1),      # 256 input channels: one strip per tile set
+    (2, 16, 16, 128, 192, 3, 3, 1, 1),      # second channel block half empty
+    (2, 32, 32, 64, 128, 3, 3, 2, 1),       # stride 2 on 32 x 32: 16 x 16 parity classes
+    (2, 28, 28, 128, 128, 3, 3, 1, 1),
+    (9, 16, 16, 128, 128, 3, 3, 1, 1),      # odd number of tile sets: a pair with one phantom set
+]
+
+
+@pytest.mark.parametrize("mode", ["dense", "two_pass", "fused", "fused_random", "fused_rescaled_1"])
+@pytest.mark.parametrize("case", HALO_CASES)
+def test_whole_filter_reuse_kernel(case, mode):
+    import paper_2202_00774_b200 as sdgp
+    B, H, Wd, Cin, Cout, R, S, stride, pad = case
+    layer = inputs.ConvLayer("t", B, H, Wd, Cin, Cout, R, S, stride, pad)
+    dO, W = inputs.conv_layer_tensors(layer, seed=H * 100 + Wd)
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    n, scheme = 2, oracle.MAGNITUDE
+    if mode == "dense":
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, stride, pad, 4, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
+        src = dO
+    else:
+        if mode == "fused_random":
+            scheme = oracle.RANDOM
+        if mode == "fused_rescaled_1":
+            n, scheme = 1, oracle.RESCALED
+        if mode == "two_pass":
+            ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(B, H, Wd, Cin, Cout, R, S, stride, pad), dtype=torch.uint8,
+                             device="cuda")
+            sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, stride, pad, n, 4, scheme, seed=3, workspace=ws)
+        else:
+            sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, stride, pad, n, 4, scheme, seed=3, flags=sdgp.FLAG_FUSED)
+        src = oracle.prune(dO.reshape(-1, Cout), n, 4, scheme, 3, want=("dense",))["dense"].reshape(dO.shape)
+    check_no_device_error()
+    got = to_f64(dD)
+    assert not np.isnan(got).any()           # every output was written
+    assert rel_fro(got, oracle.dgrad_conv2d(src, W, H, Wd, stride, pad)) <= TOL
+
+
 def test_fused_needs_groups_of_four():
     import paper_2202_00774_b200 as sdgp
     dO = torch.zeros((2, 8, 8, 128), dtype=torch.int16, device="cuda")
