@@ -129,6 +129,30 @@ __device__ __forceinline__ void build_metadata_lane(const uint8_t* raw_rows, uin
       make_uint4(prmt(lo.x, hi.x, sel), prmt(lo.y, hi.y, sel), prmt(lo.z, hi.z, sel), prmt(lo.w, hi.w, sel));
 }
 
+// The whole 128-lane image by one warp: four passes of 32 lanes, all loads before all stores
+// (the compiler cannot tell the two shared-memory regions apart and would serialise them).
+__device__ __forceinline__ void build_metadata_image(const uint8_t* raw_rows, uint8_t* hw_tile, int lane, int rows_used) {
+  const uint32_t sel = (lane & 8) ? 0x7632u : 0x5410u;
+  const uint4 k01 = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+  uint4 lo[4], hi[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int tl = 32 * i + lane;
+    const int row_a = ((tl >> 4) << 4) + (tl & 7), row_b = row_a + 8;
+    lo[i] = k01;
+    hi[i] = k01;
+    if (row_a < rows_used) lo[i] = *(const uint4*)(raw_rows + row_a * 16);
+    if (row_b < rows_used) hi[i] = *(const uint4*)(raw_rows + row_b * 16);
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint4 a = lo[i].x == 0u ? k01 : lo[i];
+    const uint4 b = hi[i].x == 0u ? k01 : hi[i];
+    *(uint4*)(hw_tile + (32 * i + lane) * 16) =
+        make_uint4(prmt(a.x, b.x, sel), prmt(a.y, b.y, sel), prmt(a.z, b.z, sel), prmt(a.w, b.w, sel));
+  }
+}
+
 // Fused pruning of one pixel row of a stage: 128 dense channels (two 128-byte-swizzled boxes of
 // 64) -> 64 compressed values written straight into the A tile's swizzled row, plus the row's 16
 // bytes of position metadata in the row-major form the rearrangement step expects.
@@ -422,8 +446,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     // ------------------------------------------------- metadata rearranger
     if (SPARSE && !FUSED) {
       // A lone warp runs a dependent chain slowly, so the four warps do not share a stage:
-      // warp k builds the TMEM metadata images of stage uses k, k+4, k+8, ... (four passes of
-      // 32 lanes per image), four stages in flight.
+      // warp k builds the TMEM metadata images of stage uses k, k+G, k+2G, ... (four passes of
+      // 32 lanes per image), G stages in flight.
       // No more warps than stages take part: a warp's previous use then needed the use two ring
       // passes back to be complete, so a parity wait can never be satisfied by a stale phase.
       const int G = STAGES < 4 ? STAGES : 4;
@@ -435,10 +459,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         if (!ptx::mbar_wait(&meta_full[st], ph, err, 0x500u + st)) break;
         for (int v = 0; v < p.rr; ++v) {
           const int row_off = reuse ? (p.R - 1 - v) * p.TW : 0;
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            build_metadata_lane(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + v * kEHwBytes,
-                                32 * i + lane, rows_used);
+          build_metadata_image(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + v * kEHwBytes, lane,
+                               rows_used);
         }
         ptx::fence_proxy_async_smem();
         __syncwarp();
@@ -838,8 +860,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // ------------------------------------------------- metadata rearranger
     if (SPARSE) {
       // A lone warp runs a dependent instruction chain slowly, so the four warps do not share
-      // one tap: warp k builds the metadata of W-ring uses k, k+4, k+8, ... (a whole TMEM image
-      // per strip: four passes of 32 lanes), four taps in flight.
+      // one tap: warp k builds the metadata of W-ring uses k, k+G, k+2G, ... (a whole TMEM image
+      // per strip: four passes of 32 lanes), G taps in flight.
       // lane = pixel column w, channel half, and odd/even pair of strip rows within a pass
       const int w = lane & 7, hsub = lane >> 4;
       const uint32_t sel = (lane & 8) ? 0x7632u : 0x5410u;
@@ -860,21 +882,31 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int r = t / p.S, s = t - r * p.S;
         const uint8_t* raw = sEraw + ast * p.eraw_bytes;
         uint8_t* dst = sEhw + wst * p.ehw_bytes + lane * 16;
-        // TMEM lane 32*i + lane holds strip rows 2*h2 and 2*h2 + 1 with h2 = 2*i + hsub
+        // TMEM lane 32*i + lane holds strip rows 2*h2 and 2*h2 + 1 with h2 = 2*i + hsub.
+        // All loads first, then all stores: the compiler cannot tell that the two shared-memory
+        // regions differ and would otherwise serialise load - store - load.
         const int px0 = (2 * hsub + (p.R - 1 - r)) * p.pitch + w + (p.S - 1 - s);
+        uint4 lo[4 * NT], hi[4 * NT];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
 #pragma unroll
           for (int j = 0; j < NT; ++j) {
             const int px = px0 + 4 * i * p.pitch + 8 * j;
-            uint4 lo = *(const uint4*)(raw + px * 16);
-            uint4 hi = *(const uint4*)(raw + (px + p.pitch) * 16);
+            lo[i * NT + j] = *(const uint4*)(raw + px * 16);
+            hi[i * NT + j] = *(const uint4*)(raw + (px + p.pitch) * 16);
+          }
+        }
+        const uint4 k01 = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+#pragma unroll
+          for (int j = 0; j < NT; ++j) {
             // pixels outside the image carry no metadata (TMA fills zeros; real metadata is never
             // zero): give them the well-formed position pair (0,1) in every chunk
-            if (lo.x == 0u) lo = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
-            if (hi.x == 0u) hi = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+            const uint4 a = lo[i * NT + j].x == 0u ? k01 : lo[i * NT + j];
+            const uint4 b = hi[i * NT + j].x == 0u ? k01 : hi[i * NT + j];
             *(uint4*)(dst + j * kEHwBytes + i * 512) =
-                make_uint4(prmt(lo.x, hi.x, sel), prmt(lo.y, hi.y, sel), prmt(lo.z, hi.z, sel), prmt(lo.w, hi.w, sel));
+                make_uint4(prmt(a.x, b.x, sel), prmt(a.y, b.y, sel), prmt(a.z, b.z, sel), prmt(a.w, b.w, sel));
           }
         }
         ptx::fence_proxy_async_smem();
