@@ -114,8 +114,14 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool sparse) {
 // lane (row%8) + 8*half + 16*(row/16) holds in its low 16 bits the four position nibbles of
 // channels 32*k2 + 16*half + [0,16) of the row with bit 3 clear, in its high 16 bits those of
 // row + 8. One call builds the 16 bytes of TMEM lane `tl` from its two rows. Rows that carry no
-// data (past the patch, or outside the image where TMA filled zeros - real metadata is never
-// zero) get the well-formed position pair (0,1) in every chunk.
+// data (past the patch, or outside the image where TMA filled zeros) get the well-formed
+// position pair (0,1) in every chunk.
+// Every position nibble of real metadata is at least 4 (p0 | p1 << 2 with p0 < p1), so a 16-bit
+// group of four nibbles is at least 0x4444; pixels outside the image arrive as zeros. The
+// per-half maximum with 0x4444 therefore leaves real metadata alone and turns a missing group
+// into the well-formed position pair (0,1) in every chunk.
+__device__ __forceinline__ uint32_t well_formed(uint32_t x) { return __vmaxu2(x, 0x44444444u); }
+
 __device__ __forceinline__ void build_metadata_lane(const uint8_t* raw_rows, uint8_t* hw_tile, int tl, int rows_used) {
   const int row_a = ((tl >> 4) << 4) + (tl & 7), row_b = row_a + 8;
   const uint32_t sel = (tl & 8) ? 0x7632u : 0x5410u;
@@ -123,10 +129,9 @@ __device__ __forceinline__ void build_metadata_lane(const uint8_t* raw_rows, uin
   uint4 lo = k01, hi = k01;
   if (row_a < rows_used) lo = *(const uint4*)(raw_rows + row_a * 16);
   if (row_b < rows_used) hi = *(const uint4*)(raw_rows + row_b * 16);
-  if (lo.x == 0u) lo = k01;
-  if (hi.x == 0u) hi = k01;
   *(uint4*)(hw_tile + tl * 16) =
-      make_uint4(prmt(lo.x, hi.x, sel), prmt(lo.y, hi.y, sel), prmt(lo.z, hi.z, sel), prmt(lo.w, hi.w, sel));
+      make_uint4(well_formed(prmt(lo.x, hi.x, sel)), well_formed(prmt(lo.y, hi.y, sel)),
+                 well_formed(prmt(lo.z, hi.z, sel)), well_formed(prmt(lo.w, hi.w, sel)));
 }
 
 // The whole 128-lane image by one warp: four passes of 32 lanes, all loads before all stores
@@ -146,10 +151,10 @@ __device__ __forceinline__ void build_metadata_image(const uint8_t* raw_rows, ui
   }
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const uint4 a = lo[i].x == 0u ? k01 : lo[i];
-    const uint4 b = hi[i].x == 0u ? k01 : hi[i];
+    const uint4 a = lo[i], b = hi[i];
     *(uint4*)(hw_tile + (32 * i + lane) * 16) =
-        make_uint4(prmt(a.x, b.x, sel), prmt(a.y, b.y, sel), prmt(a.z, b.z, sel), prmt(a.w, b.w, sel));
+        make_uint4(well_formed(prmt(a.x, b.x, sel)), well_formed(prmt(a.y, b.y, sel)),
+                   well_formed(prmt(a.z, b.z, sel)), well_formed(prmt(a.w, b.w, sel)));
   }
 }
 
@@ -896,17 +901,14 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             hi[i * NT + j] = *(const uint4*)(raw + (px + p.pitch) * 16);
           }
         }
-        const uint4 k01 = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
 #pragma unroll
           for (int j = 0; j < NT; ++j) {
-            // pixels outside the image carry no metadata (TMA fills zeros; real metadata is never
-            // zero): give them the well-formed position pair (0,1) in every chunk
-            const uint4 a = lo[i * NT + j].x == 0u ? k01 : lo[i * NT + j];
-            const uint4 b = hi[i * NT + j].x == 0u ? k01 : hi[i * NT + j];
+            const uint4 a = lo[i * NT + j], b = hi[i * NT + j];
             *(uint4*)(dst + j * kEHwBytes + i * 512) =
-                make_uint4(prmt(a.x, b.x, sel), prmt(a.y, b.y, sel), prmt(a.z, b.z, sel), prmt(a.w, b.w, sel));
+                make_uint4(well_formed(prmt(a.x, b.x, sel)), well_formed(prmt(a.y, b.y, sel)),
+                           well_formed(prmt(a.z, b.z, sel)), well_formed(prmt(a.w, b.w, sel)));
           }
         }
         ptx::fence_proxy_async_smem();
