@@ -236,6 +236,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
              const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
              const DgradParams p) {
   using C = Cfg<SPARSE, BN>;
+  ptx::launch_dependents();  // the next kernel of the stream may start its set-up
 
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle of the A, B and staging tiles
@@ -296,6 +297,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   ptx::cluster_sync();  // barrier inits and TMEM of both CTAs are ready before any cross-CTA signal
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above touched no global memory; the previous kernel's results are needed from here on
+  ptx::wait_for_previous_grid();
 
   const int rows_used = p.TW * p.TH * p.TB;
   const int taps = p.R * p.S;
@@ -634,6 +637,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
                   const HaloParams p) {
   using C = Cfg<SPARSE, BN>;
+  ptx::launch_dependents();  // the next kernel of the stream may start its set-up
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -695,6 +699,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   ptx::cluster_sync();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above touched no global memory; the previous kernel's results are needed from here on
+  ptx::wait_for_previous_grid();
 
   const int taps = p.R * p.S;
   const int pair_stride = gridDim.x >> 1;
@@ -1219,13 +1225,17 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const Dg
   cfg.blockDim = dim3(kThreadsGemm);
   cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // may be scheduled while the previous kernel of the stream drains (the kernel waits for it
+  // after its set-up)
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, tmA, tmE, tmB, tmD, p) == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
@@ -1354,13 +1364,17 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
   cfg.blockDim = dim3(FUSED ? kThreadsHaloFused : kThreadsGemm);
   cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // may be scheduled while the previous kernel of the stream drains (the kernel waits for it
+  // after its set-up)
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, tmA, tmE, tmB, tmD, p) == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 

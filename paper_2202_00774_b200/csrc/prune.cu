@@ -9,6 +9,7 @@
 #include <cuda_bf16.h>
 
 #include "prune_core.cuh"
+#include "ptx.cuh"
 #include "sdgp_internal.cuh"
 
 namespace sdgp {
@@ -23,12 +24,31 @@ __device__ __forceinline__ uint32_t chunk_nibble(uint32_t keep4) {
   return (uint32_t)(0x444E4DCC49884444ull >> (4 * keep4)) & 0xFu;
 }
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while the previous
+// kernel of the stream is still draining; it waits for that kernel before its first load.
+template <typename... Params, typename... Args>
+cudaError_t launch_after_previous(void (*kernel)(Params...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
+}
+
 // M: group size; LANES = lanes that share a group (1, 2 or 4).
 template <int M, int SCHEME>
 __global__ void __launch_bounds__(kThreads)
 prune_kernel(const uint4* __restrict__ dO, int64_t nvec, int n, uint32_t seed_lo, uint32_t seed_hi,
              uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
              uint8_t* __restrict__ mask) {
+  ptx::launch_dependents();
+  ptx::wait_for_previous_grid();
   constexpr int LANES = (M <= 8) ? 1 : M / 8;
   constexpr int SUB = (M == 4) ? 4 : 8;  // elements of this thread that share a group
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
@@ -214,6 +234,8 @@ __global__ void __launch_bounds__(kThreads)
 prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                 uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
                 uint8_t* __restrict__ mask, OutPitch pitch) {
+  ptx::launch_dependents();
+  ptx::wait_for_previous_grid();
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
   uint4 in[kVecPerThread];
 #pragma unroll
@@ -242,7 +264,7 @@ cudaError_t launch_m4_n(int scheme, const void* dO, int64_t nvec, uint64_t seed,
   const dim3 grid((unsigned)blocks), block(kThreads);
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
 #define SDGP_LAUNCH4(S)                                                                         \
-  prune_m4_kernel<N, S><<<grid, block, 0, stream>>>((const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
+  launch_after_previous(prune_m4_kernel<N, S>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
                                                     (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch)
   switch (scheme) {
     case SDGP_RANDOM: SDGP_LAUNCH4(SDGP_RANDOM); break;
@@ -271,6 +293,8 @@ __global__ void __launch_bounds__(kThreads)
 prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                   uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
                   uint8_t* __restrict__ mask, OutPitch pitch) {
+  ptx::launch_dependents();
+  ptx::wait_for_previous_grid();
   constexpr int LANES = M / 8;
   static_assert(N == 1 || N == 2, "threshold selection keeps one or two elements");
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
@@ -355,7 +379,7 @@ cudaError_t launch_top2(int scheme, const void* dO, int64_t nvec, uint64_t seed,
   const dim3 grid((unsigned)blocks), block(kThreads);
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
 #define SDGP_LAUNCH_T2(S)                                                                            \
-  prune_top2_kernel<M, N, S><<<grid, block, 0, stream>>>((const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
+  launch_after_previous(prune_top2_kernel<M, N, S>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
                                                          (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch)
   switch (scheme) {
     case SDGP_RANDOM: SDGP_LAUNCH_T2(SDGP_RANDOM); break;
@@ -376,7 +400,7 @@ cudaError_t launch_m(int scheme, const void* dO, int64_t nvec, int n, uint64_t s
   const dim3 grid((unsigned)blocks), block(kThreads);
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
 #define SDGP_LAUNCH(S)                                                                              \
-  prune_kernel<M, S><<<grid, block, 0, stream>>>((const uint4*)dO, nvec, n, lo, hi, (uint4*)dense, \
+  launch_after_previous(prune_kernel<M, S>, grid, block, stream, (const uint4*)dO, nvec, n, lo, hi, (uint4*)dense, \
                                                  (uint2*)values, (uint8_t*)meta, (uint8_t*)mask)
   switch (scheme) {
     case SDGP_RANDOM: SDGP_LAUNCH(SDGP_RANDOM); break;

@@ -27,6 +27,14 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   return t;
 }
 
+// Programmatic dependent launch. launch_dependents: the next kernel of the stream may be
+// scheduled (and run its set-up) once every CTA of this grid has got here. wait_for_previous_grid:
+// returns when the previous kernel of the stream has completed and its writes are visible; a
+// kernel must pass it before it touches global memory. Both do nothing in a kernel that was
+// launched without the attribute.
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_previous_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
