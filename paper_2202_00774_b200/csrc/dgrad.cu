@@ -584,7 +584,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
 constexpr int kHaloTH = 16;  // pixel rows of a strip: 8 x 16 pixels = the 128 rows of an accumulator
 constexpr int kHaloAStages = 2;
-constexpr int kPruneWarps = 8;  // fused pruning: warps 10..17 prune the dense A box in shared memory
+constexpr int kPruneWarps = 16;  // fused pruning: warps 10..25 prune the dense A box in shared memory
 constexpr int kThreadsHaloFused = kThreadsGemm + 32 * kPruneWarps;
 
 struct HaloParams {
@@ -929,7 +929,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   } else if (FUSED && warp >= 10) {
     // ------------------------------------------------------------ pruner
     // The dense box is pruned quarter row by quarter row (32 channels per item, items dealt to
-    // the 256 threads round-robin: a round covers 64 whole pixel rows). Within a round every
+    // the pruning threads round-robin: a round covers whole pixel rows). Within a round every
     // thread reads its input, all wait, then every thread writes: the compressed row replaces
     // the first dense half in place.
     const int tid = threadIdx.x - kThreadsGemm;  // 0 .. 32 * kPruneWarps - 1
