@@ -352,15 +352,18 @@ def test_unsupported_requests_raise():
 # ------------------------------------------------- full benchmark sizes, sampled outputs
 
 
-def _sampled_conv_check(layer, seed, n, m, scheme, samples=600):
-    """Run the two-pass path on the full layer; compare `samples` output pixels (plus the first
-    and last pixels of the tensor) with the oracle, which prunes only the rows those pixels read."""
+def _sampled_conv_check(layer, seed, n, m, scheme, samples=600, fused=False):
+    """Run the two-pass (or fused) path on the full layer; compare `samples` output pixels (plus the
+    first and last pixels of the tensor) with the oracle, which prunes only the rows those pixels read."""
     import paper_2202_00774_b200 as sdgp
     dO, W = inputs.conv_layer_tensors(layer, seed)
-    ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(layer.B, layer.H, layer.W, layer.Cin, layer.Cout, layer.R,
-                                                     layer.S, 1, layer.pad), dtype=torch.uint8, device="cuda")
     dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
-    sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, layer.pad, n, m, scheme, seed=5, workspace=ws)
+    if fused:
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, layer.pad, n, m, scheme, seed=5, flags=sdgp.FLAG_FUSED)
+    else:
+        ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(layer.B, layer.H, layer.W, layer.Cin, layer.Cout, layer.R,
+                                                         layer.S, 1, layer.pad), dtype=torch.uint8, device="cuda")
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, layer.pad, n, m, scheme, seed=5, workspace=ws)
     check_no_device_error()
     got_all = dD.cpu().numpy().view(np.uint16)
     assert not np.isnan(inputs.bf16_bits_to_f32(got_all)).any()   # every output was written
@@ -392,6 +395,14 @@ def test_resnet9_full_size_layers_sampled(index):
     layer = inputs.resnet9_layers(512)[index]
     scheme = [oracle.MAGNITUDE, oracle.RESCALED, oracle.RANDOM][index % 3]
     _sampled_conv_check(layer, seed=index, n=2, m=4, scheme=scheme)
+
+
+@pytest.mark.parametrize("index,scheme", [(0, oracle.RANDOM), (1, oracle.MAGNITUDE), (3, oracle.RESCALED), (4, oracle.MAGNITUDE),
+                                          (6, oracle.MAGNITUDE)])
+def test_resnet9_full_size_layers_fused_sampled(index, scheme):
+    """bench.py --mode fused: the same shapes with the prune inside the data-gradient kernel."""
+    layer = inputs.resnet9_layers(512)[index]
+    _sampled_conv_check(layer, seed=10 + index, n=2, m=4, scheme=scheme, fused=True)
 
 
 @pytest.mark.parametrize("n,m,scheme", [(2, 4, oracle.MAGNITUDE), (1, 4, oracle.RESCALED), (2, 8, oracle.MAGNITUDE),
