@@ -39,6 +39,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "prune_core.cuh"
 #include "ptx.cuh"
 #include "sdgp_internal.cuh"
@@ -595,6 +597,8 @@ struct HaloParams {
   int sets_w, tiles_h, tiles_n;
   int m_sets;              // sets_w * tiles_h * B
   int pair_tiles;          // ceil(m_sets / 2) * tiles_n
+  int units;               // work units: pair tiles, the last `units - split_from` of them split by strip
+  int split_from;          // units >= split_from cover one strip of a pair tile each (quantisation of the last round)
   int k_blocks;
   int pitch;               // pixel columns of the A box: 8 * nt + S - 1
   int img_h;               // pixel rows of the A box: kHaloTH + R - 1
@@ -705,12 +709,19 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int taps = p.R * p.S;
   const int pair_stride = gridDim.x >> 1;
   const int first_pair = blockIdx.x >> 1;
-  const int my_tiles = first_pair < p.pair_tiles ? (p.pair_tiles - first_pair + pair_stride - 1) / pair_stride : 0;
+  const int my_tiles = first_pair < p.units ? (p.units - first_pair + pair_stride - 1) / pair_stride : 0;
   const int n_half = (int)rank * C::kBCols;
   constexpr int set_cols = NT * BN;  // TMEM columns of one tile set's accumulators
   const int WS = p.w_stages;
-  // tile set `pt` of this CTA: first input channel, first pixel column / row, image
-  auto locate = [&p, rank](int pt, int& n0, int& w0, int& h0, int& b0) -> bool {
+  // Work unit u: a pair tile, or - for the units of the last, partly filled round - one strip of
+  // a pair tile, so that the round costs half. strip_mask: the strips unit number lt of this CTA covers.
+  auto strip_mask = [&p, first_pair, pair_stride](int lt) -> uint32_t {
+    const int u = first_pair + lt * pair_stride;
+    return u < p.split_from ? ((1u << NT) - 1u) : (1u << ((u - p.split_from) & 1));
+  };
+  // tile set of unit `u` for this CTA: first input channel, first pixel column / row, image
+  auto locate = [&p, rank](int u, int& n0, int& w0, int& h0, int& b0) -> bool {
+    const int pt = u < p.split_from ? u : p.split_from + ((u - p.split_from) >> 1);
     n0 = (pt % p.tiles_n) * BN;
     int t = 2 * (pt / p.tiles_n) + (int)rank;
     const bool in_range = t < p.m_sets;  // a set past the last one loads zeros and stores nothing
@@ -768,8 +779,9 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       int wst = 0, use = 0;
       uint32_t wph = 0;
       for (int lt = 0; alive && lt < my_tiles; ++lt) {
-        const int pt = first_pair + lt * pair_stride;
-        const int n0 = (pt % p.tiles_n) * BN + n_half;
+        int n0, w0_unused, h0_unused, b0_unused;
+        locate(first_pair + lt * pair_stride, n0, w0_unused, h0_unused, b0_unused);
+        n0 += n_half;
         for (int kb = 0; alive && kb < p.k_blocks; ++kb, ++use) {
           while (alive && ia <= use)
             if (issue_a(true) < 0) alive = false;
@@ -825,6 +837,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const uint32_t meta_base = tmem_base + (uint32_t)(p.meta_shared ? (acc ^ 1) * set_cols : p.meta_col);
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * set_cols);
+        const uint32_t strips = strip_mask(lt);
+        const bool all_strips = strips == ((1u << NT) - 1u);
         uint32_t accumulate = 0u;
         for (int kb = 0; alive && kb < p.k_blocks; ++kb) {
           if (!ptx::mbar_wait(&a_full[ast], aph, err, 0x300u + ast)) { alive = false; break; }
@@ -834,25 +848,33 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (!ptx::mbar_wait(&w_ready[wst], wph, err, 0x380u + wst)) { alive = false; break; }
             ptx::tc_fence_after_sync();
             const uint32_t e_col = meta_base + mcol;  // even: slots are 4 columns apart
-            if (SPARSE) {
+            // ALL: every strip takes part (no per-strip test in the issue path)
+            auto issue_tap = [&](auto all) {
+              constexpr bool ALL = decltype(all)::value;
+              if (SPARSE) {
 #pragma unroll
-              for (int j = 0; j < NT; ++j)
-                ptx::tc_cp_128x128b_pair(e_col + 4u * j, ((uint64_t)e_hi << 32) | (e_lo + (uint32_t)(j * (kEHwBytes / 16))));
-            }
-#pragma unroll
-            for (int j = 0; j < NT; ++j) {
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                // strip j: 8 pixels = 1024 bytes to the right; MMA q: 32 bytes along the row
-                const uint64_t a_q = ((uint64_t)a_hi << 32) | (a_lo + (uint32_t)(j * 64 + q * 2));
-                const uint64_t b_q = ((uint64_t)b_hi << 32) | (b_lo + (uint32_t)q * kBStep);
-                if (SPARSE)
-                  ptx::mma_sp_f16_ss_pair(d_tmem + (uint32_t)(j * BN), a_q, b_q, e_col + (uint32_t)(4 * j + (q & 2)),
-                                          idesc | (uint32_t)(q & 1), q == 0 ? accumulate : 1u);
-                else
-                  ptx::mma_f16_ss_pair(d_tmem + (uint32_t)(j * BN), a_q, b_q, idesc, q == 0 ? accumulate : 1u);
+                for (int j = 0; j < NT; ++j)
+                  if (ALL || (strips & (1u << j)))
+                    ptx::tc_cp_128x128b_pair(e_col + 4u * j, ((uint64_t)e_hi << 32) | (e_lo + (uint32_t)(j * (kEHwBytes / 16))));
               }
-            }
+#pragma unroll
+              for (int j = 0; j < NT; ++j) {
+                if (!ALL && !(strips & (1u << j))) continue;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  // strip j: 8 pixels = 1024 bytes to the right; MMA q: 32 bytes along the row
+                  const uint64_t a_q = ((uint64_t)a_hi << 32) | (a_lo + (uint32_t)(j * 64 + q * 2));
+                  const uint64_t b_q = ((uint64_t)b_hi << 32) | (b_lo + (uint32_t)q * kBStep);
+                  if (SPARSE)
+                    ptx::mma_sp_f16_ss_pair(d_tmem + (uint32_t)(j * BN), a_q, b_q, e_col + (uint32_t)(4 * j + (q & 2)),
+                                            idesc | (uint32_t)(q & 1), q == 0 ? accumulate : 1u);
+                  else
+                    ptx::mma_f16_ss_pair(d_tmem + (uint32_t)(j * BN), a_q, b_q, idesc, q == 0 ? accumulate : 1u);
+                }
+              }
+            };
+            if (all_strips) issue_tap(std::true_type{});
+            else issue_tap(std::false_type{});
             ptx::tc_commit_pair(&w_empty[wst], 3);
             accumulate = 1u;
             // next tap: one pixel to the left, or the end of the filter row above
@@ -891,6 +913,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // the stage's previous tiles have been copied to TMEM and used
         if (!ptx::mbar_wait(&w_empty[wst], wph ^ 1u, err, 0x580u + wst)) break;
         const int r = t / p.S, s = t - r * p.S;
+        const uint32_t strips = strip_mask(ause / p.k_blocks);
         const uint8_t* raw = sEraw + ast * p.eraw_bytes;
         uint8_t* dst = sEhw + wst * p.ehw_bytes + lane * 16;
         // TMEM lane 32*i + lane holds strip rows 2*h2 and 2*h2 + 1 with h2 = 2*i + hsub.
@@ -911,6 +934,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int i = 0; i < 4; ++i) {
 #pragma unroll
           for (int j = 0; j < NT; ++j) {
+            if (!(strips & (1u << j))) continue;  // strip not part of this unit: its image is never read
             const uint4 a = lo[i * NT + j], b = hi[i * NT + j];
             *(uint4*)(dst + j * kEHwBytes + i * 512) =
                 make_uint4(well_formed(prmt(a.x, b.x, sel)), well_formed(prmt(a.y, b.y, sel)),
@@ -992,12 +1016,14 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     for (int lt = 0; lt < my_tiles; ++lt) {
       int n0, w0, h0, b0;
       const bool in_range = locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
+      const uint32_t strips = strip_mask(lt);
       if (!ptx::mbar_wait(&acc_full[acc], cph, err, 0x600u + acc)) break;
       ptx::tc_fence_after_sync();
 #pragma unroll
       for (int j = 0; j < NT; ++j)
         store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * set_cols + j * BN), sOut,
-                              p.out_bufs, &tmD, n0, w0 + 8 * j, h0, b0, in_range && (w0 + 8 * j < p.W), row, issuer,
+                              p.out_bufs, &tmD, n0, w0 + 8 * j, h0, b0, in_range && (w0 + 8 * j < p.W) && (strips & (1u << j)), row,
+                              issuer,
                               chunk, (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr);
       ptx::tc_fence_before_sync();
       __syncwarp();
@@ -1295,6 +1321,16 @@ bool plan_halo(HaloParams* p, int nt) {
     if (m_sets * p->tiles_n > 0x3FFFFFFF) return false;
     p->m_sets = (int)m_sets;
     p->pair_tiles = (int)((m_sets + 1) / 2) * p->tiles_n;
+    // The pair tiles of a last round that fills at most half the CTA pairs are dealt out strip by
+    // strip: that round then costs about half.
+    p->units = p->pair_tiles;
+    p->split_from = p->pair_tiles;
+    const int max_pairs = sm_count() / 2;
+    const int rem = p->pair_tiles % max_pairs;
+    if (nt == 2 && p->pair_tiles > max_pairs && rem > 0 && 2 * rem <= max_pairs) {
+      p->split_from = p->pair_tiles - rem;
+      p->units = p->pair_tiles + rem;
+    }
     return true;
   }
   return false;
@@ -1358,7 +1394,7 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
     configured = true;
   }
   const int max_pairs = sm_count() / 2;
-  const int pairs = p.pair_tiles < max_pairs ? p.pair_tiles : max_pairs;
+  const int pairs = p.units < max_pairs ? p.units : max_pairs;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs));
   cfg.blockDim = dim3(FUSED ? kThreadsHaloFused : kThreadsGemm);

@@ -296,6 +296,7 @@ HALO_CASES = [
     (2, 32, 32, 64, 128, 3, 3, 2, 1),       # stride 2 on 32 x 32: 16 x 16 parity classes
     (2, 28, 28, 128, 128, 3, 3, 1, 1),
     (9, 16, 16, 128, 128, 3, 3, 1, 1),      # odd number of tile sets: a pair with one phantom set
+    (168, 16, 16, 64, 64, 3, 3, 1, 1),      # 84 pair tiles on 74 CTA pairs: the last round is dealt out strip by strip
 ]
 
 
