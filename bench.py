@@ -137,7 +137,7 @@ class OracleArm:
         return int(max(1, probe * seconds / dt))
 
 
-def cpu_baseline(layers, workload, n, m, scheme, target_s=15.0):
+def cpu_baseline(layers, workload, n, m, scheme, target_s=24.0):
     arm = OracleArm(layers, workload, n, m, scheme)
     pixels = arm.pixels_for(target_s)
     t0 = time.perf_counter()
