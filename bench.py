@@ -2,7 +2,7 @@
 """Benchmark of the SDGP hot path: N:M pruning of dL/dO followed by the sparse tensor-core
 data gradient, on synthetic tensors shaped like a network's convolution layers.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet9|gemm_large|fc_small]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet9|gemm_large|fc_small|resnet50]
                   [--scheme magnitude|rescaled|random] [--nm 2:4] [--impl ours|reference]
 
 One step = every layer of the workload once: prune kernel + sparse dgrad kernel per layer
@@ -464,19 +464,130 @@ def run_ours(args, layers):
         dist.destroy_process_group()
 
 
+def run_layer_table(args):
+    """--workload resnet50: every distinct bottleneck convolution of ResNet-50 at batch 256, one layer
+    at a time (the tensors of all 23 shapes together would not be a step any trainer runs back to
+    back with resident inputs): per layer the prune kernel, the sparse contraction, the fused kernel
+    (groups of four only) and the dense twin, each timed by CUDA events around single launches with
+    a write of 256 MB between launches (L2 flush), median of --steps launches (at most 50). The
+    printed value weighs every shape by the number of times the network holds it."""
+    import torch
+    import paper_2202_00774_b200 as sdgp
+
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    n, m = [int(v) for v in args.nm.split(":")]
+    scheme = SCHEMES[args.scheme]
+    pk = peaks()
+    reps = max(5, min(args.steps, 50))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def dev16(a):
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
+
+    def median_us(fn):
+        for _ in range(max(3, min(args.warmup, 5))):
+            fn()
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(1e3 * e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    sampler = ClockSampler(torch.cuda.current_device())
+    rows, launches = [], 0
+    tot = dict(two_pass=0.0, best=0.0, dense=0.0, flops=0.0, prune=0.0, prune_bytes=0.0, spmm=0.0)
+    for l, count in inputs.resnet50_layers(256):
+        dO_h, W_h = inputs.conv_layer_tensors(l, seed=0)
+        dO, Wt = dev16(dO_h), dev16(W_h)
+        del dO_h, W_h
+        dD = torch.empty(l.dD_shape(), dtype=torch.int16, device="cuda")
+        Cp = (l.Cout + 127) // 128 * 128
+        ws = torch.empty(max(16, sdgp.sdgp_workspace_size_conv2d(l.B, l.H, l.W, l.Cin, l.Cout, l.R, l.S, l.stride, l.pad)),
+                         dtype=torch.uint8, device="cuda")
+        pix = l.B * l.P * l.Q
+        vals = torch.empty(pix * l.Cout // 2, dtype=torch.int16, device="cuda")
+        metas = torch.empty(pix * l.Cout // 16, dtype=torch.int16, device="cuda")
+        def note(what):
+            print("[%s] %s" % (l.name, what), file=sys.stderr, flush=True)
+
+        note("two-pass")
+        t_two = median_us(lambda: sdgp.sdgp_dgrad_conv2d(dO, Wt, dD, l.stride, l.pad, n, m, scheme, seed=1234, workspace=ws))
+        note("prune")
+        t_prune = median_us(lambda: sdgp.sdgp_prune(dO.view(-1, l.Cout), n, m, scheme, 1234, values=vals, meta=metas))
+        t_spmm = None
+        if Cp == l.Cout:
+            note("sparse contraction")
+            t_spmm = median_us(lambda: sdgp.sdgp_spmm_conv2d(vals.view(l.B, l.P, l.Q, l.Cout // 2),
+                                                             metas.view(l.B, l.P, l.Q, l.Cout // 16), Wt, dD, l.stride, l.pad))
+        t_fused = None
+        if m == 4:
+            note("fused")
+            t_fused = median_us(lambda: sdgp.sdgp_dgrad_conv2d(dO, Wt, dD, l.stride, l.pad, n, m, scheme, seed=1234,
+                                                               flags=sdgp.FLAG_FUSED))
+        note("dense")
+        t_dense = median_us(lambda: sdgp.sdgp_dgrad_conv2d(dO, Wt, dD, l.stride, l.pad, n, m, scheme, flags=sdgp.FLAG_DENSE))
+        launches += (reps + 3) * (2 + 1 + (1 if t_spmm else 0) + (1 if t_fused else 0) + 1)
+        status = sdgp.sdgp_last_device_error()
+        if status != 0:
+            raise SystemExit("device error: " + sdgp.status_string(status))
+        fl = 2.0 * l.dense_macs
+        bytes_dense = 2.0 * (pix * l.Cout + l.Cout * l.R * l.S * l.Cin + l.B * l.H * l.W * l.Cin)
+        best = min(t for t in (t_two, t_fused) if t is not None)
+        t_tensor = fl / (2.0 * pk["bf16_sustained"] * 1e12) * 1e6
+        t_hbm = bytes_dense / (pk["hbm"] * 1e9) * 1e6
+        rows.append({"layer": l.name, "count": count, "gflop": fl / 1e9, "two_pass_us": t_two, "prune_us": t_prune,
+                     "spmm_us": t_spmm, "fused_us": t_fused, "dense_us": t_dense,
+                     "speedup_two_pass": t_dense / t_two, "speedup_best": t_dense / best,
+                     "speedup_spmm_alone": (t_dense / t_spmm) if t_spmm else None,
+                     "bound": "tensor" if t_tensor >= t_hbm else "hbm",
+                     "ideal_us": max(t_tensor, t_hbm), "frac_of_ideal_best": max(t_tensor, t_hbm) / best,
+                     "prune_gbs": pix * l.Cout * 3.125 / (t_prune * 1e-6) / 1e9})
+        tot["two_pass"] += count * t_two
+        tot["best"] += count * best
+        tot["dense"] += count * t_dense
+        tot["flops"] += count * fl
+        tot["prune"] += count * t_prune
+        tot["prune_bytes"] += count * pix * l.Cout * 3.125
+        del dO, Wt, dD, ws, vals, metas
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    value = tot["flops"] / (tot["two_pass"] * 1e-6) / 1e12
+    print(json.dumps({
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 1, "steps": reps, "warmup": max(3, min(args.warmup, 5)),
+        "ms_per_step": tot["two_pass"] / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "resnet50", "layers": len(rows), "convolutions": sum(r["count"] for r in rows), "batch": 256,
+                   "nm": args.nm, "scheme": args.scheme, "mode": "two_pass (per layer also fused and dense)",
+                   "l2": "256 MB written between timed launches", "launch": "one launch per event pair, median"},
+        "speedup_vs_dense": tot["dense"] / tot["two_pass"], "speedup_best_mode_vs_dense": tot["dense"] / tot["best"],
+        "dense_tflops": tot["flops"] / (tot["dense"] * 1e-6) / 1e12,
+        "prune_gbs": tot["prune_bytes"] / (tot["prune"] * 1e-6) / 1e9,
+        "prune_frac_of_hbm": tot["prune_bytes"] / (tot["prune"] * 1e-6) / 1e9 / pk["hbm"],
+        "per_layer": rows, "gpu_launches": launches, "clocks": clocks}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet9", choices=["resnet9", "gemm_large", "fc_small"])
+    ap.add_argument("--workload", default="resnet9", choices=["resnet9", "gemm_large", "fc_small", "resnet50"])
     ap.add_argument("--scheme", default="magnitude", choices=sorted(SCHEMES))
     ap.add_argument("--nm", default="2:4")
     ap.add_argument("--mode", default="two_pass", choices=["two_pass", "fused"],
                     help="two_pass: prune kernel + sparse dgrad kernel per layer; fused: one kernel prunes and contracts")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.workload == "resnet50":
+        if args.impl == "reference" or args.gpus != 1:
+            raise SystemExit("--workload resnet50 is a single-GPU per-layer table of this implementation")
+        return run_layer_table(args)
     layers = workload_layers(args.workload)
     if args.impl == "reference":
         run_reference(args, layers)

@@ -71,7 +71,12 @@ enum {
   SDGP_FLAG_TWO_PASS = 0, /* prune kernel writes compressed dL/dO into the workspace, sparse GEMM reads it */
   SDGP_FLAG_FUSED = 1,    /* pruning happens inside the dgrad kernel (needs m == 4, n <= 2); no workspace, no
                              compressed tensor in global memory */
-  SDGP_FLAG_DENSE = 2     /* no pruning: dense tensor-core data gradient of dL/dO itself (n, m, scheme ignored) */
+  SDGP_FLAG_DENSE = 2,    /* no pruning: dense tensor-core data gradient of dL/dO itself (n, m, scheme ignored) */
+  SDGP_FLAG_MASKED = 3    /* prune kernel writes the pruned tensor as a dense copy (pruned positions +0.0, the tensor
+                             Algorithm 1 returns) into the workspace and the dense tensor-core kernel contracts it:
+                             for every 1 <= n <= m, m in {4, 8, 16, 32}, in particular the patterns of Section 4.2
+                             that leave more than two survivors in some aligned 4-chunk (3:4, 4:8, 4:16, 8:16,
+                             16:32, ...), which a 2:4 sparse tensor core cannot take; no speed-up over dense */
 };
 
 /* Algorithm 1 with pruning function `scheme` on dO viewed as [rows, K], groups of m along K.
@@ -90,9 +95,10 @@ sdgp_status sdgp_prune(const void* dO, int64_t rows, int64_t K, int n, int m, sd
 /* Fully connected data gradient (Section 2.1, Fig. 2): dD[r, c] = sum_k prune(dO)[r, k] * W[k, c].
  *   dO [rows, K] bf16, W [K, N] bf16 (output channels x input channels), dD [rows, N] bf16,
  *   fp32 accumulation, round-to-nearest-even bf16 result.
- * Requirements: K % 64 == 0, N % 64 == 0 (any rows >= 0); pruned modes need n <= 2, m in {4,8,16,32}
- * dividing K (or n == m, which prunes nothing). Workspace: sdgp_workspace_size_linear() bytes,
- * 256-byte aligned (the compressed rows are padded to whole blocks of 128 channels). */
+ * Requirements: K % 64 == 0, N % 64 == 0 (any rows >= 0); m in {4,8,16,32} dividing K; the sparse
+ * modes (two-pass, fused) need n <= 2 (or n == m, which prunes nothing), SDGP_FLAG_MASKED takes any
+ * n <= m. Workspace: sdgp_workspace_size_linear() bytes, 256-byte aligned (two-pass: the compressed
+ * rows, padded to whole blocks of 128 channels; masked: the pruned dense copy, rows * K * 2 bytes). */
 sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,
                               int64_t N, int n, int m, sdgp_scheme scheme, uint64_t seed,
                               void* workspace, size_t workspace_bytes, uint32_t flags, void* stream);
@@ -137,7 +143,7 @@ sdgp_status sdgp_dgrad_linear_static(const void* dO, const void* W, void* dD, in
                                      void* stream);
 
 /* Bytes of workspace the matching dgrad call needs for these shapes and flags (0 for
- * SDGP_FLAG_DENSE and SDGP_FLAG_FUSED). */
+ * SDGP_FLAG_DENSE and SDGP_FLAG_FUSED; the size of dL/dO for SDGP_FLAG_MASKED). */
 size_t sdgp_workspace_size_linear(int64_t rows, int64_t K, int64_t N, uint32_t flags);
 size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R, int S, int stride,
                                   int pad, uint32_t flags);

@@ -14,7 +14,7 @@ import torch
 from . import build as _build
 
 RANDOM, MAGNITUDE, RESCALED_MAGNITUDE = 0, 1, 2
-FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE = 0, 1, 2
+FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE, FLAG_MASKED = 0, 1, 2, 3
 
 EXPORTS = ["sdgp_prune", "sdgp_dgrad_linear", "sdgp_dgrad_conv2d", "sdgp_spmm_linear", "sdgp_spmm_conv2d",
            "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",

@@ -72,16 +72,19 @@ sdgp_status sdgp_prune(const void* dO, int64_t rows, int64_t K, int n, int m, sd
 
 size_t sdgp_workspace_size_linear(int64_t rows, int64_t K, int64_t N, uint32_t flags) {
   (void)N;
-  if (flags != SDGP_FLAG_TWO_PASS || rows <= 0 || K <= 0) return 0;
+  if (rows <= 0 || K <= 0) return 0;
+  if (flags == SDGP_FLAG_MASKED) return round_up((size_t)rows * (size_t)K * 2, 256);
+  if (flags != SDGP_FLAG_TWO_PASS) return 0;
   return carve_compressed(nullptr, rows * pad128(K)).bytes;
 }
 
 size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R, int S, int stride,
                                   int pad, uint32_t flags) {
   (void)Cin;
-  if (flags != SDGP_FLAG_TWO_PASS || stride < 1) return 0;
+  if ((flags != SDGP_FLAG_TWO_PASS && flags != SDGP_FLAG_MASKED) || stride < 1) return 0;
   const int64_t P = (H + 2 * pad - R) / stride + 1, Q = (Wd + 2 * pad - S) / stride + 1;
   if (B <= 0 || P <= 0 || Q <= 0 || Cout <= 0) return 0;
+  if (flags == SDGP_FLAG_MASKED) return round_up((size_t)B * P * Q * Cout * 2, 256);
   return carve_compressed(nullptr, (int64_t)B * P * Q * pad128(Cout)).bytes;
 }
 
@@ -112,13 +115,13 @@ sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, in
                               size_t workspace_bytes, uint32_t flags, void* stream) {
   if (B < 0 || H < 0 || Wd < 0 || Cin < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0)
     return SDGP_ERR_INVALID_ARG;
-  if (flags > SDGP_FLAG_DENSE) return SDGP_ERR_INVALID_ARG;
+  if (flags > SDGP_FLAG_MASKED) return SDGP_ERR_INVALID_ARG;
   if (stride > 2) return SDGP_ERR_UNSUPPORTED;
   if (pad > R - 1 || pad > S - 1) return SDGP_ERR_UNSUPPORTED;
   if (flags != SDGP_FLAG_DENSE) {
     sdgp_status st = check_prune_args(0, Cout, n, m, (int)scheme);
     if (st != SDGP_OK) return st;
-    if (n > 2 && n != m) return SDGP_ERR_UNSUPPORTED;
+    if (n > 2 && n != m && flags != SDGP_FLAG_MASKED) return SDGP_ERR_UNSUPPORTED;  // not 2:4-compatible
   }
   if ((int64_t)B * H * Wd == 0) return SDGP_OK;
   const int64_t P = (H + 2 * pad - R) / stride + 1, Q = (Wd + 2 * pad - S) / stride + 1;
@@ -129,6 +132,16 @@ sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, in
   if (flags == SDGP_FLAG_DENSE || n == m)
     return sdgp::launch_dgrad(false, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s);
   if (Cin % 64 != 0 || Cout % 64 != 0) return SDGP_ERR_UNSUPPORTED;
+  if (flags == SDGP_FLAG_MASKED) {
+    // Algorithm 1 as printed: a pruned dense copy, then the dense contraction
+    const size_t need = round_up((size_t)B * P * Q * Cout * 2, 256);
+    if (!workspace || workspace_bytes < need) return SDGP_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255u) != 0) return SDGP_ERR_ALIGNMENT;
+    cudaError_t e = sdgp::launch_prune(dO, (int64_t)B * P * Q, Cout, n, m, (int)scheme, seed, workspace, nullptr,
+                                       nullptr, nullptr, s);
+    if (e != cudaSuccess) return SDGP_ERR_CUDA;
+    return sdgp::launch_dgrad(false, workspace, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s);
+  }
   if (flags == SDGP_FLAG_FUSED) {
     if (m != 4) return SDGP_ERR_UNSUPPORTED;  // the in-kernel prune handles groups of four
     const sdgp::FusedPrune fp = {n, (int)scheme, seed};

@@ -455,28 +455,35 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   } else if (warp < 6) {
     // ------------------------------------------------- metadata rearranger
     if (SPARSE && !FUSED) {
-      // A lone warp runs a dependent chain slowly, so the four warps do not share a stage:
-      // warp k builds the TMEM metadata images of stage uses k, k+G, k+2G, ... (four passes of
-      // 32 lanes per image), G stages in flight.
-      // No more warps than stages take part: a warp's previous use then needed the use two ring
-      // passes back to be complete, so a parity wait can never be satisfied by a stale phase.
+      // A lone warp runs a dependent chain slowly, so the four warps do not share a stage: warp k
+      // owns stages k, k+G, ... of the ring and builds the TMEM metadata images of every use of
+      // those stages (four passes of 32 lanes per image); consecutive uses fall to different warps,
+      // so up to G are in flight.
+      // Ownership goes by STAGE, not by use: a parity wait tells "the phase I expect has completed"
+      // from "the phase two before it has" only if the waiter saw the phase in between complete.
+      // The warp that owns a stage waits for each of its uses in turn, so it always has. (A warp
+      // that took uses k, k+G, ... regardless of stage would wait for use u of a stage without
+      // having waited for use u - STAGES; that box was requested earlier than the boxes the warp
+      // did see land, but TMA boxes may land out of request order, and a box that is late lets
+      // the wait pass one phase early.)
       const int G = STAGES < 4 ? STAGES : 4;
       const int total_uses = (warp - 2 < G) ? my_tiles * uses_per_tile : 0;
-      int st = warp - 2;
       uint32_t ph = 0;
-      for (int u = warp - 2; u < total_uses; u += G) {
-        // the metadata box was requested after the stage's previous use had been consumed
-        if (!ptx::mbar_wait(&meta_full[st], ph, err, 0x500u + st)) break;
-        for (int v = 0; v < p.rr; ++v) {
-          const int row_off = reuse ? (p.R - 1 - v) * p.TW : 0;
-          build_metadata_image(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + v * kEHwBytes, lane,
-                               rows_used);
+      for (int first = 0; first < total_uses; first += STAGES, ph ^= 1u) {  // one pass over the ring
+        bool alive = true;
+        for (int st = warp - 2; st < STAGES && first + st < total_uses; st += G) {
+          // the metadata box was requested after the stage's previous use had been consumed
+          if (!ptx::mbar_wait(&meta_full[st], ph, err, 0x500u + st)) { alive = false; break; }
+          for (int v = 0; v < p.rr; ++v) {
+            const int row_off = reuse ? (p.R - 1 - v) * p.TW : 0;
+            build_metadata_image(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + v * kEHwBytes, lane,
+                                 rows_used);
+          }
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(&full[st], 0);
         }
-        ptx::fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive_cluster(&full[st], 0);
-        st += G;
-        while (st >= STAGES) { st -= STAGES; ph ^= 1u; }
+        if (!alive) break;
       }
     } else if (SPARSE) {
       // Fused pruning: the four warps prune the stage's pixel rows together (thread = row),
@@ -899,8 +906,12 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int w = lane & 7, hsub = lane >> 4;
       const uint32_t sel = (lane & 8) ? 0x7632u : 0x5410u;
       // No more warps than W stages take part: a warp's previous use then needed the use two
-      // ring passes back to be consumed, so a parity wait can never be satisfied by a stale phase.
-      const int G = WS < 4 ? WS : 4;
+      // ring passes back to be consumed (the MMA thread frees W stages in order), so the w_empty
+      // parity wait can never be satisfied by a stale phase. And no more warps than taps: every
+      // warp then has a tap in every A-stage use and waits for each phase of meta_full in turn
+      // (boxes may land out of request order; a warp that skipped a use could otherwise pass the
+      // wait one phase early when that use's box is late).
+      const int G = (WS < 4 ? WS : 4) < taps ? (WS < 4 ? WS : 4) : taps;
       const int total_uses = (warp - 2 < G) ? my_tiles * p.k_blocks * taps : 0;
       int t = warp - 2;  // tap within the channel block
       int ause = 0;      // A stage use = (tile set, channel block)

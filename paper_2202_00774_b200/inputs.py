@@ -125,6 +125,32 @@ def resnet50_stride1_layers(batch: int = 256) -> List[ConvLayer]:
     return out
 
 
+def resnet50_layers(batch: int = 256):
+    """Every distinct 1x1 / 3x3 convolution of the ResNet-50 bottleneck stages 1-4 with the number
+    of times the network holds it: (layer, count) pairs. The stride-2 transitions sit on the 3x3
+    convolution of each stage's first block and on its 1x1 projection shortcut."""
+    out = []
+    prev_wide = 64   # channels that enter stage 1 (from the stem)
+    for stage, (hw, mid, blocks) in enumerate([(56, 64, 3), (28, 128, 4), (14, 256, 6), (7, 512, 3)], start=1):
+        wide = 4 * mid
+        s = 1 if stage == 1 else 2
+        hin = hw * s   # spatial size entering the stage
+        tag = "r50_s%d_" % stage
+        # first block: reduce at the incoming size, 3x3 carries the stride, projection shortcut
+        out.append((ConvLayer(tag + "1x1_%dto%d_at%d" % (prev_wide, mid, hin), batch, hin, hin, prev_wide, mid, 1, 1, 1, 0), 1))
+        if s == 2:
+            out.append((ConvLayer(tag + "3x3s2_%dto%d_at%d" % (mid, mid, hin), batch, hin, hin, mid, mid, 3, 3, 2, 1), 1))
+        out.append((ConvLayer(tag + "proj%s_%dto%d_at%d" % ("s2" if s == 2 else "", prev_wide, wide, hin), batch, hin, hin,
+                              prev_wide, wide, 1, 1, s, 0), 1))
+        # remaining blocks (and the stride-1 3x3 / expand convolutions of every block)
+        out.append((ConvLayer(tag + "1x1_%dto%d_at%d" % (wide, mid, hw), batch, hw, hw, wide, mid, 1, 1, 1, 0), blocks - 1))
+        out.append((ConvLayer(tag + "3x3_%dto%d_at%d" % (mid, mid, hw), batch, hw, hw, mid, mid, 3, 3, 1, 1),
+                    blocks if s == 1 else blocks - 1))
+        out.append((ConvLayer(tag + "1x1_%dto%d_at%d" % (mid, wide, hw), batch, hw, hw, mid, wide, 1, 1, 1, 0), blocks))
+        prev_wide = wide
+    return out
+
+
 def conv_layer_tensors(layer: ConvLayer, seed: int):
     """(dO, W) for one layer: dO = ReLU-masked Laplace, W = He-normal N(0, 2/(R*S*Cin))."""
     dO = relu_masked_laplace_bf16(layer.dO_shape(), seed, stream=1)

@@ -76,3 +76,10 @@ def test_dgrad_rejects_bad_arguments_before_launch(lib):
     assert C(FAKE, FAKE, FAKE, 2, 8, 8, 64, 128, 3, 3, 1, 1, 2, 4, 1, 0, None, 0, 0, None) == 4
     assert lib.sdgp_workspace_size_conv2d(2, 8, 8, 64, 128, 3, 3, 1, 1, 0) == 2 * 8 * 8 * 128 * 9 // 8
     assert lib.sdgp_workspace_size_conv2d(2, 8, 8, 64, 128, 3, 3, 1, 1, 2) == 0
+    # masked mode: any n <= m, workspace = a dense copy of dL/dO
+    assert lib.sdgp_workspace_size_linear(128, 256, 128, 3) == 128 * 256 * 2
+    assert lib.sdgp_workspace_size_conv2d(2, 8, 8, 64, 128, 3, 3, 1, 1, 3) == 2 * 8 * 8 * 128 * 2
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 3, 4, 1, 0, None, 0, 3, None) == 4        # 3:4 masked: needs the workspace
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 3, 4, 1, 0, ws, 128 * 256 * 2 - 1, 3, None) == 4
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 5, 4, 1, 0, ws, 1 << 20, 3, None) == 1    # n > m
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 2, 4, 1, 0, ws, need, 4, None) == 1       # flags past the last mode

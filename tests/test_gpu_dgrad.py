@@ -70,6 +70,54 @@ def test_pruned_linear_two_pass(n, m, scheme):
     assert rel_fro(to_f64(dD), oracle.dgrad_linear(pruned, W)) <= TOL
 
 
+# Patterns with more than two survivors in some aligned 4-chunk have no 2:4 form: the masked mode
+# prunes into a dense copy and contracts it on the dense pipe (Algorithm 1 as printed; Section 4.2's
+# sparsity sweep 4:8 ... 16:32).
+@pytest.mark.parametrize("scheme", [oracle.RANDOM, oracle.MAGNITUDE, oracle.RESCALED])
+@pytest.mark.parametrize("n,m", [(3, 4), (4, 8), (4, 16), (8, 16), (4, 32), (16, 32), (2, 4), (8, 8)])
+def test_pruned_linear_masked(n, m, scheme):
+    import paper_2202_00774_b200 as sdgp
+    rows, K, N = 301, 384, 192
+    dO, W = inputs.fc_tensors(rows, K, N, seed=3 * n + m)
+    ws = torch.empty(sdgp.sdgp_workspace_size_linear(rows, K, N, sdgp.FLAG_MASKED), dtype=torch.uint8, device="cuda")
+    dD = torch.full((rows, N), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, n, m, scheme, seed=17, workspace=ws, flags=sdgp.FLAG_MASKED)
+    check_no_device_error()
+    pruned = oracle.prune(dO, n, m, scheme, 17, want=("dense",))["dense"]
+    # the workspace holds Algorithm 1's return value, bit for bit (n == m prunes nothing: dO is read directly)
+    assert n == m or np.array_equal(ws.cpu().numpy()[:rows * K * 2].view(np.uint16).reshape(rows, K), pruned)
+    assert rel_fro(to_f64(dD), oracle.dgrad_linear(pruned, W)) <= TOL
+
+
+@pytest.mark.parametrize("n,m,scheme", [(4, 8, oracle.MAGNITUDE), (3, 4, oracle.RESCALED), (8, 32, oracle.RANDOM)])
+@pytest.mark.parametrize("case", [(3, 16, 16, 64, 128, 3, 3, 1, 1), (2, 14, 14, 128, 64, 1, 1, 1, 0),
+                                  (2, 15, 13, 64, 128, 3, 3, 2, 1), (5, 8, 8, 128, 256, 3, 3, 1, 1)])
+def test_pruned_conv_masked(case, n, m, scheme):
+    import paper_2202_00774_b200 as sdgp
+    B, H, Wd, Cin, Cout, R, S, stride, pad = case
+    layer = inputs.ConvLayer("t", B, H, Wd, Cin, Cout, R, S, stride, pad)
+    dO, W = inputs.conv_layer_tensors(layer, seed=n + Cout)
+    ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(B, H, Wd, Cin, Cout, R, S, stride, pad, sdgp.FLAG_MASKED),
+                     dtype=torch.uint8, device="cuda")
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, stride, pad, n, m, scheme, seed=23, workspace=ws, flags=sdgp.FLAG_MASKED)
+    check_no_device_error()
+    pruned = oracle.prune(dO.reshape(-1, Cout), n, m, scheme, 23, want=("dense",))["dense"].reshape(dO.shape)
+    assert rel_fro(to_f64(dD), oracle.dgrad_conv2d(pruned, W, H, Wd, stride, pad)) <= TOL
+
+
+def test_sparse_modes_refuse_patterns_without_a_2_4_form():
+    import paper_2202_00774_b200 as sdgp
+    dO = torch.zeros((64, 128), dtype=torch.int16, device="cuda")
+    W = torch.zeros((128, 64), dtype=torch.int16, device="cuda")
+    dD = torch.zeros((64, 64), dtype=torch.int16, device="cuda")
+    ws = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
+    for flags in (sdgp.FLAG_TWO_PASS, sdgp.FLAG_FUSED):
+        with pytest.raises(sdgp.SdgpError) as e:
+            sdgp.sdgp_dgrad_linear(dO, W, dD, 4, 8, sdgp.MAGNITUDE, workspace=ws, flags=flags)
+        assert e.value.status == 2
+
+
 def test_fc_small_config_full():
     """The single-FC workload: dO [256,512], W [512,256], 2:4 magnitude, seed 0."""
     import paper_2202_00774_b200 as sdgp
