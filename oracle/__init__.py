@@ -19,6 +19,7 @@ _SRC = os.path.join(_HERE, "sdgp_oracle.c")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
 RANDOM, MAGNITUDE, RESCALED = 0, 1, 2
+BF16, FP16 = 0, 1   # element type of the 16-bit tensors (bf16 unless a call says otherwise)
 
 _lock = threading.Lock()
 _lib = None
@@ -44,6 +45,16 @@ def _load():
                                       ctypes.c_double)
             lib.oracle_prune.argtypes = [vp, i64, i64, i32, i32, i32, u64, vp, vp, vp, vp]
             lib.oracle_prune.restype = i32
+            lib.oracle_prune_t.argtypes = [vp, i64, i64, i32, i32, i32, i32, u64, vp, vp, vp, vp]
+            lib.oracle_prune_t.restype = i32
+            lib.oracle_dgrad_linear_t.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, i32]
+            lib.oracle_dgrad_linear_t.restype = i32
+            lib.oracle_dgrad_conv2d_t.argtypes = [vp, vp, vp] + [i32] * 9 + [vp, i64, i32]
+            lib.oracle_dgrad_conv2d_t.restype = i32
+            lib.oracle_f32_to_f16.argtypes = [ctypes.c_float]
+            lib.oracle_f32_to_f16.restype = ctypes.c_uint16
+            lib.oracle_f16_to_f64.argtypes = [ctypes.c_uint16]
+            lib.oracle_f16_to_f64.restype = dbl
             lib.oracle_expand.argtypes = [vp, vp, i64, i64, vp]
             lib.oracle_expand.restype = i32
             lib.oracle_dgrad_linear.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64]
@@ -81,9 +92,9 @@ def compressible(n: int, m: int) -> bool:
     return n <= 2 and m % 4 == 0
 
 
-def prune(dO, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask")):
+def prune(dO, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask"), dtype=BF16):
     """Algorithm 1 with the Section 3.2 pruning function ``scheme`` on a
-    ``[rows, K]`` uint16 array. Returns a dict with the requested outputs."""
+    ``[rows, K]`` uint16 array of ``dtype`` elements. Returns a dict with the requested outputs."""
     dO = _u16(dO)
     rows, K = dO.shape
     out = {}
@@ -95,8 +106,8 @@ def prune(dO, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask")):
         out["meta"] = np.empty((rows, K // 16), np.uint16)
     if "mask" in want:
         out["mask"] = np.empty((rows, K // 32), np.uint32)
-    rc = _load().oracle_prune(_ptr(dO), rows, K, n, m, scheme, seed, _ptr(out.get("dense")),
-                              _ptr(out.get("values")), _ptr(out.get("meta")), _ptr(out.get("mask")))
+    rc = _load().oracle_prune_t(_ptr(dO), rows, K, n, m, scheme, dtype, seed, _ptr(out.get("dense")),
+                                _ptr(out.get("values")), _ptr(out.get("meta")), _ptr(out.get("mask")))
     if rc != 0:
         raise ValueError("oracle_prune rejected its arguments (rc=%d)" % rc)
     return out
@@ -112,8 +123,8 @@ def expand(values, meta):
     return dense
 
 
-def dgrad_linear(dOp, W, row_index=None):
-    """dD = dOp @ W in fp64 from bf16 bit patterns; ``row_index`` evaluates a subset of rows."""
+def dgrad_linear(dOp, W, row_index=None, dtype=BF16):
+    """dD = dOp @ W in fp64 from 16-bit bit patterns; ``row_index`` evaluates a subset of rows."""
     dOp, W = _u16(dOp), _u16(W)
     rows, K = dOp.shape
     K2, N = W.shape
@@ -122,13 +133,13 @@ def dgrad_linear(dOp, W, row_index=None):
     idx = None if row_index is None else np.ascontiguousarray(row_index, dtype=np.int64)
     count = rows if idx is None else idx.shape[0]
     dD = np.empty((count, N), np.float64)
-    rc = _load().oracle_dgrad_linear(_ptr(dOp), _ptr(W), _ptr(dD), rows, K, N, _ptr(idx), count)
+    rc = _load().oracle_dgrad_linear_t(_ptr(dOp), _ptr(W), _ptr(dD), rows, K, N, _ptr(idx), count, dtype)
     if rc != 0:
         raise ValueError("oracle_dgrad_linear rejected its arguments")
     return dD
 
 
-def dgrad_conv2d(dOp, W, H, Wd, stride=1, pad=0, pixel_index=None):
+def dgrad_conv2d(dOp, W, H, Wd, stride=1, pad=0, pixel_index=None, dtype=BF16):
     """dD (NHWC, fp64) from dOp NHWC ``[B,P,Q,Cout]`` and W ``[Cout,R,S,Cin]`` (uint16)."""
     dOp, W = _u16(dOp), _u16(W)
     B, P, Q, Cout = dOp.shape
@@ -138,8 +149,8 @@ def dgrad_conv2d(dOp, W, H, Wd, stride=1, pad=0, pixel_index=None):
     idx = None if pixel_index is None else np.ascontiguousarray(pixel_index, dtype=np.int64)
     count = B * H * Wd if idx is None else idx.shape[0]
     dD = np.empty((count, Cin), np.float64)
-    rc = _load().oracle_dgrad_conv2d(_ptr(dOp), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S, stride,
-                                     pad, _ptr(idx), count)
+    rc = _load().oracle_dgrad_conv2d_t(_ptr(dOp), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S, stride,
+                                       pad, _ptr(idx), count, dtype)
     if rc != 0:
         raise ValueError("oracle_dgrad_conv2d rejected its arguments")
     return dD.reshape(B, H, Wd, Cin) if idx is None else dD
@@ -178,6 +189,14 @@ def f32_to_bf16(x):
 
 def bf16_to_f64(bits):
     return float(_load().oracle_bf16_to_f64(int(bits)))
+
+
+def f32_to_f16(x):
+    return int(_load().oracle_f32_to_f16(float(x)))
+
+
+def f16_to_f64(bits):
+    return float(_load().oracle_f16_to_f64(int(bits)))
 
 
 def bf16_array_to_f64(a):

@@ -29,7 +29,11 @@
  * function is pinned against an independent open-source engine at test time;
  * agreement with the authors' published known-answer vectors: parity unpinned.
  *
- * Storage: bf16 tensors travel as uint16_t bit patterns, row-major.
+ * Storage: 16-bit floating-point tensors travel as uint16_t bit patterns, row-major.
+ * Element type: bf16 (ORACLE_BF16, the default of the un-suffixed entry points) or IEEE
+ * binary16 (ORACLE_FP16, the precision the paper trained in, Section 4). The type only
+ * enters where a value is read as a number: the rescale of Section 3.2 and the contraction.
+ * Ranking by the bit pattern with the sign cleared orders both formats by magnitude.
  */
 #include <math.h>
 #include <stdint.h>
@@ -40,6 +44,7 @@
 #define ORACLE_ERR_ARG 1
 
 enum { ORACLE_RANDOM = 0, ORACLE_MAGNITUDE = 1, ORACLE_RESCALED = 2 };
+enum { ORACLE_BF16 = 0, ORACLE_FP16 = 1 };
 #define ORACLE_MAX_M 32 /* Section 3.1: the implementation supports groups up to m = 32 */
 
 /* ------------------------------------------------------------------ bf16 */
@@ -65,6 +70,56 @@ uint16_t oracle_f32_to_bf16(float f) {
   u += 0x7FFFu + lsb;
   return (uint16_t)(u >> 16);
 }
+
+/* ------------------------------------------------------------------ fp16 */
+
+/* IEEE binary16 -> fp32, exact: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static float f16_to_f32(uint16_t h) {
+  int exp = (h >> 10) & 0x1F;
+  int man = h & 0x3FF;
+  float mag;
+  if (exp == 0)
+    mag = ldexpf((float)man, -24); /* zero and subnormals: man * 2^-24 */
+  else if (exp == 31)
+    mag = man ? NAN : INFINITY;
+  else
+    mag = ldexpf((float)(man + 1024), exp - 25); /* (1 + man/1024) * 2^(exp-15) */
+  return (h & 0x8000u) ? -mag : mag;
+}
+
+/* fp32 -> binary16, round to nearest, ties to even: |f| is rounded to a whole multiple of
+ * the binary16 spacing at its magnitude (2^(e-10) for 2^e <= |f| < 2^(e+1), e >= -14; 2^-24
+ * below 2^-14), then packed. Overflow gives infinity; a NaN is stored as 0x7E00 (same
+ * reading as for bf16: one canonical quiet NaN). */
+uint16_t oracle_f32_to_f16(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+  uint32_t a = u & 0x7FFFFFFFu;
+  if (a > 0x7F800000u) return (uint16_t)0x7E00u;
+  if (a == 0x7F800000u) return (uint16_t)(sign | 0x7C00u);
+  if (a == 0) return sign;
+  float x = fabsf(f);
+  int e;
+  (void)frexpf(x, &e); /* x = frac * 2^e with frac in [0.5, 1): 2^(e-1) <= x < 2^e */
+  int ue = e - 1;
+  int q = (ue < -14 ? -14 : ue) - 10;      /* exponent of the spacing */
+  float r = nearbyintf(ldexpf(x, -q));    /* exact scaling, then nearest-even (default rounding mode) */
+  if (r == 0.0f) return sign;
+  if (ue < -14) return (uint16_t)(sign | (uint16_t)r); /* subnormal; r == 1024 is the smallest normal */
+  if (r == 2048.0f) {
+    r = 1024.0f;
+    ++ue;
+  }
+  if (ue > 15) return (uint16_t)(sign | 0x7C00u);
+  return (uint16_t)(sign | (uint16_t)((ue + 15) << 10) | (uint16_t)((int)r - 1024));
+}
+
+double oracle_f16_to_f64(uint16_t h) { return (double)f16_to_f32(h); }
+
+static float elem_to_f32(uint16_t bits, int dtype) { return dtype == ORACLE_FP16 ? f16_to_f32(bits) : bf16_to_f32(bits); }
+static uint16_t elem_from_f32(float f, int dtype) { return dtype == ORACLE_FP16 ? oracle_f32_to_f16(f) : oracle_f32_to_bf16(f); }
+static double elem_to_f64(uint16_t bits, int dtype) { return (double)elem_to_f32(bits, dtype); }
 
 /* ---------------------------------------------------------------- Philox */
 
@@ -126,7 +181,7 @@ static float tree_sum_f32(const float* a, int m) {
 
 /* P(group, n): Section 3.2. Fills keep[j] in {0,1} and out[j] (bf16 bits).
  * e0 is the linear index of the group's first element (random scheme only). */
-static void prune_group(const uint16_t* x, int n, int m, int scheme, uint64_t seed, uint64_t e0,
+static void prune_group(const uint16_t* x, int n, int m, int scheme, int dtype, uint64_t seed, uint64_t e0,
                         uint8_t* keep, uint16_t* out) {
   /* Rank: an index permutation ordered best-first, by a stable insertion sort
    * so that equal keys stay in index order (the lower index wins a tie). */
@@ -165,7 +220,7 @@ static void prune_group(const uint16_t* x, int n, int m, int scheme, uint64_t se
     /* Rescale the survivors so that the group's L1 norm is preserved. */
     float mag_all[ORACLE_MAX_M], mag_kept[ORACLE_MAX_M];
     for (int j = 0; j < m; ++j) {
-      float a = fabsf(bf16_to_f32(x[j]));
+      float a = fabsf(elem_to_f32(x[j], dtype));
       mag_all[j] = a;
       mag_kept[j] = keep[j] ? a : 0.0f;
     }
@@ -174,8 +229,8 @@ static void prune_group(const uint16_t* x, int n, int m, int scheme, uint64_t se
     volatile float scale = (S == 0.0f) ? 1.0f : T / S;
     for (int j = 0; j < m; ++j)
       if (keep[j]) {
-        volatile float y = bf16_to_f32(x[j]) * scale;
-        out[j] = oracle_f32_to_bf16(y);
+        volatile float y = elem_to_f32(x[j], dtype) * scale;
+        out[j] = elem_from_f32(y, dtype);
       }
   }
 }
@@ -190,8 +245,9 @@ static int compressible(int n, int m) { return n <= 2 && (m % 4) == 0; }
  *   mask   [rows, K/32]  u32   bit k%32 of word k/32 set iff element k is kept
  * values/meta need every 4-chunk to hold at most two survivors (n <= 2, m % 4 == 0)
  * and K % 16 == 0; mask needs K % 32 == 0. */
-int oracle_prune(const uint16_t* dO, int64_t rows, int64_t K, int n, int m, int scheme,
-                 uint64_t seed, uint16_t* dense, uint16_t* values, uint16_t* meta, uint32_t* mask) {
+int oracle_prune_t(const uint16_t* dO, int64_t rows, int64_t K, int n, int m, int scheme, int dtype,
+                   uint64_t seed, uint16_t* dense, uint16_t* values, uint16_t* meta, uint32_t* mask) {
+  if (dtype != ORACLE_BF16 && dtype != ORACLE_FP16) return ORACLE_ERR_ARG;
   if (!dO || rows < 0 || K < 0 || m < 1 || m > ORACLE_MAX_M || n < 1 || n > m) return ORACLE_ERR_ARG;
   if (K % m != 0) return ORACLE_ERR_ARG;
   if (scheme < 0 || scheme > 2) return ORACLE_ERR_ARG;
@@ -206,7 +262,7 @@ int oracle_prune(const uint16_t* dO, int64_t rows, int64_t K, int n, int m, int 
     uint8_t* row_keep = (uint8_t*)malloc((size_t)(K > 0 ? K : 1));
     for (int64_t g = 0; g < K / m; ++g) {
       uint64_t e0 = (uint64_t)r * (uint64_t)K + (uint64_t)(g * m);
-      prune_group(dO + r * K + g * m, n, m, scheme, seed, e0, row_keep + g * m, row_out + g * m);
+      prune_group(dO + r * K + g * m, n, m, scheme, dtype, seed, e0, row_keep + g * m, row_out + g * m);
     }
     if (dense) memcpy(dense + r * K, row_out, (size_t)K * sizeof(uint16_t));
     if (mask)
@@ -249,6 +305,11 @@ int oracle_prune(const uint16_t* dO, int64_t rows, int64_t K, int n, int m, int 
   return ORACLE_OK;
 }
 
+int oracle_prune(const uint16_t* dO, int64_t rows, int64_t K, int n, int m, int scheme,
+                 uint64_t seed, uint16_t* dense, uint16_t* values, uint16_t* meta, uint32_t* mask) {
+  return oracle_prune_t(dO, rows, K, n, m, scheme, ORACLE_BF16, seed, dense, values, meta, mask);
+}
+
 /* Inverse of the compressed format: rebuild the dense [rows, K] tensor. */
 int oracle_expand(const uint16_t* values, const uint16_t* meta, int64_t rows, int64_t K,
                   uint16_t* dense) {
@@ -271,8 +332,9 @@ int oracle_expand(const uint16_t* values, const uint16_t* meta, int64_t rows, in
  * dOp [rows, K], W [K, N] (output channels x input channels), fp64 accumulation
  * in ascending k. Rows may be a subset: row_index (nullable) lists which rows
  * of dOp to evaluate; dD then has n_rows rows in that order. */
-int oracle_dgrad_linear(const uint16_t* dOp, const uint16_t* W, double* dD, int64_t rows, int64_t K,
-                        int64_t N, const int64_t* row_index, int64_t n_rows) {
+int oracle_dgrad_linear_t(const uint16_t* dOp, const uint16_t* W, double* dD, int64_t rows, int64_t K,
+                          int64_t N, const int64_t* row_index, int64_t n_rows, int dtype) {
+  if (dtype != ORACLE_BF16 && dtype != ORACLE_FP16) return ORACLE_ERR_ARG;
   if (!dOp || !W || !dD || rows < 0 || K < 0 || N < 0) return ORACLE_ERR_ARG;
   int64_t count = row_index ? n_rows : rows;
 #pragma omp parallel for schedule(static)
@@ -281,11 +343,16 @@ int oracle_dgrad_linear(const uint16_t* dOp, const uint16_t* W, double* dD, int6
     for (int64_t c = 0; c < N; ++c) {
       double acc = 0.0;
       for (int64_t k = 0; k < K; ++k)
-        acc += oracle_bf16_to_f64(dOp[r * K + k]) * oracle_bf16_to_f64(W[k * N + c]);
+        acc += elem_to_f64(dOp[r * K + k], dtype) * elem_to_f64(W[k * N + c], dtype);
       dD[i * N + c] = acc;
     }
   }
   return ORACLE_OK;
+}
+
+int oracle_dgrad_linear(const uint16_t* dOp, const uint16_t* W, double* dD, int64_t rows, int64_t K,
+                        int64_t N, const int64_t* row_index, int64_t n_rows) {
+  return oracle_dgrad_linear_t(dOp, W, dD, rows, K, N, row_index, n_rows, ORACLE_BF16);
 }
 
 /* Convolution data gradient (Fig. 3). Forward layer: cross-correlation
@@ -295,9 +362,10 @@ int oracle_dgrad_linear(const uint16_t* dOp, const uint16_t* W, double* dD, int6
  *                  q*stride - pad + s == w of dOp[b,p,q,co] * W[co,r,s,ci].
  * dOp NHWC [B,P,Q,Cout], W [Cout,R,S,Cin], dD NHWC [B,H,Wd,Cin] in fp64.
  * pixel_index (nullable) lists flattened (b*H + h)*Wd + w positions to evaluate. */
-int oracle_dgrad_conv2d(const uint16_t* dOp, const uint16_t* W, double* dD, int B, int H, int Wd,
-                        int Cin, int Cout, int R, int S, int stride, int pad,
-                        const int64_t* pixel_index, int64_t n_pixels) {
+int oracle_dgrad_conv2d_t(const uint16_t* dOp, const uint16_t* W, double* dD, int B, int H, int Wd,
+                          int Cin, int Cout, int R, int S, int stride, int pad,
+                          const int64_t* pixel_index, int64_t n_pixels, int dtype) {
+  if (dtype != ORACLE_BF16 && dtype != ORACLE_FP16) return ORACLE_ERR_ARG;
   if (!dOp || !W || !dD || stride < 1 || pad < 0 || R < 1 || S < 1) return ORACLE_ERR_ARG;
   int P = (H + 2 * pad - R) / stride + 1;
   int Q = (Wd + 2 * pad - S) / stride + 1;
@@ -323,14 +391,20 @@ int oracle_dgrad_conv2d(const uint16_t* dOp, const uint16_t* W, double* dD, int 
           if (q >= Q) continue;
           const uint16_t* g = dOp + (((int64_t)b * P + p) * Q + q) * Cout;
           for (int co = 0; co < Cout; ++co)
-            acc += oracle_bf16_to_f64(g[co]) *
-                   oracle_bf16_to_f64(W[(((int64_t)co * R + r) * S + s) * Cin + ci]);
+            acc += elem_to_f64(g[co], dtype) *
+                   elem_to_f64(W[(((int64_t)co * R + r) * S + s) * Cin + ci], dtype);
         }
       }
       dD[i * Cin + ci] = acc;
     }
   }
   return ORACLE_OK;
+}
+
+int oracle_dgrad_conv2d(const uint16_t* dOp, const uint16_t* W, double* dD, int B, int H, int Wd,
+                        int Cin, int Cout, int R, int S, int stride, int pad,
+                        const int64_t* pixel_index, int64_t n_pixels) {
+  return oracle_dgrad_conv2d_t(dOp, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, pixel_index, n_pixels, ORACLE_BF16);
 }
 
 /* Direct forward convolution in fp64 on fp64 inputs; used only by the adjoint
