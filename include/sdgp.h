@@ -66,6 +66,12 @@ typedef enum {
 
 typedef enum { SDGP_RANDOM = 0, SDGP_MAGNITUDE = 1, SDGP_RESCALED_MAGNITUDE = 2 } sdgp_scheme;
 
+/* Element type of the 16-bit tensors of the *_typed entry points (the un-suffixed ones are bf16). */
+typedef enum {
+  SDGP_BF16 = 0, /* bfloat16 */
+  SDGP_FP16 = 1  /* IEEE binary16, the precision the paper's experiments trained in (Section 4) */
+} sdgp_dtype;
+
 /* `flags` of the dgrad entry points. */
 enum {
   SDGP_FLAG_TWO_PASS = 0, /* prune kernel writes compressed dL/dO into the workspace, sparse GEMM reads it */
@@ -124,6 +130,35 @@ sdgp_status sdgp_spmm_linear(const void* values, const void* meta, const void* W
 sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W, void* dD, int B,
                              int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
                              void* stream);
+
+/* The same five operations for tensors of element type `dtype` (dO, W, dD, the dense pruned copy and
+ * the compressed values alike); SDGP_BF16 is exactly the un-suffixed entry point. With SDGP_FP16:
+ *   - ranking and selection are unchanged (the binary16 pattern with the sign cleared orders
+ *     magnitudes just as the bf16 pattern does; NaN > Inf > finite), random keys likewise;
+ *   - SDGP_RESCALED_MAGNITUDE widens binary16 to fp32 exactly, sums, divides and multiplies in fp32
+ *     as above and rounds to nearest-even binary16 (overflow gives infinity; a NaN result is
+ *     stored as 0x7E00);
+ *   - the contraction multiplies binary16 operands on the tensor cores with fp32 accumulation and
+ *     rounds dD to nearest-even binary16;
+ *   - SDGP_FLAG_FUSED with SDGP_RESCALED_MAGNITUDE returns SDGP_ERR_UNSUPPORTED (the in-kernel
+ *     prune of that scheme exists for bf16 only).
+ * Any other dtype value: SDGP_ERR_INVALID_ARG. */
+sdgp_status sdgp_prune_typed(const void* dO, int64_t rows, int64_t K, int n, int m, sdgp_scheme scheme,
+                             uint64_t seed, sdgp_dtype dtype, void* dOp_dense, void* values, void* meta,
+                             void* mask, void* stream);
+sdgp_status sdgp_dgrad_linear_typed(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,
+                                    int64_t N, int n, int m, sdgp_scheme scheme, uint64_t seed,
+                                    sdgp_dtype dtype, void* workspace, size_t workspace_bytes,
+                                    uint32_t flags, void* stream);
+sdgp_status sdgp_dgrad_conv2d_typed(const void* dO, const void* W, void* dD, int B, int H, int Wd, int Cin,
+                                    int Cout, int R, int S, int stride, int pad, int n, int m,
+                                    sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* workspace,
+                                    size_t workspace_bytes, uint32_t flags, void* stream);
+sdgp_status sdgp_spmm_linear_typed(const void* values, const void* meta, const void* W, void* dD,
+                                   int64_t rows, int64_t K, int64_t N, sdgp_dtype dtype, void* stream);
+sdgp_status sdgp_spmm_conv2d_typed(const void* values, const void* meta, const void* W, void* dD, int B,
+                                   int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
+                                   sdgp_dtype dtype, void* stream);
 
 /* No counterpart in the paper: a convenience variant of sdgp_dgrad_linear (two-pass mode) that
  * takes no workspace and allocates nothing - for callers that cannot call cudaMalloc where

@@ -18,7 +18,8 @@
  * Readings taken where the paper is silent (each is listed in the design notes):
  *   - ties between equal magnitudes go to the lower index;
  *   - magnitude order is the order of the bf16 bit pattern with the sign cleared;
- *   - the L1 rescale is per group, in fp32, with a fixed balanced summation tree;
+ *   - the L1 rescale is per group, in fp32, with a fixed balanced summation tree; a group
+ *     from which nothing is pruned (n == m) is returned unchanged;
  *   - "random" ranks elements by 16-bit keys drawn from Philox4x32-10
  *     (Salmon et al., SC'11) at a counter fixed by the element's linear index;
  *   - pruned positions hold +0.0.
@@ -216,8 +217,10 @@ static void prune_group(const uint16_t* x, int n, int m, int scheme, int dtype, 
     keep[order[i]] = 1;
     out[order[i]] = x[order[i]];
   }
-  if (scheme == ORACLE_RESCALED) {
-    /* Rescale the survivors so that the group's L1 norm is preserved. */
+  if (scheme == ORACLE_RESCALED && n < m) {
+    /* Rescale the survivors so that the group's L1 norm is preserved. With n == m nothing was
+     * pruned, the norm is preserved as it stands and the group is returned unchanged (no
+     * division takes place, so a group holding Inf or NaN is not turned into NaNs). */
     float mag_all[ORACLE_MAX_M], mag_kept[ORACLE_MAX_M];
     for (int j = 0; j < m; ++j) {
       float a = fabsf(elem_to_f32(x[j], dtype));

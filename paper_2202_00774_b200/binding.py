@@ -16,8 +16,10 @@ from . import build as _build
 RANDOM, MAGNITUDE, RESCALED_MAGNITUDE = 0, 1, 2
 FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE, FLAG_MASKED = 0, 1, 2, 3
 
+BF16, FP16 = 0, 1   # sdgp_dtype
 EXPORTS = ["sdgp_prune", "sdgp_dgrad_linear", "sdgp_dgrad_conv2d", "sdgp_spmm_linear", "sdgp_spmm_conv2d",
-           "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
+           "sdgp_prune_typed", "sdgp_dgrad_linear_typed", "sdgp_dgrad_conv2d_typed", "sdgp_spmm_linear_typed",
+           "sdgp_spmm_conv2d_typed", "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
            "sdgp_workspace_size_linear", "sdgp_workspace_size_conv2d", "sdgp_last_device_error",
            "sdgp_status_string"]
 
@@ -54,6 +56,16 @@ def lib() -> ctypes.CDLL:
         L.sdgp_spmm_linear.restype = i32
         L.sdgp_spmm_conv2d.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
         L.sdgp_spmm_conv2d.restype = i32
+        L.sdgp_prune_typed.argtypes = [vp, i64, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp]
+        L.sdgp_prune_typed.restype = i32
+        L.sdgp_dgrad_linear_typed.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, u64, i32, vp, sz, u32, vp]
+        L.sdgp_dgrad_linear_typed.restype = i32
+        L.sdgp_dgrad_conv2d_typed.argtypes = [vp, vp, vp] + [i32] * 9 + [i32, i32, i32, u64, i32, vp, sz, u32, vp]
+        L.sdgp_dgrad_conv2d_typed.restype = i32
+        L.sdgp_spmm_linear_typed.argtypes = [vp, vp, vp, vp, i64, i64, i64, i32, vp]
+        L.sdgp_spmm_linear_typed.restype = i32
+        L.sdgp_spmm_conv2d_typed.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [i32, vp]
+        L.sdgp_spmm_conv2d_typed.restype = i32
         L.sdgp_workspace_size_linear.argtypes = [i64, i64, i64, u32]
         L.sdgp_workspace_size_linear.restype = sz
         L.sdgp_workspace_size_conv2d.argtypes = [i32] * 9 + [u32]
@@ -160,6 +172,58 @@ def sdgp_spmm_conv2d(values, meta, W, dD, stride, pad):
     Cout, R, S, _ = W.shape
     _check(lib().sdgp_spmm_conv2d(_ptr(values), _ptr(meta), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S,
                                   stride, pad, _stream()), "sdgp_spmm_conv2d")
+
+
+# ---- the same operations on tensors of an explicit element type (sdgp_dtype: BF16 or FP16) ----
+
+
+def sdgp_prune_typed(dO, n, m, scheme, seed, dtype, dense=None, values=None, meta=None, mask=None):
+    """``sdgp_prune_typed``: :func:`sdgp_prune` for 2-byte elements of type ``dtype``."""
+    for t, name in ((dO, "dO"), (dense, "dense"), (values, "values"), (meta, "meta"), (mask, "mask")):
+        _dev(t, name)
+    K = dO.shape[-1] if dO.dim() else 0
+    rows = dO.numel() // K if K else 0
+    _check(lib().sdgp_prune_typed(_ptr(dO), rows, K, n, m, scheme, seed, dtype, _ptr(dense), _ptr(values),
+                                  _ptr(meta), _ptr(mask), _stream()), "sdgp_prune_typed")
+
+
+def sdgp_dgrad_linear_typed(dO, W, dD, n, m, scheme, seed, dtype, workspace=None, flags=FLAG_TWO_PASS):
+    for t, name in ((dO, "dO"), (W, "W"), (dD, "dD"), (workspace, "workspace")):
+        _dev(t, name)
+    rows, K = dO.shape
+    N = W.shape[1]
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().sdgp_dgrad_linear_typed(_ptr(dO), _ptr(W), _ptr(dD), rows, K, N, n, m, scheme, seed, dtype,
+                                         _ptr(workspace), ws_bytes, flags, _stream()), "sdgp_dgrad_linear_typed")
+
+
+def sdgp_dgrad_conv2d_typed(dO, W, dD, stride, pad, n, m, scheme, seed, dtype, workspace=None, flags=FLAG_TWO_PASS):
+    for t, name in ((dO, "dO"), (W, "W"), (dD, "dD"), (workspace, "workspace")):
+        _dev(t, name)
+    B, H, Wd, Cin = dD.shape
+    Cout, R, S, _ = W.shape
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().sdgp_dgrad_conv2d_typed(_ptr(dO), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S, stride, pad, n, m,
+                                         scheme, seed, dtype, _ptr(workspace), ws_bytes, flags, _stream()),
+           "sdgp_dgrad_conv2d_typed")
+
+
+def sdgp_spmm_linear_typed(values, meta, W, dD, dtype):
+    for t, name in ((values, "values"), (meta, "meta"), (W, "W"), (dD, "dD")):
+        _dev(t, name)
+    rows, N = dD.shape
+    K = W.shape[0]
+    _check(lib().sdgp_spmm_linear_typed(_ptr(values), _ptr(meta), _ptr(W), _ptr(dD), rows, K, N, dtype, _stream()),
+           "sdgp_spmm_linear_typed")
+
+
+def sdgp_spmm_conv2d_typed(values, meta, W, dD, stride, pad, dtype):
+    for t, name in ((values, "values"), (meta, "meta"), (W, "W"), (dD, "dD")):
+        _dev(t, name)
+    B, H, Wd, Cin = dD.shape
+    Cout, R, S, _ = W.shape
+    _check(lib().sdgp_spmm_conv2d_typed(_ptr(values), _ptr(meta), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S,
+                                        stride, pad, dtype, _stream()), "sdgp_spmm_conv2d_typed")
 
 
 def sdgp_selftest_bounded_wait():

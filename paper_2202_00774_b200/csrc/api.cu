@@ -5,6 +5,8 @@ namespace {
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
+bool valid_dtype(sdgp_dtype d) { return d == SDGP_BF16 || d == SDGP_FP16; }
+
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // The sparse contraction works on whole blocks of 128 channels; the compressed workspace rows are
@@ -57,6 +59,13 @@ const char* sdgp_status_string(sdgp_status status) {
 sdgp_status sdgp_prune(const void* dO, int64_t rows, int64_t K, int n, int m, sdgp_scheme scheme,
                        uint64_t seed, void* dOp_dense, void* values, void* meta, void* mask,
                        void* stream) {
+  return sdgp_prune_typed(dO, rows, K, n, m, scheme, seed, SDGP_BF16, dOp_dense, values, meta, mask, stream);
+}
+
+sdgp_status sdgp_prune_typed(const void* dO, int64_t rows, int64_t K, int n, int m, sdgp_scheme scheme,
+                             uint64_t seed, sdgp_dtype dtype, void* dOp_dense, void* values, void* meta,
+                             void* mask, void* stream) {
+  if (!valid_dtype(dtype)) return SDGP_ERR_INVALID_ARG;
   sdgp_status st = check_prune_args(rows, K, n, m, (int)scheme);
   if (st != SDGP_OK) return st;
   if (rows == 0 || K == 0) return SDGP_OK;
@@ -66,7 +75,7 @@ sdgp_status sdgp_prune(const void* dO, int64_t rows, int64_t K, int n, int m, sd
   if (!aligned16(dO) || !aligned16(dOp_dense) || !aligned16(values) || !aligned16(meta) || !aligned16(mask))
     return SDGP_ERR_ALIGNMENT;
   cudaError_t e = sdgp::launch_prune(dO, rows, K, n, m, (int)scheme, seed, dOp_dense, values, meta, mask,
-                                     (cudaStream_t)stream);
+                                     (cudaStream_t)stream, 0, (int)dtype);
   return e == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
@@ -91,6 +100,13 @@ size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R
 sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W, void* dD, int B,
                              int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
                              void* stream) {
+  return sdgp_spmm_conv2d_typed(values, meta, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, SDGP_BF16, stream);
+}
+
+sdgp_status sdgp_spmm_conv2d_typed(const void* values, const void* meta, const void* W, void* dD, int B,
+                                   int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
+                                   sdgp_dtype dtype, void* stream) {
+  if (!valid_dtype(dtype)) return SDGP_ERR_INVALID_ARG;
   if (B < 0 || H < 0 || Wd < 0 || Cin < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0)
     return SDGP_ERR_INVALID_ARG;
   if (stride > 2) return SDGP_ERR_UNSUPPORTED;
@@ -99,20 +115,35 @@ sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W
   if ((int64_t)B * H * Wd == 0) return SDGP_OK;
   if (!values || !meta || !W || !dD) return SDGP_ERR_INVALID_ARG;
   if (!aligned16(values) || !aligned16(meta) || !aligned16(W) || !aligned16(dD)) return SDGP_ERR_ALIGNMENT;
-  return sdgp::launch_dgrad(true, values, meta, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, (cudaStream_t)stream);
+  return sdgp::launch_dgrad(true, values, meta, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, (cudaStream_t)stream,
+                            nullptr, (int)dtype);
 }
 
 sdgp_status sdgp_spmm_linear(const void* values, const void* meta, const void* W, void* dD,
                              int64_t rows, int64_t K, int64_t N, void* stream) {
+  return sdgp_spmm_linear_typed(values, meta, W, dD, rows, K, N, SDGP_BF16, stream);
+}
+
+sdgp_status sdgp_spmm_linear_typed(const void* values, const void* meta, const void* W, void* dD,
+                                   int64_t rows, int64_t K, int64_t N, sdgp_dtype dtype, void* stream) {
   if (rows < 0 || K < 1 || N < 1) return SDGP_ERR_INVALID_ARG;
   if (rows > 0x7FFFFFFF || K > 0x7FFFFFFF || N > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
-  return sdgp_spmm_conv2d(values, meta, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 1, 0, stream);
+  return sdgp_spmm_conv2d_typed(values, meta, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 1, 0, dtype, stream);
 }
 
 sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, int H, int Wd, int Cin,
                               int Cout, int R, int S, int stride, int pad, int n, int m,
                               sdgp_scheme scheme, uint64_t seed, void* workspace,
                               size_t workspace_bytes, uint32_t flags, void* stream) {
+  return sdgp_dgrad_conv2d_typed(dO, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, n, m, scheme, seed, SDGP_BF16,
+                                 workspace, workspace_bytes, flags, stream);
+}
+
+sdgp_status sdgp_dgrad_conv2d_typed(const void* dO, const void* W, void* dD, int B, int H, int Wd, int Cin,
+                                    int Cout, int R, int S, int stride, int pad, int n, int m,
+                                    sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* workspace,
+                                    size_t workspace_bytes, uint32_t flags, void* stream) {
+  if (!valid_dtype(dtype)) return SDGP_ERR_INVALID_ARG;
   if (B < 0 || H < 0 || Wd < 0 || Cin < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0)
     return SDGP_ERR_INVALID_ARG;
   if (flags > SDGP_FLAG_MASKED) return SDGP_ERR_INVALID_ARG;
@@ -129,8 +160,9 @@ sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, in
   if (!dO || !W || !dD) return SDGP_ERR_INVALID_ARG;
   if (!aligned16(dO) || !aligned16(W) || !aligned16(dD)) return SDGP_ERR_ALIGNMENT;
   cudaStream_t s = (cudaStream_t)stream;
+  const int dt = (int)dtype;
   if (flags == SDGP_FLAG_DENSE || n == m)
-    return sdgp::launch_dgrad(false, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s);
+    return sdgp::launch_dgrad(false, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, nullptr, dt);
   if (Cin % 64 != 0 || Cout % 64 != 0) return SDGP_ERR_UNSUPPORTED;
   if (flags == SDGP_FLAG_MASKED) {
     // Algorithm 1 as printed: a pruned dense copy, then the dense contraction
@@ -138,32 +170,41 @@ sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, in
     if (!workspace || workspace_bytes < need) return SDGP_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255u) != 0) return SDGP_ERR_ALIGNMENT;
     cudaError_t e = sdgp::launch_prune(dO, (int64_t)B * P * Q, Cout, n, m, (int)scheme, seed, workspace, nullptr,
-                                       nullptr, nullptr, s);
+                                       nullptr, nullptr, s, 0, dt);
     if (e != cudaSuccess) return SDGP_ERR_CUDA;
-    return sdgp::launch_dgrad(false, workspace, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s);
+    return sdgp::launch_dgrad(false, workspace, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, nullptr, dt);
   }
   if (flags == SDGP_FLAG_FUSED) {
     if (m != 4) return SDGP_ERR_UNSUPPORTED;  // the in-kernel prune handles groups of four
+    if (dtype == SDGP_FP16 && scheme == SDGP_RESCALED_MAGNITUDE) return SDGP_ERR_UNSUPPORTED;  // bf16 arithmetic only
     const sdgp::FusedPrune fp = {n, (int)scheme, seed};
-    return sdgp::launch_dgrad(true, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, &fp);
+    return sdgp::launch_dgrad(true, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, &fp, dt);
   }
   const int64_t Cpad = pad128(Cout);
   const Carve c = carve_compressed(workspace, (int64_t)B * P * Q * Cpad);
   if (!workspace || workspace_bytes < c.bytes) return SDGP_ERR_WORKSPACE;
   if (((uintptr_t)workspace & 255u) != 0) return SDGP_ERR_ALIGNMENT;
   cudaError_t e = sdgp::launch_prune(dO, (int64_t)B * P * Q, Cout, n, m, (int)scheme, seed, nullptr, c.values,
-                                     c.meta, nullptr, s, Cpad);
+                                     c.meta, nullptr, s, Cpad, dt);
   if (e != cudaSuccess) return SDGP_ERR_CUDA;
-  return sdgp::launch_dgrad(true, c.values, c.meta, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s);
+  return sdgp::launch_dgrad(true, c.values, c.meta, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, nullptr, dt);
 }
 
 sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,
                               int64_t N, int n, int m, sdgp_scheme scheme, uint64_t seed,
                               void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
+  return sdgp_dgrad_linear_typed(dO, W, dD, rows, K, N, n, m, scheme, seed, SDGP_BF16, workspace, workspace_bytes,
+                                 flags, stream);
+}
+
+sdgp_status sdgp_dgrad_linear_typed(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,
+                                    int64_t N, int n, int m, sdgp_scheme scheme, uint64_t seed,
+                                    sdgp_dtype dtype, void* workspace, size_t workspace_bytes,
+                                    uint32_t flags, void* stream) {
   if (rows < 0 || K < 1 || N < 1) return SDGP_ERR_INVALID_ARG;
   if (rows > 0x7FFFFFFF || K > 0x7FFFFFFF || N > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
-  return sdgp_dgrad_conv2d(dO, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 1, 0, n, m, scheme, seed,
-                           workspace, workspace_bytes, flags, stream);
+  return sdgp_dgrad_conv2d_typed(dO, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 1, 0, n, m, scheme, seed, dtype,
+                                 workspace, workspace_bytes, flags, stream);
 }
 
 sdgp_status sdgp_last_device_error(void) { return sdgp::read_device_error(); }

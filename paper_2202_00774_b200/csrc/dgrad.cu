@@ -84,6 +84,7 @@ struct DgradParams {
   int fused_n, fused_scheme;
   uint32_t seed_lo, seed_hi;
   int P, Q;               // dO pixel grid (for the linear element index of the random scheme)
+  int f16;                // element type of A, W and dD: 0 = bf16, 1 = IEEE binary16
   int off_raw;            // dense dL/dO stages: 2 * a_bytes each (two boxes of 64 channels)
   // shared-memory carve (byte offsets from the 1024-aligned base) and per-stage sizes
   int a_bytes, b_bytes, eraw_bytes, ehw_bytes;
@@ -109,6 +110,9 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool sparse) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
          ((uint32_t)(256 >> 4) << 24) | (sparse ? (1u << 2) : 0u);
 }
+// The A-format (bits 7-9) and B-format (bits 10-12) fields: 1 = bf16, 0 = binary16. Both operands
+// always have the same type.
+constexpr uint32_t kIdescBf16Operands = (1u << 7) | (1u << 10);
 
 // Metadata of an A tile: from the row-major order TMA delivers (16 bytes per pixel row: one uint16
 // per 16 channels of a 128-channel block) to the order tcgen05.cp moves into TMEM. For the MMA
@@ -191,7 +195,7 @@ template <int BN>
 __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* staging, int out_bufs,
                                                   const CUtensorMap* tmD, int n0, int w0, int h0, int b0,
                                                   bool tile_in_range, int row, bool issuer, uint32_t& chunk,
-                                                  uint64_t* first_slab_read) {
+                                                  uint64_t* first_slab_read, bool f16) {
 #pragma unroll 1
   for (int c0 = 0; c0 < BN; c0 += 64, ++chunk) {
     uint32_t packed[32];
@@ -206,12 +210,22 @@ __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* stagi
       __syncwarp();
       if ((threadIdx.x & 31) == 0) ptx::mbar_arrive_cluster(first_slab_read, 0);
     }
+    if (f16) {
 #pragma unroll
-    for (int e = 0; e < 16; ++e) {
-      const __nv_bfloat162 a2 = __floats2bfloat162_rn(__uint_as_float(v0[2 * e]), __uint_as_float(v0[2 * e + 1]));
-      const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v1[2 * e]), __uint_as_float(v1[2 * e + 1]));
-      packed[e] = *(const uint32_t*)&a2;
-      packed[16 + e] = *(const uint32_t*)&b2;
+      for (int e = 0; e < 16; ++e) {
+        const __half2 a2 = __floats2half2_rn(__uint_as_float(v0[2 * e]), __uint_as_float(v0[2 * e + 1]));
+        const __half2 b2 = __floats2half2_rn(__uint_as_float(v1[2 * e]), __uint_as_float(v1[2 * e + 1]));
+        packed[e] = *(const uint32_t*)&a2;
+        packed[16 + e] = *(const uint32_t*)&b2;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const __nv_bfloat162 a2 = __floats2bfloat162_rn(__uint_as_float(v0[2 * e]), __uint_as_float(v0[2 * e + 1]));
+        const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v1[2 * e]), __uint_as_float(v1[2 * e + 1]));
+        packed[e] = *(const uint32_t*)&a2;
+        packed[16 + e] = *(const uint32_t*)&b2;
+      }
     }
     uint8_t* buf = staging + (out_bufs == 2 ? (chunk & 1u) : 0u) * kOutBytes;
     if (issuer) {  // the store that last used this slab has finished reading it
@@ -382,7 +396,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     // A single thread executes roughly one dependent instruction per ten clocks, so its path
     // per stage is short: one barrier wait, descriptor words kept as running sums.
     if (rank == 0 && ptx::elect_one()) {
-      constexpr uint32_t idesc = make_idesc(BN, SPARSE);
+      const uint32_t idesc = make_idesc(BN, SPARSE) & ~(p.f16 ? kIdescBf16Operands : 0u);
       bool alive = true;
       if (p.w_resident) alive = ptx::mbar_wait(w_full, 0u, err, 0x700u);
       // descriptors as two 32-bit halves: the start address only ever changes the low word
@@ -551,7 +565,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       ptx::tc_fence_after_sync();
       store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), sOut, p.out_bufs, &tmD,
                             nt * BN, wt * p.TW, ht * p.TH, bt * p.TB, mt < p.m_tiles, row, issuer, chunk,
-                            p.meta_shared ? &meta_free[acc] : nullptr);
+                            p.meta_shared ? &meta_free[acc] : nullptr, p.f16 != 0);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
@@ -619,6 +633,7 @@ struct HaloParams {
   int fused_n, fused_scheme;
   uint32_t seed_lo, seed_hi;
   int P, Q;                // dO pixel grid (linear element index of the random scheme)
+  int f16;                 // element type of A, W and dD: 0 = bf16, 1 = IEEE binary16
 };
 
 // Fused pruning of one quarter (32 channels = 4 vectors) of one pixel row of a dense A box that
@@ -814,7 +829,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // kept short: one barrier wait, running descriptor words updated by additions, compile-time
     // offsets for the strips and the four MMAs of a channel block.
     if (rank == 0 && ptx::elect_one()) {
-      constexpr uint32_t idesc = make_idesc(BN, SPARSE);
+      const uint32_t idesc = make_idesc(BN, SPARSE) & ~(p.f16 ? kIdescBf16Operands : 0u);
       // descriptors as two 32-bit halves: the start address only ever changes the low word
       const uint64_t adesc0 = ptx::make_smem_desc(0, 16, (uint32_t)p.pitch * 128u, 2);
       const uint64_t bdesc0 = ptx::make_smem_desc(0, C::kBoxBytes, 8 * C::kRowB, C::kBSwizzle);
@@ -1035,7 +1050,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * set_cols + j * BN), sOut,
                               p.out_bufs, &tmD, n0, w0 + 8 * j, h0, b0, in_range && (w0 + 8 * j < p.W) && (strips & (1u << j)), row,
                               issuer,
-                              chunk, (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr);
+                              chunk, (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr, p.f16 != 0);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
@@ -1448,8 +1463,10 @@ sdgp_status launch_halo(const void* A, const void* meta, const void* Wt, const D
 // (m = 4, n = fused->n in {1, 2}); no compressed tensor exists in global memory.
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
                          int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
-                         const FusedPrune* fused) {
+                         const FusedPrune* fused, int dtype) {
   if (fused && (!sparse || fused->n < 1 || fused->n > 2)) return SDGP_ERR_UNSUPPORTED;
+  if (dtype != SDGP_BF16 && dtype != SDGP_FP16) return SDGP_ERR_INVALID_ARG;
+  if (fused && dtype == SDGP_FP16 && fused->scheme == SDGP_RESCALED_MAGNITUDE) return SDGP_ERR_UNSUPPORTED;
   if (stride != 1 && stride != 2) return SDGP_ERR_UNSUPPORTED;
   const int P = (H + 2 * pad - R) / stride + 1, Q = (W + 2 * pad - S) / stride + 1;
   if (P < 1 || Q < 1) return SDGP_ERR_INVALID_ARG;
@@ -1496,6 +1513,7 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
       p.pair_tiles = (int)((m_tiles + 1) / 2) * p.tiles_n;
       p.k_blocks = (Cout + kb_channels - 1) / kb_channels;
       p.P = P; p.Q = Q;
+      p.f16 = dtype == SDGP_FP16 ? 1 : 0;
       if (fused) {
         p.fused_n = fused->n; p.fused_scheme = fused->scheme;
         p.seed_lo = (uint32_t)fused->seed; p.seed_hi = (uint32_t)(fused->seed >> 32);
@@ -1513,6 +1531,7 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
         hp.S_full = S;
         hp.tiles_n = p.tiles_n; hp.k_blocks = p.k_blocks;
         hp.P = P; hp.Q = Q;
+        hp.f16 = p.f16;
         if (fused) {
           hp.fused_n = p.fused_n; hp.fused_scheme = p.fused_scheme; hp.seed_lo = p.seed_lo; hp.seed_hi = p.seed_hi;
           st = BN == 256 ? launch_halo<true, 256, true>(A, meta, Wt, view, hp, stream)

@@ -42,7 +42,7 @@ cudaError_t launch_after_previous(void (*kernel)(Params...), dim3 grid, dim3 blo
 }
 
 // M: group size; LANES = lanes that share a group (1, 2 or 4).
-template <int M, int SCHEME>
+template <int M, int SCHEME, bool F16>
 __global__ void __launch_bounds__(kThreads)
 prune_kernel(const uint4* __restrict__ dO, int64_t nvec, int n, uint32_t seed_lo, uint32_t seed_hi,
              uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
@@ -117,11 +117,11 @@ prune_kernel(const uint4* __restrict__ dO, int64_t nvec, int n, uint32_t seed_lo
 
     // ---- survivor values ----
     uint32_t y[8];
-    if (SCHEME == SDGP_RESCALED_MAGNITUDE) {
+    if (SCHEME == SDGP_RESCALED_MAGNITUDE && n < M) {  // n == m: nothing pruned, nothing rescaled
       float a[8], t[8], s[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        a[i] = __uint_as_float((x[i] & 0x7FFFu) << 16);
+        a[i] = lane_lo<F16>(x[i] & 0x7FFFu);
         t[i] = a[i];
         s[i] = ((keep8 >> i) & 1u) ? a[i] : 0.0f;
       }
@@ -150,8 +150,8 @@ prune_kernel(const uint4* __restrict__ dO, int64_t nvec, int n, uint32_t seed_lo
       }
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const float xf = __uint_as_float(x[i] << 16);
-        y[i] = ((keep8 >> i) & 1u) ? f32_to_bf16_bits(__fmul_rn(xf, scale[i >> 2])) : 0u;
+        const float xf = lane_lo<F16>(x[i]);
+        y[i] = ((keep8 >> i) & 1u) ? f32_to_elem_bits<F16>(__fmul_rn(xf, scale[i >> 2])) : 0u;
       }
     } else {
 #pragma unroll
@@ -229,7 +229,7 @@ __device__ __forceinline__ void emit_packed(int64_t v, uint32_t y0, uint32_t y1,
   }
 }
 
-template <int N, int SCHEME>
+template <int N, int SCHEME, bool F16>
 __global__ void __launch_bounds__(kThreads)
 prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                 uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
@@ -249,13 +249,15 @@ prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, ui
     if (v >= nvec) continue;
     const uint4 w = in[it];
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3;
-    m4_prune_vector<N, SCHEME>(w, v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
+    m4_prune_vector<N, SCHEME, F16>(w, v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
     emit_packed<(N <= 2)>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask, pitch);
   }
 }
 
+// Only the rescaled scheme reads values as numbers: the other two run the same (bf16-named)
+// instantiation for both element types.
 template <int N>
-cudaError_t launch_m4_n(int scheme, const void* dO, int64_t nvec, uint64_t seed, void* dense, void* values,
+cudaError_t launch_m4_n(int scheme, bool f16, const void* dO, int64_t nvec, uint64_t seed, void* dense, void* values,
                         void* meta, void* mask, OutPitch pitch, cudaStream_t stream) {
   const int64_t per_block = (int64_t)kThreads * kVecPerThread;
   const int64_t blocks = (nvec + per_block - 1) / per_block;
@@ -263,13 +265,16 @@ cudaError_t launch_m4_n(int scheme, const void* dO, int64_t nvec, uint64_t seed,
   if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)blocks), block(kThreads);
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
-#define SDGP_LAUNCH4(S)                                                                         \
-  launch_after_previous(prune_m4_kernel<N, S>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
+#define SDGP_LAUNCH4(S, F)                                                                      \
+  launch_after_previous(prune_m4_kernel<N, S, F>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
                                                     (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch)
   switch (scheme) {
-    case SDGP_RANDOM: SDGP_LAUNCH4(SDGP_RANDOM); break;
-    case SDGP_MAGNITUDE: SDGP_LAUNCH4(SDGP_MAGNITUDE); break;
-    default: SDGP_LAUNCH4(SDGP_RESCALED_MAGNITUDE); break;
+    case SDGP_RANDOM: SDGP_LAUNCH4(SDGP_RANDOM, false); break;
+    case SDGP_MAGNITUDE: SDGP_LAUNCH4(SDGP_MAGNITUDE, false); break;
+    default:
+      if (f16) SDGP_LAUNCH4(SDGP_RESCALED_MAGNITUDE, true);
+      else SDGP_LAUNCH4(SDGP_RESCALED_MAGNITUDE, false);
+      break;
   }
 #undef SDGP_LAUNCH4
   return cudaGetLastError();
@@ -288,7 +293,7 @@ __device__ __forceinline__ void merge_top2(uint32_t& hi, uint32_t& lo, uint32_t 
   hi = h;
 }
 
-template <int M, int N, int SCHEME>
+template <int M, int N, int SCHEME, bool F16>
 __global__ void __launch_bounds__(kThreads)
 prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                   uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
@@ -349,28 +354,22 @@ prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, 
     uint32_t y0 = p0 & km0, y1 = p1 & km1, y2 = p2 & km2, y3 = p3 & km3;
     if (SCHEME == SDGP_RESCALED_MAGNITUDE) {
       // balanced pairwise sums in index order: elements 0..3 are the low lanes, 4..7 the high lanes
-#define SDGP_SUM8(q0, q1, q2, q3)                                                                                 \
-  __fadd_rn(__fadd_rn(__fadd_rn(__uint_as_float((q0 << 16) & 0x7FFF0000u), __uint_as_float((q1 << 16) & 0x7FFF0000u)), \
-                      __fadd_rn(__uint_as_float((q2 << 16) & 0x7FFF0000u), __uint_as_float((q3 << 16) & 0x7FFF0000u))), \
-            __fadd_rn(__fadd_rn(__uint_as_float(q0 & 0x7FFF0000u), __uint_as_float(q1 & 0x7FFF0000u)),             \
-                      __fadd_rn(__uint_as_float(q2 & 0x7FFF0000u), __uint_as_float(q3 & 0x7FFF0000u))))
-      float tsum = SDGP_SUM8(p0, p1, p2, p3);
-      float ssum = SDGP_SUM8(y0, y1, y2, y3);
-#undef SDGP_SUM8
+      float tsum = __fadd_rn(sum4_lo_abs<F16>(p0, p1, p2, p3), sum4_hi_abs<F16>(p0, p1, p2, p3));
+      float ssum = __fadd_rn(sum4_lo_abs<F16>(y0, y1, y2, y3), sum4_hi_abs<F16>(y0, y1, y2, y3));
 #pragma unroll
       for (int d = 1; d < LANES; d <<= 1) {
         tsum = __fadd_rn(tsum, __shfl_xor_sync(0xFFFFFFFFu, tsum, d));
         ssum = __fadd_rn(ssum, __shfl_xor_sync(0xFFFFFFFFu, ssum, d));
       }
       const float sc = (ssum == 0.0f) ? 1.0f : __fdiv_rn(tsum, ssum);
-      rescale_packed(y0, y1, y2, y3, km0, km1, km2, km3, sc, sc, tsum, tsum);
+      rescale_packed<F16>(y0, y1, y2, y3, km0, km1, km2, km3, sc, sc, tsum, tsum);
     }
     if (v < nvec) emit_packed<true>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask, pitch);
   }
 }
 
 template <int M, int N>
-cudaError_t launch_top2(int scheme, const void* dO, int64_t nvec, uint64_t seed, void* dense, void* values,
+cudaError_t launch_top2(int scheme, bool f16, const void* dO, int64_t nvec, uint64_t seed, void* dense, void* values,
                         void* meta, void* mask, OutPitch pitch, cudaStream_t stream) {
   const int64_t per_block = (int64_t)kThreads * kVecPerThread;
   const int64_t blocks = (nvec + per_block - 1) / per_block;
@@ -378,20 +377,23 @@ cudaError_t launch_top2(int scheme, const void* dO, int64_t nvec, uint64_t seed,
   if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)blocks), block(kThreads);
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
-#define SDGP_LAUNCH_T2(S)                                                                            \
-  launch_after_previous(prune_top2_kernel<M, N, S>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
+#define SDGP_LAUNCH_T2(S, F)                                                                         \
+  launch_after_previous(prune_top2_kernel<M, N, S, F>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
                                                          (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch)
   switch (scheme) {
-    case SDGP_RANDOM: SDGP_LAUNCH_T2(SDGP_RANDOM); break;
-    case SDGP_MAGNITUDE: SDGP_LAUNCH_T2(SDGP_MAGNITUDE); break;
-    default: SDGP_LAUNCH_T2(SDGP_RESCALED_MAGNITUDE); break;
+    case SDGP_RANDOM: SDGP_LAUNCH_T2(SDGP_RANDOM, false); break;
+    case SDGP_MAGNITUDE: SDGP_LAUNCH_T2(SDGP_MAGNITUDE, false); break;
+    default:
+      if (f16) SDGP_LAUNCH_T2(SDGP_RESCALED_MAGNITUDE, true);
+      else SDGP_LAUNCH_T2(SDGP_RESCALED_MAGNITUDE, false);
+      break;
   }
 #undef SDGP_LAUNCH_T2
   return cudaGetLastError();
 }
 
 template <int M>
-cudaError_t launch_m(int scheme, const void* dO, int64_t nvec, int n, uint64_t seed, void* dense,
+cudaError_t launch_m(int scheme, bool f16, const void* dO, int64_t nvec, int n, uint64_t seed, void* dense,
                      void* values, void* meta, void* mask, cudaStream_t stream) {
   const int64_t per_block = (int64_t)kThreads * kVecPerThread;
   const int64_t blocks = (nvec + per_block - 1) / per_block;
@@ -399,13 +401,16 @@ cudaError_t launch_m(int scheme, const void* dO, int64_t nvec, int n, uint64_t s
   if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)blocks), block(kThreads);
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
-#define SDGP_LAUNCH(S)                                                                              \
-  launch_after_previous(prune_kernel<M, S>, grid, block, stream, (const uint4*)dO, nvec, n, lo, hi, (uint4*)dense, \
+#define SDGP_LAUNCH(S, F)                                                                           \
+  launch_after_previous(prune_kernel<M, S, F>, grid, block, stream, (const uint4*)dO, nvec, n, lo, hi, (uint4*)dense, \
                                                  (uint2*)values, (uint8_t*)meta, (uint8_t*)mask)
   switch (scheme) {
-    case SDGP_RANDOM: SDGP_LAUNCH(SDGP_RANDOM); break;
-    case SDGP_MAGNITUDE: SDGP_LAUNCH(SDGP_MAGNITUDE); break;
-    default: SDGP_LAUNCH(SDGP_RESCALED_MAGNITUDE); break;
+    case SDGP_RANDOM: SDGP_LAUNCH(SDGP_RANDOM, false); break;
+    case SDGP_MAGNITUDE: SDGP_LAUNCH(SDGP_MAGNITUDE, false); break;
+    default:
+      if (f16) SDGP_LAUNCH(SDGP_RESCALED_MAGNITUDE, true);
+      else SDGP_LAUNCH(SDGP_RESCALED_MAGNITUDE, false);
+      break;
   }
 #undef SDGP_LAUNCH
   return cudaGetLastError();
@@ -415,7 +420,8 @@ cudaError_t launch_m(int scheme, const void* dO, int64_t nvec, int n, uint64_t s
 
 cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, int scheme,
                          uint64_t seed, void* dense, void* values, void* meta, void* mask,
-                         cudaStream_t stream, int64_t k_pad) {
+                         cudaStream_t stream, int64_t k_pad, int dtype) {
+  const bool f16 = dtype == SDGP_FP16;
   const int64_t nvec = rows * (K / 8);
   OutPitch pitch = {(int)(K / 8), 0};
   if (k_pad != 0 && k_pad != K) {
@@ -425,16 +431,16 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
   switch (m) {
     case 4:
       switch (n) {
-        case 1: return launch_m4_n<1>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
-        case 2: return launch_m4_n<2>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
-        case 3: return launch_m4_n<3>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
-        default: return launch_m4_n<4>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
+        case 1: return launch_m4_n<1>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
+        case 2: return launch_m4_n<2>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
+        case 3: return launch_m4_n<3>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
+        default: return launch_m4_n<4>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
       }
 #define SDGP_M_CASE(M)                                                                                     \
   case M:                                                                                                  \
-    if (n == 1) return launch_top2<M, 1>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream); \
-    if (n == 2) return launch_top2<M, 2>(scheme, dO, nvec, seed, dense, values, meta, mask, pitch, stream); \
-    return launch_m<M>(scheme, dO, nvec, n, seed, dense, values, meta, mask, stream);
+    if (n == 1) return launch_top2<M, 1>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream); \
+    if (n == 2) return launch_top2<M, 2>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream); \
+    return launch_m<M>(scheme, f16, dO, nvec, n, seed, dense, values, meta, mask, stream);
     SDGP_M_CASE(8)
     SDGP_M_CASE(16)
     SDGP_M_CASE(32)

@@ -3,6 +3,7 @@
 // per-vector m = 4 pruning function (Algorithm 1, Section 3.2).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -61,28 +62,78 @@ __host__ __device__ constexpr int threshold_lut(bool na, bool nb, bool nc) {
 }
 
 
-// Survivors of both lanes times their group's scale, rounded to bf16 (nearest even). When both
-// group sums are finite every product is finite and the hardware's packed conversion applies;
+// Element type of the 16-bit tensors. Ranking and selection only read bit patterns (the pattern
+// with the sign cleared orders bf16 and IEEE binary16 alike); the type matters where the rescale
+// of Section 3.2 reads values as numbers and rounds the survivors. F16 = false: bf16, true: binary16.
+
+// fp32 -> binary16 bits, round to nearest even (hardware conversion); any NaN becomes 0x7E00.
+__device__ __forceinline__ uint32_t f32_to_f16_bits(float f) {
+  const uint32_t h = __half_as_ushort(__float2half_rn(f));
+  return ((h & 0x7FFFu) > 0x7C00u) ? 0x7E00u : h;
+}
+
+template <bool F16>
+__device__ __forceinline__ uint32_t f32_to_elem_bits(float f) {
+  return F16 ? f32_to_f16_bits(f) : f32_to_bf16_bits(f);
+}
+
+// The element in the low / high half of a lane-paired register as fp32 (exact).
+template <bool F16>
+__device__ __forceinline__ float lane_lo(uint32_t p) {
+  return F16 ? __half2float(__ushort_as_half((unsigned short)(p & 0xFFFFu))) : __uint_as_float(p << 16);
+}
+template <bool F16>
+__device__ __forceinline__ float lane_hi(uint32_t p) {
+  return F16 ? __half2float(__ushort_as_half((unsigned short)(p >> 16))) : __uint_as_float(p & 0xFFFF0000u);
+}
+// ... and their magnitudes
+template <bool F16>
+__device__ __forceinline__ float lane_lo_abs(uint32_t p) { return lane_lo<F16>(p & 0x00007FFFu); }
+template <bool F16>
+__device__ __forceinline__ float lane_hi_abs(uint32_t p) { return lane_hi<F16>(p & 0x7FFF0000u); }
+
+// Two fp32 values rounded to nearest even and packed (low, high): hardware conversion, finite inputs.
+template <bool F16>
+__device__ __forceinline__ uint32_t pack_pair_rn(float lo, float hi) {
+  if (F16) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *(const uint32_t*)&h;
+  }
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *(const uint32_t*)&h;
+}
+
+// Balanced pairwise sum, in index order, of the magnitudes in the low (high) halves of four
+// lane-paired registers: (|e0| + |e1|) + (|e2| + |e3|), every add rounded once.
+template <bool F16>
+__device__ __forceinline__ float sum4_lo_abs(uint32_t q0, uint32_t q1, uint32_t q2, uint32_t q3) {
+  return __fadd_rn(__fadd_rn(lane_lo_abs<F16>(q0), lane_lo_abs<F16>(q1)), __fadd_rn(lane_lo_abs<F16>(q2), lane_lo_abs<F16>(q3)));
+}
+template <bool F16>
+__device__ __forceinline__ float sum4_hi_abs(uint32_t q0, uint32_t q1, uint32_t q2, uint32_t q3) {
+  return __fadd_rn(__fadd_rn(lane_hi_abs<F16>(q0), lane_hi_abs<F16>(q1)), __fadd_rn(lane_hi_abs<F16>(q2), lane_hi_abs<F16>(q3)));
+}
+
+// Survivors of both lanes times their group's scale, rounded to the element type (nearest even).
+// When both group sums are finite every fp32 product is finite and the hardware's packed
+// conversion applies (a product beyond the binary16 range rounds to infinity, as IEEE says);
 // otherwise (Inf or NaN in the group) each value goes through the explicit rounding, which
-// stores any NaN as 0x7FC0.
+// stores any NaN as the one canonical quiet NaN.
+template <bool F16>
 __device__ __forceinline__ void rescale_packed(uint32_t& y0, uint32_t& y1, uint32_t& y2, uint32_t& y3, uint32_t km0,
                                                uint32_t km1, uint32_t km2, uint32_t km3, float scA, float scB,
                                                float tA, float tB) {
   const bool finite = (__float_as_uint(tA) & 0x7F800000u) != 0x7F800000u &&
                       (__float_as_uint(tB) & 0x7F800000u) != 0x7F800000u;
   if (finite) {
-#define SDGP_RESCALE_FAST(y, km)                                                                    \
-  {                                                                                                 \
-    const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(__uint_as_float(y << 16), scA),        \
-                                                   __fmul_rn(__uint_as_float(y & 0xFFFF0000u), scB)); \
-    y = (*(const uint32_t*)&h) & km;                                                                \
-  }
+#define SDGP_RESCALE_FAST(y, km) \
+  y = pack_pair_rn<F16>(__fmul_rn(lane_lo<F16>(y), scA), __fmul_rn(lane_hi<F16>(y), scB)) & km;
     SDGP_RESCALE_FAST(y0, km0) SDGP_RESCALE_FAST(y1, km1) SDGP_RESCALE_FAST(y2, km2) SDGP_RESCALE_FAST(y3, km3)
 #undef SDGP_RESCALE_FAST
   } else {
-#define SDGP_RESCALE_SLOW(y, km)                                                                    \
-  y = (f32_to_bf16_bits(__fmul_rn(__uint_as_float(y << 16), scA)) |                                 \
-       (f32_to_bf16_bits(__fmul_rn(__uint_as_float(y & 0xFFFF0000u), scB)) << 16)) & km;
+#define SDGP_RESCALE_SLOW(y, km)                                                 \
+  y = (f32_to_elem_bits<F16>(__fmul_rn(lane_lo<F16>(y), scA)) |                  \
+       (f32_to_elem_bits<F16>(__fmul_rn(lane_hi<F16>(y), scB)) << 16)) & km;
     SDGP_RESCALE_SLOW(y0, km0) SDGP_RESCALE_SLOW(y1, km1) SDGP_RESCALE_SLOW(y2, km2) SDGP_RESCALE_SLOW(y3, km3)
 #undef SDGP_RESCALE_SLOW
   }
@@ -92,7 +143,7 @@ __device__ __forceinline__ void rescale_packed(uint32_t& y0, uint32_t& y1, uint3
 // random keys). Lane-paired form: register i holds (element i, element i + 4) in its low / high
 // 16 bits. Out: y_i = pruned (and, for the rescaled scheme, rescaled) values, km_i = 0xFFFF in
 // the lanes of kept elements.
-template <int N, int SCHEME>
+template <int N, int SCHEME, bool F16 = false>
 __device__ __forceinline__ void m4_prune_vector(const uint4& w, int64_t v, uint32_t seed_lo, uint32_t seed_hi,
                                                 uint32_t& y0, uint32_t& y1, uint32_t& y2, uint32_t& y3,
                                                 uint32_t& km0, uint32_t& km1, uint32_t& km2, uint32_t& km3) {
@@ -143,17 +194,11 @@ __device__ __forceinline__ void m4_prune_vector(const uint4& w, int64_t v, uint3
   y0 = p0 & km0; y1 = p1 & km1; y2 = p2 & km2; y3 = p3 & km3;  // pruned lanes are +0.0
   if (SCHEME == SDGP_RESCALED_MAGNITUDE && N != 4) {
     // per group: scale = sum|x| / sum|kept x|, balanced pairwise sums in index order
-    const float tA = __fadd_rn(__fadd_rn(__uint_as_float((p0 << 16) & 0x7FFF0000u), __uint_as_float((p1 << 16) & 0x7FFF0000u)),
-                               __fadd_rn(__uint_as_float((p2 << 16) & 0x7FFF0000u), __uint_as_float((p3 << 16) & 0x7FFF0000u)));
-    const float tB = __fadd_rn(__fadd_rn(__uint_as_float(p0 & 0x7FFF0000u), __uint_as_float(p1 & 0x7FFF0000u)),
-                               __fadd_rn(__uint_as_float(p2 & 0x7FFF0000u), __uint_as_float(p3 & 0x7FFF0000u)));
-    const float sA = __fadd_rn(__fadd_rn(__uint_as_float((y0 << 16) & 0x7FFF0000u), __uint_as_float((y1 << 16) & 0x7FFF0000u)),
-                               __fadd_rn(__uint_as_float((y2 << 16) & 0x7FFF0000u), __uint_as_float((y3 << 16) & 0x7FFF0000u)));
-    const float sB = __fadd_rn(__fadd_rn(__uint_as_float(y0 & 0x7FFF0000u), __uint_as_float(y1 & 0x7FFF0000u)),
-                               __fadd_rn(__uint_as_float(y2 & 0x7FFF0000u), __uint_as_float(y3 & 0x7FFF0000u)));
+    const float tA = sum4_lo_abs<F16>(p0, p1, p2, p3), tB = sum4_hi_abs<F16>(p0, p1, p2, p3);
+    const float sA = sum4_lo_abs<F16>(y0, y1, y2, y3), sB = sum4_hi_abs<F16>(y0, y1, y2, y3);
     const float scA = (sA == 0.0f) ? 1.0f : __fdiv_rn(tA, sA);
     const float scB = (sB == 0.0f) ? 1.0f : __fdiv_rn(tB, sB);
-    rescale_packed(y0, y1, y2, y3, km0, km1, km2, km3, scA, scB, tA, tB);
+    rescale_packed<F16>(y0, y1, y2, y3, km0, km1, km2, km3, scA, scB, tA, tB);
   }
 
 }

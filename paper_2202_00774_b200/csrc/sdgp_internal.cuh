@@ -12,7 +12,7 @@ namespace sdgp {
 // treat the row as k_pad channels (used to bring a channel count up to a whole 128-channel block).
 cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, int scheme,
                          uint64_t seed, void* dense, void* values, void* meta, void* mask,
-                         cudaStream_t stream, int64_t k_pad = 0);
+                         cudaStream_t stream, int64_t k_pad = 0, int dtype = SDGP_BF16);
 
 // Data gradient on the tensor cores (stride 1 or 2). sparse == false: A is dense dL/dO
 // [B,P,Q,Cout]; sparse == true: A is the compressed values [B,P,Q,Cp/2] and meta [B,P,Q,Cp/16]
@@ -24,9 +24,11 @@ struct FusedPrune {
   int scheme;
   uint64_t seed;
 };
+// dtype: element type of A, Wt and dD (SDGP_BF16 or SDGP_FP16; accumulation is fp32 either way).
+// Fused pruning with the rescaled scheme exists for bf16 only.
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
                          int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
-                         const FusedPrune* fused = nullptr);
+                         const FusedPrune* fused = nullptr, int dtype = SDGP_BF16);
 
 // Launches a one-CTA kernel whose only wait can never be satisfied (50 ms limit).
 sdgp_status launch_bounded_wait_selftest(cudaStream_t stream);

@@ -31,6 +31,21 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
     return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
+def f32_to_f16_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 to IEEE binary16 (nearest, ties to even; numpy's conversion) and return the bit patterns."""
+    with np.errstate(over="ignore"):
+        return np.ascontiguousarray(x, dtype=np.float32).astype(np.float16).view(np.uint16)
+
+
+def f16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    return np.ascontiguousarray(b, dtype=np.uint16).view(np.float16).astype(np.float32)
+
+
+def bf16_bits_as_f16_bits(b: np.ndarray) -> np.ndarray:
+    """The values of a bf16 tensor re-encoded as binary16 (rounded; the same draw in the other format)."""
+    return f32_to_f16_bits(bf16_bits_to_f32(b))
+
+
 def _rng(seed: int, stream: int) -> np.random.Generator:
     return np.random.Generator(np.random.PCG64([int(seed), int(stream)]))
 

@@ -229,6 +229,11 @@ def test_rescale_identity_when_nothing_is_pruned(m):
     x = inputs.normal_bf16((16, 64), 1.0, seed=2)
     res = oracle.prune(x, m, m, oracle.RESCALED, want=("dense",))
     assert np.array_equal(res["dense"], x)  # T == S -> scale exactly 1
+    # ... also for groups that hold Inf or NaN: with nothing pruned there is nothing to rescale
+    # (Section 3.2 rescales "the remaining n elements" of a group that lost m - n), so no Inf/Inf arises
+    y = inputs.adversarial_groups_bf16(16, 64, seed=4)
+    res = oracle.prune(y, m, m, oracle.RESCALED, want=("dense",))
+    assert np.array_equal(res["dense"], y)
 
 
 # ---------------------------------------------------------- compressed form
