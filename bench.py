@@ -58,11 +58,15 @@ def layer_flops(l):
     return 2.0 * l.B * l.H * l.W * l.Cin * l.R * l.S * l.Cout
 
 
-def layer_inputs(l, workload, seed):
-    if workload == "resnet9":
-        return inputs.conv_layer_tensors(l, seed)
-    dO, W = inputs.fc_tensors(l.W, l.Cout, l.Cin, seed)
-    return dO.reshape(l.dO_shape()), W.reshape(l.W_shape())
+def layer_inputs(l, workload, seed, dtype="bf16"):
+    if workload in ("resnet9", "resnet50"):
+        dO, W = inputs.conv_layer_tensors(l, seed)
+    else:
+        dO, W = inputs.fc_tensors(l.W, l.Cout, l.Cin, seed)
+        dO, W = dO.reshape(l.dO_shape()), W.reshape(l.W_shape())
+    if dtype == "fp16":   # the same draw, re-encoded
+        dO, W = inputs.bf16_bits_as_f16_bits(dO), inputs.bf16_bits_as_f16_bits(W)
+    return dO, W
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the seven sparse dgrad launches of one
@@ -100,16 +104,17 @@ class OracleArm:
     fp64 data gradient at `p` output pixels (the pruned neighbourhood is prepared once, outside
     the timed region). p is scaled so that a step lasts about `seconds`."""
 
-    def __init__(self, layers, workload, n, m, scheme):
+    def __init__(self, layers, workload, n, m, scheme, dtype="bf16"):
         import oracle
         oracle.build()
         self.oracle = oracle
         self.n, self.m, self.scheme = n, m, scheme
+        self.dt = oracle.FP16 if dtype == "fp16" else oracle.BF16
         # a slice of the workload large enough for ~30 s of oracle time: up to 256 images / 16384 rows
         self.layers = [inputs.ConvLayer(l.name, min(l.B, 256), l.H, min(l.W, 16384) if l.B == 1 and l.H == 1 else l.W,
                                         l.Cin, l.Cout, l.R, l.S, l.stride, l.pad) for l in layers]
-        self.tensors = [layer_inputs(l, workload, 0) for l in self.layers]
-        self.pruned = [oracle.prune(dO.reshape(-1, l.Cout), n, m, scheme, 0, want=("dense",))["dense"].reshape(dO.shape)
+        self.tensors = [layer_inputs(l, workload, 0, dtype) for l in self.layers]
+        self.pruned = [oracle.prune(dO.reshape(-1, l.Cout), n, m, scheme, 0, want=("dense",), dtype=self.dt)["dense"].reshape(dO.shape)
                        for l, (dO, _) in zip(self.layers, self.tensors)]
         self.cores = oracle.omp_threads()
 
@@ -119,8 +124,9 @@ class OracleArm:
         for l, (dO, W), pruned in zip(self.layers, self.tensors, self.pruned):
             p = int(max(1, min(pixels, l.B * l.H * l.W, l.B * l.P * l.Q)))
             self.last_pixels.append(p)
-            self.oracle.prune(dO.reshape(-1, l.Cout)[:p], self.n, self.m, self.scheme, 0, want=("dense",))
-            self.oracle.dgrad_conv2d(pruned, W, l.H, l.W, l.stride, l.pad, pixel_index=np.arange(p, dtype=np.int64))
+            self.oracle.prune(dO.reshape(-1, l.Cout)[:p], self.n, self.m, self.scheme, 0, want=("dense",), dtype=self.dt)
+            self.oracle.dgrad_conv2d(pruned, W, l.H, l.W, l.stride, l.pad, pixel_index=np.arange(p, dtype=np.int64),
+                                     dtype=self.dt)
             flops += 2.0 * p * l.Cin * l.R * l.S * l.Cout
         return flops
 
@@ -137,8 +143,8 @@ class OracleArm:
         return int(max(1, probe * seconds / dt))
 
 
-def cpu_baseline(layers, workload, n, m, scheme, target_s=24.0):
-    arm = OracleArm(layers, workload, n, m, scheme)
+def cpu_baseline(layers, workload, n, m, scheme, dtype="bf16", target_s=24.0):
+    arm = OracleArm(layers, workload, n, m, scheme, dtype)
     pixels = arm.pixels_for(target_s)
     t0 = time.perf_counter()
     flops = arm.step(pixels)
@@ -153,7 +159,7 @@ def run_reference(args, layers):
     if rank != 0:
         return
     n, m = [int(v) for v in args.nm.split(":")]
-    arm = OracleArm(layers, args.workload, n, m, SCHEMES[args.scheme])
+    arm = OracleArm(layers, args.workload, n, m, SCHEMES[args.scheme], args.dtype)
     budget = min(20.0, 150.0 / max(1, args.steps + args.warmup))  # whole run stays within a few minutes
     pixels = arm.pixels_for(budget)
     for _ in range(args.warmup):
@@ -169,7 +175,7 @@ def run_reference(args, layers):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "nm": args.nm, "scheme": args.scheme, "sample": sample},
+        "config": {"workload": args.workload, "nm": args.nm, "scheme": args.scheme, "elements": args.dtype, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": arm.cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
@@ -256,11 +262,18 @@ def run_ours(args, layers):
     def dev16(a):
         return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
 
-    host_tensors = [layer_inputs(l, args.workload, seed=rank) for l in layers]
+    DT = sdgp.FP16 if args.dtype == "fp16" else sdgp.BF16
+    # patterns with more than two survivors in some 4-chunk have no 2:4 form: pruned dense copy + dense kernel
+    masked = n > 2 and n != m
+    if masked and args.mode == "fused":
+        raise SystemExit("--mode fused needs groups of four with n <= 2")
+    step_flag = sdgp.FLAG_MASKED if masked else (sdgp.FLAG_FUSED if args.mode == "fused" else sdgp.FLAG_TWO_PASS)
+    host_tensors = [layer_inputs(l, args.workload, rank, args.dtype) for l in layers]
     dO = [dev16(t[0]) for t in host_tensors]
     Wt = [dev16(t[1]) for t in host_tensors]
     dD = [torch.empty(l.dD_shape(), dtype=torch.int16, device="cuda") for l in layers]
-    ws = [torch.empty(max(16, sdgp.sdgp_workspace_size_conv2d(l.B, l.H, l.W, l.Cin, l.Cout, l.R, l.S, l.stride, l.pad)),
+    ws = [torch.empty(max(16, sdgp.sdgp_workspace_size_conv2d(l.B, l.H, l.W, l.Cin, l.Cout, l.R, l.S, l.stride, l.pad,
+                                                              step_flag)),
                       dtype=torch.uint8, device="cuda") for l in layers]
     total_flops = sum(layer_flops(l) for l in layers)
     order = list(range(len(layers)))[::-1]  # backward pass: last layer first
@@ -268,13 +281,13 @@ def run_ours(args, layers):
     def sparse_step():
         for i in order:
             l = layers[i]
-            sdgp.sdgp_dgrad_conv2d(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, seed=1234, workspace=ws[i],
-                                   flags=sdgp.FLAG_FUSED if args.mode == "fused" else sdgp.FLAG_TWO_PASS)
+            sdgp.sdgp_dgrad_conv2d_typed(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, 1234, DT, workspace=ws[i],
+                                         flags=step_flag)
 
     def dense_step():
         for i in order:
             l = layers[i]
-            sdgp.sdgp_dgrad_conv2d(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, flags=sdgp.FLAG_DENSE)
+            sdgp.sdgp_dgrad_conv2d_typed(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, 0, DT, flags=sdgp.FLAG_DENSE)
 
     def capture(fn):
         stream = torch.cuda.Stream()
@@ -323,8 +336,24 @@ def run_ours(args, layers):
 
     # ---- per-kernel timing: the same step captured with timing events between the kernels
     # (event-record graph nodes), replayed with the same data and cache state as the timed step ----
-    vals = [torch.empty(l.B * l.P * l.Q * l.Cout // 2, dtype=torch.int16, device="cuda") for l in layers]
+    vals = [torch.empty(l.B * l.P * l.Q * l.Cout // (1 if masked else 2), dtype=torch.int16, device="cuda") for l in layers]
     metas = [torch.empty(l.B * l.P * l.Q * l.Cout // 16, dtype=torch.int16, device="cuda") for l in layers]
+
+    def prune_only(i):
+        l = layers[i]
+        if masked:
+            sdgp.sdgp_prune_typed(dO[i].view(-1, l.Cout), n, m, scheme, 1234, DT, dense=vals[i])
+        else:
+            sdgp.sdgp_prune_typed(dO[i].view(-1, l.Cout), n, m, scheme, 1234, DT, values=vals[i], meta=metas[i])
+
+    def contraction_only(i):
+        l = layers[i]
+        if masked:
+            sdgp.sdgp_dgrad_conv2d_typed(vals[i].view(l.dO_shape()), Wt[i], dD[i], l.stride, l.pad, n, m, scheme, 0, DT,
+                                         flags=sdgp.FLAG_DENSE)
+        else:
+            sdgp.sdgp_spmm_conv2d_typed(vals[i].view(l.B, l.P, l.Q, l.Cout // 2), metas[i].view(l.B, l.P, l.Q, l.Cout // 16),
+                                        Wt[i], dD[i], l.stride, l.pad, DT)
     ev_s = [torch.cuda.Event(enable_timing=True, external=True) for _ in range(2 * len(layers) + 1)]
     ev_d = [torch.cuda.Event(enable_timing=True, external=True) for _ in range(len(layers) + 1)]
 
@@ -333,10 +362,9 @@ def run_ours(args, layers):
         for i in order:
             l = layers[i]
             ev_s[k].record()
-            sdgp.sdgp_prune(dO[i].view(-1, l.Cout), n, m, scheme, 1234, values=vals[i], meta=metas[i])
+            prune_only(i)
             ev_s[k + 1].record()
-            sdgp.sdgp_spmm_conv2d(vals[i].view(l.B, l.P, l.Q, l.Cout // 2), metas[i].view(l.B, l.P, l.Q, l.Cout // 16),
-                                  Wt[i], dD[i], l.stride, l.pad)
+            contraction_only(i)
             k += 2
         ev_s[k].record()
 
@@ -344,7 +372,7 @@ def run_ours(args, layers):
         for k, i in enumerate(order):
             l = layers[i]
             ev_d[k].record()
-            sdgp.sdgp_dgrad_conv2d(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, flags=sdgp.FLAG_DENSE)
+            sdgp.sdgp_dgrad_conv2d_typed(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, 0, DT, flags=sdgp.FLAG_DENSE)
         ev_d[len(order)].record()
 
     per_steps = max(3, min(args.steps, 30))
@@ -371,25 +399,24 @@ def run_ours(args, layers):
     # the graph time is the sum of the launch durations, gaps between launches included ----
     def dgrad_only_step():
         for i in order:
-            l = layers[i]
-            sdgp.sdgp_spmm_conv2d(vals[i].view(l.B, l.P, l.Q, l.Cout // 2), metas[i].view(l.B, l.P, l.Q, l.Cout // 16),
-                                  Wt[i], dD[i], l.stride, l.pad)
+            contraction_only(i)
 
     g_dg = capture(dgrad_only_step)
     ms_dgrad_only = timed(g_dg.replay, per_steps, 3) / per_steps
     status = sdgp.sdgp_last_device_error()
     if status != 0:
         raise SystemExit("device error: " + sdgp.status_string(status))
-    prune_bytes = sum(l.B * l.P * l.Q * l.Cout * 3.125 for l in layers)
+    bytes_per_element = 4.0 if masked else 3.125   # read 2 B; write a dense copy, or values + positions
+    prune_bytes = sum(l.B * l.P * l.Q * l.Cout * bytes_per_element for l in layers)
     prune_gbs = prune_bytes * per_steps / (sum(prune_ms) * 1e-3) / 1e9
     dgrad_tflops_events = total_flops * per_steps / (sum(dgrad_ms) * 1e-3) / 1e12
     dgrad_tflops = total_flops / (ms_dgrad_only * 1e-3) / 1e12
-    sparse_peak = 2.0 * pk["bf16_sustained"]
+    sparse_peak = (1.0 if masked else 2.0) * pk["bf16_sustained"]   # binary16 has the same tensor-core rate as bf16
     per_layer = [{"layer": l.name, "prune_us": 1e3 * prune_ms[i] / per_steps, "dgrad_us": 1e3 * dgrad_ms[i] / per_steps,
                   "dense_us": 1e3 * dense_ms[i] / per_steps,
                   "dgrad_dense_equiv_tflops": layer_flops(l) / (dgrad_ms[i] / per_steps * 1e-3) / 1e12,
                   "speedup_vs_dense": dense_ms[i] / (prune_ms[i] + dgrad_ms[i]),
-                  "prune_gbs": l.B * l.P * l.Q * l.Cout * 3.125 / (prune_ms[i] / per_steps * 1e-3) / 1e9}
+                  "prune_gbs": l.B * l.P * l.Q * l.Cout * bytes_per_element / (prune_ms[i] / per_steps * 1e-3) / 1e9}
                  for i, l in enumerate(layers)]
 
     # ---- end to end: dL/dO from pinned host memory, dL/dD back to the host, every step ----
@@ -416,8 +443,8 @@ def run_ours(args, layers):
         for i in order:
             l = layers[i]
             main.wait_event(ev_in[i])
-            sdgp.sdgp_dgrad_conv2d(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, seed=1234, workspace=ws[i],
-                                   flags=sdgp.FLAG_FUSED if args.mode == "fused" else sdgp.FLAG_TWO_PASS)
+            sdgp.sdgp_dgrad_conv2d_typed(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, 1234, DT, workspace=ws[i],
+                                         flags=step_flag)
             ev_done[i].record()
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_done[i])
@@ -430,28 +457,32 @@ def run_ours(args, layers):
     e2e_value = world * total_flops / (ms_e2e / e2e_steps * 1e-3) / 1e12
 
     if rank == 0:
-        base = cpu_baseline(layers, args.workload, n, m, scheme) if world == 1 and not args.no_cpu_baseline else None
+        base = (cpu_baseline(layers, args.workload, n, m, scheme, args.dtype)
+                if world == 1 and not args.no_cpu_baseline else None)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
             "config": {"workload": args.workload, "layers": len(layers), "nm": args.nm, "scheme": args.scheme,
-                       "mode": args.mode, "flops": "2*M*N*K of the implicit GEMM per layer",
+                       "mode": "masked (pruned dense copy + dense kernel)" if masked else args.mode, "flops": "2*M*N*K of the implicit GEMM per layer",
                        "l2": "inputs larger than L2 (step touches %.0f MB)" % ((prune_bytes + d2h) / 1e6),
                        "launch": "one CUDA graph per step", "replicas": world},
             "speedup_vs_dense": value / dense_value, "dense_tflops": dense_value,
             "prune_gbs": prune_gbs, "prune_frac_of_hbm": prune_gbs / pk["hbm"],
-            "roofline": {"bound": "tensor", "kernel": "sparse dgrad (dgrad_halo_kernel<1,..>, dgrad_kernel<1,..>)",
+            "roofline": {"bound": "tensor",
+                         "kernel": ("dense dgrad on the pruned copy (dgrad_halo_kernel<0,..>, dgrad_kernel<0,..>)" if masked
+                                    else "sparse dgrad (dgrad_halo_kernel<1,..>, dgrad_kernel<1,..>)"),
                          "achieved": dgrad_tflops, "peak": sparse_peak, "unit": "TFLOP/s",
                          "frac": dgrad_tflops / sparse_peak,
-                         "traffic": measured_traffic(args.workload, args.mode),
+                         "traffic": (measured_traffic(args.workload, args.mode)
+                                     if not masked and args.dtype == "bf16" and args.nm == "2:4" else None),
                          "traffic_unit": "DRAM bytes of the sparse dgrad launches of one step (ncu)",
                          "achieved_between_event_nodes": dgrad_tflops_events,
                          "note": "dense-equivalent FLOPs of the sparse dgrad launches of one step / the time of a "
                                  "graph holding exactly those launches back to back (CUDA events around %d replays); "
                                  "achieved_between_event_nodes: the same launches timed inside the full step by "
                                  "event nodes, each of which adds a few microseconds; "
-                                 "peak = 2 x %s sustained dense bf16" % (per_steps, pk["source"])},
+                                 "peak = %d x %s sustained dense bf16" % (per_steps, 1 if masked else 2, pk["source"])},
             "per_layer": per_layer,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": (1 if args.mode == "fused" else 2) * len(layers) * args.steps,
@@ -582,6 +613,8 @@ def main():
     ap.add_argument("--nm", default="2:4")
     ap.add_argument("--mode", default="two_pass", choices=["two_pass", "fused"],
                     help="two_pass: prune kernel + sparse dgrad kernel per layer; fused: one kernel prunes and contracts")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"],
+                    help="element type of dL/dO, W and dL/dD (fp32 accumulation either way)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.workload == "resnet50":
