@@ -11,6 +11,7 @@ CIFAR-10 / ImageNet training runs, Section 4):
   * ``resnet9``        3x3 stride-1 pad-1 convolution layers of a 9-layer ResNet at batch 512
   * ``resnet50``       1x1 / 3x3 bottleneck convolutions of ResNet-50 at batch 256
   * ``gemm_large``     dO [16384, 4096], W [4096, 4096]
+  * ``resnet18``       3x3 / stride-2 / shortcut convolutions of ResNet-18 (parity shapes)
 """
 from __future__ import annotations
 
@@ -163,6 +164,21 @@ def resnet50_layers(batch: int = 256):
                     blocks if s == 1 else blocks - 1))
         out.append((ConvLayer(tag + "1x1_%dto%d_at%d" % (mid, wide, hw), batch, hw, hw, mid, wide, 1, 1, 1, 0), blocks))
         prev_wide = wide
+    return out
+
+
+def resnet18_layers(batch: int = 256) -> List[ConvLayer]:
+    """Distinct convolutions of the ResNet-18 basic-block stages (Section 4 trains it on ImageNet): 3x3 at
+    64@56, 128@28, 256@14, 512@7, the stride-2 3x3 that opens stages 2-4 and their 1x1 stride-2 shortcuts."""
+    out = []
+    prev = 64
+    for stage, (hw, ch) in enumerate([(56, 64), (28, 128), (14, 256), (7, 512)], start=1):
+        tag = "r18_s%d_" % stage
+        if stage > 1:
+            out.append(ConvLayer(tag + "3x3s2_%dto%d_at%d" % (prev, ch, 2 * hw), batch, 2 * hw, 2 * hw, prev, ch, 3, 3, 2, 1))
+            out.append(ConvLayer(tag + "projs2_%dto%d_at%d" % (prev, ch, 2 * hw), batch, 2 * hw, 2 * hw, prev, ch, 1, 1, 2, 0))
+        out.append(ConvLayer(tag + "3x3_%dto%d_at%d" % (ch, ch, hw), batch, hw, hw, ch, ch, 3, 3, 1, 1))
+        prev = ch
     return out
 
 

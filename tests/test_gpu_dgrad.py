@@ -292,6 +292,26 @@ def test_resnet50_bottleneck_shapes_small_batch():
         assert rel_fro(got, want) <= TOL, layer.name
 
 
+def test_resnet18_shapes_small_batch():
+    """Every distinct convolution of the ResNet-18 stages (batch 3; stride-2 3x3 and 1x1 shortcuts included),
+    2:4 magnitude two-pass, all outputs against the oracle."""
+    import paper_2202_00774_b200 as sdgp
+    for layer in inputs.resnet18_layers(batch=3):
+        dO, W = inputs.conv_layer_tensors(layer, seed=layer.Cin + layer.H)
+        ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(layer.B, layer.H, layer.W, layer.Cin, layer.Cout, layer.R,
+                                                         layer.S, layer.stride, layer.pad), dtype=torch.uint8, device="cuda")
+        dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, layer.stride, layer.pad, 2, 4, sdgp.MAGNITUDE, workspace=ws)
+        check_no_device_error()
+        pruned = oracle.prune(dO.reshape(-1, layer.Cout), 2, 4, oracle.MAGNITUDE, 0, want=("dense",))["dense"]
+        rng = np.random.default_rng(layer.Cout)
+        idx = np.unique(np.concatenate([rng.integers(0, layer.B * layer.H * layer.W, 500), np.arange(0, 60)]))
+        want = oracle.dgrad_conv2d(pruned.reshape(dO.shape), W, layer.H, layer.W, layer.stride, layer.pad, pixel_index=idx)
+        got_all = to_f64(dD)
+        assert not np.isnan(got_all).any(), layer.name
+        assert rel_fro(got_all.reshape(-1, layer.Cin)[idx], want) <= TOL, layer.name
+
+
 # ------------------------------------------------------------------- fused
 
 
