@@ -47,9 +47,11 @@ def _load():
             lib.oracle_prune.restype = i32
             lib.oracle_prune_t.argtypes = [vp, i64, i64, i32, i32, i32, i32, u64, vp, vp, vp, vp]
             lib.oracle_prune_t.restype = i32
-            lib.oracle_dgrad_linear_t.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, i32]
+            lib.oracle_dgrad_linear_t.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, i32, vp]
             lib.oracle_dgrad_linear_t.restype = i32
-            lib.oracle_dgrad_conv2d_t.argtypes = [vp, vp, vp] + [i32] * 9 + [vp, i64, i32]
+            lib.oracle_dgrad_conv2d_t.argtypes = [vp, vp, vp] + [i32] * 9 + [vp, i64, i32, vp]
+            lib.oracle_channel_scales.argtypes = [vp, i64, i64, i32, i32, i32, vp]
+            lib.oracle_channel_scales.restype = i32
             lib.oracle_dgrad_conv2d_t.restype = i32
             lib.oracle_f32_to_f16.argtypes = [ctypes.c_float]
             lib.oracle_f32_to_f16.restype = ctypes.c_uint16
@@ -123,8 +125,29 @@ def expand(values, meta):
     return dense
 
 
-def dgrad_linear(dOp, W, row_index=None, dtype=BF16):
-    """dD = dOp @ W in fp64 from 16-bit bit patterns; ``row_index`` evaluates a subset of rows."""
+def channel_scales(dO, n, m, dtype=BF16):
+    """Per-channel reading of the L1 rescale: one fp64 factor per column of the ``[rows, K]`` tensor,
+    sum|x| / sum|kept x| over all rows under the magnitude mask (1 where nothing of the column is kept)."""
+    dO = _u16(dO)
+    rows, K = dO.shape
+    out = np.empty(K, np.float64)
+    rc = _load().oracle_channel_scales(_ptr(dO), rows, K, n, m, dtype, _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_channel_scales rejected its arguments")
+    return out
+
+
+def _scale_arg(k_scale, K):
+    if k_scale is None:
+        return None
+    a = np.ascontiguousarray(k_scale, dtype=np.float64)
+    if a.shape != (K,):
+        raise ValueError("k_scale must have one entry per output channel")
+    return a
+
+
+def dgrad_linear(dOp, W, row_index=None, dtype=BF16, k_scale=None):
+    """dD = (dOp * k_scale) @ W in fp64 from 16-bit bit patterns; ``row_index`` evaluates a subset of rows."""
     dOp, W = _u16(dOp), _u16(W)
     rows, K = dOp.shape
     K2, N = W.shape
@@ -133,13 +156,14 @@ def dgrad_linear(dOp, W, row_index=None, dtype=BF16):
     idx = None if row_index is None else np.ascontiguousarray(row_index, dtype=np.int64)
     count = rows if idx is None else idx.shape[0]
     dD = np.empty((count, N), np.float64)
-    rc = _load().oracle_dgrad_linear_t(_ptr(dOp), _ptr(W), _ptr(dD), rows, K, N, _ptr(idx), count, dtype)
+    ks = _scale_arg(k_scale, K)
+    rc = _load().oracle_dgrad_linear_t(_ptr(dOp), _ptr(W), _ptr(dD), rows, K, N, _ptr(idx), count, dtype, _ptr(ks))
     if rc != 0:
         raise ValueError("oracle_dgrad_linear rejected its arguments")
     return dD
 
 
-def dgrad_conv2d(dOp, W, H, Wd, stride=1, pad=0, pixel_index=None, dtype=BF16):
+def dgrad_conv2d(dOp, W, H, Wd, stride=1, pad=0, pixel_index=None, dtype=BF16, k_scale=None):
     """dD (NHWC, fp64) from dOp NHWC ``[B,P,Q,Cout]`` and W ``[Cout,R,S,Cin]`` (uint16)."""
     dOp, W = _u16(dOp), _u16(W)
     B, P, Q, Cout = dOp.shape
@@ -149,8 +173,9 @@ def dgrad_conv2d(dOp, W, H, Wd, stride=1, pad=0, pixel_index=None, dtype=BF16):
     idx = None if pixel_index is None else np.ascontiguousarray(pixel_index, dtype=np.int64)
     count = B * H * Wd if idx is None else idx.shape[0]
     dD = np.empty((count, Cin), np.float64)
+    ks = _scale_arg(k_scale, Cout)
     rc = _load().oracle_dgrad_conv2d_t(_ptr(dOp), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S, stride,
-                                       pad, _ptr(idx), count, dtype)
+                                       pad, _ptr(idx), count, dtype, _ptr(ks))
     if rc != 0:
         raise ValueError("oracle_dgrad_conv2d rejected its arguments")
     return dD.reshape(B, H, Wd, Cin) if idx is None else dD

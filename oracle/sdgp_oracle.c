@@ -19,7 +19,8 @@
  *   - ties between equal magnitudes go to the lower index;
  *   - magnitude order is the order of the bf16 bit pattern with the sign cleared;
  *   - the L1 rescale is per group, in fp32, with a fixed balanced summation tree; a group
- *     from which nothing is pruned (n == m) is returned unchanged;
+ *     from which nothing is pruned (n == m) is returned unchanged; the per-channel reading of
+ *     the same sentence is offered beside it (oracle_channel_scales);
  *   - "random" ranks elements by 16-bit keys drawn from Philox4x32-10
  *     (Salmon et al., SC'11) at a counter fixed by the element's linear index;
  *   - pruned positions hold +0.0.
@@ -313,6 +314,38 @@ int oracle_prune(const uint16_t* dO, int64_t rows, int64_t K, int n, int m, int 
   return oracle_prune_t(dO, rows, K, n, m, scheme, ORACLE_BF16, seed, dense, values, meta, mask);
 }
 
+/* The other reading of the L1 rescale (Section 3.3 and the caption of Fig. 4 speak of the norm
+ * being "preserved ... per channel" across batch and spatial positions, where Section 3.2 speaks
+ * of the group): the survivors are those of the magnitude function, and every channel k gets one
+ * scale for the whole tensor,
+ *   scale[k] = sum_r |x[r,k]| / sum_r |x[r,k]| * kept[r,k]      (1 where the denominator is 0),
+ * so that each channel's L1 norm over all rows is preserved. Sums in fp64, rows in ascending order.
+ * The scaled tensor is never rounded to 16 bits: the scale multiplies the survivor inside the
+ * contraction (see the k_scale argument of the data-gradient functions). */
+int oracle_channel_scales(const uint16_t* dO, int64_t rows, int64_t K, int n, int m, int dtype, double* scale) {
+  if (dtype != ORACLE_BF16 && dtype != ORACLE_FP16) return ORACLE_ERR_ARG;
+  if (!dO || !scale || rows < 0 || K < 0 || m < 1 || m > ORACLE_MAX_M || n < 1 || n > m || K % m != 0)
+    return ORACLE_ERR_ARG;
+  double* total = (double*)calloc((size_t)(K > 0 ? K : 1), sizeof(double));
+  double* kept = (double*)calloc((size_t)(K > 0 ? K : 1), sizeof(double));
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t g = 0; g < K / m; ++g) {
+      uint8_t keep[ORACLE_MAX_M];
+      uint16_t out[ORACLE_MAX_M];
+      const uint16_t* x = dO + r * K + g * m;
+      prune_group(x, n, m, ORACLE_MAGNITUDE, dtype, 0, 0, keep, out);
+      for (int j = 0; j < m; ++j) {
+        double a = fabs(elem_to_f64(x[j], dtype));
+        total[g * m + j] += a;
+        if (keep[j]) kept[g * m + j] += a;
+      }
+    }
+  for (int64_t k = 0; k < K; ++k) scale[k] = (kept[k] == 0.0) ? 1.0 : total[k] / kept[k];
+  free(total);
+  free(kept);
+  return ORACLE_OK;
+}
+
 /* Inverse of the compressed format: rebuild the dense [rows, K] tensor. */
 int oracle_expand(const uint16_t* values, const uint16_t* meta, int64_t rows, int64_t K,
                   uint16_t* dense) {
@@ -331,12 +364,15 @@ int oracle_expand(const uint16_t* values, const uint16_t* meta, int64_t rows, in
 
 /* ----------------------------------------------------------------- dgrad */
 
+/* k_scale (nullable) in the two functions below: one factor per output channel k that multiplies
+ * dOp[., k] inside the sum (the per-channel reading of the rescale, oracle_channel_scales). */
+
 /* Fully connected data gradient (Fig. 2): dD[r, c] = sum_k dOp[r, k] * W[k, c],
  * dOp [rows, K], W [K, N] (output channels x input channels), fp64 accumulation
  * in ascending k. Rows may be a subset: row_index (nullable) lists which rows
  * of dOp to evaluate; dD then has n_rows rows in that order. */
 int oracle_dgrad_linear_t(const uint16_t* dOp, const uint16_t* W, double* dD, int64_t rows, int64_t K,
-                          int64_t N, const int64_t* row_index, int64_t n_rows, int dtype) {
+                          int64_t N, const int64_t* row_index, int64_t n_rows, int dtype, const double* k_scale) {
   if (dtype != ORACLE_BF16 && dtype != ORACLE_FP16) return ORACLE_ERR_ARG;
   if (!dOp || !W || !dD || rows < 0 || K < 0 || N < 0) return ORACLE_ERR_ARG;
   int64_t count = row_index ? n_rows : rows;
@@ -346,7 +382,7 @@ int oracle_dgrad_linear_t(const uint16_t* dOp, const uint16_t* W, double* dD, in
     for (int64_t c = 0; c < N; ++c) {
       double acc = 0.0;
       for (int64_t k = 0; k < K; ++k)
-        acc += elem_to_f64(dOp[r * K + k], dtype) * elem_to_f64(W[k * N + c], dtype);
+        acc += elem_to_f64(dOp[r * K + k], dtype) * (k_scale ? k_scale[k] : 1.0) * elem_to_f64(W[k * N + c], dtype);
       dD[i * N + c] = acc;
     }
   }
@@ -355,7 +391,7 @@ int oracle_dgrad_linear_t(const uint16_t* dOp, const uint16_t* W, double* dD, in
 
 int oracle_dgrad_linear(const uint16_t* dOp, const uint16_t* W, double* dD, int64_t rows, int64_t K,
                         int64_t N, const int64_t* row_index, int64_t n_rows) {
-  return oracle_dgrad_linear_t(dOp, W, dD, rows, K, N, row_index, n_rows, ORACLE_BF16);
+  return oracle_dgrad_linear_t(dOp, W, dD, rows, K, N, row_index, n_rows, ORACLE_BF16, NULL);
 }
 
 /* Convolution data gradient (Fig. 3). Forward layer: cross-correlation
@@ -367,7 +403,7 @@ int oracle_dgrad_linear(const uint16_t* dOp, const uint16_t* W, double* dD, int6
  * pixel_index (nullable) lists flattened (b*H + h)*Wd + w positions to evaluate. */
 int oracle_dgrad_conv2d_t(const uint16_t* dOp, const uint16_t* W, double* dD, int B, int H, int Wd,
                           int Cin, int Cout, int R, int S, int stride, int pad,
-                          const int64_t* pixel_index, int64_t n_pixels, int dtype) {
+                          const int64_t* pixel_index, int64_t n_pixels, int dtype, const double* k_scale) {
   if (dtype != ORACLE_BF16 && dtype != ORACLE_FP16) return ORACLE_ERR_ARG;
   if (!dOp || !W || !dD || stride < 1 || pad < 0 || R < 1 || S < 1) return ORACLE_ERR_ARG;
   int P = (H + 2 * pad - R) / stride + 1;
@@ -394,7 +430,7 @@ int oracle_dgrad_conv2d_t(const uint16_t* dOp, const uint16_t* W, double* dD, in
           if (q >= Q) continue;
           const uint16_t* g = dOp + (((int64_t)b * P + p) * Q + q) * Cout;
           for (int co = 0; co < Cout; ++co)
-            acc += elem_to_f64(g[co], dtype) *
+            acc += elem_to_f64(g[co], dtype) * (k_scale ? k_scale[co] : 1.0) *
                    elem_to_f64(W[(((int64_t)co * R + r) * S + s) * Cin + ci], dtype);
         }
       }
@@ -407,7 +443,8 @@ int oracle_dgrad_conv2d_t(const uint16_t* dOp, const uint16_t* W, double* dD, in
 int oracle_dgrad_conv2d(const uint16_t* dOp, const uint16_t* W, double* dD, int B, int H, int Wd,
                         int Cin, int Cout, int R, int S, int stride, int pad,
                         const int64_t* pixel_index, int64_t n_pixels) {
-  return oracle_dgrad_conv2d_t(dOp, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, pixel_index, n_pixels, ORACLE_BF16);
+  return oracle_dgrad_conv2d_t(dOp, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, pixel_index, n_pixels, ORACLE_BF16,
+                               NULL);
 }
 
 /* Direct forward convolution in fp64 on fp64 inputs; used only by the adjoint
