@@ -78,11 +78,17 @@ enum {
   SDGP_FLAG_FUSED = 1,    /* pruning happens inside the dgrad kernel (needs m == 4, n <= 2); no workspace, no
                              compressed tensor in global memory */
   SDGP_FLAG_DENSE = 2,    /* no pruning: dense tensor-core data gradient of dL/dO itself (n, m, scheme ignored) */
-  SDGP_FLAG_MASKED = 3    /* prune kernel writes the pruned tensor as a dense copy (pruned positions +0.0, the tensor
+  SDGP_FLAG_MASKED = 3,   /* prune kernel writes the pruned tensor as a dense copy (pruned positions +0.0, the tensor
                              Algorithm 1 returns) into the workspace and the dense tensor-core kernel contracts it:
                              for every 1 <= n <= m, m in {4, 8, 16, 32}, in particular the patterns of Section 4.2
                              that leave more than two survivors in some aligned 4-chunk (3:4, 4:8, 4:16, 8:16,
                              16:32, ...), which a 2:4 sparse tensor core cannot take; no speed-up over dense */
+  SDGP_FLAG_CHANNEL = 4   /* two-pass under the OTHER reading of the L1 rescale (Section 3.3, caption of Fig. 4: the
+                             norm is preserved "per channel" over batch and spatial positions): survivors of the
+                             magnitude function, one factor per output channel k for the whole tensor,
+                             sum_rows |dO[.,k]| / sum_rows |kept dO[.,k]| (1 if nothing of the channel is kept), applied
+                             inside the contraction by scaling row k of W (a scaled copy of W in the workspace).
+                             `scheme` must be SDGP_RESCALED_MAGNITUDE, n <= 2. Costs one more read of dL/dO. */
 };
 
 /* Algorithm 1 with pruning function `scheme` on dO viewed as [rows, K], groups of m along K.
@@ -160,6 +166,14 @@ sdgp_status sdgp_spmm_conv2d_typed(const void* values, const void* meta, const v
                                    int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
                                    sdgp_dtype dtype, void* stream);
 
+/* The factors of SDGP_FLAG_CHANNEL on their own: dO [rows, K] of element type `dtype`, groups of m along K,
+ * magnitude function with n survivors (any 1 <= n <= m, m in {4, 8, 16, 32}, K % m == 0, K % 8 == 0).
+ * `out` is a device array of 3 * K floats: [0, K) the factors, [K, 2K) the column sums of |dO| over all rows,
+ * [2K, 3K) the same sums over the survivors. fp32 sums (partial sums per thread, combined with atomic adds:
+ * the last bits depend on the order). */
+sdgp_status sdgp_channel_scales(const void* dO, int64_t rows, int64_t K, int n, int m, sdgp_dtype dtype, float* out,
+                                void* stream);
+
 /* No counterpart in the paper: a convenience variant of sdgp_dgrad_linear (two-pass mode) that
  * takes no workspace and allocates nothing - for callers that cannot call cudaMalloc where
  * the gradient is computed (inside another runtime's no-allocation region, in a plugin whose
@@ -178,7 +192,8 @@ sdgp_status sdgp_dgrad_linear_static(const void* dO, const void* W, void* dD, in
                                      void* stream);
 
 /* Bytes of workspace the matching dgrad call needs for these shapes and flags (0 for
- * SDGP_FLAG_DENSE and SDGP_FLAG_FUSED; the size of dL/dO for SDGP_FLAG_MASKED). */
+ * SDGP_FLAG_DENSE and SDGP_FLAG_FUSED; the size of dL/dO for SDGP_FLAG_MASKED; the compressed tensor,
+ * 3 * K floats and a copy of W for SDGP_FLAG_CHANNEL). */
 size_t sdgp_workspace_size_linear(int64_t rows, int64_t K, int64_t N, uint32_t flags);
 size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R, int S, int stride,
                                   int pad, uint32_t flags);

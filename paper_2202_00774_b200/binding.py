@@ -14,12 +14,12 @@ import torch
 from . import build as _build
 
 RANDOM, MAGNITUDE, RESCALED_MAGNITUDE = 0, 1, 2
-FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE, FLAG_MASKED = 0, 1, 2, 3
+FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE, FLAG_MASKED, FLAG_CHANNEL = 0, 1, 2, 3, 4
 
 BF16, FP16 = 0, 1   # sdgp_dtype
 EXPORTS = ["sdgp_prune", "sdgp_dgrad_linear", "sdgp_dgrad_conv2d", "sdgp_spmm_linear", "sdgp_spmm_conv2d",
            "sdgp_prune_typed", "sdgp_dgrad_linear_typed", "sdgp_dgrad_conv2d_typed", "sdgp_spmm_linear_typed",
-           "sdgp_spmm_conv2d_typed", "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
+           "sdgp_spmm_conv2d_typed", "sdgp_channel_scales", "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
            "sdgp_workspace_size_linear", "sdgp_workspace_size_conv2d", "sdgp_last_device_error",
            "sdgp_status_string"]
 
@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.sdgp_spmm_linear_typed.restype = i32
         L.sdgp_spmm_conv2d_typed.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [i32, vp]
         L.sdgp_spmm_conv2d_typed.restype = i32
+        L.sdgp_channel_scales.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp]
+        L.sdgp_channel_scales.restype = i32
         L.sdgp_workspace_size_linear.argtypes = [i64, i64, i64, u32]
         L.sdgp_workspace_size_linear.restype = sz
         L.sdgp_workspace_size_conv2d.argtypes = [i32] * 9 + [u32]
@@ -224,6 +226,17 @@ def sdgp_spmm_conv2d_typed(values, meta, W, dD, stride, pad, dtype):
     Cout, R, S, _ = W.shape
     _check(lib().sdgp_spmm_conv2d_typed(_ptr(values), _ptr(meta), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S,
                                         stride, pad, dtype, _stream()), "sdgp_spmm_conv2d_typed")
+
+
+def sdgp_channel_scales(dO, n, m, dtype, out):
+    """``sdgp_channel_scales``: ``out`` is a float32 CUDA tensor of 3*K elements (factors, sums of |dO|, sums over survivors)."""
+    _dev(dO, "dO")
+    _dev(out, "out")
+    K = dO.shape[-1]
+    rows = dO.numel() // K if K else 0
+    if out.numel() < 3 * K or out.element_size() != 4:
+        raise ValueError("out must hold 3*K float32 values")
+    _check(lib().sdgp_channel_scales(_ptr(dO), rows, K, n, m, dtype, _ptr(out), _stream()), "sdgp_channel_scales")
 
 
 def sdgp_selftest_bounded_wait():

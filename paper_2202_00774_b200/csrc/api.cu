@@ -79,22 +79,27 @@ sdgp_status sdgp_prune_typed(const void* dO, int64_t rows, int64_t K, int n, int
   return e == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
+// SDGP_FLAG_CHANNEL: behind the compressed tensor, 3 * K floats (factors, two column sums) and the scaled copy of W
+static size_t channel_floats_bytes(int64_t K) { return round_up((size_t)K * 3 * sizeof(float), 256); }
+static size_t channel_extra_bytes(int64_t K, int64_t w_row_elems) {
+  return channel_floats_bytes(K) + round_up((size_t)K * (size_t)w_row_elems * 2, 256);
+}
+
 size_t sdgp_workspace_size_linear(int64_t rows, int64_t K, int64_t N, uint32_t flags) {
-  (void)N;
   if (rows <= 0 || K <= 0) return 0;
   if (flags == SDGP_FLAG_MASKED) return round_up((size_t)rows * (size_t)K * 2, 256);
-  if (flags != SDGP_FLAG_TWO_PASS) return 0;
-  return carve_compressed(nullptr, rows * pad128(K)).bytes;
+  if (flags != SDGP_FLAG_TWO_PASS && flags != SDGP_FLAG_CHANNEL) return 0;
+  return carve_compressed(nullptr, rows * pad128(K)).bytes + (flags == SDGP_FLAG_CHANNEL ? channel_extra_bytes(K, N) : 0);
 }
 
 size_t sdgp_workspace_size_conv2d(int B, int H, int Wd, int Cin, int Cout, int R, int S, int stride,
                                   int pad, uint32_t flags) {
-  (void)Cin;
-  if ((flags != SDGP_FLAG_TWO_PASS && flags != SDGP_FLAG_MASKED) || stride < 1) return 0;
+  if ((flags != SDGP_FLAG_TWO_PASS && flags != SDGP_FLAG_MASKED && flags != SDGP_FLAG_CHANNEL) || stride < 1) return 0;
   const int64_t P = (H + 2 * pad - R) / stride + 1, Q = (Wd + 2 * pad - S) / stride + 1;
   if (B <= 0 || P <= 0 || Q <= 0 || Cout <= 0) return 0;
   if (flags == SDGP_FLAG_MASKED) return round_up((size_t)B * P * Q * Cout * 2, 256);
-  return carve_compressed(nullptr, (int64_t)B * P * Q * pad128(Cout)).bytes;
+  return carve_compressed(nullptr, (int64_t)B * P * Q * pad128(Cout)).bytes +
+         (flags == SDGP_FLAG_CHANNEL ? channel_extra_bytes(Cout, (int64_t)R * S * Cin) : 0);
 }
 
 sdgp_status sdgp_spmm_conv2d(const void* values, const void* meta, const void* W, void* dD, int B,
@@ -146,7 +151,7 @@ sdgp_status sdgp_dgrad_conv2d_typed(const void* dO, const void* W, void* dD, int
   if (!valid_dtype(dtype)) return SDGP_ERR_INVALID_ARG;
   if (B < 0 || H < 0 || Wd < 0 || Cin < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0)
     return SDGP_ERR_INVALID_ARG;
-  if (flags > SDGP_FLAG_MASKED) return SDGP_ERR_INVALID_ARG;
+  if (flags > SDGP_FLAG_CHANNEL) return SDGP_ERR_INVALID_ARG;
   if (stride > 2) return SDGP_ERR_UNSUPPORTED;
   if (pad > R - 1 || pad > S - 1) return SDGP_ERR_UNSUPPORTED;
   if (flags != SDGP_FLAG_DENSE) {
@@ -182,6 +187,21 @@ sdgp_status sdgp_dgrad_conv2d_typed(const void* dO, const void* W, void* dD, int
   }
   const int64_t Cpad = pad128(Cout);
   const Carve c = carve_compressed(workspace, (int64_t)B * P * Q * Cpad);
+  if (flags == SDGP_FLAG_CHANNEL) {
+    // per-channel reading of the rescale: magnitude survivors, factors folded into a scaled copy of W
+    if (scheme != SDGP_RESCALED_MAGNITUDE) return SDGP_ERR_INVALID_ARG;
+    const int64_t w_row = (int64_t)R * S * Cin, rows = (int64_t)B * P * Q;
+    if (!workspace || workspace_bytes < c.bytes + channel_extra_bytes(Cout, w_row)) return SDGP_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255u) != 0) return SDGP_ERR_ALIGNMENT;
+    float* floats = (float*)((uint8_t*)workspace + c.bytes);       // [0,K) factors, [K,3K) the two sums
+    void* w_scaled = (uint8_t*)floats + channel_floats_bytes(Cout);
+    if (sdgp::launch_channel_sums(dO, rows, Cout, n, m, dt, floats + Cout, s) != cudaSuccess) return SDGP_ERR_CUDA;
+    if (sdgp::launch_scale_weights(W, floats + Cout, Cout, w_row, dt, w_scaled, floats, s) != cudaSuccess) return SDGP_ERR_CUDA;
+    if (sdgp::launch_prune(dO, rows, Cout, n, m, SDGP_MAGNITUDE, seed, nullptr, c.values, c.meta, nullptr, s, Cpad, dt) !=
+        cudaSuccess)
+      return SDGP_ERR_CUDA;
+    return sdgp::launch_dgrad(true, c.values, c.meta, w_scaled, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, nullptr, dt);
+  }
   if (!workspace || workspace_bytes < c.bytes) return SDGP_ERR_WORKSPACE;
   if (((uintptr_t)workspace & 255u) != 0) return SDGP_ERR_ALIGNMENT;
   cudaError_t e = sdgp::launch_prune(dO, (int64_t)B * P * Q, Cout, n, m, (int)scheme, seed, nullptr, c.values,
@@ -205,6 +225,19 @@ sdgp_status sdgp_dgrad_linear_typed(const void* dO, const void* W, void* dD, int
   if (rows > 0x7FFFFFFF || K > 0x7FFFFFFF || N > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
   return sdgp_dgrad_conv2d_typed(dO, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 1, 0, n, m, scheme, seed, dtype,
                                  workspace, workspace_bytes, flags, stream);
+}
+
+sdgp_status sdgp_channel_scales(const void* dO, int64_t rows, int64_t K, int n, int m, sdgp_dtype dtype, float* out,
+                                void* stream) {
+  if (!valid_dtype(dtype)) return SDGP_ERR_INVALID_ARG;
+  sdgp_status st = check_prune_args(rows, K, n, m, SDGP_MAGNITUDE);
+  if (st != SDGP_OK) return st;
+  if (K == 0) return SDGP_OK;
+  if (!out || (rows > 0 && !dO)) return SDGP_ERR_INVALID_ARG;
+  if (K % 8 != 0 || !aligned16(dO) || ((uintptr_t)out & 3u) != 0) return SDGP_ERR_ALIGNMENT;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (sdgp::launch_channel_sums(dO, rows, K, n, m, (int)dtype, out + K, s) != cudaSuccess) return SDGP_ERR_CUDA;
+  return sdgp::launch_channel_scales(out + K, K, out, s) == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
 sdgp_status sdgp_last_device_error(void) { return sdgp::read_device_error(); }

@@ -1,0 +1,152 @@
+// The per-channel reading of the L1 rescale (Section 3.3 and the caption of Fig. 4: the norm is
+// preserved "per channel" over batch and spatial positions; Section 3.2 words it per group).
+// Survivors are those of the magnitude function; channel k of the whole [rows, K] tensor gets one
+// factor scale[k] = sum_r |x[r,k]| / sum_r |kept x[r,k]| (1 when nothing of the channel is kept).
+// Because the factor is the same for every row, it is folded into row k of W
+// (dD = (A diag(s)) W = A (diag(s) W)): the pruned tensor itself is never rescaled, and the sparse
+// contraction runs unchanged on the scaled copy of W.
+//
+// Cost: one more read of dL/dO (column sums cannot be known before the whole tensor has been seen)
+// and one pass over W.
+#include "prune_core.cuh"
+#include "sdgp_internal.cuh"
+
+namespace sdgp {
+namespace {
+
+constexpr int kChThreads = 256;
+
+// sums[0..K) += sum over rows of |x|, sums[K..2K) += the same over kept elements only. A thread owns
+// one chunk of whole groups (8 elements, or m when m > 8) of a set of rows and keeps the chunk's
+// sixteen-or-more partial sums in registers; the mask is the prune kernels' (larger magnitude wins,
+// equal magnitudes: lower position), found by counting.
+template <int M, bool F16>
+__global__ void __launch_bounds__(kChThreads)
+channel_sums_kernel(const uint4* __restrict__ dO, int64_t rows, int K, int n, float* __restrict__ sums) {
+  constexpr int CH = M < 8 ? 8 : M;
+  constexpr int VEC = CH / 8;
+  const int cpr = K / CH;                                  // chunks per row
+  const int ct = cpr < kChThreads ? cpr : kChThreads;      // chunk columns handled side by side
+  const int lanes = kChThreads / ct;                       // rows handled side by side
+  const int cc0 = threadIdx.x % ct, lane = threadIdx.x / ct;
+  if (lane >= lanes) return;
+  for (int cbase = 0; cbase < cpr; cbase += ct) {
+    const int cc = cbase + cc0;
+    if (cc >= cpr) continue;
+    float t[CH], s[CH];
+#pragma unroll
+    for (int i = 0; i < CH; ++i) t[i] = s[i] = 0.0f;
+    for (int64_t r = (int64_t)blockIdx.x * lanes + lane; r < rows; r += (int64_t)gridDim.x * lanes) {
+      const uint4* src = dO + (r * K + (int64_t)cc * CH) / 8;
+      uint32_t x[CH];
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) {
+        const uint4 w = __ldg(src + v);
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[8 * v + i] = (i & 1) ? (ww[i >> 1] >> 16) : (ww[i >> 1] & 0xFFFFu);
+      }
+      uint32_t c[CH];
+#pragma unroll
+      for (int i = 0; i < CH; ++i) c[i] = ((x[i] & 0x7FFFu) << 5) | (uint32_t)(31 - (i % M));
+#pragma unroll
+      for (int i = 0; i < CH; ++i) {
+        int above = 0;
+#pragma unroll
+        for (int o = 0; o < CH; ++o)
+          if (o != i && (o / M) == (i / M)) above += (c[o] > c[i]) ? 1 : 0;
+        const float a = lane_lo<F16>(x[i] & 0x7FFFu);
+        t[i] += a;
+        if (above < n) s[i] += a;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      atomicAdd(sums + (int64_t)cc * CH + i, t[i]);
+      atomicAdd(sums + K + (int64_t)cc * CH + i, s[i]);
+    }
+  }
+}
+
+__device__ __forceinline__ float channel_scale(const float* sums, int K, int k) {
+  const float t = sums[k], s = sums[K + k];
+  return s == 0.0f ? 1.0f : __fdiv_rn(t, s);
+}
+
+__global__ void channel_scales_kernel(const float* __restrict__ sums, int K, float* __restrict__ scales) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < K) scales[k] = channel_scale(sums, K, k);
+}
+
+// Wout[k, :] = round(W[k, :] * scale[k]); one thread per 8 elements, row length a multiple of 8.
+template <bool F16>
+__global__ void scale_weights_kernel(const uint4* __restrict__ W, const float* __restrict__ sums, int K, int64_t row_vecs,
+                                     uint4* __restrict__ Wout, float* __restrict__ scales) {
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v >= (int64_t)K * row_vecs) return;
+  const int k = (int)(v / row_vecs);
+  const float sc = channel_scale(sums, K, k);
+  if (v == (int64_t)k * row_vecs) scales[k] = sc;
+  const uint4 w = __ldg(W + v);
+  uint4 o;
+  o.x = pack_pair_rn<F16>(__fmul_rn(lane_lo<F16>(w.x), sc), __fmul_rn(lane_hi<F16>(w.x), sc));
+  o.y = pack_pair_rn<F16>(__fmul_rn(lane_lo<F16>(w.y), sc), __fmul_rn(lane_hi<F16>(w.y), sc));
+  o.z = pack_pair_rn<F16>(__fmul_rn(lane_lo<F16>(w.z), sc), __fmul_rn(lane_hi<F16>(w.z), sc));
+  o.w = pack_pair_rn<F16>(__fmul_rn(lane_lo<F16>(w.w), sc), __fmul_rn(lane_hi<F16>(w.w), sc));
+  Wout[v] = o;
+}
+
+template <int M>
+cudaError_t launch_sums_m(bool f16, const void* dO, int64_t rows, int K, int n, float* sums, cudaStream_t stream) {
+  constexpr int CH = M < 8 ? 8 : M;
+  const int cpr = K / CH;
+  const int ct = cpr < kChThreads ? cpr : kChThreads;
+  const int lanes = kChThreads / ct;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return cudaErrorUnknown;
+  int64_t blocks = (rows + lanes - 1) / lanes;
+  if (blocks > 4 * (int64_t)sms) blocks = 4 * (int64_t)sms;
+  if (blocks < 1) return cudaSuccess;
+  if (f16) channel_sums_kernel<M, true><<<(unsigned)blocks, kChThreads, 0, stream>>>((const uint4*)dO, rows, K, n, sums);
+  else channel_sums_kernel<M, false><<<(unsigned)blocks, kChThreads, 0, stream>>>((const uint4*)dO, rows, K, n, sums);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_channel_sums(const void* dO, int64_t rows, int64_t K, int n, int m, int dtype, float* sums,
+                                cudaStream_t stream) {
+  if (K > 0x7FFFFFFF || K % 8 != 0 || K % m != 0) return cudaErrorInvalidValue;
+  if (cudaMemsetAsync(sums, 0, (size_t)K * 2 * sizeof(float), stream) != cudaSuccess) return cudaErrorUnknown;
+  const bool f16 = dtype == SDGP_FP16;
+  switch (m) {
+    case 4: return launch_sums_m<4>(f16, dO, rows, (int)K, n, sums, stream);
+    case 8: return launch_sums_m<8>(f16, dO, rows, (int)K, n, sums, stream);
+    case 16: return launch_sums_m<16>(f16, dO, rows, (int)K, n, sums, stream);
+    case 32: return launch_sums_m<32>(f16, dO, rows, (int)K, n, sums, stream);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+cudaError_t launch_channel_scales(const float* sums, int64_t K, float* scales, cudaStream_t stream) {
+  if (K < 1) return cudaSuccess;
+  channel_scales_kernel<<<(unsigned)((K + 255) / 256), 256, 0, stream>>>(sums, (int)K, scales);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scale_weights(const void* W, const float* sums, int64_t K, int64_t row_elems, int dtype, void* Wout,
+                                 float* scales, cudaStream_t stream) {
+  if (row_elems % 8 != 0 || K < 1) return cudaErrorInvalidValue;
+  const int64_t row_vecs = row_elems / 8, total = K * row_vecs;
+  const int64_t blocks = (total + 255) / 256;
+  if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
+  if (dtype == SDGP_FP16)
+    scale_weights_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>((const uint4*)W, sums, (int)K, row_vecs, (uint4*)Wout, scales);
+  else
+    scale_weights_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>((const uint4*)W, sums, (int)K, row_vecs, (uint4*)Wout, scales);
+  return cudaGetLastError();
+}
+
+}  // namespace sdgp

@@ -14,6 +14,17 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
                          uint64_t seed, void* dense, void* values, void* meta, void* mask,
                          cudaStream_t stream, int64_t k_pad = 0, int dtype = SDGP_BF16);
 
+// Per-channel reading of the L1 rescale (channel.cu). sums: 2 * K floats (cleared by the call): the
+// column sums of |x| over all rows, then the same over the survivors of the magnitude function.
+cudaError_t launch_channel_sums(const void* dO, int64_t rows, int64_t K, int n, int m, int dtype, float* sums,
+                                cudaStream_t stream);
+// scales[k] = sums[k] / sums[K + k] (1 where the denominator is 0)
+cudaError_t launch_channel_scales(const float* sums, int64_t K, float* scales, cudaStream_t stream);
+// Wout[k, :] = W[k, :] * scale[k] rounded to the element type (row_elems elements per row, a multiple of 8); also
+// writes the K scales.
+cudaError_t launch_scale_weights(const void* W, const float* sums, int64_t K, int64_t row_elems, int dtype, void* Wout,
+                                 float* scales, cudaStream_t stream);
+
 // Data gradient on the tensor cores (stride 1 or 2). sparse == false: A is dense dL/dO
 // [B,P,Q,Cout]; sparse == true: A is the compressed values [B,P,Q,Cp/2] and meta [B,P,Q,Cp/16]
 // with Cp = Cout rounded up to a multiple of 128 (see launch_prune's k_pad).

@@ -82,4 +82,13 @@ def test_dgrad_rejects_bad_arguments_before_launch(lib):
     assert L(FAKE, FAKE, FAKE, 128, 256, 128, 3, 4, 1, 0, None, 0, 3, None) == 4        # 3:4 masked: needs the workspace
     assert L(FAKE, FAKE, FAKE, 128, 256, 128, 3, 4, 1, 0, ws, 128 * 256 * 2 - 1, 3, None) == 4
     assert L(FAKE, FAKE, FAKE, 128, 256, 128, 5, 4, 1, 0, ws, 1 << 20, 3, None) == 1    # n > m
-    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 2, 4, 1, 0, ws, need, 4, None) == 1       # flags past the last mode
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 2, 4, 1, 0, ws, need, 5, None) == 1       # flags past the last mode
+    # per-channel reading: compressed tensor + 3*K floats + a copy of W; scheme must be the rescaled one
+    need_ch = need + 256 * 3 * 4 + 256 * 128 * 2
+    assert lib.sdgp_workspace_size_linear(128, 256, 128, 4) == need_ch
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 2, 4, 2, 0, ws, need_ch - 1, 4, None) == 4
+    assert L(FAKE, FAKE, FAKE, 128, 256, 128, 2, 4, 1, 0, ws, need_ch, 4, None) == 1     # magnitude scheme with the channel mode
+    S = lib.sdgp_channel_scales
+    assert S(FAKE, 4, 64, 2, 4, 7, FAKE, None) == 1      # unknown element type
+    assert S(FAKE, 4, 66, 2, 4, 0, FAKE, None) == 1      # K % m != 0
+    assert S(FAKE, 4, 64, 2, 4, 0, None, None) == 1      # no output
