@@ -104,10 +104,13 @@ class OracleArm:
     fp64 data gradient at `p` output pixels (the pruned neighbourhood is prepared once, outside
     the timed region). p is scaled so that a step lasts about `seconds`."""
 
-    def __init__(self, layers, workload, n, m, scheme, dtype="bf16"):
+    def __init__(self, layers, workload, n, m, scheme, dtype="bf16", channel=False):
         import oracle
         oracle.build()
         self.oracle = oracle
+        self.channel = channel   # per-channel reading: magnitude survivors, one factor per channel inside the contraction
+        if channel:
+            scheme = oracle.MAGNITUDE
         self.n, self.m, self.scheme = n, m, scheme
         self.dt = oracle.FP16 if dtype == "fp16" else oracle.BF16
         # a slice of the workload large enough for ~30 s of oracle time: up to 256 images / 16384 rows
@@ -125,8 +128,9 @@ class OracleArm:
             p = int(max(1, min(pixels, l.B * l.H * l.W, l.B * l.P * l.Q)))
             self.last_pixels.append(p)
             self.oracle.prune(dO.reshape(-1, l.Cout)[:p], self.n, self.m, self.scheme, 0, want=("dense",), dtype=self.dt)
+            ks = self.oracle.channel_scales(dO.reshape(-1, l.Cout)[:p], self.n, self.m, dtype=self.dt) if self.channel else None
             self.oracle.dgrad_conv2d(pruned, W, l.H, l.W, l.stride, l.pad, pixel_index=np.arange(p, dtype=np.int64),
-                                     dtype=self.dt)
+                                     dtype=self.dt, k_scale=ks)
             flops += 2.0 * p * l.Cin * l.R * l.S * l.Cout
         return flops
 
@@ -143,8 +147,8 @@ class OracleArm:
         return int(max(1, probe * seconds / dt))
 
 
-def cpu_baseline(layers, workload, n, m, scheme, dtype="bf16", target_s=24.0):
-    arm = OracleArm(layers, workload, n, m, scheme, dtype)
+def cpu_baseline(layers, workload, n, m, scheme, dtype="bf16", channel=False, target_s=24.0):
+    arm = OracleArm(layers, workload, n, m, scheme, dtype, channel)
     pixels = arm.pixels_for(target_s)
     t0 = time.perf_counter()
     flops = arm.step(pixels)
@@ -159,7 +163,7 @@ def run_reference(args, layers):
     if rank != 0:
         return
     n, m = [int(v) for v in args.nm.split(":")]
-    arm = OracleArm(layers, args.workload, n, m, SCHEMES[args.scheme], args.dtype)
+    arm = OracleArm(layers, args.workload, n, m, SCHEMES[args.scheme], args.dtype, args.mode == "channel")
     budget = min(20.0, 150.0 / max(1, args.steps + args.warmup))  # whole run stays within a few minutes
     pixels = arm.pixels_for(budget)
     for _ in range(args.warmup):
@@ -265,9 +269,10 @@ def run_ours(args, layers):
     DT = sdgp.FP16 if args.dtype == "fp16" else sdgp.BF16
     # patterns with more than two survivors in some 4-chunk have no 2:4 form: pruned dense copy + dense kernel
     masked = n > 2 and n != m
-    if masked and args.mode == "fused":
-        raise SystemExit("--mode fused needs groups of four with n <= 2")
-    step_flag = sdgp.FLAG_MASKED if masked else (sdgp.FLAG_FUSED if args.mode == "fused" else sdgp.FLAG_TWO_PASS)
+    if masked and args.mode != "two_pass":
+        raise SystemExit("--mode %s needs n <= 2" % args.mode)
+    step_flag = sdgp.FLAG_MASKED if masked else {"fused": sdgp.FLAG_FUSED, "channel": sdgp.FLAG_CHANNEL,
+                                                 "two_pass": sdgp.FLAG_TWO_PASS}[args.mode]
     host_tensors = [layer_inputs(l, args.workload, rank, args.dtype) for l in layers]
     dO = [dev16(t[0]) for t in host_tensors]
     Wt = [dev16(t[1]) for t in host_tensors]
@@ -339,8 +344,11 @@ def run_ours(args, layers):
     vals = [torch.empty(l.B * l.P * l.Q * l.Cout // (1 if masked else 2), dtype=torch.int16, device="cuda") for l in layers]
     metas = [torch.empty(l.B * l.P * l.Q * l.Cout // 16, dtype=torch.int16, device="cuda") for l in layers]
 
+    kernel_scheme = SCHEMES["magnitude"] if args.mode == "channel" else scheme   # channel mode prunes by magnitude
+
     def prune_only(i):
         l = layers[i]
+        scheme = kernel_scheme
         if masked:
             sdgp.sdgp_prune_typed(dO[i].view(-1, l.Cout), n, m, scheme, 1234, DT, dense=vals[i])
         else:
@@ -457,7 +465,7 @@ def run_ours(args, layers):
     e2e_value = world * total_flops / (ms_e2e / e2e_steps * 1e-3) / 1e12
 
     if rank == 0:
-        base = (cpu_baseline(layers, args.workload, n, m, scheme, args.dtype)
+        base = (cpu_baseline(layers, args.workload, n, m, scheme, args.dtype, args.mode == "channel")
                 if world == 1 and not args.no_cpu_baseline else None)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -485,7 +493,7 @@ def run_ours(args, layers):
                                  "peak = %d x %s sustained dense bf16" % (per_steps, 1 if masked else 2, pk["source"])},
             "per_layer": per_layer,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": (1 if args.mode == "fused" else 2) * len(layers) * args.steps,
+            "gpu_launches": {"fused": 1, "channel": 4}.get(args.mode, 2) * len(layers) * args.steps,
             "clocks": clocks,
         }
         if base is not None:
@@ -611,12 +619,15 @@ def main():
     ap.add_argument("--workload", default="resnet9", choices=["resnet9", "gemm_large", "fc_small", "resnet50"])
     ap.add_argument("--scheme", default="magnitude", choices=sorted(SCHEMES))
     ap.add_argument("--nm", default="2:4")
-    ap.add_argument("--mode", default="two_pass", choices=["two_pass", "fused"],
-                    help="two_pass: prune kernel + sparse dgrad kernel per layer; fused: one kernel prunes and contracts")
+    ap.add_argument("--mode", default="two_pass", choices=["two_pass", "fused", "channel"],
+                    help="two_pass: prune kernel + sparse dgrad kernel per layer; fused: one kernel prunes and contracts; "
+                         "channel: two-pass under the per-channel reading of the L1 rescale (implies --scheme rescaled)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"],
                     help="element type of dL/dO, W and dL/dD (fp32 accumulation either way)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.mode == "channel":
+        args.scheme = "rescaled"
     if args.workload == "resnet50":
         if args.impl == "reference" or args.gpus != 1:
             raise SystemExit("--workload resnet50 is a single-GPU per-layer table of this implementation")

@@ -16,55 +16,78 @@ namespace {
 
 constexpr int kChThreads = 256;
 
+constexpr int kChSlots = 4096;  // channels one block pass accumulates in shared memory (2 x 16 KB)
+
+// Chunk columns a block handles side by side: as many as there are threads, chunks in a row, or
+// shared-memory slots.
+template <int CH>
+__host__ __device__ constexpr int chunk_columns(int cpr) {
+  int ct = cpr < kChThreads ? cpr : kChThreads;
+  return ct < kChSlots / CH ? ct : kChSlots / CH;
+}
+
 // sums[0..K) += sum over rows of |x|, sums[K..2K) += the same over kept elements only. A thread owns
 // one chunk of whole groups (8 elements, or m when m > 8) of a set of rows and keeps the chunk's
-// sixteen-or-more partial sums in registers; the mask is the prune kernels' (larger magnitude wins,
-// equal magnitudes: lower position), found by counting.
+// partial sums in registers; the mask is the prune kernels' (larger magnitude wins, equal
+// magnitudes: lower position), found by counting. The threads of a block that share a chunk column
+// combine their sums in shared memory, so that a block adds to each global sum once.
 template <int M, bool F16>
 __global__ void __launch_bounds__(kChThreads)
 channel_sums_kernel(const uint4* __restrict__ dO, int64_t rows, int K, int n, float* __restrict__ sums) {
   constexpr int CH = M < 8 ? 8 : M;
   constexpr int VEC = CH / 8;
+  __shared__ float sh_t[kChSlots], sh_s[kChSlots];
   const int cpr = K / CH;                                  // chunks per row
-  const int ct = cpr < kChThreads ? cpr : kChThreads;      // chunk columns handled side by side
+  const int ct = chunk_columns<CH>(cpr);
   const int lanes = kChThreads / ct;                       // rows handled side by side
   const int cc0 = threadIdx.x % ct, lane = threadIdx.x / ct;
-  if (lane >= lanes) return;
   for (int cbase = 0; cbase < cpr; cbase += ct) {
+    for (int i = threadIdx.x; i < ct * CH; i += kChThreads) sh_t[i] = sh_s[i] = 0.0f;
+    __syncthreads();
     const int cc = cbase + cc0;
-    if (cc >= cpr) continue;
-    float t[CH], s[CH];
+    if (lane < lanes && cc < cpr) {
+      float t[CH], s[CH];
 #pragma unroll
-    for (int i = 0; i < CH; ++i) t[i] = s[i] = 0.0f;
-    for (int64_t r = (int64_t)blockIdx.x * lanes + lane; r < rows; r += (int64_t)gridDim.x * lanes) {
-      const uint4* src = dO + (r * K + (int64_t)cc * CH) / 8;
-      uint32_t x[CH];
+      for (int i = 0; i < CH; ++i) t[i] = s[i] = 0.0f;
+      for (int64_t r = (int64_t)blockIdx.x * lanes + lane; r < rows; r += (int64_t)gridDim.x * lanes) {
+        const uint4* src = dO + (r * K + (int64_t)cc * CH) / 8;
+        uint32_t x[CH];
 #pragma unroll
-      for (int v = 0; v < VEC; ++v) {
-        const uint4 w = __ldg(src + v);
-        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+        for (int v = 0; v < VEC; ++v) {
+          const uint4 w = __ldg(src + v);
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-        for (int i = 0; i < 8; ++i) x[8 * v + i] = (i & 1) ? (ww[i >> 1] >> 16) : (ww[i >> 1] & 0xFFFFu);
+          for (int i = 0; i < 8; ++i) x[8 * v + i] = (i & 1) ? (ww[i >> 1] >> 16) : (ww[i >> 1] & 0xFFFFu);
+        }
+        uint32_t c[CH];
+#pragma unroll
+        for (int i = 0; i < CH; ++i) c[i] = ((x[i] & 0x7FFFu) << 5) | (uint32_t)(31 - (i % M));
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          int above = 0;
+#pragma unroll
+          for (int o = 0; o < CH; ++o)
+            if (o != i && (o / M) == (i / M)) above += (c[o] > c[i]) ? 1 : 0;
+          const float a = lane_lo<F16>(x[i] & 0x7FFFu);
+          t[i] += a;
+          if (above < n) s[i] += a;
+        }
       }
-      uint32_t c[CH];
-#pragma unroll
-      for (int i = 0; i < CH; ++i) c[i] = ((x[i] & 0x7FFFu) << 5) | (uint32_t)(31 - (i % M));
 #pragma unroll
       for (int i = 0; i < CH; ++i) {
-        int above = 0;
-#pragma unroll
-        for (int o = 0; o < CH; ++o)
-          if (o != i && (o / M) == (i / M)) above += (c[o] > c[i]) ? 1 : 0;
-        const float a = lane_lo<F16>(x[i] & 0x7FFFu);
-        t[i] += a;
-        if (above < n) s[i] += a;
+        atomicAdd(&sh_t[cc0 * CH + i], t[i]);
+        atomicAdd(&sh_s[cc0 * CH + i], s[i]);
       }
     }
-#pragma unroll
-    for (int i = 0; i < CH; ++i) {
-      atomicAdd(sums + (int64_t)cc * CH + i, t[i]);
-      atomicAdd(sums + K + (int64_t)cc * CH + i, s[i]);
+    __syncthreads();
+    for (int i = threadIdx.x; i < ct * CH; i += kChThreads) {
+      const int64_t k = (int64_t)cbase * CH + i;
+      if (k < K) {
+        atomicAdd(sums + k, sh_t[i]);
+        atomicAdd(sums + K + k, sh_s[i]);
+      }
     }
+    __syncthreads();
   }
 }
 
@@ -100,7 +123,7 @@ template <int M>
 cudaError_t launch_sums_m(bool f16, const void* dO, int64_t rows, int K, int n, float* sums, cudaStream_t stream) {
   constexpr int CH = M < 8 ? 8 : M;
   const int cpr = K / CH;
-  const int ct = cpr < kChThreads ? cpr : kChThreads;
+  const int ct = chunk_columns<CH>(cpr);
   const int lanes = kChThreads / ct;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
