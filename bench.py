@@ -141,7 +141,7 @@ class OracleArm:
             t0 = time.perf_counter()
             self.step(probe)
             dt = max(time.perf_counter() - t0, 1e-6)
-            if dt >= min(0.5, seconds / 4) or probe >= (1 << 20):
+            if dt >= min(2.0, seconds / 4) or probe >= (1 << 20):   # long enough that fixed costs no longer count
                 break
             probe *= 4
         return int(max(1, probe * seconds / dt))
