@@ -59,6 +59,25 @@ channel_sums_kernel(const uint4* __restrict__ dO, int64_t rows, int K, int n, fl
 #pragma unroll
           for (int i = 0; i < 8; ++i) x[8 * v + i] = (i & 1) ? (ww[i >> 1] >> 16) : (ww[i >> 1] & 0xFFFFu);
         }
+        if (M == 4) {
+          // groups of four: the packed-lane selection of the prune kernel (register i = elements i and i + 4)
+          const uint4 w = make_uint4(x[0] | (x[1] << 16), x[2] | (x[3] << 16), x[4] | (x[5] << 16), x[6] | (x[7] << 16));
+          uint32_t y[4], km[4];
+          switch (n) {
+            case 1: m4_prune_vector<1, SDGP_MAGNITUDE, F16>(w, 0, 0u, 0u, y[0], y[1], y[2], y[3], km[0], km[1], km[2], km[3]); break;
+            case 2: m4_prune_vector<2, SDGP_MAGNITUDE, F16>(w, 0, 0u, 0u, y[0], y[1], y[2], y[3], km[0], km[1], km[2], km[3]); break;
+            case 3: m4_prune_vector<3, SDGP_MAGNITUDE, F16>(w, 0, 0u, 0u, y[0], y[1], y[2], y[3], km[0], km[1], km[2], km[3]); break;
+            default: m4_prune_vector<4, SDGP_MAGNITUDE, F16>(w, 0, 0u, 0u, y[0], y[1], y[2], y[3], km[0], km[1], km[2], km[3]); break;
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            t[i] += lane_lo<F16>(x[i] & 0x7FFFu);
+            t[4 + i] += lane_lo<F16>(x[4 + i] & 0x7FFFu);
+            s[i] += lane_lo_abs<F16>(y[i]);          // pruned lanes are +0
+            s[4 + i] += lane_hi_abs<F16>(y[i]);
+          }
+          continue;
+        }
         uint32_t c[CH];
 #pragma unroll
         for (int i = 0; i < CH; ++i) c[i] = ((x[i] & 0x7FFFu) << 5) | (uint32_t)(31 - (i % M));
@@ -130,6 +149,7 @@ cudaError_t launch_sums_m(bool f16, const void* dO, int64_t rows, int K, int n, 
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return cudaErrorUnknown;
   int64_t blocks = (rows + lanes - 1) / lanes;
+  // measured: twice as many blocks cost more in the closing adds than they gain in loads in flight, half as many the reverse
   if (blocks > 4 * (int64_t)sms) blocks = 4 * (int64_t)sms;
   if (blocks < 1) return cudaSuccess;
   if (f16) channel_sums_kernel<M, true><<<(unsigned)blocks, kChThreads, 0, stream>>>((const uint4*)dO, rows, K, n, sums);
