@@ -312,6 +312,41 @@ def test_resnet18_shapes_small_batch():
         assert rel_fro(got_all.reshape(-1, layer.Cin)[idx], want) <= TOL, layer.name
 
 
+def test_memory_bound_1x1_layer_cold_inputs_repeated():
+    """A 1x1 convolution with many short tiles per CTA (ResNet-50 128->512 at 28 x 28, batch 256) launched again and
+    again with its inputs flushed from L2 in between: operand boxes then arrive late and out of request order,
+    which the stage hand-over between the loader, the metadata warps and the MMA thread must tolerate.
+    The tensors are drawn on the device (same law as the other convolution inputs); sampled rows go to the oracle."""
+    import paper_2202_00774_b200 as sdgp
+    B, HW, Cin, Cout = 256, 28, 128, 512
+    rows = B * HW * HW
+    g = torch.Generator(device="cuda").manual_seed(5)
+    u = torch.rand((rows, Cout), generator=g, device="cuda") - 0.5
+    lap = -torch.sign(u) * torch.log1p(-2 * u.abs())                       # Laplace(0, 1)
+    lap[torch.rand((rows, Cout), generator=g, device="cuda") < 0.5] = 0.0   # ReLU zeros
+    dO = lap.to(torch.bfloat16).view(torch.int16)
+    del u, lap
+    W = (torch.randn((Cout, Cin), generator=g, device="cuda") * (2.0 / Cin) ** 0.5).to(torch.bfloat16).view(torch.int16)
+    vals = torch.empty((rows, Cout // 2), dtype=torch.int16, device="cuda")
+    meta = torch.empty((rows, Cout // 16), dtype=torch.int16, device="cuda")
+    dD = torch.full((B, HW, HW, Cin), -1, dtype=torch.int16, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    sdgp.sdgp_prune(dO, 2, 4, sdgp.MAGNITUDE, 0, values=vals, meta=meta)
+    for _ in range(25):
+        flush.zero_()
+        sdgp.sdgp_spmm_conv2d(vals.view(B, HW, HW, Cout // 2), meta.view(B, HW, HW, Cout // 16), W.view(Cout, 1, 1, Cin), dD, 1, 0)
+        sdgp.sdgp_spmm_conv2d(vals.view(B, HW, HW, Cout // 2), meta.view(B, HW, HW, Cout // 16), W.view(Cout, 1, 1, Cin), dD, 1, 0)
+    torch.cuda.synchronize()
+    check_no_device_error()
+    idx = torch.from_numpy(np.unique(np.concatenate([np.random.default_rng(2).integers(0, rows, 400), [0, rows - 1]]))).cuda()
+    sample = dO[idx].cpu().numpy().view(np.uint16)
+    pruned = oracle.prune(sample, 2, 4, oracle.MAGNITUDE, want=("dense",))["dense"]
+    want = oracle.dgrad_linear(pruned, W.cpu().numpy().view(np.uint16))
+    got = to_f64(dD.view(rows, Cin)[idx])
+    assert rel_fro(got, want) <= TOL
+    assert not np.isnan(to_f64(dD)).any()
+
+
 # ------------------------------------------------------------------- fused
 
 
