@@ -509,6 +509,55 @@ def test_resnet9_full_size_layers_fused_sampled(index, scheme):
     _sampled_conv_check(layer, seed=10 + index, n=2, m=4, scheme=scheme, fused=True)
 
 
+def _device_conv_tensors(layer, seed):
+    """dO (ReLU-masked Laplace) and W (He-normal) drawn on the device: the full-size ResNet-50 tensors take
+    too long to draw on the host. Returned as int16 views of bf16."""
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    shape = layer.dO_shape()
+    u = torch.rand(shape, generator=g, device="cuda") - 0.5
+    lap = -torch.sign(u) * torch.log1p(-2 * u.abs())
+    lap[torch.rand(shape, generator=g, device="cuda") < 0.5] = 0.0
+    dO = lap.to(torch.bfloat16).view(torch.int16)
+    del u, lap
+    std = (2.0 / (layer.R * layer.S * layer.Cin)) ** 0.5
+    W = (torch.randn(layer.W_shape(), generator=g, device="cuda") * std).to(torch.bfloat16).view(torch.int16)
+    return dO, W
+
+
+R50_FULL = ["r50_s1_3x3_64to64_at56", "r50_s1_1x1_256to64_at56", "r50_s2_3x3s2_128to128_at56", "r50_s2_1x1_512to128_at28",
+            "r50_s3_3x3_256to256_at14", "r50_s4_projs2_1024to2048_at14", "r50_s4_3x3_512to512_at7", "r50_s4_1x1_512to2048_at7"]
+
+
+@pytest.mark.parametrize("name", R50_FULL)
+def test_resnet50_full_size_layers_sampled(name):
+    """ResNet-50 bottleneck shapes at batch 256, as `bench.py --workload resnet50` launches them (two-pass, 2:4
+    magnitude): whole sampled images (first, last, three random) go to the oracle, 600 of their output pixels are compared."""
+    import paper_2202_00774_b200 as sdgp
+    layer = dict((l.name, l) for l, _ in inputs.resnet50_layers(256))[name]
+    dO, W = _device_conv_tensors(layer, seed=len(name))
+    ws = torch.empty(sdgp.sdgp_workspace_size_conv2d(layer.B, layer.H, layer.W, layer.Cin, layer.Cout, layer.R, layer.S,
+                                                     layer.stride, layer.pad), dtype=torch.uint8, device="cuda")
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_conv2d(dO, W, dD, layer.stride, layer.pad, 2, 4, sdgp.MAGNITUDE, workspace=ws)
+    check_no_device_error()
+    assert not bool(torch.isnan(dD.view(torch.bfloat16)).any())          # every output was written
+    rng = np.random.default_rng(len(name))
+    imgs = np.unique(np.concatenate([[0, layer.B - 1], rng.integers(0, layer.B, 3)]))
+    sub = dO[torch.from_numpy(imgs).cuda()].cpu().numpy().view(np.uint16)           # [len(imgs), P, Q, Cout]
+    Wh = W.cpu().numpy().view(np.uint16)
+    Cpad = (layer.Cout + 31) // 32 * 32
+    flat = np.zeros((sub.size // layer.Cout, Cpad), np.uint16)
+    flat[:, :layer.Cout] = sub.reshape(-1, layer.Cout)
+    pruned = oracle.prune(flat, 2, 4, oracle.MAGNITUDE, want=("dense",))["dense"][:, :layer.Cout]
+    pruned = np.ascontiguousarray(pruned).reshape(sub.shape)
+    per_img = layer.H * layer.W
+    idx = np.unique(np.concatenate([k * per_img + rng.integers(0, per_img, 120) for k in range(len(imgs))] +
+                                   [np.arange(0, min(40, per_img)), len(imgs) * per_img - 1 - np.arange(0, min(40, per_img))]))
+    want = oracle.dgrad_conv2d(pruned, Wh, layer.H, layer.W, layer.stride, layer.pad, pixel_index=idx)
+    got = to_f64(dD[torch.from_numpy(imgs).cuda()]).reshape(-1, layer.Cin)[idx]
+    assert rel_fro(got, want) <= TOL
+
+
 @pytest.mark.parametrize("n,m,scheme", [(2, 4, oracle.MAGNITUDE), (1, 4, oracle.RESCALED), (2, 8, oracle.MAGNITUDE),
                                         (2, 16, oracle.RESCALED)])
 def test_gemm_large_full_size_sampled_rows(n, m, scheme):
