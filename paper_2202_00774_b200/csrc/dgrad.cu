@@ -53,6 +53,12 @@ namespace {
 
 constexpr int kBM = 128;             // output pixels (rows) per CTA tile = TMEM lanes
 constexpr int kThreadsGemm = 320;    // 10 warps
+// Fused pruning in the general kernel: eight more warps (10..17) prune beside warps 2..5. A lone warp
+// runs the pruning code at a quarter of an instruction per clock; twelve of them keep up with the
+// rate at which a memory-bound layer's dense dL/dO arrives.
+constexpr int kFusedHelperWarps = 8;
+constexpr int kThreadsGemmFused = kThreadsGemm + 32 * kFusedHelperWarps;
+constexpr int kFusedPruners = 128 + 32 * kFusedHelperWarps;
 constexpr int kEHwBytes = kBM * 16;  // rearranged metadata of one (tap, channel block): 128 lanes x 16 B
 constexpr int kOutBytes = kBM * 128; // epilogue staging slab: 128 rows x 64 bf16 columns
 constexpr uint32_t kTmemCols = 512;
@@ -164,26 +170,29 @@ __device__ __forceinline__ void build_metadata_image(const uint8_t* raw_rows, ui
   }
 }
 
-// Fused pruning of one pixel row of a stage: 128 dense channels (two 128-byte-swizzled boxes of
-// 64) -> 64 compressed values written straight into the A tile's swizzled row, plus the row's 16
-// bytes of position metadata in the row-major form the rearrangement step expects.
-// vbase = number of the row's first 8-element vector in the whole dL/dO tensor (random keys).
+// Fused pruning of one eighth of a pixel row of a stage (the unit of work the pruning threads share
+// out): the row's 128 dense channels lie in two 128-byte-swizzled boxes of 64; 16 of them = two
+// vectors become one 16-byte chunk of the compressed row, written straight into the A tile's swizzled
+// row, and two of the row's sixteen bytes of position metadata (row-major form, as the rearrangement
+// step expects). vbase = number of the row's first 8-element vector in the whole dL/dO tensor (random keys).
 template <int N, int SCHEME>
-__device__ __forceinline__ void fused_prune_row(const uint8_t* raw, int a_bytes, uint8_t* a_tile, uint8_t* meta_rows,
-                                                int i, int64_t vbase, uint32_t seed_lo, uint32_t seed_hi) {
-  uint32_t metaw[4] = {0u, 0u, 0u, 0u};
+__device__ __forceinline__ void fused_prune_eighth(const uint8_t* raw, int a_bytes, uint8_t* a_tile, uint8_t* meta_rows,
+                                                   int i, int e, int64_t vbase, uint32_t seed_lo, uint32_t seed_hi) {
   const int sw = i & 7;
-#pragma unroll 4
-  for (int j = 0; j < 16; ++j) {
+  uint32_t nibs = 0u;
+  uint2 out[2];
+#pragma unroll
+  for (int jj = 0; jj < 2; ++jj) {
+    const int j = 2 * e + jj;
     const uint4 w = *(const uint4*)(raw + (j >> 3) * a_bytes + i * 128 + (((j & 7) ^ sw) << 4));
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2;
     m4_prune_vector<N, SCHEME>(w, vbase + j, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
     compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
-    *(uint2*)(a_tile + i * 128 + (((j >> 1) ^ sw) << 4) + (j & 1) * 8) =
-        make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
-    metaw[j >> 2] |= nib2 << (8 * (j & 3));
+    out[jj] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
+    nibs |= nib2 << (8 * jj);
   }
-  *(uint4*)(meta_rows + i * 16) = make_uint4(metaw[0], metaw[1], metaw[2], metaw[3]);
+  *(uint4*)(a_tile + i * 128 + ((e ^ sw) << 4)) = make_uint4(out[0].x, out[0].y, out[1].x, out[1].y);
+  *(uint16_t*)(meta_rows + i * 16 + 2 * e) = (uint16_t)nibs;
 }
 
 // The four epilogue warps move one 128-row x BN accumulator to global memory in 64-column
@@ -247,7 +256,7 @@ __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* stagi
 }
 
 template <bool SPARSE, int BN, bool FUSED>
-__global__ void __launch_bounds__(kThreadsGemm, 1)
+__global__ void __launch_bounds__(FUSED ? kThreadsGemmFused : kThreadsGemm, 1)
 dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmE,
              const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
              const DgradParams p) {
@@ -466,7 +475,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         if (++acc == NACC) { acc = 0; aph ^= 1u; }
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < 6 || warp >= 10) {  // warps 10.. exist only in the fused instantiation
     // ------------------------------------------------- metadata rearranger
     if (SPARSE && !FUSED) {
       // A lone warp runs a dependent chain slowly, so the four warps do not share a stage: warp k
@@ -500,9 +509,10 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         if (!alive) break;
       }
     } else if (SPARSE) {
-      // Fused pruning: the four warps prune the stage's pixel rows together (thread = row),
-      // then each thread builds one TMEM lane of every metadata image.
-      const int row = threadIdx.x - 64;
+      // Fused pruning: warps 2..5 and the helper warps 10.. share out the stage's pixel rows in eighths
+      // (item = row, eighth); then each thread of warps 2..5 builds one TMEM lane of every metadata image.
+      const int pruner = warp < 6 ? (int)threadIdx.x - 64 : 128 + (int)threadIdx.x - kThreadsGemm;  // 0 .. kFusedPruners - 1
+      const int row = threadIdx.x - 64;  // warps 2..5 only
       bool alive = true;
       int st = 0;
       uint32_t ph = 0;
@@ -514,31 +524,35 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int w0 = wt * p.TW, h0 = ht * p.TH, b0 = t * p.TB;
         int r = reuse ? (p.R - 1) : 0, s = 0, cb = 0;
         for (int k = 0; k < uses_per_tile; ++k) {
-          // the four warps stay or leave together: they meet at a named barrier below
-          if (!ptx::named_bar_all(2, 128, ptx::mbar_wait(&raw_full[st], ph, err, 0x900u + st))) { alive = false; break; }
+          // the pruning warps stay or leave together: they meet at a named barrier below
+          if (!ptx::named_bar_all(2, kFusedPruners, ptx::mbar_wait(&raw_full[st], ph, err, 0x900u + st))) { alive = false; break; }
           const int q0 = w0 + p.pad_w - s, p0 = h0 + p.pad_h - r;
-          for (int i = row; i < p.img_rows; i += 128) {
+          const uint8_t* raw = sRaw + st * 2 * p.a_bytes;
+          uint8_t* a_tile = sA + st * p.a_bytes;
+          uint8_t* meta_rows = sEraw + st * p.eraw_bytes;
+          for (int item = pruner; item < 8 * p.img_rows; item += kFusedPruners) {
+            const int i = item >> 3, e = item & 7;
             const int iw = i % p.TW, ih = (i / p.TW) % img_h, ib = i / (p.TW * img_h);
             const int64_t pixel = ((int64_t)(b0 + ib) * p.P + (p0 + ih)) * p.Q + (q0 + iw);  // any value when outside
             const int64_t vbase = pixel * (p.Cout >> 3) + cb * 16;
-            const uint8_t* raw = sRaw + st * 2 * p.a_bytes;
-            uint8_t* a_tile = sA + st * p.a_bytes;
-            uint8_t* meta_rows = sEraw + st * p.eraw_bytes;
-#define SDGP_FUSED_ROW(NN, SS) fused_prune_row<NN, SS>(raw, p.a_bytes, a_tile, meta_rows, i, vbase, p.seed_lo, p.seed_hi)
-            if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_MAGNITUDE); else SDGP_FUSED_ROW(2, SDGP_MAGNITUDE); }
-            else if (p.fused_scheme == SDGP_RANDOM) { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_RANDOM); else SDGP_FUSED_ROW(2, SDGP_RANDOM); }
-            else { if (p.fused_n == 1) SDGP_FUSED_ROW(1, SDGP_RESCALED_MAGNITUDE); else SDGP_FUSED_ROW(2, SDGP_RESCALED_MAGNITUDE); }
-#undef SDGP_FUSED_ROW
+#define SDGP_FUSED_ITEM(NN, SS) fused_prune_eighth<NN, SS>(raw, p.a_bytes, a_tile, meta_rows, i, e, vbase, p.seed_lo, p.seed_hi)
+            if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_ITEM(1, SDGP_MAGNITUDE); else SDGP_FUSED_ITEM(2, SDGP_MAGNITUDE); }
+            else if (p.fused_scheme == SDGP_RANDOM) { if (p.fused_n == 1) SDGP_FUSED_ITEM(1, SDGP_RANDOM); else SDGP_FUSED_ITEM(2, SDGP_RANDOM); }
+            else { if (p.fused_n == 1) SDGP_FUSED_ITEM(1, SDGP_RESCALED_MAGNITUDE); else SDGP_FUSED_ITEM(2, SDGP_RESCALED_MAGNITUDE); }
+#undef SDGP_FUSED_ITEM
           }
-          ptx::named_bar_sync(2, 128);  // every row's metadata is in place before it is rearranged
-          for (int u = 0; u < p.rr; ++u) {
-            const int row_off = reuse ? (p.R - 1 - u) * p.TW : 0;
-            build_metadata_lane(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + u * kEHwBytes, row,
-                                rows_used);
+          ptx::fence_proxy_async_smem();                // the compressed tile is read by the tensor core
+          ptx::named_bar_sync(2, kFusedPruners);        // every row's metadata is in place before it is rearranged
+          if (warp < 6) {
+            for (int u = 0; u < p.rr; ++u) {
+              const int row_off = reuse ? (p.R - 1 - u) * p.TW : 0;
+              build_metadata_lane(sEraw + st * p.eraw_bytes + row_off * 16, sEhw + st * p.ehw_bytes + u * kEHwBytes, row,
+                                  rows_used);
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(&full[st], 0);
           }
-          ptx::fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive_cluster(&full[st], 0);
           if (++st == STAGES) { st = 0; ph ^= 1u; }
           if (++cb == p.k_blocks) {
             cb = 0;
@@ -1274,7 +1288,7 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const Dg
   const int pairs = p.pair_tiles < max_pairs ? p.pair_tiles : max_pairs;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3(kThreadsGemm);
+  cfg.blockDim = dim3(FUSED ? kThreadsGemmFused : kThreadsGemm);
   cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
