@@ -401,9 +401,14 @@ cudaError_t launch_m(int scheme, bool f16, const void* dO, int64_t nvec, int n, 
   if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)blocks), block(kThreads);
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
+  // Plain launch, without programmatic stream serialisation (the kernel's griddepcontrol
+  // instructions then do nothing). With the attribute, a stream of back-to-back masked-mode steps
+  // (this kernel, dense data-gradient kernel, this kernel, ...) stopped making progress on B200 after
+  // a few steps, at 4:8, 8:16 and 4:32 alike; the m = 4 and top-2 kernels run thousands of such steps
+  // with it. The cause was not found; the overlap it would buy on this slower path is small.
 #define SDGP_LAUNCH(S, F)                                                                           \
-  launch_after_previous(prune_kernel<M, S, F>, grid, block, stream, (const uint4*)dO, nvec, n, lo, hi, (uint4*)dense, \
-                                                 (uint2*)values, (uint8_t*)meta, (uint8_t*)mask)
+  prune_kernel<M, S, F><<<grid, block, 0, stream>>>((const uint4*)dO, nvec, n, lo, hi, (uint4*)dense,       \
+                                                    (uint2*)values, (uint8_t*)meta, (uint8_t*)mask)
   switch (scheme) {
     case SDGP_RANDOM: SDGP_LAUNCH(SDGP_RANDOM, false); break;
     case SDGP_MAGNITUDE: SDGP_LAUNCH(SDGP_MAGNITUDE, false); break;
