@@ -558,6 +558,29 @@ def test_resnet50_full_size_layers_sampled(name):
     assert rel_fro(got, want) <= TOL
 
 
+@pytest.mark.timeout(240, method="thread")
+def test_masked_mode_steps_back_to_back():
+    """Thirty-two masked-mode steps (4:8: generic prune kernel, dense data-gradient kernel) over three full-size ResNet-9
+    layers, enqueued without a host synchronisation in between; the last results are checked against the oracle."""
+    import paper_2202_00774_b200 as sdgp
+    layers = [inputs.resnet9_layers(512)[i] for i in (6, 3, 1)]
+    data = [_device_conv_tensors(l, seed=40 + i) for i, l in enumerate(layers)]
+    ws = [torch.empty(sdgp.sdgp_workspace_size_conv2d(l.B, l.H, l.W, l.Cin, l.Cout, 3, 3, 1, 1, sdgp.FLAG_MASKED),
+                      dtype=torch.uint8, device="cuda") for l in layers]
+    dD = [torch.full(l.dD_shape(), -1, dtype=torch.int16, device="cuda") for l in layers]
+    for _ in range(32):
+        for l, (dO, W), w, o in zip(layers, data, ws, dD):
+            sdgp.sdgp_dgrad_conv2d(dO, W, o, 1, 1, 4, 8, sdgp.MAGNITUDE, workspace=w, flags=sdgp.FLAG_MASKED)
+    torch.cuda.synchronize()
+    check_no_device_error()
+    for l, (dO, W), o in zip(layers, data, dD):
+        sub = dO[:2].cpu().numpy().view(np.uint16)                       # the first two images
+        pruned = oracle.prune(sub.reshape(-1, l.Cout), 4, 8, oracle.MAGNITUDE, want=("dense",))["dense"].reshape(sub.shape)
+        idx = np.unique(np.random.default_rng(l.Cin).integers(0, 2 * l.H * l.W, 200))
+        want = oracle.dgrad_conv2d(pruned, W.cpu().numpy().view(np.uint16), l.H, l.W, 1, 1, pixel_index=idx)
+        assert rel_fro(to_f64(o[:2]).reshape(-1, l.Cin)[idx], want) <= TOL, l.name
+
+
 @pytest.mark.parametrize("n,m,scheme", [(2, 4, oracle.MAGNITUDE), (1, 4, oracle.RESCALED), (2, 8, oracle.MAGNITUDE),
                                         (2, 16, oracle.RESCALED)])
 def test_gemm_large_full_size_sampled_rows(n, m, scheme):
