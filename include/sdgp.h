@@ -128,7 +128,8 @@ sdgp_status sdgp_dgrad_conv2d(const void* dO, const void* W, void* dD, int B, in
                               sdgp_scheme scheme, uint64_t seed, void* workspace,
                               size_t workspace_bytes, uint32_t flags, void* stream);
 
-/* The contraction alone, from an already compressed dL/dO (output of sdgp_prune):
+/* The contraction of Section 2.1 (Fig. 2, fully connected) / Section 3.1 (Fig. 3, convolution) alone, from
+ * an already compressed dL/dO (output of sdgp_prune):
  * values [rows, K/2] bf16 and meta [rows, K/16] u16 in place of dO. No workspace. Needs
  * K % 128 == 0 (Cout % 128 == 0 for the convolution), N % 64 == 0, stride 1 or 2. */
 sdgp_status sdgp_spmm_linear(const void* values, const void* meta, const void* W, void* dD,
@@ -181,9 +182,12 @@ sdgp_status sdgp_channel_scales(const void* dO, int64_t rows, int64_t K, int n, 
  * 9 MiB array that is part of the library image in device memory, so every GPU that loads the
  * library holds those 9 MiB until the process exits.
  *   Limit: rows * K <= 8,388,608 elements (e.g. 4096 x 2048); larger -> SDGP_ERR_TOO_LARGE.
- *   Same requirements as sdgp_dgrad_linear otherwise (K % 128 == 0, N % 64 == 0, n <= 2, ...).
+ *   Requirements: K % 128 == 0, N % 64 == 0, m in {4, 8, 16, 32} dividing K, n <= 2 or n == m
+ *   (n == m prunes nothing: the dense kernel reads dO directly and the array is not used),
+ *   16-byte aligned pointers; violations are reported before anything is launched.
  *   The first call on each device looks up the array's device address (one host-side runtime
- *   query, no allocation); make that first call outside any stream capture.
+ *   query, no allocation); make that first call outside any stream capture. First calls made
+ *   from several host threads at once are safe: each stores the same address.
  *   All calls on a device share the one array: two calls whose kernels may overlap on the GPU
  *   (different streams, no dependency) race on it and give wrong results - serialise them.
  *   Nothing in the array has to be cleared between calls: each call rewrites what it reads. */

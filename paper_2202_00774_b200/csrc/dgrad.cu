@@ -261,8 +261,6 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
              const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
              const DgradParams p) {
   using C = Cfg<SPARSE, BN>;
-  ptx::launch_dependents();  // the next kernel of the stream may start its set-up
-
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle of the A, B and staging tiles
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -324,6 +322,12 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   const uint32_t tmem_base = *tmem_slot;
   // everything above touched no global memory; the previous kernel's results are needed from here on
   ptx::wait_for_previous_grid();
+  // Only now may the next kernel of the stream be scheduled: every CTA of this grid owns its TMEM
+  // and has passed its cluster barrier and its wait for the previous grid, so a younger grid can
+  // never sit between this grid and a resource it still needs, and at most one grid is resident
+  // behind a running one. The younger grid's own TMEM allocation then simply waits for this grid
+  // to free its columns, which it does without anyone's help.
+  ptx::launch_dependents();
 
   const int rows_used = p.TW * p.TH * p.TB;
   const int taps = p.R * p.S;
@@ -677,8 +681,6 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
                   const HaloParams p) {
   using C = Cfg<SPARSE, BN>;
-  ptx::launch_dependents();  // the next kernel of the stream may start its set-up
-
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;
@@ -741,6 +743,12 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
   // everything above touched no global memory; the previous kernel's results are needed from here on
   ptx::wait_for_previous_grid();
+  // Only now may the next kernel of the stream be scheduled: every CTA of this grid owns its TMEM
+  // and has passed its cluster barrier and its wait for the previous grid, so a younger grid can
+  // never sit between this grid and a resource it still needs, and at most one grid is resident
+  // behind a running one. The younger grid's own TMEM allocation then simply waits for this grid
+  // to free its columns, which it does without anyone's help.
+  ptx::launch_dependents();
 
   const int taps = p.R * p.S;
   const int pair_stride = gridDim.x >> 1;
@@ -1142,15 +1150,39 @@ void choose_patch(int B, int H, int W, int* TW, int* TH, int* TB) {
   }
 }
 
+// Per-device caches, indexed by the ordinal of the CURRENT device (the library follows the caller's
+// current device, and a process may drive several). Filled on first use; concurrent first uses store the
+// same values.
+constexpr int kMaxDevices = 64;
+
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
 int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
+  static int n[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0) return 148;
+  if (!n[dev]) {
+    int v = 0;
+    cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+    n[dev] = v > 0 ? v : 148;
   }
-  return n;
+  return n[dev];
+}
+
+// Opts `kernel` in to the large dynamic shared-memory carve, once per device and instantiation.
+template <typename K>
+bool configure_once(K kernel, bool (&done)[kMaxDevices]) {
+  const int dev = current_device();
+  if (dev < 0) return false;
+  if (!done[dev]) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) return false;
+    done[dev] = true;
+  }
+  return true;
 }
 
 int round_up(int x, int a) { return (x + a - 1) / a * a; }
@@ -1277,13 +1309,9 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const Dg
       return SDGP_ERR_CUDA;
   }
 
-  static bool configured = false;
+  static bool configured[kMaxDevices] = {};
   auto kernel = dgrad_kernel<SPARSE, BN, FUSED>;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
-      return SDGP_ERR_CUDA;
-    configured = true;
-  }
+  if (!configure_once(kernel, configured)) return SDGP_ERR_CUDA;
   const int max_pairs = sm_count() / 2;
   const int pairs = p.pair_tiles < max_pairs ? p.pair_tiles : max_pairs;
   cudaLaunchConfig_t cfg = {};
@@ -1426,13 +1454,9 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
       return SDGP_ERR_CUDA;
   }
 
-  static bool configured = false;
+  static bool configured[kMaxDevices] = {};
   auto kernel = dgrad_halo_kernel<SPARSE, BN, NT, FUSED>;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
-      return SDGP_ERR_CUDA;
-    configured = true;
-  }
+  if (!configure_once(kernel, configured)) return SDGP_ERR_CUDA;
   const int max_pairs = sm_count() / 2;
   const int pairs = p.units < max_pairs ? p.units : max_pairs;
   cudaLaunchConfig_t cfg = {};

@@ -47,8 +47,8 @@ __global__ void __launch_bounds__(kThreads)
 prune_kernel(const uint4* __restrict__ dO, int64_t nvec, int n, uint32_t seed_lo, uint32_t seed_hi,
              uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
              uint8_t* __restrict__ mask) {
-  ptx::launch_dependents();
   ptx::wait_for_previous_grid();
+  ptx::launch_dependents();  // only once this grid's own predecessor is done: at most one grid ever waits behind a running one
   constexpr int LANES = (M <= 8) ? 1 : M / 8;
   constexpr int SUB = (M == 4) ? 4 : 8;  // elements of this thread that share a group
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
@@ -234,8 +234,8 @@ __global__ void __launch_bounds__(kThreads)
 prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                 uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
                 uint8_t* __restrict__ mask, OutPitch pitch) {
-  ptx::launch_dependents();
   ptx::wait_for_previous_grid();
+  ptx::launch_dependents();  // only once this grid's own predecessor is done: at most one grid ever waits behind a running one
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
   uint4 in[kVecPerThread];
 #pragma unroll
@@ -298,8 +298,8 @@ __global__ void __launch_bounds__(kThreads)
 prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                   uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
                   uint8_t* __restrict__ mask, OutPitch pitch) {
-  ptx::launch_dependents();
   ptx::wait_for_previous_grid();
+  ptx::launch_dependents();  // only once this grid's own predecessor is done: at most one grid ever waits behind a running one
   constexpr int LANES = M / 8;
   static_assert(N == 1 || N == 2, "threshold selection keeps one or two elements");
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;

@@ -31,7 +31,10 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 // scheduled (and run its set-up) once every CTA of this grid has got here. wait_for_previous_grid:
 // returns when the previous kernel of the stream has completed and its writes are visible; a
 // kernel must pass it before it touches global memory. Both do nothing in a kernel that was
-// launched without the attribute.
+// launched without the attribute. Every kernel of this library signals launch_dependents AFTER its
+// own wait_for_previous_grid (and after any other wait that has no time limit: TMEM allocation,
+// cluster barrier), so at most one younger grid is ever resident behind a running one and no
+// chain of waiting grids can build up.
 __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void wait_for_previous_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

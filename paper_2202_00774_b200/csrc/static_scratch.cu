@@ -21,6 +21,8 @@ unsigned char* g_scratch_addr[kMaxDevices] = {};
 
 // In host code `g_static_scratch` is only a handle for the symbol, not a device address;
 // the address the kernels need is asked for once per device, with that device current.
+// Threads that make their first call on a device at the same time may each do the lookup; they
+// all store the same address, so no lock is taken.
 sdgp_status scratch_for_current_device(unsigned char** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SDGP_ERR_CUDA;
@@ -43,20 +45,22 @@ extern "C" sdgp_status sdgp_dgrad_linear_static(const void* dO, const void* W, v
   if (m < 1 || m > 32 || n < 1 || n > m) return SDGP_ERR_INVALID_ARG;
   if (m != 4 && m != 8 && m != 16 && m != 32) return SDGP_ERR_UNSUPPORTED;
   if (K % m != 0) return SDGP_ERR_INVALID_ARG;
-  if (n > 2) return SDGP_ERR_UNSUPPORTED;
+  if (n > 2 && n != m) return SDGP_ERR_UNSUPPORTED;
   if (K % 128 != 0 || N % 64 != 0) return SDGP_ERR_UNSUPPORTED;
   if (rows > 0x7FFFFFFF || K > 0x7FFFFFFF || N > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;
   if ((uint64_t)rows * (uint64_t)K > kMaxElements) return SDGP_ERR_TOO_LARGE;
   if (rows == 0) return SDGP_OK;
   if (!dO || !W || !dD) return SDGP_ERR_INVALID_ARG;
   if (((uintptr_t)dO | (uintptr_t)W | (uintptr_t)dD) & 15u) return SDGP_ERR_ALIGNMENT;
+  cudaStream_t s = (cudaStream_t)stream;
+  // n == m prunes nothing: the dense kernel reads dO itself and the scratch is not touched
+  if (n == m) return sdgp::launch_dgrad(false, dO, nullptr, W, dD, 1, 1, (int)rows, (int)N, (int)K, 1, 1, 1, 0, s);
 
   unsigned char* scratch = nullptr;
   sdgp_status st = scratch_for_current_device(&scratch);
   if (st != SDGP_OK) return st;
   void* values = scratch;
   void* meta = scratch + kValuesBytes;
-  cudaStream_t s = (cudaStream_t)stream;
   // Every byte of values/meta that the contraction reads is rewritten by the prune kernel
   // first, so what an earlier call left in the array never shows.
   if (sdgp::launch_prune(dO, rows, K, n, m, (int)scheme, seed, nullptr, values, meta, nullptr, s) != cudaSuccess)

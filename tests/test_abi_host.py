@@ -34,8 +34,8 @@ def test_binding_lists_the_same_symbols():
 
 
 def test_status_strings(lib):
-    seen = {lib.sdgp_status_string(i).decode() for i in range(7)}
-    assert len(seen) == 7 and "ok" in seen
+    seen = {lib.sdgp_status_string(i).decode() for i in range(8)}
+    assert len(seen) == 8 and "ok" in seen and "unknown status" not in seen
     assert lib.sdgp_status_string(99).decode() == "unknown status"
 
 
@@ -92,3 +92,21 @@ def test_dgrad_rejects_bad_arguments_before_launch(lib):
     assert S(FAKE, 4, 64, 2, 4, 7, FAKE, None) == 1      # unknown element type
     assert S(FAKE, 4, 66, 2, 4, 0, FAKE, None) == 1      # K % m != 0
     assert S(FAKE, 4, 64, 2, 4, 0, None, None) == 1      # no output
+
+
+def test_static_scratch_variant_rejects_bad_arguments_before_launch(lib):
+    """sdgp_dgrad_linear_static validates on the host: nothing below reaches a launch or the scratch lookup."""
+    T = lib.sdgp_dgrad_linear_static
+    T.restype = ctypes.c_int
+    T.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] * 3 + [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_uint64,
+                                                                ctypes.c_void_p]
+    assert T(FAKE, FAKE, FAKE, 64, 192, 64, 2, 4, 1, 0, None) == 2                      # K % 128 != 0
+    assert T(FAKE, FAKE, FAKE, 64, 256, 96, 2, 4, 1, 0, None) == 2                      # N % 64 != 0
+    assert T(FAKE, FAKE, FAKE, 64, 256, 64, 3, 4, 1, 0, None) == 2                      # 3:4 has no compressed form
+    assert T(FAKE, FAKE, FAKE, 64, 256, 64, 0, 4, 1, 0, None) == 1                      # n < 1
+    assert T(FAKE, FAKE, FAKE, 64, 256, 64, 2, 4, 9, 0, None) == 1                      # unknown scheme
+    assert T(ctypes.c_void_p(0x1008), FAKE, FAKE, 64, 256, 64, 2, 4, 1, 0, None) == 3   # misaligned dO
+    assert T(FAKE, FAKE, ctypes.c_void_p(0x1004), 64, 256, 64, 2, 4, 1, 0, None) == 3   # misaligned dD
+    assert T(None, FAKE, FAKE, 64, 256, 64, 2, 4, 1, 0, None) == 1                      # null input
+    assert T(FAKE, FAKE, FAKE, 8193, 1024, 64, 2, 4, 1, 0, None) == 7                   # beyond the fixed scratch
+    assert T(FAKE, FAKE, FAKE, 0, 256, 64, 2, 4, 1, 0, None) == 0                       # rows == 0: no-op

@@ -1,7 +1,12 @@
 """GPU data-gradient kernels vs the fp64 CPU oracle, through the C ABI.
 
 Tolerance: relative Frobenius error <= 5e-3 against the fp64 result computed from the same
-pruned bf16 inputs (fp32 accumulation plus one bf16 rounding per output sits near 2e-3)."""
+pruned bf16 inputs (fp32 accumulation plus one bf16 rounding per output sits near 2e-3). A norm alone
+would let a few wholly wrong rows through, so the full-tensor cases also bound EVERY element:
+|got - ref| <= 2^-7 |ref| + 2^-16 sum_k |a_k| |b_k|  (one rounding to bf16, relative 2^-8, with a factor two
+to spare; fp32 accumulation of up to a few thousand products, each step off by at most 2^-24 of the
+running magnitude, again with room to spare). The second term comes from the oracle run on the operands'
+magnitudes."""
 import numpy as np
 import pytest
 
@@ -26,6 +31,29 @@ def rel_fro(got, ref):
     return np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
 
 
+def magnitudes(bits):
+    """The same 16-bit patterns with the sign cleared."""
+    return (np.asarray(bits).view(np.uint16) & np.uint16(0x7FFF)).astype(np.uint16)
+
+
+def assert_close(got, want, absdot=None, what=""):
+    """Norm bound, and - when the oracle's sum of |a||b| per output is given - the bound on every element."""
+    assert rel_fro(got, want) <= TOL, what
+    if absdot is not None:
+        bound = 2.0 ** -7 * np.abs(want) + 2.0 ** -16 * absdot
+        bad = np.abs(got - want) > bound
+        assert not bad.any(), "%s: %d elements off, first at %s" % (what, int(bad.sum()), np.argwhere(bad)[0])
+
+
+def linear_ref(src, W):
+    return oracle.dgrad_linear(src, W), oracle.dgrad_linear(magnitudes(src), magnitudes(W))
+
+
+def conv_ref(src, W, H, Wd, stride, pad, **kw):
+    return (oracle.dgrad_conv2d(src, W, H, Wd, stride, pad, **kw),
+            oracle.dgrad_conv2d(magnitudes(src), magnitudes(W), H, Wd, stride, pad, **kw))
+
+
 def check_no_device_error():
     import paper_2202_00774_b200 as sdgp
     assert sdgp.sdgp_last_device_error() == 0
@@ -41,7 +69,7 @@ def test_dense_linear(rows, K, N):
     dD = torch.full((rows, N), -1, dtype=torch.int16, device="cuda")
     sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, 4, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
     check_no_device_error()
-    assert rel_fro(to_f64(dD), oracle.dgrad_linear(dO, W)) <= TOL
+    assert_close(to_f64(dD), *linear_ref(dO, W))
 
 
 @pytest.mark.parametrize("rows,K,N", [(256, 512, 256), (300, 256, 128), (77, 128, 64), (1000, 384, 192)])
@@ -53,7 +81,7 @@ def test_spmm_linear_from_oracle_compressed(rows, K, N):
     dD = torch.full((rows, N), -1, dtype=torch.int16, device="cuda")
     sdgp.sdgp_spmm_linear(dev16(ref["values"]), dev16(ref["meta"]), dev16(W), dD)
     check_no_device_error()
-    assert rel_fro(to_f64(dD), oracle.dgrad_linear(ref["dense"], W)) <= TOL
+    assert_close(to_f64(dD), *linear_ref(ref["dense"], W))
 
 
 @pytest.mark.parametrize("scheme", [oracle.RANDOM, oracle.MAGNITUDE, oracle.RESCALED])
@@ -67,7 +95,7 @@ def test_pruned_linear_two_pass(n, m, scheme):
     sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, n, m, scheme, seed=42, workspace=ws)
     check_no_device_error()
     pruned = oracle.prune(dO, n, m, scheme, 42, want=("dense",))["dense"]
-    assert rel_fro(to_f64(dD), oracle.dgrad_linear(pruned, W)) <= TOL
+    assert_close(to_f64(dD), *linear_ref(pruned, W))
 
 
 # Patterns with more than two survivors in some aligned 4-chunk have no 2:4 form: the masked mode
@@ -86,7 +114,7 @@ def test_pruned_linear_masked(n, m, scheme):
     pruned = oracle.prune(dO, n, m, scheme, 17, want=("dense",))["dense"]
     # the workspace holds Algorithm 1's return value, bit for bit (n == m prunes nothing: dO is read directly)
     assert n == m or np.array_equal(ws.cpu().numpy()[:rows * K * 2].view(np.uint16).reshape(rows, K), pruned)
-    assert rel_fro(to_f64(dD), oracle.dgrad_linear(pruned, W)) <= TOL
+    assert_close(to_f64(dD), *linear_ref(pruned, W))
 
 
 @pytest.mark.parametrize("n,m,scheme", [(4, 8, oracle.MAGNITUDE), (3, 4, oracle.RESCALED), (8, 32, oracle.RANDOM)])
@@ -103,7 +131,7 @@ def test_pruned_conv_masked(case, n, m, scheme):
     sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, stride, pad, n, m, scheme, seed=23, workspace=ws, flags=sdgp.FLAG_MASKED)
     check_no_device_error()
     pruned = oracle.prune(dO.reshape(-1, Cout), n, m, scheme, 23, want=("dense",))["dense"].reshape(dO.shape)
-    assert rel_fro(to_f64(dD), oracle.dgrad_conv2d(pruned, W, H, Wd, stride, pad)) <= TOL
+    assert_close(to_f64(dD), *conv_ref(pruned, W, H, Wd, stride, pad))
 
 
 def test_sparse_modes_refuse_patterns_without_a_2_4_form():
@@ -128,7 +156,7 @@ def test_fc_small_config_full():
     sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, 2, 4, sdgp.MAGNITUDE, workspace=ws)
     check_no_device_error()
     pruned = oracle.prune(dO, 2, 4, oracle.MAGNITUDE, want=("dense",))["dense"]
-    assert rel_fro(to_f64(dD), oracle.dgrad_linear(pruned, W)) <= TOL
+    assert_close(to_f64(dD), *linear_ref(pruned, W))
 
 
 # --------------------------------------------------------------------- conv
@@ -156,7 +184,7 @@ def test_dense_conv(case):
     dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
     sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, pad, 4, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
     check_no_device_error()
-    assert rel_fro(to_f64(dD), oracle.dgrad_conv2d(dO, W, H, Wd, 1, pad)) <= TOL
+    assert_close(to_f64(dD), *conv_ref(dO, W, H, Wd, 1, pad))
 
 
 @pytest.mark.parametrize("scheme", [oracle.RANDOM, oracle.MAGNITUDE, oracle.RESCALED])
@@ -172,7 +200,7 @@ def test_pruned_conv_two_pass(case, scheme):
     sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, pad, 2, 4, scheme, seed=7, workspace=ws)
     check_no_device_error()
     pruned = oracle.prune(dO.reshape(-1, Cout), 2, 4, scheme, 7, want=("dense",))["dense"].reshape(dO.shape)
-    assert rel_fro(to_f64(dD), oracle.dgrad_conv2d(pruned, W, H, Wd, 1, pad)) <= TOL
+    assert_close(to_f64(dD), *conv_ref(pruned, W, H, Wd, 1, pad))
 
 
 # Shapes that switch on the kernel's shared-memory reuse modes: enough tiles that every CTA
@@ -210,9 +238,8 @@ def test_conv_reuse_modes_sampled(case, mode):
     rng = np.random.default_rng(1)
     npix = B * H * Wd
     idx = np.unique(np.concatenate([rng.integers(0, npix, 1500), np.arange(0, 300), np.arange(npix - 300, npix)]))
-    want = oracle.dgrad_conv2d(src, W, H, Wd, 1, pad, pixel_index=idx)
     got = to_f64(dD).reshape(npix, Cin)[idx]
-    assert rel_fro(got, want) <= TOL
+    assert_close(got, *conv_ref(src, W, H, Wd, 1, pad, pixel_index=idx))
     # nothing outside the sample is left unwritten (the buffer was pre-filled with 0xFFFF = NaN)
     assert not np.isnan(to_f64(dD)).any()
 
@@ -246,7 +273,7 @@ def test_conv_stride2(case, mode):
     check_no_device_error()
     got = to_f64(dD)
     assert not np.isnan(got).any()
-    assert rel_fro(got, oracle.dgrad_conv2d(src, W, H, Wd, 2, pad)) <= TOL
+    assert_close(got, *conv_ref(src, W, H, Wd, 2, pad))
 
 
 # Output-channel counts that are not whole 128-channel blocks: the compressed rows are padded.
@@ -271,7 +298,7 @@ def test_pruned_conv_partial_channel_block(case, scheme):
     sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, stride, pad, 2, 4, scheme, seed=11, workspace=ws)
     check_no_device_error()
     pruned = oracle.prune(dO.reshape(-1, Cout), 2, 4, scheme, 11, want=("dense",))["dense"].reshape(dO.shape)
-    assert rel_fro(to_f64(dD), oracle.dgrad_conv2d(pruned, W, H, Wd, stride, pad)) <= TOL
+    assert_close(to_f64(dD), *conv_ref(pruned, W, H, Wd, stride, pad))
 
 
 def test_resnet50_bottleneck_shapes_small_batch():
@@ -378,7 +405,7 @@ def test_fused_prune_and_dgrad(case, scheme, n):
     pruned = oracle.prune(dO.reshape(-1, Cout), n, 4, scheme, 21, want=("dense",))["dense"].reshape(dO.shape)
     got = to_f64(dD)
     assert not np.isnan(got).any()
-    assert rel_fro(got, oracle.dgrad_conv2d(pruned, W, H, Wd, stride, pad)) <= TOL
+    assert_close(got, *conv_ref(pruned, W, H, Wd, stride, pad))
 
 
 # Shapes for the whole-filter-reuse kernel (more than one tap, images at least one 8 x 16 strip
@@ -430,7 +457,7 @@ def test_whole_filter_reuse_kernel(case, mode):
     check_no_device_error()
     got = to_f64(dD)
     assert not np.isnan(got).any()           # every output was written
-    assert rel_fro(got, oracle.dgrad_conv2d(src, W, H, Wd, stride, pad)) <= TOL
+    assert_close(got, *conv_ref(src, W, H, Wd, stride, pad))
 
 
 def test_fused_needs_groups_of_four():
@@ -488,9 +515,8 @@ def _sampled_conv_check(layer, seed, n, m, scheme, samples=600, fused=False):
     idx = np.concatenate([b * per_img + rng.integers(0, per_img, samples // len(imgs)) for b in imgs])
     edge = min(64, per_img)   # first pixels of the first image, last pixels of the last one
     idx = np.unique(np.concatenate([idx, np.arange(0, edge), np.arange(layer.B * per_img - edge, layer.B * per_img)]))
-    want = oracle.dgrad_conv2d(pruned, W, layer.H, layer.W, 1, layer.pad, pixel_index=idx)
     got = inputs.bf16_bits_to_f32(got_all.reshape(-1, layer.Cin)[idx]).astype(np.float64)
-    assert rel_fro(got, want) <= TOL
+    assert_close(got, *conv_ref(pruned, W, layer.H, layer.W, 1, layer.pad, pixel_index=idx), what=layer.name)
 
 
 @pytest.mark.parametrize("index", range(7))
@@ -524,8 +550,7 @@ def _device_conv_tensors(layer, seed):
     return dO, W
 
 
-R50_FULL = ["r50_s1_3x3_64to64_at56", "r50_s1_1x1_256to64_at56", "r50_s2_3x3s2_128to128_at56", "r50_s2_1x1_512to128_at28",
-            "r50_s3_3x3_256to256_at14", "r50_s4_projs2_1024to2048_at14", "r50_s4_3x3_512to512_at7", "r50_s4_1x1_512to2048_at7"]
+R50_FULL = [l.name for l, _ in inputs.resnet50_layers(256)]   # every distinct bottleneck convolution (23 shapes)
 
 
 @pytest.mark.parametrize("name", R50_FULL)
@@ -553,32 +578,8 @@ def test_resnet50_full_size_layers_sampled(name):
     per_img = layer.H * layer.W
     idx = np.unique(np.concatenate([k * per_img + rng.integers(0, per_img, 120) for k in range(len(imgs))] +
                                    [np.arange(0, min(40, per_img)), len(imgs) * per_img - 1 - np.arange(0, min(40, per_img))]))
-    want = oracle.dgrad_conv2d(pruned, Wh, layer.H, layer.W, layer.stride, layer.pad, pixel_index=idx)
     got = to_f64(dD[torch.from_numpy(imgs).cuda()]).reshape(-1, layer.Cin)[idx]
-    assert rel_fro(got, want) <= TOL
-
-
-@pytest.mark.timeout(240, method="thread")
-def test_masked_mode_steps_back_to_back():
-    """Thirty-two masked-mode steps (4:8: generic prune kernel, dense data-gradient kernel) over three full-size ResNet-9
-    layers, enqueued without a host synchronisation in between; the last results are checked against the oracle."""
-    import paper_2202_00774_b200 as sdgp
-    layers = [inputs.resnet9_layers(512)[i] for i in (6, 3, 1)]
-    data = [_device_conv_tensors(l, seed=40 + i) for i, l in enumerate(layers)]
-    ws = [torch.empty(sdgp.sdgp_workspace_size_conv2d(l.B, l.H, l.W, l.Cin, l.Cout, 3, 3, 1, 1, sdgp.FLAG_MASKED),
-                      dtype=torch.uint8, device="cuda") for l in layers]
-    dD = [torch.full(l.dD_shape(), -1, dtype=torch.int16, device="cuda") for l in layers]
-    for _ in range(32):
-        for l, (dO, W), w, o in zip(layers, data, ws, dD):
-            sdgp.sdgp_dgrad_conv2d(dO, W, o, 1, 1, 4, 8, sdgp.MAGNITUDE, workspace=w, flags=sdgp.FLAG_MASKED)
-    torch.cuda.synchronize()
-    check_no_device_error()
-    for l, (dO, W), o in zip(layers, data, dD):
-        sub = dO[:2].cpu().numpy().view(np.uint16)                       # the first two images
-        pruned = oracle.prune(sub.reshape(-1, l.Cout), 4, 8, oracle.MAGNITUDE, want=("dense",))["dense"].reshape(sub.shape)
-        idx = np.unique(np.random.default_rng(l.Cin).integers(0, 2 * l.H * l.W, 200))
-        want = oracle.dgrad_conv2d(pruned, W.cpu().numpy().view(np.uint16), l.H, l.W, 1, 1, pixel_index=idx)
-        assert rel_fro(to_f64(o[:2]).reshape(-1, l.Cin)[idx], want) <= TOL, l.name
+    assert_close(got, *conv_ref(pruned, Wh, layer.H, layer.W, layer.stride, layer.pad, pixel_index=idx), what=name)
 
 
 @pytest.mark.parametrize("n,m,scheme", [(2, 4, oracle.MAGNITUDE), (1, 4, oracle.RESCALED), (2, 8, oracle.MAGNITUDE),
@@ -595,9 +596,8 @@ def test_gemm_large_full_size_sampled_rows(n, m, scheme):
     rng = np.random.default_rng(n * 10 + m)
     rows = np.unique(np.concatenate([[0, 127, 128, c["rows"] - 1], rng.integers(0, c["rows"], 92)]))
     pruned = oracle.prune(dO[rows], n, m, scheme, 9, want=("dense",))["dense"]   # magnitude schemes: row-local
-    want = oracle.dgrad_linear(pruned, W)
     got = inputs.bf16_bits_to_f32(dD[torch.from_numpy(rows).cuda()].cpu().numpy().view(np.uint16)).astype(np.float64)
-    assert rel_fro(got, want) <= TOL
+    assert_close(got, *linear_ref(pruned, W))
 
 
 def test_bounded_wait_reports_timeout_and_context_survives():
@@ -612,4 +612,4 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     dD = torch.empty((128, 64), dtype=torch.int16, device="cuda")
     sdgp.sdgp_dgrad_linear(dev16(dO), dev16(W), dD, 4, 4, sdgp.MAGNITUDE, flags=sdgp.FLAG_DENSE)
     check_no_device_error()
-    assert rel_fro(to_f64(dD), oracle.dgrad_linear(dO, W)) <= TOL
+    assert_close(to_f64(dD), *linear_ref(dO, W))

@@ -1,10 +1,12 @@
 """sdgp_dgrad_linear_static - the entry point for callers that cannot allocate device memory
 (its scratch is a fixed array inside the library) - must give what sdgp_dgrad_linear gives
-with a caller-supplied workspace. Two calls in a row with different inputs share the array;
-the second must not see anything the first left behind. Collected last on purpose."""
+with a caller-supplied workspace, bit for bit: both run the same two kernels on the same inputs.
+Two calls in a row with different inputs share the array; the second must not see anything the
+first left behind. Each result is also checked against the CPU oracle. Collected last on purpose."""
 import numpy as np
 import pytest
 
+import oracle
 from paper_2202_00774_b200 import inputs
 
 torch = pytest.importorskip("torch")
@@ -23,7 +25,10 @@ def _dev16(a):
 
 def test_static_scratch_matches_workspace_variant_twice():
     import paper_2202_00774_b200 as sdgp
-    calls = [(700, 512, 256, 2, 4, sdgp.MAGNITUDE, 11), (333, 1024, 128, 2, 8, sdgp.RESCALED_MAGNITUDE, 12)]
+    # the second call is smaller in rows, larger in K: its rows lie over the first call's leftovers;
+    # the third prunes nothing (n == m) and must leave the shared array alone
+    calls = [(700, 512, 256, 2, 4, sdgp.MAGNITUDE, 11), (333, 1024, 128, 2, 8, sdgp.RESCALED_MAGNITUDE, 12),
+             (200, 256, 64, 4, 4, sdgp.MAGNITUDE, 13)]
     for rows, K, N, n, m, scheme, seed in calls:
         dO, W = inputs.fc_tensors(rows, K, N, seed=seed)
         d_dO, d_W = _dev16(dO), _dev16(W)
@@ -34,8 +39,10 @@ def test_static_scratch_matches_workspace_variant_twice():
         sdgp.sdgp_dgrad_linear_static(d_dO, d_W, got, n, m, scheme, seed=seed)
         torch.cuda.synchronize()
         assert sdgp.sdgp_last_device_error() == 0
-        a, b = _f64(got), _f64(want)
-        assert np.linalg.norm(a - b) <= TOL * np.linalg.norm(b)
+        assert torch.equal(got, want)          # same kernels, same inputs: identical bits
+        pruned = oracle.prune(dO, n, m, scheme, seed, want=("dense",))["dense"]
+        ref = oracle.dgrad_linear(pruned, W)
+        assert np.linalg.norm(_f64(got) - ref) <= TOL * np.linalg.norm(ref)
 
 
 def test_static_scratch_rejects_oversized_problems():
