@@ -625,8 +625,24 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
 constexpr int kHaloTH = 16;  // pixel rows of a strip: 8 x 16 pixels = the 128 rows of an accumulator
 constexpr int kHaloAStages = 2;
-constexpr int kPruneWarps = 16;  // fused pruning: warps 10..25 prune the dense A box in shared memory
-constexpr int kThreadsHaloFused = kThreadsGemm + 32 * kPruneWarps;
+// Warp roles of the fused whole-filter-reuse kernel (24 warps: registers are granted to warps in fours, and
+// 24 x 80 registers is what fits). Warp w runs on scheduler w % 4, and the thread that issues the MMAs
+// (warp 1) is what bounds these kernels, so the busy pruning warps keep off its scheduler: warp 0 streams W,
+// warp 1 issues the MMAs, warps 4..7 are the epilogue (one per TMEM lane quarter), and of the rest those
+// with w % 4 != 1 prune (2, 3, 8, 10..12, 14..16, 18..20, 22, 23: fourteen warps); warps 9, 13, 17 and 21
+// have no role.
+constexpr int kPruneWarps = 14;
+constexpr unsigned kIdleWaitNs = 200;  // sleep between polls of the waits that are off the critical path
+constexpr int kThreadsHaloFused = 24 * 32;
+
+// Division by a divisor fixed for the launch: m = floor(2^32 / d) (0xFFFFFFFF for d = 1) gives a quotient
+// that is at most one too small for any 32-bit x; one correction step makes it exact.
+__host__ __device__ inline uint32_t div_magic(uint32_t d) { return d <= 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / d); }
+__device__ __forceinline__ void divmod(uint32_t x, uint32_t d, uint32_t m, uint32_t& q, uint32_t& r) {
+  q = __umulhi(x, m);
+  r = x - q * d;
+  if (r >= d) { ++q; r -= d; }
+}
 
 struct HaloParams {
   int B, H, W, Cin, Cout;
@@ -635,6 +651,7 @@ struct HaloParams {
   int nt;                  // strips per CTA tile set (1 or 2), side by side, sharing every W stage
   int sets_w, tiles_h, tiles_n;
   int m_sets;              // sets_w * tiles_h * B
+  uint32_t mg_tiles_n, mg_sets_w, mg_tiles_h;  // div_magic of the three counts above
   int pair_tiles;          // ceil(m_sets / 2) * tiles_n
   int units;               // work units: pair tiles, the last `units - split_from` of them split by strip
   int split_from;          // units >= split_from cover one strip of a pair tile each (quantisation of the last round)
@@ -644,35 +661,51 @@ struct HaloParams {
   int img_rows;            // pitch * img_h
   int w_stages;
   int meta_col, meta_shared, out_bufs;
-  int a_bytes, eraw_bytes, w_bytes, ehw_bytes;  // per stage
-  int off_eraw, off_half1, off_w, off_ehw, off_out, off_bar;
+  int a_bytes, eraw_bytes, w_bytes;  // per stage
+  // Position metadata of an A box in the order the tensor core wants, stored ONCE per box and shared by every
+  // tap: "master" pi (pi = 0, 1) pairs box rows (pi + 2m, pi + 2m + 1); its 16-byte line ((2m + e) * pitch + x)
+  // holds, for the four MMAs of a channel block, the metadata of channels 16e .. 16e+15 of the MMA's 32 at
+  // box pixel (pi + 2m, x) in the low half-words and of the pixel below it in the high half-words. The
+  // TMEM image of tap (r, s) and strip j is then the window of 16 groups of 8 lines that starts at line
+  // ((R-1-r - pi) * pitch + 8j + S-1-s) of master pi = (R-1-r) % 2, groups pitch lines apart: one
+  // tcgen05.cp whose descriptor carries that start address and stride.
+  int pairs0, pairs1;      // row pairs of the two masters
+  int m0_bytes, meta_bytes;  // bytes of master 0; of both (one A stage)
+  int off_eraw, off_meta, off_w, off_out, off_bar;
   int smem_bytes;
-  // fused pruning (A is the dense dL/dO; m = 4)
+  // fused pruning (A is the dense dL/dO; m = 4): the pruning warps read it straight from global memory
+  const uint8_t* a_dense;  // dL/dO [B, P, Q, Cout], 16-bit elements
+  uint32_t pitch_magic;    // ceil(2^20 / pitch): i / pitch == (i * pitch_magic) >> 20 for every box pixel row i
   int fused_n, fused_scheme;
   uint32_t seed_lo, seed_hi;
   int P, Q;                // dO pixel grid (linear element index of the random scheme)
   int f16;                 // element type of A, W and dD: 0 = bf16, 1 = IEEE binary16
 };
 
-// Fused pruning of one quarter (32 channels = 4 vectors) of one pixel row of a dense A box that
-// lies in shared memory as two 128-byte-swizzled halves of 64 channels: `half` points at the half
-// holding the quarter, c = quarter number (0..3). The results stay in registers (out, metaw)
-// until every thread of the round has read its input, because the compressed row overwrites the
-// first half in place.
+// Fused pruning of four vectors (8 channels each, already in registers) of one pixel row: out[v] = the 8
+// compressed bytes of vector v, metaw = their four bytes of position metadata (byte v = the two nibbles of
+// vector v). vnum(v) = number of vector v in the whole dL/dO tensor (random keys): vbase + vstep * v.
 template <int N, int SCHEME>
-__device__ __forceinline__ void fused_prune_quarter(const uint8_t* half, int i, int c, int64_t vbase, uint32_t seed_lo,
+__device__ __forceinline__ void fused_prune_vectors(const uint4 (&w)[4], int64_t vbase, int vstep, uint32_t seed_lo,
                                                     uint32_t seed_hi, uint2 (&out)[4], uint32_t& metaw) {
-  const int sw = i & 7;
   metaw = 0u;
 #pragma unroll
   for (int v = 0; v < 4; ++v) {
-    const uint4 w = *(const uint4*)(half + i * 128 + (((4 * (c & 1) + v) ^ sw) << 4));
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2;
-    m4_prune_vector<N, SCHEME>(w, vbase + 4 * c + v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
+    m4_prune_vector<N, SCHEME>(w[v], vbase + vstep * v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
     compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
     out[v] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
     metaw |= nib2 << (8 * v);
   }
+}
+
+// 16 bytes from global memory, read-only path, kept out of L1 (each byte is used once by this SM).
+__device__ __forceinline__ uint4 ldg_stream(const uint8_t* ptr) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(ptr));
+  return v;
 }
 
 template <bool SPARSE, int BN, int NT, bool FUSED>
@@ -681,19 +714,19 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmD,
                   const HaloParams p) {
   using C = Cfg<SPARSE, BN>;
+  constexpr int kEpilogueWarp0 = FUSED ? 4 : 6;  // first of the four epilogue warps
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;
-  uint8_t* sEraw = smem + p.off_eraw;
-  uint8_t* sHalf1 = smem + p.off_half1;  // fused: channels 64..127 of the dense box being pruned
+  uint8_t* sEraw = smem + p.off_eraw;    // two-pass: the row-major metadata box as TMA delivers it
+  uint8_t* sMeta = smem + p.off_meta;    // the two metadata masters of each A stage
   uint8_t* sW = smem + p.off_w;
-  uint8_t* sEhw = smem + p.off_ehw;
   uint8_t* sOut = smem + p.off_out;
   uint64_t* a_full = (uint64_t*)(smem + p.off_bar);
   uint64_t* a_empty = a_full + kHaloAStages;
   uint64_t* meta_full = a_empty + kHaloAStages;
-  uint64_t* raw_full = meta_full + kHaloAStages;  // fused: the dense box has landed
-  uint64_t* w_ready = raw_full + kHaloAStages;    // W bytes landed AND (sparse) metadata tiles built
+  uint64_t* meta_ready = meta_full + kHaloAStages;  // two-pass: the masters of the A stage are built (both CTAs)
+  uint64_t* w_ready = meta_ready + kHaloAStages;    // W bytes landed
   uint64_t* w_empty = w_ready + kMaxStages;
   uint64_t* acc_full = w_empty + kMaxStages;
   uint64_t* acc_empty = acc_full + 2;
@@ -709,15 +742,14 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     for (int s = 0; s < kHaloAStages; ++s) {
       // fused: A and its metadata rows are complete when every pruning warp has arrived
       // (a_full: the warps of both CTAs; meta_full: this CTA's)
-      ptx::mbar_init(&a_full[s], FUSED ? 2 * kPruneWarps : 1);
+      // (one arrival per work unit of the box: 8 pixel rows)
+      ptx::mbar_init(&a_full[s], FUSED ? 2 * ((p.img_rows + 7) >> 3) : 1);
       ptx::mbar_init(&a_empty[s], 1);
-      ptx::mbar_init(&meta_full[s], FUSED ? kPruneWarps : 1);
-      ptx::mbar_init(&raw_full[s], 1);
+      ptx::mbar_init(&meta_full[s], 1);
+      ptx::mbar_init(&meta_ready[s], 8);  // four metadata warps in each CTA
     }
     for (int s = 0; s < kMaxStages; ++s) {
-      // one arrival from the producer (with the byte count) plus, for sparse A, one from the
-      // metadata warp of each CTA that built the tap: the MMA thread waits once per tap
-      ptx::mbar_init(&w_ready[s], SPARSE ? 3 : 1);
+      ptx::mbar_init(&w_ready[s], 1);  // the producer's arrival with the byte count
       ptx::mbar_init(&w_empty[s], 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -766,12 +798,16 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   // tile set of unit `u` for this CTA: first input channel, first pixel column / row, image
   auto locate = [&p, rank](int u, int& n0, int& w0, int& h0, int& b0) -> bool {
     const int pt = u < p.split_from ? u : p.split_from + ((u - p.split_from) >> 1);
-    n0 = (pt % p.tiles_n) * BN;
-    int t = 2 * (pt / p.tiles_n) + (int)rank;
-    const bool in_range = t < p.m_sets;  // a set past the last one loads zeros and stores nothing
-    w0 = (t % p.sets_w) * 8 * NT; t /= p.sets_w;
-    h0 = (t % p.tiles_h) * kHaloTH;
-    b0 = t / p.tiles_h;
+    uint32_t q, r;
+    divmod((uint32_t)pt, (uint32_t)p.tiles_n, p.mg_tiles_n, q, r);
+    n0 = (int)r * BN;
+    const uint32_t t = 2u * q + rank;
+    const bool in_range = (int)t < p.m_sets;  // a set past the last one loads zeros and stores nothing
+    divmod(t, (uint32_t)p.sets_w, p.mg_sets_w, q, r);
+    w0 = (int)r * 8 * NT;
+    divmod(q, (uint32_t)p.tiles_h, p.mg_tiles_h, q, r);
+    h0 = (int)r * kHaloTH;
+    b0 = (int)q;
     return in_range;
   };
 
@@ -787,34 +823,21 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // Loads the A box (and raw metadata) of stage use `ia`. blocking == false: only if the
       // stage is free right now. Returns 1 issued, 0 not free, -1 wait gave up.
       auto issue_a = [&](bool blocking) -> int {
-        // fused: the box before this one must have been pruned, its second half lies in the
-        // single scratch buffer this load overwrites
-        uint64_t* pruned = &meta_full[ast ^ 1];
-        const uint32_t pruned_ph = ((uint32_t)(ia - 1) >> 1) & 1u;
         if (blocking) {
           if (!ptx::mbar_wait(&a_empty[ast], aph ^ 1u, err, 0x100u + ast)) return -1;
-          if (FUSED && ia > 0 && !ptx::mbar_wait(pruned, pruned_ph, err, 0x140u + ast)) return -1;
-        } else if (!ptx::mbar_test(&a_empty[ast], aph ^ 1u) || (FUSED && ia > 0 && !ptx::mbar_test(pruned, pruned_ph))) {
+        } else if (!ptx::mbar_test(&a_empty[ast], aph ^ 1u)) {
           return 0;
         }
         const int lt = ia / p.k_blocks, kb = ia - lt * p.k_blocks;
         int n0, w0, h0, b0;
         locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
         const int q0 = w0 + p.pad_w - (p.S - 1), p0 = h0 + p.pad_h - (p.R - 1);
-        if (FUSED) {
-          // dense dL/dO of this CTA's box: 128 channels as two halves of 64; the first half lands
-          // in the A stage itself and is compressed in place
-          ptx::mbar_arrive_expect_tx(&raw_full[ast], 2u * (uint32_t)(p.img_rows * 128));
-          ptx::tma_load_4d(sA + ast * p.a_bytes, &tmA, &raw_full[ast], kb * 128, q0, p0, b0);
-          ptx::tma_load_4d(sHalf1, &tmA, &raw_full[ast], kb * 128 + 64, q0, p0, b0);
-        } else {
-          if (rank == 0) ptx::mbar_arrive_expect_tx(&a_full[ast], a_tx);
-          if (SPARSE) {
-            ptx::mbar_arrive_expect_tx(&meta_full[ast], meta_tx);
-            ptx::tma_load_4d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, p0, b0);
-          }
-          ptx::tma_load_4d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, p0, b0);
+        if (rank == 0) ptx::mbar_arrive_expect_tx(&a_full[ast], a_tx);
+        if (SPARSE) {
+          ptx::mbar_arrive_expect_tx(&meta_full[ast], meta_tx);
+          ptx::tma_load_4d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, p0, b0);
         }
+        ptx::tma_load_4d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, p0, b0);
         ++ia;
         if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
         return 1;
@@ -827,12 +850,13 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         locate(first_pair + lt * pair_stride, n0, w0_unused, h0_unused, b0_unused);
         n0 += n_half;
         for (int kb = 0; alive && kb < p.k_blocks; ++kb, ++use) {
-          while (alive && ia <= use)
+          // (fused: the dense boxes are another warp's job, chunk by chunk; this thread streams W only)
+          while (!FUSED && alive && ia <= use)
             if (issue_a(true) < 0) alive = false;
           for (int t = 0; alive && t < taps; ++t) {
             // the next A box goes out as soon as its stage is released, between W taps
-            if (ia < a_uses && ia < use + kHaloAStages && issue_a(false) < 0) { alive = false; break; }
-            if (!ptx::mbar_wait(&w_empty[wst], wph ^ 1u, err, 0x180u + wst)) { alive = false; break; }
+            if (!FUSED && ia < a_uses && ia < use + kHaloAStages && issue_a(false) < 0) { alive = false; break; }
+            if (!ptx::mbar_wait<kIdleWaitNs>(&w_empty[wst], wph ^ 1u, err, 0x180u + wst)) { alive = false; break; }
             if (rank == 0) ptx::mbar_arrive_expect_tx(&w_ready[wst], w_tx);
             const int r = t / p.S, s = t - r * p.S;
             const int ft = (p.r_first + p.r_step * r) * p.S_full + p.s_first + p.s_step * s;
@@ -855,13 +879,18 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // descriptors as two 32-bit halves: the start address only ever changes the low word
       const uint64_t adesc0 = ptx::make_smem_desc(0, 16, (uint32_t)p.pitch * 128u, 2);
       const uint64_t bdesc0 = ptx::make_smem_desc(0, C::kBoxBytes, 8 * C::kRowB, C::kBSwizzle);
-      const uint64_t edesc0 = ptx::make_smem_desc(0, 128, 128, 0);
+      // metadata window: 16 groups of 8 consecutive 16-byte lines, one pitch of lines apart
+      const uint64_t edesc0 = ptx::make_smem_desc(0, 128, (uint32_t)p.pitch * 16u, 0);
       const uint32_t a_hi = (uint32_t)(adesc0 >> 32), b_hi = (uint32_t)(bdesc0 >> 32), e_hi = (uint32_t)(edesc0 >> 32);
       const uint32_t a_lo0 = (uint32_t)adesc0 + (ptx::smem_u32(sA) >> 4);
       const uint32_t b_lo0 = (uint32_t)bdesc0 + (ptx::smem_u32(sW) >> 4);
-      const uint32_t e_lo0 = (uint32_t)edesc0 + (ptx::smem_u32(sEhw) >> 4);
+      const uint32_t e_lo0 = (uint32_t)edesc0 + (ptx::smem_u32(sMeta) >> 4);
       const uint32_t a_stage16 = (uint32_t)p.a_bytes >> 4, w_stage16 = (uint32_t)p.w_bytes >> 4,
-                     e_stage16 = (uint32_t)p.ehw_bytes >> 4;
+                     e_stage16 = (uint32_t)p.meta_bytes >> 4, m1_off16 = (uint32_t)p.m0_bytes >> 4;
+      // first line (16-byte units) of the window of vertical tap offset dr = R-1-r: master dr % 2, pair dr / 2
+      auto meta_row16 = [&p, m1_off16](int dr) -> uint32_t {
+        return ((dr & 1) ? m1_off16 : 0u) + (uint32_t)((dr >> 1) * 2 * p.pitch);
+      };
       const uint32_t a_first16 = (uint32_t)(((p.R - 1) * p.pitch + (p.S - 1)) * 8);  // tap (0,0), in 16-byte units
       const uint32_t a_rowstep16 = (uint32_t)((p.pitch - (p.S - 1)) * 8);            // last tap of a filter row -> first of the next
       constexpr uint32_t kBStep = (uint32_t)((C::kKB / 4) * C::kRowB / 16);  // W rows of one MMA
@@ -869,8 +898,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       bool alive = true;
       int ast = 0, acc = 0, wst = 0;
       uint32_t aph = 0, wph = 0, cph = 0;
-      // running words of the W ring: W descriptor, metadata descriptor, metadata column (relative)
-      uint32_t b_lo = b_lo0, e_lo = e_lo0, mcol = 0;
+      // running words of the W ring: W descriptor, metadata column (relative)
+      uint32_t b_lo = b_lo0, mcol = 0;
       for (int lt = 0; alive && lt < my_tiles; ++lt) {
         if (!ptx::mbar_wait(&acc_empty[acc], cph ^ 1u, err, 0x200u + acc)) break;
         // shared metadata region: the first columns of the other tile set's accumulators,
@@ -886,8 +915,11 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         uint32_t accumulate = 0u;
         for (int kb = 0; alive && kb < p.k_blocks; ++kb) {
           if (!ptx::mbar_wait(&a_full[ast], aph, err, 0x300u + ast)) { alive = false; break; }
+          if (SPARSE && !FUSED && !ptx::mbar_wait(&meta_ready[ast], aph, err, 0x340u + ast)) { alive = false; break; }
           uint32_t a_lo = a_lo0 + (uint32_t)ast * a_stage16 + a_first16;
-          int s = p.S;
+          int s = p.S, dr = p.R - 1;
+          const uint32_t e_stage = e_lo0 + (uint32_t)ast * e_stage16;
+          uint32_t e_lo = e_stage + meta_row16(dr) + (uint32_t)(p.S - 1);
           for (int t = 0; t < taps; ++t) {
             if (!ptx::mbar_wait(&w_ready[wst], wph, err, 0x380u + wst)) { alive = false; break; }
             ptx::tc_fence_after_sync();
@@ -899,7 +931,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < NT; ++j)
                   if (ALL || (strips & (1u << j)))
-                    ptx::tc_cp_128x128b_pair(e_col + 4u * j, ((uint64_t)e_hi << 32) | (e_lo + (uint32_t)(j * (kEHwBytes / 16))));
+                    ptx::tc_cp_128x128b_pair(e_col + 4u * j, ((uint64_t)e_hi << 32) | (e_lo + (uint32_t)(8 * j)));
               }
 #pragma unroll
               for (int j = 0; j < NT; ++j) {
@@ -922,9 +954,10 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             ptx::tc_commit_pair(&w_empty[wst], 3);
             accumulate = 1u;
             // next tap: one pixel to the left, or the end of the filter row above
-            if (--s == 0) { s = p.S; a_lo -= a_rowstep16; } else { a_lo -= 8u; }
-            if (++wst == WS) { wst = 0; wph ^= 1u; b_lo = b_lo0; e_lo = e_lo0; mcol = 0; }
-            else { b_lo += w_stage16; e_lo += e_stage16; mcol += kSlotCols; }
+            if (--s == 0) { s = p.S; a_lo -= a_rowstep16; --dr; e_lo = e_stage + meta_row16(dr) + (uint32_t)(p.S - 1); }
+            else { a_lo -= 8u; e_lo -= 1u; }
+            if (++wst == WS) { wst = 0; wph ^= 1u; b_lo = b_lo0; mcol = 0; }
+            else { b_lo += w_stage16; mcol += kSlotCols; }
           }
           if (alive) ptx::tc_commit_pair(&a_empty[ast], 3);
           if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
@@ -933,139 +966,222 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (++acc == 2) { acc = 0; cph ^= 1u; }
       }
     }
-  } else if (warp < 6) {
-    // ------------------------------------------------- metadata rearranger
+  } else if (!FUSED && warp < 6) {
+    // ------------------------------------------------- metadata rearranger (two-pass)
+    // Once per A box the four warps turn the row-major metadata box TMA delivered into the two masters
+    // (one 16-byte line per lane and pass: two 16-byte loads, four prmt, one 16-byte store), then arrive
+    // on meta_ready. Every warp waits for every box in turn (a parity wait must see each phase).
     if (SPARSE) {
-      // A lone warp runs a dependent instruction chain slowly, so the four warps do not share
-      // one tap: warp k builds the metadata of W-ring uses k, k+G, k+2G, ... (a whole TMEM image
-      // per strip: four passes of 32 lanes), G taps in flight.
-      // lane = pixel column w, channel half, and odd/even pair of strip rows within a pass
-      const int w = lane & 7, hsub = lane >> 4;
-      const uint32_t sel = (lane & 8) ? 0x7632u : 0x5410u;
-      // No more warps than W stages take part: a warp's previous use then needed the use two
-      // ring passes back to be consumed (the MMA thread frees W stages in order), so the w_empty
-      // parity wait can never be satisfied by a stale phase. And no more warps than taps: every
-      // warp then has a tap in every A-stage use and waits for each phase of meta_full in turn
-      // (boxes may land out of request order; a warp that skipped a use could otherwise pass the
-      // wait one phase early when that use's box is late).
-      const int G = (WS < 4 ? WS : 4) < taps ? (WS < 4 ? WS : 4) : taps;
-      const int total_uses = (warp - 2 < G) ? my_tiles * p.k_blocks * taps : 0;
-      int t = warp - 2;  // tap within the channel block
-      int ause = 0;      // A stage use = (tile set, channel block)
-      while (t >= taps) { t -= taps; ++ause; }
-      int wst = warp - 2;
-      uint32_t wph = 0;
-      for (int u = warp - 2; u < total_uses; u += G) {
+      const int mw = warp - 2;
+      const int lines0 = p.pairs0 * 2 * p.pitch, lines = (p.pairs0 + p.pairs1) * 2 * p.pitch;
+      const int a_uses = my_tiles * p.k_blocks;
+      constexpr int kBatch = 3;  // lines per lane whose loads are issued before any store
+      for (int ause = 0; ause < a_uses; ++ause) {
         const int ast = ause & 1;  // kHaloAStages == 2
         if (!ptx::mbar_wait(&meta_full[ast], (uint32_t)(ause >> 1) & 1u, err, 0x500u + ast)) break;
-        // the stage's previous tiles have been copied to TMEM and used
-        if (!ptx::mbar_wait(&w_empty[wst], wph ^ 1u, err, 0x580u + wst)) break;
-        const int r = t / p.S, s = t - r * p.S;
-        const uint32_t strips = strip_mask(ause / p.k_blocks);
         const uint8_t* raw = sEraw + ast * p.eraw_bytes;
-        uint8_t* dst = sEhw + wst * p.ehw_bytes + lane * 16;
-        // TMEM lane 32*i + lane holds strip rows 2*h2 and 2*h2 + 1 with h2 = 2*i + hsub.
-        // All loads first, then all stores: the compiler cannot tell that the two shared-memory
-        // regions differ and would otherwise serialise load - store - load.
-        const int px0 = (2 * hsub + (p.R - 1 - r)) * p.pitch + w + (p.S - 1 - s);
-        uint4 lo[4 * NT], hi[4 * NT];
+        uint8_t* master = sMeta + ast * p.meta_bytes;
+        for (int first = mw * 32 + lane; first < lines; first += 128 * kBatch) {
+          uint4 lo[kBatch], hi[kBatch];
+          uint32_t sel[kBatch];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-#pragma unroll
-          for (int j = 0; j < NT; ++j) {
-            const int px = px0 + 4 * i * p.pitch + 8 * j;
-            lo[i * NT + j] = *(const uint4*)(raw + px * 16);
-            hi[i * NT + j] = *(const uint4*)(raw + (px + p.pitch) * 16);
+          for (int k = 0; k < kBatch; ++k) {
+            const int L = first + 128 * k;
+            if (L < lines) {
+              const int pi = L >= lines0 ? 1 : 0;
+              const int l = L - pi * lines0;
+              const int m2e = (int)(((uint32_t)l * p.pitch_magic) >> 20), x = l - m2e * p.pitch;  // 2m + e, pixel column
+              const int row_a = (pi + (m2e & ~1)) * p.pitch + x;  // box pixel (pi + 2m, x); its partner is one box row down
+              lo[k] = *(const uint4*)(raw + row_a * 16);
+              hi[k] = *(const uint4*)(raw + (row_a + p.pitch) * 16);
+              sel[k] = (m2e & 1) ? 0x7632u : 0x5410u;
+            }
           }
-        }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-#pragma unroll
-          for (int j = 0; j < NT; ++j) {
-            if (!(strips & (1u << j))) continue;  // strip not part of this unit: its image is never read
-            const uint4 a = lo[i * NT + j], b = hi[i * NT + j];
-            *(uint4*)(dst + j * kEHwBytes + i * 512) =
-                make_uint4(well_formed(prmt(a.x, b.x, sel)), well_formed(prmt(a.y, b.y, sel)),
-                           well_formed(prmt(a.z, b.z, sel)), well_formed(prmt(a.w, b.w, sel)));
+          for (int k = 0; k < kBatch; ++k) {
+            const int L = first + 128 * k;
+            if (L < lines)
+              *(uint4*)(master + L * 16) =
+                  make_uint4(well_formed(prmt(lo[k].x, hi[k].x, sel[k])), well_formed(prmt(lo[k].y, hi[k].y, sel[k])),
+                             well_formed(prmt(lo[k].z, hi[k].z, sel[k])), well_formed(prmt(lo[k].w, hi[k].w, sel[k])));
           }
         }
         ptx::fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive_cluster(&w_ready[wst], 0);
-        t += G;
-        while (t >= taps) { t -= taps; ++ause; }
-        wst += G;
-        while (wst >= WS) { wst -= WS; wph ^= 1u; }
+        if (lane == 0) ptx::mbar_arrive_cluster(&meta_ready[ast], 0);
       }
     }
-  } else if (FUSED && warp >= 10) {
+  } else if (FUSED && (warp & 3) != 1 && (warp < 4 || warp >= 8)) {
     // ------------------------------------------------------------ pruner
-    // The dense box is pruned quarter row by quarter row (32 channels per item, items dealt to
-    // the pruning threads round-robin: a round covers whole pixel rows). Within a round every
-    // thread reads its input, all wait, then every thread writes: the compressed row replaces
-    // the first dense half in place.
-    const int tid = threadIdx.x - kThreadsGemm;  // 0 .. 32 * kPruneWarps - 1
-    constexpr int kPruners = 32 * kPruneWarps;
-    const int items = p.img_rows * 4;
-    const int rounds = (items + kPruners - 1) / kPruners;
-    const int a_uses = my_tiles * p.k_blocks;
-    int lt = 0, kb = 0;
-    for (int ia = 0; ia < a_uses; ++ia) {
-      const int ast = ia & 1;  // kHaloAStages == 2
-      // all pruning threads stay or leave together: they meet at named barriers below
-      if (!ptx::named_bar_all(3, kPruners, ptx::mbar_wait(&raw_full[ast], ((uint32_t)ia >> 1) & 1u, err, 0x900u + ast)))
-        break;
-      int n0, w0, h0, b0;
-      locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
-      const int q0 = w0 + p.pad_w - (p.S - 1), p0 = h0 + p.pad_h - (p.R - 1);
-      uint8_t* a_tile = sA + ast * p.a_bytes;
-      uint8_t* meta_rows = sEraw + ast * p.eraw_bytes;
-      for (int rd = 0; rd < rounds; ++rd) {
-        const int item = rd * kPruners + tid;
-        const int i = item >> 2, c = item & 3;  // pixel row of the box, quarter
-        const bool active = item < items;
-        uint2 out[4];
-        uint32_t metaw = 0u;
-        if (active) {
-          const int ih = i / p.pitch, iw = i - ih * p.pitch;
-          const int64_t pixel = ((int64_t)b0 * p.P + (p0 + ih)) * p.Q + (q0 + iw);  // any value when outside the image
-          const int64_t vbase = pixel * (p.Cout >> 3) + kb * 16;
-          const uint8_t* half = (c < 2) ? a_tile : sHalf1;
-#define SDGP_FUSED_Q(NN, SS) fused_prune_quarter<NN, SS>(half, i, c, vbase, p.seed_lo, p.seed_hi, out, metaw)
-          if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_Q(1, SDGP_MAGNITUDE); else SDGP_FUSED_Q(2, SDGP_MAGNITUDE); }
-          else if (p.fused_scheme == SDGP_RANDOM) { if (p.fused_n == 1) SDGP_FUSED_Q(1, SDGP_RANDOM); else SDGP_FUSED_Q(2, SDGP_RANDOM); }
-          else { if (p.fused_n == 1) SDGP_FUSED_Q(1, SDGP_RESCALED_MAGNITUDE); else SDGP_FUSED_Q(2, SDGP_RESCALED_MAGNITUDE); }
-#undef SDGP_FUSED_Q
+    // Work unit = 8 pixel rows of a box = one pass of a warp: lane = (row, c), and the thread owns vectors
+    // c, c + 4, c + 8 and c + 12 (8 channels each) of the row's 16, so that every load instruction of the
+    // warp reads 64 contiguous bytes per pixel. Units are numbered through all boxes of this CTA and dealt
+    // round-robin to the pruning warps. A thread reads its 64 bytes of dense dL/dO straight from global
+    // memory into registers (the loads of the next unit go out as soon as this one is pruned, and the lines
+    // of the next box are asked into L2 a box ahead), prunes them and writes the compressed vectors and their
+    // metadata into the A stage. These stores replace the TMA write of the compressed box, so the fused mode adds no
+    // shared-memory traffic to the two-pass kernel's - which matters because with 64 or 128 input
+    // channels the MMAs themselves are bound by shared-memory reads.
+    {
+      // number of this pruning warp, 0 .. kPruneWarps - 1: warps 2, 3, 8, then 10.. without those on scheduler 1
+      const int pw = warp < 4 ? warp - 2 : warp == 8 ? 2 : 3 + (warp - 10) - ((warp - 9) >> 2);
+      const int upb = (p.img_rows + 7) >> 3;  // units per box
+      const int a_uses = my_tiles * p.k_blocks;
+      const int row8 = lane >> 2, c = lane & 3;
+      const uint32_t px_bytes = (uint32_t)p.Cout * 2u;
+      auto prune_units = [&](auto n_tag, auto scheme_tag) {
+        constexpr int N = decltype(n_tag)::value;
+        constexpr int SCHEME = decltype(scheme_tag)::value;
+        // ---- load cursor: the unit whose loads go out next, and the box it lies in
+        int ia = 0, o = pw, lt = 0, kb = 0;
+        auto normalise = [&]() { while (o >= upb) { o -= upb; ++ia; if (++kb == p.k_blocks) { kb = 0; ++lt; } } };
+        normalise();
+        int org_box = -1;             // box the origin below belongs to
+        const uint8_t* org_ptr = p.a_dense;  // address of box pixel (0, 0), channel block kb, quarter c (may lie outside the tensor)
+        int org_p = 0, org_q = 0;     // dO pixel of box pixel (0, 0)
+        int64_t org_pix = 0;          // its linear pixel number (random keys)
+        bool org_ok = false;
+        auto set_origin = [&](int box_lt, int box_kb, const uint8_t*& ptr, int& p0, int& q0, int64_t& pix, bool& ok) {
+          int n0, w0, h0, b0;
+          ok = locate(first_pair + box_lt * pair_stride, n0, w0, h0, b0);
+          q0 = w0 + p.pad_w - (p.S - 1);
+          p0 = h0 + p.pad_h - (p.R - 1);
+          pix = ((int64_t)b0 * p.P + p0) * p.Q + q0;
+          ptr = p.a_dense + pix * (int64_t)px_bytes + box_kb * 256 + c * 16;
+        };
+        // The unit whose loads are in flight: its 64 bytes, its pixel row in the box, its box
+        uint4 w[4];
+        int u_i = 0, u_ia = 0, u_kb = 0;
+        int64_t u_pix = 0;
+        auto fetch = [&]() {
+          if (org_box != ia) {
+            set_origin(lt, kb, org_ptr, org_p, org_q, org_pix, org_ok);
+            org_box = ia;
+            // ask the lines of the NEXT box into L2 now, a whole box ahead of their loads: 2 lines of 128
+            // bytes per box pixel, dealt to the pruning threads
+            int nlt = lt, nkb = kb + 1;
+            if (nkb == p.k_blocks) { nkb = 0; ++nlt; }
+            if (ia + 1 < a_uses) {
+              const uint8_t* nptr;
+              int np0, nq0;
+              int64_t npix;
+              bool nok;
+              set_origin(nlt, nkb, nptr, np0, nq0, npix, nok);
+              for (int line = pw * 32 + lane; line < 2 * p.img_rows; line += 32 * kPruneWarps) {
+                const int px = line >> 1;
+                const int ih = (int)(((uint32_t)px * p.pitch_magic) >> 20), iw = px - ih * p.pitch;
+                if (nok && (unsigned)(np0 + ih) < (unsigned)p.P && (unsigned)(nq0 + iw) < (unsigned)p.Q)
+                  asm volatile("prefetch.global.L2 [%0];" ::"l"(nptr - c * 16 + (uint32_t)(ih * p.Q + iw) * px_bytes + (line & 1) * 128));
+              }
+            }
+          }
+          u_i = 8 * o + row8;
+          u_ia = ia;
+          u_kb = kb;
+          const int ih = (int)(((uint32_t)u_i * p.pitch_magic) >> 20), iw = u_i - ih * p.pitch;
+          const uint32_t off = (uint32_t)(ih * p.Q + iw);
+          u_pix = org_pix + off;
+          const bool valid = org_ok && u_i < p.img_rows && (unsigned)(org_p + ih) < (unsigned)p.P &&
+                             (unsigned)(org_q + iw) < (unsigned)p.Q;
+#pragma unroll
+          for (int v = 0; v < 4; ++v) w[v] = make_uint4(0u, 0u, 0u, 0u);
+          if (valid) {
+            const uint8_t* src = org_ptr + off * px_bytes;
+            // vector c + 4v: channels beyond Cout (a last channel block that is half empty) read as zero
+            const int chan0 = kb * 128 + c * 8;
+#pragma unroll
+            for (int v = 0; v < 4; ++v)
+              if (chan0 + 32 * v < p.Cout) w[v] = ldg_stream(src + 64 * v);
+          }
+          o += kPruneWarps;
+          normalise();
+        };
+        int boxes_seen = 0;  // stage hand-backs (a_empty phases) this warp has observed, one per box, in order
+        int pending_ast = -1;  // stage of the unit whose stores are out but not yet announced
+        // Makes the stores of the previous unit visible to the tensor core and announces them. Called a whole
+        // unit later than the stores were issued, so the fence finds them done.
+        auto announce = [&]() {
+          if (pending_ast >= 0) {
+            ptx::fence_proxy_async_smem();  // the tensor core reads A and the masters through the async proxy
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(&a_full[pending_ast], 0);
+          }
+        };
+        bool more = ia < a_uses;  // a unit is in flight
+        if (more) fetch();
+        while (more) {
+          const int i = u_i, cia = u_ia;
+          if (boxes_seen <= cia) {  // the MMAs that read this stage's previous contents (box cia - 2) have completed
+            bool ok = true;
+            while (boxes_seen <= cia) {
+              if (!ptx::mbar_wait<kIdleWaitNs>(&a_empty[boxes_seen & 1], (((uint32_t)boxes_seen >> 1) & 1u) ^ 1u, err, 0x900u + (boxes_seen & 1))) { ok = false; break; }
+              ++boxes_seen;
+            }
+            if (!__all_sync(0xFFFFFFFFu, ok)) break;
+          }
+          const int ast = cia & 1;
+          uint2 out[4];
+          uint32_t metaw;
+          fused_prune_vectors<N, SCHEME>(w, u_pix * (p.Cout >> 3) + u_kb * 16 + c, 4, p.seed_lo, p.seed_hi, out, metaw);
+          // the registers of this unit are free: the loads of the next one go out before this one's stores
+          more = ia < a_uses;
+          if (more) fetch();
+          announce();
+          const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, metaw, 1);  // (all lanes: before the rows part ways)
+          if (i < p.img_rows) {
+            const int sw = i & 7;
+            // vector j = c + 4v -> 8 bytes at 16-byte chunk j / 2 = 2v + c / 2 (swizzled), half j % 2 = c % 2
+            uint8_t* a_row = sA + ast * p.a_bytes + i * 128 + 8 * (c & 1);
+            const int ch0 = (c >> 1) ^ sw;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) *(uint2*)(a_row + ((ch0 ^ (2 * v)) << 4)) = out[v];
+            // Metadata: byte v of metaw belongs to the 16-channel group 2v + c / 2, i.e. to 32-bit word v of the
+            // master line e = c / 2, byte c % 2 of its low or high half-word. Lanes c and c ^ 1 hold the two bytes
+            // of each half-word: they trade words, the even lane writes the half-words of v = 0, 1, the odd one
+            // those of v = 2, 3.
+            const uint32_t lo = (c & 1) ? other : metaw, hi = (c & 1) ? metaw : other;  // bytes of c even / c odd
+            const uint32_t pair = (c & 1) ? prmt(lo, hi, 0x7362) : prmt(lo, hi, 0x5140);  // two half-words
+            const int ih = (int)(((uint32_t)i * p.pitch_magic) >> 20), iw = i - ih * p.pitch;
+            uint8_t* master = sMeta + ast * p.meta_bytes + (iw << 4) + 8 * (c & 1) + (c >> 1) * (p.pitch << 4);
+            if (ih < 2 * p.pairs0) {
+              uint8_t* dst = master + (((ih & ~1) * p.pitch) << 4) + 2 * (ih & 1);
+              *(uint16_t*)dst = (uint16_t)pair;
+              *(uint16_t*)(dst + 4) = (uint16_t)(pair >> 16);
+            }
+            if (ih >= 1 && ih <= 2 * p.pairs1) {
+              uint8_t* dst = master + p.m0_bytes + ((((ih - 1) & ~1) * p.pitch) << 4) + 2 * ((ih - 1) & 1);
+              *(uint16_t*)dst = (uint16_t)pair;
+              *(uint16_t*)(dst + 4) = (uint16_t)(pair >> 16);
+            }
+          }
+          pending_ast = ast;
         }
-        ptx::named_bar_sync(3, kPruners);  // the round's inputs are in registers
-        if (active) {
-          const int sw = i & 7;
-          // vectors 4c .. 4c+3 of the row -> 8 bytes each at chunk (j >> 1), half (j & 1)
-          *(uint4*)(a_tile + i * 128 + (((2 * c) ^ sw) << 4)) = make_uint4(out[0].x, out[0].y, out[1].x, out[1].y);
-          *(uint4*)(a_tile + i * 128 + (((2 * c + 1) ^ sw) << 4)) = make_uint4(out[2].x, out[2].y, out[3].x, out[3].y);
-          *(uint32_t*)(meta_rows + i * 16 + 4 * c) = metaw;
-        }
+        announce();
+      };
+      using std::integral_constant;
+      if (p.fused_scheme == SDGP_MAGNITUDE) {
+        if (p.fused_n == 1) prune_units(integral_constant<int, 1>{}, integral_constant<int, SDGP_MAGNITUDE>{});
+        else prune_units(integral_constant<int, 2>{}, integral_constant<int, SDGP_MAGNITUDE>{});
+      } else if (p.fused_scheme == SDGP_RANDOM) {
+        if (p.fused_n == 1) prune_units(integral_constant<int, 1>{}, integral_constant<int, SDGP_RANDOM>{});
+        else prune_units(integral_constant<int, 2>{}, integral_constant<int, SDGP_RANDOM>{});
+      } else {
+        if (p.fused_n == 1) prune_units(integral_constant<int, 1>{}, integral_constant<int, SDGP_RESCALED_MAGNITUDE>{});
+        else prune_units(integral_constant<int, 2>{}, integral_constant<int, SDGP_RESCALED_MAGNITUDE>{});
       }
-      ptx::fence_proxy_async_smem();  // the tensor core reads A through the async proxy
-      __syncwarp();
-      if (lane == 0) {
-        ptx::mbar_arrive(&meta_full[ast]);
-        ptx::mbar_arrive_cluster(&a_full[ast], 0);
-      }
-      if (++kb == p.k_blocks) { kb = 0; ++lt; }
     }
-  } else {
+  } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + 4) {
     // ------------------------------------------------------------ epilogue
     const int q = warp & 3;
     const int row = q * 32 + lane;
-    const bool issuer = (threadIdx.x == 192);
+    const bool issuer = (threadIdx.x == kEpilogueWarp0 * 32);
     uint32_t chunk = 0, cph = 0;
     int acc = 0;
     for (int lt = 0; lt < my_tiles; ++lt) {
       int n0, w0, h0, b0;
       const bool in_range = locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
       const uint32_t strips = strip_mask(lt);
-      if (!ptx::mbar_wait(&acc_full[acc], cph, err, 0x600u + acc)) break;
+      if (!ptx::mbar_wait<kIdleWaitNs>(&acc_full[acc], cph, err, 0x600u + acc)) break;
       ptx::tc_fence_after_sync();
 #pragma unroll
       for (int j = 0; j < NT; ++j)
@@ -1347,16 +1463,18 @@ bool plan_halo(HaloParams* p, int nt) {
     p->img_rows = p->pitch * p->img_h;
     if (p->pitch > 256 || p->img_h > 256) return false;
     p->a_bytes = round_up(p->img_rows * 128, 1024);
-    p->eraw_bytes = SPARSE ? round_up(p->img_rows * 16, 128) : 0;
+    p->eraw_bytes = (SPARSE && !FUSED) ? round_up(p->img_rows * 16, 128) : 0;
     p->w_bytes = C::kTapBBytes;
-    p->ehw_bytes = SPARSE ? nt * kEHwBytes : 0;
-    const int half1_bytes = FUSED ? p->a_bytes : 0;  // scratch for the second dense half
-    const int fixed = kHaloAStages * (p->a_bytes + p->eraw_bytes) + half1_bytes + 1024;
+    p->pairs0 = 8 + ((p->R - 1) >> 1);
+    p->pairs1 = p->R > 1 ? 8 + ((p->R - 2) >> 1) : 0;
+    p->m0_bytes = SPARSE ? p->pairs0 * 2 * p->pitch * 16 : 0;
+    p->meta_bytes = SPARSE ? round_up((p->pairs0 + p->pairs1) * 2 * p->pitch * 16, 128) : 0;
+    const int fixed = kHaloAStages * (p->a_bytes + p->eraw_bytes + p->meta_bytes) + 1024;
     int out_bufs = 2;
-    int w_stages = (budget - fixed - out_bufs * kOutBytes) / (p->w_bytes + p->ehw_bytes);
+    int w_stages = (budget - fixed - out_bufs * kOutBytes) / p->w_bytes;
     if (w_stages < 4) {
       out_bufs = 1;
-      w_stages = (budget - fixed - out_bufs * kOutBytes) / (p->w_bytes + p->ehw_bytes);
+      w_stages = (budget - fixed - out_bufs * kOutBytes) / p->w_bytes;
     }
     if (w_stages > kMaxStages) w_stages = kMaxStages;
     p->meta_shared = 0;
@@ -1376,10 +1494,10 @@ bool plan_halo(HaloParams* p, int nt) {
     p->w_stages = w_stages;
     p->out_bufs = out_bufs;
     p->off_eraw = kHaloAStages * p->a_bytes;
-    p->off_half1 = round_up(p->off_eraw + kHaloAStages * p->eraw_bytes, 1024);
-    p->off_w = p->off_half1 + half1_bytes;
-    p->off_ehw = p->off_w + w_stages * p->w_bytes;
-    p->off_out = round_up(p->off_ehw + w_stages * p->ehw_bytes, 1024);
+    p->off_meta = p->off_eraw + kHaloAStages * p->eraw_bytes;
+    p->off_w = round_up(p->off_meta + kHaloAStages * p->meta_bytes, 1024);
+    p->pitch_magic = ((1u << 20) + (uint32_t)p->pitch - 1u) / (uint32_t)p->pitch;
+    p->off_out = round_up(p->off_w + w_stages * p->w_bytes, 1024);
     p->off_bar = p->off_out + out_bufs * kOutBytes;
     p->smem_bytes = p->off_bar + 512 + 1024;
     if (p->smem_bytes > kSmemLimit) return false;
@@ -1389,6 +1507,9 @@ bool plan_halo(HaloParams* p, int nt) {
     if (m_sets * p->tiles_n > 0x3FFFFFFF) return false;
     p->m_sets = (int)m_sets;
     p->pair_tiles = (int)((m_sets + 1) / 2) * p->tiles_n;
+    p->mg_tiles_n = div_magic((uint32_t)p->tiles_n);
+    p->mg_sets_w = div_magic((uint32_t)p->sets_w);
+    p->mg_tiles_h = div_magic((uint32_t)p->tiles_h);
     // The pair tiles of a last round that fills at most half the CTA pairs are dealt out strip by
     // strip: that round then costs about half.
     p->units = p->pair_tiles;
@@ -1424,9 +1545,12 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
   {
     const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
     const uint64_t strides[3] = {CA * 2, CA * 2 * Q, CA * 2 * Q * P};
+    // (fused: the pruning warps read dL/dO with plain loads and this map goes unused)
     const uint32_t box[4] = {64, (uint32_t)p.pitch, (uint32_t)p.img_h, 1};
     if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
+    tmE = tmA;
+    p.a_dense = (const uint8_t*)A;
   }
   if (SPARSE && !FUSED) {
     const uint64_t CE = (uint64_t)view.a_channels / 16;
@@ -1435,8 +1559,6 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
     const uint32_t box[4] = {8, (uint32_t)p.pitch, (uint32_t)p.img_h, 1};
     if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
       return SDGP_ERR_CUDA;
-  } else {
-    tmE = tmA;
   }
   {
     const uint64_t dims[2] = {(uint64_t)view.w_cols, (uint64_t)p.Cout};

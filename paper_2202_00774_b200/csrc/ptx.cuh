@@ -71,15 +71,20 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 
 // Bounded wait: gives up after ~2 s of wall time (or as soon as another wait has given up),
 // records `code` in *error_word and returns false; the caller carries on, so the kernel
-// always terminates.
+// always terminates. SLEEP_NS > 0: the waiter sleeps that long between polls - for roles whose wake-up
+// may come a fraction of a microsecond late (epilogue, loaders, pruning warps) and whose polling would
+// otherwise take issue slots from the warps that share their scheduler.
+template <unsigned SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* error_word,
                                           unsigned int code, uint64_t limit_ns = 2000000000ull) {
   if (mbar_test(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 256; ++i)
+    for (int i = 0; i < 256; ++i) {
+      if (SLEEP_NS) __nanosleep(SLEEP_NS);
       if (mbar_test(bar, parity)) return true;
+    }
     // once any wait of any CTA has given up, no other wait lingers
     if (*(volatile unsigned int*)error_word != 0u) return false;
     if (globaltimer_ns() - t0 > limit_ns) {
