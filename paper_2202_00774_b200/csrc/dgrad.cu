@@ -623,7 +623,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 // rearranged metadata tiles of that tap). Roles as in dgrad_kernel; the metadata warps build one
 // 2 KB TMEM image per (tap, strip) from the raw metadata box of the A stage.
 
-constexpr int kHaloTH = 16;  // pixel rows of a strip: 8 x 16 pixels = the 128 rows of an accumulator
+constexpr int kHaloRows = 16;  // 8-pixel rows of a strip: the 128 rows of an accumulator
 constexpr int kHaloAStages = 2;
 // Warp roles of the fused whole-filter-reuse kernel (24 warps: registers are granted to warps in fours, and
 // 24 x 80 registers is what fits). Warp w runs on scheduler w % 4, and the thread that issues the MMAs
@@ -657,7 +657,10 @@ struct HaloParams {
   int split_from;          // units >= split_from cover one strip of a pair tile each (quantisation of the last round)
   int k_blocks;
   int pitch;               // pixel columns of the A box: 8 * nt + S - 1
-  int img_h;               // pixel rows of the A box: kHaloTH + R - 1
+  int th, tb;              // a strip is 8 pixels wide and covers th pixel rows of tb images, th * tb = 16: 16 x 1, or 8 x 2
+                           // for images at most 8 pixels tall. Its 16 rows are ordered (pixel row, image), so a vertical
+                           // tap is still one uniform row offset (tb rows).
+  int img_h;               // rows of the A box: (th + R - 1) * tb, ordered (pixel row, image)
   int img_rows;            // pitch * img_h
   int w_stages;
   int meta_col, meta_shared, out_bufs;
@@ -806,8 +809,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     divmod(t, (uint32_t)p.sets_w, p.mg_sets_w, q, r);
     w0 = (int)r * 8 * NT;
     divmod(q, (uint32_t)p.tiles_h, p.mg_tiles_h, q, r);
-    h0 = (int)r * kHaloTH;
-    b0 = (int)q;
+    h0 = (int)r * p.th;
+    b0 = (int)q * p.tb;
     return in_range;
   };
 
@@ -835,9 +838,9 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (rank == 0) ptx::mbar_arrive_expect_tx(&a_full[ast], a_tx);
         if (SPARSE) {
           ptx::mbar_arrive_expect_tx(&meta_full[ast], meta_tx);
-          ptx::tma_load_4d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, p0, b0);
+          ptx::tma_load_4d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, b0, p0);
         }
-        ptx::tma_load_4d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, p0, b0);
+        ptx::tma_load_4d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, b0, p0);
         ++ia;
         if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
         return 1;
@@ -889,10 +892,11 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                      e_stage16 = (uint32_t)p.meta_bytes >> 4, m1_off16 = (uint32_t)p.m0_bytes >> 4;
       // first line (16-byte units) of the window of vertical tap offset dr = R-1-r: master dr % 2, pair dr / 2
       auto meta_row16 = [&p, m1_off16](int dr) -> uint32_t {
-        return ((dr & 1) ? m1_off16 : 0u) + (uint32_t)((dr >> 1) * 2 * p.pitch);
+        const int off = dr * p.tb;  // box rows
+        return ((off & 1) ? m1_off16 : 0u) + (uint32_t)((off >> 1) * 2 * p.pitch);
       };
-      const uint32_t a_first16 = (uint32_t)(((p.R - 1) * p.pitch + (p.S - 1)) * 8);  // tap (0,0), in 16-byte units
-      const uint32_t a_rowstep16 = (uint32_t)((p.pitch - (p.S - 1)) * 8);            // last tap of a filter row -> first of the next
+      const uint32_t a_first16 = (uint32_t)(((p.R - 1) * p.tb * p.pitch + (p.S - 1)) * 8);  // tap (0,0), in 16-byte units
+      const uint32_t a_rowstep16 = (uint32_t)((p.tb * p.pitch - (p.S - 1)) * 8);            // last tap of a filter row -> first of the next
       constexpr uint32_t kBStep = (uint32_t)((C::kKB / 4) * C::kRowB / 16);  // W rows of one MMA
       constexpr uint32_t kSlotCols = 4u * NT;                                // metadata columns of one W stage
       bool alive = true;
@@ -1029,6 +1033,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int a_uses = my_tiles * p.k_blocks;
       const int row8 = lane >> 2, c = lane & 3;
       const uint32_t px_bytes = (uint32_t)p.Cout * 2u;
+      const int tb_shift = p.tb >> 1;  // tb is 1 or 2
       auto prune_units = [&](auto n_tag, auto scheme_tag) {
         constexpr int N = decltype(n_tag)::value;
         constexpr int SCHEME = decltype(scheme_tag)::value;
@@ -1039,10 +1044,11 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int org_box = -1;             // box the origin below belongs to
         const uint8_t* org_ptr = p.a_dense;  // address of box pixel (0, 0), channel block kb, quarter c (may lie outside the tensor)
         int org_p = 0, org_q = 0;     // dO pixel of box pixel (0, 0)
+        int org_b = 0;                // its image
         int64_t org_pix = 0;          // its linear pixel number (random keys)
         bool org_ok = false;
-        auto set_origin = [&](int box_lt, int box_kb, const uint8_t*& ptr, int& p0, int& q0, int64_t& pix, bool& ok) {
-          int n0, w0, h0, b0;
+        auto set_origin = [&](int box_lt, int box_kb, const uint8_t*& ptr, int& p0, int& q0, int& b0, int64_t& pix, bool& ok) {
+          int n0, w0, h0;
           ok = locate(first_pair + box_lt * pair_stride, n0, w0, h0, b0);
           q0 = w0 + p.pad_w - (p.S - 1);
           p0 = h0 + p.pad_h - (p.R - 1);
@@ -1055,7 +1061,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int64_t u_pix = 0;
         auto fetch = [&]() {
           if (org_box != ia) {
-            set_origin(lt, kb, org_ptr, org_p, org_q, org_pix, org_ok);
+            set_origin(lt, kb, org_ptr, org_p, org_q, org_b, org_pix, org_ok);
             org_box = ia;
             // ask the lines of the NEXT box into L2 now, a whole box ahead of their loads: 2 lines of 128
             // bytes per box pixel, dealt to the pruning threads
@@ -1063,25 +1069,27 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (nkb == p.k_blocks) { nkb = 0; ++nlt; }
             if (ia + 1 < a_uses) {
               const uint8_t* nptr;
-              int np0, nq0;
+              int np0, nq0, nb0;
               int64_t npix;
               bool nok;
-              set_origin(nlt, nkb, nptr, np0, nq0, npix, nok);
+              set_origin(nlt, nkb, nptr, np0, nq0, nb0, npix, nok);
               for (int line = pw * 32 + lane; line < 2 * p.img_rows; line += 32 * kPruneWarps) {
                 const int px = line >> 1;
-                const int ih = (int)(((uint32_t)px * p.pitch_magic) >> 20), iw = px - ih * p.pitch;
-                if (nok && (unsigned)(np0 + ih) < (unsigned)p.P && (unsigned)(nq0 + iw) < (unsigned)p.Q)
-                  asm volatile("prefetch.global.L2 [%0];" ::"l"(nptr - c * 16 + (uint32_t)(ih * p.Q + iw) * px_bytes + (line & 1) * 128));
+                const int br = (int)(((uint32_t)px * p.pitch_magic) >> 20), iw = px - br * p.pitch;  // box row, column
+                const int ih = br >> tb_shift, ib = br & (p.tb - 1);                                 // pixel row, image
+                if (nok && nb0 + ib < p.B && (unsigned)(np0 + ih) < (unsigned)p.P && (unsigned)(nq0 + iw) < (unsigned)p.Q)
+                  asm volatile("prefetch.global.L2 [%0];" ::"l"(nptr - c * 16 + (uint32_t)((ib * p.P + ih) * p.Q + iw) * px_bytes + (line & 1) * 128));
               }
             }
           }
           u_i = 8 * o + row8;
           u_ia = ia;
           u_kb = kb;
-          const int ih = (int)(((uint32_t)u_i * p.pitch_magic) >> 20), iw = u_i - ih * p.pitch;
-          const uint32_t off = (uint32_t)(ih * p.Q + iw);
+          const int br = (int)(((uint32_t)u_i * p.pitch_magic) >> 20), iw = u_i - br * p.pitch;  // box row, column
+          const int ih = br >> tb_shift, ib = br & (p.tb - 1);                                   // pixel row, image
+          const uint32_t off = (uint32_t)((ib * p.P + ih) * p.Q + iw);
           u_pix = org_pix + off;
-          const bool valid = org_ok && u_i < p.img_rows && (unsigned)(org_p + ih) < (unsigned)p.P &&
+          const bool valid = org_ok && u_i < p.img_rows && org_b + ib < p.B && (unsigned)(org_p + ih) < (unsigned)p.P &&
                              (unsigned)(org_q + iw) < (unsigned)p.Q;
 #pragma unroll
           for (int v = 0; v < 4; ++v) w[v] = make_uint4(0u, 0u, 0u, 0u);
@@ -1141,7 +1149,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             // those of v = 2, 3.
             const uint32_t lo = (c & 1) ? other : metaw, hi = (c & 1) ? metaw : other;  // bytes of c even / c odd
             const uint32_t pair = (c & 1) ? prmt(lo, hi, 0x7362) : prmt(lo, hi, 0x5140);  // two half-words
-            const int ih = (int)(((uint32_t)i * p.pitch_magic) >> 20), iw = i - ih * p.pitch;
+            const int ih = (int)(((uint32_t)i * p.pitch_magic) >> 20), iw = i - ih * p.pitch;  // ih: box row
             uint8_t* master = sMeta + ast * p.meta_bytes + (iw << 4) + 8 * (c & 1) + (c >> 1) * (p.pitch << 4);
             if (ih < 2 * p.pairs0) {
               uint8_t* dst = master + (((ih & ~1) * p.pitch) << 4) + 2 * (ih & 1);
@@ -1186,7 +1194,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
       for (int j = 0; j < NT; ++j)
         store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * set_cols + j * BN), sOut,
-                              p.out_bufs, &tmD, n0, w0 + 8 * j, h0, b0, in_range && (w0 + 8 * j < p.W) && (strips & (1u << j)), row,
+                              p.out_bufs, &tmD, n0, w0 + 8 * j, b0, h0, in_range && (w0 + 8 * j < p.W) && (strips & (1u << j)), row,
                               issuer,
                               chunk, (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr, p.f16 != 0);
       ptx::tc_fence_before_sync();
@@ -1459,14 +1467,17 @@ bool plan_halo(HaloParams* p, int nt) {
     if (nt == 2 && p->W <= 8) return false;  // a second strip would be empty
     p->nt = nt;
     p->pitch = 8 * nt + p->S - 1;
-    p->img_h = kHaloTH + p->R - 1;
+    p->th = p->H <= 8 ? 8 : kHaloRows;
+    p->tb = kHaloRows / p->th;
+    p->img_h = (p->th + p->R - 1) * p->tb;
     p->img_rows = p->pitch * p->img_h;
     if (p->pitch > 256 || p->img_h > 256) return false;
     p->a_bytes = round_up(p->img_rows * 128, 1024);
     p->eraw_bytes = (SPARSE && !FUSED) ? round_up(p->img_rows * 16, 128) : 0;
     p->w_bytes = C::kTapBBytes;
-    p->pairs0 = 8 + ((p->R - 1) >> 1);
-    p->pairs1 = p->R > 1 ? 8 + ((p->R - 2) >> 1) : 0;
+    // vertical tap offset dr = 0 .. R-1 starts tb * dr box rows down: master (tb * dr) % 2, pair (tb * dr) / 2
+    p->pairs0 = 8 + (p->tb == 2 ? p->R - 1 : (p->R - 1) >> 1);
+    p->pairs1 = (p->tb == 1 && p->R > 1) ? 8 + ((p->R - 2) >> 1) : 0;
     p->m0_bytes = SPARSE ? p->pairs0 * 2 * p->pitch * 16 : 0;
     p->meta_bytes = SPARSE ? round_up((p->pairs0 + p->pairs1) * 2 * p->pitch * 16, 128) : 0;
     const int fixed = kHaloAStages * (p->a_bytes + p->eraw_bytes + p->meta_bytes) + 1024;
@@ -1502,8 +1513,8 @@ bool plan_halo(HaloParams* p, int nt) {
     p->smem_bytes = p->off_bar + 512 + 1024;
     if (p->smem_bytes > kSmemLimit) return false;
     p->sets_w = (p->W + 8 * nt - 1) / (8 * nt);
-    p->tiles_h = (p->H + kHaloTH - 1) / kHaloTH;
-    const int64_t m_sets = (int64_t)p->sets_w * p->tiles_h * p->B;
+    p->tiles_h = (p->H + p->th - 1) / p->th;
+    const int64_t m_sets = (int64_t)p->sets_w * p->tiles_h * ((p->B + p->tb - 1) / p->tb);
     if (m_sets * p->tiles_n > 0x3FFFFFFF) return false;
     p->m_sets = (int)m_sets;
     p->pair_tiles = (int)((m_sets + 1) / 2) * p->tiles_n;
@@ -1528,8 +1539,9 @@ bool plan_halo(HaloParams* p, int nt) {
 // Whole-filter reuse pays when there is more than one tap and strips of 8 x 16 pixels cover the
 // image without much padding.
 bool halo_applies(int H, int W, int taps) {
-  if (taps < 2 || W < 8 || H < 12) return false;
-  const int64_t covered = (int64_t)((W + 7) / 8 * 8) * ((H + kHaloTH - 1) / kHaloTH * kHaloTH);
+  if (taps < 2 || W < 8 || (H < 12 && H > 8) || H < 6) return false;
+  const int th = H <= 8 ? 8 : kHaloRows;  // images at most 8 pixels tall: strips of 8 rows of two images
+  const int64_t covered = (int64_t)((W + 7) / 8 * 8) * ((H + th - 1) / th * th);
   return covered * 100 <= (int64_t)H * W * 135;
 }
 
@@ -1543,10 +1555,11 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
   const int P = view.P, Q = view.Q;
   const uint64_t CA = (SPARSE && !FUSED) ? (uint64_t)view.a_channels / 2 : (uint64_t)view.a_channels;
   {
-    const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
-    const uint64_t strides[3] = {CA * 2, CA * 2 * Q, CA * 2 * Q * P};
+    // dimensions ordered (channel, pixel column, image, pixel row): a box then holds its rows in (pixel row, image) order
+    const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)view.batch, (uint64_t)P};
+    const uint64_t strides[3] = {CA * 2, CA * 2 * Q * P, CA * 2 * Q};
     // (fused: the pruning warps read dL/dO with plain loads and this map goes unused)
-    const uint32_t box[4] = {64, (uint32_t)p.pitch, (uint32_t)p.img_h, 1};
+    const uint32_t box[4] = {64, (uint32_t)p.pitch, (uint32_t)p.tb, (uint32_t)(p.img_h / p.tb)};
     if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
     tmE = tmA;
@@ -1554,9 +1567,9 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
   }
   if (SPARSE && !FUSED) {
     const uint64_t CE = (uint64_t)view.a_channels / 16;
-    const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch};
-    const uint64_t strides[3] = {CE * 2, CE * 2 * Q, CE * 2 * Q * P};
-    const uint32_t box[4] = {8, (uint32_t)p.pitch, (uint32_t)p.img_h, 1};
+    const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)view.batch, (uint64_t)P};
+    const uint64_t strides[3] = {CE * 2, CE * 2 * Q * P, CE * 2 * Q};
+    const uint32_t box[4] = {8, (uint32_t)p.pitch, (uint32_t)p.tb, (uint32_t)(p.img_h / p.tb)};
     if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
       return SDGP_ERR_CUDA;
   }
@@ -1569,9 +1582,9 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
       return SDGP_ERR_CUDA;
   }
   {
-    const uint64_t dims[4] = {(uint64_t)p.Cin, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.B};
-    const uint64_t strides[3] = {view.d_stride_w, view.d_stride_h, view.d_stride_b};
-    const uint32_t box[4] = {64, 8, (uint32_t)kHaloTH, 1};
+    const uint64_t dims[4] = {(uint64_t)p.Cin, (uint64_t)p.W, (uint64_t)p.B, (uint64_t)p.H};
+    const uint64_t strides[3] = {view.d_stride_w, view.d_stride_b, view.d_stride_h};
+    const uint32_t box[4] = {64, 8, (uint32_t)p.tb, (uint32_t)p.th};
     if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, view.d_base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
   }

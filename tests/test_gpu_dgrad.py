@@ -427,6 +427,11 @@ HALO_CASES = [
     (2, 28, 28, 128, 128, 3, 3, 1, 1),
     (9, 16, 16, 128, 128, 3, 3, 1, 1),      # odd number of tile sets: a pair with one phantom set
     (168, 16, 16, 64, 64, 3, 3, 1, 1),      # 84 pair tiles on 74 CTA pairs: the last round is dealt out strip by strip
+    (5, 8, 8, 256, 128, 3, 3, 1, 1),        # images 8 pixels tall: a strip is 8 rows of TWO images; odd batch
+    (4, 8, 16, 64, 128, 3, 3, 1, 1),        # the same with two strips side by side
+    (3, 6, 8, 128, 128, 3, 3, 1, 1),        # 6 pixel rows: two of the strip's eight are padding
+    (2, 8, 8, 64, 128, 5, 5, 1, 2),         # 5 x 5 filter on 8 x 8 images
+    (6, 8, 8, 128, 256, 3, 3, 1, 1),        # two channel blocks
 ]
 
 
