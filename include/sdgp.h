@@ -75,8 +75,9 @@ typedef enum {
 /* `flags` of the dgrad entry points. */
 enum {
   SDGP_FLAG_TWO_PASS = 0, /* prune kernel writes compressed dL/dO into the workspace, sparse GEMM reads it */
-  SDGP_FLAG_FUSED = 1,    /* pruning happens inside the dgrad kernel (needs m == 4, n <= 2); no workspace, no
-                             compressed tensor in global memory */
+  SDGP_FLAG_FUSED = 1,    /* pruning happens inside the dgrad kernel (n <= 2; m = 4, 8 or 16, also 32 for convolutions
+                             that run on the whole-filter-reuse kernel); no workspace, no compressed tensor in
+                             global memory */
   SDGP_FLAG_DENSE = 2,    /* no pruning: dense tensor-core data gradient of dL/dO itself (n, m, scheme ignored) */
   SDGP_FLAG_MASKED = 3,   /* prune kernel writes the pruned tensor as a dense copy (pruned positions +0.0, the tensor
                              Algorithm 1 returns) into the workspace and the dense tensor-core kernel contracts it:

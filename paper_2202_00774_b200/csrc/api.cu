@@ -180,9 +180,8 @@ sdgp_status sdgp_dgrad_conv2d_typed(const void* dO, const void* W, void* dD, int
     return sdgp::launch_dgrad(false, workspace, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, nullptr, dt);
   }
   if (flags == SDGP_FLAG_FUSED) {
-    if (m != 4) return SDGP_ERR_UNSUPPORTED;  // the in-kernel prune handles groups of four
     if (dtype == SDGP_FP16 && scheme == SDGP_RESCALED_MAGNITUDE) return SDGP_ERR_UNSUPPORTED;  // bf16 arithmetic only
-    const sdgp::FusedPrune fp = {n, (int)scheme, seed};
+    const sdgp::FusedPrune fp = {n, m, (int)scheme, seed};
     return sdgp::launch_dgrad(true, dO, nullptr, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, &fp, dt);
   }
   const int64_t Cpad = pad128(Cout);

@@ -87,7 +87,7 @@ struct DgradParams {
   int w_resident;         // whole W half-slice kept in shared memory
   int out_bufs;           // epilogue staging slabs (1 or 2)
   // fused pruning (the kernel reads dense dL/dO and prunes it while staging A)
-  int fused_n, fused_scheme;
+  int fused_n, fused_m, fused_scheme;
   uint32_t seed_lo, seed_hi;
   int P, Q;               // dO pixel grid (for the linear element index of the random scheme)
   int f16;                // element type of A, W and dD: 0 = bf16, 1 = IEEE binary16
@@ -175,19 +175,36 @@ __device__ __forceinline__ void build_metadata_image(const uint8_t* raw_rows, ui
 // vectors become one 16-byte chunk of the compressed row, written straight into the A tile's swizzled
 // row, and two of the row's sixteen bytes of position metadata (row-major form, as the rearrangement
 // step expects). vbase = number of the row's first 8-element vector in the whole dL/dO tensor (random keys).
-template <int N, int SCHEME>
+template <int M, int N, int SCHEME>
 __device__ __forceinline__ void fused_prune_eighth(const uint8_t* raw, int a_bytes, uint8_t* a_tile, uint8_t* meta_rows,
                                                    int i, int e, int64_t vbase, uint32_t seed_lo, uint32_t seed_hi) {
   const int sw = i & 7;
   uint32_t nibs = 0u;
   uint2 out[2];
+  uint4 w[2];
 #pragma unroll
   for (int jj = 0; jj < 2; ++jj) {
     const int j = 2 * e + jj;
-    const uint4 w = *(const uint4*)(raw + (j >> 3) * a_bytes + i * 128 + (((j & 7) ^ sw) << 4));
-    uint32_t y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2;
-    m4_prune_vector<N, SCHEME>(w, vbase + j, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
-    compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
+    w[jj] = *(const uint4*)(raw + (j >> 3) * a_bytes + i * 128 + (((j & 7) ^ sw) << 4));
+  }
+  uint32_t y[2][4], km[2][4];
+  if (M == 16) {  // the thread's two vectors are one group
+    top2_prune_group16<SCHEME>(w[0], w[1], vbase + 2 * e, seed_lo, seed_hi, N, y[0], km[0], y[1], km[1]);
+  } else {
+#pragma unroll
+    for (int jj = 0; jj < 2; ++jj) {
+      if (M == 4)
+        m4_prune_vector<N, SCHEME>(w[jj], vbase + 2 * e + jj, seed_lo, seed_hi, y[jj][0], y[jj][1], y[jj][2], y[jj][3], km[jj][0],
+                                   km[jj][1], km[jj][2], km[jj][3]);
+      else
+        top2_prune_vector<8, SCHEME>(w[jj], vbase + 2 * e + jj, seed_lo, seed_hi, N, 0, 0u, y[jj][0], y[jj][1], y[jj][2], y[jj][3],
+                                     km[jj][0], km[jj][1], km[jj][2], km[jj][3]);
+    }
+  }
+#pragma unroll
+  for (int jj = 0; jj < 2; ++jj) {
+    uint32_t slot0, slot1, nib2;
+    compressed_slots(y[jj][0], y[jj][1], y[jj][2], y[jj][3], km[jj][0], km[jj][1], km[jj][2], km[jj][3], slot0, slot1, nib2);
     out[jj] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
     nibs |= nib2 << (8 * jj);
   }
@@ -539,10 +556,13 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const int iw = i % p.TW, ih = (i / p.TW) % img_h, ib = i / (p.TW * img_h);
             const int64_t pixel = ((int64_t)(b0 + ib) * p.P + (p0 + ih)) * p.Q + (q0 + iw);  // any value when outside
             const int64_t vbase = pixel * (p.Cout >> 3) + cb * 16;
-#define SDGP_FUSED_ITEM(NN, SS) fused_prune_eighth<NN, SS>(raw, p.a_bytes, a_tile, meta_rows, i, e, vbase, p.seed_lo, p.seed_hi)
-            if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_ITEM(1, SDGP_MAGNITUDE); else SDGP_FUSED_ITEM(2, SDGP_MAGNITUDE); }
-            else if (p.fused_scheme == SDGP_RANDOM) { if (p.fused_n == 1) SDGP_FUSED_ITEM(1, SDGP_RANDOM); else SDGP_FUSED_ITEM(2, SDGP_RANDOM); }
-            else { if (p.fused_n == 1) SDGP_FUSED_ITEM(1, SDGP_RESCALED_MAGNITUDE); else SDGP_FUSED_ITEM(2, SDGP_RESCALED_MAGNITUDE); }
+#define SDGP_FUSED_ITEM(MM, NN, SS) fused_prune_eighth<MM, NN, SS>(raw, p.a_bytes, a_tile, meta_rows, i, e, vbase, p.seed_lo, p.seed_hi)
+#define SDGP_FUSED_M(MM)                                                                                                   \
+  if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_ITEM(MM, 1, SDGP_MAGNITUDE); else SDGP_FUSED_ITEM(MM, 2, SDGP_MAGNITUDE); } \
+  else if (p.fused_scheme == SDGP_RANDOM) { if (p.fused_n == 1) SDGP_FUSED_ITEM(MM, 1, SDGP_RANDOM); else SDGP_FUSED_ITEM(MM, 2, SDGP_RANDOM); }    \
+  else { if (p.fused_n == 1) SDGP_FUSED_ITEM(MM, 1, SDGP_RESCALED_MAGNITUDE); else SDGP_FUSED_ITEM(MM, 2, SDGP_RESCALED_MAGNITUDE); }
+            if (p.fused_m == 4) { SDGP_FUSED_M(4) } else if (p.fused_m == 8) { SDGP_FUSED_M(8) } else { SDGP_FUSED_M(16) }
+#undef SDGP_FUSED_M
 #undef SDGP_FUSED_ITEM
           }
           ptx::fence_proxy_async_smem();                // the compressed tile is read by the tensor core
@@ -679,7 +699,7 @@ struct HaloParams {
   // fused pruning (A is the dense dL/dO; m = 4): the pruning warps read it straight from global memory
   const uint8_t* a_dense;  // dL/dO [B, P, Q, Cout], 16-bit elements
   uint32_t pitch_magic;    // ceil(2^20 / pitch): i / pitch == (i * pitch_magic) >> 20 for every box pixel row i
-  int fused_n, fused_scheme;
+  int fused_n, fused_m, fused_scheme;
   uint32_t seed_lo, seed_hi;
   int P, Q;                // dO pixel grid (linear element index of the random scheme)
   int f16;                 // element type of A, W and dD: 0 = bf16, 1 = IEEE binary16
@@ -687,15 +707,21 @@ struct HaloParams {
 
 // Fused pruning of four vectors (8 channels each, already in registers) of one pixel row: out[v] = the 8
 // compressed bytes of vector v, metaw = their four bytes of position metadata (byte v = the two nibbles of
-// vector v). vnum(v) = number of vector v in the whole dL/dO tensor (random keys): vbase + vstep * v.
-template <int N, int SCHEME>
+// vector v). Number of vector v in the whole dL/dO tensor (random keys): vbase + vstep * v. Groups of M = 8, 16
+// or 32 channels span 1, 2 or 4 vectors held by neighbouring lanes (lane bits 0 and up; `part` = which of
+// them this lane's vectors are); all 32 lanes must call together.
+template <int M, int N, int SCHEME>
 __device__ __forceinline__ void fused_prune_vectors(const uint4 (&w)[4], int64_t vbase, int vstep, uint32_t seed_lo,
-                                                    uint32_t seed_hi, uint2 (&out)[4], uint32_t& metaw) {
+                                                    uint32_t seed_hi, int part, uint2 (&out)[4], uint32_t& metaw) {
   metaw = 0u;
 #pragma unroll
   for (int v = 0; v < 4; ++v) {
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2;
-    m4_prune_vector<N, SCHEME>(w[v], vbase + vstep * v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
+    if (M == 4)
+      m4_prune_vector<N, SCHEME>(w[v], vbase + vstep * v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
+    else
+      top2_prune_vector<(M == 4 ? 8 : M), SCHEME>(w[v], vbase + vstep * v, seed_lo, seed_hi, N, part, 0xFFFFFFFFu, y0, y1, y2, y3,
+                                                  km0, km1, km2, km3);
     compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
     out[v] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
     metaw |= nib2 << (8 * v);
@@ -1034,7 +1060,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int row8 = lane >> 2, c = lane & 3;
       const uint32_t px_bytes = (uint32_t)p.Cout * 2u;
       const int tb_shift = p.tb >> 1;  // tb is 1 or 2
-      auto prune_units = [&](auto n_tag, auto scheme_tag) {
+      auto prune_units = [&](auto m_tag, auto n_tag, auto scheme_tag) {
+        constexpr int M = decltype(m_tag)::value;
         constexpr int N = decltype(n_tag)::value;
         constexpr int SCHEME = decltype(scheme_tag)::value;
         // ---- load cursor: the unit whose loads go out next, and the box it lies in
@@ -1130,7 +1157,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int ast = cia & 1;
           uint2 out[4];
           uint32_t metaw;
-          fused_prune_vectors<N, SCHEME>(w, u_pix * (p.Cout >> 3) + u_kb * 16 + c, 4, p.seed_lo, p.seed_hi, out, metaw);
+          // (a group of M channels = vectors c + 4v of M / 8 neighbouring lanes c, same v)
+          fused_prune_vectors<M, N, SCHEME>(w, u_pix * (p.Cout >> 3) + u_kb * 16 + c, 4, p.seed_lo, p.seed_hi, c & (M / 8 - 1), out, metaw);
           // the registers of this unit are free: the loads of the next one go out before this one's stores
           more = ia < a_uses;
           if (more) fetch();
@@ -1167,16 +1195,22 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         announce();
       };
       using std::integral_constant;
-      if (p.fused_scheme == SDGP_MAGNITUDE) {
-        if (p.fused_n == 1) prune_units(integral_constant<int, 1>{}, integral_constant<int, SDGP_MAGNITUDE>{});
-        else prune_units(integral_constant<int, 2>{}, integral_constant<int, SDGP_MAGNITUDE>{});
-      } else if (p.fused_scheme == SDGP_RANDOM) {
-        if (p.fused_n == 1) prune_units(integral_constant<int, 1>{}, integral_constant<int, SDGP_RANDOM>{});
-        else prune_units(integral_constant<int, 2>{}, integral_constant<int, SDGP_RANDOM>{});
-      } else {
-        if (p.fused_n == 1) prune_units(integral_constant<int, 1>{}, integral_constant<int, SDGP_RESCALED_MAGNITUDE>{});
-        else prune_units(integral_constant<int, 2>{}, integral_constant<int, SDGP_RESCALED_MAGNITUDE>{});
-      }
+      auto with_m = [&](auto m_tag) {
+        if (p.fused_scheme == SDGP_MAGNITUDE) {
+          if (p.fused_n == 1) prune_units(m_tag, integral_constant<int, 1>{}, integral_constant<int, SDGP_MAGNITUDE>{});
+          else prune_units(m_tag, integral_constant<int, 2>{}, integral_constant<int, SDGP_MAGNITUDE>{});
+        } else if (p.fused_scheme == SDGP_RANDOM) {
+          if (p.fused_n == 1) prune_units(m_tag, integral_constant<int, 1>{}, integral_constant<int, SDGP_RANDOM>{});
+          else prune_units(m_tag, integral_constant<int, 2>{}, integral_constant<int, SDGP_RANDOM>{});
+        } else {
+          if (p.fused_n == 1) prune_units(m_tag, integral_constant<int, 1>{}, integral_constant<int, SDGP_RESCALED_MAGNITUDE>{});
+          else prune_units(m_tag, integral_constant<int, 2>{}, integral_constant<int, SDGP_RESCALED_MAGNITUDE>{});
+        }
+      };
+      if (p.fused_m == 4) with_m(integral_constant<int, 4>{});
+      else if (p.fused_m == 8) with_m(integral_constant<int, 8>{});
+      else if (p.fused_m == 16) with_m(integral_constant<int, 16>{});
+      else with_m(integral_constant<int, 32>{});
     }
   } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + 4) {
     // ------------------------------------------------------------ epilogue
@@ -1638,6 +1672,7 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
                          int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
                          const FusedPrune* fused, int dtype) {
   if (fused && (!sparse || fused->n < 1 || fused->n > 2)) return SDGP_ERR_UNSUPPORTED;
+  if (fused && fused->m != 4 && fused->m != 8 && fused->m != 16 && fused->m != 32) return SDGP_ERR_UNSUPPORTED;
   if (dtype != SDGP_BF16 && dtype != SDGP_FP16) return SDGP_ERR_INVALID_ARG;
   if (fused && dtype == SDGP_FP16 && fused->scheme == SDGP_RESCALED_MAGNITUDE) return SDGP_ERR_UNSUPPORTED;
   if (stride != 1 && stride != 2) return SDGP_ERR_UNSUPPORTED;
@@ -1688,7 +1723,7 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
       p.P = P; p.Q = Q;
       p.f16 = dtype == SDGP_FP16 ? 1 : 0;
       if (fused) {
-        p.fused_n = fused->n; p.fused_scheme = fused->scheme;
+        p.fused_n = fused->n; p.fused_m = fused->m; p.fused_scheme = fused->scheme;
         p.seed_lo = (uint32_t)fused->seed; p.seed_hi = (uint32_t)(fused->seed >> 32);
       }
       view.d_base = (uint8_t*)dD + ((size_t)ph * W + pw) * Cin * 2;
@@ -1706,7 +1741,7 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
         hp.P = P; hp.Q = Q;
         hp.f16 = p.f16;
         if (fused) {
-          hp.fused_n = p.fused_n; hp.fused_scheme = p.fused_scheme; hp.seed_lo = p.seed_lo; hp.seed_hi = p.seed_hi;
+          hp.fused_n = p.fused_n; hp.fused_m = p.fused_m; hp.fused_scheme = p.fused_scheme; hp.seed_lo = p.seed_lo; hp.seed_hi = p.seed_hi;
           st = BN == 256 ? launch_halo<true, 256, true>(A, meta, Wt, view, hp, stream)
              : BN == 128 ? launch_halo<true, 128, true>(A, meta, Wt, view, hp, stream)
                          : launch_halo<true, 64, true>(A, meta, Wt, view, hp, stream);
@@ -1723,6 +1758,7 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
         if (st != SDGP_ERR_UNSUPPORTED) return st;  // otherwise: does not fit, use the general kernel
       }
       if (fused) {
+        if (fused->m == 32) return SDGP_ERR_UNSUPPORTED;  // this kernel's threads hold 16 channels each: groups of up to 16
         st = BN == 256 ? launch_cfg<true, 256, true>(A, meta, Wt, view, p, stream)
            : BN == 128 ? launch_cfg<true, 128, true>(A, meta, Wt, view, p, stream)
                        : launch_cfg<true, 64, true>(A, meta, Wt, view, p, stream);

@@ -287,12 +287,6 @@ cudaError_t launch_m4_n(int scheme, bool f16, const void* dO, int64_t nvec, uint
 // span 2 or 4 lanes merge their pairs through xor-shuffles, and the outputs are written from the
 // same lane-paired form as the m = 4 path.
 
-__device__ __forceinline__ void merge_top2(uint32_t& hi, uint32_t& lo, uint32_t hi2, uint32_t lo2) {
-  const uint32_t h = max(hi, hi2);
-  lo = max(min(hi, hi2), max(lo, lo2));
-  hi = h;
-}
-
 template <int M, int N, int SCHEME, bool F16>
 __global__ void __launch_bounds__(kThreads)
 prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
@@ -303,7 +297,6 @@ prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, 
   constexpr int LANES = M / 8;
   static_assert(N == 1 || N == 2, "threshold selection keeps one or two elements");
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
-  const uint32_t pos0 = 31u - 8u * (uint32_t)(threadIdx.x & (LANES - 1));  // tie-break bits of element 0
   uint4 in[kVecPerThread];
 #pragma unroll
   for (int it = 0; it < kVecPerThread; ++it) {
@@ -313,57 +306,9 @@ prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, 
 #pragma unroll
   for (int it = 0; it < kVecPerThread; ++it) {
     const int64_t v = base + (int64_t)it * kThreads;
-    const uint4 w = in[it];
-    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-    uint32_t c[8];
-    if (SCHEME == SDGP_RANDOM) {
-      const uint4 o = philox4x32_10((uint32_t)v, (uint32_t)((uint64_t)v >> 32), 0u, 0u, seed_lo, seed_hi);
-      const uint32_t r[4] = {~o.x, ~o.y, ~o.z, ~o.w};  // smallest random key ranks first
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-        c[i] = (((i & 1) ? (r[i >> 1] >> 11) : (r[i >> 1] << 5)) & 0x1FFFE0u) | (pos0 - i);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-        c[i] = (((i & 1) ? (ww[i >> 1] >> 11) : (ww[i >> 1] << 5)) & 0xFFFE0u) | (pos0 - i);  // |x| << 5 | tie-break
-    }
-    uint32_t hi, lo = 0;
-    if (N == 1) {
-      hi = max(max(max(c[0], c[1]), max(c[2], c[3])), max(max(c[4], c[5]), max(c[6], c[7])));
-#pragma unroll
-      for (int d = 1; d < LANES; d <<= 1) hi = max(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, d));
-    } else {
-      uint32_t h1 = max(c[2], c[3]), l1 = min(c[2], c[3]), h2 = max(c[4], c[5]), l2 = min(c[4], c[5]),
-               h3 = max(c[6], c[7]), l3 = min(c[6], c[7]);
-      hi = max(c[0], c[1]);
-      lo = min(c[0], c[1]);
-      merge_top2(hi, lo, h1, l1);
-      merge_top2(h2, l2, h3, l3);
-      merge_top2(hi, lo, h2, l2);
-#pragma unroll
-      for (int d = 1; d < LANES; d <<= 1) {
-        const uint32_t oh = __shfl_xor_sync(0xFFFFFFFFu, hi, d), ol = __shfl_xor_sync(0xFFFFFFFFu, lo, d);
-        merge_top2(hi, lo, oh, ol);
-      }
-    }
-    const uint32_t t1 = ((N == 1) ? hi : lo) - 1u;  // keep <=> key > t1; (t1 - key) is then negative
-    const uint32_t p0 = prmt(w.x, w.z, 0x5410), p1 = prmt(w.x, w.z, 0x7632);
-    const uint32_t p2 = prmt(w.y, w.w, 0x5410), p3 = prmt(w.y, w.w, 0x7632);
-    const uint32_t km0 = prmt(t1 - c[0], t1 - c[4], 0xFFBB), km1 = prmt(t1 - c[1], t1 - c[5], 0xFFBB);
-    const uint32_t km2 = prmt(t1 - c[2], t1 - c[6], 0xFFBB), km3 = prmt(t1 - c[3], t1 - c[7], 0xFFBB);
-    uint32_t y0 = p0 & km0, y1 = p1 & km1, y2 = p2 & km2, y3 = p3 & km3;
-    if (SCHEME == SDGP_RESCALED_MAGNITUDE) {
-      // balanced pairwise sums in index order: elements 0..3 are the low lanes, 4..7 the high lanes
-      float tsum = __fadd_rn(sum4_lo_abs<F16>(p0, p1, p2, p3), sum4_hi_abs<F16>(p0, p1, p2, p3));
-      float ssum = __fadd_rn(sum4_lo_abs<F16>(y0, y1, y2, y3), sum4_hi_abs<F16>(y0, y1, y2, y3));
-#pragma unroll
-      for (int d = 1; d < LANES; d <<= 1) {
-        tsum = __fadd_rn(tsum, __shfl_xor_sync(0xFFFFFFFFu, tsum, d));
-        ssum = __fadd_rn(ssum, __shfl_xor_sync(0xFFFFFFFFu, ssum, d));
-      }
-      const float sc = (ssum == 0.0f) ? 1.0f : __fdiv_rn(tsum, ssum);
-      rescale_packed<F16>(y0, y1, y2, y3, km0, km1, km2, km3, sc, sc, tsum, tsum);
-    }
+    uint32_t y0, y1, y2, y3, km0, km1, km2, km3;
+    top2_prune_vector<M, SCHEME, F16>(in[it], v, seed_lo, seed_hi, N, (int)(threadIdx.x & (LANES - 1)), 0xFFFFFFFFu, y0, y1, y2,
+                                      y3, km0, km1, km2, km3);
     if (v < nvec) emit_packed<true>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask, pitch);
   }
 }

@@ -219,5 +219,115 @@ __device__ __forceinline__ void compressed_slots(uint32_t y0, uint32_t y1, uint3
   nib2 = (nib & 0xFu) | ((nib >> 12) & 0xF0u);
 }
 
+// Groups of 8, 16 or 32 with n <= 2 (Algorithm 1 with the same three pruning functions): the survivors are the
+// elements whose composite key (rank key << 5 | 31 - position, unique inside a group) reaches the group's n-th
+// largest. The M / 8 vectors of a group are held by M / 8 neighbouring lanes (lane bits 0 and up; `part` = this
+// lane's number among them, i.e. which eighth of the group the vector is); each lane finds the two largest keys
+// of its 8 elements with a max/min network and the lanes merge their pairs through xor-shuffles, which every
+// lane named in `lanes` must execute together. Output in the lane-paired form of m4_prune_vector.
+__device__ __forceinline__ void merge_top2(uint32_t& hi, uint32_t& lo, uint32_t hi2, uint32_t lo2) {
+  const uint32_t h = max(hi, hi2);
+  lo = max(min(hi, hi2), max(lo, lo2));
+  hi = h;
+}
+
+// Composite keys of the 8 elements of vector w (number v in the tensor); pos0 = tie-break bits of element 0.
+template <int SCHEME>
+__device__ __forceinline__ void top2_keys(const uint4& w, int64_t v, uint32_t seed_lo, uint32_t seed_hi, uint32_t pos0,
+                                          uint32_t (&c)[8]) {
+  const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+  if (SCHEME == SDGP_RANDOM) {
+    const uint4 o = philox4x32_10((uint32_t)v, (uint32_t)((uint64_t)v >> 32), 0u, 0u, seed_lo, seed_hi);
+    const uint32_t r[4] = {~o.x, ~o.y, ~o.z, ~o.w};  // smallest random key ranks first
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      c[i] = (((i & 1) ? (r[i >> 1] >> 11) : (r[i >> 1] << 5)) & 0x1FFFE0u) | (pos0 - i);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      c[i] = (((i & 1) ? (ww[i >> 1] >> 11) : (ww[i >> 1] << 5)) & 0xFFFE0u) | (pos0 - i);  // |x| << 5 | tie-break
+  }
+}
+
+// The two largest of eight keys.
+__device__ __forceinline__ void top2_of_8(const uint32_t (&c)[8], uint32_t& hi, uint32_t& lo) {
+  uint32_t h1 = max(c[2], c[3]), l1 = min(c[2], c[3]), h2 = max(c[4], c[5]), l2 = min(c[4], c[5]),
+           h3 = max(c[6], c[7]), l3 = min(c[6], c[7]);
+  hi = max(c[0], c[1]);
+  lo = min(c[0], c[1]);
+  merge_top2(hi, lo, h1, l1);
+  merge_top2(h2, l2, h3, l3);
+  merge_top2(hi, lo, h2, l2);
+}
+
+// Lane-paired values and keep masks of a vector whose elements with key > t1 survive.
+__device__ __forceinline__ void top2_apply(const uint4& w, const uint32_t (&c)[8], uint32_t t1, uint32_t& p0, uint32_t& p1,
+                                           uint32_t& p2, uint32_t& p3, uint32_t& y0, uint32_t& y1, uint32_t& y2, uint32_t& y3,
+                                           uint32_t& km0, uint32_t& km1, uint32_t& km2, uint32_t& km3) {
+  p0 = prmt(w.x, w.z, 0x5410); p1 = prmt(w.x, w.z, 0x7632);
+  p2 = prmt(w.y, w.w, 0x5410); p3 = prmt(w.y, w.w, 0x7632);
+  km0 = prmt(t1 - c[0], t1 - c[4], 0xFFBB); km1 = prmt(t1 - c[1], t1 - c[5], 0xFFBB);  // (t1 - key) negative <=> kept
+  km2 = prmt(t1 - c[2], t1 - c[6], 0xFFBB); km3 = prmt(t1 - c[3], t1 - c[7], 0xFFBB);
+  y0 = p0 & km0; y1 = p1 & km1; y2 = p2 & km2; y3 = p3 & km3;
+}
+
+template <int M, int SCHEME, bool F16 = false>
+__device__ __forceinline__ void top2_prune_vector(const uint4& w, int64_t v, uint32_t seed_lo, uint32_t seed_hi, int n,
+                                                  int part, unsigned lanes, uint32_t& y0, uint32_t& y1, uint32_t& y2,
+                                                  uint32_t& y3, uint32_t& km0, uint32_t& km1, uint32_t& km2,
+                                                  uint32_t& km3) {
+  constexpr int LANES = M / 8;
+  uint32_t c[8], hi, lo;
+  top2_keys<SCHEME>(w, v, seed_lo, seed_hi, 31u - 8u * (uint32_t)part, c);
+  top2_of_8(c, hi, lo);
+#pragma unroll
+  for (int d = 1; d < LANES; d <<= 1) {
+    const uint32_t oh = __shfl_xor_sync(lanes, hi, d), ol = __shfl_xor_sync(lanes, lo, d);
+    merge_top2(hi, lo, oh, ol);
+  }
+  uint32_t p0, p1, p2, p3;
+  top2_apply(w, c, ((n == 1) ? hi : lo) - 1u, p0, p1, p2, p3, y0, y1, y2, y3, km0, km1, km2, km3);
+  if (SCHEME == SDGP_RESCALED_MAGNITUDE) {
+    // balanced pairwise sums in index order: elements 0..3 are the low lanes, 4..7 the high lanes
+    float tsum = __fadd_rn(sum4_lo_abs<F16>(p0, p1, p2, p3), sum4_hi_abs<F16>(p0, p1, p2, p3));
+    float ssum = __fadd_rn(sum4_lo_abs<F16>(y0, y1, y2, y3), sum4_hi_abs<F16>(y0, y1, y2, y3));
+#pragma unroll
+    for (int d = 1; d < LANES; d <<= 1) {
+      tsum = __fadd_rn(tsum, __shfl_xor_sync(lanes, tsum, d));
+      ssum = __fadd_rn(ssum, __shfl_xor_sync(lanes, ssum, d));
+    }
+    const float sc = (ssum == 0.0f) ? 1.0f : __fdiv_rn(tsum, ssum);
+    rescale_packed<F16>(y0, y1, y2, y3, km0, km1, km2, km3, sc, sc, tsum, tsum);
+  }
+}
+
+// One group of 16 whose two vectors (numbers v and v + 1) are held by the same thread.
+template <int SCHEME, bool F16 = false>
+__device__ __forceinline__ void top2_prune_group16(const uint4& wa, const uint4& wb, int64_t v, uint32_t seed_lo,
+                                                   uint32_t seed_hi, int n, uint32_t (&ya)[4], uint32_t (&kma)[4],
+                                                   uint32_t (&yb)[4], uint32_t (&kmb)[4]) {
+  uint32_t ca[8], cb[8], hi, lo, hb, lb;
+  top2_keys<SCHEME>(wa, v, seed_lo, seed_hi, 31u, ca);
+  top2_keys<SCHEME>(wb, v + 1, seed_lo, seed_hi, 23u, cb);
+  top2_of_8(ca, hi, lo);
+  top2_of_8(cb, hb, lb);
+  merge_top2(hi, lo, hb, lb);
+  const uint32_t t1 = ((n == 1) ? hi : lo) - 1u;
+  uint32_t pa[4], pb[4];
+  top2_apply(wa, ca, t1, pa[0], pa[1], pa[2], pa[3], ya[0], ya[1], ya[2], ya[3], kma[0], kma[1], kma[2], kma[3]);
+  top2_apply(wb, cb, t1, pb[0], pb[1], pb[2], pb[3], yb[0], yb[1], yb[2], yb[3], kmb[0], kmb[1], kmb[2], kmb[3]);
+  if (SCHEME == SDGP_RESCALED_MAGNITUDE) {
+    // the same tree as across two lanes: (sum of elements 0..7) + (sum of elements 8..15)
+    const float ta = __fadd_rn(sum4_lo_abs<F16>(pa[0], pa[1], pa[2], pa[3]), sum4_hi_abs<F16>(pa[0], pa[1], pa[2], pa[3]));
+    const float tb = __fadd_rn(sum4_lo_abs<F16>(pb[0], pb[1], pb[2], pb[3]), sum4_hi_abs<F16>(pb[0], pb[1], pb[2], pb[3]));
+    const float sa = __fadd_rn(sum4_lo_abs<F16>(ya[0], ya[1], ya[2], ya[3]), sum4_hi_abs<F16>(ya[0], ya[1], ya[2], ya[3]));
+    const float sb = __fadd_rn(sum4_lo_abs<F16>(yb[0], yb[1], yb[2], yb[3]), sum4_hi_abs<F16>(yb[0], yb[1], yb[2], yb[3]));
+    const float tsum = __fadd_rn(ta, tb), ssum = __fadd_rn(sa, sb);
+    const float sc = (ssum == 0.0f) ? 1.0f : __fdiv_rn(tsum, ssum);
+    rescale_packed<F16>(ya[0], ya[1], ya[2], ya[3], kma[0], kma[1], kma[2], kma[3], sc, sc, tsum, tsum);
+    rescale_packed<F16>(yb[0], yb[1], yb[2], yb[3], kmb[0], kmb[1], kmb[2], kmb[3], sc, sc, tsum, tsum);
+  }
+}
+
 }  // namespace
 }  // namespace sdgp

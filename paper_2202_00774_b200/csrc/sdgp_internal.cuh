@@ -29,9 +29,10 @@ cudaError_t launch_scale_weights(const void* W, const float* sums, int64_t K, in
 // [B,P,Q,Cout]; sparse == true: A is the compressed values [B,P,Q,Cp/2] and meta [B,P,Q,Cp/16]
 // with Cp = Cout rounded up to a multiple of 128 (see launch_prune's k_pad).
 // Wt [Cout,R,S,Cin], dD [B,H,W,Cin]. A fully connected layer is B = H = 1, W = rows, R = S = 1.
-// fused != nullptr: A is the dense dL/dO and the kernel prunes it on the fly (groups of 4).
+// fused != nullptr: A is the dense dL/dO and the kernel prunes it on the fly (n <= 2).
 struct FusedPrune {
   int n;
+  int m;  // group size: 4, 8, 16 (32 in the whole-filter-reuse kernel only)
   int scheme;
   uint64_t seed;
 };

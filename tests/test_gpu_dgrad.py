@@ -465,13 +465,47 @@ def test_whole_filter_reuse_kernel(case, mode):
     assert_close(got, *conv_ref(src, W, H, Wd, stride, pad))
 
 
-def test_fused_needs_groups_of_four():
+@pytest.mark.parametrize("n,m,scheme", [(2, 8, oracle.MAGNITUDE), (1, 8, oracle.RESCALED), (2, 16, oracle.MAGNITUDE),
+                                        (2, 16, oracle.RANDOM), (2, 8, oracle.RANDOM), (1, 16, oracle.RESCALED)])
+@pytest.mark.parametrize("case", [(3, 16, 16, 64, 128, 3, 3, 1, 1),      # whole-filter-reuse kernel, two strips
+                                  (5, 8, 8, 256, 128, 3, 3, 1, 1),       # ... strips of two images
+                                  (2, 16, 16, 128, 256, 3, 3, 1, 1),     # two channel blocks
+                                  (5, 4, 4, 64, 256, 3, 3, 1, 1),        # general kernel, several images per tile
+                                  (1, 1, 333, 128, 512, 1, 1, 1, 0),     # fully connected
+                                  (2, 14, 14, 64, 128, 1, 1, 1, 0)])     # 1 x 1
+def test_fused_groups_of_8_and_16(case, n, m, scheme):
+    """SDGP_FLAG_FUSED for groups larger than four (n <= 2): the in-kernel prune finds the group's two largest
+    keys; a group's vectors sit in one thread or in neighbouring lanes."""
     import paper_2202_00774_b200 as sdgp
-    dO = torch.zeros((2, 8, 8, 128), dtype=torch.int16, device="cuda")
-    W = torch.zeros((128, 3, 3, 64), dtype=torch.int16, device="cuda")
-    dD = torch.zeros((2, 8, 8, 64), dtype=torch.int16, device="cuda")
+    B, H, Wd, Cin, Cout, R, S, stride, pad = case
+    layer = inputs.ConvLayer("t", B, H, Wd, Cin, Cout, R, S, stride, pad)
+    dO, W = inputs.conv_layer_tensors(layer, seed=B + Cout + m)
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, stride, pad, n, m, scheme, seed=31, flags=sdgp.FLAG_FUSED)
+    check_no_device_error()
+    pruned = oracle.prune(dO.reshape(-1, Cout), n, m, scheme, 31, want=("dense",))["dense"].reshape(dO.shape)
+    got = to_f64(dD)
+    assert not np.isnan(got).any()
+    assert_close(got, *conv_ref(pruned, W, H, Wd, stride, pad))
+
+
+def test_fused_groups_of_32():
+    """Groups of 32 span four lanes of the whole-filter-reuse kernel's pruning warps; the general kernel (whose
+    threads hold 16 channels) refuses them."""
+    import paper_2202_00774_b200 as sdgp
+    layer = inputs.ConvLayer("t", 3, 16, 16, 64, 128, 3, 3, 1, 1)
+    dO, W = inputs.conv_layer_tensors(layer, seed=77)
+    dD = torch.full(layer.dD_shape(), -1, dtype=torch.int16, device="cuda")
+    for n, scheme in ((2, oracle.MAGNITUDE), (1, oracle.RANDOM), (2, oracle.RESCALED)):
+        sdgp.sdgp_dgrad_conv2d(dev16(dO), dev16(W), dD, 1, 1, n, 32, scheme, seed=5, flags=sdgp.FLAG_FUSED)
+        check_no_device_error()
+        pruned = oracle.prune(dO.reshape(-1, 128), n, 32, scheme, 5, want=("dense",))["dense"].reshape(dO.shape)
+        assert_close(to_f64(dD), *conv_ref(pruned, W, 16, 16, 1, 1))
+    x = torch.zeros((64, 128), dtype=torch.int16, device="cuda")
+    w = torch.zeros((128, 64), dtype=torch.int16, device="cuda")
+    y = torch.zeros((64, 64), dtype=torch.int16, device="cuda")
     with pytest.raises(sdgp.SdgpError) as e:
-        sdgp.sdgp_dgrad_conv2d(dO, W, dD, 1, 1, 2, 8, sdgp.MAGNITUDE, flags=sdgp.FLAG_FUSED)
+        sdgp.sdgp_dgrad_linear(x, w, y, 2, 32, sdgp.MAGNITUDE, flags=sdgp.FLAG_FUSED)
     assert e.value.status == 2
 
 
