@@ -57,6 +57,8 @@ def _load():
             lib.oracle_f32_to_f16.restype = ctypes.c_uint16
             lib.oracle_f16_to_f64.argtypes = [ctypes.c_uint16]
             lib.oracle_f16_to_f64.restype = dbl
+            lib.oracle_relu_backward.argtypes = [vp, vp, i64, i32, vp]
+            lib.oracle_relu_backward.restype = i32
             lib.oracle_expand.argtypes = [vp, vp, i64, i64, vp]
             lib.oracle_expand.restype = i32
             lib.oracle_dgrad_linear.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64]
@@ -112,6 +114,28 @@ def prune(dO, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask"), dt
                                 _ptr(out.get("values")), _ptr(out.get("meta")), _ptr(out.get("mask")))
     if rc != 0:
         raise ValueError("oracle_prune rejected its arguments (rc=%d)" % rc)
+    return out
+
+
+def relu_backward(dY, act, dtype=BF16):
+    """dL/dO below a ReLU (Section 2.1, Fig. 2): dY where the ReLU's activation ``act`` is positive, +0.0 elsewhere.
+    Arrays of 16-bit patterns of the same shape."""
+    dY, act = _u16(dY), _u16(act)
+    if dY.shape != act.shape:
+        raise ValueError("dY and act must have the same shape")
+    out = np.empty(dY.shape, np.uint16)
+    rc = _load().oracle_relu_backward(_ptr(dY), _ptr(act), dY.size, dtype, _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_relu_backward rejected its arguments")
+    return out
+
+
+def relu_backward_prune(dY, act, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask"), dtype=BF16):
+    """The producer of the pruned dL/dO: ReLU backward, then Algorithm 1 on the result. Returns the dict of
+    ``prune`` plus ``"grad"``, the unpruned dL/dO that the weight gradient still needs (Section 3.1)."""
+    grad = relu_backward(dY, act, dtype)
+    out = prune(grad, n, m, scheme, seed, want, dtype)
+    out["grad"] = grad
     return out
 
 

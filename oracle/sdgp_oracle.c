@@ -14,6 +14,10 @@
  *     restore survivors to their original positions);
  *   - Section 2.1 / Fig. 2-3 data-gradient contraction (the reduction runs over the
  *     output-channel dimension, which is the pruned one).
+ *   - Section 2.1 / Fig. 2 (backward pass: a layer's dL/dO is what the layer above hands down), Section 3.1
+ *     (the pruned tensor is a copy: the unpruned dL/dO still feeds the weight gradient) and Section 3.3
+ *     (the many exact zeros of dL/dO come from the ReLU): oracle_relu_backward forms dL/dO from the
+ *     gradient above a ReLU and that ReLU's activation; pruning it is then Algorithm 1 unchanged.
  *
  * Readings taken where the paper is silent (each is listed in the design notes):
  *   - ties between equal magnitudes go to the lower index;
@@ -469,6 +473,22 @@ int oracle_conv2d_forward_f64(const double* D, const uint16_t* W, double* O, int
             }
           O[(((int64_t)b * P + p) * Q + q) * Cout + co] = acc;
         }
+  return ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------- the producer of dL/dO
+ *
+ * Section 2.1 / Fig. 2: in the backward pass a layer's dL/dO is the gradient handed down by what follows
+ * it. For a ReLU that is dO[e] = dY[e] where the ReLU's activation is positive and +0.0 elsewhere (its
+ * derivative is 1 for positive inputs and 0 otherwise; the ReLU's output is positive exactly where its
+ * input is, so either may be passed as `act`). An activation that is not a number passes nothing.
+ * The survivors keep the exact bits of dY. */
+int oracle_relu_backward(const uint16_t* dY, const uint16_t* act, int64_t count, int dtype, uint16_t* dO) {
+  if (!dY || !act || !dO || count < 0 || (dtype != ORACLE_BF16 && dtype != ORACLE_FP16)) return ORACLE_ERR_ARG;
+  for (int64_t e = 0; e < count; ++e) {
+    const float a = elem_to_f32(act[e], dtype);
+    dO[e] = (a > 0.0f) ? dY[e] : (uint16_t)0; /* a NaN compares false */
+  }
   return ORACLE_OK;
 }
 
