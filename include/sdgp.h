@@ -168,6 +168,21 @@ sdgp_status sdgp_spmm_conv2d_typed(const void* values, const void* meta, const v
                                    int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
                                    sdgp_dtype dtype, void* stream);
 
+/* The producer of the pruned dL/dO (Section 2.1, Fig. 2: in the backward pass a layer's dL/dO is what the layer above
+ * hands down; Section 3.1: the pruned tensor is a copy, the unpruned one still feeds the weight gradient; Section 3.3: its
+ * many exact zeros come from the ReLU). One pass over the gradient dY above a ReLU and that ReLU's activation `act`
+ * (its output or its input, [rows, K] each, element type `dtype`) forms
+ *     dL/dO[r, k] = dY[r, k] if act[r, k] > 0 (a number greater than zero; NaN passes nothing), else +0.0
+ * and applies Algorithm 1 to it, so that no separate pass has to read dL/dO again before the sparse contraction
+ * (sdgp_spmm_*) can run:
+ *   grad      [rows, K]   the unpruned dL/dO (survivors keep the bits of dY)           - optional
+ *   dOp_dense, values, meta, mask: as sdgp_prune, computed from that dL/dO            - each optional
+ * Requirements as sdgp_prune; groups of 8, 16 and 32 need n <= 2 (n == m is allowed for m == 4: nothing is pruned and
+ * the call is a plain ReLU backward). */
+sdgp_status sdgp_relu_backward_prune(const void* dY, const void* act, int64_t rows, int64_t K, int n, int m,
+                                     sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad, void* dOp_dense,
+                                     void* values, void* meta, void* mask, void* stream);
+
 /* The factors of SDGP_FLAG_CHANNEL on their own: dO [rows, K] of element type `dtype`, groups of m along K,
  * magnitude function with n survivors (any 1 <= n <= m, m in {4, 8, 16, 32}, K % m == 0, K % 8 == 0).
  * `out` is a device array of 3 * K floats: [0, K) the factors, [K, 2K) the column sums of |dO| over all rows,

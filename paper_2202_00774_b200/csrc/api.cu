@@ -79,6 +79,25 @@ sdgp_status sdgp_prune_typed(const void* dO, int64_t rows, int64_t K, int n, int
   return e == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
+sdgp_status sdgp_relu_backward_prune(const void* dY, const void* act, int64_t rows, int64_t K, int n, int m,
+                                     sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad, void* dOp_dense,
+                                     void* values, void* meta, void* mask, void* stream) {
+  if (!valid_dtype(dtype)) return SDGP_ERR_INVALID_ARG;
+  sdgp_status st = check_prune_args(rows, K, n, m, (int)scheme);
+  if (st != SDGP_OK) return st;
+  if (n > 2 && !(m == 4)) return SDGP_ERR_UNSUPPORTED;   // groups of 8, 16, 32: the threshold selection keeps one or two
+  if (rows == 0 || K == 0) return SDGP_OK;
+  if (!dY || !act) return SDGP_ERR_INVALID_ARG;
+  if ((values || meta) && n > 2) return SDGP_ERR_UNSUPPORTED;
+  if (K % 16 != 0 || (mask && K % 32 != 0)) return SDGP_ERR_ALIGNMENT;
+  if (!aligned16(dY) || !aligned16(act) || !aligned16(grad) || !aligned16(dOp_dense) || !aligned16(values) ||
+      !aligned16(meta) || !aligned16(mask))
+    return SDGP_ERR_ALIGNMENT;
+  cudaError_t e = sdgp::launch_relu_backward_prune(dY, act, rows, K, n, m, (int)scheme, seed, grad, dOp_dense, values, meta,
+                                                   mask, (cudaStream_t)stream, (int)dtype);
+  return e == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
+}
+
 // SDGP_FLAG_CHANNEL: behind the compressed tensor, 3 * K floats (factors, two column sums) and the scaled copy of W
 static size_t channel_floats_bytes(int64_t K) { return round_up((size_t)K * 3 * sizeof(float), 256); }
 static size_t channel_extra_bytes(int64_t K, int64_t w_row_elems) {

@@ -41,6 +41,35 @@ cudaError_t launch_after_previous(void (*kernel)(Params...), dim3 grid, dim3 blo
   return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
 }
 
+// The producer of dL/dO below a ReLU (Section 2.1, Fig. 2): the 8 gradients g above the ReLU pass where the
+// ReLU's activation a is positive (a number greater than zero: sign clear, magnitude between 1 and the
+// pattern of infinity) and become +0.0 elsewhere. nan_add = 0x7FFF - (pattern of infinity) in both half-words:
+// adding it to a magnitude sets the half-word's top bit exactly for the NaN patterns.
+struct ReluSource {
+  const uint4* act;   // the ReLU's activation, same shape as the gradient; nullptr: no ReLU, the input is dL/dO itself
+  uint4* grad;        // optional: the unpruned dL/dO (kept for the weight gradient, Section 3.1)
+  uint32_t nan_add;
+};
+
+__device__ __forceinline__ uint32_t relu_pass2(uint32_t g, uint32_t a, uint32_t nan_add) {
+  const uint32_t mag = a & 0x7FFF7FFFu;
+  const uint32_t nonzero = mag + 0x7FFF7FFFu, nan = mag + nan_add;   // top bit of each half-word
+  const uint32_t ok = nonzero & ~nan & ~a;
+  return g & prmt(ok, 0u, 0xBB99);  // top bits replicated over their half-words
+}
+
+template <bool RELU>
+__device__ __forceinline__ uint4 load_gradient(const uint4* __restrict__ dO, int64_t v, const ReluSource& src) {
+  uint4 g = __ldg(dO + v);
+  if (RELU) {
+    const uint4 a = __ldg(src.act + v);
+    g = make_uint4(relu_pass2(g.x, a.x, src.nan_add), relu_pass2(g.y, a.y, src.nan_add), relu_pass2(g.z, a.z, src.nan_add),
+                   relu_pass2(g.w, a.w, src.nan_add));
+    if (src.grad) src.grad[v] = g;
+  }
+  return g;
+}
+
 // M: group size; LANES = lanes that share a group (1, 2 or 4).
 template <int M, int SCHEME, bool F16>
 __global__ void __launch_bounds__(kThreads)
@@ -229,11 +258,11 @@ __device__ __forceinline__ void emit_packed(int64_t v, uint32_t y0, uint32_t y1,
   }
 }
 
-template <int N, int SCHEME, bool F16>
+template <int N, int SCHEME, bool F16, bool RELU>
 __global__ void __launch_bounds__(kThreads)
 prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                 uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
-                uint8_t* __restrict__ mask, OutPitch pitch) {
+                uint8_t* __restrict__ mask, OutPitch pitch, ReluSource src) {
   ptx::wait_for_previous_grid();
   ptx::launch_dependents();  // only once this grid's own predecessor is done: at most one grid ever waits behind a running one
   const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
@@ -241,7 +270,7 @@ prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, ui
 #pragma unroll
   for (int it = 0; it < kVecPerThread; ++it) {
     const int64_t v = base + (int64_t)it * kThreads;
-    in[it] = (v < nvec) ? __ldg(dO + v) : make_uint4(0, 0, 0, 0);
+    in[it] = (v < nvec) ? load_gradient<RELU>(dO, v, src) : make_uint4(0, 0, 0, 0);
   }
 #pragma unroll
   for (int it = 0; it < kVecPerThread; ++it) {
@@ -256,9 +285,9 @@ prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, ui
 
 // Only the rescaled scheme reads values as numbers: the other two run the same (bf16-named)
 // instantiation for both element types.
-template <int N>
+template <int N, bool RELU>
 cudaError_t launch_m4_n(int scheme, bool f16, const void* dO, int64_t nvec, uint64_t seed, void* dense, void* values,
-                        void* meta, void* mask, OutPitch pitch, cudaStream_t stream) {
+                        void* meta, void* mask, OutPitch pitch, cudaStream_t stream, ReluSource src) {
   const int64_t per_block = (int64_t)kThreads * kVecPerThread;
   const int64_t blocks = (nvec + per_block - 1) / per_block;
   if (blocks == 0) return cudaSuccess;
@@ -266,8 +295,8 @@ cudaError_t launch_m4_n(int scheme, bool f16, const void* dO, int64_t nvec, uint
   const dim3 grid((unsigned)blocks), block(kThreads);
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
 #define SDGP_LAUNCH4(S, F)                                                                      \
-  launch_after_previous(prune_m4_kernel<N, S, F>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
-                                                    (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch)
+  launch_after_previous(prune_m4_kernel<N, S, F, RELU>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
+                                                    (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch, src)
   switch (scheme) {
     case SDGP_RANDOM: SDGP_LAUNCH4(SDGP_RANDOM, false); break;
     case SDGP_MAGNITUDE: SDGP_LAUNCH4(SDGP_MAGNITUDE, false); break;
@@ -287,11 +316,11 @@ cudaError_t launch_m4_n(int scheme, bool f16, const void* dO, int64_t nvec, uint
 // span 2 or 4 lanes merge their pairs through xor-shuffles, and the outputs are written from the
 // same lane-paired form as the m = 4 path.
 
-template <int M, int N, int SCHEME, bool F16>
+template <int M, int N, int SCHEME, bool F16, bool RELU>
 __global__ void __launch_bounds__(kThreads)
 prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, uint32_t seed_hi,
                   uint4* __restrict__ dense, uint2* __restrict__ values, uint8_t* __restrict__ meta,
-                  uint8_t* __restrict__ mask, OutPitch pitch) {
+                  uint8_t* __restrict__ mask, OutPitch pitch, ReluSource src) {
   ptx::wait_for_previous_grid();
   ptx::launch_dependents();  // only once this grid's own predecessor is done: at most one grid ever waits behind a running one
   constexpr int LANES = M / 8;
@@ -301,7 +330,7 @@ prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, 
 #pragma unroll
   for (int it = 0; it < kVecPerThread; ++it) {
     const int64_t v = base + (int64_t)it * kThreads;
-    in[it] = (v < nvec) ? __ldg(dO + v) : make_uint4(0, 0, 0, 0);
+    in[it] = (v < nvec) ? load_gradient<RELU>(dO, v, src) : make_uint4(0, 0, 0, 0);
   }
 #pragma unroll
   for (int it = 0; it < kVecPerThread; ++it) {
@@ -313,9 +342,9 @@ prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, 
   }
 }
 
-template <int M, int N>
+template <int M, int N, bool RELU>
 cudaError_t launch_top2(int scheme, bool f16, const void* dO, int64_t nvec, uint64_t seed, void* dense, void* values,
-                        void* meta, void* mask, OutPitch pitch, cudaStream_t stream) {
+                        void* meta, void* mask, OutPitch pitch, cudaStream_t stream, ReluSource src) {
   const int64_t per_block = (int64_t)kThreads * kVecPerThread;
   const int64_t blocks = (nvec + per_block - 1) / per_block;
   if (blocks == 0) return cudaSuccess;
@@ -323,8 +352,8 @@ cudaError_t launch_top2(int scheme, bool f16, const void* dO, int64_t nvec, uint
   const dim3 grid((unsigned)blocks), block(kThreads);
   const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
 #define SDGP_LAUNCH_T2(S, F)                                                                         \
-  launch_after_previous(prune_top2_kernel<M, N, S, F>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
-                                                         (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch)
+  launch_after_previous(prune_top2_kernel<M, N, S, F, RELU>, grid, block, stream, (const uint4*)dO, nvec, lo, hi, (uint4*)dense, \
+                                                         (uint2*)values, (uint8_t*)meta, (uint8_t*)mask, pitch, src)
   switch (scheme) {
     case SDGP_RANDOM: SDGP_LAUNCH_T2(SDGP_RANDOM, false); break;
     case SDGP_MAGNITUDE: SDGP_LAUNCH_T2(SDGP_MAGNITUDE, false); break;
@@ -366,11 +395,10 @@ cudaError_t launch_m(int scheme, bool f16, const void* dO, int64_t nvec, int n, 
   return cudaGetLastError();
 }
 
-}  // namespace
-
-cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, int scheme,
-                         uint64_t seed, void* dense, void* values, void* meta, void* mask,
-                         cudaStream_t stream, int64_t k_pad, int dtype) {
+template <bool RELU>
+cudaError_t launch_prune_src(const void* dO, int64_t rows, int64_t K, int n, int m, int scheme, uint64_t seed, void* dense,
+                             void* values, void* meta, void* mask, cudaStream_t stream, int64_t k_pad, int dtype,
+                             ReluSource src) {
   const bool f16 = dtype == SDGP_FP16;
   const int64_t nvec = rows * (K / 8);
   OutPitch pitch = {(int)(K / 8), 0};
@@ -381,15 +409,16 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
   switch (m) {
     case 4:
       switch (n) {
-        case 1: return launch_m4_n<1>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
-        case 2: return launch_m4_n<2>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
-        case 3: return launch_m4_n<3>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
-        default: return launch_m4_n<4>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream);
+        case 1: return launch_m4_n<1, RELU>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream, src);
+        case 2: return launch_m4_n<2, RELU>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream, src);
+        case 3: return launch_m4_n<3, RELU>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream, src);
+        default: return launch_m4_n<4, RELU>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream, src);
       }
 #define SDGP_M_CASE(M)                                                                                     \
   case M:                                                                                                  \
-    if (n == 1) return launch_top2<M, 1>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream); \
-    if (n == 2) return launch_top2<M, 2>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream); \
+    if (n == 1) return launch_top2<M, 1, RELU>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream, src); \
+    if (n == 2) return launch_top2<M, 2, RELU>(scheme, f16, dO, nvec, seed, dense, values, meta, mask, pitch, stream, src); \
+    if (RELU) return cudaErrorInvalidValue; /* the generic kernel reads dL/dO itself */                      \
     return launch_m<M>(scheme, f16, dO, nvec, n, seed, dense, values, meta, mask, stream);
     SDGP_M_CASE(8)
     SDGP_M_CASE(16)
@@ -397,6 +426,22 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
 #undef SDGP_M_CASE
     default: return cudaErrorInvalidValue;
   }
+}
+
+}  // namespace
+
+cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, int scheme,
+                         uint64_t seed, void* dense, void* values, void* meta, void* mask,
+                         cudaStream_t stream, int64_t k_pad, int dtype) {
+  return launch_prune_src<false>(dO, rows, K, n, m, scheme, seed, dense, values, meta, mask, stream, k_pad, dtype,
+                                 ReluSource{nullptr, nullptr, 0u});
+}
+
+cudaError_t launch_relu_backward_prune(const void* dY, const void* act, int64_t rows, int64_t K, int n, int m, int scheme,
+                                       uint64_t seed, void* grad, void* dense, void* values, void* meta, void* mask,
+                                       cudaStream_t stream, int dtype) {
+  const ReluSource src = {(const uint4*)act, (uint4*)grad, dtype == SDGP_FP16 ? 0x03FF03FFu : 0x007F007Fu};
+  return launch_prune_src<true>(dY, rows, K, n, m, scheme, seed, dense, values, meta, mask, stream, 0, dtype, src);
 }
 
 }  // namespace sdgp

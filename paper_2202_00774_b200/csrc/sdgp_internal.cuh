@@ -14,6 +14,13 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
                          uint64_t seed, void* dense, void* values, void* meta, void* mask,
                          cudaStream_t stream, int64_t k_pad = 0, int dtype = SDGP_BF16);
 
+// The producer of dL/dO below a ReLU fused with its pruning: the gradient above the ReLU (dY) passes where the
+// activation `act` is positive; `grad` (optional) receives that unpruned dL/dO, the other outputs are
+// launch_prune's. n <= 2, or n == m (nothing pruned: only `grad` and the mask make sense then).
+cudaError_t launch_relu_backward_prune(const void* dY, const void* act, int64_t rows, int64_t K, int n, int m, int scheme,
+                                       uint64_t seed, void* grad, void* dense, void* values, void* meta, void* mask,
+                                       cudaStream_t stream, int dtype = SDGP_BF16);
+
 // Per-channel reading of the L1 rescale (channel.cu). sums: 2 * K floats (cleared by the call): the
 // column sums of |x| over all rows, then the same over the survivors of the magnitude function.
 cudaError_t launch_channel_sums(const void* dO, int64_t rows, int64_t K, int n, int m, int dtype, float* sums,

@@ -1,0 +1,103 @@
+"""sdgp_relu_backward_prune on the GPU against the oracle's producer (ReLU backward, then Algorithm 1): every output
+bit for bit, and the sparse contraction fed from it within the data-gradient tolerance."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2202_00774_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = 5e-3
+
+
+def dev16(a):
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
+
+
+def host16(t):
+    return t.cpu().numpy().view(np.uint16)
+
+
+def make(rows, K, seed, dtype=oracle.BF16):
+    rng = np.random.default_rng(seed)
+    to_bits = inputs.f32_to_bf16_bits if dtype == oracle.BF16 else (lambda x: x.astype(np.float16).view(np.uint16))
+    dY = to_bits(rng.laplace(size=(rows, K)).astype(np.float32))
+    act = to_bits(np.maximum(rng.standard_normal((rows, K)), 0.0).astype(np.float32))
+    # a few special activations: -0.0, NaN, +Inf, the smallest subnormal, a negative number
+    flat = act.reshape(-1)
+    special = [0x8000, 0x7FC0 if dtype == oracle.BF16 else 0x7E00, 0x7F80 if dtype == oracle.BF16 else 0x7C00, 0x0001, 0xBF80]
+    flat[rng.integers(0, flat.size, 400)] = np.resize(np.array(special, np.uint16), 400)
+    return dY, act
+
+
+@pytest.mark.parametrize("n,m", [(2, 4), (1, 4), (2, 8), (1, 8), (2, 16), (2, 32)])
+@pytest.mark.parametrize("scheme", [oracle.MAGNITUDE, oracle.RESCALED, oracle.RANDOM])
+def test_producer_outputs_bit_exact(n, m, scheme):
+    import paper_2202_00774_b200 as sdgp
+    rows, K = 1237, 160                 # ragged: not a whole number of thread blocks
+    dY, act = make(rows, K, seed=n * 10 + m)
+    grad = torch.full((rows, K), -1, dtype=torch.int16, device="cuda")
+    dense = torch.full((rows, K), -1, dtype=torch.int16, device="cuda")
+    values = torch.full((rows, K // 2), -1, dtype=torch.int16, device="cuda")
+    meta = torch.full((rows, K // 16), -1, dtype=torch.int16, device="cuda")
+    mask = torch.full((rows, K // 32), -1, dtype=torch.int32, device="cuda")
+    sdgp.sdgp_relu_backward_prune(dev16(dY), dev16(act), n, m, scheme, seed=77, grad=grad, dense=dense, values=values,
+                                  meta=meta, mask=mask)
+    ref = oracle.relu_backward_prune(dY, act, n, m, scheme, seed=77)
+    assert np.array_equal(host16(grad), ref["grad"])
+    assert np.array_equal(host16(dense), ref["dense"])
+    assert np.array_equal(host16(values), ref["values"])
+    assert np.array_equal(host16(meta), ref["meta"])
+    assert np.array_equal(mask.cpu().numpy().view(np.uint32), ref["mask"])
+
+
+def test_producer_binary16_and_plain_relu_backward():
+    import paper_2202_00774_b200 as sdgp
+    rows, K = 515, 128
+    dY, act = make(rows, K, seed=3, dtype=oracle.FP16)
+    grad = torch.full((rows, K), -1, dtype=torch.int16, device="cuda")
+    values = torch.full((rows, K // 2), -1, dtype=torch.int16, device="cuda")
+    meta = torch.full((rows, K // 16), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_relu_backward_prune(dev16(dY), dev16(act), 2, 4, sdgp.RESCALED_MAGNITUDE, seed=1, dtype=sdgp.FP16, grad=grad,
+                                  values=values, meta=meta)
+    ref = oracle.relu_backward_prune(dY, act, 2, 4, oracle.RESCALED, seed=1, dtype=oracle.FP16)
+    assert np.array_equal(host16(grad), ref["grad"])
+    assert np.array_equal(host16(values), ref["values"])
+    assert np.array_equal(host16(meta), ref["meta"])
+    # n == m: nothing pruned, the call is the ReLU backward alone
+    grad.fill_(-1)
+    sdgp.sdgp_relu_backward_prune(dev16(dY), dev16(act), 4, 4, sdgp.MAGNITUDE, dtype=sdgp.FP16, grad=grad)
+    assert np.array_equal(host16(grad), oracle.relu_backward(dY, act, oracle.FP16))
+
+
+def test_producer_feeds_the_sparse_contraction():
+    """ReLU backward + prune in one pass, then the contraction alone: a 1 x 1 convolution of ResNet-50's shape family."""
+    import paper_2202_00774_b200 as sdgp
+    B, HW, Cin, Cout = 4, 14, 256, 1024
+    rows = B * HW * HW
+    dY, act = make(rows, Cout, seed=8)
+    W = inputs.f32_to_bf16_bits((np.random.default_rng(1).standard_normal((Cout, Cin)) * (2.0 / Cin) ** 0.5).astype(np.float32))
+    values = torch.empty((rows, Cout // 2), dtype=torch.int16, device="cuda")
+    meta = torch.empty((rows, Cout // 16), dtype=torch.int16, device="cuda")
+    dD = torch.full((B, HW, HW, Cin), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_relu_backward_prune(dev16(dY), dev16(act), 2, 4, sdgp.MAGNITUDE, values=values, meta=meta)
+    sdgp.sdgp_spmm_conv2d(values.view(B, HW, HW, Cout // 2), meta.view(B, HW, HW, Cout // 16), dev16(W).view(Cout, 1, 1, Cin), dD, 1, 0)
+    assert sdgp.sdgp_last_device_error() == 0
+    ref = oracle.relu_backward_prune(dY, act, 2, 4, oracle.MAGNITUDE, want=("dense",))
+    want = oracle.dgrad_linear(ref["dense"], W)
+    got = inputs.bf16_bits_to_f32(host16(dD)).astype(np.float64).reshape(rows, Cin)
+    assert np.linalg.norm(got - want) <= TOL * np.linalg.norm(want)
+
+
+def test_producer_rejects_bad_arguments():
+    import paper_2202_00774_b200 as sdgp
+    x = torch.zeros((8, 64), dtype=torch.int16, device="cuda")
+    v = torch.zeros((8, 32), dtype=torch.int16, device="cuda")
+    with pytest.raises(sdgp.SdgpError) as e:
+        sdgp.sdgp_relu_backward_prune(x, x, 4, 8, sdgp.MAGNITUDE, values=v)      # 4:8 has no compressed form
+    assert e.value.status == 2
+    with pytest.raises(sdgp.SdgpError) as e:
+        sdgp.sdgp_relu_backward_prune(x, x, 0, 4, sdgp.MAGNITUDE, grad=x)
+    assert e.value.status == 1
