@@ -638,7 +638,7 @@ def run_layer_table(args):
 
     sampler = ClockSampler(torch.cuda.current_device())
     rows, launches = [], 0
-    tot = dict(two_pass=0.0, best=0.0, dense=0.0, flops=0.0, prune=0.0, prune_bytes=0.0, spmm=0.0)
+    tot = dict(two_pass=0.0, best=0.0, dense=0.0, flops=0.0, prune=0.0, prune_bytes=0.0, spmm=0.0, chain_sparse=0.0, chain_dense=0.0)
     for l, count in inputs.resnet50_layers(256):
         dO_h, W_h = inputs.conv_layer_tensors(l, seed=0)
         dO, Wt = dev16(dO_h), dev16(W_h)
@@ -669,6 +669,21 @@ def run_layer_table(args):
                                                                flags=sdgp.FLAG_FUSED))
         note("dense")
         t_dense = median_us(lambda: sdgp.sdgp_dgrad_conv2d(dO, Wt, dD, l.stride, l.pad, n, m, scheme, flags=sdgp.FLAG_DENSE))
+        # The backward chain through the ReLU above the layer: the producer forms dL/dO from the gradient above the
+        # ReLU and its activation and prunes it in the same pass (it also writes the unpruned dL/dO the weight
+        # gradient needs), against a plain ReLU backward followed by the dense twin. Both sides pay for the pass.
+        t_relu_prune = t_relu = None
+        if t_spmm is not None and n <= 2:
+            act = torch.randn(dO.shape, device="cuda").clamp_(min=0).to(torch.bfloat16).view(torch.int16)
+            grad = torch.empty_like(dO)
+            note("relu backward + prune")
+            t_relu_prune = median_us(lambda: sdgp.sdgp_relu_backward_prune(dO.view(-1, l.Cout), act.view(-1, l.Cout), n, m, scheme, 1234,
+                                                                          grad=grad.view(-1, l.Cout), values=vals, meta=metas))
+            note("relu backward")
+            t_relu = median_us(lambda: sdgp.sdgp_relu_backward_prune(dO.view(-1, l.Cout), act.view(-1, l.Cout), 4, 4, scheme, 0,
+                                                                    grad=grad.view(-1, l.Cout)))
+            launches += 2 * (reps + 3)
+            del act, grad
         launches += (reps + 3) * (2 + 1 + (1 if t_spmm else 0) + (1 if t_fused else 0) + 1)
         status = sdgp.sdgp_last_device_error()
         if status != 0:
@@ -684,7 +699,14 @@ def run_layer_table(args):
                      "speedup_spmm_alone": (t_dense / t_spmm) if t_spmm else None,
                      "bound": "tensor" if t_tensor >= t_hbm else "hbm",
                      "ideal_us": max(t_tensor, t_hbm), "frac_of_ideal_best": max(t_tensor, t_hbm) / best,
-                     "prune_gbs": pix * l.Cout * 3.125 / (t_prune * 1e-6) / 1e9})
+                     "prune_gbs": pix * l.Cout * 3.125 / (t_prune * 1e-6) / 1e9,
+                     "relu_prune_us": t_relu_prune, "relu_us": t_relu,
+                     "chain_sparse_us": (t_relu_prune + t_spmm) if t_relu_prune else None,
+                     "chain_dense_us": (t_relu + t_dense) if t_relu else None,
+                     "chain_speedup": ((t_relu + t_dense) / (t_relu_prune + t_spmm)) if t_relu_prune else None})
+        if t_relu_prune:
+            tot["chain_sparse"] += count * (t_relu_prune + t_spmm)
+            tot["chain_dense"] += count * (t_relu + t_dense)
         tot["two_pass"] += count * t_two
         tot["best"] += count * best
         tot["dense"] += count * t_dense
@@ -703,6 +725,10 @@ def run_layer_table(args):
                    "nm": args.nm, "scheme": args.scheme, "mode": "two_pass (per layer also fused and dense)",
                    "l2": "256 MB written between timed launches", "launch": "one launch per event pair, median"},
         "speedup_vs_dense": tot["dense"] / tot["two_pass"], "speedup_best_mode_vs_dense": tot["dense"] / tot["best"],
+        "relu_chain": {"what": "per layer [ReLU backward + prune in one pass, then the sparse contraction] against [plain ReLU "
+                               "backward, then the dense twin], over the shapes whose channel count needs no padding",
+                       "sparse_us": tot["chain_sparse"], "dense_us": tot["chain_dense"],
+                       "speedup": (tot["chain_dense"] / tot["chain_sparse"]) if tot["chain_sparse"] else None},
         "dense_tflops": tot["flops"] / (tot["dense"] * 1e-6) / 1e12,
         "prune_gbs": tot["prune_bytes"] / (tot["prune"] * 1e-6) / 1e9,
         "prune_frac_of_hbm": tot["prune_bytes"] / (tot["prune"] * 1e-6) / 1e9 / pk["hbm"],
