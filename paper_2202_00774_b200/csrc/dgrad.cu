@@ -217,11 +217,12 @@ __device__ __forceinline__ void fused_prune_eighth(const uint8_t* raw, int a_byt
 // whole pixel patch (full-line writes; pixels outside the tensor are clipped by the TMA unit).
 // With two staging slabs the store of one overlaps the packing of the next. `chunk` counts
 // slabs over the kernel's lifetime and picks the slab.
-template <int BN>
+// FIVE: dD's tensor map has five dimensions and (w0, h0, b0, e0) are coordinates 1..4.
+template <int BN, bool FIVE = false>
 __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* staging, int out_bufs,
                                                   const CUtensorMap* tmD, int n0, int w0, int h0, int b0,
                                                   bool tile_in_range, int row, bool issuer, uint32_t& chunk,
-                                                  uint64_t* first_slab_read, bool f16) {
+                                                  uint64_t* first_slab_read, bool f16, int e0 = 0) {
 #pragma unroll 1
   for (int c0 = 0; c0 < BN; c0 += 64, ++chunk) {
     uint32_t packed[32];
@@ -266,7 +267,8 @@ __device__ __forceinline__ void store_accumulator(uint32_t taddr, uint8_t* stagi
     ptx::fence_proxy_async_smem();
     ptx::named_bar_sync(1, 128);
     if (issuer && tile_in_range) {
-      ptx::tma_store_4d(tmD, buf, n0 + c0, w0, h0, b0);
+      if (FIVE) ptx::tma_store_5d(tmD, buf, n0 + c0, w0, h0, b0, e0);
+      else ptx::tma_store_4d(tmD, buf, n0 + c0, w0, h0, b0);
       ptx::bulk_commit_group();
     }
   }
@@ -644,7 +646,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 // 2 KB TMEM image per (tap, strip) from the raw metadata box of the A stage.
 
 constexpr int kHaloRows = 16;  // 8-pixel rows of a strip: the 128 rows of an accumulator
-constexpr int kHaloAStages = 2;
+constexpr int kHaloAStages = 4;  // at most: A stages in use are p.a_stages = 2, or 4 when the boxes are small (a power of two)
 // Warp roles of the fused whole-filter-reuse kernel (24 warps: registers are granted to warps in fours, and
 // 24 x 80 registers is what fits). Warp w runs on scheduler w % 4, and the thread that issues the MMAs
 // (warp 1) is what bounds these kernels, so the busy pruning warps keep off its scheduler: warp 0 streams W,
@@ -681,6 +683,14 @@ struct HaloParams {
                            // for images at most 8 pixels tall. Its 16 rows are ordered (pixel row, image), so a vertical
                            // tap is still one uniform row offset (tb rows).
   int img_h;               // rows of the A box: (th + R - 1) * tb, ordered (pixel row, image)
+  // Images 4 pixels wide: the 8 pixels of a strip row are the same pixel row of TWO images, a box row holds
+  // img_per_row = 2 * nt images side by side with no column halo (an image's neighbour is another image), and
+  // the horizontal taps are served by separate boxes: ss = S boxes per channel block, each fetched with its
+  // own column offset (the tensor map zero-fills beyond an image's edge), sb = 1 filter column per box.
+  // Otherwise img_per_row = 1, ss = 1, sb = S.
+  int split, img_per_row, ss, sb;
+  int k_uses;              // A boxes per tile set: k_blocks * ss
+  int a_stages, a_shift;   // A ring depth (2 or 4) and its log2
   int img_rows;            // pitch * img_h
   int w_stages;
   int meta_col, meta_shared, out_bufs;
@@ -811,7 +821,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   // to free its columns, which it does without anyone's help.
   ptx::launch_dependents();
 
-  const int taps = p.R * p.S;
+  const int taps = p.R * p.sb;  // filter taps served by one A box
   const int pair_stride = gridDim.x >> 1;
   const int first_pair = blockIdx.x >> 1;
   const int my_tiles = first_pair < p.units ? (p.units - first_pair + pair_stride - 1) / pair_stride : 0;
@@ -836,7 +846,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     w0 = (int)r * 8 * NT;
     divmod(q, (uint32_t)p.tiles_h, p.mg_tiles_h, q, r);
     h0 = (int)r * p.th;
-    b0 = (int)q * p.tb;
+    b0 = (int)q * p.tb * p.img_per_row;
     return in_range;
   };
 
@@ -846,7 +856,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const uint32_t a_tx = 2u * (uint32_t)(p.img_rows * 128);
       const uint32_t meta_tx = (uint32_t)(p.img_rows * 16);
       const uint32_t w_tx = 2u * (uint32_t)C::kTapBBytes;
-      const int a_uses = my_tiles * p.k_blocks;
+      const int a_uses = my_tiles * p.k_uses;
       int ia = 0, ast = 0;
       uint32_t aph = 0;
       // Loads the A box (and raw metadata) of stage use `ia`. blocking == false: only if the
@@ -857,18 +867,21 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         } else if (!ptx::mbar_test(&a_empty[ast], aph ^ 1u)) {
           return 0;
         }
-        const int lt = ia / p.k_blocks, kb = ia - lt * p.k_blocks;
+        const int lt = ia / p.k_uses, ku = ia - lt * p.k_uses;
+        const int kb = ku / p.ss, si = ku - kb * p.ss;  // channel block, filter column of the box (column-split mode)
         int n0, w0, h0, b0;
         locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
-        const int q0 = w0 + p.pad_w - (p.S - 1), p0 = h0 + p.pad_h - (p.R - 1);
+        const int q0 = w0 + p.pad_w - (p.sb - 1) - si, p0 = h0 + p.pad_h - (p.R - 1);
+        // coordinates: channel, pixel column, image within a box row, image group, pixel row
+        const int bg = b0 / p.img_per_row;
         if (rank == 0) ptx::mbar_arrive_expect_tx(&a_full[ast], a_tx);
         if (SPARSE) {
           ptx::mbar_arrive_expect_tx(&meta_full[ast], meta_tx);
-          ptx::tma_load_4d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, b0, p0);
+          ptx::tma_load_5d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, 0, bg, p0);
         }
-        ptx::tma_load_4d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, b0, p0);
+        ptx::tma_load_5d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, 0, bg, p0);
         ++ia;
-        if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
+        if (++ast == p.a_stages) { ast = 0; aph ^= 1u; }
         return 1;
       };
       bool alive = true;
@@ -878,16 +891,17 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int n0, w0_unused, h0_unused, b0_unused;
         locate(first_pair + lt * pair_stride, n0, w0_unused, h0_unused, b0_unused);
         n0 += n_half;
-        for (int kb = 0; alive && kb < p.k_blocks; ++kb, ++use) {
-          // (fused: the dense boxes are another warp's job, chunk by chunk; this thread streams W only)
+        for (int ku = 0; alive && ku < p.k_uses; ++ku, ++use) {
+          const int kb = ku / p.ss, si = ku - kb * p.ss;
+          // (fused: the pruning warps fetch dL/dO themselves; this thread streams W only)
           while (!FUSED && alive && ia <= use)
             if (issue_a(true) < 0) alive = false;
           for (int t = 0; alive && t < taps; ++t) {
             // the next A box goes out as soon as its stage is released, between W taps
-            if (!FUSED && ia < a_uses && ia < use + kHaloAStages && issue_a(false) < 0) { alive = false; break; }
+            if (!FUSED && ia < a_uses && ia < use + p.a_stages && issue_a(false) < 0) { alive = false; break; }
             if (!ptx::mbar_wait<kIdleWaitNs>(&w_empty[wst], wph ^ 1u, err, 0x180u + wst)) { alive = false; break; }
             if (rank == 0) ptx::mbar_arrive_expect_tx(&w_ready[wst], w_tx);
-            const int r = t / p.S, s = t - r * p.S;
+            const int r = t / p.sb, s = t - r * p.sb + si;
             const int ft = (p.r_first + p.r_step * r) * p.S_full + p.s_first + p.s_step * s;
 #pragma unroll
             for (int j = 0; j < C::kBoxes; ++j)
@@ -921,8 +935,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int off = dr * p.tb;  // box rows
         return ((off & 1) ? m1_off16 : 0u) + (uint32_t)((off >> 1) * 2 * p.pitch);
       };
-      const uint32_t a_first16 = (uint32_t)(((p.R - 1) * p.tb * p.pitch + (p.S - 1)) * 8);  // tap (0,0), in 16-byte units
-      const uint32_t a_rowstep16 = (uint32_t)((p.tb * p.pitch - (p.S - 1)) * 8);            // last tap of a filter row -> first of the next
+      const uint32_t a_first16 = (uint32_t)(((p.R - 1) * p.tb * p.pitch + (p.sb - 1)) * 8);  // tap (0,0), in 16-byte units
+      const uint32_t a_rowstep16 = (uint32_t)((p.tb * p.pitch - (p.sb - 1)) * 8);            // last tap of a filter row -> first of the next
       constexpr uint32_t kBStep = (uint32_t)((C::kKB / 4) * C::kRowB / 16);  // W rows of one MMA
       constexpr uint32_t kSlotCols = 4u * NT;                                // metadata columns of one W stage
       bool alive = true;
@@ -943,13 +957,13 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const uint32_t strips = strip_mask(lt);
         const bool all_strips = strips == ((1u << NT) - 1u);
         uint32_t accumulate = 0u;
-        for (int kb = 0; alive && kb < p.k_blocks; ++kb) {
+        for (int ku = 0; alive && ku < p.k_uses; ++ku) {
           if (!ptx::mbar_wait(&a_full[ast], aph, err, 0x300u + ast)) { alive = false; break; }
           if (SPARSE && !FUSED && !ptx::mbar_wait(&meta_ready[ast], aph, err, 0x340u + ast)) { alive = false; break; }
           uint32_t a_lo = a_lo0 + (uint32_t)ast * a_stage16 + a_first16;
-          int s = p.S, dr = p.R - 1;
+          int s = p.sb, dr = p.R - 1;
           const uint32_t e_stage = e_lo0 + (uint32_t)ast * e_stage16;
-          uint32_t e_lo = e_stage + meta_row16(dr) + (uint32_t)(p.S - 1);
+          uint32_t e_lo = e_stage + meta_row16(dr) + (uint32_t)(p.sb - 1);
           for (int t = 0; t < taps; ++t) {
             if (!ptx::mbar_wait(&w_ready[wst], wph, err, 0x380u + wst)) { alive = false; break; }
             ptx::tc_fence_after_sync();
@@ -984,13 +998,13 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             ptx::tc_commit_pair(&w_empty[wst], 3);
             accumulate = 1u;
             // next tap: one pixel to the left, or the end of the filter row above
-            if (--s == 0) { s = p.S; a_lo -= a_rowstep16; --dr; e_lo = e_stage + meta_row16(dr) + (uint32_t)(p.S - 1); }
+            if (--s == 0) { s = p.sb; a_lo -= a_rowstep16; --dr; e_lo = e_stage + meta_row16(dr) + (uint32_t)(p.sb - 1); }
             else { a_lo -= 8u; e_lo -= 1u; }
             if (++wst == WS) { wst = 0; wph ^= 1u; b_lo = b_lo0; mcol = 0; }
             else { b_lo += w_stage16; mcol += kSlotCols; }
           }
           if (alive) ptx::tc_commit_pair(&a_empty[ast], 3);
-          if (++ast == kHaloAStages) { ast = 0; aph ^= 1u; }
+          if (++ast == p.a_stages) { ast = 0; aph ^= 1u; }
         }
         if (alive) ptx::tc_commit_pair(&acc_full[acc], 3);
         if (++acc == 2) { acc = 0; cph ^= 1u; }
@@ -1004,11 +1018,11 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (SPARSE) {
       const int mw = warp - 2;
       const int lines0 = p.pairs0 * 2 * p.pitch, lines = (p.pairs0 + p.pairs1) * 2 * p.pitch;
-      const int a_uses = my_tiles * p.k_blocks;
+      const int a_uses = my_tiles * p.k_uses;
       constexpr int kBatch = 3;  // lines per lane whose loads are issued before any store
       for (int ause = 0; ause < a_uses; ++ause) {
-        const int ast = ause & 1;  // kHaloAStages == 2
-        if (!ptx::mbar_wait(&meta_full[ast], (uint32_t)(ause >> 1) & 1u, err, 0x500u + ast)) break;
+        const int ast = ause & (p.a_stages - 1);
+        if (!ptx::mbar_wait(&meta_full[ast], (uint32_t)(ause >> p.a_shift) & 1u, err, 0x500u + ast)) break;
         const uint8_t* raw = sEraw + ast * p.eraw_bytes;
         uint8_t* master = sMeta + ast * p.meta_bytes;
         for (int first = mw * 32 + lane; first < lines; first += 128 * kBatch) {
@@ -1056,17 +1070,17 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // number of this pruning warp, 0 .. kPruneWarps - 1: warps 2, 3, 8, then 10.. without those on scheduler 1
       const int pw = warp < 4 ? warp - 2 : warp == 8 ? 2 : 3 + (warp - 10) - ((warp - 9) >> 2);
       const int upb = (p.img_rows + 7) >> 3;  // units per box
-      const int a_uses = my_tiles * p.k_blocks;
+      const int a_uses = my_tiles * p.k_uses;
       const int row8 = lane >> 2, c = lane & 3;
       const uint32_t px_bytes = (uint32_t)p.Cout * 2u;
-      const int tb_shift = p.tb >> 1;  // tb is 1 or 2
+      const int tb_shift = p.tb == 4 ? 2 : p.tb >> 1;  // tb is 1, 2 or 4
       auto prune_units = [&](auto m_tag, auto n_tag, auto scheme_tag) {
         constexpr int M = decltype(m_tag)::value;
         constexpr int N = decltype(n_tag)::value;
         constexpr int SCHEME = decltype(scheme_tag)::value;
         // ---- load cursor: the unit whose loads go out next, and the box it lies in
-        int ia = 0, o = pw, lt = 0, kb = 0;
-        auto normalise = [&]() { while (o >= upb) { o -= upb; ++ia; if (++kb == p.k_blocks) { kb = 0; ++lt; } } };
+        int ia = 0, o = pw, lt = 0, ku = 0;  // ku: box of the tile set (channel block ku / ss, filter column ku % ss)
+        auto normalise = [&]() { while (o >= upb) { o -= upb; ++ia; if (++ku == p.k_uses) { ku = 0; ++lt; } } };
         normalise();
         int org_box = -1;             // box the origin below belongs to
         const uint8_t* org_ptr = p.a_dense;  // address of box pixel (0, 0), channel block kb, quarter c (may lie outside the tensor)
@@ -1074,26 +1088,34 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int org_b = 0;                // its image
         int64_t org_pix = 0;          // its linear pixel number (random keys)
         bool org_ok = false;
-        auto set_origin = [&](int box_lt, int box_kb, const uint8_t*& ptr, int& p0, int& q0, int& b0, int64_t& pix, bool& ok) {
+        auto set_origin = [&](int box_lt, int box_ku, const uint8_t*& ptr, int& p0, int& q0, int& b0, int64_t& pix, bool& ok) {
           int n0, w0, h0;
           ok = locate(first_pair + box_lt * pair_stride, n0, w0, h0, b0);
-          q0 = w0 + p.pad_w - (p.S - 1);
+          const int box_kb = box_ku / p.ss, si = box_ku - box_kb * p.ss;
+          q0 = w0 + p.pad_w - (p.sb - 1) - si;
           p0 = h0 + p.pad_h - (p.R - 1);
           pix = ((int64_t)b0 * p.P + p0) * p.Q + q0;
           ptr = p.a_dense + pix * (int64_t)px_bytes + box_kb * 256 + c * 16;
         };
+        // box pixel (box row br, column col) -> image offset, pixel row and pixel column relative to the origin
+        auto box_pixel = [&](int br, int col, int& ib, int& ih, int& iw) {
+          ih = br >> tb_shift;
+          ib = (br & (p.tb - 1)) * p.img_per_row;
+          iw = col;
+          if (p.split) { ib += col >> 2; iw = col & 3; }
+        };
         // The unit whose loads are in flight: its 64 bytes, its pixel row in the box, its box
         uint4 w[4];
-        int u_i = 0, u_ia = 0, u_kb = 0;
+        int u_i = 0, u_ia = 0, u_kb = 0;  // (u_kb: channel block)
         int64_t u_pix = 0;
         auto fetch = [&]() {
           if (org_box != ia) {
-            set_origin(lt, kb, org_ptr, org_p, org_q, org_b, org_pix, org_ok);
+            set_origin(lt, ku, org_ptr, org_p, org_q, org_b, org_pix, org_ok);
             org_box = ia;
             // ask the lines of the NEXT box into L2 now, a whole box ahead of their loads: 2 lines of 128
             // bytes per box pixel, dealt to the pruning threads
-            int nlt = lt, nkb = kb + 1;
-            if (nkb == p.k_blocks) { nkb = 0; ++nlt; }
+            int nlt = lt, nkb = ku + 1;
+            if (nkb == p.k_uses) { nkb = 0; ++nlt; }
             if (ia + 1 < a_uses) {
               const uint8_t* nptr;
               int np0, nq0, nb0;
@@ -1102,8 +1124,9 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               set_origin(nlt, nkb, nptr, np0, nq0, nb0, npix, nok);
               for (int line = pw * 32 + lane; line < 2 * p.img_rows; line += 32 * kPruneWarps) {
                 const int px = line >> 1;
-                const int br = (int)(((uint32_t)px * p.pitch_magic) >> 20), iw = px - br * p.pitch;  // box row, column
-                const int ih = br >> tb_shift, ib = br & (p.tb - 1);                                 // pixel row, image
+                const int br = (int)(((uint32_t)px * p.pitch_magic) >> 20);  // box row
+                int ib, ih, iw;
+                box_pixel(br, px - br * p.pitch, ib, ih, iw);
                 if (nok && nb0 + ib < p.B && (unsigned)(np0 + ih) < (unsigned)p.P && (unsigned)(nq0 + iw) < (unsigned)p.Q)
                   asm volatile("prefetch.global.L2 [%0];" ::"l"(nptr - c * 16 + (uint32_t)((ib * p.P + ih) * p.Q + iw) * px_bytes + (line & 1) * 128));
               }
@@ -1111,9 +1134,11 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
           u_i = 8 * o + row8;
           u_ia = ia;
+          const int kb = ku / p.ss;
           u_kb = kb;
-          const int br = (int)(((uint32_t)u_i * p.pitch_magic) >> 20), iw = u_i - br * p.pitch;  // box row, column
-          const int ih = br >> tb_shift, ib = br & (p.tb - 1);                                   // pixel row, image
+          const int br = (int)(((uint32_t)u_i * p.pitch_magic) >> 20);  // box row
+          int ib, ih, iw;
+          box_pixel(br, u_i - br * p.pitch, ib, ih, iw);
           const uint32_t off = (uint32_t)((ib * p.P + ih) * p.Q + iw);
           u_pix = org_pix + off;
           const bool valid = org_ok && u_i < p.img_rows && org_b + ib < p.B && (unsigned)(org_p + ih) < (unsigned)p.P &&
@@ -1149,12 +1174,13 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (boxes_seen <= cia) {  // the MMAs that read this stage's previous contents (box cia - 2) have completed
             bool ok = true;
             while (boxes_seen <= cia) {
-              if (!ptx::mbar_wait<kIdleWaitNs>(&a_empty[boxes_seen & 1], (((uint32_t)boxes_seen >> 1) & 1u) ^ 1u, err, 0x900u + (boxes_seen & 1))) { ok = false; break; }
+              const int bs = boxes_seen & (p.a_stages - 1);
+              if (!ptx::mbar_wait<kIdleWaitNs>(&a_empty[bs], (((uint32_t)boxes_seen >> p.a_shift) & 1u) ^ 1u, err, 0x900u + bs)) { ok = false; break; }
               ++boxes_seen;
             }
             if (!__all_sync(0xFFFFFFFFu, ok)) break;
           }
-          const int ast = cia & 1;
+          const int ast = cia & (p.a_stages - 1);
           uint2 out[4];
           uint32_t metaw;
           // (a group of M channels = vectors c + 4v of M / 8 neighbouring lanes c, same v)
@@ -1227,10 +1253,11 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ptx::tc_fence_after_sync();
 #pragma unroll
       for (int j = 0; j < NT; ++j)
-        store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * set_cols + j * BN), sOut,
-                              p.out_bufs, &tmD, n0, w0 + 8 * j, b0, h0, in_range && (w0 + 8 * j < p.W) && (strips & (1u << j)), row,
-                              issuer,
-                              chunk, (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr, p.f16 != 0);
+        // coordinates of strip j: pixel column, image within the box row, image group, pixel row
+        store_accumulator<BN, true>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * set_cols + j * BN), sOut, p.out_bufs,
+                                    &tmD, n0, p.split ? 0 : w0 + 8 * j, p.split ? 2 * j : 0, b0 / p.img_per_row,
+                                    in_range && (p.split || w0 + 8 * j < p.W) && (strips & (1u << j)), row, issuer, chunk,
+                                    (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr, p.f16 != 0, h0);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
@@ -1498,10 +1525,16 @@ bool plan_halo(HaloParams* p, int nt) {
   const int budget = kSmemLimit - kSmemSlack;
   {
     if (nt * BN > 256) return false;         // two tile sets of accumulators must fit the 512 TMEM columns
-    if (nt == 2 && p->W <= 8) return false;  // a second strip would be empty
+    p->split = (p->W == 4) ? 1 : 0;  // images 4 pixels wide: two per strip row, horizontal taps by separate boxes
+    if (!p->split && nt == 2 && p->W <= 8) return false;  // a second strip would be empty
     p->nt = nt;
-    p->pitch = 8 * nt + p->S - 1;
-    p->th = p->H <= 8 ? 8 : kHaloRows;
+    p->img_per_row = p->split ? 2 * nt : 1;
+    if (p->B % p->img_per_row != 0) return false;  // a box row of images must not reach past the batch
+    p->ss = p->split ? p->S : 1;
+    p->sb = p->split ? 1 : p->S;
+    p->k_uses = p->k_blocks * p->ss;
+    p->pitch = 8 * nt + p->sb - 1;
+    p->th = p->H <= 4 ? 4 : p->H <= 8 ? 8 : kHaloRows;
     p->tb = kHaloRows / p->th;
     p->img_h = (p->th + p->R - 1) * p->tb;
     p->img_rows = p->pitch * p->img_h;
@@ -1510,11 +1543,17 @@ bool plan_halo(HaloParams* p, int nt) {
     p->eraw_bytes = (SPARSE && !FUSED) ? round_up(p->img_rows * 16, 128) : 0;
     p->w_bytes = C::kTapBBytes;
     // vertical tap offset dr = 0 .. R-1 starts tb * dr box rows down: master (tb * dr) % 2, pair (tb * dr) / 2
-    p->pairs0 = 8 + (p->tb == 2 ? p->R - 1 : (p->R - 1) >> 1);
+    p->pairs0 = 8 + (p->tb == 1 ? (p->R - 1) >> 1 : (p->tb >> 1) * (p->R - 1));
     p->pairs1 = (p->tb == 1 && p->R > 1) ? 8 + ((p->R - 2) >> 1) : 0;
     p->m0_bytes = SPARSE ? p->pairs0 * 2 * p->pitch * 16 : 0;
     p->meta_bytes = SPARSE ? round_up((p->pairs0 + p->pairs1) * 2 * p->pitch * 16, 128) : 0;
-    const int fixed = kHaloAStages * (p->a_bytes + p->eraw_bytes + p->meta_bytes) + 1024;
+    // A ring: two stages; four where a box feeds few taps (column-split mode: R taps per box), so that the loads
+    // run further ahead of the MMAs, if that still leaves three W stages
+    p->a_stages = 2;
+    const int per_a = p->a_bytes + p->eraw_bytes + p->meta_bytes;
+    if (p->split && (budget - 4 * per_a - 1024 - kOutBytes) / p->w_bytes >= 3) p->a_stages = 4;
+    p->a_shift = p->a_stages == 4 ? 2 : 1;
+    const int fixed = p->a_stages * per_a + 1024;
     int out_bufs = 2;
     int w_stages = (budget - fixed - out_bufs * kOutBytes) / p->w_bytes;
     if (w_stages < 4) {
@@ -1538,17 +1577,18 @@ bool plan_halo(HaloParams* p, int nt) {
     if (w_stages < 3) return false;
     p->w_stages = w_stages;
     p->out_bufs = out_bufs;
-    p->off_eraw = kHaloAStages * p->a_bytes;
-    p->off_meta = p->off_eraw + kHaloAStages * p->eraw_bytes;
-    p->off_w = round_up(p->off_meta + kHaloAStages * p->meta_bytes, 1024);
+    p->off_eraw = p->a_stages * p->a_bytes;
+    p->off_meta = p->off_eraw + p->a_stages * p->eraw_bytes;
+    p->off_w = round_up(p->off_meta + p->a_stages * p->meta_bytes, 1024);
     p->pitch_magic = ((1u << 20) + (uint32_t)p->pitch - 1u) / (uint32_t)p->pitch;
     p->off_out = round_up(p->off_w + w_stages * p->w_bytes, 1024);
     p->off_bar = p->off_out + out_bufs * kOutBytes;
     p->smem_bytes = p->off_bar + 512 + 1024;
     if (p->smem_bytes > kSmemLimit) return false;
-    p->sets_w = (p->W + 8 * nt - 1) / (8 * nt);
+    p->sets_w = p->split ? 1 : (p->W + 8 * nt - 1) / (8 * nt);
     p->tiles_h = (p->H + p->th - 1) / p->th;
-    const int64_t m_sets = (int64_t)p->sets_w * p->tiles_h * ((p->B + p->tb - 1) / p->tb);
+    const int tile_imgs = p->tb * p->img_per_row;  // images of one tile set
+    const int64_t m_sets = (int64_t)p->sets_w * p->tiles_h * ((p->B + tile_imgs - 1) / tile_imgs);
     if (m_sets * p->tiles_n > 0x3FFFFFFF) return false;
     p->m_sets = (int)m_sets;
     p->pair_tiles = (int)((m_sets + 1) / 2) * p->tiles_n;
@@ -1573,7 +1613,9 @@ bool plan_halo(HaloParams* p, int nt) {
 // Whole-filter reuse pays when there is more than one tap and strips of 8 x 16 pixels cover the
 // image without much padding.
 bool halo_applies(int H, int W, int taps) {
-  if (taps < 2 || W < 8 || (H < 12 && H > 8) || H < 6) return false;
+  if (taps < 2) return false;
+  if (W == 4 && H >= 3 && H <= 4) return true;  // two images per strip row, four pixel rows of eight images per strip
+  if (W < 8 || (H < 12 && H > 8) || H < 6) return false;
   const int th = H <= 8 ? 8 : kHaloRows;  // images at most 8 pixels tall: strips of 8 rows of two images
   const int64_t covered = (int64_t)((W + 7) / 8 * 8) * ((H + th - 1) / th * th);
   return covered * 100 <= (int64_t)H * W * 135;
@@ -1588,23 +1630,29 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
   CUtensorMap tmA, tmE, tmB, tmD;
   const int P = view.P, Q = view.Q;
   const uint64_t CA = (SPARSE && !FUSED) ? (uint64_t)view.a_channels / 2 : (uint64_t)view.a_channels;
+  // Five dimensions: channel, pixel column, image within a box row (img_per_row of them: one, or the images that lie
+  // side by side in column-split mode), image group, pixel row. A box then holds its rows in (pixel row, image group)
+  // order and, inside a row, image after image.
+  const uint64_t ipr = (uint64_t)p.img_per_row, groups = (uint64_t)view.batch / ipr;
+  const uint32_t box_w = (uint32_t)(p.split ? 4 : p.pitch), box_h = (uint32_t)(p.img_h / p.tb);
   {
-    // dimensions ordered (channel, pixel column, image, pixel row): a box then holds its rows in (pixel row, image) order
-    const uint64_t dims[4] = {CA, (uint64_t)Q, (uint64_t)view.batch, (uint64_t)P};
-    const uint64_t strides[3] = {CA * 2, CA * 2 * Q * P, CA * 2 * Q};
+    const uint64_t img = CA * 2 * Q * P;
+    const uint64_t dims[5] = {CA, (uint64_t)Q, ipr, groups, (uint64_t)P};
+    const uint64_t strides[4] = {CA * 2, img, img * ipr, CA * 2 * Q};
     // (fused: the pruning warps read dL/dO with plain loads and this map goes unused)
-    const uint32_t box[4] = {64, (uint32_t)p.pitch, (uint32_t)p.tb, (uint32_t)(p.img_h / p.tb)};
-    if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+    const uint32_t box[5] = {64, box_w, (uint32_t)ipr, (uint32_t)p.tb, box_h};
+    if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
     tmE = tmA;
     p.a_dense = (const uint8_t*)A;
   }
   if (SPARSE && !FUSED) {
     const uint64_t CE = (uint64_t)view.a_channels / 16;
-    const uint64_t dims[4] = {CE, (uint64_t)Q, (uint64_t)view.batch, (uint64_t)P};
-    const uint64_t strides[3] = {CE * 2, CE * 2 * Q * P, CE * 2 * Q};
-    const uint32_t box[4] = {8, (uint32_t)p.pitch, (uint32_t)p.tb, (uint32_t)(p.img_h / p.tb)};
-    if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
+    const uint64_t img = CE * 2 * Q * P;
+    const uint64_t dims[5] = {CE, (uint64_t)Q, ipr, groups, (uint64_t)P};
+    const uint64_t strides[4] = {CE * 2, img, img * ipr, CE * 2 * Q};
+    const uint32_t box[5] = {8, box_w, (uint32_t)ipr, (uint32_t)p.tb, box_h};
+    if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 5, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
       return SDGP_ERR_CUDA;
   }
   {
@@ -1616,10 +1664,11 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
       return SDGP_ERR_CUDA;
   }
   {
-    const uint64_t dims[4] = {(uint64_t)p.Cin, (uint64_t)p.W, (uint64_t)p.B, (uint64_t)p.H};
-    const uint64_t strides[3] = {view.d_stride_w, view.d_stride_b, view.d_stride_h};
-    const uint32_t box[4] = {64, 8, (uint32_t)p.tb, (uint32_t)p.th};
-    if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, view.d_base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+    // one strip: 8 pixel columns of one image, or (column-split mode) the 4 columns of two neighbouring images
+    const uint64_t dims[5] = {(uint64_t)p.Cin, (uint64_t)p.W, ipr, (uint64_t)p.B / ipr, (uint64_t)p.H};
+    const uint64_t strides[4] = {view.d_stride_w, view.d_stride_b, view.d_stride_b * ipr, view.d_stride_h};
+    const uint32_t box[5] = {64, (uint32_t)(p.split ? 4 : 8), (uint32_t)(p.split ? 2 : 1), (uint32_t)p.tb, (uint32_t)p.th};
+    if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, view.d_base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
       return SDGP_ERR_CUDA;
   }
 
@@ -1731,7 +1780,11 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
       view.d_stride_h = (uint64_t)stride * W * Cin * 2;
       view.d_stride_b = (uint64_t)H * W * Cin * 2;
       sdgp_status st = SDGP_ERR_UNSUPPORTED;
-      if (halo_applies(Hs, Ws, p.R * p.S)) {
+      // Images 4 pixels wide take the whole-filter-reuse kernel (column-split mode) with a sparse A: fused, it prunes
+      // each box S times instead of R * S times; two-pass it measured the same as the general kernel; the dense twin
+      // measured slower there (one tile per CTA pair: set-up and the single epilogue dominate either way) and stays
+      // on the general kernel.
+      if (halo_applies(Hs, Ws, p.R * p.S) && (Ws != 4 || sparse)) {
         HaloParams hp = {};
         hp.B = B; hp.H = Hs; hp.W = Ws; hp.Cin = Cin; hp.Cout = Cout;
         hp.R = p.R; hp.S = p.S; hp.pad_h = p.pad_h; hp.pad_w = p.pad_w;

@@ -432,6 +432,12 @@ HALO_CASES = [
     (3, 6, 8, 128, 128, 3, 3, 1, 1),        # 6 pixel rows: two of the strip's eight are padding
     (2, 8, 8, 64, 128, 5, 5, 1, 2),         # 5 x 5 filter on 8 x 8 images
     (6, 8, 8, 128, 256, 3, 3, 1, 1),        # two channel blocks
+    (16, 4, 4, 512, 512, 3, 3, 1, 1),       # images 4 pixels wide: two per strip row, a box per filter column
+    (8, 4, 4, 64, 128, 3, 3, 1, 1),         # ... two strips (four images) per box row
+    (6, 4, 4, 128, 128, 3, 3, 1, 1),        # ... six images: the tile set of eight is partly empty
+    (4, 3, 4, 64, 128, 3, 3, 1, 1),         # ... three pixel rows
+    (10, 4, 4, 64, 128, 5, 5, 1, 2),        # ... 5 x 5 filter
+    (8, 8, 8, 64, 128, 3, 3, 2, 1),         # stride 2 on 8 x 8: 4 x 4 parity classes written through strided views
 ]
 
 
