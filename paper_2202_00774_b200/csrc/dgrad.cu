@@ -875,11 +875,14 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // coordinates: channel, pixel column, image within a box row, image group, pixel row
         const int bg = b0 / p.img_per_row;
         if (rank == 0) ptx::mbar_arrive_expect_tx(&a_full[ast], a_tx);
+        // (the tensor maps have the image-within-row dimension only in column-split mode)
         if (SPARSE) {
           ptx::mbar_arrive_expect_tx(&meta_full[ast], meta_tx);
-          ptx::tma_load_5d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, 0, bg, p0);
+          if (p.split) ptx::tma_load_5d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, 0, bg, p0);
+          else ptx::tma_load_4d(sEraw + ast * p.eraw_bytes, &tmE, &meta_full[ast], kb * 8, q0, b0, p0);
         }
-        ptx::tma_load_5d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, 0, bg, p0);
+        if (p.split) ptx::tma_load_5d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, 0, bg, p0);
+        else ptx::tma_load_4d_pair(sA + ast * p.a_bytes, &tmA, &a_full[ast], kb * 64, q0, b0, p0);
         ++ia;
         if (++ast == p.a_stages) { ast = 0; aph ^= 1u; }
         return 1;
@@ -1253,11 +1256,14 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ptx::tc_fence_after_sync();
 #pragma unroll
       for (int j = 0; j < NT; ++j)
-        // coordinates of strip j: pixel column, image within the box row, image group, pixel row
-        store_accumulator<BN, true>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * set_cols + j * BN), sOut, p.out_bufs,
-                                    &tmD, n0, p.split ? 0 : w0 + 8 * j, p.split ? 2 * j : 0, b0 / p.img_per_row,
-                                    in_range && (p.split || w0 + 8 * j < p.W) && (strips & (1u << j)), row, issuer, chunk,
-                                    (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr, p.f16 != 0, h0);
+        if (p.split)  // coordinates of strip j: pixel column, image within the box row, image group, pixel row
+          store_accumulator<BN, true>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * set_cols + j * BN), sOut, p.out_bufs,
+                                      &tmD, n0, 0, 2 * j, b0 / p.img_per_row, in_range && (strips & (1u << j)), row, issuer, chunk,
+                                      (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr, p.f16 != 0, h0);
+        else          // pixel column, image, pixel row
+          store_accumulator<BN>(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * set_cols + j * BN), sOut, p.out_bufs, &tmD,
+                                n0, w0 + 8 * j, b0, h0, in_range && (w0 + 8 * j < p.W) && (strips & (1u << j)), row, issuer, chunk,
+                                (p.meta_shared && j == 0) ? &meta_free[acc] : nullptr, p.f16 != 0);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
@@ -1630,29 +1636,36 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
   CUtensorMap tmA, tmE, tmB, tmD;
   const int P = view.P, Q = view.Q;
   const uint64_t CA = (SPARSE && !FUSED) ? (uint64_t)view.a_channels / 2 : (uint64_t)view.a_channels;
-  // Five dimensions: channel, pixel column, image within a box row (img_per_row of them: one, or the images that lie
-  // side by side in column-split mode), image group, pixel row. A box then holds its rows in (pixel row, image group)
-  // order and, inside a row, image after image.
+  // Dimensions: channel, pixel column, [column-split mode only: image within a box row (img_per_row images lie side by
+  // side),] image (group), pixel row. A box then holds its rows in (pixel row, image group) order and, inside a row,
+  // image after image.
   const uint64_t ipr = (uint64_t)p.img_per_row, groups = (uint64_t)view.batch / ipr;
   const uint32_t box_w = (uint32_t)(p.split ? 4 : p.pitch), box_h = (uint32_t)(p.img_h / p.tb);
-  {
-    const uint64_t img = CA * 2 * Q * P;
-    const uint64_t dims[5] = {CA, (uint64_t)Q, ipr, groups, (uint64_t)P};
-    const uint64_t strides[4] = {CA * 2, img, img * ipr, CA * 2 * Q};
-    // (fused: the pruning warps read dL/dO with plain loads and this map goes unused)
-    const uint32_t box[5] = {64, box_w, (uint32_t)ipr, (uint32_t)p.tb, box_h};
-    if (!encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
-      return SDGP_ERR_CUDA;
-    tmE = tmA;
-    p.a_dense = (const uint8_t*)A;
-  }
+  // builds the map of a [B, rows, cols, chan] tensor of 2-byte elements with the given strides and box extents
+  auto encode_nhwc = [&](CUtensorMap* tm, CUtensorMapDataType dt, const void* base, uint64_t chan, uint64_t cols, uint64_t rows,
+                         uint64_t images, uint64_t s_col, uint64_t s_row, uint64_t s_img, uint32_t b_chan, uint32_t b_col,
+                         uint32_t b_ipr, uint32_t b_grp, uint32_t b_row, CUtensorMapSwizzle swz) -> bool {
+    if (p.split) {
+      const uint64_t dims[5] = {chan, cols, ipr, images / ipr, rows};
+      const uint64_t strides[4] = {s_col, s_img, s_img * ipr, s_row};
+      const uint32_t box[5] = {b_chan, b_col, b_ipr, b_grp, b_row};
+      return encode(tm, dt, 5, base, dims, strides, box, swz);
+    }
+    const uint64_t dims[4] = {chan, cols, images, rows};
+    const uint64_t strides[3] = {s_col, s_img, s_row};
+    const uint32_t box[4] = {b_chan, b_col, b_grp, b_row};
+    return encode(tm, dt, 4, base, dims, strides, box, swz);
+  };
+  // (fused: the pruning warps read dL/dO with plain loads and the A map goes unused)
+  if (!encode_nhwc(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, A, CA, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch, CA * 2, CA * 2 * Q,
+                   CA * 2 * Q * P, 64, box_w, (uint32_t)ipr, (uint32_t)p.tb, box_h, CU_TENSOR_MAP_SWIZZLE_128B))
+    return SDGP_ERR_CUDA;
+  tmE = tmA;
+  p.a_dense = (const uint8_t*)A;
   if (SPARSE && !FUSED) {
     const uint64_t CE = (uint64_t)view.a_channels / 16;
-    const uint64_t img = CE * 2 * Q * P;
-    const uint64_t dims[5] = {CE, (uint64_t)Q, ipr, groups, (uint64_t)P};
-    const uint64_t strides[4] = {CE * 2, img, img * ipr, CE * 2 * Q};
-    const uint32_t box[5] = {8, box_w, (uint32_t)ipr, (uint32_t)p.tb, box_h};
-    if (!encode(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, 5, meta, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
+    if (!encode_nhwc(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT16, meta, CE, (uint64_t)Q, (uint64_t)P, (uint64_t)view.batch, CE * 2, CE * 2 * Q,
+                     CE * 2 * Q * P, 8, box_w, (uint32_t)ipr, (uint32_t)p.tb, box_h, CU_TENSOR_MAP_SWIZZLE_NONE))
       return SDGP_ERR_CUDA;
   }
   {
@@ -1663,14 +1676,11 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
                 C::kRowB == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
       return SDGP_ERR_CUDA;
   }
-  {
-    // one strip: 8 pixel columns of one image, or (column-split mode) the 4 columns of two neighbouring images
-    const uint64_t dims[5] = {(uint64_t)p.Cin, (uint64_t)p.W, ipr, (uint64_t)p.B / ipr, (uint64_t)p.H};
-    const uint64_t strides[4] = {view.d_stride_w, view.d_stride_b, view.d_stride_b * ipr, view.d_stride_h};
-    const uint32_t box[5] = {64, (uint32_t)(p.split ? 4 : 8), (uint32_t)(p.split ? 2 : 1), (uint32_t)p.tb, (uint32_t)p.th};
-    if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, view.d_base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
-      return SDGP_ERR_CUDA;
-  }
+  // dD, one strip per store: 8 pixel columns of one image, or (column-split mode) the 4 columns of two neighbouring images
+  if (!encode_nhwc(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, view.d_base, (uint64_t)p.Cin, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.B,
+                   view.d_stride_w, view.d_stride_h, view.d_stride_b, 64, (uint32_t)(p.split ? 4 : 8), 2, (uint32_t)p.tb,
+                   (uint32_t)p.th, CU_TENSOR_MAP_SWIZZLE_128B))
+    return SDGP_ERR_CUDA;
 
   static bool configured[kMaxDevices] = {};
   auto kernel = dgrad_halo_kernel<SPARSE, BN, NT, FUSED>;
