@@ -1111,6 +1111,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         uint4 w[4];
         int u_i = 0, u_ia = 0, u_kb = 0;  // (u_kb: channel block)
         int64_t u_pix = 0;
+        bool u_live = false;  // some pixel of the unit lies inside the tensor (halo rows above / below an image: none does)
         auto fetch = [&]() {
           if (org_box != ia) {
             set_origin(lt, ku, org_ptr, org_p, org_q, org_b, org_pix, org_ok);
@@ -1146,6 +1147,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           u_pix = org_pix + off;
           const bool valid = org_ok && u_i < p.img_rows && org_b + ib < p.B && (unsigned)(org_p + ih) < (unsigned)p.P &&
                              (unsigned)(org_q + iw) < (unsigned)p.Q;
+          u_live = __any_sync(0xFFFFFFFFu, valid);
 #pragma unroll
           for (int v = 0; v < 4; ++v) w[v] = make_uint4(0u, 0u, 0u, 0u);
           if (valid) {
@@ -1174,6 +1176,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (more) fetch();
         while (more) {
           const int i = u_i, cia = u_ia;
+          const bool live = u_live;
           if (boxes_seen <= cia) {  // the MMAs that read this stage's previous contents (box cia - 2) have completed
             bool ok = true;
             while (boxes_seen <= cia) {
@@ -1187,7 +1190,14 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           uint2 out[4];
           uint32_t metaw;
           // (a group of M channels = vectors c + 4v of M / 8 neighbouring lanes c, same v)
-          fused_prune_vectors<M, N, SCHEME>(w, u_pix * (p.Cout >> 3) + u_kb * 16 + c, 4, p.seed_lo, p.seed_hi, c & (M / 8 - 1), out, metaw);
+          if (live) {
+            fused_prune_vectors<M, N, SCHEME>(w, u_pix * (p.Cout >> 3) + u_kb * 16 + c, 4, p.seed_lo, p.seed_hi, c & (M / 8 - 1), out, metaw);
+          } else {
+            // a unit of padding only: zeros, whatever positions the metadata names (it names the pair (0, 1))
+#pragma unroll
+            for (int v = 0; v < 4; ++v) out[v] = make_uint2(0u, 0u);
+            metaw = 0x44444444u;
+          }
           // the registers of this unit are free: the loads of the next one go out before this one's stores
           more = ia < a_uses;
           if (more) fetch();
