@@ -53,6 +53,8 @@ def _load():
             lib.oracle_channel_scales.argtypes = [vp, i64, i64, i32, i32, i32, vp]
             lib.oracle_channel_scales.restype = i32
             lib.oracle_dgrad_conv2d_t.restype = i32
+            lib.oracle_dgrad_conv2d_grouped_t.argtypes = [vp, vp, vp] + [i32] * 10 + [vp, i64, i32]
+            lib.oracle_dgrad_conv2d_grouped_t.restype = i32
             lib.oracle_f32_to_f16.argtypes = [ctypes.c_float]
             lib.oracle_f32_to_f16.restype = ctypes.c_uint16
             lib.oracle_f16_to_f64.argtypes = [ctypes.c_uint16]
@@ -202,6 +204,24 @@ def dgrad_conv2d(dOp, W, H, Wd, stride=1, pad=0, pixel_index=None, dtype=BF16, k
                                        pad, _ptr(idx), count, dtype, _ptr(ks))
     if rc != 0:
         raise ValueError("oracle_dgrad_conv2d rejected its arguments")
+    return dD.reshape(B, H, Wd, Cin) if idx is None else dD
+
+
+def dgrad_conv2d_grouped(dOp, W, H, Wd, groups, stride=1, pad=0, pixel_index=None, dtype=BF16):
+    """dD (NHWC, fp64) of a grouped convolution: dOp NHWC ``[B,P,Q,Cout]``, W ``[Cout,R,S,Cin/groups]`` (uint16)."""
+    dOp, W = _u16(dOp), _u16(W)
+    B, P, Q, Cout = dOp.shape
+    Cout2, R, S, cin_g = W.shape
+    if Cout != Cout2 or P != (H + 2 * pad - R) // stride + 1 or Q != (Wd + 2 * pad - S) // stride + 1:
+        raise ValueError("shape mismatch")
+    Cin = cin_g * groups
+    idx = None if pixel_index is None else np.ascontiguousarray(pixel_index, dtype=np.int64)
+    count = B * H * Wd if idx is None else idx.shape[0]
+    dD = np.empty((count, Cin), np.float64)
+    rc = _load().oracle_dgrad_conv2d_grouped_t(_ptr(dOp), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S, stride,
+                                               pad, groups, _ptr(idx), count, dtype)
+    if rc != 0:
+        raise ValueError("oracle_dgrad_conv2d_grouped rejected its arguments")
     return dD.reshape(B, H, Wd, Cin) if idx is None else dD
 
 

@@ -451,6 +451,57 @@ int oracle_dgrad_conv2d(const uint16_t* dOp, const uint16_t* W, double* dD, int 
                                NULL);
 }
 
+/* Grouped convolution (the 3x3 convolutions of RegNetX, Section 4): the channels fall into `groups` groups;
+ * output channel co belongs to group co / (Cout / groups) and sees only the Cin / groups input channels of
+ * its group, so W is [Cout, R, S, Cin / groups] and
+ *   O[b,p,q,co] = sum_{r,s,cj} D[b, p*stride - pad + r, q*stride - pad + s, g(co) * Cin/groups + cj] * W[co,r,s,cj].
+ * The gradient w.r.t. the input therefore sums, for input channel ci of group g = ci / (Cin / groups), over
+ * the output channels of that group only:
+ *   dD[b,h,w,ci] = sum over (r,s), the (p,q) with p*stride - pad + r == h, q*stride - pad + s == w, and the
+ *                  co of group g, of dOp[b,p,q,co] * W[co,r,s, ci - g * Cin/groups].
+ * Pruning (Algorithm 1) runs along the output channels of dL/dO as for any other layer; it does not know
+ * about the convolution's groups. groups == 1 is oracle_dgrad_conv2d_t. */
+int oracle_dgrad_conv2d_grouped_t(const uint16_t* dOp, const uint16_t* W, double* dD, int B, int H, int Wd,
+                                  int Cin, int Cout, int R, int S, int stride, int pad, int groups,
+                                  const int64_t* pixel_index, int64_t n_pixels, int dtype) {
+  if (dtype != ORACLE_BF16 && dtype != ORACLE_FP16) return ORACLE_ERR_ARG;
+  if (!dOp || !W || !dD || stride < 1 || pad < 0 || R < 1 || S < 1 || groups < 1) return ORACLE_ERR_ARG;
+  if (Cin % groups != 0 || Cout % groups != 0) return ORACLE_ERR_ARG;
+  int P = (H + 2 * pad - R) / stride + 1;
+  int Q = (Wd + 2 * pad - S) / stride + 1;
+  if (P < 1 || Q < 1) return ORACLE_ERR_ARG;
+  const int cin_g = Cin / groups, cout_g = Cout / groups;
+  int64_t count = pixel_index ? n_pixels : (int64_t)B * H * Wd;
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < count; ++i) {
+    int64_t pix = pixel_index ? pixel_index[i] : i;
+    int w = (int)(pix % Wd);
+    int h = (int)((pix / Wd) % H);
+    int b = (int)(pix / ((int64_t)Wd * H));
+    for (int ci = 0; ci < Cin; ++ci) {
+      const int g = ci / cin_g, cj = ci - g * cin_g;
+      double acc = 0.0;
+      for (int r = 0; r < R; ++r) {
+        int hp = h + pad - r;
+        if (hp < 0 || hp % stride != 0) continue;
+        int p = hp / stride;
+        if (p >= P) continue;
+        for (int s = 0; s < S; ++s) {
+          int wq = w + pad - s;
+          if (wq < 0 || wq % stride != 0) continue;
+          int q = wq / stride;
+          if (q >= Q) continue;
+          const uint16_t* grad = dOp + (((int64_t)b * P + p) * Q + q) * Cout;
+          for (int co = g * cout_g; co < (g + 1) * cout_g; ++co)
+            acc += elem_to_f64(grad[co], dtype) * elem_to_f64(W[(((int64_t)co * R + r) * S + s) * cin_g + cj], dtype);
+        }
+      }
+      dD[i * Cin + ci] = acc;
+    }
+  }
+  return ORACLE_OK;
+}
+
 /* Direct forward convolution in fp64 on fp64 inputs; used only by the adjoint
  * identity test <conv(D), G> == <D, dgrad(G)>. */
 int oracle_conv2d_forward_f64(const double* D, const uint16_t* W, double* O, int B, int H, int Wd,

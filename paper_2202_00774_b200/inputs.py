@@ -97,6 +97,7 @@ class ConvLayer:
     S: int
     stride: int
     pad: int
+    groups: int = 1   # grouped convolution: W is [Cout, R, S, Cin / groups]
 
     @property
     def P(self) -> int:
@@ -109,13 +110,13 @@ class ConvLayer:
     @property
     def dense_macs(self) -> int:
         """True multiply-accumulates of the dense data-gradient contraction."""
-        return self.B * self.P * self.Q * self.Cout * self.R * self.S * self.Cin
+        return self.B * self.P * self.Q * self.Cout * self.R * self.S * (self.Cin // self.groups)
 
     def dO_shape(self):
         return (self.B, self.P, self.Q, self.Cout)
 
     def W_shape(self):
-        return (self.Cout, self.R, self.S, self.Cin)
+        return (self.Cout, self.R, self.S, self.Cin // self.groups)
 
     def dD_shape(self):
         return (self.B, self.H, self.W, self.Cin)
@@ -182,10 +183,30 @@ def resnet18_layers(batch: int = 256) -> List[ConvLayer]:
     return out
 
 
+def regnetx_400mf_layers(batch: int = 256) -> List[ConvLayer]:
+    """Distinct convolutions of the RegNetX-400MF body (Section 4 trains it on ImageNet): stage widths 32, 64,
+    160, 384 at 56, 28, 14, 7 pixels, group width 16 (so 2, 4, 10, 24 groups), bottleneck ratio 1. A block is
+    1x1 -> grouped 3x3 -> 1x1; the first block of a stage takes the previous stage's width at twice the
+    resolution, strides in its 3x3 and has a 1x1 stride-2 shortcut."""
+    out = []
+    prev = 32
+    for stage, (hw, ch, depth) in enumerate([(56, 32, 1), (28, 64, 2), (14, 160, 7), (7, 384, 12)], start=1):
+        tag = "rx_s%d_" % stage
+        g = ch // 16
+        out.append(ConvLayer(tag + "1x1_%dto%d_at%d" % (prev, ch, 2 * hw), batch, 2 * hw, 2 * hw, prev, ch, 1, 1, 1, 0))
+        out.append(ConvLayer(tag + "3x3s2g%d_%d_at%d" % (g, ch, 2 * hw), batch, 2 * hw, 2 * hw, ch, ch, 3, 3, 2, 1, g))
+        out.append(ConvLayer(tag + "projs2_%dto%d_at%d" % (prev, ch, 2 * hw), batch, 2 * hw, 2 * hw, prev, ch, 1, 1, 2, 0))
+        out.append(ConvLayer(tag + "1x1_%dto%d_at%d" % (ch, ch, hw), batch, hw, hw, ch, ch, 1, 1, 1, 0))
+        if depth > 1:
+            out.append(ConvLayer(tag + "3x3g%d_%d_at%d" % (g, ch, hw), batch, hw, hw, ch, ch, 3, 3, 1, 1, g))
+        prev = ch
+    return out
+
+
 def conv_layer_tensors(layer: ConvLayer, seed: int):
     """(dO, W) for one layer: dO = ReLU-masked Laplace, W = He-normal N(0, 2/(R*S*Cin))."""
     dO = relu_masked_laplace_bf16(layer.dO_shape(), seed, stream=1)
-    W = normal_bf16(layer.W_shape(), float(np.sqrt(2.0 / (layer.R * layer.S * layer.Cin))), seed, stream=2)
+    W = normal_bf16(layer.W_shape(), float(np.sqrt(2.0 / (layer.R * layer.S * (layer.Cin // layer.groups)))), seed, stream=2)
     return dO, W
 
 
