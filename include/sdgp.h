@@ -183,6 +183,29 @@ sdgp_status sdgp_relu_backward_prune(const void* dY, const void* act, int64_t ro
                                      sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad, void* dOp_dense,
                                      void* values, void* meta, void* mask, void* stream);
 
+/* Data gradient of a GROUPED convolution (the 3x3 convolutions of RegNetX, one of the networks of Section 4; the
+ * contraction is Section 2.1 / Fig. 2 and Section 3.1 / Fig. 3 with the sum over output channels restricted to the
+ * group of the input channel): output channel co belongs to group co / (Cout/groups) and is connected to the
+ * Cin/groups input channels of that group only, so
+ *   dD[b,h,w,ci] = sum over r, s, the (p, q) with p*stride - pad + r == h and q*stride - pad + s == w, and the co of
+ *                  group ci / (Cin/groups), of prune(dO)[b,p,q,co] * W[co,r,s, ci % (Cin/groups)].
+ *   dO [B,P,Q,Cout], W [Cout,R,S,Cin/groups], dD [B,H,Wd,Cin], element type `dtype`. Algorithm 1 runs along Cout as
+ *   for any layer (the groups of m know nothing of the convolution's groups).
+ * groups == 1 is an ordinary convolution; unlike sdgp_dgrad_conv2d this entry point also takes channel counts that
+ * are not multiples of 64 (RegNetX-400MF has 32 and 160): Cout % 16 == 0 when anything is pruned (% 8 otherwise),
+ * (Cin/groups) % 8 == 0. flags: SDGP_FLAG_TWO_PASS, SDGP_FLAG_DENSE, SDGP_FLAG_MASKED, and SDGP_FLAG_FUSED where both
+ * channel counts are multiples of 64 (SDGP_ERR_UNSUPPORTED otherwise). Other requirements as sdgp_dgrad_conv2d.
+ * The call first writes the filters as the block-diagonal filters of an ordinary convolution, channel counts
+ * rounded up to multiples of 64, into the workspace (read again by the contraction on `stream`), then runs the
+ * ordinary kernels on them; dL/dO and dD are used as stored, without padded copies.
+ * Workspace: sdgp_workspace_size_conv2d_grouped() bytes (every mode needs one), 256-byte aligned, owned by the caller. */
+size_t sdgp_workspace_size_conv2d_grouped(int B, int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
+                                          int groups, uint32_t flags);
+sdgp_status sdgp_dgrad_conv2d_grouped(const void* dO, const void* W, void* dD, int B, int H, int Wd, int Cin, int Cout,
+                                      int R, int S, int stride, int pad, int groups, int n, int m, sdgp_scheme scheme,
+                                      uint64_t seed, sdgp_dtype dtype, void* workspace, size_t workspace_bytes,
+                                      uint32_t flags, void* stream);
+
 /* The factors of SDGP_FLAG_CHANNEL on their own: dO [rows, K] of element type `dtype`, groups of m along K,
  * magnitude function with n survivors (any 1 <= n <= m, m in {4, 8, 16, 32}, K % m == 0, K % 8 == 0).
  * `out` is a device array of 3 * K floats: [0, K) the factors, [K, 2K) the column sums of |dO| over all rows,

@@ -20,7 +20,8 @@ BF16, FP16 = 0, 1   # sdgp_dtype
 EXPORTS = ["sdgp_prune", "sdgp_dgrad_linear", "sdgp_dgrad_conv2d", "sdgp_spmm_linear", "sdgp_spmm_conv2d",
            "sdgp_prune_typed", "sdgp_dgrad_linear_typed", "sdgp_dgrad_conv2d_typed", "sdgp_spmm_linear_typed",
            "sdgp_spmm_conv2d_typed", "sdgp_channel_scales", "sdgp_relu_backward_prune", "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
-           "sdgp_workspace_size_linear", "sdgp_workspace_size_conv2d", "sdgp_last_device_error",
+           "sdgp_workspace_size_linear", "sdgp_workspace_size_conv2d", "sdgp_workspace_size_conv2d_grouped",
+           "sdgp_dgrad_conv2d_grouped", "sdgp_last_device_error",
            "sdgp_status_string"]
 
 _lib = None
@@ -74,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.sdgp_workspace_size_linear.restype = sz
         L.sdgp_workspace_size_conv2d.argtypes = [i32] * 9 + [u32]
         L.sdgp_workspace_size_conv2d.restype = sz
+        L.sdgp_workspace_size_conv2d_grouped.argtypes = [i32] * 10 + [u32]
+        L.sdgp_workspace_size_conv2d_grouped.restype = sz
+        L.sdgp_dgrad_conv2d_grouped.argtypes = [vp, vp, vp] + [i32] * 10 + [i32, i32, i32, u64, i32, vp, sz, u32, vp]
+        L.sdgp_dgrad_conv2d_grouped.restype = i32
         L.sdgp_last_device_error.argtypes = []
         L.sdgp_last_device_error.restype = i32
         L.sdgp_selftest_bounded_wait.argtypes = [vp]
@@ -225,6 +230,23 @@ def sdgp_dgrad_conv2d_typed(dO, W, dD, stride, pad, n, m, scheme, seed, dtype, w
     _check(lib().sdgp_dgrad_conv2d_typed(_ptr(dO), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S, stride, pad, n, m,
                                          scheme, seed, dtype, _ptr(workspace), ws_bytes, flags, _stream()),
            "sdgp_dgrad_conv2d_typed")
+
+
+def sdgp_workspace_size_conv2d_grouped(B, H, Wd, Cin, Cout, R, S, stride, pad, groups, flags=FLAG_TWO_PASS) -> int:
+    return int(lib().sdgp_workspace_size_conv2d_grouped(B, H, Wd, Cin, Cout, R, S, stride, pad, groups, flags))
+
+
+def sdgp_dgrad_conv2d_grouped(dO, W, dD, stride, pad, groups, n, m, scheme, seed=0, dtype=BF16, workspace=None,
+                              flags=FLAG_TWO_PASS):
+    """``sdgp_dgrad_conv2d_grouped``: dO NHWC [B,P,Q,Cout], W [Cout,R,S,Cin/groups], dD NHWC [B,H,W,Cin]."""
+    for t, name in ((dO, "dO"), (W, "W"), (dD, "dD"), (workspace, "workspace")):
+        _dev(t, name)
+    B, H, Wd, Cin = dD.shape
+    Cout, R, S, _ = W.shape
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().sdgp_dgrad_conv2d_grouped(_ptr(dO), _ptr(W), _ptr(dD), B, H, Wd, Cin, Cout, R, S, stride, pad, groups,
+                                           n, m, scheme, seed, dtype, _ptr(workspace), ws_bytes, flags, _stream()),
+           "sdgp_dgrad_conv2d_grouped")
 
 
 def sdgp_spmm_linear_typed(values, meta, W, dD, dtype):

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsdgp.so")
-SOURCES = ["prune.cu", "dgrad.cu", "api.cu", "static_scratch.cu", "channel.cu"]
+SOURCES = ["prune.cu", "dgrad.cu", "api.cu", "static_scratch.cu", "channel.cu", "grouped.cu"]
 HEADERS = ["ptx.cuh", "sdgp_internal.cuh", "prune_core.cuh", os.path.join("..", "..", "include", "sdgp.h")]
 
 

@@ -228,6 +228,86 @@ sdgp_status sdgp_dgrad_conv2d_typed(const void* dO, const void* W, void* dD, int
   return sdgp::launch_dgrad(true, c.values, c.meta, W, dD, B, H, Wd, Cin, Cout, R, S, stride, pad, s, nullptr, dt);
 }
 
+// Grouped convolution: the expanded (block-diagonal, channel-padded) filters sit at the start of the workspace
+static int round64(int c) { return (c + 63) / 64 * 64; }
+static size_t grouped_weights_bytes(int Cin, int Cout, int R, int S) {
+  return round_up((size_t)round64(Cout) * R * S * round64(Cin) * 2, 256);
+}
+
+size_t sdgp_workspace_size_conv2d_grouped(int B, int H, int Wd, int Cin, int Cout, int R, int S, int stride, int pad,
+                                          int groups, uint32_t flags) {
+  if (flags > SDGP_FLAG_MASKED || stride < 1 || groups < 1 || Cin < 1 || Cout < 1 || R < 1 || S < 1) return 0;
+  const int64_t P = (H + 2 * pad - R) / stride + 1, Q = (Wd + 2 * pad - S) / stride + 1;
+  if (B <= 0 || P <= 0 || Q <= 0) return 0;
+  const size_t w = grouped_weights_bytes(Cin, Cout, R, S);
+  if (flags == SDGP_FLAG_MASKED) return w + round_up((size_t)B * P * Q * Cout * 2, 256);
+  if (flags == SDGP_FLAG_TWO_PASS) return w + carve_compressed(nullptr, (int64_t)B * P * Q * pad128(Cout)).bytes;
+  return w;
+}
+
+sdgp_status sdgp_dgrad_conv2d_grouped(const void* dO, const void* W, void* dD, int B, int H, int Wd, int Cin, int Cout,
+                                      int R, int S, int stride, int pad, int groups, int n, int m, sdgp_scheme scheme,
+                                      uint64_t seed, sdgp_dtype dtype, void* workspace, size_t workspace_bytes,
+                                      uint32_t flags, void* stream) {
+  if (!valid_dtype(dtype)) return SDGP_ERR_INVALID_ARG;
+  if (B < 0 || H < 0 || Wd < 0 || Cin < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0 || groups < 1)
+    return SDGP_ERR_INVALID_ARG;
+  if (Cin % groups != 0 || Cout % groups != 0) return SDGP_ERR_INVALID_ARG;
+  if (flags > SDGP_FLAG_MASKED) return SDGP_ERR_INVALID_ARG;
+  if (stride > 2) return SDGP_ERR_UNSUPPORTED;
+  if (pad > R - 1 || pad > S - 1) return SDGP_ERR_UNSUPPORTED;
+  if ((Cin / groups) % 8 != 0 || Cout % 8 != 0) return SDGP_ERR_UNSUPPORTED;  // 16-byte vectors and tensor-map strides
+  const bool prunes = flags != SDGP_FLAG_DENSE && n != m;
+  if (flags != SDGP_FLAG_DENSE) {
+    sdgp_status st = check_prune_args(0, Cout, n, m, (int)scheme);
+    if (st != SDGP_OK) return st;
+    if (n > 2 && n != m && flags != SDGP_FLAG_MASKED) return SDGP_ERR_UNSUPPORTED;  // not 2:4-compatible
+    if (prunes && Cout % 16 != 0) return SDGP_ERR_ALIGNMENT;
+  }
+  if ((int64_t)B * H * Wd == 0) return SDGP_OK;
+  const int64_t P = (H + 2 * pad - R) / stride + 1, Q = (Wd + 2 * pad - S) / stride + 1;
+  if (P < 1 || Q < 1) return SDGP_ERR_INVALID_ARG;
+  if (!dO || !W || !dD) return SDGP_ERR_INVALID_ARG;
+  if (!aligned16(dO) || !aligned16(W) || !aligned16(dD)) return SDGP_ERR_ALIGNMENT;
+  const int cin_k = round64(Cin), cout_k = round64(Cout);  // the channel counts the kernels tile by
+  const size_t w_bytes = grouped_weights_bytes(Cin, Cout, R, S);
+  if (!workspace || workspace_bytes < sdgp_workspace_size_conv2d_grouped(B, H, Wd, Cin, Cout, R, S, stride, pad, groups,
+                                                                          prunes ? flags : SDGP_FLAG_DENSE))
+    return SDGP_ERR_WORKSPACE;
+  if (((uintptr_t)workspace & 255u) != 0) return SDGP_ERR_ALIGNMENT;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int dt = (int)dtype;
+  void* w_full = workspace;
+  void* rest = (uint8_t*)workspace + w_bytes;
+  if (sdgp::launch_expand_grouped_weights(W, Cout, R * S, Cin, groups, cout_k, cin_k, w_full, s) != cudaSuccess)
+    return SDGP_ERR_CUDA;
+  const sdgp::StoredChannels dense_view = {Cout != cout_k ? Cout : 0, Cin != cin_k ? Cin : 0};
+  const sdgp::StoredChannels sparse_view = {0, dense_view.d};  // a compressed dL/dO is padded by the prune kernel
+  const bool padded = dense_view.a != 0 || dense_view.d != 0;
+  if (!prunes)
+    return sdgp::launch_dgrad(false, dO, nullptr, w_full, dD, B, H, Wd, cin_k, cout_k, R, S, stride, pad, s, nullptr, dt,
+                              padded ? &dense_view : nullptr);
+  const int64_t rows = (int64_t)B * P * Q;
+  if (flags == SDGP_FLAG_MASKED) {
+    if (sdgp::launch_prune(dO, rows, Cout, n, m, (int)scheme, seed, rest, nullptr, nullptr, nullptr, s, 0, dt) != cudaSuccess)
+      return SDGP_ERR_CUDA;
+    return sdgp::launch_dgrad(false, rest, nullptr, w_full, dD, B, H, Wd, cin_k, cout_k, R, S, stride, pad, s, nullptr, dt,
+                              padded ? &dense_view : nullptr);
+  }
+  if (flags == SDGP_FLAG_FUSED) {
+    if (padded) return SDGP_ERR_UNSUPPORTED;  // the in-kernel prune reads dL/dO by the channel count it tiles by
+    if (dtype == SDGP_FP16 && scheme == SDGP_RESCALED_MAGNITUDE) return SDGP_ERR_UNSUPPORTED;
+    const sdgp::FusedPrune fp = {n, m, (int)scheme, seed};
+    return sdgp::launch_dgrad(true, dO, nullptr, w_full, dD, B, H, Wd, cin_k, cout_k, R, S, stride, pad, s, &fp, dt);
+  }
+  const int64_t Cpad = pad128(Cout);
+  const Carve c = carve_compressed(rest, rows * Cpad);
+  if (sdgp::launch_prune(dO, rows, Cout, n, m, (int)scheme, seed, nullptr, c.values, c.meta, nullptr, s, Cpad, dt) != cudaSuccess)
+    return SDGP_ERR_CUDA;
+  return sdgp::launch_dgrad(true, c.values, c.meta, w_full, dD, B, H, Wd, cin_k, cout_k, R, S, stride, pad, s, nullptr, dt,
+                            sparse_view.d ? &sparse_view : nullptr);
+}
+
 sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,
                               int64_t N, int n, int m, sdgp_scheme scheme, uint64_t seed,
                               void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {

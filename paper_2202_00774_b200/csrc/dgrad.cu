@@ -1462,6 +1462,7 @@ bool plan(DgradParams* p) {
 struct DgradView {
   int P, Q, batch;
   int a_channels;
+  int d_channels;                 // channels per pixel of dD as stored (<= Cin: a store is clipped there)
   int64_t w_cols;                 // R_full * S_full * Cin
   void* d_base;
   uint64_t d_stride_w, d_stride_h, d_stride_b;  // bytes
@@ -1503,7 +1504,7 @@ sdgp_status launch_cfg(const void* A, const void* meta, const void* Wt, const Dg
       return SDGP_ERR_CUDA;
   }
   {
-    const uint64_t dims[4] = {(uint64_t)p.Cin, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.B};
+    const uint64_t dims[4] = {(uint64_t)view.d_channels, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.B};
     const uint64_t strides[3] = {view.d_stride_w, view.d_stride_h, view.d_stride_b};
     const uint32_t box[4] = {64, (uint32_t)p.TW, (uint32_t)p.TH, (uint32_t)p.TB};
     if (!encode(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, view.d_base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
@@ -1687,7 +1688,7 @@ sdgp_status launch_halo_nt(const void* A, const void* meta, const void* Wt, cons
       return SDGP_ERR_CUDA;
   }
   // dD, one strip per store: 8 pixel columns of one image, or (column-split mode) the 4 columns of two neighbouring images
-  if (!encode_nhwc(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, view.d_base, (uint64_t)p.Cin, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.B,
+  if (!encode_nhwc(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, view.d_base, (uint64_t)view.d_channels, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.B,
                    view.d_stride_w, view.d_stride_h, view.d_stride_b, 64, (uint32_t)(p.split ? 4 : 8), 2, (uint32_t)p.tb,
                    (uint32_t)p.th, CU_TENSOR_MAP_SWIZZLE_128B))
     return SDGP_ERR_CUDA;
@@ -1739,7 +1740,10 @@ sdgp_status launch_halo(const void* A, const void* meta, const void* Wt, const D
 // (m = 4, n = fused->n in {1, 2}); no compressed tensor exists in global memory.
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
                          int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
-                         const FusedPrune* fused, int dtype) {
+                         const FusedPrune* fused, int dtype, const StoredChannels* stored) {
+  if (fused && stored) return SDGP_ERR_UNSUPPORTED;  // the pruning warps address dL/dO by the channel count they tile by
+  if (stored && (stored->a < 0 || stored->a > Cout || stored->a % 8 != 0 || stored->d < 0 || stored->d > Cin || stored->d % 8 != 0))
+    return SDGP_ERR_INVALID_ARG;
   if (fused && (!sparse || fused->n < 1 || fused->n > 2)) return SDGP_ERR_UNSUPPORTED;
   if (fused && fused->m != 4 && fused->m != 8 && fused->m != 16 && fused->m != 32) return SDGP_ERR_UNSUPPORTED;
   if (dtype != SDGP_BF16 && dtype != SDGP_FP16) return SDGP_ERR_INVALID_ARG;
@@ -1756,15 +1760,17 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
 
   DgradView view;
   view.P = P; view.Q = Q; view.batch = B;
-  view.a_channels = (sparse && !fused) ? (Cout + 127) / 128 * 128 : Cout;
+  view.a_channels = (sparse && !fused) ? (Cout + 127) / 128 * 128 : (stored && stored->a) ? stored->a : Cout;
+  view.d_channels = (stored && stored->d) ? stored->d : Cin;
   view.w_cols = (int64_t)R * S * Cin;
+  const size_t Cd = (size_t)view.d_channels;
 
   // Output parities that no tap reaches are zero: clear dD first if there is any such class.
   bool any_empty = false;
   for (int ph = 0; ph < stride; ++ph)
     for (int pw = 0; pw < stride; ++pw)
       if ((ph + pad) % stride >= R || (pw + pad) % stride >= S) any_empty = true;
-  if (any_empty && cudaMemsetAsync(dD, 0, (size_t)B * H * W * Cin * 2, stream) != cudaSuccess) return SDGP_ERR_CUDA;
+  if (any_empty && cudaMemsetAsync(dD, 0, (size_t)B * H * W * Cd * 2, stream) != cudaSuccess) return SDGP_ERR_CUDA;
   for (int ph = 0; ph < stride; ++ph) {
     for (int pw = 0; pw < stride; ++pw) {
       const int Hs = (H - ph + stride - 1) / stride, Ws = (W - pw + stride - 1) / stride;  // pixels of this class
@@ -1795,10 +1801,10 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
         p.fused_n = fused->n; p.fused_m = fused->m; p.fused_scheme = fused->scheme;
         p.seed_lo = (uint32_t)fused->seed; p.seed_hi = (uint32_t)(fused->seed >> 32);
       }
-      view.d_base = (uint8_t*)dD + ((size_t)ph * W + pw) * Cin * 2;
-      view.d_stride_w = (uint64_t)stride * Cin * 2;
-      view.d_stride_h = (uint64_t)stride * W * Cin * 2;
-      view.d_stride_b = (uint64_t)H * W * Cin * 2;
+      view.d_base = (uint8_t*)dD + ((size_t)ph * W + pw) * Cd * 2;
+      view.d_stride_w = (uint64_t)stride * Cd * 2;
+      view.d_stride_h = (uint64_t)stride * W * Cd * 2;
+      view.d_stride_b = (uint64_t)H * W * Cd * 2;
       sdgp_status st = SDGP_ERR_UNSUPPORTED;
       // Images 4 pixels wide take the whole-filter-reuse kernel (column-split mode) with a sparse A: fused, it prunes
       // each box S times instead of R * S times; two-pass it measured the same as the general kernel; the dense twin

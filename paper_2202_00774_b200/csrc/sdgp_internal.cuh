@@ -45,9 +45,22 @@ struct FusedPrune {
 };
 // dtype: element type of A, Wt and dD (SDGP_BF16 or SDGP_FP16; accumulation is fp32 either way).
 // Fused pruning with the rescaled scheme exists for bf16 only.
+// stored != nullptr: Cin and Cout are the channel counts the kernels tile by (multiples of 64; Wt has that
+// many rows and columns, the extra ones zero) while the tensors in global memory hold fewer channels per
+// pixel: `a` for a dense A (0 = Cout; a compressed A is always padded to whole 128-channel blocks), `d` for dD
+// (0 = Cin), both multiples of 8. TMA reads the missing channels of A as zeros and clips the stores of dD.
+struct StoredChannels {
+  int a;
+  int d;
+};
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
                          int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
-                         const FusedPrune* fused = nullptr, int dtype = SDGP_BF16);
+                         const FusedPrune* fused = nullptr, int dtype = SDGP_BF16, const StoredChannels* stored = nullptr);
+
+// Filters of a grouped convolution, Wg [Cout, R*S, Cin/groups], written as the block-diagonal filters of an
+// ordinary one, Wfull [cout_pad, R*S, cin_pad] (zeros outside each group's block and in the padding).
+cudaError_t launch_expand_grouped_weights(const void* Wg, int Cout, int taps, int Cin, int groups, int cout_pad, int cin_pad,
+                                          void* Wfull, cudaStream_t stream);
 
 // Launches a one-CTA kernel whose only wait can never be satisfied (50 ms limit).
 sdgp_status launch_bounded_wait_selftest(cudaStream_t stream);
