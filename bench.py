@@ -2,7 +2,7 @@
 """Benchmark of the SDGP hot path: N:M pruning of dL/dO followed by the sparse tensor-core
 data gradient, on synthetic tensors shaped like a network's convolution layers.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet9|gemm_large|fc_small|resnet50]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet9|gemm_large|fc_small|resnet50|regnetx]
                   [--scheme magnitude|rescaled|random] [--nm 2:4] [--impl ours|reference]
 
 One step = every layer of the workload once: prune kernel + sparse dgrad kernel per layer
@@ -735,13 +735,97 @@ def run_layer_table(args):
         "per_layer": rows, "gpu_launches": launches, "clocks": clocks}))
 
 
+def run_grouped_table(args):
+    """--workload regnetx: every distinct convolution of the RegNetX-400MF body at batch 256 through
+    sdgp_dgrad_conv2d_grouped (grouped 3x3 convolutions, channel counts 32 and 160 that are not multiples of 64), one
+    layer at a time: two-pass, the dense twin and - where both channel counts are multiples of 64 - the fused
+    kernel, each timed as in the ResNet-50 table (CUDA events around single calls, 256 MB written between them,
+    median). FLOPs are the true ones of the grouped layer (Cin / groups input channels per output channel)."""
+    import torch
+    import paper_2202_00774_b200 as sdgp
+
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    n, m = [int(v) for v in args.nm.split(":")]
+    scheme = SCHEMES[args.scheme]
+    pk = peaks()
+    reps = max(5, min(args.steps, 50))
+    warm = max(3, min(args.warmup, 5))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def median_us(fn):
+        for _ in range(warm):
+            fn()
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(1e3 * e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    sampler = ClockSampler(torch.cuda.current_device())
+    rows, launches = [], 0
+    tot = dict(two_pass=0.0, dense=0.0, flops=0.0)
+    for l, count in inputs.regnetx_400mf_layer_counts(256):
+        dO_h, W_h = inputs.conv_layer_tensors(l, seed=0)
+        dO = torch.from_numpy(np.ascontiguousarray(dO_h).view(np.int16)).cuda()
+        Wt = torch.from_numpy(np.ascontiguousarray(W_h).view(np.int16)).cuda()
+        del dO_h, W_h
+        dD = torch.empty(l.dD_shape(), dtype=torch.int16, device="cuda")
+        ws = torch.empty(sdgp.sdgp_workspace_size_conv2d_grouped(l.B, l.H, l.W, l.Cin, l.Cout, l.R, l.S, l.stride, l.pad, l.groups),
+                         dtype=torch.uint8, device="cuda")
+
+        def call(flags):
+            sdgp.sdgp_dgrad_conv2d_grouped(dO, Wt, dD, l.stride, l.pad, l.groups, n, m, scheme, seed=1234, workspace=ws, flags=flags)
+
+        print("[%s]" % l.name, file=sys.stderr, flush=True)
+        t_two = median_us(lambda: call(sdgp.FLAG_TWO_PASS))
+        t_dense = median_us(lambda: call(sdgp.FLAG_DENSE))
+        t_fused = None
+        if l.Cin % 64 == 0 and l.Cout % 64 == 0 and n <= 2:
+            t_fused = median_us(lambda: call(sdgp.FLAG_FUSED))
+        launches += (reps + warm) * (3 + 2 + (2 if t_fused else 0))   # filter expansion + (prune) + contraction
+        status = sdgp.sdgp_last_device_error()
+        if status != 0:
+            raise SystemExit("device error: " + sdgp.status_string(status))
+        fl = 2.0 * l.dense_macs
+        pix = l.B * l.P * l.Q
+        bytes_dense = 2.0 * (pix * l.Cout + l.Cout * l.R * l.S * (l.Cin // l.groups) + l.B * l.H * l.W * l.Cin)
+        t_tensor = fl / (2.0 * pk["bf16_sustained"] * 1e12) * 1e6
+        t_hbm = bytes_dense / (pk["hbm"] * 1e9) * 1e6
+        rows.append({"layer": l.name, "count": count, "groups": l.groups, "gflop": fl / 1e9, "two_pass_us": t_two,
+                     "fused_us": t_fused, "dense_us": t_dense, "speedup_two_pass": t_dense / t_two,
+                     "bound": "tensor" if t_tensor >= t_hbm else "hbm", "ideal_dense_us": max(t_tensor, t_hbm),
+                     "dense_frac_of_ideal": max(t_tensor, t_hbm) / t_dense})
+        tot["two_pass"] += count * t_two
+        tot["dense"] += count * t_dense
+        tot["flops"] += count * fl
+        del dO, Wt, dD, ws
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    print(json.dumps({
+        "metric": METRIC, "value": tot["flops"] / (tot["two_pass"] * 1e-6) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": reps,
+        "warmup": warm, "ms_per_step": tot["two_pass"] / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "regnetx", "layers": len(rows), "convolutions": sum(r["count"] for r in rows), "batch": 256,
+                   "nm": args.nm, "scheme": args.scheme, "mode": "two_pass (per layer also dense and, where it applies, fused)",
+                   "flops": "true FLOPs of the grouped layers", "l2": "256 MB written between timed calls",
+                   "launch": "one call per event pair (filter expansion included), median"},
+        "speedup_vs_dense": tot["dense"] / tot["two_pass"],
+        "dense_tflops": tot["flops"] / (tot["dense"] * 1e-6) / 1e12,
+        "per_layer": rows, "gpu_launches": launches, "clocks": clocks}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet9", choices=["resnet9", "gemm_large", "fc_small", "resnet50"])
+    ap.add_argument("--workload", default="resnet9", choices=["resnet9", "gemm_large", "fc_small", "resnet50", "regnetx"])
     ap.add_argument("--scheme", default="magnitude", choices=sorted(SCHEMES))
     ap.add_argument("--nm", default="2:4")
     ap.add_argument("--mode", default="two_pass", choices=["two_pass", "fused", "channel"],
@@ -755,10 +839,10 @@ def main():
     args = ap.parse_args()
     if args.mode == "channel":
         args.scheme = "rescaled"
-    if args.workload == "resnet50":
+    if args.workload in ("resnet50", "regnetx"):
         if args.impl == "reference" or args.gpus != 1:
-            raise SystemExit("--workload resnet50 is a single-GPU per-layer table of this implementation")
-        return run_layer_table(args)
+            raise SystemExit("--workload %s is a single-GPU per-layer table of this implementation" % args.workload)
+        return run_layer_table(args) if args.workload == "resnet50" else run_grouped_table(args)
     layers = workload_layers(args.workload)
     if args.impl == "reference":
         run_reference(args, layers)

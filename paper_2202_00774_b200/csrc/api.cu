@@ -277,35 +277,40 @@ sdgp_status sdgp_dgrad_conv2d_grouped(const void* dO, const void* W, void* dD, i
   if (((uintptr_t)workspace & 255u) != 0) return SDGP_ERR_ALIGNMENT;
   cudaStream_t s = (cudaStream_t)stream;
   const int dt = (int)dtype;
-  void* w_full = workspace;
+  const void* w_full = W;  // one group and whole 64-channel blocks: the filters are already in the kernels' form
   void* rest = (uint8_t*)workspace + w_bytes;
-  if (sdgp::launch_expand_grouped_weights(W, Cout, R * S, Cin, groups, cout_k, cin_k, w_full, s) != cudaSuccess)
-    return SDGP_ERR_CUDA;
+  if (groups > 1 || Cin != cin_k || Cout != cout_k) {
+    if (sdgp::launch_expand_grouped_weights(W, Cout, R * S, Cin, groups, cout_k, cin_k, workspace, s) != cudaSuccess)
+      return SDGP_ERR_CUDA;
+    w_full = workspace;
+  }
   const sdgp::StoredChannels dense_view = {Cout != cout_k ? Cout : 0, Cin != cin_k ? Cin : 0};
   const sdgp::StoredChannels sparse_view = {0, dense_view.d};  // a compressed dL/dO is padded by the prune kernel
   const bool padded = dense_view.a != 0 || dense_view.d != 0;
+  const sdgp::ConvGroups cg = {Cin / groups, Cout / groups};
+  const sdgp::ConvGroups* cgp = groups > 1 ? &cg : nullptr;
   if (!prunes)
     return sdgp::launch_dgrad(false, dO, nullptr, w_full, dD, B, H, Wd, cin_k, cout_k, R, S, stride, pad, s, nullptr, dt,
-                              padded ? &dense_view : nullptr);
+                              padded ? &dense_view : nullptr, cgp);
   const int64_t rows = (int64_t)B * P * Q;
   if (flags == SDGP_FLAG_MASKED) {
     if (sdgp::launch_prune(dO, rows, Cout, n, m, (int)scheme, seed, rest, nullptr, nullptr, nullptr, s, 0, dt) != cudaSuccess)
       return SDGP_ERR_CUDA;
     return sdgp::launch_dgrad(false, rest, nullptr, w_full, dD, B, H, Wd, cin_k, cout_k, R, S, stride, pad, s, nullptr, dt,
-                              padded ? &dense_view : nullptr);
+                              padded ? &dense_view : nullptr, cgp);
   }
   if (flags == SDGP_FLAG_FUSED) {
     if (padded) return SDGP_ERR_UNSUPPORTED;  // the in-kernel prune reads dL/dO by the channel count it tiles by
     if (dtype == SDGP_FP16 && scheme == SDGP_RESCALED_MAGNITUDE) return SDGP_ERR_UNSUPPORTED;
     const sdgp::FusedPrune fp = {n, m, (int)scheme, seed};
-    return sdgp::launch_dgrad(true, dO, nullptr, w_full, dD, B, H, Wd, cin_k, cout_k, R, S, stride, pad, s, &fp, dt);
+    return sdgp::launch_dgrad(true, dO, nullptr, w_full, dD, B, H, Wd, cin_k, cout_k, R, S, stride, pad, s, &fp, dt, nullptr, cgp);
   }
   const int64_t Cpad = pad128(Cout);
   const Carve c = carve_compressed(rest, rows * Cpad);
   if (sdgp::launch_prune(dO, rows, Cout, n, m, (int)scheme, seed, nullptr, c.values, c.meta, nullptr, s, Cpad, dt) != cudaSuccess)
     return SDGP_ERR_CUDA;
   return sdgp::launch_dgrad(true, c.values, c.meta, w_full, dD, B, H, Wd, cin_k, cout_k, R, S, stride, pad, s, nullptr, dt,
-                            sparse_view.d ? &sparse_view : nullptr);
+                            sparse_view.d ? &sparse_view : nullptr, cgp);
 }
 
 sdgp_status sdgp_dgrad_linear(const void* dO, const void* W, void* dD, int64_t rows, int64_t K,

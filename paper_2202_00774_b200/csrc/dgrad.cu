@@ -91,6 +91,9 @@ struct DgradParams {
   uint32_t seed_lo, seed_hi;
   int P, Q;               // dO pixel grid (for the linear element index of the random scheme)
   int f16;                // element type of A, W and dD: 0 = bf16, 1 = IEEE binary16
+  // grouped convolution (block-diagonal W): a tile of input channels sees only k_blocks channel blocks of dL/dO,
+  // starting at first_k_block(); diag_cin_g == 0: every tile sees all of them
+  int diag_cin_g, diag_cout_g, diag_last;
   int off_raw;            // dense dL/dO stages: 2 * a_bytes each (two boxes of 64 channels)
   // shared-memory carve (byte offsets from the 1024-aligned base) and per-stage sizes
   int a_bytes, b_bytes, eraw_bytes, ehw_bytes;
@@ -110,6 +113,17 @@ struct Cfg {
   static constexpr int kTapBBytes = kBoxBytes * kBoxes;       // one CTA's W bytes of one (tap, channel block)
   static_assert(kBCols == 32 || kBCols % 64 == 0, "W half must be 32 columns or whole 64-column blocks");
 };
+
+// Grouped convolution: input channels n0 .. n0 + BN - 1 belong to groups n0 / cin_g and up, whose output channels
+// start at (n0 / cin_g) * cout_g; the tile's window of channel blocks (kbc channels each) starts at that channel's
+// block, or at `diag_last` where the window would otherwise run past the last block (W is zero outside the groups'
+// own blocks, so a window that covers more than it must changes nothing).
+template <class P>
+__device__ __forceinline__ int first_k_block(const P& p, int n0, int kbc) {
+  if (p.diag_cin_g == 0) return 0;
+  const int kb = ((n0 / p.diag_cin_g) * p.diag_cout_g) / kbc;
+  return kb < p.diag_last ? kb : p.diag_last;
+}
 
 // Instruction descriptor: fp32 accumulate, bf16 A and B, A K-major, B MN-major, M = 256 (pair).
 __host__ __device__ constexpr uint32_t make_idesc(int n, bool sparse) {
@@ -387,6 +401,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int ht = t % p.tiles_h; t /= p.tiles_h;
         const int bt = t;
         const int n0 = nt * BN + n_half;
+        const int cb0 = first_k_block(p, nt * BN, C::kKB);
         const int w0 = wt * p.TW, h0 = ht * p.TH, b0 = bt * p.TB;
         // reuse: a group is the horizontal tap s and the image starts R-1 rows above the row
         // the last vertical tap needs; otherwise a group is the single tap (r, s).
@@ -399,14 +414,14 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             if (FUSED) {
               // dense dL/dO of this CTA's patch: 128 channels as two boxes of 64
               ptx::mbar_arrive_expect_tx(&raw_full[st], 2u * (uint32_t)(p.img_rows * 128));
-              ptx::tma_load_4d(sRaw + st * 2 * p.a_bytes, &tmA, &raw_full[st], cb * 128, q0, p0, b0);
-              ptx::tma_load_4d(sRaw + st * 2 * p.a_bytes + p.a_bytes, &tmA, &raw_full[st], cb * 128 + 64, q0, p0, b0);
+              ptx::tma_load_4d(sRaw + st * 2 * p.a_bytes, &tmA, &raw_full[st], (cb0 + cb) * 128, q0, p0, b0);
+              ptx::tma_load_4d(sRaw + st * 2 * p.a_bytes + p.a_bytes, &tmA, &raw_full[st], (cb0 + cb) * 128 + 64, q0, p0, b0);
             } else {
               if (SPARSE) {
                 ptx::mbar_arrive_expect_tx(&meta_full[st], meta_tx);
-                ptx::tma_load_4d(sEraw + st * p.eraw_bytes, &tmE, &meta_full[st], cb * 8, q0, p0, b0);
+                ptx::tma_load_4d(sEraw + st * p.eraw_bytes, &tmE, &meta_full[st], (cb0 + cb) * 8, q0, p0, b0);
               }
-              ptx::tma_load_4d_pair(sA + st * p.a_bytes, &tmA, &full[st], cb * 64, q0, p0, b0);
+              ptx::tma_load_4d_pair(sA + st * p.a_bytes, &tmA, &full[st], (cb0 + cb) * 64, q0, p0, b0);
             }
             if (!p.w_resident) {
               for (int u = 0; u < p.rr; ++u) {
@@ -414,7 +429,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 #pragma unroll
                 for (int j = 0; j < C::kBoxes; ++j)
                   ptx::tma_load_2d_pair(sB + st * p.b_bytes + (u * C::kBoxes + j) * C::kBoxBytes, &tmB, &full[st],
-                                        tap * p.Cin + n0 + C::kBoxCols * j, cb * C::kKB);
+                                        tap * p.Cin + n0 + C::kBoxCols * j, (cb0 + cb) * C::kKB);
               }
             }
             if (++st == STAGES) { st = 0; ph ^= 1u; }
@@ -545,6 +560,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int wt = t % p.tiles_w; t /= p.tiles_w;
         const int ht = t % p.tiles_h; t /= p.tiles_h;
         const int w0 = wt * p.TW, h0 = ht * p.TH, b0 = t * p.TB;
+        const int cb0 = first_k_block(p, (pt % p.tiles_n) * BN, C::kKB);
         int r = reuse ? (p.R - 1) : 0, s = 0, cb = 0;
         for (int k = 0; k < uses_per_tile; ++k) {
           // the pruning warps stay or leave together: they meet at a named barrier below
@@ -557,7 +573,7 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const int i = item >> 3, e = item & 7;
             const int iw = i % p.TW, ih = (i / p.TW) % img_h, ib = i / (p.TW * img_h);
             const int64_t pixel = ((int64_t)(b0 + ib) * p.P + (p0 + ih)) * p.Q + (q0 + iw);  // any value when outside
-            const int64_t vbase = pixel * (p.Cout >> 3) + cb * 16;
+            const int64_t vbase = pixel * (p.Cout >> 3) + (cb0 + cb) * 16;
 #define SDGP_FUSED_ITEM(MM, NN, SS) fused_prune_eighth<MM, NN, SS>(raw, p.a_bytes, a_tile, meta_rows, i, e, vbase, p.seed_lo, p.seed_hi)
 #define SDGP_FUSED_M(MM)                                                                                                   \
   if (p.fused_scheme == SDGP_MAGNITUDE) { if (p.fused_n == 1) SDGP_FUSED_ITEM(MM, 1, SDGP_MAGNITUDE); else SDGP_FUSED_ITEM(MM, 2, SDGP_MAGNITUDE); } \
@@ -708,6 +724,7 @@ struct HaloParams {
   int smem_bytes;
   // fused pruning (A is the dense dL/dO; m = 4): the pruning warps read it straight from global memory
   const uint8_t* a_dense;  // dL/dO [B, P, Q, Cout], 16-bit elements
+  int diag_cin_g, diag_cout_g, diag_last;  // grouped convolution: see first_k_block()
   uint32_t pitch_magic;    // ceil(2^20 / pitch): i / pitch == (i * pitch_magic) >> 20 for every box pixel row i
   int fused_n, fused_m, fused_scheme;
   uint32_t seed_lo, seed_hi;
@@ -868,9 +885,10 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           return 0;
         }
         const int lt = ia / p.k_uses, ku = ia - lt * p.k_uses;
-        const int kb = ku / p.ss, si = ku - kb * p.ss;  // channel block, filter column of the box (column-split mode)
+        const int kl = ku / p.ss, si = ku - kl * p.ss;  // channel block of the tile's window, filter column of the box (column-split mode)
         int n0, w0, h0, b0;
         locate(first_pair + lt * pair_stride, n0, w0, h0, b0);
+        const int kb = first_k_block(p, n0, C::kKB) + kl;
         const int q0 = w0 + p.pad_w - (p.sb - 1) - si, p0 = h0 + p.pad_h - (p.R - 1);
         // coordinates: channel, pixel column, image within a box row, image group, pixel row
         const int bg = b0 / p.img_per_row;
@@ -893,9 +911,10 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       for (int lt = 0; alive && lt < my_tiles; ++lt) {
         int n0, w0_unused, h0_unused, b0_unused;
         locate(first_pair + lt * pair_stride, n0, w0_unused, h0_unused, b0_unused);
+        const int kb0 = first_k_block(p, n0, C::kKB);
         n0 += n_half;
         for (int ku = 0; alive && ku < p.k_uses; ++ku, ++use) {
-          const int kb = ku / p.ss, si = ku - kb * p.ss;
+          const int kl = ku / p.ss, si = ku - kl * p.ss, kb = kb0 + kl;
           // (fused: the pruning warps fetch dL/dO themselves; this thread streams W only)
           while (!FUSED && alive && ia <= use)
             if (issue_a(true) < 0) alive = false;
@@ -1091,10 +1110,13 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int org_b = 0;                // its image
         int64_t org_pix = 0;          // its linear pixel number (random keys)
         bool org_ok = false;
-        auto set_origin = [&](int box_lt, int box_ku, const uint8_t*& ptr, int& p0, int& q0, int& b0, int64_t& pix, bool& ok) {
+        int org_kb0 = 0;              // first channel block of its tile's window
+        auto set_origin = [&](int box_lt, int box_ku, const uint8_t*& ptr, int& p0, int& q0, int& b0, int64_t& pix, bool& ok, int& kb0) {
           int n0, w0, h0;
           ok = locate(first_pair + box_lt * pair_stride, n0, w0, h0, b0);
-          const int box_kb = box_ku / p.ss, si = box_ku - box_kb * p.ss;
+          const int box_kl = box_ku / p.ss, si = box_ku - box_kl * p.ss;
+          kb0 = first_k_block(p, n0, 128);
+          const int box_kb = kb0 + box_kl;
           q0 = w0 + p.pad_w - (p.sb - 1) - si;
           p0 = h0 + p.pad_h - (p.R - 1);
           pix = ((int64_t)b0 * p.P + p0) * p.Q + q0;
@@ -1114,7 +1136,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         bool u_live = false;  // some pixel of the unit lies inside the tensor (halo rows above / below an image: none does)
         auto fetch = [&]() {
           if (org_box != ia) {
-            set_origin(lt, ku, org_ptr, org_p, org_q, org_b, org_pix, org_ok);
+            set_origin(lt, ku, org_ptr, org_p, org_q, org_b, org_pix, org_ok, org_kb0);
             org_box = ia;
             // ask the lines of the NEXT box into L2 now, a whole box ahead of their loads: 2 lines of 128
             // bytes per box pixel, dealt to the pruning threads
@@ -1122,10 +1144,10 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (nkb == p.k_uses) { nkb = 0; ++nlt; }
             if (ia + 1 < a_uses) {
               const uint8_t* nptr;
-              int np0, nq0, nb0;
+              int np0, nq0, nb0, nkb0;
               int64_t npix;
               bool nok;
-              set_origin(nlt, nkb, nptr, np0, nq0, nb0, npix, nok);
+              set_origin(nlt, nkb, nptr, np0, nq0, nb0, npix, nok, nkb0);
               for (int line = pw * 32 + lane; line < 2 * p.img_rows; line += 32 * kPruneWarps) {
                 const int px = line >> 1;
                 const int br = (int)(((uint32_t)px * p.pitch_magic) >> 20);  // box row
@@ -1138,7 +1160,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
           u_i = 8 * o + row8;
           u_ia = ia;
-          const int kb = ku / p.ss;
+          const int kb = org_kb0 + ku / p.ss;
           u_kb = kb;
           const int br = (int)(((uint32_t)u_i * p.pitch_magic) >> 20);  // box row
           int ib, ih, iw;
@@ -1398,7 +1420,7 @@ bool plan(DgradParams* p) {
   // Filter-row reuse needs a single-image patch whose rows are whole groups of 8 pixels, so
   // that every vertical tap is an offset of whole 1024-byte swizzle periods.
   const bool can_reuse = p->R > 1 && p->TB == 1 && p->TW % 8 == 0 && p->TW * (p->TH + p->R - 1) <= kMaxImgRows;
-  const bool can_reside = p->tiles_n == 1 && p->pair_tiles > sm_count() / 2;  // pays only if tiles repeat
+  const bool can_reside = p->tiles_n == 1 && p->diag_cin_g == 0 && p->pair_tiles > sm_count() / 2;  // pays only if tiles repeat
   for (int attempt = 0; attempt < 4; ++attempt) {
     // attempt 0: reuse with streamed W (measured best where it fits: more stages in flight),
     // 1: reuse + resident W, 2: resident W, 3: neither
@@ -1740,7 +1762,7 @@ sdgp_status launch_halo(const void* A, const void* meta, const void* Wt, const D
 // (m = 4, n = fused->n in {1, 2}); no compressed tensor exists in global memory.
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
                          int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
-                         const FusedPrune* fused, int dtype, const StoredChannels* stored) {
+                         const FusedPrune* fused, int dtype, const StoredChannels* stored, const ConvGroups* conv_groups) {
   if (fused && stored) return SDGP_ERR_UNSUPPORTED;  // the pruning warps address dL/dO by the channel count they tile by
   if (stored && (stored->a < 0 || stored->a > Cout || stored->a % 8 != 0 || stored->d < 0 || stored->d > Cin || stored->d % 8 != 0))
     return SDGP_ERR_INVALID_ARG;
@@ -1795,6 +1817,22 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
       p.m_tiles = (int)m_tiles;
       p.pair_tiles = (int)((m_tiles + 1) / 2) * p.tiles_n;
       p.k_blocks = (Cout + kb_channels - 1) / kb_channels;
+      if (conv_groups && conv_groups->cin_g > 0 && conv_groups->cout_g > 0) {
+        // block-diagonal W: the widest window of channel blocks any tile of input channels needs
+        int widest = 0;
+        for (int nt = 0; nt < p.tiles_n; ++nt) {
+          const int lo = ((nt * BN) / conv_groups->cin_g) * conv_groups->cout_g / kb_channels;
+          int co_end = ((nt * BN + BN + conv_groups->cin_g - 1) / conv_groups->cin_g) * conv_groups->cout_g;
+          if (co_end > Cout) co_end = Cout;
+          const int hi = (co_end + kb_channels - 1) / kb_channels;
+          if (hi - lo > widest) widest = hi - lo;
+        }
+        if (widest > 0 && widest < p.k_blocks) {
+          p.diag_cin_g = conv_groups->cin_g; p.diag_cout_g = conv_groups->cout_g;
+          p.diag_last = p.k_blocks - widest;
+          p.k_blocks = widest;
+        }
+      }
       p.P = P; p.Q = Q;
       p.f16 = dtype == SDGP_FP16 ? 1 : 0;
       if (fused) {
@@ -1817,6 +1855,7 @@ sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const voi
         hp.r_first = p.r_first; hp.r_step = p.r_step; hp.s_first = p.s_first; hp.s_step = p.s_step;
         hp.S_full = S;
         hp.tiles_n = p.tiles_n; hp.k_blocks = p.k_blocks;
+        hp.diag_cin_g = p.diag_cin_g; hp.diag_cout_g = p.diag_cout_g; hp.diag_last = p.diag_last;
         hp.P = P; hp.Q = Q;
         hp.f16 = p.f16;
         if (fused) {

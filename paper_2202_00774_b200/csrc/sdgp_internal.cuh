@@ -53,9 +53,17 @@ struct StoredChannels {
   int a;
   int d;
 };
+// conv_groups != nullptr: Wt is block-diagonal - input channels [g * cin_g, (g + 1) * cin_g) are connected to output
+// channels [g * cout_g, (g + 1) * cout_g) only, everything else in Wt is zero - so a tile of input channels skips
+// the channel blocks of dL/dO that only meet zeros.
+struct ConvGroups {
+  int cin_g;
+  int cout_g;
+};
 sdgp_status launch_dgrad(bool sparse, const void* A, const void* meta, const void* Wt, void* dD, int B,
                          int H, int W, int Cin, int Cout, int R, int S, int stride, int pad, cudaStream_t stream,
-                         const FusedPrune* fused = nullptr, int dtype = SDGP_BF16, const StoredChannels* stored = nullptr);
+                         const FusedPrune* fused = nullptr, int dtype = SDGP_BF16, const StoredChannels* stored = nullptr,
+                         const ConvGroups* conv_groups = nullptr);
 
 // Filters of a grouped convolution, Wg [Cout, R*S, Cin/groups], written as the block-diagonal filters of an
 // ordinary one, Wfull [cout_pad, R*S, cin_pad] (zeros outside each group's block and in the padding).

@@ -183,24 +183,29 @@ def resnet18_layers(batch: int = 256) -> List[ConvLayer]:
     return out
 
 
-def regnetx_400mf_layers(batch: int = 256) -> List[ConvLayer]:
-    """Distinct convolutions of the RegNetX-400MF body (Section 4 trains it on ImageNet): stage widths 32, 64,
-    160, 384 at 56, 28, 14, 7 pixels, group width 16 (so 2, 4, 10, 24 groups), bottleneck ratio 1. A block is
-    1x1 -> grouped 3x3 -> 1x1; the first block of a stage takes the previous stage's width at twice the
-    resolution, strides in its 3x3 and has a 1x1 stride-2 shortcut."""
+def regnetx_400mf_layer_counts(batch: int = 256):
+    """Distinct convolutions of the RegNetX-400MF body (Section 4 trains it on ImageNet) with the number of times
+    the network holds each: stage widths 32, 64, 160, 384 at 56, 28, 14, 7 pixels, depths 1, 2, 7, 12, group width
+    16 (so 2, 4, 10, 24 groups), bottleneck ratio 1. A block is 1x1 -> grouped 3x3 -> 1x1; the first block of a
+    stage takes the previous stage's width at twice the resolution, strides in its 3x3 and has a 1x1 stride-2
+    shortcut."""
     out = []
     prev = 32
     for stage, (hw, ch, depth) in enumerate([(56, 32, 1), (28, 64, 2), (14, 160, 7), (7, 384, 12)], start=1):
         tag = "rx_s%d_" % stage
         g = ch // 16
-        out.append(ConvLayer(tag + "1x1_%dto%d_at%d" % (prev, ch, 2 * hw), batch, 2 * hw, 2 * hw, prev, ch, 1, 1, 1, 0))
-        out.append(ConvLayer(tag + "3x3s2g%d_%d_at%d" % (g, ch, 2 * hw), batch, 2 * hw, 2 * hw, ch, ch, 3, 3, 2, 1, g))
-        out.append(ConvLayer(tag + "projs2_%dto%d_at%d" % (prev, ch, 2 * hw), batch, 2 * hw, 2 * hw, prev, ch, 1, 1, 2, 0))
-        out.append(ConvLayer(tag + "1x1_%dto%d_at%d" % (ch, ch, hw), batch, hw, hw, ch, ch, 1, 1, 1, 0))
+        out.append((ConvLayer(tag + "1x1_%dto%d_at%d" % (prev, ch, 2 * hw), batch, 2 * hw, 2 * hw, prev, ch, 1, 1, 1, 0), 1))
+        out.append((ConvLayer(tag + "3x3s2g%d_%d_at%d" % (g, ch, 2 * hw), batch, 2 * hw, 2 * hw, ch, ch, 3, 3, 2, 1, g), 1))
+        out.append((ConvLayer(tag + "projs2_%dto%d_at%d" % (prev, ch, 2 * hw), batch, 2 * hw, 2 * hw, prev, ch, 1, 1, 2, 0), 1))
+        out.append((ConvLayer(tag + "1x1_%dto%d_at%d" % (ch, ch, hw), batch, hw, hw, ch, ch, 1, 1, 1, 0), 2 * depth - 1))
         if depth > 1:
-            out.append(ConvLayer(tag + "3x3g%d_%d_at%d" % (g, ch, hw), batch, hw, hw, ch, ch, 3, 3, 1, 1, g))
+            out.append((ConvLayer(tag + "3x3g%d_%d_at%d" % (g, ch, hw), batch, hw, hw, ch, ch, 3, 3, 1, 1, g), depth - 1))
         prev = ch
     return out
+
+
+def regnetx_400mf_layers(batch: int = 256) -> List[ConvLayer]:
+    return [layer for layer, _ in regnetx_400mf_layer_counts(batch)]
 
 
 def conv_layer_tensors(layer: ConvLayer, seed: int):
