@@ -627,7 +627,8 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
       if (++acc == NACC) { acc = 0; aph ^= 1u; }
     }
-    if (issuer) ptx::bulk_wait_group_all();  // dD is written before the CTA leaves
+    // the staging slabs have been read; the writes themselves complete with the grid (whoever depends on dD waits for that)
+    if (issuer) ptx::bulk_wait_group_read<0>();
   }
 
   __syncwarp();
@@ -828,7 +829,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   ptx::tc_fence_before_sync();
   ptx::cluster_sync();
   ptx::tc_fence_after_sync();
-  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_base_any = *tmem_slot;
+  const uint32_t tmem_base = tmem_base_any;
   // everything above touched no global memory; the previous kernel's results are needed from here on
   ptx::wait_for_previous_grid();
   // Only now may the next kernel of the stream be scheduled: every CTA of this grid owns its TMEM
@@ -936,10 +938,14 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
   } else if (warp == 1) {
     // ------------------------------------------- MMA issuer (first CTA only)
-    // One thread executes a few dependent instructions per ~10 clocks, so its path per tap is
-    // kept short: one barrier wait, running descriptor words updated by additions, compile-time
-    // offsets for the strips and the four MMAs of a channel block.
-    if (rank == 0 && ptx::elect_one()) {
+    // The whole warp walks the loops together and one elected lane issues the tensor-core instructions: every
+    // address and descriptor word is then the same in all lanes, which lets the compiler keep them in the warp's
+    // uniform registers, where those instructions take their operands from. The path per tap is kept short: one
+    // barrier wait, running descriptor words updated by additions, compile-time offsets for the strips and the four
+    // MMAs of a channel block.
+    if (rank == 0) {
+      const bool leader = ptx::elect_one();
+      const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, tmem_base_any, 0);  // one value for the warp, and known to be
       const uint32_t idesc = make_idesc(BN, SPARSE) & ~(p.f16 ? kIdescBf16Operands : 0u);
       // descriptors as two 32-bit halves: the start address only ever changes the low word
       const uint64_t adesc0 = ptx::make_smem_desc(0, 16, (uint32_t)p.pitch * 128u, 2);
@@ -966,13 +972,15 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       uint32_t aph = 0, wph = 0, cph = 0;
       // running words of the W ring: W descriptor, metadata column (relative)
       uint32_t b_lo = b_lo0, mcol = 0;
+      // (a wait that gives up in one lane ends the role for the whole warp)
+      auto wait_all = [&](uint64_t* bar, uint32_t parity, unsigned int code) -> bool {
+        return __all_sync(0xFFFFFFFFu, ptx::mbar_wait(bar, parity, err, code));
+      };
       for (int lt = 0; alive && lt < my_tiles; ++lt) {
-        if (!ptx::mbar_wait(&acc_empty[acc], cph ^ 1u, err, 0x200u + acc)) break;
+        if (!wait_all(&acc_empty[acc], cph ^ 1u, 0x200u + acc)) break;
         // shared metadata region: the first columns of the other tile set's accumulators,
         // which the epilogue of the previous tile set reads out first
-        if (p.meta_shared && lt > 0 &&
-            !ptx::mbar_wait(&meta_free[acc ^ 1], (((uint32_t)lt - 1u) >> 1) & 1u, err, 0x800u + acc))
-          break;
+        if (p.meta_shared && lt > 0 && !wait_all(&meta_free[acc ^ 1], (((uint32_t)lt - 1u) >> 1) & 1u, 0x800u + acc)) break;
         const uint32_t meta_base = tmem_base + (uint32_t)(p.meta_shared ? (acc ^ 1) * set_cols : p.meta_col);
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * set_cols);
@@ -980,14 +988,14 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const bool all_strips = strips == ((1u << NT) - 1u);
         uint32_t accumulate = 0u;
         for (int ku = 0; alive && ku < p.k_uses; ++ku) {
-          if (!ptx::mbar_wait(&a_full[ast], aph, err, 0x300u + ast)) { alive = false; break; }
-          if (SPARSE && !FUSED && !ptx::mbar_wait(&meta_ready[ast], aph, err, 0x340u + ast)) { alive = false; break; }
+          if (!wait_all(&a_full[ast], aph, 0x300u + ast)) { alive = false; break; }
+          if (SPARSE && !FUSED && !wait_all(&meta_ready[ast], aph, 0x340u + ast)) { alive = false; break; }
           uint32_t a_lo = a_lo0 + (uint32_t)ast * a_stage16 + a_first16;
           int s = p.sb, dr = p.R - 1;
           const uint32_t e_stage = e_lo0 + (uint32_t)ast * e_stage16;
           uint32_t e_lo = e_stage + meta_row16(dr) + (uint32_t)(p.sb - 1);
           for (int t = 0; t < taps; ++t) {
-            if (!ptx::mbar_wait(&w_ready[wst], wph, err, 0x380u + wst)) { alive = false; break; }
+            if (!wait_all(&w_ready[wst], wph, 0x380u + wst)) { alive = false; break; }
             ptx::tc_fence_after_sync();
             const uint32_t e_col = meta_base + mcol;  // even: slots are 4 columns apart
             // ALL: every strip takes part (no per-strip test in the issue path)
@@ -1015,9 +1023,11 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 }
               }
             };
-            if (all_strips) issue_tap(std::true_type{});
-            else issue_tap(std::false_type{});
-            ptx::tc_commit_pair(&w_empty[wst], 3);
+            if (leader) {
+              if (all_strips) issue_tap(std::true_type{});
+              else issue_tap(std::false_type{});
+              ptx::tc_commit_pair(&w_empty[wst], 3);
+            }
             accumulate = 1u;
             // next tap: one pixel to the left, or the end of the filter row above
             if (--s == 0) { s = p.sb; a_lo -= a_rowstep16; --dr; e_lo = e_stage + meta_row16(dr) + (uint32_t)(p.sb - 1); }
@@ -1025,10 +1035,10 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (++wst == WS) { wst = 0; wph ^= 1u; b_lo = b_lo0; mcol = 0; }
             else { b_lo += w_stage16; mcol += kSlotCols; }
           }
-          if (alive) ptx::tc_commit_pair(&a_empty[ast], 3);
+          if (alive && leader) ptx::tc_commit_pair(&a_empty[ast], 3);
           if (++ast == p.a_stages) { ast = 0; aph ^= 1u; }
         }
-        if (alive) ptx::tc_commit_pair(&acc_full[acc], 3);
+        if (alive && leader) ptx::tc_commit_pair(&acc_full[acc], 3);
         if (++acc == 2) { acc = 0; cph ^= 1u; }
       }
     }
@@ -1301,7 +1311,8 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       if (lane == 0) ptx::mbar_arrive_cluster(&acc_empty[acc], 0);
       if (++acc == 2) { acc = 0; cph ^= 1u; }
     }
-    if (issuer) ptx::bulk_wait_group_all();
+    // the staging slabs have been read; the writes themselves complete with the grid (whoever depends on dD waits for that)
+    if (issuer) ptx::bulk_wait_group_read<0>();
   }
 
   __syncwarp();
