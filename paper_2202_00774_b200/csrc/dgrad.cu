@@ -24,8 +24,8 @@
 //               four MMAs per (tap, channel block), tcgen05.commit to the stage's "empty" barrier.
 //   warps 2-5   (sparse only) build the stage's metadata images: from the row-major order TMA
 //               delivers to the lane/column order the tensor core reads from TMEM. Each warp
-//               takes every fourth stage use (four stages in flight); with fused pruning the
-//               four warps first prune the stage's pixel rows together.
+//               owns every fourth stage; with fused pruning these four warps and eight helper
+//               warps (10-17) first prune the stage's pixel rows together.
 //   warps 6-9   epilogue: TMEM -> registers -> bf16 -> swizzled staging tile -> TMA store,
 //               overlapped with the next tile's main loop through a second accumulator.
 //
@@ -648,25 +648,31 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
 // ---------------------------------------------------------------- whole-filter reuse
 //
-// Convolutions with more than one filter tap on images at least a strip (8 x 16 pixels) large.
+// Convolutions with more than one filter tap.
 // The shared-memory matrix descriptor swizzles by absolute address bits, so an A operand may
 // start at ANY 128-byte row of a swizzled tile and its 8-row groups may lie any number of rows
-// apart. A tile is therefore an 8-pixel-wide, 16-pixel-tall strip of one image, and one TMA box
-// holding the strip plus its (R-1, S-1) halo serves EVERY filter tap: tap (r, s) is the row
-// offset (R-1-r) * pitch + (S-1-s) in the A descriptor, group stride = pitch rows. dL/dO is
+// apart. A tile is therefore a strip of 16 rows of 8 pixels, and one TMA box holding the strip plus
+// its (R-1, S-1) halo serves EVERY filter tap: tap (r, s) is the row offset
+// (R-1-r) * tb * pitch + (S-1-s) in the A descriptor, group stride = pitch rows. dL/dO is
 // read from L2 once per strip (plus halo) instead of once per horizontal tap, and with two
 // neighbouring strips per CTA (two accumulators) each W stage feeds twice the MMAs.
+// Strip geometries (th pixel rows x tb images, th * tb = 16): 16 rows of one image; 8 rows of two images
+// (images at most 8 pixels tall; the box's rows are ordered (pixel row, image)); and, for images 4 pixels
+// wide, 4 rows of eight images with two images side by side in a strip row and one box per filter column
+// (column-split mode: no column halo, five-dimensional tensor maps).
 //
-// Rings: A images (2 stages; one stage = one tile set and one block of output channels),
-// W taps (w_stages; one stage = the W rows of one tap and channel block, plus, for sparse A, the
-// rearranged metadata tiles of that tap). Roles as in dgrad_kernel; the metadata warps build one
-// 2 KB TMEM image per (tap, strip) from the raw metadata box of the A stage.
+// Rings: A boxes (2 or 4 stages; one stage = one tile set and one block of output channels, with the raw
+// metadata box TMA delivers and the two metadata masters built from it), W taps (w_stages; one stage = the W
+// rows of one tap and channel block, and a slot of TMEM columns for that tap's metadata).
+// Metadata masters: the position metadata of a box is stored once, in the order the tensor core wants, and every
+// tap copies a window of it into TMEM (see HaloParams). Two-pass: warps 2..5 build the masters of each box;
+// fused: the pruning warps write them directly.
 
 constexpr int kHaloRows = 16;  // 8-pixel rows of a strip: the 128 rows of an accumulator
 constexpr int kHaloAStages = 4;  // at most: A stages in use are p.a_stages = 2, or 4 when the boxes are small (a power of two)
 // Warp roles of the fused whole-filter-reuse kernel (24 warps: registers are granted to warps in fours, and
-// 24 x 80 registers is what fits). Warp w runs on scheduler w % 4, and the thread that issues the MMAs
-// (warp 1) is what bounds these kernels, so the busy pruning warps keep off its scheduler: warp 0 streams W,
+// 24 x 80 registers is what fits). Warp w runs on scheduler w % 4; the busy pruning warps keep off the scheduler
+// of the warp that issues the MMAs (with them on it a tap took 900 instead of 750 clocks): warp 0 streams W,
 // warp 1 issues the MMAs, warps 4..7 are the epilogue (one per TMEM lane quarter), and of the rest those
 // with w % 4 != 1 prune (2, 3, 8, 10..12, 14..16, 18..20, 22, 23: fourteen warps); warps 9, 13, 17 and 21
 // have no role.
