@@ -39,6 +39,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <string.h>
+
 #include <type_traits>
 
 #include "prune_core.cuh"
@@ -1353,14 +1355,43 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// A tensor map is a pure function of these arguments (it holds the address, not the memory), and a training
+// loop asks for the same few maps every step: each host thread keeps the last kMapCache it encoded. Outside a CUDA
+// graph the four encodes of a launch otherwise cost about as much as a small layer's kernel.
+struct MapKey {
+  const void* base;
+  uint64_t dims[5], strides[4];
+  uint32_t box[5];
+  int dt, rank, swz;
+};
+constexpr int kMapCache = 64;
+
 bool encode(CUtensorMap* tm, CUtensorMapDataType dt, int rank, const void* base, const uint64_t* dims,
             const uint64_t* strides_bytes, const uint32_t* box, CUtensorMapSwizzle swz) {
+  static thread_local MapKey keys[kMapCache];
+  static thread_local CUtensorMap maps[kMapCache];
+  static thread_local int used = 0, next = 0;
+  MapKey key;
+  memset(&key, 0, sizeof(key));
+  key.base = base; key.dt = (int)dt; key.rank = rank; key.swz = (int)swz;
+  for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides_bytes[i];
+  for (int i = 0; i < used; ++i)
+    if (memcmp(&keys[i], &key, sizeof(key)) == 0) {
+      *tm = maps[i];
+      return true;
+    }
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-  return fn(tm, dt, (cuuint32_t)rank, const_cast<void*>(base), (const cuuint64_t*)dims,
-            (const cuuint64_t*)strides_bytes, (const cuuint32_t*)box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  if (fn(tm, dt, (cuuint32_t)rank, const_cast<void*>(base), (const cuuint64_t*)dims, (const cuuint64_t*)strides_bytes,
+         (const cuuint32_t*)box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  const int slot = used < kMapCache ? used++ : (next = (next + 1) % kMapCache);
+  keys[slot] = key;
+  maps[slot] = *tm;
+  return true;
 }
 
 int largest_divisor_at_most(int x, int cap) {
