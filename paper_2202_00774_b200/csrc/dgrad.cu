@@ -220,7 +220,10 @@ __device__ __forceinline__ void fused_prune_eighth(const uint8_t* raw, int a_byt
 #pragma unroll
   for (int jj = 0; jj < 2; ++jj) {
     uint32_t slot0, slot1, nib2;
-    compressed_slots(y[jj][0], y[jj][1], y[jj][2], y[jj][3], km[jj][0], km[jj][1], km[jj][2], km[jj][3], slot0, slot1, nib2);
+    if (M == 4 && SCHEME == SDGP_RESCALED_MAGNITUDE)  // (the lanes above are dead code then: the slots are rescaled, not the lanes)
+      m4_rescaled_compressed<N, false>(w[jj], slot0, slot1, nib2, km[jj][0], km[jj][1], km[jj][2], km[jj][3]);
+    else
+      compressed_slots(y[jj][0], y[jj][1], y[jj][2], y[jj][3], km[jj][0], km[jj][1], km[jj][2], km[jj][3], slot0, slot1, nib2);
     out[jj] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
     nibs |= nib2 << (8 * jj);
   }
@@ -753,12 +756,16 @@ __device__ __forceinline__ void fused_prune_vectors(const uint4 (&w)[4], int64_t
 #pragma unroll
   for (int v = 0; v < 4; ++v) {
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2;
-    if (M == 4)
-      m4_prune_vector<N, SCHEME>(w[v], vbase + vstep * v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
-    else
-      top2_prune_vector<(M == 4 ? 8 : M), SCHEME>(w[v], vbase + vstep * v, seed_lo, seed_hi, N, part, 0xFFFFFFFFu, y0, y1, y2, y3,
-                                                  km0, km1, km2, km3);
-    compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
+    if (M == 4 && SCHEME == SDGP_RESCALED_MAGNITUDE) {
+      m4_rescaled_compressed<N, false>(w[v], slot0, slot1, nib2, km0, km1, km2, km3);  // the slots are rescaled, not the lanes
+    } else {
+      if (M == 4)
+        m4_prune_vector<N, SCHEME>(w[v], vbase + vstep * v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
+      else
+        top2_prune_vector<(M == 4 ? 8 : M), SCHEME>(w[v], vbase + vstep * v, seed_lo, seed_hi, N, part, 0xFFFFFFFFu, y0, y1, y2,
+                                                    y3, km0, km1, km2, km3);
+      compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
+    }
     out[v] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
     metaw |= nib2 << (8 * v);
   }

@@ -226,30 +226,40 @@ struct OutPitch {
 
 // Writes one vector's outputs from the lane-paired form (see m4_prune_vector). COMPRESS: every
 // 4-chunk holds at most two survivors, so values / meta can be produced.
+// Output position of vector v's compressed outputs; writes the padding of a padded row when v is the row's last vector.
+__device__ __forceinline__ int64_t compressed_index(int64_t v, uint2* __restrict__ values, uint8_t* __restrict__ meta,
+                                                    OutPitch pitch) {
+  if (pitch.kpad8 == 0) return v;
+  const int64_t row = v / pitch.k8;
+  const int kv = (int)(v - row * pitch.k8);
+  const int64_t vo = row * pitch.kpad8 + kv;
+  if (kv == pitch.k8 - 1) {
+    for (int t = 1; t <= pitch.kpad8 - pitch.k8; ++t) {
+      if (values) values[vo + t] = make_uint2(0u, 0u);
+      if (meta) meta[vo + t] = (uint8_t)0x44;
+    }
+  }
+  return vo;
+}
+
+__device__ __forceinline__ void emit_mask(int64_t v, uint32_t km0, uint32_t km1, uint32_t km2, uint32_t km3,
+                                          uint8_t* __restrict__ mask) {
+  const uint32_t t = (km0 & 0x00010001u) | (km1 & 0x00020002u) | (km2 & 0x00040004u) | (km3 & 0x00080008u);
+  mask[v] = (uint8_t)((t & 0xFu) | (t >> 12));
+}
+
+// Writes one vector's outputs from the lane-paired form (see m4_prune_vector). COMPRESS: every
+// 4-chunk holds at most two survivors, so values / meta can be produced.
 template <bool COMPRESS>
 __device__ __forceinline__ void emit_packed(int64_t v, uint32_t y0, uint32_t y1, uint32_t y2, uint32_t y3,
                                             uint32_t km0, uint32_t km1, uint32_t km2, uint32_t km3,
                                             uint4* __restrict__ dense, uint2* __restrict__ values,
                                             uint8_t* __restrict__ meta, uint8_t* __restrict__ mask,
                                             OutPitch pitch) {
-  int64_t vo = v;
-  if (pitch.kpad8 != 0) {
-    const int64_t row = v / pitch.k8;
-    const int kv = (int)(v - row * pitch.k8);
-    vo = row * pitch.kpad8 + kv;
-    if (COMPRESS && kv == pitch.k8 - 1) {
-      for (int t = 1; t <= pitch.kpad8 - pitch.k8; ++t) {
-        if (values) values[vo + t] = make_uint2(0u, 0u);
-        if (meta) meta[vo + t] = (uint8_t)0x44;
-      }
-    }
-  }
+  const int64_t vo = COMPRESS ? compressed_index(v, values, meta, pitch) : v;
   if (dense)
     dense[v] = make_uint4(prmt(y0, y1, 0x5410), prmt(y2, y3, 0x5410), prmt(y0, y1, 0x7632), prmt(y2, y3, 0x7632));
-  if (mask) {
-    const uint32_t t = (km0 & 0x00010001u) | (km1 & 0x00020002u) | (km2 & 0x00040004u) | (km3 & 0x00080008u);
-    mask[v] = (uint8_t)((t & 0xFu) | (t >> 12));
-  }
+  if (mask) emit_mask(v, km0, km1, km2, km3, mask);
   if (COMPRESS && (values || meta)) {
     uint32_t slot0, slot1, nib2;
     compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
@@ -278,6 +288,17 @@ prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, ui
     if (v >= nvec) continue;
     const uint4 w = in[it];
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3;
+    if constexpr (SCHEME == SDGP_RESCALED_MAGNITUDE && N <= 2) {
+      if (!dense) {  // only the compressed form is wanted: rescale the two slots instead of the eight lanes
+        uint32_t slot0, slot1, nib2;
+        m4_rescaled_compressed<N, F16>(w, slot0, slot1, nib2, km0, km1, km2, km3);
+        const int64_t vo = compressed_index(v, values, meta, pitch);
+        if (mask) emit_mask(v, km0, km1, km2, km3, mask);
+        if (values) values[vo] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
+        if (meta) meta[vo] = (uint8_t)nib2;
+        continue;
+      }
+    }
     m4_prune_vector<N, SCHEME, F16>(w, v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);
     emit_packed<(N <= 2)>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask, pitch);
   }

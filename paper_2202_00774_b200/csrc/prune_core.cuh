@@ -87,10 +87,12 @@ __device__ __forceinline__ float lane_hi(uint32_t p) {
   return F16 ? __half2float(__ushort_as_half((unsigned short)(p >> 16))) : __uint_as_float(p & 0xFFFF0000u);
 }
 // ... and their magnitudes
+// (the absolute value of the fp32 number clears the same sign bit, NaN payloads included, and rides on the add that
+// consumes it instead of costing an integer instruction)
 template <bool F16>
-__device__ __forceinline__ float lane_lo_abs(uint32_t p) { return lane_lo<F16>(p & 0x00007FFFu); }
+__device__ __forceinline__ float lane_lo_abs(uint32_t p) { return fabsf(lane_lo<F16>(p)); }
 template <bool F16>
-__device__ __forceinline__ float lane_hi_abs(uint32_t p) { return lane_hi<F16>(p & 0x7FFF0000u); }
+__device__ __forceinline__ float lane_hi_abs(uint32_t p) { return fabsf(lane_hi<F16>(p)); }
 
 // Two fp32 values rounded to nearest even and packed (low, high): hardware conversion, finite inputs.
 template <bool F16>
@@ -217,6 +219,40 @@ __device__ __forceinline__ void compressed_slots(uint32_t y0, uint32_t y1, uint3
   const uint32_t pos1 = 0x00010001u + (k23 & 0x00010001u) + (km3 & 0x00010001u);
   const uint32_t nib = pos0 + 4u * pos1;
   nib2 = (nib & 0xFu) | ((nib >> 12) & 0xF0u);
+}
+
+// Magnitude function with the L1 rescale of Section 3.2 for callers that want only the compressed form (n <= 2):
+// the same survivors, sums, divisions and roundings as m4_prune_vector, but the survivors are gathered into their two
+// slots first, so that the sum over the kept elements is one addition of the slots' magnitudes (the other terms of
+// the tree are +0, which changes nothing) and only the slots are multiplied and rounded: half the conversions,
+// products and roundings of the lane-by-lane form. A slot that holds the pad of a chunk with one survivor is +0 and
+// stays +0 (its product with a finite positive scale is +0; where the scale is not finite it is masked out: with one
+// survivor the pad is slot 1 if the survivor is element 0 and slot 0 otherwise).
+// km_i: keep masks as m4_prune_vector returns them (for the bit mask output).
+template <int N, bool F16>
+__device__ __forceinline__ void m4_rescaled_compressed(const uint4& w, uint32_t& slot0, uint32_t& slot1, uint32_t& nib2,
+                                                       uint32_t& km0, uint32_t& km1, uint32_t& km2, uint32_t& km3) {
+  static_assert(N == 1 || N == 2, "a compressed form exists for one or two survivors");
+  uint32_t y0, y1, y2, y3;
+  m4_prune_vector<N, SDGP_MAGNITUDE, F16>(w, 0, 0u, 0u, y0, y1, y2, y3, km0, km1, km2, km3);  // survivors, not yet rescaled
+  const uint32_t p0 = prmt(w.x, w.z, 0x5410), p1 = prmt(w.x, w.z, 0x7632);
+  const uint32_t p2 = prmt(w.y, w.w, 0x5410), p3 = prmt(w.y, w.w, 0x7632);
+  const float tA = sum4_lo_abs<F16>(p0, p1, p2, p3), tB = sum4_hi_abs<F16>(p0, p1, p2, p3);
+  compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
+  const float a0 = lane_lo<F16>(slot0), b0 = lane_hi<F16>(slot0), a1 = lane_lo<F16>(slot1), b1 = lane_hi<F16>(slot1);
+  const float sA = __fadd_rn(fabsf(a0), fabsf(a1)), sB = __fadd_rn(fabsf(b0), fabsf(b1));
+  const float scA = (sA == 0.0f) ? 1.0f : __fdiv_rn(tA, sA);
+  const float scB = (sB == 0.0f) ? 1.0f : __fdiv_rn(tB, sB);
+  const bool finite = (__float_as_uint(tA) & 0x7F800000u) != 0x7F800000u &&
+                      (__float_as_uint(tB) & 0x7F800000u) != 0x7F800000u;
+  if (finite) {  // every product is finite: the hardware's packed rounding applies (see rescale_packed)
+    slot0 = pack_pair_rn<F16>(__fmul_rn(a0, scA), __fmul_rn(b0, scB));
+    slot1 = pack_pair_rn<F16>(__fmul_rn(a1, scA), __fmul_rn(b1, scB));
+  } else {
+    const uint32_t keep0 = N == 2 ? 0xFFFFFFFFu : km0, keep1 = N == 2 ? 0xFFFFFFFFu : ~km0;
+    slot0 = (f32_to_elem_bits<F16>(__fmul_rn(a0, scA)) | (f32_to_elem_bits<F16>(__fmul_rn(b0, scB)) << 16)) & keep0;
+    slot1 = (f32_to_elem_bits<F16>(__fmul_rn(a1, scA)) | (f32_to_elem_bits<F16>(__fmul_rn(b1, scB)) << 16)) & keep1;
+  }
 }
 
 // Groups of 8, 16 or 32 with n <= 2 (Algorithm 1 with the same three pruning functions): the survivors are the

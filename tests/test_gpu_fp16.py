@@ -62,6 +62,24 @@ def test_prune_fp16_bit_exact(n, m, scheme, adversarial):
         assert np.array_equal(host16(meta), ref["meta"])
 
 
+@pytest.mark.parametrize("adversarial", [False, True])
+@pytest.mark.parametrize("scheme", [oracle.RANDOM, oracle.MAGNITUDE, oracle.RESCALED])
+@pytest.mark.parametrize("n,m", [(2, 4), (1, 4), (2, 8), (2, 16)])
+def test_prune_fp16_compressed_outputs_alone(n, m, scheme, adversarial):
+    """What the two-pass path asks for: values, metadata and mask, no dense copy."""
+    import paper_2202_00774_b200 as sdgp
+    rows, K = 203, 256
+    x = fp16_rows(rows, K, seed=n * 5 + m, adversarial=adversarial)
+    mask = torch.full((rows, K // 32), -1, dtype=torch.int32, device="cuda")
+    values = torch.full((rows, K // 2), -1, dtype=torch.int16, device="cuda")
+    meta = torch.full((rows, K // 16), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_prune_typed(dev16(x), n, m, scheme, 78, sdgp.FP16, values=values, meta=meta, mask=mask)
+    ref = oracle.prune(x, n, m, scheme, 78, want=("mask", "values", "meta"), dtype=oracle.FP16)
+    assert np.array_equal(host16(values), ref["values"])
+    assert np.array_equal(host16(meta), ref["meta"])
+    assert np.array_equal(mask.cpu().numpy().view(np.uint32), ref["mask"])
+
+
 def test_fp16_rescale_differs_from_bf16_rescale_on_the_same_bits():
     # guards against the typed entry point silently running the bf16 arithmetic
     import paper_2202_00774_b200 as sdgp

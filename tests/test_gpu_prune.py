@@ -42,6 +42,19 @@ def compare(x, n, m, scheme, seed=0):
         assert np.array_equal(got[key], ref[key]), "%s differs for %d:%d scheme %d" % (key, n, m, scheme)
 
 
+def compare_compressed_only(x, n, m, scheme, seed=0):
+    """The call the two-pass path makes: values and metadata, no dense copy (the rescaled scheme then scales the
+    gathered survivors instead of every lane)."""
+    import paper_2202_00774_b200 as sdgp
+    rows, K = x.shape
+    ref = oracle.prune(x, n, m, scheme, seed, want=("values", "meta"))
+    values = torch.full((rows, K // 2), -1, dtype=torch.int16, device="cuda")
+    meta = torch.full((rows, K // 16), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_prune(dev(x), n, m, scheme, seed, values=values, meta=meta)
+    assert np.array_equal(values.cpu().numpy().view(np.uint16), ref["values"]), "values differ for %d:%d scheme %d" % (n, m, scheme)
+    assert np.array_equal(meta.cpu().numpy().view(np.uint16), ref["meta"]), "meta differs for %d:%d scheme %d" % (n, m, scheme)
+
+
 SCHEMES = [oracle.RANDOM, oracle.MAGNITUDE, oracle.RESCALED]
 NM = [(1, 4), (2, 4), (3, 4), (4, 4), (1, 8), (2, 8), (4, 8), (2, 16), (5, 16), (2, 32), (4, 32), (16, 32)]
 
@@ -98,3 +111,10 @@ def test_prune_full_size_fc_and_sampled_large():
         ref = oracle.prune(big, 2, 4, scheme, 77)
         for key in ("dense", "values", "meta", "mask"):
             assert np.array_equal(got[key], ref[key]), key
+
+
+@pytest.mark.parametrize("scheme", SCHEMES)
+@pytest.mark.parametrize("n,m", [(1, 4), (2, 4), (1, 8), (2, 8), (2, 16), (2, 32)])
+def test_prune_compressed_outputs_alone(n, m, scheme):
+    compare_compressed_only(inputs.relu_masked_laplace_bf16((1237, 160), seed=n * 10 + m), n, m, scheme, seed=3)
+    compare_compressed_only(inputs.adversarial_groups_bf16(513, 96, seed=m + 1), n, m, scheme, seed=4)
