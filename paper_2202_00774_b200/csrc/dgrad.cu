@@ -758,6 +758,8 @@ __device__ __forceinline__ void fused_prune_vectors(const uint4 (&w)[4], int64_t
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2;
     if (M == 4 && SCHEME == SDGP_RESCALED_MAGNITUDE) {
       m4_rescaled_compressed<N, false>(w[v], slot0, slot1, nib2, km0, km1, km2, km3);  // the slots are rescaled, not the lanes
+    } else if (SCHEME == SDGP_RESCALED_MAGNITUDE) {
+      top2_rescaled_compressed<(M == 4 ? 8 : M), false>(w[v], N, part, 0xFFFFFFFFu, slot0, slot1, nib2, km0, km1, km2, km3);
     } else {
       if (M == 4)
         m4_prune_vector<N, SCHEME>(w[v], vbase + vstep * v, seed_lo, seed_hi, y0, y1, y2, y3, km0, km1, km2, km3);

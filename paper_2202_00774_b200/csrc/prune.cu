@@ -357,6 +357,20 @@ prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, 
   for (int it = 0; it < kVecPerThread; ++it) {
     const int64_t v = base + (int64_t)it * kThreads;
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3;
+    if constexpr (SCHEME == SDGP_RESCALED_MAGNITUDE) {
+      if (!dense) {  // (uniform over the grid: every lane of a group takes the same branch and meets in the shuffles)
+        uint32_t slot0, slot1, nib2;
+        top2_rescaled_compressed<M, F16>(in[it], N, (int)(threadIdx.x & (LANES - 1)), 0xFFFFFFFFu, slot0, slot1, nib2, km0, km1,
+                                         km2, km3);
+        if (v < nvec) {
+          const int64_t vo = compressed_index(v, values, meta, pitch);
+          if (mask) emit_mask(v, km0, km1, km2, km3, mask);
+          if (values) values[vo] = make_uint2(prmt(slot0, slot1, 0x5410), prmt(slot0, slot1, 0x7632));
+          if (meta) meta[vo] = (uint8_t)nib2;
+        }
+        continue;
+      }
+    }
     top2_prune_vector<M, SCHEME, F16>(in[it], v, seed_lo, seed_hi, N, (int)(threadIdx.x & (LANES - 1)), 0xFFFFFFFFu, y0, y1, y2,
                                       y3, km0, km1, km2, km3);
     if (v < nvec) emit_packed<true>(v, y0, y1, y2, y3, km0, km1, km2, km3, dense, values, meta, mask, pitch);

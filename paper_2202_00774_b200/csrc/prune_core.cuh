@@ -337,6 +337,40 @@ __device__ __forceinline__ void top2_prune_vector(const uint4& w, int64_t v, uin
   }
 }
 
+// top2_prune_vector for the magnitude function with the L1 rescale, for callers that want only the compressed form:
+// as m4_rescaled_compressed, the survivors of the vector's two chunks are gathered into the slots first; a chunk's share of
+// the sum over the kept elements is then one addition of its slots' magnitudes (a group keeps at most two elements, so
+// every other term of the oracle's tree is +0) and only the slots are scaled and rounded.
+template <int M, bool F16>
+__device__ __forceinline__ void top2_rescaled_compressed(const uint4& w, int n, int part, unsigned lanes, uint32_t& slot0,
+                                                         uint32_t& slot1, uint32_t& nib2, uint32_t& km0, uint32_t& km1,
+                                                         uint32_t& km2, uint32_t& km3) {
+  constexpr int LANES = M / 8;
+  uint32_t y0, y1, y2, y3;
+  top2_prune_vector<M, SDGP_MAGNITUDE, F16>(w, 0, 0u, 0u, n, part, lanes, y0, y1, y2, y3, km0, km1, km2, km3);  // not yet rescaled
+  const uint32_t p0 = prmt(w.x, w.z, 0x5410), p1 = prmt(w.x, w.z, 0x7632);
+  const uint32_t p2 = prmt(w.y, w.w, 0x5410), p3 = prmt(w.y, w.w, 0x7632);
+  float tsum = __fadd_rn(sum4_lo_abs<F16>(p0, p1, p2, p3), sum4_hi_abs<F16>(p0, p1, p2, p3));
+  compressed_slots(y0, y1, y2, y3, km0, km1, km2, km3, slot0, slot1, nib2);
+  const float a0 = lane_lo<F16>(slot0), b0 = lane_hi<F16>(slot0), a1 = lane_lo<F16>(slot1), b1 = lane_hi<F16>(slot1);
+  float ssum = __fadd_rn(__fadd_rn(fabsf(a0), fabsf(a1)), __fadd_rn(fabsf(b0), fabsf(b1)));
+#pragma unroll
+  for (int d = 1; d < LANES; d <<= 1) {
+    tsum = __fadd_rn(tsum, __shfl_xor_sync(lanes, tsum, d));
+    ssum = __fadd_rn(ssum, __shfl_xor_sync(lanes, ssum, d));
+  }
+  const float sc = (ssum == 0.0f) ? 1.0f : __fdiv_rn(tsum, ssum);
+  if ((__float_as_uint(tsum) & 0x7F800000u) != 0x7F800000u) {  // finite sums: finite scale, a +0 pad stays +0
+    slot0 = pack_pair_rn<F16>(__fmul_rn(a0, sc), __fmul_rn(b0, sc));
+    slot1 = pack_pair_rn<F16>(__fmul_rn(a1, sc), __fmul_rn(b1, sc));
+  } else {
+    // which slots hold survivors: slot 1 if anything but element 0 of the chunk is kept, slot 0 if element 0 is kept or two are
+    const uint32_t keep1 = km1 | km2 | km3, keep0 = km0 | (km1 & km2) | (km3 & (km1 | km2));
+    slot0 = (f32_to_elem_bits<F16>(__fmul_rn(a0, sc)) | (f32_to_elem_bits<F16>(__fmul_rn(b0, sc)) << 16)) & keep0;
+    slot1 = (f32_to_elem_bits<F16>(__fmul_rn(a1, sc)) | (f32_to_elem_bits<F16>(__fmul_rn(b1, sc)) << 16)) & keep1;
+  }
+}
+
 // One group of 16 whose two vectors (numbers v and v + 1) are held by the same thread.
 template <int SCHEME, bool F16 = false>
 __device__ __forceinline__ void top2_prune_group16(const uint4& wa, const uint4& wb, int64_t v, uint32_t seed_lo,
