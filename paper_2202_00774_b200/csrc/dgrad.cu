@@ -676,12 +676,11 @@ dgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 constexpr int kHaloRows = 16;  // 8-pixel rows of a strip: the 128 rows of an accumulator
 constexpr int kHaloAStages = 4;  // at most: A stages in use are p.a_stages = 2, or 4 when the boxes are small (a power of two)
 // Warp roles of the fused whole-filter-reuse kernel (24 warps: registers are granted to warps in fours, and
-// 24 x 80 registers is what fits). Warp w runs on scheduler w % 4; the busy pruning warps keep off the scheduler
-// of the warp that issues the MMAs (with them on it a tap took 900 instead of 750 clocks): warp 0 streams W,
-// warp 1 issues the MMAs, warps 4..7 are the epilogue (one per TMEM lane quarter), and of the rest those
-// with w % 4 != 1 prune (2, 3, 8, 10..12, 14..16, 18..20, 22, 23: fourteen warps); warps 9, 13, 17 and 21
-// have no role.
-constexpr int kPruneWarps = 14;
+// 24 x 80 registers is what fits): warp 0 streams W, warp 1 issues the MMAs, warps 4..7 are the epilogue (one per
+// TMEM lane quarter) and the other eighteen prune. Warp w runs on scheduler w % 4, so four pruning warps (9, 13, 17,
+// 21) share the scheduler of the MMA-issuing warp; measured, their integer-pipe time is worth more than the issue
+// slots they take from it (14 -> 16 -> 18 pruning warps: 1062 -> 1107 -> 1111 TFLOP/s on the ResNet-9 chain).
+constexpr int kPruneWarps = 18;
 constexpr unsigned kIdleWaitNs = 200;  // sleep between polls of the waits that are off the critical path
 constexpr int kThreadsHaloFused = 24 * 32;
 
@@ -1104,7 +1103,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (lane == 0) ptx::mbar_arrive_cluster(&meta_ready[ast], 0);
       }
     }
-  } else if (FUSED && (warp & 3) != 1 && (warp < 4 || warp >= 8)) {
+  } else if (FUSED && (((warp & 3) != 1 && (warp < 4 || warp >= 8)) || warp == 9 || warp == 13 || warp == 17 || warp == 21)) {
     // ------------------------------------------------------------ pruner
     // Work unit = 8 pixel rows of a box = one pass of a warp: lane = (row, c), and the thread owns vectors
     // c, c + 4, c + 8 and c + 12 (8 channels each) of the row's 16, so that every load instruction of the
@@ -1116,8 +1115,9 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // shared-memory traffic to the two-pass kernel's - which matters because with 64 or 128 input
     // channels the MMAs themselves are bound by shared-memory reads.
     {
-      // number of this pruning warp, 0 .. kPruneWarps - 1: warps 2, 3, 8, then 10.. without those on scheduler 1
-      const int pw = warp < 4 ? warp - 2 : warp == 8 ? 2 : 3 + (warp - 10) - ((warp - 9) >> 2);
+      // number of this pruning warp, 0 .. kPruneWarps - 1: warps 2, 3, 8, then 10.. without those on scheduler 1 (0..13),
+      // then the four on scheduler 1
+      const int pw = warp == 9 ? 14 : warp == 13 ? 15 : warp == 17 ? 16 : warp == 21 ? 17 : warp < 4 ? warp - 2 : warp == 8 ? 2 : 3 + (warp - 10) - ((warp - 9) >> 2);
       const int upb = (p.img_rows + 7) >> 3;  // units per box
       const int a_uses = my_tiles * p.k_uses;
       const int row8 = lane >> 2, c = lane & 3;
