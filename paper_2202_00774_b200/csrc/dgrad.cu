@@ -719,6 +719,13 @@ struct HaloParams {
   int k_uses;              // A boxes per tile set: k_blocks * ss
   int a_stages, a_shift;   // A ring depth (2 or 4) and its log2
   int img_rows;            // pitch * img_h
+  // Fused mode, work units of the pruning warps (8 box pixels each). static_pad == 0: unit u = box pixels 8u .. 8u + 7
+  // in row-major order, units_per_box = ceil(img_rows / 8). static_pad == 1 (a tile set spans its images from edge to
+  // edge, so the halo rows and columns of EVERY box are padding): the stages are cleared once when the kernel starts and
+  // only the units inside the images are ever pruned and written - unit u = 8 pixels from column unit_col0 + 8 * (u % nt)
+  // of box row unit_row0 + u / nt, units_per_box = H * tb * nt. Fewer units per box also means fewer rounds of units
+  // per pruning warp, which is what sets the time a box takes.
+  int static_pad, units_per_box, unit_row0, unit_col0;
   int w_stages;
   int meta_col, meta_shared, out_bufs;
   int a_bytes, eraw_bytes, w_bytes;  // per stage
@@ -816,7 +823,7 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // fused: A and its metadata rows are complete when every pruning warp has arrived
       // (a_full: the warps of both CTAs; meta_full: this CTA's)
       // (one arrival per work unit of the box: 8 pixel rows)
-      ptx::mbar_init(&a_full[s], FUSED ? 2 * ((p.img_rows + 7) >> 3) : 1);
+      ptx::mbar_init(&a_full[s], FUSED ? 2 * p.units_per_box : 1);
       ptx::mbar_init(&a_empty[s], 1);
       ptx::mbar_init(&meta_full[s], 1);
       ptx::mbar_init(&meta_ready[s], 8);  // four metadata warps in each CTA
@@ -1118,7 +1125,17 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // number of this pruning warp, 0 .. kPruneWarps - 1: warps 2, 3, 8, then 10.. without those on scheduler 1 (0..13),
       // then the four on scheduler 1
       const int pw = warp == 9 ? 14 : warp == 13 ? 15 : warp == 17 ? 16 : warp == 21 ? 17 : warp < 4 ? warp - 2 : warp == 8 ? 2 : 3 + (warp - 10) - ((warp - 9) >> 2);
-      const int upb = (p.img_rows + 7) >> 3;  // units per box
+      const int upb = p.units_per_box;
+      if (p.static_pad) {
+        // every stage starts out as padding: zero values, metadata naming the position pair (0, 1)
+        const int words = p.a_stages * p.a_bytes >> 4;
+        for (int k = pw * 32 + lane; k < words; k += 32 * kPruneWarps) ((uint4*)sA)[k] = make_uint4(0u, 0u, 0u, 0u);
+        const int mwords = p.a_stages * p.meta_bytes >> 4;
+        for (int k = pw * 32 + lane; k < mwords; k += 32 * kPruneWarps)
+          ((uint4*)sMeta)[k] = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+        ptx::fence_proxy_async_smem();
+        ptx::named_bar_sync(3, 32 * kPruneWarps);  // no unit is announced before every stage is cleared
+      }
       const int a_uses = my_tiles * p.k_uses;
       const int row8 = lane >> 2, c = lane & 3;
       const uint32_t px_bytes = (uint32_t)p.Cout * 2u;
@@ -1185,7 +1202,12 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               }
             }
           }
-          u_i = 8 * o + row8;
+          if (p.static_pad) {
+            const int ur = NT == 2 ? (o >> 1) : o, uc = NT == 2 ? (o & 1) : 0;
+            u_i = (p.unit_row0 + ur) * p.pitch + p.unit_col0 + 8 * uc + row8;
+          } else {
+            u_i = 8 * o + row8;
+          }
           u_ia = ia;
           const int kb = org_kb0 + ku / p.ss;
           u_kb = kb;
@@ -1227,6 +1249,10 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int i = u_i, cia = u_ia;
           const bool live = u_live;
           if (boxes_seen <= cia) {  // the MMAs that read this stage's previous contents (box cia - 2) have completed
+            // (whatever this warp still owes an earlier box goes out first: with fewer units per box than pruning warps
+            // the stage waited for here can be the very one that unit belongs to)
+            announce();
+            pending_ast = -1;
             bool ok = true;
             while (boxes_seen <= cia) {
               const int bs = boxes_seen & (p.a_stages - 1);
@@ -1634,6 +1660,8 @@ bool plan_halo(HaloParams* p, int nt) {
     p->tb = kHaloRows / p->th;
     p->img_h = (p->th + p->R - 1) * p->tb;
     p->img_rows = p->pitch * p->img_h;
+    p->static_pad = 0;
+    p->units_per_box = (p->img_rows + 7) / 8;
     if (p->pitch > 256 || p->img_h > 256) return false;
     p->a_bytes = round_up(p->img_rows * 128, 1024);
     p->eraw_bytes = (SPARSE && !FUSED) ? round_up(p->img_rows * 16, 128) : 0;
@@ -1683,6 +1711,21 @@ bool plan_halo(HaloParams* p, int nt) {
     if (p->smem_bytes > kSmemLimit) return false;
     p->sets_w = p->split ? 1 : (p->W + 8 * nt - 1) / (8 * nt);
     p->tiles_h = (p->H + p->th - 1) / p->th;
+    if (FUSED && p->sets_w == 1 && p->tiles_h == 1 && p->a_bytes % 16 == 0 && p->meta_bytes % 16 == 0) {
+      // Box pixel row 0 is dL/dO row p0 and box column 0 is dL/dO column q0 (every tile set starts at h0 = w0 = 0); the
+      // rows and columns of the box that lie inside dL/dO's P x Q pixels are the same for every box.
+      const int p0 = p->pad_h - (p->R - 1), q0 = p->pad_w - (p->sb - 1);
+      const int row_lo = p0 < 0 ? -p0 : 0;
+      const int row_hi = (p->th + p->R - 1) < (p->P - p0) ? (p->th + p->R - 1) : (p->P - p0);
+      const int col_lo = p->split ? 0 : (q0 < 0 ? -q0 : 0);
+      const bool cols_fit = p->split ? p->Q <= 4 : (p->Q - q0 <= col_lo + 8 * nt);
+      if (row_hi > row_lo && cols_fit) {
+        p->static_pad = 1;
+        p->unit_row0 = row_lo * p->tb;
+        p->unit_col0 = col_lo;
+        p->units_per_box = (row_hi - row_lo) * p->tb * nt;
+      }
+    }
     const int tile_imgs = p->tb * p->img_per_row;  // images of one tile set
     const int64_t m_sets = (int64_t)p->sets_w * p->tiles_h * ((p->B + tile_imgs - 1) / tile_imgs);
     if (m_sets * p->tiles_n > 0x3FFFFFFF) return false;

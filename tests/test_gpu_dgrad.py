@@ -438,6 +438,12 @@ HALO_CASES = [
     (4, 3, 4, 64, 128, 3, 3, 1, 1),         # ... three pixel rows
     (10, 4, 4, 64, 128, 5, 5, 1, 2),        # ... 5 x 5 filter
     (8, 8, 8, 64, 128, 3, 3, 2, 1),         # stride 2 on 8 x 8: 4 x 4 parity classes written through strided views
+    (3, 15, 15, 64, 128, 3, 3, 2, 1),       # stride 2 on 15 x 15: a class of 7 rows reads all 8 rows of dL/dO
+    (2, 14, 14, 128, 128, 3, 3, 1, 1),      # 14 columns under two strips of 8
+    (2, 12, 16, 64, 128, 3, 3, 1, 1),       # 12 rows under a strip of 16
+    (3, 16, 16, 64, 128, 3, 3, 1, 0),       # no padding: dL/dO is 14 x 14 and the box starts two pixels inside it
+    (3, 7, 8, 64, 128, 3, 3, 1, 1),         # 7 rows of two images
+    (5, 16, 16, 64, 128, 3, 3, 1, 2),       # padding 2: dL/dO is 18 x 18, larger than the image
 ]
 
 
