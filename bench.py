@@ -72,7 +72,7 @@ def layer_inputs(l, workload, seed, dtype="bf16"):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the seven sparse dgrad launches of one
 # resnet9 two-pass step, from the ncu capture summarised in profiles/traffic_dgrad_sparse_resnet9.md,
 # and the hash of the kernel sources it was taken with (the figure is dropped once they change).
-NCU_TRAFFIC = {"workload": "resnet9", "mode": "two_pass", "bytes_per_step": 214.2e6, "sources_sha": "78eed029538da942"}
+NCU_TRAFFIC = {"workload": "resnet9", "mode": "two_pass", "bytes_per_step": 213.0e6, "sources_sha": "ce36a0ae91d3cc31"}
 KERNEL_SOURCES = ["dgrad.cu", "ptx.cuh"]   # all the code of the non-fused data-gradient kernels
 
 
@@ -372,6 +372,22 @@ def run_ours(args, layers):
     value = world * total_flops / (ms_per_step * 1e-3) / 1e12
     dense_value = world * total_flops / (ms_dense / dense_steps * 1e-3) / 1e12
 
+    # The same chain with the prune inside the data-gradient kernel (one launch per layer), beside the two-pass step
+    # of a default run: same tensors, same graph treatment, same number of timed replays as the dense twin.
+    fused_chain = None
+    if (args.mode == "two_pass" and not masked and n <= 2 and args.workload == "resnet9"
+            and not (args.dtype == "fp16" and args.scheme == "rescaled")):
+        def fused_step():
+            for i in order:
+                l = layers[i]
+                sdgp.sdgp_dgrad_conv2d_typed(dO[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, 1234, DT, flags=sdgp.FLAG_FUSED)
+        g_fused = capture(fused_step)
+        ms_fused = timed(g_fused.replay, dense_steps, max(3, args.warmup // 2))
+        fused_value = world * total_flops / (ms_fused / dense_steps * 1e-3) / 1e12
+        fused_chain = {"value": fused_value, "unit": UNIT, "ms_per_step": ms_fused / dense_steps,
+                       "speedup_vs_dense": fused_value / dense_value, "steps": dense_steps,
+                       "what": "the step as %d fused prune + sparse dgrad launches (SDGP_FLAG_FUSED), one CUDA graph" % len(layers)}
+
     # ---- per-kernel timing: the same step captured with timing events between the kernels
     # (event-record graph nodes), replayed with the same data and cache state as the timed step ----
     vals = [torch.empty(l.B * l.P * l.Q * l.Cout // (1 if masked else 2), dtype=torch.int16, device="cuda") for l in layers]
@@ -575,7 +591,7 @@ def run_ours(args, layers):
                        "mode": "masked (pruned dense copy + dense kernel)" if masked else args.mode, "flops": "2*M*N*K of the implicit GEMM per layer",
                        "l2": "inputs larger than L2 (step touches %.0f MB)" % ((prune_bytes + d2h) / 1e6),
                        "launch": "one CUDA graph per step", "replicas": world},
-            "speedup_vs_dense": value / dense_value, "dense_tflops": dense_value,
+            "speedup_vs_dense": value / dense_value, "dense_tflops": dense_value, "fused_chain": fused_chain,
             "prune_gbs": prune_gbs, "prune_frac_of_hbm": (prune_gbs / pk["hbm"]) if prune_gbs else None,
             "prune_frac_of_nominal_8tbs": (prune_gbs / 8000.0) if prune_gbs else None,
             "prune_gbs_between_event_nodes": prune_gbs_events,
