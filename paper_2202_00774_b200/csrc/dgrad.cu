@@ -1248,19 +1248,6 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         while (more) {
           const int i = u_i, cia = u_ia;
           const bool live = u_live;
-          if (boxes_seen <= cia) {  // the MMAs that read this stage's previous contents (box cia - 2) have completed
-            // (whatever this warp still owes an earlier box goes out first: with fewer units per box than pruning warps
-            // the stage waited for here can be the very one that unit belongs to)
-            announce();
-            pending_ast = -1;
-            bool ok = true;
-            while (boxes_seen <= cia) {
-              const int bs = boxes_seen & (p.a_stages - 1);
-              if (!ptx::mbar_wait<kIdleWaitNs>(&a_empty[bs], (((uint32_t)boxes_seen >> p.a_shift) & 1u) ^ 1u, err, 0x900u + bs)) { ok = false; break; }
-              ++boxes_seen;
-            }
-            if (!__all_sync(0xFFFFFFFFu, ok)) break;
-          }
           const int ast = cia & (p.a_stages - 1);
           uint2 out[4];
           uint32_t metaw;
@@ -1276,6 +1263,20 @@ dgrad_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           // the registers of this unit are free: the loads of the next one go out before this one's stores
           more = ia < a_uses;
           if (more) fetch();
+          // only now, with the unit pruned and the next one's loads in flight, does the warp need the stage
+          if (boxes_seen <= cia) {  // the MMAs that read this stage's previous contents (box cia - 2) have completed
+            // (whatever this warp still owes an earlier box goes out first: with fewer units per box than pruning warps
+            // the stage waited for here can be the very one that unit belongs to)
+            announce();
+            pending_ast = -1;
+            bool ok = true;
+            while (boxes_seen <= cia) {
+              const int bs = boxes_seen & (p.a_stages - 1);
+              if (!ptx::mbar_wait<kIdleWaitNs>(&a_empty[bs], (((uint32_t)boxes_seen >> p.a_shift) & 1u) ^ 1u, err, 0x900u + bs)) { ok = false; break; }
+              ++boxes_seen;
+            }
+            if (!__all_sync(0xFFFFFFFFu, ok)) break;
+          }
           announce();
           const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, metaw, 1);  // (all lanes: before the rows part ways)
           if (i < p.img_rows) {
