@@ -72,7 +72,7 @@ def layer_inputs(l, workload, seed, dtype="bf16"):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the seven sparse dgrad launches of one
 # resnet9 two-pass step, from the ncu capture summarised in profiles/traffic_dgrad_sparse_resnet9.md,
 # and the hash of the kernel sources it was taken with (the figure is dropped once they change).
-NCU_TRAFFIC = {"workload": "resnet9", "mode": "two_pass", "bytes_per_step": 213.0e6, "sources_sha": "ce36a0ae91d3cc31"}
+NCU_TRAFFIC = {"workload": "resnet9", "mode": "two_pass", "bytes_per_step": 213.0e6, "sources_sha": "9e2b4e39f6d4dd4c"}
 KERNEL_SOURCES = ["dgrad.cu", "ptx.cuh"]   # all the code of the non-fused data-gradient kernels
 
 
