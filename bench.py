@@ -365,7 +365,7 @@ def run_ours(args, layers):
     # Clocks are sampled over the timed regions of the step and of the kernel-only graphs below (the step
     # itself may last only a few milliseconds; those graphs are replayed for at least 0.3 s each).
     ms_sparse = timed(g_sparse.replay, args.steps, args.warmup, sample_clocks=True)
-    dense_steps = max(3, args.steps // 4)
+    dense_steps = max(20, args.steps // 4)   # a replay lasts about 0.3 ms
     ms_dense = timed(g_dense.replay, dense_steps, max(3, args.warmup // 2))
 
     ms_per_step = ms_sparse / args.steps
@@ -387,6 +387,44 @@ def run_ours(args, layers):
         fused_chain = {"value": fused_value, "unit": UNIT, "ms_per_step": ms_fused / dense_steps,
                        "speedup_vs_dense": fused_value / dense_value, "steps": dense_steps,
                        "what": "the step as %d fused prune + sparse dgrad launches (SDGP_FLAG_FUSED), one CUDA graph" % len(layers)}
+
+    # ---- the chain with the ReLU below every convolution (Section 2.1, Fig. 2: dL/dO comes out of the layer above;
+    # Section 3.1: the unpruned tensor is kept for the weight gradient). Sparse side: the producer forms dL/dO from
+    # the gradient above the ReLU and the activation, writes it and its compressed pruned copy in one pass, then the
+    # sparse contraction. Dense side: a plain ReLU backward (the same kernel with n = m, which writes dL/dO only),
+    # then the dense twin. Both sides pay for the pass over the gradient; each is one CUDA graph of 14 launches. ----
+    relu_chain = None
+    if (args.mode == "two_pass" and not masked and n <= 2 and args.workload == "resnet9" and not args.no_other_configs
+            and all(l.Cout % 128 == 0 for l in layers)):
+        act = [torch.randn(t.shape, device="cuda").clamp_(min=0).to(torch.float16 if args.dtype == "fp16" else torch.bfloat16)
+               .view(torch.int16) for t in dO]
+        grad = [torch.empty_like(t) for t in dO]
+        cv = [torch.empty(l.B * l.P * l.Q * l.Cout // 2, dtype=torch.int16, device="cuda") for l in layers]
+        cm = [torch.empty(l.B * l.P * l.Q * l.Cout // 16, dtype=torch.int16, device="cuda") for l in layers]
+
+        def relu_sparse_step():
+            for i in order:
+                l = layers[i]
+                sdgp.sdgp_relu_backward_prune(dO[i].view(-1, l.Cout), act[i].view(-1, l.Cout), n, m, scheme, 1234, dtype=DT,
+                                              grad=grad[i].view(-1, l.Cout), values=cv[i], meta=cm[i])
+                sdgp.sdgp_spmm_conv2d_typed(cv[i].view(l.B, l.P, l.Q, l.Cout // 2), cm[i].view(l.B, l.P, l.Q, l.Cout // 16),
+                                            Wt[i], dD[i], l.stride, l.pad, DT)
+
+        def relu_dense_step():
+            for i in order:
+                l = layers[i]
+                sdgp.sdgp_relu_backward_prune(dO[i].view(-1, l.Cout), act[i].view(-1, l.Cout), m, m, scheme, 0, dtype=DT,
+                                              grad=grad[i].view(-1, l.Cout))
+                sdgp.sdgp_dgrad_conv2d_typed(grad[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, 0, DT, flags=sdgp.FLAG_DENSE)
+
+        g_rs, g_rd = capture(relu_sparse_step), capture(relu_dense_step)
+        ms_rs = timed(g_rs.replay, dense_steps, max(3, args.warmup // 2)) / dense_steps
+        ms_rd = timed(g_rd.replay, dense_steps, max(3, args.warmup // 2)) / dense_steps
+        relu_chain = {"sparse_ms_per_step": ms_rs, "dense_ms_per_step": ms_rd, "speedup_vs_dense": ms_rd / ms_rs,
+                      "steps": dense_steps,
+                      "what": "every layer as [ReLU backward + prune in one pass (unpruned dL/dO kept), sparse contraction] "
+                              "against [plain ReLU backward, dense twin], one CUDA graph each"}
+        del act, grad, cv, cm, g_rs, g_rd
 
     # ---- per-kernel timing: the same step captured with timing events between the kernels
     # (event-record graph nodes), replayed with the same data and cache state as the timed step ----
@@ -592,6 +630,7 @@ def run_ours(args, layers):
                        "l2": "inputs larger than L2 (step touches %.0f MB)" % ((prune_bytes + d2h) / 1e6),
                        "launch": "one CUDA graph per step", "replicas": world},
             "speedup_vs_dense": value / dense_value, "dense_tflops": dense_value, "fused_chain": fused_chain,
+            "relu_chain": relu_chain,
             "prune_gbs": prune_gbs, "prune_frac_of_hbm": (prune_gbs / pk["hbm"]) if prune_gbs else None,
             "prune_frac_of_nominal_8tbs": (prune_gbs / 8000.0) if prune_gbs else None,
             "prune_gbs_between_event_nodes": prune_gbs_events,
