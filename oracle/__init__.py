@@ -61,6 +61,8 @@ def _load():
             lib.oracle_f16_to_f64.restype = dbl
             lib.oracle_relu_backward.argtypes = [vp, vp, i64, i32, vp]
             lib.oracle_relu_backward.restype = i32
+            lib.oracle_residual_relu_backward.argtypes = [vp, vp, vp, i64, i32, vp]
+            lib.oracle_residual_relu_backward.restype = i32
             lib.oracle_expand.argtypes = [vp, vp, i64, i64, vp]
             lib.oracle_expand.restype = i32
             lib.oracle_dgrad_linear.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64]
@@ -136,6 +138,28 @@ def relu_backward_prune(dY, act, n, m, scheme, seed=0, want=("dense", "values", 
     """The producer of the pruned dL/dO: ReLU backward, then Algorithm 1 on the result. Returns the dict of
     ``prune`` plus ``"grad"``, the unpruned dL/dO that the weight gradient still needs (Section 3.1)."""
     grad = relu_backward(dY, act, dtype)
+    out = prune(grad, n, m, scheme, seed, want, dtype)
+    out["grad"] = grad
+    return out
+
+
+def residual_relu_backward(dY, dSkip, act, dtype=BF16):
+    """dL/dO below the ReLU that follows a residual addition (the ResNets of Section 4): the two gradients handed down
+    to the ReLU's output are added (single precision, rounded to the 16-bit type), and the sum passes where ``act`` is
+    positive. Arrays of 16-bit patterns of the same shape."""
+    dY, dSkip, act = _u16(dY), _u16(dSkip), _u16(act)
+    if dY.shape != act.shape or dY.shape != dSkip.shape:
+        raise ValueError("dY, dSkip and act must have the same shape")
+    out = np.empty(dY.shape, np.uint16)
+    rc = _load().oracle_residual_relu_backward(_ptr(dY), _ptr(dSkip), _ptr(act), dY.size, dtype, _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_residual_relu_backward rejected its arguments")
+    return out
+
+
+def residual_relu_backward_prune(dY, dSkip, act, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask"), dtype=BF16):
+    """``residual_relu_backward`` followed by Algorithm 1; ``"grad"`` is the unpruned dL/dO (Section 3.1)."""
+    grad = residual_relu_backward(dY, dSkip, act, dtype)
     out = prune(grad, n, m, scheme, seed, want, dtype)
     out["grad"] = grad
     return out

@@ -543,6 +543,24 @@ int oracle_relu_backward(const uint16_t* dY, const uint16_t* act, int64_t count,
   return ORACLE_OK;
 }
 
+/* Where a residual connection joins its branch (the ResNets of Section 4: y = ReLU(x + F(x))), the gradient
+ * that reaches the ReLU is the SUM of what the two consumers of y hand down (Section 2.1 / Fig. 2: each
+ * hands down its own data gradient). The producer of dL/dO below such a ReLU therefore adds the two
+ * gradients first: s[e] = dY[e] + dSkip[e], one IEEE single-precision addition of the two 16-bit values
+ * (both exact in single precision), rounded to the tensors' 16-bit type to nearest-even (a NaN sum is stored
+ * as the canonical quiet NaN, as everywhere in this file); then dO[e] = s[e] where the activation is
+ * positive and +0.0 elsewhere. */
+int oracle_residual_relu_backward(const uint16_t* dY, const uint16_t* dSkip, const uint16_t* act, int64_t count, int dtype,
+                                  uint16_t* dO) {
+  if (!dY || !dSkip || !act || !dO || count < 0 || (dtype != ORACLE_BF16 && dtype != ORACLE_FP16)) return ORACLE_ERR_ARG;
+  for (int64_t e = 0; e < count; ++e) {
+    const float a = elem_to_f32(act[e], dtype);
+    volatile float s = elem_to_f32(dY[e], dtype) + elem_to_f32(dSkip[e], dtype); /* one rounding, to single precision */
+    dO[e] = (a > 0.0f) ? elem_from_f32(s, dtype) : (uint16_t)0;
+  }
+  return ORACLE_OK;
+}
+
 /* Section 4.3 estimator: removing a fraction (1 - n/m) of a pass that takes
  * share f of the runtime reduces the total by f * (1 - n/m). */
 double oracle_runtime_reduction(double share, int n, int m) {

@@ -66,3 +66,82 @@ def test_worked_example_passes_through_an_open_relu():
     act[0, 1] = 0
     out = oracle.relu_backward_prune(dY, act, 2, 4, oracle.MAGNITUDE, want=("dense",))
     assert np.array_equal(out["dense"][0, :4], bits([0.0, 0.0, -3.0, 2.0]))
+
+
+# ---- the producer below the ReLU that follows a residual addition (the two gradients are added first) ----
+
+
+def test_residual_sum_hand_examples_of_rounding():
+    # bf16 keeps 8 significant bits: 1 + 2^-8 lies exactly between 1 and 1 + 2^-7 and goes to the even one (1);
+    # (1 + 2^-7) + 2^-8 lies between 1 + 2^-7 (odd) and 1 + 2^-6 (even) and goes up; 1 + 3 * 2^-9 is above the midpoint
+    one, ulp, half_ulp = 0x3F80, 0x3C00, 0x3B80          # 1.0, 2^-7, 2^-8
+    act = np.full(8, 0x3F80, np.uint16)
+    dY = np.array([one, one + 1, one, 0x4049, 0xC049, 0x7F80, 0x7F80, 0x0000], np.uint16)
+    dSkip = np.array([half_ulp, half_ulp, 0x3BC0, 0xC049, 0x4049, 0xFF80, 0x3F80, 0x8000], np.uint16)
+    got = oracle.residual_relu_backward(dY, dSkip, act)
+    #            tie->even  tie->even(up)  above the tie   x + (-x)  (-x) + x   inf - inf   inf + 1   +0 + -0
+    want = np.array([one,    one + 2,       one + 1,        0x0000,   0x0000,    0x7FC0,     0x7F80,   0x0000], np.uint16)
+    assert np.array_equal(got, want)
+    assert ulp == 0x3C00 and inputs.bf16_bits_to_f32(np.array([one + 1], np.uint16))[0] == 1.0078125
+
+
+def test_residual_sum_equals_the_libraries_16_bit_addition():
+    # torch adds bfloat16 tensors, numpy adds float16 arrays: both libraries round the sum of the two numbers to the
+    # 16-bit type, which is what the gradient accumulation of a framework does at a residual connection
+    import torch
+    rng = np.random.default_rng(11)
+    shape = (96, 128)
+    act = np.full(shape, 0x3F80, np.uint16)
+    for scale in (1.0, 1e-3, 300.0):
+        a = bits(rng.standard_normal(shape) * scale)
+        b = bits(rng.laplace(size=shape))
+        want = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) + torch.from_numpy(b.view(np.int16)).view(torch.bfloat16))
+        assert np.array_equal(oracle.residual_relu_backward(a, b, act), want.view(torch.int16).numpy().view(np.uint16))
+    # every pair of exponents, so that one operand vanishes, half-vanishes or cancels against the other
+    a = np.repeat(np.arange(0x0080, 0x7F80, 0x0155, dtype=np.uint16), 64)
+    b = np.tile(np.arange(0x8080, 0xFF80, 0x0200, dtype=np.uint16), a.size // 64 + 1)[:a.size]
+    want = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) + torch.from_numpy(b.view(np.int16)).view(torch.bfloat16)
+    assert np.array_equal(oracle.residual_relu_backward(a, b, np.full(a.shape, 0x3F80, np.uint16)),
+                          want.view(torch.int16).numpy().view(np.uint16))
+    # binary16
+    h = rng.standard_normal(shape).astype(np.float16)
+    k = (rng.standard_normal(shape) * 0.01).astype(np.float16)
+    got = oracle.residual_relu_backward(h.view(np.uint16), k.view(np.uint16), np.full(shape, 0x3C00, np.uint16), oracle.FP16)
+    assert np.array_equal(got, (h + k).view(np.uint16))
+    big = np.array([65504.0, 65504.0, -65504.0, 6.1e-5, 5.96e-8], np.float16)        # overflow to infinity, subnormal sums
+    small = np.array([32.0, 8.0, -32.0, -6.0e-5, 5.96e-8], np.float16)
+    got = oracle.residual_relu_backward(big.view(np.uint16), small.view(np.uint16), np.full(5, 0x3C00, np.uint16), oracle.FP16)
+    with np.errstate(over="ignore"):
+        assert np.array_equal(got, (big + small).view(np.uint16))
+
+
+def test_residual_sum_symmetry_gate_and_reduction_to_the_plain_producer():
+    rng = np.random.default_rng(12)
+    shape = (64, 96)
+    dY, dSkip = bits(rng.laplace(size=shape)), bits(rng.laplace(size=shape) * 0.25)
+    act = bits(np.maximum(rng.standard_normal(shape), 0.0))
+    got = oracle.residual_relu_backward(dY, dSkip, act)
+    assert np.array_equal(got, oracle.residual_relu_backward(dSkip, dY, act))           # addition commutes, bit for bit
+    blocked = inputs.bf16_bits_to_f32(act) <= 0
+    assert blocked.any() and np.all(got[blocked] == 0)
+    # the gate is the plain producer's: the sum, formed everywhere, then passed through relu_backward
+    everywhere = oracle.residual_relu_backward(dY, dSkip, np.full(shape, 0x3F80, np.uint16))
+    assert np.array_equal(got, oracle.relu_backward(everywhere, act))
+    # with nothing on the skip path the sum is dY itself (its zeros are +0.0 here)
+    assert np.array_equal(oracle.residual_relu_backward(dY, np.zeros(shape, np.uint16), act), oracle.relu_backward(dY, act))
+    # an activation that is not a number, negative zero or negative passes nothing
+    odd = np.array([0x7FC0, 0x8000, 0xBF80, 0xFF80], np.uint16)
+    assert not oracle.residual_relu_backward(dY.ravel()[:4], dSkip.ravel()[:4], odd).any()
+
+
+def test_residual_producer_is_the_sum_followed_by_algorithm_1():
+    rng = np.random.default_rng(13)
+    dY, dSkip = bits(rng.laplace(size=(48, 64))), bits(rng.laplace(size=(48, 64)))
+    act = bits(np.maximum(rng.standard_normal((48, 64)), 0.0))
+    out = oracle.residual_relu_backward_prune(dY, dSkip, act, 2, 4, oracle.MAGNITUDE)
+    ref = oracle.prune(out["grad"], 2, 4, oracle.MAGNITUDE)
+    for key in ("dense", "values", "meta", "mask"):
+        assert np.array_equal(out[key], ref[key])
+    f = inputs.bf16_bits_to_f32
+    kept = f(out["dense"]) != 0
+    assert np.all(f(out["dense"])[kept] == f(out["grad"])[kept]) and kept.reshape(48, 16, 4).sum(-1).max() <= 2
