@@ -424,7 +424,19 @@ def run_ours(args, layers):
                       "steps": dense_steps,
                       "what": "every layer as [ReLU backward + prune in one pass (unpruned dL/dO kept), sparse contraction] "
                               "against [plain ReLU backward, dense twin], one CUDA graph each"}
-        del act, grad, cv, cm, g_rs, g_rd
+        # the producer below a ReLU that follows a residual addition (two gradients added in the same pass), on the largest
+        # tensor of the set: 3 reads + the unpruned dL/dO + values + positions = 9.125 B per element
+        big = max(order, key=lambda i: dO[i].numel())
+        lb = layers[big]
+        skip = (torch.randn(dO[big].shape, device="cuda") * 0.5).to(torch.float16 if args.dtype == "fp16" else torch.bfloat16).view(torch.int16)
+        g_res = capture(lambda: sdgp.sdgp_residual_relu_backward_prune(
+            dO[big].view(-1, lb.Cout), skip.view(-1, lb.Cout), act[big].view(-1, lb.Cout), n, m, scheme, 1234, dtype=DT,
+            grad=grad[big].view(-1, lb.Cout), values=cv[big], meta=cm[big]))
+        ms_res = timed(g_res.replay, 50, 3) / 50
+        res_gbs = dO[big].numel() * 9.125 / (ms_res * 1e-3) / 1e9
+        relu_chain["residual_producer"] = {"layer": lb.name, "us": 1e3 * ms_res, "gbs": res_gbs, "frac_of_hbm": res_gbs / pk["hbm"],
+                                           "bytes_per_element": 9.125}
+        del act, grad, cv, cm, g_rs, g_rd, skip, g_res
 
     # ---- per-kernel timing: the same step captured with timing events between the kernels
     # (event-record graph nodes), replayed with the same data and cache state as the timed step ----

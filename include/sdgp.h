@@ -183,6 +183,18 @@ sdgp_status sdgp_relu_backward_prune(const void* dY, const void* act, int64_t ro
                                      sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad, void* dOp_dense,
                                      void* values, void* meta, void* mask, void* stream);
 
+/* The same producer below the ReLU that FOLLOWS A RESIDUAL ADDITION, y = ReLU(x + F(x)) (the ResNets of Section 4): two
+ * consumers of y hand down a data gradient each (Section 2.1, Fig. 2) - the next block's branch and its skip path - and the
+ * gradient that reaches the ReLU is their sum. One pass reads both gradients and the activation and forms
+ *     dL/dO[r, k] = round16(dY[r, k] + dSkip[r, k]) if act[r, k] > 0, else +0.0
+ * (one IEEE single-precision addition of the two 16-bit values, rounded to `dtype` to nearest-even; a NaN sum is stored as
+ * the canonical quiet NaN 0x7FC0 / 0x7E00), then applies Algorithm 1 to it. dSkip: [rows, K], element type `dtype`,
+ * 16-byte aligned, never written; everything else as sdgp_relu_backward_prune. A null dSkip is SDGP_ERR_INVALID_ARG
+ * (unless rows * K == 0). */
+sdgp_status sdgp_residual_relu_backward_prune(const void* dY, const void* dSkip, const void* act, int64_t rows, int64_t K,
+                                              int n, int m, sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad,
+                                              void* dOp_dense, void* values, void* meta, void* mask, void* stream);
+
 /* Data gradient of a GROUPED convolution (the 3x3 convolutions of RegNetX, one of the networks of Section 4; the
  * contraction is Section 2.1 / Fig. 2 and Section 3.1 / Fig. 3 with the sum over output channels restricted to the
  * group of the input channel): output channel co belongs to group co / (Cout/groups) and is connected to the

@@ -19,7 +19,7 @@ FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE, FLAG_MASKED, FLAG_CHANNEL = 0, 1, 2, 3, 4
 BF16, FP16 = 0, 1   # sdgp_dtype
 EXPORTS = ["sdgp_prune", "sdgp_dgrad_linear", "sdgp_dgrad_conv2d", "sdgp_spmm_linear", "sdgp_spmm_conv2d",
            "sdgp_prune_typed", "sdgp_dgrad_linear_typed", "sdgp_dgrad_conv2d_typed", "sdgp_spmm_linear_typed",
-           "sdgp_spmm_conv2d_typed", "sdgp_channel_scales", "sdgp_relu_backward_prune", "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
+           "sdgp_spmm_conv2d_typed", "sdgp_channel_scales", "sdgp_relu_backward_prune", "sdgp_residual_relu_backward_prune", "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
            "sdgp_workspace_size_linear", "sdgp_workspace_size_conv2d", "sdgp_workspace_size_conv2d_grouped",
            "sdgp_dgrad_conv2d_grouped", "sdgp_last_device_error",
            "sdgp_status_string"]
@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.sdgp_channel_scales.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp]
         L.sdgp_relu_backward_prune.argtypes = [vp, vp, i64, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
         L.sdgp_relu_backward_prune.restype = i32
+        L.sdgp_residual_relu_backward_prune.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
+        L.sdgp_residual_relu_backward_prune.restype = i32
         L.sdgp_channel_scales.restype = i32
         L.sdgp_workspace_size_linear.argtypes = [i64, i64, i64, u32]
         L.sdgp_workspace_size_linear.restype = sz
@@ -209,6 +211,22 @@ def sdgp_relu_backward_prune(dY, act, n, m, scheme, seed=0, dtype=BF16, grad=Non
     rows = dY.numel() // K if K else 0
     _check(lib().sdgp_relu_backward_prune(_ptr(dY), _ptr(act), rows, K, n, m, scheme, seed, dtype, _ptr(grad), _ptr(dense),
                                           _ptr(values), _ptr(meta), _ptr(mask), _stream()), "sdgp_relu_backward_prune")
+
+
+def sdgp_residual_relu_backward_prune(dY, dSkip, act, n, m, scheme, seed=0, dtype=BF16, grad=None, dense=None, values=None,
+                                      meta=None, mask=None):
+    """``sdgp_residual_relu_backward_prune``: dL/dO = dY + dSkip (rounded to the 16-bit type) where ``act`` > 0, pruned in
+    the same pass. The three inputs are 2-byte-element tensors of the same shape whose last dimension is K."""
+    for t, name in ((dY, "dY"), (dSkip, "dSkip"), (act, "act"), (grad, "grad"), (dense, "dense"), (values, "values"),
+                    (meta, "meta"), (mask, "mask")):
+        _dev(t, name)
+    if dY.shape != act.shape or (dSkip is not None and dY.shape != dSkip.shape):   # (a missing dSkip is the library's to reject)
+        raise ValueError("dY, dSkip and act must have the same shape")
+    K = dY.shape[-1] if dY.dim() else 0
+    rows = dY.numel() // K if K else 0
+    _check(lib().sdgp_residual_relu_backward_prune(_ptr(dY), _ptr(dSkip), _ptr(act), rows, K, n, m, scheme, seed, dtype,
+                                                   _ptr(grad), _ptr(dense), _ptr(values), _ptr(meta), _ptr(mask), _stream()),
+           "sdgp_residual_relu_backward_prune")
 
 
 def sdgp_dgrad_linear_typed(dO, W, dD, n, m, scheme, seed, dtype, workspace=None, flags=FLAG_TWO_PASS):

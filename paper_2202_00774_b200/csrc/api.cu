@@ -79,9 +79,9 @@ sdgp_status sdgp_prune_typed(const void* dO, int64_t rows, int64_t K, int n, int
   return e == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 
-sdgp_status sdgp_relu_backward_prune(const void* dY, const void* act, int64_t rows, int64_t K, int n, int m,
-                                     sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad, void* dOp_dense,
-                                     void* values, void* meta, void* mask, void* stream) {
+static sdgp_status relu_backward_prune(const void* dY, const void* dSkip, const void* act, int64_t rows, int64_t K, int n,
+                                       int m, sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad,
+                                       void* dOp_dense, void* values, void* meta, void* mask, void* stream) {
   if (!valid_dtype(dtype)) return SDGP_ERR_INVALID_ARG;
   sdgp_status st = check_prune_args(rows, K, n, m, (int)scheme);
   if (st != SDGP_OK) return st;
@@ -93,9 +93,23 @@ sdgp_status sdgp_relu_backward_prune(const void* dY, const void* act, int64_t ro
   if (!aligned16(dY) || !aligned16(act) || !aligned16(grad) || !aligned16(dOp_dense) || !aligned16(values) ||
       !aligned16(meta) || !aligned16(mask))
     return SDGP_ERR_ALIGNMENT;
+  if (!aligned16(dSkip)) return SDGP_ERR_ALIGNMENT;
   cudaError_t e = sdgp::launch_relu_backward_prune(dY, act, rows, K, n, m, (int)scheme, seed, grad, dOp_dense, values, meta,
-                                                   mask, (cudaStream_t)stream, (int)dtype);
+                                                   mask, (cudaStream_t)stream, (int)dtype, dSkip);
   return e == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
+}
+
+sdgp_status sdgp_relu_backward_prune(const void* dY, const void* act, int64_t rows, int64_t K, int n, int m,
+                                     sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad, void* dOp_dense,
+                                     void* values, void* meta, void* mask, void* stream) {
+  return relu_backward_prune(dY, nullptr, act, rows, K, n, m, scheme, seed, dtype, grad, dOp_dense, values, meta, mask, stream);
+}
+
+sdgp_status sdgp_residual_relu_backward_prune(const void* dY, const void* dSkip, const void* act, int64_t rows, int64_t K,
+                                              int n, int m, sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad,
+                                              void* dOp_dense, void* values, void* meta, void* mask, void* stream) {
+  if (!dSkip && rows != 0 && K != 0) return SDGP_ERR_INVALID_ARG;
+  return relu_backward_prune(dY, dSkip, act, rows, K, n, m, scheme, seed, dtype, grad, dOp_dense, values, meta, mask, stream);
 }
 
 // SDGP_FLAG_CHANNEL: behind the compressed tensor, 3 * K floats (factors, two column sums) and the scaled copy of W

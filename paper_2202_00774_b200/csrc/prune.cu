@@ -49,7 +49,18 @@ struct ReluSource {
   const uint4* act;   // the ReLU's activation, same shape as the gradient; nullptr: no ReLU, the input is dL/dO itself
   uint4* grad;        // optional: the unpruned dL/dO (kept for the weight gradient, Section 3.1)
   uint32_t nan_add;
+  const uint4* skip;  // optional: the second gradient that reaches the ReLU where a residual connection joins its
+                      // branch; the two are added before the gate
+  int f16;            // element type of the sum (only read when skip is set)
 };
+
+// Two 16-bit elements of each gradient, added in fp32 (one rounding) and rounded to the 16-bit type to nearest-even;
+// a NaN sum becomes the canonical quiet NaN.
+template <bool F16>
+__device__ __forceinline__ uint32_t add_pair(uint32_t g, uint32_t s) {
+  const float lo = __fadd_rn(lane_lo<F16>(g), lane_lo<F16>(s)), hi = __fadd_rn(lane_hi<F16>(g), lane_hi<F16>(s));
+  return f32_to_elem_bits<F16>(lo) | (f32_to_elem_bits<F16>(hi) << 16);
+}
 
 __device__ __forceinline__ uint32_t relu_pass2(uint32_t g, uint32_t a, uint32_t nan_add) {
   const uint32_t mag = a & 0x7FFF7FFFu;
@@ -63,6 +74,12 @@ __device__ __forceinline__ uint4 load_gradient(const uint4* __restrict__ dO, int
   uint4 g = __ldg(dO + v);
   if (RELU) {
     const uint4 a = __ldg(src.act + v);
+    if (src.skip) {
+      const uint4 k = __ldg(src.skip + v);
+      g = src.f16 ? make_uint4(add_pair<true>(g.x, k.x), add_pair<true>(g.y, k.y), add_pair<true>(g.z, k.z), add_pair<true>(g.w, k.w))
+                  : make_uint4(add_pair<false>(g.x, k.x), add_pair<false>(g.y, k.y), add_pair<false>(g.z, k.z),
+                               add_pair<false>(g.w, k.w));
+    }
     g = make_uint4(relu_pass2(g.x, a.x, src.nan_add), relu_pass2(g.y, a.y, src.nan_add), relu_pass2(g.z, a.z, src.nan_add),
                    relu_pass2(g.w, a.w, src.nan_add));
     if (src.grad) src.grad[v] = g;
@@ -469,13 +486,14 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
                          uint64_t seed, void* dense, void* values, void* meta, void* mask,
                          cudaStream_t stream, int64_t k_pad, int dtype) {
   return launch_prune_src<false>(dO, rows, K, n, m, scheme, seed, dense, values, meta, mask, stream, k_pad, dtype,
-                                 ReluSource{nullptr, nullptr, 0u});
+                                 ReluSource{nullptr, nullptr, 0u, nullptr, 0});
 }
 
 cudaError_t launch_relu_backward_prune(const void* dY, const void* act, int64_t rows, int64_t K, int n, int m, int scheme,
                                        uint64_t seed, void* grad, void* dense, void* values, void* meta, void* mask,
-                                       cudaStream_t stream, int dtype) {
-  const ReluSource src = {(const uint4*)act, (uint4*)grad, dtype == SDGP_FP16 ? 0x03FF03FFu : 0x007F007Fu};
+                                       cudaStream_t stream, int dtype, const void* skip) {
+  const ReluSource src = {(const uint4*)act, (uint4*)grad, dtype == SDGP_FP16 ? 0x03FF03FFu : 0x007F007Fu,
+                          (const uint4*)skip, dtype == SDGP_FP16 ? 1 : 0};
   return launch_prune_src<true>(dY, rows, K, n, m, scheme, seed, dense, values, meta, mask, stream, 0, dtype, src);
 }
 

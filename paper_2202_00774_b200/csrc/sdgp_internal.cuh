@@ -16,10 +16,11 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
 
 // The producer of dL/dO below a ReLU fused with its pruning: the gradient above the ReLU (dY) passes where the
 // activation `act` is positive; `grad` (optional) receives that unpruned dL/dO, the other outputs are
-// launch_prune's. n <= 2, or n == m (nothing pruned: only `grad` and the mask make sense then).
+// launch_prune's. n <= 2, or n == m (nothing pruned: only `grad` and the mask make sense then). skip (optional): a second
+// gradient of the same shape, added to dY (fp32 sum, rounded to the 16-bit type) before the gate.
 cudaError_t launch_relu_backward_prune(const void* dY, const void* act, int64_t rows, int64_t K, int n, int m, int scheme,
                                        uint64_t seed, void* grad, void* dense, void* values, void* meta, void* mask,
-                                       cudaStream_t stream, int dtype = SDGP_BF16);
+                                       cudaStream_t stream, int dtype = SDGP_BF16, const void* skip = nullptr);
 
 // Per-channel reading of the L1 rescale (channel.cu). sums: 2 * K floats (cleared by the call): the
 // column sums of |x| over all rows, then the same over the survivors of the magnitude function.

@@ -60,6 +60,20 @@ def test_prune_rejects_bad_arguments_before_launch(lib):
     assert P(None, 0, 64, 2, 4, 1, 0, None, None, None, None, None) == 0   # empty tensor: no-op
 
 
+def test_producers_reject_bad_arguments_before_launch(lib):
+    i64, i32, u64, vp = ctypes.c_int64, ctypes.c_int, ctypes.c_uint64, ctypes.c_void_p
+    Pr, Rs = lib.sdgp_relu_backward_prune, lib.sdgp_residual_relu_backward_prune
+    Pr.argtypes = [vp, vp, i64, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
+    Rs.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
+    assert Pr(FAKE, None, 4, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 1       # no activation
+    assert Rs(FAKE, None, FAKE, 4, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 1  # no second gradient
+    assert Rs(FAKE, FAKE, None, 4, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 1
+    assert Rs(FAKE, ctypes.c_void_p(0x1002), FAKE, 4, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 3
+    assert Rs(FAKE, FAKE, FAKE, 4, 64, 4, 8, 1, 0, 0, None, None, FAKE, FAKE, None, None) == 2   # 4:8 has no compressed form
+    assert Rs(FAKE, FAKE, FAKE, 4, 64, 2, 4, 1, 0, 9, FAKE, None, None, None, None, None) == 1   # unknown element type
+    assert Rs(None, None, None, 0, 64, 2, 4, 1, 0, 0, None, None, None, None, None, None) == 0   # empty tensor: no-op
+
+
 def test_dgrad_rejects_bad_arguments_before_launch(lib):
     L, C = lib.sdgp_dgrad_linear, lib.sdgp_dgrad_conv2d
     ws = ctypes.c_void_p(0x10000)

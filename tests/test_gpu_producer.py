@@ -101,3 +101,87 @@ def test_producer_rejects_bad_arguments():
     with pytest.raises(sdgp.SdgpError) as e:
         sdgp.sdgp_relu_backward_prune(x, x, 0, 4, sdgp.MAGNITUDE, grad=x)
     assert e.value.status == 1
+
+
+# ---- the producer below the ReLU that follows a residual addition: two gradients are added before the gate ----
+
+
+def make_skip(rows, K, seed, dtype=oracle.BF16):
+    """A second gradient with the cases of the addition that matter: a different scale (operands that half-vanish), exact
+    negatives of dY (cancellation to +0.0), zeros of both signs, infinities of both signs and NaNs."""
+    rng = np.random.default_rng(seed + 1000)
+    to_bits = inputs.f32_to_bf16_bits if dtype == oracle.BF16 else (lambda x: x.astype(np.float16).view(np.uint16))
+    scale = np.exp2(rng.integers(-12, 4, size=(rows, K))).astype(np.float32)
+    dSkip = to_bits((rng.laplace(size=(rows, K)) * scale).astype(np.float32))
+    return dSkip
+
+
+@pytest.mark.parametrize("n,m,scheme", [(2, 4, oracle.MAGNITUDE), (2, 4, oracle.RESCALED), (1, 4, oracle.RANDOM),
+                                        (2, 8, oracle.MAGNITUDE), (2, 16, oracle.RESCALED), (2, 32, oracle.RANDOM)])
+@pytest.mark.parametrize("dtype", [oracle.BF16, oracle.FP16])
+def test_residual_producer_outputs_bit_exact(n, m, scheme, dtype):
+    import paper_2202_00774_b200 as sdgp
+    rows, K = 1237, 160
+    dY, act = make(rows, K, seed=n * 10 + m, dtype=dtype)
+    dSkip = make_skip(rows, K, seed=n * 10 + m, dtype=dtype)
+    inf, nan = (0x7F80, 0x7FC1) if dtype == oracle.BF16 else (0x7C00, 0x7E01)
+    fy, fs = dY.reshape(-1), dSkip.reshape(-1)
+    fs[0:4000:7] = fy[0:4000:7] ^ 0x8000                      # x + (-x)
+    fy[1:3000:11], fs[1:3000:11] = 0x8000, 0x0000             # -0 + +0
+    fy[2:3000:13], fs[2:3000:13] = 0x8000, 0x8000             # -0 + -0 (stays -0.0 where the ReLU passes it)
+    fy[3:3000:17], fs[3:3000:17] = inf, inf | 0x8000          # inf - inf: the canonical NaN
+    fy[4:3000:19] = nan                                       # a NaN with a payload: canonical after the addition
+    fy[5:3000:23], fs[5:3000:23] = inf - 1, inf - 1           # the largest finite number twice: overflow to infinity
+    dt = sdgp.BF16 if dtype == oracle.BF16 else sdgp.FP16
+    grad = torch.full((rows, K), -1, dtype=torch.int16, device="cuda")
+    dense = torch.full((rows, K), -1, dtype=torch.int16, device="cuda")
+    values = torch.full((rows, K // 2), -1, dtype=torch.int16, device="cuda")
+    meta = torch.full((rows, K // 16), -1, dtype=torch.int16, device="cuda")
+    mask = torch.full((rows, K // 32), -1, dtype=torch.int32, device="cuda")
+    d_dY, d_skip, d_act = dev16(dY), dev16(dSkip), dev16(act)
+    sdgp.sdgp_residual_relu_backward_prune(d_dY, d_skip, d_act, n, m, scheme, seed=77, dtype=dt, grad=grad, dense=dense,
+                                           values=values, meta=meta, mask=mask)
+    ref = oracle.residual_relu_backward_prune(dY, dSkip, act, n, m, scheme, seed=77, dtype=dtype)
+    assert np.array_equal(host16(grad), ref["grad"])
+    assert np.array_equal(host16(dense), ref["dense"])
+    assert np.array_equal(host16(values), ref["values"])
+    assert np.array_equal(host16(meta), ref["meta"])
+    assert np.array_equal(mask.cpu().numpy().view(np.uint32), ref["mask"])
+    # the inputs are never written
+    assert np.array_equal(host16(d_dY), dY) and np.array_equal(host16(d_skip), dSkip) and np.array_equal(host16(d_act), act)
+
+
+def test_residual_producer_plain_sum_and_the_sparse_contraction():
+    import paper_2202_00774_b200 as sdgp
+    B, HW, Cin, Cout = 4, 14, 128, 512
+    rows = B * HW * HW
+    dY, act = make(rows, Cout, seed=21)
+    dSkip = make_skip(rows, Cout, seed=21)
+    # n == m: the gated sum alone (what the weight gradient reads)
+    grad = torch.full((rows, Cout), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_residual_relu_backward_prune(dev16(dY), dev16(dSkip), dev16(act), 4, 4, sdgp.MAGNITUDE, grad=grad)
+    assert np.array_equal(host16(grad), oracle.residual_relu_backward(dY, dSkip, act))
+    # compressed outputs straight into the contraction
+    W = inputs.f32_to_bf16_bits((np.random.default_rng(2).standard_normal((Cout, Cin)) * (2.0 / Cin) ** 0.5).astype(np.float32))
+    values = torch.empty((rows, Cout // 2), dtype=torch.int16, device="cuda")
+    meta = torch.empty((rows, Cout // 16), dtype=torch.int16, device="cuda")
+    dD = torch.full((B, HW, HW, Cin), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_residual_relu_backward_prune(dev16(dY), dev16(dSkip), dev16(act), 2, 4, sdgp.MAGNITUDE, values=values, meta=meta)
+    sdgp.sdgp_spmm_conv2d(values.view(B, HW, HW, Cout // 2), meta.view(B, HW, HW, Cout // 16), dev16(W).view(Cout, 1, 1, Cin), dD, 1, 0)
+    assert sdgp.sdgp_last_device_error() == 0
+    ref = oracle.residual_relu_backward_prune(dY, dSkip, act, 2, 4, oracle.MAGNITUDE, want=("dense",))
+    want = oracle.dgrad_linear(ref["dense"], W)
+    got = inputs.bf16_bits_to_f32(host16(dD)).astype(np.float64).reshape(rows, Cin)
+    assert np.linalg.norm(got - want) <= TOL * np.linalg.norm(want)
+
+
+def test_residual_producer_rejects_bad_arguments():
+    import paper_2202_00774_b200 as sdgp
+    x = torch.zeros((8, 64), dtype=torch.int16, device="cuda")
+    with pytest.raises(sdgp.SdgpError) as e:
+        sdgp.sdgp_residual_relu_backward_prune(x, None, x, 2, 4, sdgp.MAGNITUDE, grad=x)
+    assert e.value.status == 1
+    with pytest.raises(sdgp.SdgpError) as e:
+        odd = torch.zeros(8 * 64 + 8, dtype=torch.int16, device="cuda")[1:1 + 8 * 64].view(8, 64)   # 2 bytes off a 16-byte boundary
+        sdgp.sdgp_residual_relu_backward_prune(x, odd, x, 2, 4, sdgp.MAGNITUDE, grad=torch.zeros_like(x))
+    assert e.value.status == 3
