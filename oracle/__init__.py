@@ -63,6 +63,8 @@ def _load():
             lib.oracle_relu_backward.restype = i32
             lib.oracle_residual_relu_backward.argtypes = [vp, vp, vp, i64, i32, vp]
             lib.oracle_residual_relu_backward.restype = i32
+            lib.oracle_maxpool_relu_backward.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp]
+            lib.oracle_maxpool_relu_backward.restype = i32
             lib.oracle_expand.argtypes = [vp, vp, i64, i64, vp]
             lib.oracle_expand.restype = i32
             lib.oracle_dgrad_linear.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64]
@@ -161,6 +163,30 @@ def residual_relu_backward_prune(dY, dSkip, act, n, m, scheme, seed=0, want=("de
     """``residual_relu_backward`` followed by Algorithm 1; ``"grad"`` is the unpruned dL/dO (Section 3.1)."""
     grad = residual_relu_backward(dY, dSkip, act, dtype)
     out = prune(grad, n, m, scheme, seed, want, dtype)
+    out["grad"] = grad
+    return out
+
+
+def maxpool_relu_backward(dYp, act, dtype=BF16):
+    """dL/dO below a ReLU that is followed by a 2 x 2 max pooling of stride 2 (ResNet-9's blocks, Section 4): ``dYp``
+    [B, H/2, W/2, K] is the gradient above the pooling, ``act`` [B, H, W, K] the ReLU's activation; each pooled
+    gradient goes to the first largest activation of its window if that is positive. Returns [B, H, W, K]."""
+    dYp, act = _u16(dYp), _u16(act)
+    B, H, W, K = act.shape
+    if dYp.shape != (B, H // 2, W // 2, K) or H % 2 or W % 2:
+        raise ValueError("dYp must be [B, H/2, W/2, K] for act [B, H, W, K] with even H and W")
+    out = np.empty(act.shape, np.uint16)
+    rc = _load().oracle_maxpool_relu_backward(_ptr(dYp), _ptr(act), B, H, W, K, dtype, _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_maxpool_relu_backward rejected its arguments")
+    return out
+
+
+def maxpool_relu_backward_prune(dYp, act, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask"), dtype=BF16):
+    """``maxpool_relu_backward`` followed by Algorithm 1 along K; outputs as [B*H*W, ...]; ``"grad"`` is the unpruned
+    dL/dO [B, H, W, K] (Section 3.1)."""
+    grad = maxpool_relu_backward(dYp, act, dtype)
+    out = prune(grad.reshape(-1, grad.shape[-1]), n, m, scheme, seed, want, dtype)
     out["grad"] = grad
     return out
 

@@ -561,6 +561,44 @@ int oracle_residual_relu_backward(const uint16_t* dY, const uint16_t* dSkip, con
   return ORACLE_OK;
 }
 
+/* Where the ReLU is followed by a 2 x 2 max pooling of stride 2 (the convolution blocks of ResNet-9, Section 4:
+ * convolution, normalisation, ReLU, pooling), the gradient handed down (Section 2.1 / Fig. 2) has the POOLED shape
+ * [B, H/2, W/2, K]. Pooling backward sends each of its elements to the position of its window's maximum, the first
+ * one in the order (0,0), (0,1), (1,0), (1,1) when several are equal, and the ReLU below passes it only where its
+ * activation is positive. Both rules together: in every window and channel the gradient goes to the first largest
+ * activation if that activation is a number greater than zero; every other position of dL/dO, and the whole window
+ * if nothing in it is positive, is +0.0. `act` is the ReLU's output or input, [B, H, W, K]; H and W are even. The
+ * survivor keeps the exact bits of the pooled gradient. */
+int oracle_maxpool_relu_backward(const uint16_t* dYp, const uint16_t* act, int B, int H, int W, int K, int dtype,
+                                 uint16_t* dO) {
+  if (!dYp || !act || !dO || B < 0 || H < 0 || W < 0 || K < 0 || (H & 1) || (W & 1) ||
+      (dtype != ORACLE_BF16 && dtype != ORACLE_FP16))
+    return ORACLE_ERR_ARG;
+  const int Hp = H / 2, Wp = W / 2;
+  for (int b = 0; b < B; ++b)
+    for (int i = 0; i < Hp; ++i)
+      for (int j = 0; j < Wp; ++j)
+        for (int k = 0; k < K; ++k) {
+          int best = -1;
+          float best_a = 0.0f;
+          for (int pos = 0; pos < 4; ++pos) {
+            const int h = 2 * i + (pos >> 1), w = 2 * j + (pos & 1);
+            const int64_t e = (((int64_t)b * H + h) * W + w) * K + k;
+            const float a = elem_to_f32(act[e], dtype);
+            dO[e] = 0;
+            if (a > 0.0f && (best < 0 || a > best_a)) { /* a NaN compares false: it is never the maximum */
+              best = pos;
+              best_a = a;
+            }
+          }
+          if (best >= 0) {
+            const int h = 2 * i + (best >> 1), w = 2 * j + (best & 1);
+            dO[(((int64_t)b * H + h) * W + w) * K + k] = dYp[(((int64_t)b * Hp + i) * Wp + j) * K + k];
+          }
+        }
+  return ORACLE_OK;
+}
+
 /* Section 4.3 estimator: removing a fraction (1 - n/m) of a pass that takes
  * share f of the runtime reduces the total by f * (1 - n/m). */
 double oracle_runtime_reduction(double share, int n, int m) {

@@ -1,6 +1,7 @@
 """Pins of the oracle's producer of dL/dO (ReLU backward, then Algorithm 1): Section 2.1 / Fig. 2 (dL/dO is what the
 layer above hands down), Section 3.1 (the unpruned tensor is kept), Section 3.3 (ReLU zeros)."""
 import numpy as np
+import pytest
 
 import oracle
 from paper_2202_00774_b200 import inputs
@@ -145,3 +146,83 @@ def test_residual_producer_is_the_sum_followed_by_algorithm_1():
     f = inputs.bf16_bits_to_f32
     kept = f(out["dense"]) != 0
     assert np.all(f(out["dense"])[kept] == f(out["grad"])[kept]) and kept.reshape(48, 16, 4).sum(-1).max() <= 2
+
+
+# ---- the producer below a ReLU that is followed by 2 x 2 max pooling (the pooled gradient goes to the window's maximum) ----
+
+
+def test_maxpool_hand_example():
+    # one image of 2 x 4 pixels (two windows), one channel per column of the tables below, K = 4
+    f = lambda rows: bits(np.array(rows, np.float32))
+    #                 channel: 0 (plain max)  1 (tie: first wins)  2 (nothing positive)  3 (max at the last position)
+    act = np.stack([f([[1.0, 2.0, -1.0, 0.5], [3.0, 2.0, 0.0, 0.25]]),        # pixel row 0: window 0 = columns 0, 1
+                    f([[2.0, 1.0, -2.0, 0.5], [0.5, 2.0, -0.0, 4.0]])])       # pixel row 1
+    act = np.concatenate([act, act[:, ::-1]], axis=1)[None]                   # second window: the first one mirrored left-right
+    g = bits(np.array([[[[10.0, 20.0, 30.0, 40.0], [50.0, 60.0, 70.0, 80.0]]]], np.float32))
+    got = inputs.bf16_bits_to_f32(oracle.maxpool_relu_backward(g, act))
+    want = np.zeros((1, 2, 4, 4), np.float32)
+    want[0, 0, 1, 0] = 10.0      # 3.0 at (0, 1)
+    want[0, 0, 0, 1] = 20.0      # 2.0 three times: (0, 0) comes first
+    want[0, 1, 1, 3] = 40.0      # 4.0 at (1, 1)
+    want[0, 0, 2, 0] = 50.0      # mirrored window: 3.0 now at (0, 0) -> pixel column 2
+    want[0, 0, 2, 1] = 60.0      # mirrored tie: the first of the three 2.0 is at (0, 0) again
+    want[0, 1, 2, 3] = 80.0      # 4.0 now at (1, 0)
+    assert np.array_equal(got, want)
+
+
+def test_maxpool_equals_the_librarys_pooling_and_relu_backward():
+    import torch
+    rng = np.random.default_rng(21)
+    B, H, W, K = 3, 8, 12, 16
+    # coarse values, so that equal activations inside a window are common
+    pre = bits(np.round(rng.standard_normal((B, H, W, K)) * 2.0) / 2.0)
+    g = bits(rng.laplace(size=(B, H // 2, W // 2, K)))
+    x = torch.from_numpy(inputs.bf16_bits_to_f32(pre)).double().permute(0, 3, 1, 2).contiguous().requires_grad_(True)
+    y = torch.nn.functional.max_pool2d(torch.relu(x), 2)
+    y.backward(torch.from_numpy(inputs.bf16_bits_to_f32(g)).double().permute(0, 3, 1, 2).contiguous())
+    want = x.grad.permute(0, 2, 3, 1).numpy()
+    for act in (pre, bits(np.maximum(inputs.bf16_bits_to_f32(pre), 0.0))):       # the ReLU's input, or its output
+        got = oracle.maxpool_relu_backward(g, act)
+        assert np.array_equal(inputs.bf16_bits_to_f32(got).astype(np.float64), want)
+    ties = (inputs.bf16_bits_to_f32(pre).reshape(B, H // 2, 2, W // 2, 2, K).transpose(0, 1, 3, 5, 2, 4).reshape(-1, 4))
+    assert np.any((ties == ties.max(1, keepdims=True)).sum(1) > 1)              # the draw does hold ties
+
+
+def test_maxpool_invariants_bits_and_special_activations():
+    rng = np.random.default_rng(22)
+    B, H, W, K = 2, 6, 4, 32
+    act = bits(rng.standard_normal((B, H, W, K)))
+    flat = act.reshape(-1)
+    flat[rng.integers(0, flat.size, 300)] = np.resize(np.array([0x7FC0, 0x7F80, 0x8000, 0x0001, 0xFF80], np.uint16), 300)
+    g = np.arange(1, 1 + B * (H // 2) * (W // 2) * K, dtype=np.uint16).reshape(B, H // 2, W // 2, K) * 37     # every kind of pattern
+    got = oracle.maxpool_relu_backward(g, act)
+    win = got.reshape(B, H // 2, 2, W // 2, 2, K).transpose(0, 1, 3, 5, 2, 4).reshape(B, H // 2, W // 2, K, 4)
+    awin = inputs.bf16_bits_to_f32(act).reshape(B, H // 2, 2, W // 2, 2, K).transpose(0, 1, 3, 5, 2, 4).reshape(B, H // 2, W // 2, K, 4)
+    with np.errstate(invalid="ignore"):
+        positive = awin > 0                                                     # NaN: False
+    assert np.all((win != 0).sum(-1) <= 1)
+    has = positive.any(-1)
+    assert np.array_equal(win.sum(-1, dtype=np.uint32)[has], g[has].astype(np.uint32))     # the survivor is g, bit for bit
+    assert not win[~has].any()
+    # the survivor sits on a positive activation that no other positive activation of the window exceeds
+    sel = win != 0
+    cand = np.where(positive, awin, -np.inf)
+    assert np.all(cand[sel] == cand.max(-1)[sel.any(-1)])
+    # an infinite activation wins its window; a NaN never does
+    a = np.full((1, 2, 2, 8), 0x3F80, np.uint16)
+    a[0, 1, 0, :] = 0x7F80
+    a[0, 0, 0, :] = 0x7FC0
+    out = oracle.maxpool_relu_backward(np.full((1, 1, 1, 8), 0x4000, np.uint16), a)
+    assert np.all(out[0, 1, 0] == 0x4000) and not out[0, 0].any() and not out[0, 1, 1].any()
+
+
+def test_maxpool_producer_is_the_scatter_followed_by_algorithm_1():
+    rng = np.random.default_rng(23)
+    act = bits(rng.standard_normal((2, 4, 4, 64)))
+    g = bits(rng.laplace(size=(2, 2, 2, 64)))
+    out = oracle.maxpool_relu_backward_prune(g, act, 2, 8, oracle.MAGNITUDE)
+    ref = oracle.prune(out["grad"].reshape(-1, 64), 2, 8, oracle.MAGNITUDE)
+    for key in ("dense", "values", "meta", "mask"):
+        assert np.array_equal(out[key], ref[key])
+    with pytest.raises(ValueError):
+        oracle.maxpool_relu_backward(g, act[:, :3])                              # odd height
