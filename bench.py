@@ -436,7 +436,18 @@ def run_ours(args, layers):
         res_gbs = dO[big].numel() * 9.125 / (ms_res * 1e-3) / 1e9
         relu_chain["residual_producer"] = {"layer": lb.name, "us": 1e3 * ms_res, "gbs": res_gbs, "frac_of_hbm": res_gbs / pk["hbm"],
                                            "bytes_per_element": 9.125}
-        del act, grad, cv, cm, g_rs, g_rd, skip, g_res
+        # ... and below a ReLU that is followed by 2 x 2 max pooling (the pooled gradient is scattered to each window's
+        # maximum in the same pass): activation + a quarter-size gradient read, the unpruned dL/dO + values + positions
+        # written = 5.625 B per element
+        pooled = dO[big].view(lb.B, lb.P, lb.Q, lb.Cout)[:, : lb.P // 2, : lb.Q // 2].contiguous()
+        g_pool = capture(lambda: sdgp.sdgp_maxpool_relu_backward_prune(
+            pooled, act[big].view(lb.B, lb.P, lb.Q, lb.Cout), n, m, scheme, 1234, dtype=DT,
+            grad=grad[big].view(lb.B, lb.P, lb.Q, lb.Cout), values=cv[big], meta=cm[big]))
+        ms_pool = timed(g_pool.replay, 50, 3) / 50
+        pool_gbs = dO[big].numel() * 5.625 / (ms_pool * 1e-3) / 1e9
+        relu_chain["pool_producer"] = {"layer": lb.name, "us": 1e3 * ms_pool, "gbs": pool_gbs, "frac_of_hbm": pool_gbs / pk["hbm"],
+                                       "bytes_per_element": 5.625}
+        del act, grad, cv, cm, g_rs, g_rd, skip, g_res, pooled, g_pool
 
     # ---- per-kernel timing: the same step captured with timing events between the kernels
     # (event-record graph nodes), replayed with the same data and cache state as the timed step ----

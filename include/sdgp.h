@@ -195,6 +195,18 @@ sdgp_status sdgp_residual_relu_backward_prune(const void* dY, const void* dSkip,
                                               int n, int m, sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad,
                                               void* dOp_dense, void* values, void* meta, void* mask, void* stream);
 
+/* The same producer below a ReLU that is FOLLOWED BY A 2 x 2 MAX POOLING of stride 2 (the blocks of ResNet-9, Section 4:
+ * convolution, normalisation, ReLU, pooling): the gradient handed down (Section 2.1, Fig. 2) has the pooled shape
+ * dYp [B, H/2, Wd/2, K]; `act` [B, H, Wd, K] is the ReLU's activation (output or input), NHWC, element type `dtype`.
+ * One pass forms dL/dO [B, H, Wd, K]: in every window and channel the pooled gradient goes to the window's largest
+ * activation - the first one in the order (0,0), (0,1), (1,0), (1,1) if several are equal, as the usual pooling backward
+ * does - provided that activation is a number greater than zero; every other position is +0.0 (a NaN is never the
+ * maximum). Algorithm 1 then runs along K on that tensor viewed as [B*H*Wd, K]; grad, dOp_dense, values, meta, mask as
+ * sdgp_relu_backward_prune. H and Wd must be even (else SDGP_ERR_INVALID_ARG); B*H*Wd*K / 32 must be below 2^31. */
+sdgp_status sdgp_maxpool_relu_backward_prune(const void* dYp, const void* act, int B, int H, int Wd, int64_t K, int n, int m,
+                                             sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad, void* dOp_dense,
+                                             void* values, void* meta, void* mask, void* stream);
+
 /* Data gradient of a GROUPED convolution (the 3x3 convolutions of RegNetX, one of the networks of Section 4; the
  * contraction is Section 2.1 / Fig. 2 and Section 3.1 / Fig. 3 with the sum over output channels restricted to the
  * group of the input channel): output channel co belongs to group co / (Cout/groups) and is connected to the

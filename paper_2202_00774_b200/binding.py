@@ -19,7 +19,7 @@ FLAG_TWO_PASS, FLAG_FUSED, FLAG_DENSE, FLAG_MASKED, FLAG_CHANNEL = 0, 1, 2, 3, 4
 BF16, FP16 = 0, 1   # sdgp_dtype
 EXPORTS = ["sdgp_prune", "sdgp_dgrad_linear", "sdgp_dgrad_conv2d", "sdgp_spmm_linear", "sdgp_spmm_conv2d",
            "sdgp_prune_typed", "sdgp_dgrad_linear_typed", "sdgp_dgrad_conv2d_typed", "sdgp_spmm_linear_typed",
-           "sdgp_spmm_conv2d_typed", "sdgp_channel_scales", "sdgp_relu_backward_prune", "sdgp_residual_relu_backward_prune", "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
+           "sdgp_spmm_conv2d_typed", "sdgp_channel_scales", "sdgp_relu_backward_prune", "sdgp_residual_relu_backward_prune", "sdgp_maxpool_relu_backward_prune", "sdgp_dgrad_linear_static", "sdgp_selftest_bounded_wait",
            "sdgp_workspace_size_linear", "sdgp_workspace_size_conv2d", "sdgp_workspace_size_conv2d_grouped",
            "sdgp_dgrad_conv2d_grouped", "sdgp_last_device_error",
            "sdgp_status_string"]
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.sdgp_relu_backward_prune.restype = i32
         L.sdgp_residual_relu_backward_prune.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
         L.sdgp_residual_relu_backward_prune.restype = i32
+        L.sdgp_maxpool_relu_backward_prune.argtypes = [vp, vp, i32, i32, i32, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
+        L.sdgp_maxpool_relu_backward_prune.restype = i32
         L.sdgp_channel_scales.restype = i32
         L.sdgp_workspace_size_linear.argtypes = [i64, i64, i64, u32]
         L.sdgp_workspace_size_linear.restype = sz
@@ -227,6 +229,23 @@ def sdgp_residual_relu_backward_prune(dY, dSkip, act, n, m, scheme, seed=0, dtyp
     _check(lib().sdgp_residual_relu_backward_prune(_ptr(dY), _ptr(dSkip), _ptr(act), rows, K, n, m, scheme, seed, dtype,
                                                    _ptr(grad), _ptr(dense), _ptr(values), _ptr(meta), _ptr(mask), _stream()),
            "sdgp_residual_relu_backward_prune")
+
+
+def sdgp_maxpool_relu_backward_prune(dYp, act, n, m, scheme, seed=0, dtype=BF16, grad=None, dense=None, values=None, meta=None,
+                                     mask=None):
+    """``sdgp_maxpool_relu_backward_prune``: ``dYp`` [B, H/2, W/2, K] is the gradient above a 2 x 2 max pooling, ``act``
+    [B, H, W, K] the activation of the ReLU below it; dL/dO [B, H, W, K] is formed and pruned in one pass."""
+    for t, name in ((dYp, "dYp"), (act, "act"), (grad, "grad"), (dense, "dense"), (values, "values"), (meta, "meta"),
+                    (mask, "mask")):
+        _dev(t, name)
+    if act.dim() != 4 or dYp.dim() != 4:
+        raise ValueError("dYp and act must be NHWC tensors")
+    B, H, W, K = act.shape
+    if tuple(dYp.shape) != (B, H // 2, W // 2, K):
+        raise ValueError("dYp must be [B, H/2, W/2, K]")
+    _check(lib().sdgp_maxpool_relu_backward_prune(_ptr(dYp), _ptr(act), B, H, W, K, n, m, scheme, seed, dtype, _ptr(grad),
+                                                  _ptr(dense), _ptr(values), _ptr(meta), _ptr(mask), _stream()),
+           "sdgp_maxpool_relu_backward_prune")
 
 
 def sdgp_dgrad_linear_typed(dO, W, dD, n, m, scheme, seed, dtype, workspace=None, flags=FLAG_TWO_PASS):

@@ -52,6 +52,9 @@ struct ReluSource {
   const uint4* skip;  // optional: the second gradient that reaches the ReLU where a residual connection joins its
                       // branch; the two are added before the gate
   int f16;            // element type of the sum (only read when skip is set)
+  // 2 x 2 max pooling of stride 2 above the ReLU (pool_k8 != 0): the input gradient has the pooled shape
+  // [B, H/2, W/2, K] and `act` the full one [B, H, W, K]; pool_k8 = K / 8, pool_hp = H / 2, pool_wp = W / 2.
+  int pool_k8, pool_hp, pool_wp;
 };
 
 // Two 16-bit elements of each gradient, added in fp32 (one rounding) and rounded to the 16-bit type to nearest-even;
@@ -85,6 +88,76 @@ __device__ __forceinline__ uint4 load_gradient(const uint4* __restrict__ dO, int
     if (src.grad) src.grad[v] = g;
   }
   return g;
+}
+
+// Pooling backward for one 32-bit word (two channels) of a window: a[0..3] are the activation words at the window's
+// four positions in the order (0,0), (0,1), (1,0), (1,1), g the pooled gradient's word. Per channel the gradient goes
+// to the first largest activation if that is a number greater than zero (patterns of positive numbers order like the
+// numbers; composite = pattern * 4 + 3 - position is unique, so exactly one position wins or none does).
+__device__ __forceinline__ void pool_select2(const uint32_t (&a)[4], uint32_t g, uint32_t nan_add, uint32_t (&out)[4]) {
+  uint32_t lo[4], hi[4];
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    const uint32_t key = relu_pass2(a[t], a[t], nan_add);  // the pattern where it is a positive number, else 0
+    lo[t] = ((key & 0xFFFFu) << 2) | (uint32_t)(3 - t);
+    hi[t] = ((key >> 16) << 2) | (uint32_t)(3 - t);
+  }
+  const uint32_t mlo = max(max(lo[0], lo[1]), max(lo[2], lo[3])), mhi = max(max(hi[0], hi[1]), max(hi[2], hi[3]));
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    const uint32_t keep = ((lo[t] == mlo && mlo > 3u) ? 0x0000FFFFu : 0u) | ((hi[t] == mhi && mhi > 3u) ? 0xFFFF0000u : 0u);
+    out[t] = g & keep;
+  }
+}
+
+// The four vectors a thread prunes and their numbers in dL/dO (>= nvec: none). Without pooling they are the thread's
+// slots of four consecutive 256-vector stripes (every load of a warp is one contiguous 512 bytes). With pooling a
+// thread owns the four pixels of one window for one 8-channel vector: it reads the pooled gradient once and the four
+// activation vectors, and its lanes still hold neighbouring channel vectors of the same pixel.
+template <bool RELU>
+__device__ __forceinline__ void load_unit(const uint4* __restrict__ dO, int64_t nvec, const ReluSource& src,
+                                          int64_t (&vi)[kVecPerThread], uint4 (&in)[kVecPerThread]) {
+  if (RELU && src.pool_k8 != 0) {
+    const int64_t u = (int64_t)blockIdx.x * kThreads + threadIdx.x;  // number of the pooled gradient's vector
+    const bool live = u < (nvec >> 2);
+    int64_t pix00 = 0;
+    int cv = 0;
+    if (live) {  // (the host checked that the number of pooled vectors fits 32 bits)
+      const uint32_t window = (uint32_t)u / (uint32_t)src.pool_k8;
+      cv = (int)((uint32_t)u - window * (uint32_t)src.pool_k8);
+      const uint32_t t = window / (uint32_t)src.pool_wp;
+      const uint32_t j = window - t * (uint32_t)src.pool_wp;
+      const uint32_t b = t / (uint32_t)src.pool_hp;
+      const uint32_t i = t - b * (uint32_t)src.pool_hp;
+      pix00 = (((int64_t)b * src.pool_hp * 2 + 2 * i) * src.pool_wp + j) * 2;  // pixel (2i, 2j) of image b
+    }
+    uint4 a[4];
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      vi[it] = live ? (pix00 + (it >> 1) * (2 * src.pool_wp) + (it & 1)) * src.pool_k8 + cv : nvec;
+      a[it] = live ? __ldg(src.act + vi[it]) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    const uint4 g = live ? __ldg(dO + u) : make_uint4(0u, 0u, 0u, 0u);
+    uint32_t ox[4], oy[4], oz[4], ow[4];
+    const uint32_t ax[4] = {a[0].x, a[1].x, a[2].x, a[3].x}, ay[4] = {a[0].y, a[1].y, a[2].y, a[3].y},
+                   az[4] = {a[0].z, a[1].z, a[2].z, a[3].z}, aw[4] = {a[0].w, a[1].w, a[2].w, a[3].w};
+    pool_select2(ax, g.x, src.nan_add, ox);
+    pool_select2(ay, g.y, src.nan_add, oy);
+    pool_select2(az, g.z, src.nan_add, oz);
+    pool_select2(aw, g.w, src.nan_add, ow);
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      in[it] = make_uint4(ox[it], oy[it], oz[it], ow[it]);
+      if (live && src.grad) src.grad[vi[it]] = in[it];
+    }
+    return;
+  }
+  const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
+#pragma unroll
+  for (int it = 0; it < kVecPerThread; ++it) {
+    vi[it] = base + (int64_t)it * kThreads;
+    in[it] = (vi[it] < nvec) ? load_gradient<RELU>(dO, vi[it], src) : make_uint4(0, 0, 0, 0);
+  }
 }
 
 // M: group size; LANES = lanes that share a group (1, 2 or 4).
@@ -292,16 +365,12 @@ prune_m4_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, ui
                 uint8_t* __restrict__ mask, OutPitch pitch, ReluSource src) {
   ptx::wait_for_previous_grid();
   ptx::launch_dependents();  // only once this grid's own predecessor is done: at most one grid ever waits behind a running one
-  const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
   uint4 in[kVecPerThread];
+  int64_t vi[kVecPerThread];
+  load_unit<RELU>(dO, nvec, src, vi, in);
 #pragma unroll
   for (int it = 0; it < kVecPerThread; ++it) {
-    const int64_t v = base + (int64_t)it * kThreads;
-    in[it] = (v < nvec) ? load_gradient<RELU>(dO, v, src) : make_uint4(0, 0, 0, 0);
-  }
-#pragma unroll
-  for (int it = 0; it < kVecPerThread; ++it) {
-    const int64_t v = base + (int64_t)it * kThreads;
+    const int64_t v = vi[it];
     if (v >= nvec) continue;
     const uint4 w = in[it];
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3;
@@ -363,16 +432,12 @@ prune_top2_kernel(const uint4* __restrict__ dO, int64_t nvec, uint32_t seed_lo, 
   ptx::launch_dependents();  // only once this grid's own predecessor is done: at most one grid ever waits behind a running one
   constexpr int LANES = M / 8;
   static_assert(N == 1 || N == 2, "threshold selection keeps one or two elements");
-  const int64_t base = (int64_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
   uint4 in[kVecPerThread];
+  int64_t vi[kVecPerThread];
+  load_unit<RELU>(dO, nvec, src, vi, in);
 #pragma unroll
   for (int it = 0; it < kVecPerThread; ++it) {
-    const int64_t v = base + (int64_t)it * kThreads;
-    in[it] = (v < nvec) ? load_gradient<RELU>(dO, v, src) : make_uint4(0, 0, 0, 0);
-  }
-#pragma unroll
-  for (int it = 0; it < kVecPerThread; ++it) {
-    const int64_t v = base + (int64_t)it * kThreads;
+    const int64_t v = vi[it];
     uint32_t y0, y1, y2, y3, km0, km1, km2, km3;
     if constexpr (SCHEME == SDGP_RESCALED_MAGNITUDE) {
       if (!dense) {  // (uniform over the grid: every lane of a group takes the same branch and meets in the shuffles)
@@ -486,15 +551,23 @@ cudaError_t launch_prune(const void* dO, int64_t rows, int64_t K, int n, int m, 
                          uint64_t seed, void* dense, void* values, void* meta, void* mask,
                          cudaStream_t stream, int64_t k_pad, int dtype) {
   return launch_prune_src<false>(dO, rows, K, n, m, scheme, seed, dense, values, meta, mask, stream, k_pad, dtype,
-                                 ReluSource{nullptr, nullptr, 0u, nullptr, 0});
+                                 ReluSource{nullptr, nullptr, 0u, nullptr, 0, 0, 0, 0});
 }
 
 cudaError_t launch_relu_backward_prune(const void* dY, const void* act, int64_t rows, int64_t K, int n, int m, int scheme,
                                        uint64_t seed, void* grad, void* dense, void* values, void* meta, void* mask,
                                        cudaStream_t stream, int dtype, const void* skip) {
   const ReluSource src = {(const uint4*)act, (uint4*)grad, dtype == SDGP_FP16 ? 0x03FF03FFu : 0x007F007Fu,
-                          (const uint4*)skip, dtype == SDGP_FP16 ? 1 : 0};
+                          (const uint4*)skip, dtype == SDGP_FP16 ? 1 : 0, 0, 0, 0};
   return launch_prune_src<true>(dY, rows, K, n, m, scheme, seed, dense, values, meta, mask, stream, 0, dtype, src);
+}
+
+cudaError_t launch_maxpool_relu_backward_prune(const void* dYp, const void* act, int B, int H, int W, int64_t K, int n, int m,
+                                               int scheme, uint64_t seed, void* grad, void* dense, void* values, void* meta,
+                                               void* mask, cudaStream_t stream, int dtype) {
+  const ReluSource src = {(const uint4*)act, (uint4*)grad, dtype == SDGP_FP16 ? 0x03FF03FFu : 0x007F007Fu,
+                          nullptr, 0, (int)(K / 8), H / 2, W / 2};
+  return launch_prune_src<true>(dYp, (int64_t)B * H * W, K, n, m, scheme, seed, dense, values, meta, mask, stream, 0, dtype, src);
 }
 
 }  // namespace sdgp

@@ -185,3 +185,92 @@ def test_residual_producer_rejects_bad_arguments():
         odd = torch.zeros(8 * 64 + 8, dtype=torch.int16, device="cuda")[1:1 + 8 * 64].view(8, 64)   # 2 bytes off a 16-byte boundary
         sdgp.sdgp_residual_relu_backward_prune(x, odd, x, 2, 4, sdgp.MAGNITUDE, grad=torch.zeros_like(x))
     assert e.value.status == 3
+
+
+# ---- the producer below a ReLU followed by 2 x 2 max pooling: the pooled gradient goes to each window's maximum ----
+
+
+def make_pool(B, H, W, K, seed, dtype=oracle.BF16, nan_gradients=True):
+    rng = np.random.default_rng(seed + 2000)
+    to_bits = inputs.f32_to_bf16_bits if dtype == oracle.BF16 else (lambda x: x.astype(np.float16).view(np.uint16))
+    # coarse activations: equal values inside a window are common; all-negative windows occur too
+    act = to_bits((np.round(rng.standard_normal((B, H, W, K)) * 2.0) / 2.0).astype(np.float32))
+    flat = act.reshape(-1)
+    special = [0x8000, 0x7FC0 if dtype == oracle.BF16 else 0x7E00, 0x7F80 if dtype == oracle.BF16 else 0x7C00, 0x0001, 0xBF80]
+    flat[rng.integers(0, flat.size, 600)] = np.resize(np.array(special, np.uint16), 600)
+    g = to_bits(rng.laplace(size=(B, H // 2, W // 2, K)).astype(np.float32))
+    if nan_gradients:
+        g.reshape(-1)[rng.integers(0, g.size, 50)] = 0x7FC1   # payloads travel unchanged
+    return g, act
+
+
+@pytest.mark.parametrize("n,m,scheme", [(2, 4, oracle.MAGNITUDE), (2, 4, oracle.RESCALED), (1, 4, oracle.RANDOM),
+                                        (3, 4, oracle.MAGNITUDE), (2, 8, oracle.MAGNITUDE), (2, 16, oracle.RESCALED),
+                                        (2, 32, oracle.RANDOM)])
+@pytest.mark.parametrize("shape", [(3, 6, 10, 160), (5, 2, 2, 32), (2, 16, 16, 128)])
+def test_maxpool_producer_outputs_bit_exact(n, m, scheme, shape):
+    import paper_2202_00774_b200 as sdgp
+    B, H, W, K = shape
+    if K % m:
+        pytest.skip("K is not a multiple of m")
+    g, act = make_pool(B, H, W, K, seed=n * 10 + m)
+    rows = B * H * W
+    compressed = n <= 2
+    grad = torch.full((B, H, W, K), -1, dtype=torch.int16, device="cuda")
+    dense = torch.full((rows, K), -1, dtype=torch.int16, device="cuda")
+    values = torch.full((rows, K // 2), -1, dtype=torch.int16, device="cuda") if compressed else None
+    meta = torch.full((rows, K // 16), -1, dtype=torch.int16, device="cuda") if compressed else None
+    mask = torch.full((rows, K // 32), -1, dtype=torch.int32, device="cuda")
+    d_g, d_act = dev16(g), dev16(act)
+    sdgp.sdgp_maxpool_relu_backward_prune(d_g, d_act, n, m, scheme, seed=99, grad=grad, dense=dense, values=values, meta=meta,
+                                          mask=mask)
+    want = ("dense", "values", "meta", "mask") if compressed else ("dense", "mask")
+    ref = oracle.maxpool_relu_backward_prune(g, act, n, m, scheme, seed=99, want=want)
+    assert np.array_equal(host16(grad), ref["grad"])
+    assert np.array_equal(host16(dense), ref["dense"])
+    if compressed:
+        assert np.array_equal(host16(values), ref["values"])
+        assert np.array_equal(host16(meta), ref["meta"])
+    assert np.array_equal(mask.cpu().numpy().view(np.uint32), ref["mask"])
+    assert np.array_equal(host16(d_g), g) and np.array_equal(host16(d_act), act)
+
+
+def test_maxpool_producer_binary16_plain_backward_and_the_sparse_contraction():
+    import paper_2202_00774_b200 as sdgp
+    B, H, W, Cin, Cout = 4, 8, 8, 64, 128
+    g, act = make_pool(B, H, W, Cout, seed=5, dtype=oracle.FP16)
+    grad = torch.full((B, H, W, Cout), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_maxpool_relu_backward_prune(dev16(g), dev16(act), 4, 4, sdgp.MAGNITUDE, dtype=sdgp.FP16, grad=grad)   # n == m: no pruning
+    assert np.array_equal(host16(grad), oracle.maxpool_relu_backward(g, act, oracle.FP16))
+    # bf16, compressed outputs straight into a 3 x 3 convolution's contraction
+    g, act = make_pool(B, H, W, Cout, seed=6, nan_gradients=False)
+    layer = inputs.ConvLayer("pool", B, H, W, Cin, Cout, 3, 3, 1, 1)
+    _, Wt = inputs.conv_layer_tensors(layer, seed=3)
+    rows = B * H * W
+    values = torch.empty((rows, Cout // 2), dtype=torch.int16, device="cuda")
+    meta = torch.empty((rows, Cout // 16), dtype=torch.int16, device="cuda")
+    dD = torch.full((B, H, W, Cin), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_maxpool_relu_backward_prune(dev16(g), dev16(act), 2, 4, sdgp.MAGNITUDE, values=values, meta=meta)
+    sdgp.sdgp_spmm_conv2d(values.view(B, H, W, Cout // 2), meta.view(B, H, W, Cout // 16), dev16(Wt), dD, 1, 1)
+    assert sdgp.sdgp_last_device_error() == 0
+    ref = oracle.maxpool_relu_backward_prune(g, act, 2, 4, oracle.MAGNITUDE, want=("dense",))
+    pruned = ref["dense"].reshape(B, H, W, Cout)
+    want = oracle.dgrad_conv2d(pruned, Wt, H, W, 1, 1)
+    got = inputs.bf16_bits_to_f32(host16(dD)).astype(np.float64)
+    assert np.linalg.norm(got - want) <= TOL * np.linalg.norm(want)
+
+
+def test_maxpool_producer_rejects_bad_arguments():
+    import paper_2202_00774_b200 as sdgp
+    act = torch.zeros((2, 3, 4, 64), dtype=torch.int16, device="cuda")      # odd height
+    g = torch.zeros((2, 1, 2, 64), dtype=torch.int16, device="cuda")
+    with pytest.raises(sdgp.SdgpError) as e:
+        sdgp.sdgp_maxpool_relu_backward_prune(g, act, 2, 4, sdgp.MAGNITUDE, grad=act)
+    assert e.value.status == 1
+    act = torch.zeros((2, 4, 4, 64), dtype=torch.int16, device="cuda")
+    g = torch.zeros((2, 2, 2, 64), dtype=torch.int16, device="cuda")
+    with pytest.raises(sdgp.SdgpError) as e:
+        sdgp.sdgp_maxpool_relu_backward_prune(g, act, 4, 8, sdgp.MAGNITUDE, grad=act)     # groups of 8 keep one or two
+    assert e.value.status == 2
+    with pytest.raises(ValueError):
+        sdgp.sdgp_maxpool_relu_backward_prune(act, act, 2, 4, sdgp.MAGNITUDE, grad=act)   # gradient not of the pooled shape
