@@ -182,9 +182,13 @@ def maxpool_relu_backward(dYp, act, dtype=BF16):
     return out
 
 
-def maxpool_relu_backward_prune(dYp, act, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask"), dtype=BF16):
+def maxpool_relu_backward_prune(dYp, act, n, m, scheme, seed=0, want=("dense", "values", "meta", "mask"), dtype=BF16, skip=None):
     """``maxpool_relu_backward`` followed by Algorithm 1 along K; outputs as [B*H*W, ...]; ``"grad"`` is the unpruned
-    dL/dO [B, H, W, K] (Section 3.1)."""
+    dL/dO [B, H, W, K] (Section 3.1). ``skip``: a second gradient of the pooled shape (a residual block below the pooling),
+    added to ``dYp`` first as ``residual_relu_backward`` adds (through a gate that is open everywhere)."""
+    if skip is not None:
+        one = np.full(np.shape(dYp), 0x3C00 if dtype == FP16 else 0x3F80, np.uint16)
+        dYp = residual_relu_backward(dYp, skip, one, dtype)
     grad = maxpool_relu_backward(dYp, act, dtype)
     out = prune(grad.reshape(-1, grad.shape[-1]), n, m, scheme, seed, want, dtype)
     out["grad"] = grad

@@ -226,3 +226,16 @@ def test_maxpool_producer_is_the_scatter_followed_by_algorithm_1():
         assert np.array_equal(out[key], ref[key])
     with pytest.raises(ValueError):
         oracle.maxpool_relu_backward(g, act[:, :3])                              # odd height
+
+
+def test_maxpool_producer_with_a_second_gradient_adds_before_it_scatters():
+    rng = np.random.default_rng(24)
+    act = bits(rng.standard_normal((2, 4, 4, 32)))
+    g, k = bits(rng.laplace(size=(2, 2, 2, 32))), bits(rng.laplace(size=(2, 2, 2, 32)) * 0.125)
+    out = oracle.maxpool_relu_backward_prune(g, act, 2, 4, oracle.MAGNITUDE, skip=k)
+    import torch
+    total = (torch.from_numpy(g.view(np.int16)).view(torch.bfloat16) + torch.from_numpy(k.view(np.int16)).view(torch.bfloat16))
+    total = total.view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(out["grad"], oracle.maxpool_relu_backward(total, act))
+    assert np.array_equal(oracle.maxpool_relu_backward_prune(g, act, 2, 4, oracle.MAGNITUDE, skip=np.zeros_like(g))["grad"],
+                          oracle.maxpool_relu_backward(g, act))
