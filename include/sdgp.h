@@ -202,8 +202,10 @@ sdgp_status sdgp_residual_relu_backward_prune(const void* dY, const void* dSkip,
  * activation - the first one in the order (0,0), (0,1), (1,0), (1,1) if several are equal, as the usual pooling backward
  * does - provided that activation is a number greater than zero; every other position is +0.0 (a NaN is never the
  * maximum). Algorithm 1 then runs along K on that tensor viewed as [B*H*Wd, K]; grad, dOp_dense, values, meta, mask as
- * sdgp_relu_backward_prune. H and Wd must be even (else SDGP_ERR_INVALID_ARG); B*H*Wd*K / 32 must be below 2^31. */
-sdgp_status sdgp_maxpool_relu_backward_prune(const void* dYp, const void* act, int B, int H, int Wd, int64_t K, int n, int m,
+ * sdgp_relu_backward_prune. dSkipP (optional, may be null): a second gradient of the pooled shape - in ResNet-9 a residual
+ * block follows the pooling, so two gradients reach the pooling's output - added to dYp first, with the arithmetic of
+ * sdgp_residual_relu_backward_prune. H and Wd must be even (else SDGP_ERR_INVALID_ARG); B*H*Wd*K / 32 must be below 2^31. */
+sdgp_status sdgp_maxpool_relu_backward_prune(const void* dYp, const void* dSkipP, const void* act, int B, int H, int Wd, int64_t K, int n, int m,
                                              sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad, void* dOp_dense,
                                              void* values, void* meta, void* mask, void* stream);
 

@@ -72,7 +72,7 @@ def lib() -> ctypes.CDLL:
         L.sdgp_relu_backward_prune.restype = i32
         L.sdgp_residual_relu_backward_prune.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
         L.sdgp_residual_relu_backward_prune.restype = i32
-        L.sdgp_maxpool_relu_backward_prune.argtypes = [vp, vp, i32, i32, i32, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
+        L.sdgp_maxpool_relu_backward_prune.argtypes = [vp, vp, vp, i32, i32, i32, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
         L.sdgp_maxpool_relu_backward_prune.restype = i32
         L.sdgp_channel_scales.restype = i32
         L.sdgp_workspace_size_linear.argtypes = [i64, i64, i64, u32]
@@ -232,18 +232,21 @@ def sdgp_residual_relu_backward_prune(dY, dSkip, act, n, m, scheme, seed=0, dtyp
 
 
 def sdgp_maxpool_relu_backward_prune(dYp, act, n, m, scheme, seed=0, dtype=BF16, grad=None, dense=None, values=None, meta=None,
-                                     mask=None):
+                                     mask=None, skip=None):
     """``sdgp_maxpool_relu_backward_prune``: ``dYp`` [B, H/2, W/2, K] is the gradient above a 2 x 2 max pooling, ``act``
-    [B, H, W, K] the activation of the ReLU below it; dL/dO [B, H, W, K] is formed and pruned in one pass."""
+    [B, H, W, K] the activation of the ReLU below it; dL/dO [B, H, W, K] is formed and pruned in one pass. ``skip``
+    (optional, the shape of ``dYp``) is a second gradient added to ``dYp`` first."""
     for t, name in ((dYp, "dYp"), (act, "act"), (grad, "grad"), (dense, "dense"), (values, "values"), (meta, "meta"),
-                    (mask, "mask")):
+                    (mask, "mask"), (skip, "skip")):
         _dev(t, name)
+    if skip is not None and skip.shape != dYp.shape:
+        raise ValueError("skip must have the shape of dYp")
     if act.dim() != 4 or dYp.dim() != 4:
         raise ValueError("dYp and act must be NHWC tensors")
     B, H, W, K = act.shape
     if tuple(dYp.shape) != (B, H // 2, W // 2, K):
         raise ValueError("dYp must be [B, H/2, W/2, K]")
-    _check(lib().sdgp_maxpool_relu_backward_prune(_ptr(dYp), _ptr(act), B, H, W, K, n, m, scheme, seed, dtype, _ptr(grad),
+    _check(lib().sdgp_maxpool_relu_backward_prune(_ptr(dYp), _ptr(skip), _ptr(act), B, H, W, K, n, m, scheme, seed, dtype, _ptr(grad),
                                                   _ptr(dense), _ptr(values), _ptr(meta), _ptr(mask), _stream()),
            "sdgp_maxpool_relu_backward_prune")
 

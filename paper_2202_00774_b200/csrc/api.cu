@@ -105,7 +105,7 @@ sdgp_status sdgp_relu_backward_prune(const void* dY, const void* act, int64_t ro
   return relu_backward_prune(dY, nullptr, act, rows, K, n, m, scheme, seed, dtype, grad, dOp_dense, values, meta, mask, stream);
 }
 
-sdgp_status sdgp_maxpool_relu_backward_prune(const void* dYp, const void* act, int B, int H, int Wd, int64_t K, int n, int m,
+sdgp_status sdgp_maxpool_relu_backward_prune(const void* dYp, const void* dSkipP, const void* act, int B, int H, int Wd, int64_t K, int n, int m,
                                              sdgp_scheme scheme, uint64_t seed, sdgp_dtype dtype, void* grad, void* dOp_dense,
                                              void* values, void* meta, void* mask, void* stream) {
   if (!valid_dtype(dtype)) return SDGP_ERR_INVALID_ARG;
@@ -118,12 +118,12 @@ sdgp_status sdgp_maxpool_relu_backward_prune(const void* dYp, const void* act, i
   if (!dYp || !act) return SDGP_ERR_INVALID_ARG;
   if ((values || meta) && n > 2) return SDGP_ERR_UNSUPPORTED;
   if (K % 16 != 0 || (mask && K % 32 != 0)) return SDGP_ERR_ALIGNMENT;
-  if (!aligned16(dYp) || !aligned16(act) || !aligned16(grad) || !aligned16(dOp_dense) || !aligned16(values) ||
+  if (!aligned16(dYp) || !aligned16(dSkipP) || !aligned16(act) || !aligned16(grad) || !aligned16(dOp_dense) || !aligned16(values) ||
       !aligned16(meta) || !aligned16(mask))
     return SDGP_ERR_ALIGNMENT;
   if (rows * (K / 8) / 4 > 0x7FFFFFFF) return SDGP_ERR_UNSUPPORTED;   // the kernel numbers the pooled vectors in 32 bits
   cudaError_t e = sdgp::launch_maxpool_relu_backward_prune(dYp, act, B, H, Wd, K, n, m, (int)scheme, seed, grad, dOp_dense, values,
-                                                           meta, mask, (cudaStream_t)stream, (int)dtype);
+                                                           meta, mask, (cudaStream_t)stream, (int)dtype, dSkipP);
   return e == cudaSuccess ? SDGP_OK : SDGP_ERR_CUDA;
 }
 

@@ -137,7 +137,13 @@ __device__ __forceinline__ void load_unit(const uint4* __restrict__ dO, int64_t 
       vi[it] = live ? (pix00 + (it >> 1) * (2 * src.pool_wp) + (it & 1)) * src.pool_k8 + cv : nvec;
       a[it] = live ? __ldg(src.act + vi[it]) : make_uint4(0u, 0u, 0u, 0u);
     }
-    const uint4 g = live ? __ldg(dO + u) : make_uint4(0u, 0u, 0u, 0u);
+    uint4 g = live ? __ldg(dO + u) : make_uint4(0u, 0u, 0u, 0u);
+    if (live && src.skip) {  // a second gradient of the pooled shape (a residual connection joins below the pooling)
+      const uint4 k = __ldg(src.skip + u);
+      g = src.f16 ? make_uint4(add_pair<true>(g.x, k.x), add_pair<true>(g.y, k.y), add_pair<true>(g.z, k.z), add_pair<true>(g.w, k.w))
+                  : make_uint4(add_pair<false>(g.x, k.x), add_pair<false>(g.y, k.y), add_pair<false>(g.z, k.z),
+                               add_pair<false>(g.w, k.w));
+    }
     uint32_t ox[4], oy[4], oz[4], ow[4];
     const uint32_t ax[4] = {a[0].x, a[1].x, a[2].x, a[3].x}, ay[4] = {a[0].y, a[1].y, a[2].y, a[3].y},
                    az[4] = {a[0].z, a[1].z, a[2].z, a[3].z}, aw[4] = {a[0].w, a[1].w, a[2].w, a[3].w};
@@ -564,9 +570,9 @@ cudaError_t launch_relu_backward_prune(const void* dY, const void* act, int64_t 
 
 cudaError_t launch_maxpool_relu_backward_prune(const void* dYp, const void* act, int B, int H, int W, int64_t K, int n, int m,
                                                int scheme, uint64_t seed, void* grad, void* dense, void* values, void* meta,
-                                               void* mask, cudaStream_t stream, int dtype) {
+                                               void* mask, cudaStream_t stream, int dtype, const void* skip_pooled) {
   const ReluSource src = {(const uint4*)act, (uint4*)grad, dtype == SDGP_FP16 ? 0x03FF03FFu : 0x007F007Fu,
-                          nullptr, 0, (int)(K / 8), H / 2, W / 2};
+                          (const uint4*)skip_pooled, dtype == SDGP_FP16 ? 1 : 0, (int)(K / 8), H / 2, W / 2};
   return launch_prune_src<true>(dYp, (int64_t)B * H * W, K, n, m, scheme, seed, dense, values, meta, mask, stream, 0, dtype, src);
 }
 

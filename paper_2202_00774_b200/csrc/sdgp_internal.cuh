@@ -24,10 +24,12 @@ cudaError_t launch_relu_backward_prune(const void* dY, const void* act, int64_t 
 
 // The same producer below a ReLU that is followed by 2 x 2 max pooling of stride 2: dYp is the pooled gradient
 // [B, H/2, W/2, K], act the activation [B, H, W, K]; each pooled gradient goes to the first largest activation of its
-// window if that is positive. B * H * W * K / 32 must fit 31 bits; H and W even.
+// window if that is positive. skip_pooled (optional): a second gradient of the pooled shape, added to dYp first.
+// B * H * W * K / 32 must fit 31 bits; H and W even.
 cudaError_t launch_maxpool_relu_backward_prune(const void* dYp, const void* act, int B, int H, int W, int64_t K, int n, int m,
                                                int scheme, uint64_t seed, void* grad, void* dense, void* values, void* meta,
-                                               void* mask, cudaStream_t stream, int dtype = SDGP_BF16);
+                                               void* mask, cudaStream_t stream, int dtype = SDGP_BF16,
+                                               const void* skip_pooled = nullptr);
 
 // Per-channel reading of the L1 rescale (channel.cu). sums: 2 * K floats (cleared by the call): the
 // column sums of |x| over all rows, then the same over the survivors of the magnitude function.

@@ -73,14 +73,15 @@ def test_producers_reject_bad_arguments_before_launch(lib):
     assert Rs(FAKE, FAKE, FAKE, 4, 64, 2, 4, 1, 0, 9, FAKE, None, None, None, None, None) == 1   # unknown element type
     assert Rs(None, None, None, 0, 64, 2, 4, 1, 0, 0, None, None, None, None, None, None) == 0   # empty tensor: no-op
     Mp = lib.sdgp_maxpool_relu_backward_prune
-    Mp.argtypes = [vp, vp, i32, i32, i32, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
-    assert Mp(FAKE, FAKE, 2, 3, 4, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 1    # odd height
-    assert Mp(FAKE, FAKE, 2, 4, 6, 72, 2, 16, 1, 0, 0, FAKE, None, None, None, None, None) == 1   # K % m != 0
-    assert Mp(FAKE, None, 2, 4, 4, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 1    # no activation
-    assert Mp(FAKE, FAKE, 2, 4, 4, 64, 4, 8, 1, 0, 0, FAKE, None, None, None, None, None) == 2
-    assert Mp(FAKE, FAKE, 2, 4, 4, 40, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 3    # K % 16 != 0
-    assert Mp(FAKE, FAKE, 1 << 20, 1 << 10, 1 << 10, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 2   # too many vectors
-    assert Mp(None, None, 0, 4, 4, 64, 2, 4, 1, 0, 0, None, None, None, None, None, None) == 0
+    Mp.argtypes = [vp, vp, vp, i32, i32, i32, i64, i32, i32, i32, u64, i32, vp, vp, vp, vp, vp, vp]
+    assert Mp(FAKE, None, FAKE, 2, 3, 4, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 1    # odd height
+    assert Mp(FAKE, None, FAKE, 2, 4, 6, 72, 2, 16, 1, 0, 0, FAKE, None, None, None, None, None) == 1   # K % m != 0
+    assert Mp(FAKE, None, None, 2, 4, 4, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 1    # no activation
+    assert Mp(FAKE, FAKE, FAKE, 2, 4, 4, 64, 4, 8, 1, 0, 0, FAKE, None, None, None, None, None) == 2
+    assert Mp(FAKE, None, FAKE, 2, 4, 4, 40, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 3    # K % 16 != 0
+    assert Mp(FAKE, None, FAKE, 1 << 20, 1 << 10, 1 << 10, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 2   # too many vectors
+    assert Mp(FAKE, ctypes.c_void_p(0x1004), FAKE, 2, 4, 4, 64, 2, 4, 1, 0, 0, FAKE, None, None, None, None, None) == 3   # misaligned second gradient
+    assert Mp(None, None, None, 0, 4, 4, 64, 2, 4, 1, 0, 0, None, None, None, None, None, None) == 0
 
 
 def test_dgrad_rejects_bad_arguments_before_launch(lib):

@@ -274,3 +274,24 @@ def test_maxpool_producer_rejects_bad_arguments():
     assert e.value.status == 2
     with pytest.raises(ValueError):
         sdgp.sdgp_maxpool_relu_backward_prune(act, act, 2, 4, sdgp.MAGNITUDE, grad=act)   # gradient not of the pooled shape
+
+
+@pytest.mark.parametrize("dtype", [oracle.BF16, oracle.FP16])
+def test_maxpool_producer_with_a_second_pooled_gradient(dtype):
+    """ResNet-9: a residual block follows the pooling, so the pooling's output receives two gradients."""
+    import paper_2202_00774_b200 as sdgp
+    B, H, W, K = 3, 8, 6, 128
+    g, act = make_pool(B, H, W, K, seed=31, dtype=dtype)
+    skip = make_skip(B * (H // 2) * (W // 2), K, seed=31, dtype=dtype).reshape(g.shape)
+    skip.reshape(-1)[0:500:3] = g.reshape(-1)[0:500:3] ^ 0x8000           # cancellations
+    dt = sdgp.BF16 if dtype == oracle.BF16 else sdgp.FP16
+    rows = B * H * W
+    grad = torch.full((B, H, W, K), -1, dtype=torch.int16, device="cuda")
+    values = torch.full((rows, K // 2), -1, dtype=torch.int16, device="cuda")
+    meta = torch.full((rows, K // 16), -1, dtype=torch.int16, device="cuda")
+    sdgp.sdgp_maxpool_relu_backward_prune(dev16(g), dev16(act), 2, 8, sdgp.RESCALED_MAGNITUDE, seed=5, dtype=dt, grad=grad,
+                                          values=values, meta=meta, skip=dev16(skip))
+    ref = oracle.maxpool_relu_backward_prune(g, act, 2, 8, oracle.RESCALED, seed=5, want=("values", "meta"), dtype=dtype, skip=skip)
+    assert np.array_equal(host16(grad), ref["grad"])
+    assert np.array_equal(host16(values), ref["values"])
+    assert np.array_equal(host16(meta), ref["meta"])
