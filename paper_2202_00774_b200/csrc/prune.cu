@@ -92,22 +92,26 @@ __device__ __forceinline__ uint4 load_gradient(const uint4* __restrict__ dO, int
 
 // Pooling backward for one 32-bit word (two channels) of a window: a[0..3] are the activation words at the window's
 // four positions in the order (0,0), (0,1), (1,0), (1,1), g the pooled gradient's word. Per channel the gradient goes
-// to the first largest activation if that is a number greater than zero (patterns of positive numbers order like the
-// numbers; composite = pattern * 4 + 3 - position is unique, so exactly one position wins or none does).
+// to the first largest activation if that is a number greater than zero. Both channels at once, in 16-bit lanes:
+// key = the pattern where it is a positive number, else 0 (15 bits; patterns of positive numbers order like the
+// numbers); (key_a | 0x8000) - key_b keeps the lane's top bit exactly when key_a >= key_b, and no borrow leaves the
+// lane. Position t wins when its key is strictly above every earlier one and not below any later one; position 0
+// must also be non-zero (a later winner is above a key that is at least zero).
 __device__ __forceinline__ void pool_select2(const uint32_t (&a)[4], uint32_t g, uint32_t nan_add, uint32_t (&out)[4]) {
-  uint32_t lo[4], hi[4];
+  constexpr uint32_t H = 0x80008000u;
+  uint32_t k[4];
 #pragma unroll
-  for (int t = 0; t < 4; ++t) {
-    const uint32_t key = relu_pass2(a[t], a[t], nan_add);  // the pattern where it is a positive number, else 0
-    lo[t] = ((key & 0xFFFFu) << 2) | (uint32_t)(3 - t);
-    hi[t] = ((key >> 16) << 2) | (uint32_t)(3 - t);
-  }
-  const uint32_t mlo = max(max(lo[0], lo[1]), max(lo[2], lo[3])), mhi = max(max(hi[0], hi[1]), max(hi[2], hi[3]));
+  for (int t = 0; t < 4; ++t) k[t] = relu_pass2(a[t], a[t], nan_add);
+  const uint32_t ge01 = (k[0] | H) - k[1], ge02 = (k[0] | H) - k[2], ge03 = (k[0] | H) - k[3];
+  const uint32_t ge12 = (k[1] | H) - k[2], ge13 = (k[1] | H) - k[3], ge23 = (k[2] | H) - k[3];
+  const uint32_t nz0 = k[0] + 0x7FFF7FFFu;  // top bit of a lane: its key is not zero
+  uint32_t win[4];
+  win[0] = (ge01 & ge02 & ge03) & (nz0 & H);
+  win[1] = (~ge01 & ge12 & ge13) & H;
+  win[2] = (~ge02 & ~ge12 & ge23) & H;
+  win[3] = (~ge03 & ~ge13 & ~ge23) & H;
 #pragma unroll
-  for (int t = 0; t < 4; ++t) {
-    const uint32_t keep = ((lo[t] == mlo && mlo > 3u) ? 0x0000FFFFu : 0u) | ((hi[t] == mhi && mhi > 3u) ? 0xFFFF0000u : 0u);
-    out[t] = g & keep;
-  }
+  for (int t = 0; t < 4; ++t) out[t] = g & prmt(win[t], 0u, 0xBB99);  // top bits replicated over their half-words
 }
 
 // The four vectors a thread prunes and their numbers in dL/dO (>= nvec: none). Without pooling they are the thread's
