@@ -447,6 +447,42 @@ def run_ours(args, layers):
         pool_gbs = dO[big].numel() * 5.625 / (ms_pool * 1e-3) / 1e9
         relu_chain["pool_producer"] = {"layer": lb.name, "us": 1e3 * ms_pool, "gbs": pool_gbs, "frac_of_hbm": pool_gbs / pk["hbm"],
                                        "bytes_per_element": 5.625}
+        # ---- the chain with the producer each layer of ResNet-9 has above it (the normalisation layers left out): the
+        # convolutions 64->128@32, 128->256@16 and 256->512@8 are followed by ReLU and 2 x 2 max pooling, the first and the
+        # last of them with a residual block behind the pooling (two gradients reach the pooling's output); the other four
+        # convolutions sit below a plain ReLU. Sparse side and dense side run the same producers (dense: n = m). ----
+        if len(layers) == 7:
+            pooled_layers = {0: True, 3: False, 4: True}    # layer index -> a residual block follows the pooling
+            gp = {i: dO[i].view(layers[i].B, layers[i].P, layers[i].Q, layers[i].Cout)[:, : layers[i].P // 2, : layers[i].Q // 2]
+                  .contiguous() for i in pooled_layers}
+            gs = {i: (gp[i].view(torch.float16 if args.dtype == "fp16" else torch.bfloat16).float() * 0.5)
+                  .to(torch.float16 if args.dtype == "fp16" else torch.bfloat16).view(torch.int16).flip(0).contiguous()
+                  for i, res in pooled_layers.items() if res}
+
+            def glue_step(sparse):
+                for i in order:
+                    l = layers[i]
+                    nn = n if sparse else m
+                    outs = dict(values=cv[i], meta=cm[i]) if sparse else {}
+                    if i in pooled_layers:
+                        sdgp.sdgp_maxpool_relu_backward_prune(gp[i], act[i].view(l.B, l.P, l.Q, l.Cout), nn, m, scheme, 1234, dtype=DT,
+                                                              grad=grad[i].view(l.B, l.P, l.Q, l.Cout), skip=gs.get(i), **outs)
+                    else:
+                        sdgp.sdgp_relu_backward_prune(dO[i].view(-1, l.Cout), act[i].view(-1, l.Cout), nn, m, scheme, 1234, dtype=DT,
+                                                      grad=grad[i].view(-1, l.Cout), **outs)
+                    if sparse:
+                        sdgp.sdgp_spmm_conv2d_typed(cv[i].view(l.B, l.P, l.Q, l.Cout // 2), cm[i].view(l.B, l.P, l.Q, l.Cout // 16),
+                                                    Wt[i], dD[i], l.stride, l.pad, DT)
+                    else:
+                        sdgp.sdgp_dgrad_conv2d_typed(grad[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, 0, DT, flags=sdgp.FLAG_DENSE)
+            g_gs, g_gd = capture(lambda: glue_step(True)), capture(lambda: glue_step(False))
+            ms_gs = timed(g_gs.replay, dense_steps, max(3, args.warmup // 2)) / dense_steps
+            ms_gd = timed(g_gd.replay, dense_steps, max(3, args.warmup // 2)) / dense_steps
+            relu_chain["resnet9_producers"] = {
+                "sparse_ms_per_step": ms_gs, "dense_ms_per_step": ms_gd, "speedup_vs_dense": ms_gd / ms_gs,
+                "what": "as above, but layers 0, 3, 4 below ReLU + 2 x 2 max pooling (0 and 4 with a second pooled gradient), "
+                        "the others below a plain ReLU"}
+            del gp, gs, g_gs, g_gd
         del act, grad, cv, cm, g_rs, g_rd, skip, g_res, pooled, g_pool
 
     # ---- per-kernel timing: the same step captured with timing events between the kernels
