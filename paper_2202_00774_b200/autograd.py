@@ -89,3 +89,62 @@ def sdgp_conv2d(x, weight, stride=1, padding=0, n=2, m=4, scheme=_b.MAGNITUDE, s
     one padding value for both axes) whose input gradient is computed from dL/dO pruned N:M along
     the output channels. Channel counts must be multiples of 64."""
     return _SDGPConv2dFn.apply(x, weight, stride, padding, n, m, scheme, seed)
+
+
+class _SDGPConv2dReLUFn(torch.autograd.Function):
+    """``relu(conv2d(x, weight))``, optionally followed by 2 x 2 max pooling. The backward pass forms the
+    convolution's dL/dO from the gradient above the ReLU (or above the pooling) with the library's producer, which
+    writes the unpruned dL/dO - the weight gradient's operand (Section 3.1) - and its compressed pruned copy in one
+    pass; the sparse contraction then gives the input gradient (Section 2.1, Fig. 2)."""
+
+    @staticmethod
+    def forward(ctx, x, weight, stride, padding, pool, n, m, scheme, seed):
+        act = torch.relu(torch.nn.functional.conv2d(x, weight, None, stride, padding))
+        act = act.contiguous(memory_format=torch.channels_last)
+        ctx.save_for_backward(x, weight, act)
+        ctx.cfg = (stride, padding, pool, n, m, scheme, seed)
+        return torch.nn.functional.max_pool2d(act, 2) if pool else act
+
+    @staticmethod
+    def backward(ctx, grad_out):
+        x, weight, act = ctx.saved_tensors
+        stride, padding, pool, n, m, scheme, seed = ctx.cfg
+        dt = _dtype_code(grad_out)
+        B, Cin, H, Wd = x.shape
+        Cout, _, R, S = weight.shape
+        P, Q = act.shape[2], act.shape[3]
+        dY = grad_out.contiguous(memory_format=torch.channels_last).permute(0, 2, 3, 1)   # NHWC views
+        a = act.permute(0, 2, 3, 1)
+        dO = torch.empty((B, P, Q, Cout), dtype=dY.dtype, device=dY.device)
+        compressed = n <= 2 and Cout % 128 == 0 and ctx.needs_input_grad[0]
+        vals = torch.empty((B, P, Q, Cout // 2), dtype=dY.dtype, device=dY.device) if compressed else None
+        meta = torch.empty((B, P, Q, Cout // 16), dtype=torch.int16, device=dY.device) if compressed else None
+        pn, pm = (n, m) if compressed else (4, 4)   # n == m: nothing is pruned, the producer only writes dL/dO
+        if pool:
+            _b.sdgp_maxpool_relu_backward_prune(dY, a, pn, pm, scheme, seed, dt, grad=dO, values=vals, meta=meta)
+        else:
+            _b.sdgp_relu_backward_prune(dY, a, pn, pm, scheme, seed, dt, grad=dO, values=vals, meta=meta)
+        grad_x = grad_w = None
+        if ctx.needs_input_grad[0]:
+            W = weight.contiguous(memory_format=torch.channels_last).permute(0, 2, 3, 1)   # [Cout,R,S,Cin]
+            dD = torch.empty((B, H, Wd, Cin), dtype=dY.dtype, device=dY.device)
+            if compressed:
+                _b.sdgp_spmm_conv2d_typed(vals, meta, W, dD, stride, padding, dt)
+            else:   # no compressed form to hand over: prune dL/dO in a pass of its own
+                ws = torch.empty(max(16, _b.sdgp_workspace_size_conv2d(B, H, Wd, Cin, Cout, R, S, stride, padding,
+                                                                       _b.FLAG_TWO_PASS if n <= 2 else _b.FLAG_MASKED)),
+                                 dtype=torch.uint8, device=dY.device)
+                _b.sdgp_dgrad_conv2d_typed(dO, W, dD, stride, padding, n, m, scheme, seed, dt, workspace=ws,
+                                           flags=_b.FLAG_TWO_PASS if n <= 2 else _b.FLAG_MASKED)
+            grad_x = dD.permute(0, 3, 1, 2)
+        if ctx.needs_input_grad[1]:
+            grad_w = torch.nn.grad.conv2d_weight(x, weight.shape, dO.permute(0, 3, 1, 2), stride, padding)   # unpruned dL/dO
+        return grad_x, grad_w, None, None, None, None, None, None, None
+
+
+def sdgp_conv2d_relu(x, weight, stride=1, padding=0, pool=False, n=2, m=4, scheme=_b.MAGNITUDE, seed=0):
+    """``relu(conv2d(x, weight))`` - with ``pool=True`` followed by ``max_pool2d(., 2)`` - whose backward pass
+    forms and prunes the convolution's dL/dO in one pass over the incoming gradient (ReLU backward, pooling
+    backward and Algorithm 1 together) and computes the input gradient from the pruned copy. Same tensor
+    requirements as ``sdgp_conv2d``; with ``pool=True`` the convolution's output height and width must be even."""
+    return _SDGPConv2dReLUFn.apply(x, weight, stride, padding, pool, n, m, scheme, seed)
