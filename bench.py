@@ -413,8 +413,8 @@ def run_ours(args, layers):
         def relu_dense_step():
             for i in order:
                 l = layers[i]
-                sdgp.sdgp_relu_backward_prune(dO[i].view(-1, l.Cout), act[i].view(-1, l.Cout), m, m, scheme, 0, dtype=DT,
-                                              grad=grad[i].view(-1, l.Cout))
+                sdgp.sdgp_relu_backward_prune(dO[i].view(-1, l.Cout), act[i].view(-1, l.Cout), 4, 4, scheme, 0, dtype=DT,
+                                              grad=grad[i].view(-1, l.Cout))   # n == m: nothing pruned
                 sdgp.sdgp_dgrad_conv2d_typed(grad[i], Wt[i], dD[i], l.stride, l.pad, n, m, scheme, 0, DT, flags=sdgp.FLAG_DENSE)
 
         g_rs, g_rd = capture(relu_sparse_step), capture(relu_dense_step)
@@ -462,13 +462,13 @@ def run_ours(args, layers):
             def glue_step(sparse):
                 for i in order:
                     l = layers[i]
-                    nn = n if sparse else m
+                    nn, mm = (n, m) if sparse else (4, 4)   # n == m: nothing pruned
                     outs = dict(values=cv[i], meta=cm[i]) if sparse else {}
                     if i in pooled_layers:
-                        sdgp.sdgp_maxpool_relu_backward_prune(gp[i], act[i].view(l.B, l.P, l.Q, l.Cout), nn, m, scheme, 1234, dtype=DT,
+                        sdgp.sdgp_maxpool_relu_backward_prune(gp[i], act[i].view(l.B, l.P, l.Q, l.Cout), nn, mm, scheme, 1234, dtype=DT,
                                                               grad=grad[i].view(l.B, l.P, l.Q, l.Cout), skip=gs.get(i), **outs)
                     else:
-                        sdgp.sdgp_relu_backward_prune(dO[i].view(-1, l.Cout), act[i].view(-1, l.Cout), nn, m, scheme, 1234, dtype=DT,
+                        sdgp.sdgp_relu_backward_prune(dO[i].view(-1, l.Cout), act[i].view(-1, l.Cout), nn, mm, scheme, 1234, dtype=DT,
                                                       grad=grad[i].view(-1, l.Cout), **outs)
                     if sparse:
                         sdgp.sdgp_spmm_conv2d_typed(cv[i].view(l.B, l.P, l.Q, l.Cout // 2), cm[i].view(l.B, l.P, l.Q, l.Cout // 16),
