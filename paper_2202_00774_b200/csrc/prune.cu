@@ -20,7 +20,8 @@ constexpr int kVecPerThread = 4;
 // Resident blocks per SM the compiler is asked to make room for. Six (at most 40 registers per thread instead of the 42-46
 // it takes unasked, which round up to five blocks) measured 7 % more bytes per second for the magnitude function, 6 % for
 // groups of 8 and 3 % for the random function; the rescaled function and the producers below a ReLU spill at 40 registers
-// and measured slower, so they keep the compiler's own choice.
+// and measured slower, so they keep the compiler's own choice. Eight blocks (32 registers, 64-72 bytes spilled per thread)
+// measured 9 % fewer bytes per second than six.
 template <int SCHEME, bool RELU>
 constexpr int kBlocksPerSm = (!RELU && SCHEME != SDGP_RESCALED_MAGNITUDE) ? 6 : 0;
 
